@@ -1,0 +1,211 @@
+"""Seeded synthetic inputs for the ComFuse joint compute-memory fusion path.
+
+This module only *generates data*: tensor shapes, value distributions and the
+bf16 storage format.  It contains none of the method's arithmetic (no GEMM, no
+normalisation, no softmax) and is the one module that both the CPU oracle's
+tests and the CUDA path's tests / benchmark import, so that both sides see the
+same bytes.
+
+Every tensor is produced as fp32 from a numpy ``Generator`` (PCG64) seeded with
+``[seed, tensor_index]``, rounded to bfloat16 with round-to-nearest-even, and
+returned as the raw ``uint16`` bit pattern.  ``bf16_to_f64`` widens those bits
+exactly, which is what the oracle consumes; the GPU side reinterprets the same
+bits as ``torch.bfloat16``.
+
+The five named workloads follow the paper's two experiment families: a MatMul
+followed by a reduction-bearing epilogue (post-norm / softmax patterns,
+Sec. 6.1) and a back-to-back GEMM MLP (Sec. 6.2, Table II).  The paper uses
+synthetic microbenchmarks without public datasets; so do these.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+# ----------------------------------------------------------------------------
+# bf16 storage helpers (format conversion only)
+# ----------------------------------------------------------------------------
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp32 to bfloat16 (round-to-nearest-even); returns uint16 bits."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    # NaN stays NaN (quiet); everything else: add 0x7FFF + lsb, truncate.
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    rounded = (u + np.uint32(0x7FFF) + lsb) >> np.uint32(16)
+    nan = np.isnan(x)
+    out = rounded.astype(np.uint16)
+    if nan.any():
+        out[nan] = np.uint16(0x7FC0)
+    return out
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """Exact widening of bfloat16 bits to fp32."""
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def bf16_to_f64(b: np.ndarray) -> np.ndarray:
+    """Exact widening of bfloat16 bits to fp64 (what the oracle consumes)."""
+    return bf16_bits_to_f32(b).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------
+# random tensors
+# ----------------------------------------------------------------------------
+
+
+def _rng(seed: int, index: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64([int(seed), int(index)]))
+
+
+def normal_bf16(seed: int, index: int, shape, mean: float = 0.0, std: float = 1.0) -> np.ndarray:
+    g = _rng(seed, index)
+    x = g.standard_normal(size=shape, dtype=np.float32)
+    if std != 1.0:
+        x *= np.float32(std)
+    if mean != 0.0:
+        x += np.float32(mean)
+    return f32_to_bf16_bits(x)
+
+
+def uniform_bf16(seed: int, index: int, shape, lo: float, hi: float) -> np.ndarray:
+    g = _rng(seed, index)
+    x = g.random(size=shape, dtype=np.float32)
+    x = x * np.float32(hi - lo) + np.float32(lo)
+    return f32_to_bf16_bits(x)
+
+
+# ----------------------------------------------------------------------------
+# workload descriptions
+# ----------------------------------------------------------------------------
+
+KIND_BIAS_RES_LAYERNORM = "bias_res_layernorm"
+KIND_BIAS_GELU_RES_RMSNORM_MAX = "bias_gelu_res_rmsnorm_max"
+KIND_SCALE_MASK_SOFTMAX = "scale_mask_softmax"
+KIND_B2B_MLP_LAYERNORM = "b2b_mlp_layernorm"
+
+
+@dataclass
+class Workload:
+    """One problem instance: a kind, its sizes, scalars and bf16 tensors (uint16 bits)."""
+
+    name: str
+    kind: str
+    dims: dict
+    scalars: dict
+    tensors: dict = field(default_factory=dict)
+
+    def gemm_flops(self) -> float:
+        d = self.dims
+        if self.kind == KIND_B2B_MLP_LAYERNORM:
+            return 2.0 * d["M"] * d["K"] * d["N1"] + 2.0 * d["M"] * d["N1"] * d["N2"]
+        return 2.0 * d.get("batch", 1) * d["M"] * d["N"] * d["K"]
+
+    def min_hbm_bytes(self) -> float:
+        """Every operand read once and every output written once, nothing else."""
+        d = self.dims
+        if self.kind == KIND_B2B_MLP_LAYERNORM:
+            M, K, N1, N2 = d["M"], d["K"], d["N1"], d["N2"]
+            return 2.0 * (M * K + K * N1 + N1 * N2 + N1 + N2 + M * N2) + (
+                4.0 * N2 if "gamma" in self.tensors else 0.0
+            )
+        b, M, N, K = d.get("batch", 1), d["M"], d["N"], d["K"]
+        total = 2.0 * b * (M * K + K * N + M * N)
+        if self.kind == KIND_BIAS_RES_LAYERNORM:
+            total += 2.0 * (M * N + N)  # residual, bias
+            total += 2.0 * 2 * N if "gamma" in self.tensors else 0.0
+        elif self.kind == KIND_BIAS_GELU_RES_RMSNORM_MAX:
+            total += 2.0 * (M * N + 2 * N) + 8.0 * M  # residual, bias, g, rowmax+argmax
+        return total
+
+
+def _gemm_epilogue_ln(name, seed, M, N, K, affine):
+    t = {
+        "A": normal_bf16(seed, 0, (M, K)),
+        "B": normal_bf16(seed, 1, (K, N), std=1.0 / math.sqrt(K)),
+        "bias": uniform_bf16(seed, 2, (N,), -0.1, 0.1),
+        "residual": normal_bf16(seed, 3, (M, N)),
+    }
+    if affine:
+        t["gamma"] = normal_bf16(seed, 4, (N,), mean=1.0, std=0.02)
+        t["beta"] = normal_bf16(seed, 5, (N,), mean=0.0, std=0.02)
+    return Workload(name, KIND_BIAS_RES_LAYERNORM, {"M": M, "N": N, "K": K},
+                    {"alpha": 1.0, "eps": 1e-5}, t)
+
+
+def post_norm(M=256, N=256, K=256, seed=0, affine=False, name=None) -> Workload:
+    """Y = LayerNorm(X.W + b + R).  X,R ~ N(0,1); W ~ N(0, var 1/K); b ~ U(-0.1, 0.1)."""
+    return _gemm_epilogue_ln(name or f"post_norm_{M}x{N}x{K}", seed, M, N, K, affine)
+
+
+def complex_subgraph(M=8192, N=4096, K=4096, seed=2, name=None) -> Workload:
+    """Z = X.W + b; H = GELU_tanh(Z) + R; Y = RMSNorm(H).g; row max / argmax of Y."""
+    t = {
+        "A": normal_bf16(seed, 0, (M, K)),
+        "B": normal_bf16(seed, 1, (K, N), std=1.0 / math.sqrt(K)),
+        "bias": uniform_bf16(seed, 2, (N,), -0.1, 0.1),
+        "residual": normal_bf16(seed, 3, (M, N)),
+        "gamma": normal_bf16(seed, 4, (N,), mean=1.0, std=0.02),
+    }
+    return Workload(name or f"complex_subgraph_{M}x{N}x{K}", KIND_BIAS_GELU_RES_RMSNORM_MAX,
+                    {"M": M, "N": N, "K": K}, {"alpha": 1.0, "eps": 1e-5}, t)
+
+
+def scaled_masked_softmax(batch=64, M=2048, N=2048, K=64, seed=3, causal=True, name=None) -> Workload:
+    """P = softmax(alpha * A.B + mask) per batch; alpha = 1/sqrt(K); causal 0 / -inf mask."""
+    t = {
+        "A": normal_bf16(seed, 0, (batch, M, K)),
+        "B": normal_bf16(seed, 1, (batch, K, N)),
+    }
+    return Workload(name or f"softmax_{batch}x{M}x{N}x{K}", KIND_SCALE_MASK_SOFTMAX,
+                    {"batch": batch, "M": M, "N": N, "K": K},
+                    {"alpha": 1.0 / math.sqrt(K), "causal": bool(causal)}, t)
+
+
+def b2b_mlp(M=32768, K=128, N1=512, N2=128, seed=4, affine=False, name=None) -> Workload:
+    """O = LayerNorm(GELU_tanh(X.W1 + b1).W2 + b2 + X); needs N2 == K for the residual."""
+    assert N2 == K
+    t = {
+        "X": normal_bf16(seed, 0, (M, K)),
+        "W1": normal_bf16(seed, 1, (K, N1), std=1.0 / math.sqrt(K)),
+        "b1": uniform_bf16(seed, 2, (N1,), -0.1, 0.1),
+        "W2": normal_bf16(seed, 3, (N1, N2), std=1.0 / math.sqrt(N1)),
+        "b2": uniform_bf16(seed, 4, (N2,), -0.1, 0.1),
+    }
+    if affine:
+        t["gamma"] = normal_bf16(seed, 5, (N2,), mean=1.0, std=0.02)
+        t["beta"] = normal_bf16(seed, 6, (N2,), mean=0.0, std=0.02)
+    return Workload(name or f"b2b_mlp_{M}x{K}x{N1}x{N2}", KIND_B2B_MLP_LAYERNORM,
+                    {"M": M, "K": K, "N1": N1, "N2": N2}, {"eps": 1e-5}, t)
+
+
+# The five named configurations (index = position in the benchmark's config list).
+def config(index: int) -> Workload:
+    if index == 0:   # post-norm tiny, gamma = 1, beta = 0, seed 0
+        return post_norm(256, 256, 256, seed=0, affine=False, name="c1_post_norm_tiny")
+    if index == 1:   # BERT-base-shaped post-norm FFN output (batch 16 x seq 512)
+        return post_norm(8192, 768, 3072, seed=1, affine=True, name="c2_bert_ffn_out_post_norm")
+    if index == 2:   # complex subgraph over wide rows
+        return complex_subgraph(8192, 4096, 4096, seed=2, name="c3_complex_subgraph")
+    if index == 3:   # GEMM + scaled causal row softmax
+        return scaled_masked_softmax(64, 2048, 2048, 64, seed=3, name="c4_scaled_causal_softmax")
+    if index == 4:   # back-to-back GEMM MLP with post-norm
+        return b2b_mlp(32768, 128, 512, 128, seed=4, name="c5_b2b_mlp")
+    raise IndexError(index)
+
+
+def sample_rows(M: int, count: int, seed: int = 12345) -> np.ndarray:
+    """A sorted sample of row indices that always includes the first and last rows
+    and both sides of every 128-row boundary near the ends."""
+    g = _rng(seed, M)
+    fixed = {0, 1, 127, 128, M - 129 if M > 129 else 0, M - 128 if M > 128 else 0, M - 2 if M > 1 else 0, M - 1}
+    fixed = {r for r in fixed if 0 <= r < M}
+    extra = max(0, count - len(fixed))
+    pool = g.choice(M, size=min(M, extra), replace=False)
+    rows = sorted(fixed.union(int(r) for r in pool))
+    return np.asarray(rows[:max(count, len(fixed))], dtype=np.int64)
