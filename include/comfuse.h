@@ -1,0 +1,127 @@
+/*
+ * comfuse.h -- C ABI of the B200 (sm_100a) joint compute-memory fusion library.
+ *
+ * One bf16 tensor-core GEMM (or a back-to-back pair of GEMMs) whose fp32 result is consumed on-chip by
+ * an elementwise/reduction subgraph, without writing the GEMM result to global memory (ComFuse, Sec. 1:
+ * "joint compute-memory operator fusion"; Sec. 3: Stage-Stream Execution Model; Sec. 4: B2BGEMM).
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers unless stated otherwise; the caller owns every buffer.
+ *     The library allocates no device memory; its only device state is a small status word that lives
+ *     in the loaded module.
+ *   - Tensors are row-major bf16 (2 bytes/element); leading dimensions are in ELEMENTS.
+ *     Pointers must be 16-byte aligned and leading dimensions / batch strides multiples of 8 elements.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     return without synchronising.  Arguments are validated before anything is launched; a non-OK
+ *     return means nothing was enqueued.
+ *   - Device-side waits are bounded.  A wait that expires makes the kernel finish early and records
+ *     COMFUSE_ERR_TIMEOUT in the status word, read with comfuse_last_device_status().
+ *   - `fused = 1` selects the single fused kernel; `fused = 0` selects the in-library unfused path with
+ *     identical semantics (GEMM kernel writes a bf16 intermediate to `workspace`, a row kernel finishes).
+ *   - No C++ exceptions cross this boundary.  The library needs compute capability 10.x.
+ */
+#ifndef COMFUSE_H_
+#define COMFUSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COMFUSE_OK = 0,
+  COMFUSE_ERR_INVALID_ARG = 1,  /* NULL where a pointer is required, non-positive size, bad enum        */
+  COMFUSE_ERR_UNSUPPORTED = 2,  /* shape / op list has no compiled fused instantiation (try fused = 0)    */
+  COMFUSE_ERR_ALIGNMENT = 3,    /* pointer not 16-byte aligned or leading dimension not a multiple of 8  */
+  COMFUSE_ERR_WORKSPACE = 4,    /* workspace NULL or smaller than comfuse_*_workspace_size() reports      */
+  COMFUSE_ERR_ARCH = 5,         /* current device is not compute capability 10.x                           */
+  COMFUSE_ERR_CUDA = 6,         /* a CUDA runtime / driver call failed (launch, tensor-map encode, ...)   */
+  COMFUSE_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (reported by last_device_status)    */
+} comfuse_status_t;
+
+/* The memory-intensive subgraph fused behind the GEMM, as a fixed, topologically ordered op list
+ * (Sec. 5.2: the Fusion Spec IR is an ordered node list plus a table of runtime parameters; here the
+ * list is chosen by enum and the parameter table is comfuse_epilogue_args_t).  Reductions are over the
+ * last dimension N and are the stage boundaries of Sec. 3. */
+typedef enum {
+  /* Y = LayerNorm(alpha*A.B + bias + R) * gamma + beta  -- Sec. 3.2 / Fig. 3 (x = alpha*Acc + Bias; mean; x - mean) */
+  COMFUSE_EPI_BIAS_RES_LAYERNORM = 0,
+  /* H = GELU_tanh(alpha*A.B + bias) + R;  Y = H * rsqrt(mean(H^2) + eps) * gamma;  then a second, chained
+   * reduction: row_max[i] = max_j Y, row_argmax[i] = lowest such j  -- Sec. 2.2 (MatMul + RMSNorm), Sec. 3.2 */
+  COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX = 1,
+  /* P = softmax(alpha*A.B + mask) over the last dim  -- Sec. 5 (ReduceMode softmax), Sec. 6.1 (attention scores) */
+  COMFUSE_EPI_SCALE_MASK_SOFTMAX = 2
+} comfuse_epilogue_kind_t;
+
+typedef enum {
+  COMFUSE_MASK_NONE = 0,
+  COMFUSE_MASK_CAUSAL = 1,   /* 0 where column <= row, -inf elsewhere; requires M == N            */
+  COMFUSE_MASK_ADDITIVE = 2  /* bf16 [M, N] tensor (ld = N) added to the scaled scores, shared by all
+                                batches; may hold -inf; unfused path only                         */
+} comfuse_mask_t;
+
+typedef struct {
+  int32_t batch;            /* >= 1; A, B, R, Y, row_max, row_argmax are batched, vectors are shared   */
+  int32_t M, N, K;          /* A is [M, K], B is [K, N] (N contiguous), Y and R are [M, N]              */
+  int64_t lda, ldb, ldr, ldy;
+  int64_t batch_stride_a, batch_stride_b, batch_stride_r, batch_stride_y;   /* elements */
+  int32_t kind;             /* comfuse_epilogue_kind_t */
+  int32_t mask;             /* comfuse_mask_t, SOFTMAX kind only */
+  float alpha;              /* scales the accumulator before anything else */
+  float eps;                /* added to the variance / mean square inside the square root */
+  int32_t fused;            /* 1 = fused kernel, 0 = in-library unfused path */
+  int32_t reserved;         /* must be 0 */
+} comfuse_gemm_desc_t;
+
+/* Runtime-parameter table of the op list.  bf16 device vectors of length N; NULL means absent
+ * (bias, residual: 0; gamma: 1; beta: 0).  row_max / row_argmax: [batch*M] outputs of the
+ * RMSNORM_MAX kind, required there and ignored elsewhere. */
+typedef struct {
+  const void* bias;
+  const void* residual;
+  const void* gamma;
+  const void* beta;
+  const void* mask;
+  float* row_max;
+  int32_t* row_argmax;
+} comfuse_epilogue_args_t;
+
+/* Bytes of caller-provided workspace the described call needs (0 for fused calls). */
+comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes);
+
+/* GEMM -> subgraph (Sec. 3).  A, B inputs; Y output [batch, M, N] bf16, rounded once, at the store. */
+comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const void* A, const void* B, void* Y,
+                                       const comfuse_epilogue_args_t* args, void* workspace,
+                                       size_t workspace_bytes, void* cuda_stream);
+
+/* Back-to-back GEMM (Sec. 4, Eq. 2) with F = GELU_tanh(. + b1) and the tail
+ *   O = LayerNorm(S.W2 + b2 + X) * gamma + beta,   S = F(X.W1),
+ * X [M, K], W1 [K, N1], W2 [N1, N2], all dense row-major bf16, N2 == K.  In the fused path S (and P) never
+ * leave the chip: S is rounded to bf16 as the second GEMM's tensor-core operand. */
+typedef struct {
+  int32_t M, K, N1, N2;
+  float eps;
+  int32_t fused;
+} comfuse_b2b_desc_t;
+
+comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size_t* bytes);
+
+comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X, const void* W1, const void* b1,
+                                  const void* W2, const void* b2, const void* gamma, const void* beta, void* O,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device status word of the current device:
+ * COMFUSE_OK, COMFUSE_ERR_TIMEOUT, or COMFUSE_ERR_CUDA if the stream reports an error. */
+comfuse_status_t comfuse_last_device_status(void* cuda_stream);
+
+/* Number of kernels this library has launched in this process since it was loaded (for accounting). */
+uint64_t comfuse_launch_count(void);
+
+const char* comfuse_status_string(comfuse_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMFUSE_H_ */

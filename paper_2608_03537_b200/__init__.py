@@ -1,0 +1,185 @@
+"""Python binding of libcomfuse.so -- argument marshalling only.
+
+Every step of the hot path (GEMM, epilogue subgraph, reductions, stores) runs inside the CUDA library; this
+module turns torch tensors into the plain pointers and sizes of the C ABI declared in include/comfuse.h and
+raises if the library reports an error.  There is no CPU fallback: if the shared library is missing the
+import of :func:`lib` fails loudly.
+
+Functions mirror the C entry points:
+    gemm_epilogue(...)      -> comfuse_gemm_epilogue      (GEMM -> elementwise/reduction subgraph, Sec. 3)
+    b2b_gemm(...)           -> comfuse_b2b_gemm           (GEMM -> F -> GEMM -> post-norm tail, Sec. 4)
+    workspace_size(...)     -> comfuse_workspace_size
+    b2b_workspace_size(...) -> comfuse_b2b_workspace_size
+    last_device_status()    -> comfuse_last_device_status
+    launch_count()          -> comfuse_launch_count
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_float, c_int32, c_int64, c_size_t, c_uint64, c_void_p
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libcomfuse.so")
+
+# status codes / enums of include/comfuse.h
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
+EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 0, 1, 2
+MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
+
+EXPORTED_SYMBOLS = (
+    "comfuse_workspace_size",
+    "comfuse_gemm_epilogue",
+    "comfuse_b2b_workspace_size",
+    "comfuse_b2b_gemm",
+    "comfuse_last_device_status",
+    "comfuse_launch_count",
+    "comfuse_status_string",
+)
+
+
+class GemmDesc(Structure):
+    _fields_ = [
+        ("batch", c_int32), ("M", c_int32), ("N", c_int32), ("K", c_int32),
+        ("lda", c_int64), ("ldb", c_int64), ("ldr", c_int64), ("ldy", c_int64),
+        ("batch_stride_a", c_int64), ("batch_stride_b", c_int64), ("batch_stride_r", c_int64), ("batch_stride_y", c_int64),
+        ("kind", c_int32), ("mask", c_int32), ("alpha", c_float), ("eps", c_float),
+        ("fused", c_int32), ("reserved", c_int32),
+    ]
+
+
+class EpilogueArgs(Structure):
+    _fields_ = [
+        ("bias", c_void_p), ("residual", c_void_p), ("gamma", c_void_p), ("beta", c_void_p), ("mask", c_void_p),
+        ("row_max", c_void_p), ("row_argmax", c_void_p),
+    ]
+
+
+class B2bDesc(Structure):
+    _fields_ = [("M", c_int32), ("K", c_int32), ("N1", c_int32), ("N2", c_int32), ("eps", c_float), ("fused", c_int32)]
+
+
+class ComfuseError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        msg = lib().comfuse_status_string(self.status).decode()
+        super().__init__(f"{where}: {msg} (status {self.status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libcomfuse.so (built by ``python -m paper_2608_03537_b200.build``).  Fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} not found: build the CUDA library first (python -m paper_2608_03537_b200.build). "
+                "There is no CPU fallback."
+            )
+        L = ctypes.CDLL(LIB_PATH)
+        L.comfuse_workspace_size.argtypes = [POINTER(GemmDesc), POINTER(c_size_t)]
+        L.comfuse_workspace_size.restype = c_int32
+        L.comfuse_gemm_epilogue.argtypes = [POINTER(GemmDesc), c_void_p, c_void_p, c_void_p, POINTER(EpilogueArgs),
+                                            c_void_p, c_size_t, c_void_p]
+        L.comfuse_gemm_epilogue.restype = c_int32
+        L.comfuse_b2b_workspace_size.argtypes = [POINTER(B2bDesc), POINTER(c_size_t)]
+        L.comfuse_b2b_workspace_size.restype = c_int32
+        L.comfuse_b2b_gemm.argtypes = [POINTER(B2bDesc)] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
+        L.comfuse_b2b_gemm.restype = c_int32
+        L.comfuse_last_device_status.argtypes = [c_void_p]
+        L.comfuse_last_device_status.restype = c_int32
+        L.comfuse_launch_count.argtypes = []
+        L.comfuse_launch_count.restype = c_uint64
+        L.comfuse_status_string.argtypes = [c_int32]
+        L.comfuse_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return c_void_p(s.cuda_stream)
+
+
+def make_gemm_desc(A, B, Y, kind, *, residual=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True) -> GemmDesc:
+    """Describe A [b, M, K] (or [M, K]), B [b, K, N] (or [K, N]), Y [b, M, N] from torch tensors' shapes and strides."""
+    batched = A.dim() == 3
+    batch = A.shape[0] if batched else 1
+    M, K = A.shape[-2], A.shape[-1]
+    N = B.shape[-1]
+    assert B.shape[-2] == K and Y.shape[-2] == M and Y.shape[-1] == N
+    assert A.stride(-1) == 1 and B.stride(-1) == 1 and Y.stride(-1) == 1
+    d = GemmDesc()
+    d.batch, d.M, d.N, d.K = batch, M, N, K
+    d.lda, d.ldb, d.ldy = A.stride(-2), B.stride(-2), Y.stride(-2)
+    d.ldr = residual.stride(-2) if residual is not None else N
+    d.batch_stride_a = A.stride(0) if batched else M * d.lda
+    d.batch_stride_b = B.stride(0) if batched else K * d.ldb
+    d.batch_stride_y = Y.stride(0) if batched else M * d.ldy
+    d.batch_stride_r = (residual.stride(0) if batched else M * d.ldr) if residual is not None else M * N
+    d.kind, d.mask, d.alpha, d.eps, d.fused, d.reserved = int(kind), int(mask), float(alpha), float(eps), int(bool(fused)), 0
+    return d
+
+
+def workspace_size(desc: GemmDesc) -> int:
+    n = c_size_t(0)
+    st = lib().comfuse_workspace_size(byref(desc), byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_workspace_size")
+    return int(n.value)
+
+
+def gemm_epilogue(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=None, mask_tensor=None, row_max=None,
+                  row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, workspace=None, stream=None):
+    """Enqueue Y = subgraph(alpha * A.B) on the current (or given) stream.  Tensors are CUDA bf16 (row_max fp32,
+    row_argmax int32).  ``workspace`` is a CUDA uint8 tensor of at least workspace_size(desc) bytes (unfused path)."""
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused)
+    args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_gemm_epilogue(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_epilogue")
+    return Y
+
+
+def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True) -> B2bDesc:
+    return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)))
+
+
+def b2b_workspace_size(desc: B2bDesc) -> int:
+    n = c_size_t(0)
+    st = lib().comfuse_b2b_workspace_size(byref(desc), byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_workspace_size")
+    return int(n.value)
+
+
+def b2b_gemm(X, W1, b1, W2, b2, O, *, gamma=None, beta=None, eps=1e-5, fused=True, workspace=None, stream=None):
+    """Enqueue O = LayerNorm(GELU_tanh(X.W1 + b1).W2 + b2 + X) * gamma + beta.  Dense row-major CUDA bf16 tensors."""
+    M, K = X.shape
+    N1, N2 = W1.shape[1], W2.shape[1]
+    for t in (X, W1, W2, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, eps, fused)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm(byref(d), _ptr(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gamma), _ptr(beta), _ptr(O),
+                                ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm")
+    return O
+
+
+def last_device_status(stream=None) -> int:
+    """Synchronise the stream and return (and clear) the device status word: OK or ERR_TIMEOUT."""
+    return int(lib().comfuse_last_device_status(_stream(stream)))
+
+
+def launch_count() -> int:
+    return int(lib().comfuse_launch_count())

@@ -1,0 +1,26 @@
+// Parameter block and launcher of the fused back-to-back GEMM kernel (plain data).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace comfuse {
+
+struct B2bParams {
+  int M, K, N1, N2;
+  int mblocks;
+  float eps;
+  const uint16_t* X;  // also the residual of the tail
+  const uint16_t* b1;
+  const uint16_t* b2;
+  const uint16_t* gamma;
+  const uint16_t* beta;
+  uint16_t* O;
+  unsigned int* status;
+  unsigned long long timeout_ns;
+};
+
+bool b2b_fused_supported(int K, int N1, int N2);
+cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
+
+}  // namespace comfuse

@@ -1,0 +1,386 @@
+// C ABI of the library: argument validation, tensor-map construction, dispatch to the fused kernels or to the
+// in-library unfused path.  Nothing here allocates device memory.
+#include "../../include/comfuse.h"
+
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "b2b_params.h"
+#include "host_common.h"
+#include "row_params.h"
+
+namespace comfuse {
+
+__device__ unsigned int g_status_word = 0;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::mutex g_mutex;
+constexpr int kMaxDev = 64;
+DeviceInfo g_dev[kMaxDev];
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+
+EncodeFn get_encode_fn() {
+  if (g_encode) return g_encode;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_encode) return g_encode;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  g_encode = reinterpret_cast<EncodeFn>(fn);
+  return g_encode;
+}
+
+unsigned long long timeout_ns() {
+  static unsigned long long v = [] {
+    const char* e = std::getenv("COMFUSE_TIMEOUT_MS");
+    long ms = e ? std::atol(e) : 2000;
+    if (ms < 1) ms = 1;
+    return static_cast<unsigned long long>(ms) * 1000000ull;
+  }();
+  return v;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool mult8(long long v) { return (v & 7) == 0; }
+
+}  // namespace
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+const DeviceInfo* current_device_info() {
+  int d = -1;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDev) return nullptr;
+  if (g_dev[d].device == d) return &g_dev[d];
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_dev[d].device == d) return &g_dev[d];
+  DeviceInfo info;
+  if (cudaDeviceGetAttribute(&info.cc_major, cudaDevAttrComputeCapabilityMajor, d) != cudaSuccess) return nullptr;
+  if (cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, d) != cudaSuccess) return nullptr;
+  if (info.cc_major == 10) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_status_word) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    info.status_word = static_cast<unsigned int*>(addr);
+  }
+  g_dev[d] = info;
+  g_dev[d].device = d;
+  return &g_dev[d];
+}
+
+bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                         uint64_t stride2_bytes, uint32_t box_rows) {
+  EncodeFn enc = get_encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+// Tensor maps of a GEMM's operands: A [batch, M, K] (K contiguous), B [batch, K, N] (N contiguous).
+bool make_operand_maps(CUtensorMap* tmA, CUtensorMap* tmB, const void* A, const void* B, int batch, int M, int N, int K,
+                       long long lda, long long ldb, long long bsa, long long bsb) {
+  const uint64_t sa2 = static_cast<uint64_t>(batch > 1 ? bsa : static_cast<long long>(M) * lda) * 2;
+  const uint64_t sb2 = static_cast<uint64_t>(batch > 1 ? bsb : static_cast<long long>(K) * ldb) * 2;
+  return encode_tmap_bf16_3d(tmA, A, K, M, batch, static_cast<uint64_t>(lda) * 2, sa2, 128) &&
+         encode_tmap_bf16_3d(tmB, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, sb2, 64);
+}
+
+comfuse_status_t check_device(const DeviceInfo** out) {
+  const DeviceInfo* dev = current_device_info();
+  if (!dev) return COMFUSE_ERR_CUDA;
+  if (dev->cc_major != 10) return COMFUSE_ERR_ARCH;
+  *out = dev;
+  return COMFUSE_OK;
+}
+
+int kind_to_epi(int kind) {
+  switch (kind) {
+    case COMFUSE_EPI_BIAS_RES_LAYERNORM: return EPI_LN;
+    case COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX: return EPI_RMS_MAX;
+    case COMFUSE_EPI_SCALE_MASK_SOFTMAX: return EPI_SOFTMAX;
+    default: return -1;
+  }
+}
+
+comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
+  if (!d) return COMFUSE_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->M < 1 || d->N < 1 || d->K < 1) return COMFUSE_ERR_INVALID_ARG;
+  if (kind_to_epi(d->kind) < 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->mask < COMFUSE_MASK_NONE || d->mask > COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_INVALID_ARG;
+  if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
+  if (d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->lda < d->K || d->ldb < d->N || d->ldy < d->N) return COMFUSE_ERR_INVALID_ARG;
+  if (d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && d->mask != COMFUSE_MASK_NONE) return COMFUSE_ERR_INVALID_ARG;
+  if (!mult8(d->N) || !mult8(d->K)) return COMFUSE_ERR_ALIGNMENT;
+  if (!mult8(d->lda) || !mult8(d->ldb) || !mult8(d->ldy)) return COMFUSE_ERR_ALIGNMENT;
+  if (d->batch > 1) {
+    if (d->batch_stride_a < static_cast<long long>(d->M - 1) * d->lda + d->K) return COMFUSE_ERR_INVALID_ARG;
+    if (d->batch_stride_b < static_cast<long long>(d->K - 1) * d->ldb + d->N) return COMFUSE_ERR_INVALID_ARG;
+    if (d->batch_stride_y < static_cast<long long>(d->M - 1) * d->ldy + d->N) return COMFUSE_ERR_INVALID_ARG;
+    if (!mult8(d->batch_stride_a) || !mult8(d->batch_stride_b) || !mult8(d->batch_stride_y)) return COMFUSE_ERR_ALIGNMENT;
+  }
+  if (d->mask == COMFUSE_MASK_CAUSAL && d->M != d->N) return COMFUSE_ERR_UNSUPPORTED;
+  return COMFUSE_OK;
+}
+
+// Does a fused instantiation exist for this description?
+comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
+  if (d->mask == COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_UNSUPPORTED;
+  FusedParams p = {};
+  p.N = d->N;
+  CUtensorMap dummy;
+  std::memset(&dummy, 0, sizeof(dummy));
+  cudaError_t e = cudaErrorInvalidValue;
+  switch (kind_to_epi(d->kind)) {
+    case EPI_LN: e = launch_fused_layernorm(dummy, dummy, p, nullptr, true); break;
+    case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(dummy, dummy, p, nullptr, true); break;
+    case EPI_SOFTMAX: e = launch_fused_softmax(dummy, dummy, p, nullptr, true); break;
+    default: break;
+  }
+  return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+}  // namespace comfuse
+
+using namespace comfuse;
+
+extern "C" {
+
+const char* comfuse_status_string(comfuse_status_t s) {
+  switch (s) {
+    case COMFUSE_OK: return "ok";
+    case COMFUSE_ERR_INVALID_ARG: return "invalid argument";
+    case COMFUSE_ERR_UNSUPPORTED: return "unsupported shape or op list for the fused path";
+    case COMFUSE_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+    case COMFUSE_ERR_WORKSPACE: return "workspace missing or too small";
+    case COMFUSE_ERR_ARCH: return "device is not compute capability 10.x";
+    case COMFUSE_ERR_CUDA: return "CUDA call failed";
+    case COMFUSE_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+uint64_t comfuse_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes) {
+  if (!bytes) return COMFUSE_ERR_INVALID_ARG;
+  comfuse_status_t s = validate_gemm_desc(desc);
+  if (s != COMFUSE_OK) return s;
+  if (desc->fused) {
+    s = fused_supported(desc);
+    if (s != COMFUSE_OK) return s;
+    *bytes = 0;
+  } else {
+    if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
+    *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
+  }
+  return COMFUSE_OK;
+}
+
+comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const void* A, const void* B, void* Y,
+                                       const comfuse_epilogue_args_t* args, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream) {
+  comfuse_status_t s = validate_gemm_desc(desc);
+  if (s != COMFUSE_OK) return s;
+  if (!A || !B || !Y) return COMFUSE_ERR_INVALID_ARG;
+  comfuse_epilogue_args_t a;
+  std::memset(&a, 0, sizeof(a));
+  if (args) a = *args;
+  const int epi = kind_to_epi(desc->kind);
+  if (epi == EPI_RMS_MAX && (!a.row_max || !a.row_argmax)) return COMFUSE_ERR_INVALID_ARG;
+  if (desc->mask == COMFUSE_MASK_ADDITIVE && !a.mask) return COMFUSE_ERR_INVALID_ARG;
+  if (a.residual && (desc->ldr < desc->N || !mult8(desc->ldr) ||
+                     (desc->batch > 1 && (!mult8(desc->batch_stride_r) ||
+                                          desc->batch_stride_r < static_cast<long long>(desc->M - 1) * desc->ldr + desc->N))))
+    return desc->ldr < desc->N ? COMFUSE_ERR_INVALID_ARG : COMFUSE_ERR_ALIGNMENT;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(Y) || !aligned16(a.bias) || !aligned16(a.residual) ||
+      !aligned16(a.gamma) || !aligned16(a.beta) || !aligned16(a.mask))
+    return COMFUSE_ERR_ALIGNMENT;
+
+  size_t need = 0;
+  s = comfuse_workspace_size(desc, &need);
+  if (s != COMFUSE_OK) return s;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return COMFUSE_ERR_WORKSPACE;
+  if (need > 0 && !aligned16(workspace)) return COMFUSE_ERR_ALIGNMENT;
+
+  const DeviceInfo* dev = nullptr;
+  s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  CUtensorMap tmA, tmB;
+  if (!make_operand_maps(&tmA, &tmB, A, B, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, desc->batch_stride_a,
+                         desc->batch_stride_b))
+    return COMFUSE_ERR_CUDA;
+
+  FusedParams p = {};
+  p.M = desc->M; p.N = desc->N; p.K = desc->K; p.batch = desc->batch;
+  p.mblocks = (desc->M + 127) / 128;
+  p.nblocks = 1;
+  p.total_tiles = p.batch * p.mblocks;
+  p.alpha = desc->alpha; p.eps = desc->eps;
+  p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
+  p.status = dev->status_word;
+  p.timeout_ns = timeout_ns();
+  const long long bsr = desc->batch > 1 ? desc->batch_stride_r : 0;
+  const long long bsy = desc->batch > 1 ? desc->batch_stride_y : 0;
+
+  cudaError_t e;
+  if (desc->fused) {
+    p.bias = static_cast<const uint16_t*>(a.bias);
+    p.gamma = static_cast<const uint16_t*>(a.gamma);
+    p.beta = static_cast<const uint16_t*>(a.beta);
+    p.residual = static_cast<const uint16_t*>(a.residual);
+    p.ldr = desc->ldr; p.batch_stride_r = bsr;
+    p.Y = static_cast<uint16_t*>(Y);
+    p.ldy = desc->ldy; p.batch_stride_y = bsy;
+    p.row_max = a.row_max; p.row_argmax = a.row_argmax;
+    switch (epi) {
+      case EPI_LN: e = launch_fused_layernorm(tmA, tmB, p, st, false); break;
+      case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(tmA, tmB, p, st, false); break;
+      default: e = launch_fused_softmax(tmA, tmB, p, st, false); break;
+    }
+    return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+  }
+
+  // unfused: GEMM writes dense bf16 Z [batch, M, N] into the workspace, a row kernel finishes
+  p.Y = static_cast<uint16_t*>(workspace);
+  p.ldy = desc->N;
+  p.batch_stride_y = static_cast<long long>(desc->M) * desc->N;
+  e = launch_plain_gemm(tmA, tmB, p, st);
+  if (e != cudaSuccess) return COMFUSE_ERR_CUDA;
+  RowParams r = {};
+  r.batch = desc->batch; r.M = desc->M; r.N = desc->N;
+  r.Z = static_cast<const uint16_t*>(workspace);
+  r.ldz = desc->N; r.batch_stride_z = static_cast<long long>(desc->M) * desc->N;
+  r.bias = static_cast<const uint16_t*>(a.bias);
+  r.gamma = static_cast<const uint16_t*>(a.gamma);
+  r.beta = static_cast<const uint16_t*>(a.beta);
+  r.residual = static_cast<const uint16_t*>(a.residual);
+  r.ldr = desc->ldr; r.batch_stride_r = bsr;
+  r.mask = desc->mask == COMFUSE_MASK_ADDITIVE ? static_cast<const uint16_t*>(a.mask) : nullptr;
+  r.causal = p.causal;
+  r.alpha = desc->alpha; r.eps = desc->eps;
+  r.Y = static_cast<uint16_t*>(Y);
+  r.ldy = desc->ldy; r.batch_stride_y = bsy;
+  r.row_max = a.row_max; r.row_argmax = a.row_argmax;
+  e = launch_row_epilogue(epi, r, st);
+  return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
+static comfuse_status_t validate_b2b_desc(const comfuse_b2b_desc_t* d) {
+  if (!d) return COMFUSE_ERR_INVALID_ARG;
+  if (d->M < 1 || d->K < 1 || d->N1 < 1 || d->N2 < 1) return COMFUSE_ERR_INVALID_ARG;
+  if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
+  if (d->N2 != d->K) return COMFUSE_ERR_INVALID_ARG;  // the residual is X itself
+  if (!mult8(d->K) || !mult8(d->N1) || !mult8(d->N2)) return COMFUSE_ERR_ALIGNMENT;
+  if (d->fused && !b2b_fused_supported(d->K, d->N1, d->N2)) return COMFUSE_ERR_UNSUPPORTED;
+  if (!d->fused && d->N2 > 8192) return COMFUSE_ERR_UNSUPPORTED;
+  return COMFUSE_OK;
+}
+
+comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size_t* bytes) {
+  if (!bytes) return COMFUSE_ERR_INVALID_ARG;
+  comfuse_status_t s = validate_b2b_desc(desc);
+  if (s != COMFUSE_OK) return s;
+  *bytes = desc->fused ? 0 : (static_cast<size_t>(desc->M) * desc->N1 + static_cast<size_t>(desc->M) * desc->N2) * 2;
+  return COMFUSE_OK;
+}
+
+comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X, const void* W1, const void* b1,
+                                  const void* W2, const void* b2, const void* gamma, const void* beta, void* O,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  comfuse_status_t s = validate_b2b_desc(desc);
+  if (s != COMFUSE_OK) return s;
+  if (!X || !W1 || !W2 || !O) return COMFUSE_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W1) || !aligned16(W2) || !aligned16(O) || !aligned16(b1) || !aligned16(b2) ||
+      !aligned16(gamma) || !aligned16(beta))
+    return COMFUSE_ERR_ALIGNMENT;
+  size_t need = 0;
+  s = comfuse_b2b_workspace_size(desc, &need);
+  if (s != COMFUSE_OK) return s;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return COMFUSE_ERR_WORKSPACE;
+  if (need > 0 && !aligned16(workspace)) return COMFUSE_ERR_ALIGNMENT;
+  const DeviceInfo* dev = nullptr;
+  s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int M = desc->M, K = desc->K, N1 = desc->N1, N2 = desc->N2;
+
+  if (desc->fused) {
+    B2bParams bp = {};
+    bp.M = M; bp.K = K; bp.N1 = N1; bp.N2 = N2;
+    bp.eps = desc->eps;
+    bp.X = static_cast<const uint16_t*>(X);
+    bp.b1 = static_cast<const uint16_t*>(b1);
+    bp.b2 = static_cast<const uint16_t*>(b2);
+    bp.gamma = static_cast<const uint16_t*>(gamma);
+    bp.beta = static_cast<const uint16_t*>(beta);
+    bp.O = static_cast<uint16_t*>(O);
+    bp.status = dev->status_word;
+    bp.timeout_ns = timeout_ns();
+    cudaError_t e = launch_b2b_fused(X, W1, W2, bp, st);
+    return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+  }
+
+  // unfused: P = X.W1 -> S = GELU(P + b1) in place -> O' = S.W2 -> LayerNorm(O' + b2 + X)
+  uint16_t* P = static_cast<uint16_t*>(workspace);
+  uint16_t* Op = P + static_cast<size_t>(M) * N1;
+  CUtensorMap tmA, tmB;
+  FusedParams p = {};
+  p.batch = 1; p.mblocks = (M + 127) / 128; p.alpha = 1.f;
+  p.status = dev->status_word; p.timeout_ns = timeout_ns();
+  if (!make_operand_maps(&tmA, &tmB, X, W1, 1, M, N1, K, K, N1, 0, 0)) return COMFUSE_ERR_CUDA;
+  p.M = M; p.N = N1; p.K = K; p.Y = P; p.ldy = N1;
+  if (launch_plain_gemm(tmA, tmB, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (launch_bias_gelu(P, static_cast<const uint16_t*>(b1), M, N1, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (!make_operand_maps(&tmA, &tmB, P, W2, 1, M, N2, N1, N1, N2, 0, 0)) return COMFUSE_ERR_CUDA;
+  p.N = N2; p.K = N1; p.Y = Op; p.ldy = N2;
+  if (launch_plain_gemm(tmA, tmB, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  RowParams r = {};
+  r.batch = 1; r.M = M; r.N = N2;
+  r.Z = Op; r.ldz = N2;
+  r.bias = static_cast<const uint16_t*>(b2);
+  r.gamma = static_cast<const uint16_t*>(gamma);
+  r.beta = static_cast<const uint16_t*>(beta);
+  r.residual = static_cast<const uint16_t*>(X); r.ldr = K;
+  r.alpha = 1.f; r.eps = desc->eps;
+  r.Y = static_cast<uint16_t*>(O); r.ldy = N2;
+  return launch_row_epilogue(EPI_LN, r, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
+comfuse_status_t comfuse_last_device_status(void* cuda_stream) {
+  const DeviceInfo* dev = nullptr;
+  comfuse_status_t s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  unsigned int word = 0;
+  if (cudaMemcpy(&word, dev->status_word, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (word != 0) {
+    const unsigned int zero = 0;
+    if (cudaMemcpy(dev->status_word, &zero, sizeof(zero), cudaMemcpyHostToDevice) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    return COMFUSE_ERR_TIMEOUT;
+  }
+  return COMFUSE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,30 @@
+// Kernel parameter block of the GEMM -> subgraph kernels (plain data, shared by host and device code).
+#pragma once
+
+#include <stdint.h>
+
+namespace comfuse {
+
+enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3 };
+
+struct FusedParams {
+  int M, N, K, batch;
+  int mblocks;      // ceil(M / 128)
+  int nblocks;      // column blocks of BN per row block (1 unless the epilogue is EPI_NONE)
+  int total_tiles;  // batch * mblocks * nblocks
+  float alpha, eps;
+  int causal;
+  const uint16_t* bias;
+  const uint16_t* gamma;
+  const uint16_t* beta;
+  const uint16_t* residual;
+  long long ldr, batch_stride_r;
+  uint16_t* Y;
+  long long ldy, batch_stride_y;
+  float* row_max;
+  int* row_argmax;
+  unsigned int* status;
+  unsigned long long timeout_ns;
+};
+
+}  // namespace comfuse

@@ -1,0 +1,42 @@
+// Host-side helpers shared by the translation units of the library: tensor-map encoding through the
+// driver entry point (no link-time dependency on libcuda), per-device facts, launch accounting.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fused_params.h"
+
+namespace comfuse {
+
+struct DeviceInfo {
+  int device = -1;
+  int cc_major = 0;
+  int sm_count = 0;
+  unsigned int* status_word = nullptr;  // device address of the module's status word
+};
+
+// Facts about the current device (cached per device).  Returns nullptr if a CUDA call fails.
+const DeviceInfo* current_device_info();
+
+void count_launch();
+
+// Encode a 3-D bf16 tiled tensor map with 128-byte swizzle: dims/strides innermost first; strides in BYTES for
+// dims 1 and 2; box = {64, box_rows, 1}.
+bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                         uint64_t stride2_bytes, uint32_t box_rows);
+
+// Launchers implemented one per translation unit.  Each returns cudaSuccess or the launch error, and
+// cudaErrorInvalidValue if no instantiation covers (N, kind).  `supported_only` asks whether an instantiation
+// exists without launching.
+cudaError_t launch_fused_layernorm(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
+                                   bool supported_only);
+cudaError_t launch_fused_rmsnorm_max(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
+                                     bool supported_only);
+cudaError_t launch_fused_softmax(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
+                                 bool supported_only);
+// Plain GEMM, Z = bf16(A.B), any N that is a multiple of 8.  Fills p.nblocks / p.total_tiles itself.
+cudaError_t launch_plain_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, FusedParams p, cudaStream_t st);
+
+}  // namespace comfuse
