@@ -1,0 +1,74 @@
+"""GPU parity at the full sizes of the named configurations, in the launch configuration the benchmark times.
+The oracle evaluates a seeded sample of rows (always including both sides of the first and last 128-row block
+boundary) one by one; properties that hold at any size cover the rest of the output."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _finite_everywhere(Y):
+    assert torch.isfinite(Y.float()).all().item(), "some output elements were never written (NaN poison left)"
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_config_bert_ffn_out_post_norm(fused, cuda_device):
+    w = wl.config(1)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    _finite_everywhere(got["Y"])
+    rows = wl.sample_rows(w.dims["M"], 192)
+    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c2 fused={fused}")
+    # property over every row: undoing the affine step leaves mean ~0 and variance ~1
+    g = torch.from_numpy(wl.bf16_bits_to_f32(w.tensors["gamma"])).to(got["Y"].device)
+    b = torch.from_numpy(wl.bf16_bits_to_f32(w.tensors["beta"])).to(got["Y"].device)
+    Yn = (got["Y"].float() - b) / g
+    assert Yn.mean(-1).abs().max().item() < 2e-2
+    assert (Yn.var(-1, unbiased=False) - 1).abs().max().item() < 3e-2
+    print("c2", fused, res)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_config_complex_subgraph(fused, cuda_device):
+    w = wl.config(2)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    _finite_everywhere(got["Y"])
+    rows = wl.sample_rows(w.dims["M"], 96)
+    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c3 fused={fused}",
+                          rowmax_tol=5e-3 if fused else 3e-2)
+    # property over every row: the stored row attains its maximum at the reported column, and bf16(row_max) is it
+    Y = got["Y"].float()
+    ymax = Y.max(-1).values
+    picked = Y.gather(-1, got["row_argmax"].long()[:, None])[:, 0]
+    assert torch.equal(picked, ymax)
+    assert torch.equal(got["row_max"].to(torch.bfloat16).float(), ymax)
+    print("c3", fused, res)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_config_scaled_causal_softmax(fused, cuda_device):
+    w = wl.config(3)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    _finite_everywhere(got["Y"])
+    batches = [0, 17, 63]
+    rows = wl.sample_rows(w.dims["M"], 96)
+    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches,
+                          label=f"c4 fused={fused}", softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+    # properties over every row of every batch: strictly upper triangle exactly zero, rows sum to ~1, P[.,0,0] = 1
+    Y = got["Y"]
+    M = w.dims["M"]
+    upper = torch.triu(torch.ones(M, M, dtype=torch.bool, device=Y.device), diagonal=1)
+    assert (Y[:, upper] == 0).all().item()
+    assert (Y.float().sum(-1) - 1).abs().max().item() < 2e-2
+    assert (Y[:, 0, 0] == 1).all().item()
+    print("c4", fused, res)
+
+
+def test_config_tiny_post_norm_full(cuda_device):
+    w = wl.config(0)
+    for fused in (True, False):
+        got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+        print("c1", fused, P.check_outputs(w, got, P.run_oracle(w), label=f"c1 fused={fused}"))

@@ -1,0 +1,173 @@
+"""GPU parity: the fused kernels and the in-library unfused path against the fp64 oracle, element by element, on
+seeded inputs small enough for the oracle to finish in seconds yet spanning several tiles, clusters of 1, 2, 4 and 8
+CTAs, ragged row-block tails and K tails."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+LN_SHAPES = [
+    (256, 256, 256),    # the tiny post-norm configuration: 2 row blocks, 1 CTA per block
+    (300, 768, 200),    # 2-CTA cluster, ragged M (300 = 2*128 + 44), K tail (200 = 3*64 + 8)
+    (130, 512, 72),     # single CTA, 512 TMEM columns
+    (257, 1024, 128),   # 2-CTA cluster of 512 columns
+    (200, 2048, 96),    # 4-CTA cluster
+    (200, 4096, 128),   # 8-CTA cluster, TMEM completely full
+    (1, 256, 8),        # degenerate: one row, one 16-byte K line
+]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,N,K", LN_SHAPES)
+def test_layernorm_epilogue(M, N, K, fused, cuda_device):
+    w = wl.post_norm(M, N, K, seed=M + N + K, affine=(N != 256))
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN {M}x{N}x{K} fused={fused}")
+
+
+def test_layernorm_without_bias_or_residual(cuda_device):
+    w = wl.post_norm(200, 768, 128, seed=9, affine=True)
+    del w.tensors["bias"], w.tensors["residual"]
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label="LN no bias/residual")
+
+
+def test_layernorm_alpha_and_padded_leading_dims(cuda_device):
+    """alpha != 1 and leading dimensions larger than the row length (strided views)."""
+    import paper_2608_03537_b200 as cf
+    from oracle import comfuse_oracle as orc
+    w = wl.post_norm(260, 768, 136, seed=21, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+    Abig = torch.zeros(260, 136 + 24, dtype=torch.bfloat16, device=dev); Abig[:, :136] = T["A"]
+    Bbig = torch.zeros(136, 768 + 8, dtype=torch.bfloat16, device=dev); Bbig[:, :768] = T["B"]
+    Rbig = torch.zeros(260, 768 + 16, dtype=torch.bfloat16, device=dev); Rbig[:, :768] = T["residual"]
+    Ybig = torch.full((260, 768 + 32), 7.0, dtype=torch.bfloat16, device=dev)
+    A, B, R, Y = Abig[:, :136], Bbig[:, :768], Rbig[:, :768], Ybig[:, :768]
+    cf.gemm_epilogue(A, B, Y, cf.EPI_BIAS_RES_LAYERNORM, bias=T["bias"], residual=R, gamma=T["gamma"], beta=T["beta"],
+                     alpha=0.5, eps=1e-3, fused=True)
+    ref = orc.bias_res_layernorm(P.f64(w, "A"), P.f64(w, "B"), P.f64(w, "bias"), P.f64(w, "residual"), P.f64(w, "gamma"),
+                                 P.f64(w, "beta"), 0.5, 1e-3)
+    err = np.abs(P.to_f64(Y) - ref)
+    assert err.max() <= P.TOL_NORM_MAX and err.mean() <= P.TOL_NORM_MEAN
+    assert (Ybig[:, 768:] == 7.0).all()      # the pad columns of the output were not touched
+
+
+RMS_SHAPES = [(300, 256, 200), (140, 768, 64), (200, 1024, 128), (150, 4096, 128)]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,N,K", RMS_SHAPES)
+def test_gelu_rmsnorm_max_epilogue(M, N, K, fused, cuda_device):
+    w = wl.complex_subgraph(M, N, K, seed=M + N)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"RMS {M}x{N}x{K} fused={fused}",
+                    rowmax_tol=5e-3 if fused else 3e-2)
+
+
+def test_argmax_planted_spike(cuda_device):
+    """A residual spike pins the arg max of chosen rows, in every CTA of the cluster and at the chunk borders."""
+    M, N, K = 128, 768, 64
+    w = wl.complex_subgraph(M, N, K, seed=5)
+    R = wl.bf16_bits_to_f32(w.tensors["residual"]).copy()
+    cols = {0: 0, 1: 767, 2: 383, 3: 384, 64: 500, 127: 31}
+    for r, c in cols.items():
+        R[r, c] = 8.0
+    w.tensors["residual"] = wl.f32_to_bf16_bits(R)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    ref = P.run_oracle(w)
+    P.check_outputs(w, got, ref, label="argmax spike")
+    am = got["row_argmax"].cpu().numpy()
+    for r, c in cols.items():
+        assert am[r] == c == ref["row_argmax"][r]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_argmax_exact_tie_reports_lowest_column(fused, cuda_device):
+    """With A = 0 and bias = 0 the pre-norm value is the residual itself (GELU(0) = 0) and gain 1 keeps equal
+    entries equal, so equal spikes are exact ties: the lower column must win across threads, halves and CTAs."""
+    M, N, K = 128, 768, 64
+    w = wl.complex_subgraph(M, N, K, seed=8)
+    w.tensors["A"][:] = 0
+    w.tensors["bias"][:] = 0
+    w.tensors["gamma"] = wl.f32_to_bf16_bits(np.ones(N, dtype=np.float32))
+    R = wl.bf16_bits_to_f32(w.tensors["residual"]).copy()
+    ties = {0: (5, 6), 1: (10, 50), 2: (31, 32), 3: (100, 500), 4: (383, 384), 5: (700, 767), 77: (0, 767)}
+    for r, (c1, c2) in ties.items():
+        R[r, c1] = 8.0
+        R[r, c2] = 8.0
+    w.tensors["residual"] = wl.f32_to_bf16_bits(R)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    ref = P.run_oracle(w)
+    P.check_outputs(w, got, ref, label="argmax tie", rowmax_tol=5e-3 if fused else 3e-2)
+    am = got["row_argmax"].cpu().numpy()
+    for r, (c1, _) in ties.items():
+        assert am[r] == c1 == ref["row_argmax"][r]
+
+
+SOFTMAX_CASES = [
+    # batch, M, N, K, causal
+    (2, 256, 256, 64, True),
+    (3, 512, 512, 64, True),
+    (2, 1024, 1024, 32, True),
+    (2, 2048, 2048, 64, True),     # the 8-CTA cluster instantiation of the attention-score configuration
+    (1, 300, 512, 64, False),      # no mask, ragged M
+    (2, 200, 2048, 40, False),
+    (1, 4096, 4096, 16, True),
+]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M,N,K,causal", SOFTMAX_CASES)
+def test_scaled_masked_softmax_epilogue(batch, M, N, K, causal, fused, cuda_device):
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=N + K, causal=causal)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    ref = P.run_oracle(w)
+    res = P.check_outputs(w, got, ref, label=f"softmax b{batch} {M}x{N}x{K} causal={causal} fused={fused}",
+                          softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+    rowsum = got["Y"].float().sum(-1)
+    assert (rowsum - 1).abs().max().item() < 2e-2       # bf16-rounded probabilities still sum to ~1
+
+
+def test_softmax_large_scores_do_not_overflow(cuda_device):
+    """Scores of magnitude ~1e2 (alpha = 4): exp(x - max) must stay finite, rows must sum to one."""
+    w = wl.scaled_masked_softmax(1, 256, 256, 64, seed=77, causal=True)
+    w.scalars["alpha"] = 4.0
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label="softmax large scores")
+
+
+def test_softmax_additive_mask_unfused_with_fully_masked_row(cuda_device):
+    """The additive-mask variant (unfused path): -inf entries give exact zeros; a fully masked row gives zeros."""
+    batch, M, N, K = 2, 96, 256, 64
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=31, causal=False)
+    g = np.random.default_rng(0)
+    mask = (g.standard_normal((M, N)) * 0.5).astype(np.float32)
+    mask[g.random((M, N)) < 0.3] = -np.inf
+    mask[5, :] = -np.inf
+    w.tensors["mask"] = wl.f32_to_bf16_bits(mask)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=False)
+    ref = P.run_oracle(w)
+    P.check_outputs(w, got, ref, label="softmax additive mask", softmax_tol=P.TOL_SOFTMAX_UNFUSED)
+    assert (got["Y"][:, 5, :] == 0).all()
+
+
+def test_fused_and_unfused_runs_are_bitwise_repeatable(cuda_device):
+    """Merge order across the cluster is fixed (rank order), so two runs give identical bits."""
+    for w in (wl.post_norm(300, 768, 200, seed=3, affine=True), wl.complex_subgraph(150, 4096, 128, seed=4),
+              wl.scaled_masked_softmax(2, 2048, 2048, 64, seed=6)):
+        T = P.dev_tensors(w)
+        a = P.run_gpu(w, T, fused=True)
+        b = P.run_gpu(w, T, fused=True)
+        for k in a:
+            assert torch.equal(a[k].view(torch.int16) if a[k].dtype == torch.bfloat16 else a[k],
+                               b[k].view(torch.int16) if b[k].dtype == torch.bfloat16 else b[k]), (w.name, k)
+
+
+def test_no_timeout_recorded(cuda_device):
+    import paper_2608_03537_b200 as cf
+    assert cf.last_device_status() == cf.OK
