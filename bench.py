@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the joint compute-memory fusion path (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl comfuse|reference]
+
+A step is one pass of the whole hot path over one batch of synthetic input: for the default workload (c2, the
+BERT-base-shaped post-norm FFN output) that is one launch of the fused GEMM + bias + residual + LayerNorm kernel.
+`value` is GEMM TFLOP/s over the K timed steps with every input already resident in HBM; `e2e` repeats the
+measurement with the step's activations copied from pinned host memory and the result copied back inside the
+timed region.  The working set of one step fits the L2 cache, so the steps rotate over several distinct buffer
+sets whose total exceeds L2 (see config.l2).  `--impl reference` times the fp64 CPU oracle on host cores instead.
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank processes its own batch of rows with
+replicated weights -- the path has no exchange step, so there is no collective in the data path -- and `value`
+is the sum over ranks divided by the slowest rank's time (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
+WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
+# captures summarised under profiles/, in bytes; None = not captured.
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": None, "c3": None, "c4": None, "c5": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.001)
+
+    def start(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_call(w, rows):
+    """One evaluation of the fp64 oracle on `rows` of workload `w` (inputs already widened to fp64)."""
+    from oracle import comfuse_oracle as orc
+    t = w._f64
+    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        return orc.b2b_mlp_layernorm(t["X"][rows], t["W1"], t["b1"], t["W2"], t["b2"], t.get("gamma"), t.get("beta"), w.scalars["eps"])
+    if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+        return orc.bias_res_layernorm(t["A"][rows], t["B"], t["bias"], t["residual"][rows], t.get("gamma"), t.get("beta"),
+                                      w.scalars["alpha"], w.scalars["eps"])
+    if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+        return orc.bias_gelu_res_rmsnorm_max(t["A"][rows], t["B"], t["bias"], t["residual"][rows], t["gamma"],
+                                             w.scalars["alpha"], w.scalars["eps"])
+    mask = orc.causal_mask(w.dims["M"], w.dims["N"], rows=rows) if w.scalars.get("causal") else None
+    return orc.scale_mask_softmax(t["A"][0][rows], t["B"][0], w.scalars["alpha"], mask)
+
+
+def widen_for_oracle(w, softmax_batches=1):
+    w._f64 = {}
+    for k, v in w.tensors.items():
+        if w.kind == wl.KIND_SCALE_MASK_SOFTMAX:
+            v = v[:softmax_batches]
+        w._f64[k] = wl.bf16_to_f64(v)
+
+
+def sample_flops(w, nrows):
+    d = w.dims
+    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        return 2.0 * nrows * (d["K"] * d["N1"] + d["N1"] * d["N2"])
+    return 2.0 * nrows * d["N"] * d["K"]
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return int(max(n)) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(w, nrows, steps, warmup):
+    rows = np.arange(min(nrows, w.dims["M"]))
+    for _ in range(warmup):
+        oracle_call(w, rows)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_call(w, rows)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    return dt, sample_flops(w, len(rows))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    name = args.workload
+    w = wl.config(WORKLOADS[name])
+    widen_for_oracle(w)
+    # size the per-step sample so that steps + warmup stay within a couple of minutes
+    probe_rows = 64
+    dt, fl = time_oracle(w, probe_rows, 1, 1)
+    budget_s = 120.0 / max(args.steps + args.warmup, 1)
+    nrows = int(min(w.dims["M"], max(probe_rows, probe_rows * min(budget_s, 2.0) / max(dt, 1e-6))))
+    nrows = max(64, (nrows // 64) * 64)
+    dt, fl = time_oracle(w, nrows, args.steps, args.warmup)
+    tflops = fl / dt / 1e12
+    cores = blas_threads()
+    sample = f"rows 0..{nrows - 1} of {w.name} per step, fp64 numpy oracle"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, **w.dims, "sample_rows_per_step": nrows},
+        "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ CUDA arm
+def run_comfuse(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2608_03537_b200 as cf
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    cf.lib()  # fail loudly if the CUDA library is missing
+
+    name = args.workload
+    w = wl.config(WORKLOADS[name])
+    peaks = load_peaks()
+    fused = not args.unfused
+
+    def to_dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(dev)
+
+    # ---- buffer sets: per-step activations (inputs read once per step and the outputs) are replicated until the
+    # rotation exceeds 3x the L2 capacity; weights and row vectors are shared (they are meant to be L2 resident)
+    act_names = {"A", "residual", "X"} if w.kind != wl.KIND_SCALE_MASK_SOFTMAX else {"A", "B"}
+    base = {k: to_dev(v) for k, v in w.tensors.items()}
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    d = w.dims
+    out_shape = (d["batch"], d["M"], d["N"]) if "batch" in d else (d["M"], d.get("N", d.get("N2")))
+    per_set = sum(base[k].numel() * 2 for k in base if k in act_names) + int(np.prod(out_shape)) * 2
+    nsets = int(max(2, min(16, -(-3 * l2_bytes // per_set))))
+    sets = []
+    for i in range(nsets):
+        s = {k: (v.clone() if (k in act_names and i > 0) else v) for k, v in base.items()}
+        s["Y"] = torch.zeros(out_shape, dtype=torch.bfloat16, device=dev)
+        if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+            s["row_max"] = torch.zeros(out_shape[:-1], dtype=torch.float32, device=dev)
+            s["row_argmax"] = torch.zeros(out_shape[:-1], dtype=torch.int32, device=dev)
+        sets.append(s)
+
+    # workspace (unfused path only)
+    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        ws_bytes = cf.b2b_workspace_size(cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused))
+    else:
+        kind = {wl.KIND_BIAS_RES_LAYERNORM: cf.EPI_BIAS_RES_LAYERNORM,
+                wl.KIND_BIAS_GELU_RES_RMSNORM_MAX: cf.EPI_BIAS_GELU_RES_RMSNORM_MAX,
+                wl.KIND_SCALE_MASK_SOFTMAX: cf.EPI_SCALE_MASK_SOFTMAX}[w.kind]
+        mask = cf.MASK_CAUSAL if w.scalars.get("causal") else cf.MASK_NONE
+        desc = cf.make_gemm_desc(base["A"], base["B"], sets[0]["Y"], kind, residual=base.get("residual"), mask=mask, fused=fused)
+        ws_bytes = cf.workspace_size(desc)
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+
+    def step(s, use_fused=fused, workspace=ws):
+        if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+            cf.b2b_gemm(s["X"], s["W1"], s["b1"], s["W2"], s["b2"], s["Y"], gamma=s.get("gamma"), beta=s.get("beta"),
+                        eps=w.scalars["eps"], fused=use_fused, workspace=workspace)
+        elif w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+            cf.gemm_epilogue(s["A"], s["B"], s["Y"], cf.EPI_BIAS_RES_LAYERNORM, bias=s.get("bias"), residual=s.get("residual"),
+                             gamma=s.get("gamma"), beta=s.get("beta"), alpha=w.scalars["alpha"], eps=w.scalars["eps"],
+                             fused=use_fused, workspace=workspace)
+        elif w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+            cf.gemm_epilogue(s["A"], s["B"], s["Y"], cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, bias=s.get("bias"),
+                             residual=s.get("residual"), gamma=s.get("gamma"), alpha=w.scalars["alpha"], eps=w.scalars["eps"],
+                             row_max=s["row_max"], row_argmax=s["row_argmax"], fused=use_fused, workspace=workspace)
+        else:
+            cf.gemm_epilogue(s["A"], s["B"], s["Y"], cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"],
+                             mask=cf.MASK_CAUSAL if w.scalars.get("causal") else cf.MASK_NONE, fused=use_fused,
+                             workspace=workspace)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(nsteps, fn):
+        """K steps bracketed by barrier + synchronize; device time from CUDA events on the launching stream."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for i in range(nsteps):
+            fn(i)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ---- warm-up, then the timed region
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % nsets])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    launches0 = cf.launch_count()
+    sampler.start()
+    ms_total = timed(args.steps, lambda i: step(sets[i % nsets]))
+    clocks = sampler.stop()
+    launches = cf.launch_count() - launches0
+    status = cf.last_device_status()
+    if status != cf.OK:
+        raise SystemExit(f"device status {status} after the timed region")
+    ms_step = ms_total / args.steps
+    flops = w.gemm_flops()
+    bytes_min = w.min_hbm_bytes()
+    value = world * flops / (ms_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the fused kernel; one launch per step)
+    t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = bytes_min / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        roof = {"bound": "tensor", "achieved": flops / (ms_step * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": bytes_min / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
+    roof["peak_source"] = f"of {peaks['source']} (burst figure, kernel timed alone)"
+    roof["kernel"] = "fused_gemm_kernel" if w.kind != wl.KIND_B2B_MLP_LAYERNORM else "b2b_gemm_kernel"
+    roof["algorithmic_flops_per_launch"] = flops
+    roof["algorithmic_bytes_per_launch"] = bytes_min
+    roof["roofline_us"] = max(t_tensor, t_hbm) * 1e6
+
+    extra = {}
+    if not args.kernel_only:
+        # ---- the in-library unfused path on the same buffers (context: speedup of fusion)
+        try:
+            other = not fused
+            if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+                ob = cf.b2b_workspace_size(cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], other))
+            else:
+                desc.fused = int(other)
+                ob = cf.workspace_size(desc)
+            ws2 = torch.empty(max(ob, 16), dtype=torch.uint8, device=dev)
+            for i in range(3):
+                step(sets[i % nsets], other, ws2)
+            n2 = max(3, min(args.steps, 50))
+            ms_other = timed(n2, lambda i: step(sets[i % nsets], other, ws2)) / n2
+            key = "unfused_ms_per_step" if fused else "fused_ms_per_step"
+            extra[key] = ms_other
+            extra["speedup_vs_unfused"] = (ms_other / ms_step) if fused else (ms_step / ms_other)
+            del ws2
+        except cf.ComfuseError as e:
+            extra["unfused_error"] = str(e)
+
+    # ---- end to end: activations from pinned host memory, result back to pinned host memory, every step
+    if args.kernel_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": "TFLOP/s", "ms_per_step": ms_step, "steps": args.steps,
+                              "config": {"workload": w.name}, "roofline": roof, "gpu_launches": int(launches), "kernel_only": True}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    host_in = {k: torch.from_numpy(np.ascontiguousarray(w.tensors[k]).view(np.int16)).view(torch.bfloat16).pin_memory()
+               for k in w.tensors if k in act_names}
+    host_out = torch.empty(out_shape, dtype=torch.bfloat16).pin_memory()
+    h2d = sum(t.numel() * 2 for t in host_in.values())
+    d2h = host_out.numel() * 2
+
+    def e2e_step(i):
+        s = sets[i % nsets]
+        for k, t in host_in.items():
+            s[k].copy_(t, non_blocking=True)
+        step(s)
+        host_out.copy_(s["Y"], non_blocking=True)
+
+    n_e2e = max(3, min(args.steps, 20))
+    for i in range(2):
+        e2e_step(i)
+    ms_e2e = timed(n_e2e, e2e_step) / n_e2e
+    e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e}
+
+    # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only, on a bounded sample
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.kernel_only:
+        widen_for_oracle(w)
+        dt, fl = time_oracle(w, 64, 1, 1)
+        nrows = int(min(w.dims["M"], max(64, 64 * 10.0 / max(dt, 1e-6))))   # aim at ~10 s of CPU work
+        nrows = max(64, (nrows // 64) * 64)
+        dt, fl = time_oracle(w, nrows, 1, 0)
+        cpu = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle",
+               "sample": f"rows 0..{nrows - 1} of {w.name}, one pass, {dt:.2f} s", "seconds": dt}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": w.name, **w.dims, "path": "fused" if fused else "unfused",
+                       "parallelism": f"replicas x{world}, rows sharded, no collective",
+                       "l2": f"rotating {nsets} buffer sets of {per_set / 1e6:.1f} MB activations+outputs "
+                             f"({nsets * per_set / 1e6:.0f} MB > L2 {l2_bytes / 1e6:.0f} MB), weights shared"},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            **extra,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="comfuse", choices=["comfuse", "reference"])
+    ap.add_argument("--unfused", action="store_true", help="time the in-library unfused path as the main number")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the unfused, end-to-end and CPU legs (for profiler runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_comfuse(args)
+
+
+if __name__ == "__main__":
+    main()
