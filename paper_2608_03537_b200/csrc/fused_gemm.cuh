@@ -24,6 +24,7 @@
 //   stage 3  (RMSNorm+max only) a second reduction (row max / argmax) through the same exchange buffers.
 #pragma once
 
+#include "epilogue_common.cuh"
 #include "fused_params.h"
 #include "sm100_primitives.cuh"
 
@@ -53,83 +54,6 @@ struct FusedCfg {
   static_assert((BNS / 32) % 2 == 0, "two epilogue warps split the 32-column chunks evenly");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
-
-// ------------------------------------------------------------------------------------------------ merges
-// Partials are float2.  The functors merge `b` (nb elements) into `a` (na elements).
-struct MergeWelford {  // (mean, M2); pairwise update of Chan et al.
-  __device__ __forceinline__ float2 operator()(float2 a, float na, float2 b, float nb) const {
-    const float n = na + nb;
-    const float delta = b.x - a.x;
-    return make_float2(fmaf(delta, nb / n, a.x), a.y + b.y + delta * delta * (na * nb / n));
-  }
-};
-struct MergeSum {  // (sum, unused)
-  __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const { return make_float2(a.x + b.x, 0.f); }
-};
-struct MergeMaxSumExp2 {  // (max, sum of 2^(t - max)); a partial with max = -inf carries nothing
-  __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const {
-    const float m = fmaxf(a.x, b.x);
-    const float fa = (a.x == -INFINITY) ? 0.f : ex2_approx(a.x - m);
-    const float fb = (b.x == -INFINITY) ? 0.f : ex2_approx(b.x - m);
-    return make_float2(m, a.y * fa + b.y * fb);
-  }
-};
-struct MergeArgmax {  // (value, column index bits); ties -> lower index
-  __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const {
-    const int ia = __float_as_int(a.y), ib = __float_as_int(b.y);
-    const bool take_b = (b.x > a.x) || (b.x == a.x && ib < ia);
-    return take_b ? b : a;
-  }
-};
-
-// The reduce phase above thread level.  All 256 epilogue threads of every CTA of the cluster call this the same
-// number of times.  `per_thread_count` = elements behind each thread's partial (half of the CTA's columns).
-template <int CN, class Merge>
-__device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thread_count, Merge merge, float2* s_pre,
-                                                     float2* s_stats, uint32_t stats_bar, int row, int h,
-                                                     uint32_t rank, int& xpar, uint32_t& xphase, const WaitCtx& w) {
-  // level 2: the two column-halves of the row, through shared memory
-  s_pre[(xpar * 2 + h) * 128 + row] = mine;
-  named_barrier_sync(1, 256);
-  const float2 cta_partial = merge(s_pre[(xpar * 2 + 0) * 128 + row], per_thread_count,
-                                   s_pre[(xpar * 2 + 1) * 128 + row], per_thread_count);
-  const float cta_count = 2.f * per_thread_count;
-  // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks of parity h
-  float2* slot = s_stats + (xpar * CN + rank) * 128 + row;
-  if constexpr (CN == 1) {
-    if (h == 0) {
-      *slot = cta_partial;
-      mbar_arrive(stats_bar);
-    }
-  } else {
-    const uint32_t slot_addr = smem_u32(slot);
-#pragma unroll
-    for (int dst = 0; dst < CN; ++dst) {
-      if ((dst & 1) == h) {
-        st_cluster_f32x2(map_to_cta(slot_addr, dst), cta_partial.x, cta_partial.y);
-        mbar_arrive_cluster(map_to_cta(stats_bar, dst));
-      }
-    }
-  }
-  if constexpr (CN == 1) {
-    mbar_wait<false>(stats_bar, xphase, w);
-  } else {
-    mbar_wait<true>(stats_bar, xphase, w);
-  }
-  float2 acc = s_stats[(xpar * CN + 0) * 128 + row];
-#pragma unroll
-  for (int c = 1; c < CN; ++c) acc = merge(acc, cta_count * c, s_stats[(xpar * CN + c) * 128 + row], cta_count);
-  xpar ^= 1;
-  xphase ^= 1;
-  __syncwarp();
-  return acc;
-}
-
-__device__ __forceinline__ void store_chunk_bf16(uint16_t* dst, const uint32_t (&pk)[16]) {
-  uint4* d = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) d[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-}
 
 // ------------------------------------------------------------------------------------------------ kernel
 template <int EPI, int BNS, int NSUB, int CN, int NSTAGES>

@@ -10,6 +10,7 @@ enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3 };
 struct FusedParams {
   int M, N, K, batch;
   int mblocks;      // ceil(M / 128)
+  int mpairs;       // ceil(mblocks / 2): pairs of row blocks (CTA-pair kernels)
   int nblocks;      // column blocks of BN per row block (1 unless the epilogue is EPI_NONE)
   int total_tiles;  // batch * mblocks * nblocks
   float alpha, eps;
