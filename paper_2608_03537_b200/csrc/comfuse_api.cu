@@ -94,13 +94,19 @@ bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t d0, uint64
 
 namespace {
 
-// Tensor maps of a GEMM's operands: A [batch, M, K] (K contiguous), B [batch, K, N] (N contiguous).
-bool make_operand_maps(CUtensorMap* tmA, CUtensorMap* tmB, const void* A, const void* B, int batch, int M, int N, int K,
-                       long long lda, long long ldb, long long bsa, long long bsb) {
-  const uint64_t sa2 = static_cast<uint64_t>(batch > 1 ? bsa : static_cast<long long>(M) * lda) * 2;
-  const uint64_t sb2 = static_cast<uint64_t>(batch > 1 ? bsb : static_cast<long long>(K) * ldb) * 2;
-  return encode_tmap_bf16_3d(tmA, A, K, M, batch, static_cast<uint64_t>(lda) * 2, sa2, 128) &&
-         encode_tmap_bf16_3d(tmB, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, sb2, 64);
+// Tensor maps of a GEMM -> subgraph call.  R may be null (no residual): its map is then left zeroed and never used.
+bool make_gemm_maps(GemmMaps* maps, const void* A, const void* B, const void* R, const void* Y, int batch, int M, int N, int K,
+                    long long lda, long long ldb, long long ldr, long long ldy, long long bsa, long long bsb, long long bsr,
+                    long long bsy) {
+  std::memset(maps, 0, sizeof(*maps));
+  auto bs = [&](long long given, long long rows, long long ld) {
+    return static_cast<uint64_t>(batch > 1 ? given : rows * ld) * 2;
+  };
+  if (!encode_tmap_bf16_3d(&maps->A, A, K, M, batch, static_cast<uint64_t>(lda) * 2, bs(bsa, M, lda), 128)) return false;
+  if (!encode_tmap_bf16_3d(&maps->B, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, K, ldb), 64)) return false;
+  if (!encode_tmap_bf16_3d(&maps->Y, Y, N, M, batch, static_cast<uint64_t>(ldy) * 2, bs(bsy, M, ldy), 128)) return false;
+  if (R && !encode_tmap_bf16_3d(&maps->R, R, N, M, batch, static_cast<uint64_t>(ldr) * 2, bs(bsr, M, ldr), 128)) return false;
+  return true;
 }
 
 comfuse_status_t check_device(const DeviceInfo** out) {
@@ -146,13 +152,13 @@ comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
   if (d->mask == COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
   p.N = d->N;
-  CUtensorMap dummy;
+  GemmMaps dummy;
   std::memset(&dummy, 0, sizeof(dummy));
   cudaError_t e = cudaErrorInvalidValue;
   switch (kind_to_epi(d->kind)) {
-    case EPI_LN: e = launch_fused_layernorm(dummy, dummy, p, nullptr, true); break;
-    case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(dummy, dummy, p, nullptr, true); break;
-    case EPI_SOFTMAX: e = launch_fused_softmax(dummy, dummy, p, nullptr, true); break;
+    case EPI_LN: e = launch_fused_layernorm(dummy, p, nullptr, true); break;
+    case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(dummy, p, nullptr, true); break;
+    case EPI_SOFTMAX: e = launch_fused_softmax(dummy, p, nullptr, true); break;
     default: break;
   }
   return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
@@ -227,10 +233,18 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   if (s != COMFUSE_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
-  CUtensorMap tmA, tmB;
-  if (!make_operand_maps(&tmA, &tmB, A, B, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, desc->batch_stride_a,
-                         desc->batch_stride_b))
-    return COMFUSE_ERR_CUDA;
+  const long long bsr = desc->batch > 1 ? desc->batch_stride_r : 0;
+  const long long bsy = desc->batch > 1 ? desc->batch_stride_y : 0;
+  GemmMaps maps;
+  if (desc->fused) {
+    if (!make_gemm_maps(&maps, A, B, a.residual, Y, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, desc->ldr,
+                        desc->ldy, desc->batch_stride_a, desc->batch_stride_b, bsr, bsy))
+      return COMFUSE_ERR_CUDA;
+  } else {  // the GEMM's output is the dense bf16 Z in the workspace
+    if (!make_gemm_maps(&maps, A, B, nullptr, workspace, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, 0, desc->N,
+                        desc->batch_stride_a, desc->batch_stride_b, 0, static_cast<long long>(desc->M) * desc->N))
+      return COMFUSE_ERR_CUDA;
+  }
 
   FusedParams p = {};
   p.M = desc->M; p.N = desc->N; p.K = desc->K; p.batch = desc->batch;
@@ -241,8 +255,6 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
   p.status = dev->status_word;
   p.timeout_ns = timeout_ns();
-  const long long bsr = desc->batch > 1 ? desc->batch_stride_r : 0;
-  const long long bsy = desc->batch > 1 ? desc->batch_stride_y : 0;
 
   cudaError_t e;
   if (desc->fused) {
@@ -255,9 +267,9 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
     p.ldy = desc->ldy; p.batch_stride_y = bsy;
     p.row_max = a.row_max; p.row_argmax = a.row_argmax;
     switch (epi) {
-      case EPI_LN: e = launch_fused_layernorm(tmA, tmB, p, st, false); break;
-      case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(tmA, tmB, p, st, false); break;
-      default: e = launch_fused_softmax(tmA, tmB, p, st, false); break;
+      case EPI_LN: e = launch_fused_layernorm(maps, p, st, false); break;
+      case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(maps, p, st, false); break;
+      default: e = launch_fused_softmax(maps, p, st, false); break;
     }
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }
@@ -266,7 +278,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.Y = static_cast<uint16_t*>(workspace);
   p.ldy = desc->N;
   p.batch_stride_y = static_cast<long long>(desc->M) * desc->N;
-  e = launch_plain_gemm(tmA, tmB, p, st);
+  e = launch_plain_gemm(maps, p, st);
   if (e != cudaSuccess) return COMFUSE_ERR_CUDA;
   RowParams r = {};
   r.batch = desc->batch; r.M = desc->M; r.N = desc->N;
@@ -345,17 +357,17 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
   // unfused: P = X.W1 -> S = GELU(P + b1) in place -> O' = S.W2 -> LayerNorm(O' + b2 + X)
   uint16_t* P = static_cast<uint16_t*>(workspace);
   uint16_t* Op = P + static_cast<size_t>(M) * N1;
-  CUtensorMap tmA, tmB;
+  GemmMaps maps;
   FusedParams p = {};
   p.batch = 1; p.mblocks = (M + 127) / 128; p.alpha = 1.f;
   p.status = dev->status_word; p.timeout_ns = timeout_ns();
-  if (!make_operand_maps(&tmA, &tmB, X, W1, 1, M, N1, K, K, N1, 0, 0)) return COMFUSE_ERR_CUDA;
+  if (!make_gemm_maps(&maps, X, W1, nullptr, P, 1, M, N1, K, K, N1, 0, N1, 0, 0, 0, 0)) return COMFUSE_ERR_CUDA;
   p.M = M; p.N = N1; p.K = K; p.Y = P; p.ldy = N1;
-  if (launch_plain_gemm(tmA, tmB, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (launch_plain_gemm(maps, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
   if (launch_bias_gelu(P, static_cast<const uint16_t*>(b1), M, N1, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
-  if (!make_operand_maps(&tmA, &tmB, P, W2, 1, M, N2, N1, N1, N2, 0, 0)) return COMFUSE_ERR_CUDA;
+  if (!make_gemm_maps(&maps, P, W2, nullptr, Op, 1, M, N2, N1, N1, N2, 0, N2, 0, 0, 0, 0)) return COMFUSE_ERR_CUDA;
   p.N = N2; p.K = N1; p.Y = Op; p.ldy = N2;
-  if (launch_plain_gemm(tmA, tmB, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (launch_plain_gemm(maps, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
   RowParams r = {};
   r.batch = 1; r.M = M; r.N = N2;
   r.Z = Op; r.ldz = N2;

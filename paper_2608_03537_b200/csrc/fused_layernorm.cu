@@ -1,25 +1,19 @@
-// Instantiations of the fused kernels for  Y = LayerNorm(alpha*A.B + bias + R) * gamma + beta  (Sec. 3.2, Fig. 3 case).
-#include <cstdlib>
-
+// Instantiations of the fused kernel for  Y = LayerNorm(alpha*A.B + bias + R) * gamma + beta  (Sec. 3.2, Fig. 3 case).
 #include "fused_launch.cuh"
 
 namespace comfuse {
 
-cudaError_t launch_fused_layernorm(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
-                                bool supported_only) {
-  static const bool single_cta = std::getenv("COMFUSE_SINGLE_CTA_MMA") != nullptr;  // bring-up: the 1-CTA UMMA kernels
-#define COMFUSE_CASE(n, b0, b1, cn, nacc, nst, sbns, snsub, scn, snst)                                   \
-  case n:                                                                                                \
-    if (supported_only) return cudaSuccess;                                                              \
-    return single_cta ? launch_fused_instance<EPI_LN, sbns, snsub, scn, snst>(tmA, tmB, p, st)           \
-                      : launch_pair_instance<EPI_LN, b0, b1, cn, nacc, nst>(tmA, tmB, p, st);
+cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
+#define COMFUSE_CASE(n, b0, b1, cn, nst) \
+  case n:                                \
+    return supported_only ? cudaSuccess : launch_pair_instance<EPI_LN, b0, b1, cn, nst>(maps, p, st);
   switch (p.N) {
-    COMFUSE_CASE(256, 256, 0, 1, 2, 6, 128, 2, 1, 6)
-    COMFUSE_CASE(512, 256, 256, 1, 1, 4, 256, 2, 1, 4)
-    COMFUSE_CASE(768, 256, 128, 2, 1, 5, 192, 2, 2, 5)
-    COMFUSE_CASE(1024, 256, 256, 2, 1, 4, 256, 2, 2, 4)
-    COMFUSE_CASE(2048, 256, 256, 4, 1, 4, 256, 2, 4, 4)
-    COMFUSE_CASE(4096, 256, 256, 8, 1, 4, 256, 2, 8, 4)
+    COMFUSE_CASE(256, 256, 0, 1, 5)
+    COMFUSE_CASE(512, 256, 256, 1, 5)
+    COMFUSE_CASE(768, 256, 128, 2, 5)
+    COMFUSE_CASE(1024, 256, 256, 2, 5)
+    COMFUSE_CASE(2048, 256, 256, 4, 5)
+    COMFUSE_CASE(4096, 256, 256, 8, 5)
     default:
       return cudaErrorInvalidValue;
   }

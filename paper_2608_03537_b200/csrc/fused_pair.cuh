@@ -1,4 +1,4 @@
-// GEMM -> row-reduction subgraph in one kernel, CTA-pair edition (Stage-Stream Execution Model, Sec. 3).
+// GEMM -> row-reduction subgraph in one kernel (Stage-Stream Execution Model, Sec. 3), built on CTA pairs.
 //
 // Why pairs: one SM's shared memory delivers 128 B/clk, and a 128 x 256 x 16 bf16 UMMA that reads both operands
 // from shared memory already needs 96 B/clk before TMA has written the next tiles.  With cta_group::2 two CTAs
@@ -13,9 +13,19 @@
 // block pairs with a stride of the cluster count.
 //
 // Inside a CTA (10 warps): warp 0 = TMA producer, warp 1 = TMEM allocation and (even CTA only) UMMA issue,
-// warps 2-9 = epilogue (thread = one accumulator row; the two warps of a lane quarter split the 32-column chunks).
-// The CTA's BN = BNS0 + BNS1 accumulator columns advance in lock step (A is fetched once per K block), NACC
-// accumulator buffers let the next tile's MainLoop overlap this tile's epilogue when 2*BN <= 512 columns.
+// warps 2-9 = epilogue (thread = one accumulator row; the two warps of a lane quarter split every 64-column
+// group into two 32-column fragments).
+//
+// Pipelining (Sec. 3.3, PingPong at sub-tile grain).  The CTA's BN columns are one or two sub-tiles, each with its
+// own TMEM slot and full/empty barriers.  The MainLoop of sub-tile 1 runs while the epilogue's stage 1 works on
+// sub-tile 0, and the next tile's sub-tile 0 starts as soon as stage 2 has drained that slot.  A CTA with a single
+// sub-tile of at most 256 columns alternates between the two slots from tile to tile.
+//
+// One circular shared-memory buffer feeds both consumers (the unified multi-stage buffer of Sec. 4.2, applied to
+// the epilogue operand): after the K blocks of a sub-tile the producer pushes that sub-tile's residual tile through
+// the same ring, 128 rows x 64 columns per TMA box, so the epilogue reads the residual from swizzled shared memory
+// instead of issuing one scattered global load per row.  Results leave the same way: 128 x 64 bf16 boxes are
+// written to a swizzled staging buffer and stored with TMA.
 #pragma once
 
 #include "epilogue_common.cuh"
@@ -24,39 +34,63 @@
 
 namespace comfuse {
 
-template <int EPI, int BNS0, int BNS1, int CN, int NACC, int NSTAGES>
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES>
 struct PairCfg {
   static constexpr int kThreads = 320;
   static constexpr int kEpiThreads = 256;
+  static constexpr int NSUB = BNS1 > 0 ? 2 : 1;
   static constexpr int BN = BNS0 + BNS1;
+  static constexpr int BNSMAX = BNS0 > BNS1 ? BNS0 : BNS1;
   static constexpr int A_BYTES = 128 * 64 * 2;
-  static constexpr int B0_BYTES = (BNS0 / 2) * 64 * 2;  // this CTA's half of sub-tile 0's B tile
-  static constexpr int B1_BYTES = (BNS1 / 2) * 64 * 2;
-  static constexpr int STAGE_BYTES = A_BYTES + B0_BYTES + B1_BYTES;
-  static constexpr int ACC_COLS = NACC * BN;
+  static constexpr int GROUP_BYTES = 128 * 64 * 2;                        // one 128 x 64 bf16 box
+  static constexpr int STAGE_BYTES = A_BYTES + (BNSMAX / 2) * 64 * 2;     // A tile + this CTA's half of the B tile
+  static constexpr int GROUPS_PER_STAGE = STAGE_BYTES / GROUP_BYTES;      // residual boxes one ring stage can carry
+  static constexpr int ACC_COLS = NSUB == 2 ? BN : 2 * BNS0;              // two TMEM slots
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
-  static constexpr int OFF_VEC = NSTAGES * STAGE_BYTES;
+  static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
+  static constexpr int YBUF_BYTES = 2 * GROUP_BYTES;
+  static constexpr int OFF_VEC = OFF_YBUF + YBUF_BYTES;
   static constexpr int VEC_BYTES = 3 * BN * 4;
   static constexpr int OFF_STATS = OFF_VEC + VEC_BYTES;
   static constexpr int STATS_BYTES = 2 * CN * 128 * 8;
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
   static constexpr int PRE_BYTES = 2 * 2 * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 2 * NSTAGES + 2 * NACC + 2;
+  static constexpr int NUM_BARS = 3 * NSTAGES + 4 + 2;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
   static_assert(BNS0 > 0 && ACC_COLS <= 512, "accumulators must fit the 512 TMEM columns");
+  static_assert(NSTAGES <= 8, "per-stage phase bits are kept in one byte");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
 };
 
-template <int EPI, int BNS0, int BNS1, int CN, int NACC, int NSTAGES>
+// Position in the circular buffer; every role walks the same sequence of stage uses.
+template <int NSTAGES>
+struct RingPos {
+  int stage = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance() {
+    if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+  }
+  __device__ __forceinline__ void skip(int n) {
+    stage += n;
+    while (stage >= NSTAGES) { stage -= NSTAGES; phase ^= 1u; }
+  }
+};
+
+// 16-byte chunk `c` (0..7) of row `r` inside a 128-byte-swizzled 128 x 64 bf16 box.
+__device__ __forceinline__ uint32_t swz128(int r, int c) { return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES>
 __global__ void __launch_bounds__(320, 1)
-fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FusedParams p) {
-  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NACC, NSTAGES>;
+fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
+  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES>;
   constexpr int BN = Cfg::BN;
-  constexpr int CHUNK_PAIRS = BN / 64;  // each epilogue thread handles one 32-column chunk of every 64 columns
+  constexpr int NSUB = Cfg::NSUB;
+  constexpr int GPS = Cfg::GROUPS_PER_STAGE;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -69,11 +103,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   float2* s_stats = reinterpret_cast<float2*>(smem + Cfg::OFF_STATS);
   float2* s_pre = reinterpret_cast<float2*>(smem + Cfg::OFF_PRE);
   const uint32_t bar_base = smem_base + Cfg::OFF_BAR;
-  auto bar_full = [&](int s) { return bar_base + 8u * s; };
-  auto bar_empty = [&](int s) { return bar_base + 8u * (NSTAGES + s); };
-  auto bar_tfull = [&](int a) { return bar_base + 8u * (2 * NSTAGES + a); };
-  auto bar_tempty = [&](int a) { return bar_base + 8u * (2 * NSTAGES + NACC + a); };
-  const uint32_t bar_stats = bar_base + 8u * (2 * NSTAGES + 2 * NACC);
+  auto bar_full = [&](int s) { return bar_base + 8u * s; };                     // K-block stage landed (even CTA)
+  auto bar_empty = [&](int s) { return bar_base + 8u * (NSTAGES + s); };        // stage may be overwritten
+  auto bar_rfull = [&](int s) { return bar_base + 8u * (2 * NSTAGES + s); };    // residual stage landed (own CTA)
+  auto bar_tfull = [&](int a) { return bar_base + 8u * (3 * NSTAGES + a); };    // accumulator slot complete
+  auto bar_tempty = [&](int a) { return bar_base + 8u * (3 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
+  const uint32_t bar_stats = bar_base + 8u * (3 * NSTAGES + 4);
   const uint32_t bar_drain = bar_stats + 8u;
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
@@ -81,25 +116,27 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
-  const uint32_t pm = rank & 1u;           // which row block of the pair
-  const uint32_t crank = rank >> 1;        // which column range
-  const uint32_t leader = rank & ~1u;      // cluster rank of the CTA that issues the pair's UMMAs
+  const uint32_t pm = rank & 1u;       // which row block of the pair
+  const uint32_t crank = rank >> 1;    // which column range
+  const uint32_t leader = rank & ~1u;  // cluster rank of the CTA that issues the pair's UMMAs
   const uint32_t peer = rank ^ 1u;
   constexpr int CLUSTER = 2 * CN;
   const int cluster_id = blockIdx.x / CLUSTER;
   const int num_clusters = gridDim.x / CLUSTER;
   const int KB = (p.K + 63) >> 6;
+  const bool has_res = (EPI == EPI_LN || EPI == EPI_RMS_MAX) && p.residual != nullptr;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
 
   // -------------------------------------------------------------------------------------------- set-up
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
-      mbar_init(bar_full(s), 2);   // one arrive.expect_tx from each CTA of the pair (used in the even CTA only)
-      mbar_init(bar_empty(s), 1);  // one commit from the issuing CTA
+      mbar_init(bar_full(s), 2);   // one arrive.expect_tx from each CTA of the pair
+      mbar_init(bar_empty(s), 1);  // one commit from the issuing CTA, or one arrive from the epilogue (residual stage)
+      mbar_init(bar_rfull(s), 1);
     }
-    for (int a = 0; a < NACC; ++a) {
+    for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull(a), 1);
-      mbar_init(bar_tempty(a), 2 * Cfg::kEpiThreads);  // both CTAs' epilogue threads (used in the even CTA only)
+      mbar_init(bar_tempty(a), 2 * Cfg::kEpiThreads);  // both CTAs' epilogue threads
     }
     mbar_init(bar_stats, CN * 128);
     mbar_init(bar_drain, 1);
@@ -107,12 +144,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     fence_mbar_init();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
+    prefetch_tensormap(&tmY);
+    if (has_res) prefetch_tensormap(&tmR);
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(s_tmem_base), Cfg::TMEM_COLS);
     tmem_relinquish_alloc_permit_pair();
   }
   if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
+    // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once
     const int c0 = crank * BN;
     for (int i = threadIdx.x; i < BN; i += Cfg::kThreads) {
       const int c = c0 + i;
@@ -138,91 +178,97 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     mpair0 = mp * 256;
     ncta0 = (nb * CN + static_cast<int>(crank)) * BN;
   };
-  // Number of leading sub-tiles the pair has to compute: a sub-tile is dropped when it lies past N, or when the
-  // causal mask removes it for BOTH row blocks of the pair.  Every role evaluates the same predicate.
-  auto live_subtiles = [&](int mpair0, int ncta0) {
-    auto dead = [&](int n0) { return n0 >= p.N || (EPI == EPI_SOFTMAX && p.causal && n0 > mpair0 + 255); };
-    if (dead(ncta0)) return 0;
-    if (BNS1 == 0 || dead(ncta0 + BNS0)) return 1;
-    return 2;
-  };
+  // A sub-tile is not computed when it lies past N, or when the causal mask removes it for BOTH row blocks of the
+  // pair.  Every role evaluates the same predicate.
+  auto unit_live = [&](int mpair0, int n0) { return n0 < p.N && !(EPI == EPI_SOFTMAX && p.causal && n0 > mpair0 + 255); };
 
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      RingPos<NSTAGES> ring;
       bool ok = true;
       for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
-        const int nlive = live_subtiles(mpair0, ncta0);
-        if (nlive == 0) continue;
         const int m0 = mpair0 + static_cast<int>(pm) * 128;
-        const uint32_t bytes = Cfg::A_BYTES + Cfg::B0_BYTES + (nlive > 1 ? Cfg::B1_BYTES : 0);
-        for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait<false>(bar_empty(stage), phase ^ 1u, w)) { ok = false; break; }
-          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
-          const uint32_t sb0 = sa + Cfg::A_BYTES;
-          const uint32_t sb1 = sb0 + Cfg::B0_BYTES;
-          const uint32_t full = map_to_cta(bar_full(stage), leader);
-          mbar_arrive_expect_tx_cluster(full, bytes);
-          tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
 #pragma unroll
-          for (int j = 0; j < BNS0 / 128; ++j)
-            tma_load_3d_pair(sb0 + j * 8192, &tmB, full, ncta0 + static_cast<int>(pm) * (BNS0 / 2) + j * 64, kb * 64, b);
-          if (nlive > 1) {
-#pragma unroll
-            for (int j = 0; j < BNS1 / 128; ++j)
-              tma_load_3d_pair(sb1 + j * 8192, &tmB, full, ncta0 + BNS0 + static_cast<int>(pm) * (BNS1 / 2) + j * 64, kb * 64, b);
+        for (int sub = 0; sub < NSUB; ++sub) {
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          if (!ok || !unit_live(mpair0, n0)) continue;
+          const uint32_t bytes = Cfg::A_BYTES + (W / 2) * 128;
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; break; }
+            const uint32_t sa = smem_base + ring.stage * Cfg::STAGE_BYTES;
+            const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
+            mbar_arrive_expect_tx_cluster(full, bytes);
+            tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
+            for (int j = 0; j < W / 128; ++j)
+              tma_load_3d_pair(sa + Cfg::A_BYTES + j * 8192, &tmB, full, n0 + static_cast<int>(pm) * (W / 2) + j * 64, kb * 64, b);
+            ring.advance();
           }
-          if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+          if (ok && has_res) {
+            // the sub-tile's residual tile rides the same ring, right behind its last K block
+            const int groups = W / 64;
+            for (int g0 = 0; g0 < groups; g0 += GPS) {
+              if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; break; }
+              const int ng = groups - g0 < GPS ? groups - g0 : GPS;
+              const uint32_t sr = smem_base + ring.stage * Cfg::STAGE_BYTES;
+              mbar_arrive_expect_tx(bar_rfull(ring.stage), ng * Cfg::GROUP_BYTES);
+              for (int g = 0; g < ng; ++g)
+                tma_load_3d(sr + g * Cfg::GROUP_BYTES, &tmR, bar_rfull(ring.stage), n0 + (g0 + g) * 64, m0, b);
+              ring.advance();
+            }
+          }
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------------------------------ UMMA issuer (even CTA)
     if (lane == 0 && pm == 0) {
-      constexpr uint32_t idesc0 = make_idesc_bf16(256, BNS0, false, true);
-      constexpr uint32_t idesc1 = make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true);
-      int stage = 0;
-      uint32_t phase = 0;
-      int acc_it = 0;
+      RingPos<NSTAGES> ring;
+      uint32_t full_bits = 0;     // per-stage phase of bar_full (a stage is not a K-block stage on every lap)
+      uint32_t slot_uses[2] = {0, 0};
+      uint32_t unit_count = 0;
       bool ok = true;
       for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
-        const int nlive = live_subtiles(mpair0, ncta0);
-        if (nlive == 0) continue;
-        const int buf = acc_it % NACC;
-        const uint32_t aphase = static_cast<uint32_t>(acc_it / NACC) & 1u;
-        ++acc_it;
-        if (!mbar_wait<true>(bar_tempty(buf), aphase ^ 1u, w)) { ok = false; break; }
-        tcgen05_fence_after_sync();
-        const uint32_t d0 = tmem_base + buf * BN;
-        const uint32_t d1 = d0 + BNS0;
-        for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait<false>(bar_full(stage), phase, w)) { ok = false; break; }
-          tcgen05_fence_after_sync();
-          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
-          const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
-          const uint64_t bdesc0 = make_smem_desc_sw128(sa + Cfg::A_BYTES, 8192, 1024);
-          const uint64_t bdesc1 = make_smem_desc_sw128(sa + Cfg::A_BYTES + Cfg::B0_BYTES, 8192, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-            umma_bf16_ss_pair(d0, adesc + static_cast<uint64_t>(k * 2), bdesc0 + static_cast<uint64_t>(k * 128), idesc0, acc);
-            if (BNS1 > 0 && nlive > 1)
-              umma_bf16_ss_pair(d1, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc1, acc);
+        for (int sub = 0; sub < NSUB; ++sub) {
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          if (!ok || !unit_live(mpair0, n0)) continue;
+          const int slot = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
+          ++unit_count;
+          if (!mbar_wait<true>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; continue; }
+          ++slot_uses[slot];
+          tcgen05_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + (slot ? BNS0 : 0);
+          const uint32_t idesc = sub ? make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true) : make_idesc_bf16(256, BNS0, false, true);
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!mbar_wait<false>(bar_full(ring.stage), (full_bits >> ring.stage) & 1u, w)) { ok = false; break; }
+            full_bits ^= 1u << ring.stage;
+            tcgen05_fence_after_sync();
+            const uint32_t sa = smem_base + ring.stage * Cfg::STAGE_BYTES;
+            const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
+            const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              // K advances by 16 elements: 32 bytes inside A's swizzled row, 16 K-lines (2048 bytes) in B
+              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
+                                (kb | k) != 0 ? 1u : 0u);
+            }
+            // the stage is free in both CTAs once these UMMAs have read it
+            umma_commit_pair(bar_empty(ring.stage));
+            umma_commit_pair(map_to_cta(bar_empty(ring.stage), peer));
+            ring.advance();
           }
-          // the stage is free in both CTAs once these UMMAs have read it
-          umma_commit_pair(bar_empty(stage));
-          umma_commit_pair(map_to_cta(bar_empty(stage), peer));
-          if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (ok) {
-          umma_commit_pair(bar_tfull(buf));
-          umma_commit_pair(map_to_cta(bar_tfull(buf), peer));
+          if (ok) {
+            umma_commit_pair(bar_tfull(slot));
+            umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
+            if (has_res) ring.skip((W / 64 + GPS - 1) / GPS);  // the residual stages belong to the epilogue
+          }
         }
       }
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
@@ -233,225 +279,315 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int q = warp & 3;
     const int h = (warp - 2) >> 2;
     const int row = q * 32 + lane;
+    const int epi_tid = threadIdx.x - 64;
+    const bool store_thread = epi_tid == 0;
+    const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
     int xpar = 0;
     uint32_t xphase = 0;
-    int acc_it = 0;
     (void)xpar; (void)xphase; (void)s_pre; (void)s_stats; (void)s_bias; (void)s_gamma; (void)s_beta;
+    RingPos<NSTAGES> ring;
+    uint32_t rfull_bits = 0;
+    uint32_t slot_uses[2] = {0, 0};
+    uint32_t unit_count = 0;
+    uint32_t ygroup = 0;  // running count of output boxes: selects the staging buffer
     constexpr float kThreadCount = static_cast<float>(BN / 2);
-    const uint32_t tempty_leader_base = map_to_cta(bar_tempty(0), leader);
+    const uint32_t tempty_leader = map_to_cta(bar_tempty(0), leader);
+    const uint32_t ybuf = smem_base + Cfg::OFF_YBUF;
+
+    // Stage one 128 x 64 box of packed bf16 (this thread: 32 columns of its row) and store it with TMA.
+    auto store_group = [&](const uint32_t (&pk)[16], int col0, int m0, int b) {
+      const uint32_t buf = ybuf + (ygroup & 1u) * Cfg::GROUP_BYTES;
+      ++ygroup;
+      if (store_thread) tma_store_wait_read<1>();  // the box that used this buffer two stores ago has been read out
+      named_barrier_sync(3, 256);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t a = buf + swz128(row, h * 4 + i);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                     "r"(pk[4 * i + 3])
+                     : "memory");
+      }
+      fence_proxy_async_smem();
+      named_barrier_sync(3, 256);
+      if (store_thread) {
+        tma_store_3d(&tmY, buf, col0, m0, b);
+        tma_store_commit();
+      }
+    };
+    // This thread's 32 residual values of group `g` of a residual stage, as 16 packed bf16 pairs.
+    auto load_residual = [&](uint32_t stage_addr, int g, uint32_t (&r32)[16]) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t a = stage_addr + g * Cfg::GROUP_BYTES + swz128(row, h * 4 + i);
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(r32[4 * i]), "=r"(r32[4 * i + 1]), "=r"(r32[4 * i + 2]), "=r"(r32[4 * i + 3])
+                     : "r"(a));
+      }
+    };
 
     for (int tile = cluster_id; tile < p.total_tiles; tile += num_clusters) {
       int b, mpair0, ncta0;
       decode_tile(tile, b, mpair0, ncta0);
-      const int nlive = live_subtiles(mpair0, ncta0);
       const int m0 = mpair0 + static_cast<int>(pm) * 128;
       const int grow = m0 + row;
       const bool valid = grow < p.M;
-      uint16_t* yrow = p.Y + static_cast<long long>(b) * p.batch_stride_y + static_cast<long long>(grow) * p.ldy;
-      const uint16_t* rrow =
-          p.residual ? p.residual + static_cast<long long>(b) * p.batch_stride_r + static_cast<long long>(grow) * p.ldr
-                     : nullptr;
-      const int buf = acc_it % NACC;
-      const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * BN;
-      if (nlive > 0) {
-        mbar_wait<false>(bar_tfull(buf), static_cast<uint32_t>(acc_it / NACC) & 1u, w);
-        ++acc_it;
-        __syncwarp();
-        tcgen05_fence_after_sync();
+
+      // the slot of each sub-tile of this tile, and whether it is computed at all
+      bool live[NSUB];
+      int slot[NSUB];
+#pragma unroll
+      for (int sub = 0; sub < NSUB; ++sub) {
+        live[sub] = unit_live(mpair0, ncta0 + (sub ? BNS0 : 0));
+        slot[sub] = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
+        if (live[sub]) ++unit_count;
       }
-      auto release_accumulator = [&]() {
-        if (nlive > 0) {
-          tcgen05_fence_before_sync();
-          mbar_arrive_cluster(tempty_leader_base + 8u * buf);
+      auto wait_accumulator = [&](int sub) {
+        if (live[sub]) {
+          mbar_wait<false>(bar_tfull(slot[sub]), slot_uses[slot[sub]] & 1u, w);
+          ++slot_uses[slot[sub]];
+          __syncwarp();
+          tcgen05_fence_after_sync();
+          ring.skip(KB);  // the K-block stages of this sub-tile were the UMMA's
         }
       };
+      auto release_accumulator = [&](int sub) {
+        if (live[sub]) {
+          tcgen05_fence_before_sync();
+          mbar_arrive_cluster(tempty_leader + 8u * slot[sub]);
+        }
+      };
+      auto tmem_of = [&](int sub) { return tmem_base + lane_sel + (slot[sub] ? BNS0 : 0); };
 
       if constexpr (EPI == EPI_NONE) {
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          const int col = ncta0 + lc;
-          if (col >= p.N) continue;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          uint32_t pk[16];
+        for (int sub = 0; sub < NSUB; ++sub) {
+          if (!live[sub]) continue;
+          wait_accumulator(sub);
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          for (int g = 0; g < W / 64; ++g) {
+            if (n0 + g * 64 >= p.N) break;
+            uint32_t v[32];
+            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
+            uint32_t pk[16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-          if (valid) {
-            if (col + 32 <= p.N) {
-              store_chunk_bf16(yrow + col, pk);
-            } else {
-#pragma unroll
-              for (int g = 0; g < 4; ++g)
-                if (col + 8 * g + 8 <= p.N)
-                  *reinterpret_cast<uint4*>(yrow + col + 8 * g) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
-            }
+            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            store_group(pk, n0 + g * 64, m0, b);
           }
+          release_accumulator(sub);
         }
-        release_accumulator();
-      } else if constexpr (EPI == EPI_LN) {
-        // ---------------- stage 1: x = alpha*Acc + bias + R ; thread-local (mean, M2); x written back (bypass path)
+      } else if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
+        // ---------------- stage 1 (compute): x = f(alpha*Acc + bias, R); thread-local partial statistic; x is written
+        // back over the accumulator in TMEM (the bypass path of Sec. 3.2)
         float2 part = make_float2(0.f, 0.f);
         float n_run = 0.f;
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          uint4 rr[4];
+        for (int sub = 0; sub < NSUB; ++sub) {
+          wait_accumulator(sub);
+          const int W = sub ? BNS1 : BNS0;
+          const int lsub = sub ? BNS0 : 0;  // first column of the sub-tile inside the CTA's column range
+          const uint32_t taddr = tmem_of(sub);
+          for (int g0 = 0; g0 < W / 64; g0 += GPS) {
+            uint32_t stage_addr = 0;
+            if (has_res) {
+              mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
+              rfull_bits ^= 1u << ring.stage;
+              __syncwarp();
+              stage_addr = smem_base + ring.stage * Cfg::STAGE_BYTES;
+            }
 #pragma unroll
-          for (int g = 0; g < 4; ++g)
-            rr[g] = (valid && rrow) ? __ldg(reinterpret_cast<const uint4*>(rrow + ncta0 + lc) + g) : make_uint4(0, 0, 0, 0);
-          const uint32_t* r32 = reinterpret_cast<const uint32_t*>(rr);
-          float sum = 0.f;
+            for (int gg = 0; gg < GPS; ++gg) {
+              const int g = g0 + gg;
+              if (g >= W / 64) break;
+              const int lc = lsub + g * 64 + h * 32;
+              uint32_t v[32];
+              tmem_ld_32cols(taddr + g * 64 + h * 32, v);
+              uint32_t r32[16];
+              if (has_res) {
+                load_residual(stage_addr, gg, r32);
+              } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float x0 = fmaf(p.alpha, __uint_as_float(v[2 * j]), s_bias[lc + 2 * j]) + bf16_lo(r32[j]);
-            const float x1 = fmaf(p.alpha, __uint_as_float(v[2 * j + 1]), s_bias[lc + 2 * j + 1]) + bf16_hi(r32[j]);
-            v[2 * j] = __float_as_uint(x0);
-            v[2 * j + 1] = __float_as_uint(x1);
-            sum += x0 + x1;
+                for (int j = 0; j < 16; ++j) r32[j] = 0u;
+              }
+              const float4* bias4 = reinterpret_cast<const float4*>(s_bias + lc);
+              if constexpr (EPI == EPI_LN) {
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 bb = bias4[j];
+                  const float x0 = fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x) + bf16_lo(r32[2 * j]);
+                  const float x1 = fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y) + bf16_hi(r32[2 * j]);
+                  const float x2 = fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z) + bf16_lo(r32[2 * j + 1]);
+                  const float x3 = fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w) + bf16_hi(r32[2 * j + 1]);
+                  v[4 * j] = __float_as_uint(x0); v[4 * j + 1] = __float_as_uint(x1);
+                  v[4 * j + 2] = __float_as_uint(x2); v[4 * j + 3] = __float_as_uint(x3);
+                  s0 += x0; s1 += x1; s2 += x2; s3 += x3;
+                }
+                const float cmean = ((s0 + s1) + (s2 + s3)) * (1.f / 32.f);
+                float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float d0 = __uint_as_float(v[4 * j]) - cmean, d1 = __uint_as_float(v[4 * j + 1]) - cmean;
+                  const float d2 = __uint_as_float(v[4 * j + 2]) - cmean, d3 = __uint_as_float(v[4 * j + 3]) - cmean;
+                  q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1); q2 = fmaf(d2, d2, q2); q3 = fmaf(d3, d3, q3);
+                }
+                const float2 cpart = make_float2(cmean, (q0 + q1) + (q2 + q3));
+                part = (n_run == 0.f) ? cpart : MergeWelford()(part, n_run, cpart, 32.f);
+                n_run += 32.f;
+              } else {
+                float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 bb = bias4[j];
+                  const float h0 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x)) + bf16_lo(r32[2 * j]);
+                  const float h1 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y)) + bf16_hi(r32[2 * j]);
+                  const float h2 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z)) + bf16_lo(r32[2 * j + 1]);
+                  const float h3 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w)) + bf16_hi(r32[2 * j + 1]);
+                  v[4 * j] = __float_as_uint(h0); v[4 * j + 1] = __float_as_uint(h1);
+                  v[4 * j + 2] = __float_as_uint(h2); v[4 * j + 3] = __float_as_uint(h3);
+                  q0 = fmaf(h0, h0, q0); q1 = fmaf(h1, h1, q1); q2 = fmaf(h2, h2, q2); q3 = fmaf(h3, h3, q3);
+                }
+                part.x += (q0 + q1) + (q2 + q3);
+              }
+              tmem_st_32cols(taddr + g * 64 + h * 32, v);
+            }
+            if (has_res) {
+              // all 256 threads are done with this residual stage: hand it back to the producer
+              __syncwarp();
+              named_barrier_sync(2, 256);
+              if (store_thread) mbar_arrive(bar_empty(ring.stage));
+              ring.advance();
+            }
           }
-          const float cmean = sum * (1.f / 32.f);
-          float cm2 = 0.f;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float d = __uint_as_float(v[j]) - cmean;
-            cm2 = fmaf(d, d, cm2);
-          }
-          part = (n_run == 0.f) ? make_float2(cmean, cm2) : MergeWelford()(part, n_run, make_float2(cmean, cm2), 32.f);
-          n_run += 32.f;
-          tmem_st_32cols(lane_base + lc, v);
         }
         tmem_st_wait();
-        const float2 tot = cluster_row_reduce<CN>(part, kThreadCount, MergeWelford(), s_pre, s_stats, bar_stats, row, h, crank,
-                                                  xpar, xphase, w, 2u, pm);
-        const float mu = tot.x;
-        const float rstd = rsqrtf(tot.y * (1.f / static_cast<float>(CN * BN)) + p.eps);
-        // ---------------- stage 2: normalise the resident x, round once, store
-#pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float y0 = fmaf((__uint_as_float(v[2 * j]) - mu) * rstd, s_gamma[lc + 2 * j], s_beta[lc + 2 * j]);
-            const float y1 = fmaf((__uint_as_float(v[2 * j + 1]) - mu) * rstd, s_gamma[lc + 2 * j + 1], s_beta[lc + 2 * j + 1]);
-            pk[j] = pack_bf16x2_rn(y0, y1);
-          }
-          if (valid) store_chunk_bf16(yrow + ncta0 + lc, pk);
+        // ---------------- stage 1 (reduce): thread pair, then the CTAs that share these rows
+        float2 tot;
+        if constexpr (EPI == EPI_LN) {
+          tot = cluster_row_reduce<CN>(part, kThreadCount, MergeWelford(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w,
+                                       2u, pm);
+        } else {
+          tot = cluster_row_reduce<CN>(part, kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u,
+                                       pm);
         }
-        release_accumulator();
-      } else if constexpr (EPI == EPI_RMS_MAX) {
-        // ---------------- stage 1: H = GELU(alpha*Acc + bias) + R ; thread-local sum of squares; H written back
-        float ss = 0.f;
-#pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          uint4 rr[4];
-#pragma unroll
-          for (int g = 0; g < 4; ++g)
-            rr[g] = (valid && rrow) ? __ldg(reinterpret_cast<const uint4*>(rrow + ncta0 + lc) + g) : make_uint4(0, 0, 0, 0);
-          const uint32_t* r32 = reinterpret_cast<const uint32_t*>(rr);
-          float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float z0 = fmaf(p.alpha, __uint_as_float(v[2 * j]), s_bias[lc + 2 * j]);
-            const float z1 = fmaf(p.alpha, __uint_as_float(v[2 * j + 1]), s_bias[lc + 2 * j + 1]);
-            const float h0 = gelu_tanh_f32(z0) + bf16_lo(r32[j]);
-            const float h1 = gelu_tanh_f32(z1) + bf16_hi(r32[j]);
-            v[2 * j] = __float_as_uint(h0);
-            v[2 * j + 1] = __float_as_uint(h1);
-            s0 = fmaf(h0, h0, s0);
-            s1 = fmaf(h1, h1, s1);
-          }
-          ss += s0 + s1;
-          tmem_st_32cols(lane_base + lc, v);
-        }
-        tmem_st_wait();
-        const float2 tot = cluster_row_reduce<CN>(make_float2(ss, 0.f), kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row,
-                                                  h, crank, xpar, xphase, w, 2u, pm);
-        const float rstd = rsqrtf(tot.x * (1.f / static_cast<float>(CN * BN)) + p.eps);
-        // ---------------- stage 2: Y = H * rstd * g ; thread-local (max, argmax) of the unrounded Y
+        const float mu = EPI == EPI_LN ? tot.x : 0.f;
+        const float sq = EPI == EPI_LN ? tot.y : tot.x;
+        const float rstd = rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
+        // ---------------- stage 2 (PostOp): normalise the resident x, round once, store
         float best = -INFINITY;
         int best_col = 0x7FFFFFFF;
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          uint32_t pk[16];
+        for (int sub = 0; sub < NSUB; ++sub) {
+          const int W = sub ? BNS1 : BNS0;
+          const int lsub = sub ? BNS0 : 0;
+          const uint32_t taddr = tmem_of(sub);
+          for (int g = 0; g < W / 64; ++g) {
+            const int lc = lsub + g * 64 + h * 32;
+            uint32_t v[32];
+            tmem_ld_32cols(taddr + g * 64 + h * 32, v);
+            const float4* g4 = reinterpret_cast<const float4*>(s_gamma + lc);
+            const float4* b4 = reinterpret_cast<const float4*>(s_beta + lc);
+            uint32_t pk[16];
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float y0 = __uint_as_float(v[2 * j]) * rstd * s_gamma[lc + 2 * j];
-            const float y1 = __uint_as_float(v[2 * j + 1]) * rstd * s_gamma[lc + 2 * j + 1];
-            if (y0 > best) { best = y0; best_col = ncta0 + lc + 2 * j; }
-            if (y1 > best) { best = y1; best_col = ncta0 + lc + 2 * j + 1; }
-            pk[j] = pack_bf16x2_rn(y0, y1);
+            for (int j = 0; j < 8; ++j) {
+              const float4 gg = g4[j];
+              float y0, y1, y2, y3;
+              if constexpr (EPI == EPI_LN) {
+                const float4 be = b4[j];
+                y0 = fmaf((__uint_as_float(v[4 * j]) - mu) * rstd, gg.x, be.x);
+                y1 = fmaf((__uint_as_float(v[4 * j + 1]) - mu) * rstd, gg.y, be.y);
+                y2 = fmaf((__uint_as_float(v[4 * j + 2]) - mu) * rstd, gg.z, be.z);
+                y3 = fmaf((__uint_as_float(v[4 * j + 3]) - mu) * rstd, gg.w, be.w);
+              } else {
+                y0 = __uint_as_float(v[4 * j]) * rstd * gg.x;
+                y1 = __uint_as_float(v[4 * j + 1]) * rstd * gg.y;
+                y2 = __uint_as_float(v[4 * j + 2]) * rstd * gg.z;
+                y3 = __uint_as_float(v[4 * j + 3]) * rstd * gg.w;
+                const int c = ncta0 + lc + 4 * j;
+                if (y0 > best) { best = y0; best_col = c; }
+                if (y1 > best) { best = y1; best_col = c + 1; }
+                if (y2 > best) { best = y2; best_col = c + 2; }
+                if (y3 > best) { best = y3; best_col = c + 3; }
+              }
+              pk[2 * j] = pack_bf16x2_rn(y0, y1);
+              pk[2 * j + 1] = pack_bf16x2_rn(y2, y3);
+            }
+            store_group(pk, ncta0 + lsub + g * 64, m0, b);
           }
-          if (valid) store_chunk_bf16(yrow + ncta0 + lc, pk);
+          release_accumulator(sub);
         }
-        release_accumulator();
-        // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
-        const float2 mx = cluster_row_reduce<CN>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
-                                                 s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
-        if (crank == 0 && h == 0 && valid) {
-          const long long o = static_cast<long long>(b) * p.M + grow;
-          p.row_max[o] = mx.x;
-          p.row_argmax[o] = __float_as_int(mx.y);
+        if constexpr (EPI == EPI_RMS_MAX) {
+          // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
+          const float2 mx = cluster_row_reduce<CN>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
+                                                   s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
+          if (crank == 0 && h == 0 && valid) {
+            const long long o = static_cast<long long>(b) * p.M + grow;
+            p.row_max[o] = mx.x;
+            p.row_argmax[o] = __float_as_int(mx.y);
+          }
         }
       } else {  // EPI_SOFTMAX
         // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
         const float sc = p.alpha * 1.4426950408889634f;
-        // chunk classification under the causal mask, uniform over the warp's 32 rows so that the warp-wide TMEM
+        // fragment classification under the causal mask, uniform over the warp's 32 rows so that the warp-wide TMEM
         // loads stay convergent: 2 = all live, 1 = crosses the diagonal, 0 = all masked
         const int wrow0 = m0 + q * 32;
-        auto chunk_state = [&](int col0) { return !p.causal ? 2 : (col0 + 31 <= wrow0 ? 2 : (col0 > wrow0 + 31 ? 0 : 1)); };
+        auto frag_state = [&](int col0) { return !p.causal ? 2 : (col0 + 31 <= wrow0 ? 2 : (col0 > wrow0 + 31 ? 0 : 1)); };
         // ---------------- pass A: thread-local row max
         float mloc = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          const int st = chunk_state(ncta0 + lc);
-          if (st == 0) continue;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
+        for (int sub = 0; sub < NSUB; ++sub) {
+          wait_accumulator(sub);
+          if (!live[sub]) continue;
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          for (int g = 0; g < W / 64; ++g) {
+            const int col0 = n0 + g * 64 + h * 32;
+            const int st = frag_state(col0);
+            if (st == 0) continue;
+            uint32_t v[32];
+            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
+            float m0v = -INFINITY, m1v = -INFINITY;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float t = __uint_as_float(v[j]) * sc;
-            if (st == 2 || ncta0 + lc + j <= grow) mloc = fmaxf(mloc, t);
+            for (int j = 0; j < 32; j += 2) {
+              const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
+              if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
+              if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+            }
+            mloc = fmaxf(mloc, fmaxf(m0v, m1v));
           }
         }
         // ---------------- pass B: e = 2^(t - mloc), thread-local sum, e written back over the scores
         float lloc = 0.f;
         const float msub = (mloc == -INFINITY) ? 0.f : mloc;
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          const int st = chunk_state(ncta0 + lc);
-          if (st == 0) continue;
-          uint32_t v[32];
-          tmem_ld_32cols(lane_base + lc, v);
-          float s0 = 0.f, s1 = 0.f;
+        for (int sub = 0; sub < NSUB; ++sub) {
+          if (!live[sub]) continue;
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          for (int g = 0; g < W / 64; ++g) {
+            const int col0 = n0 + g * 64 + h * 32;
+            const int st = frag_state(col0);
+            if (st == 0) continue;
+            uint32_t v[32];
+            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
+            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float e0 = ex2_approx(fmaf(__uint_as_float(v[j]), sc, -msub));
-            float e1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), sc, -msub));
-            if (st != 2) {
-              if (ncta0 + lc + j > grow) e0 = 0.f;
-              if (ncta0 + lc + j + 1 > grow) e1 = 0.f;
+            for (int j = 0; j < 32; j += 2) {
+              float e0 = ex2_approx(fmaf(__uint_as_float(v[j]), sc, -msub));
+              float e1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), sc, -msub));
+              if (st != 2) {
+                if (col0 + j > grow) e0 = 0.f;
+                if (col0 + j + 1 > grow) e1 = 0.f;
+              }
+              v[j] = __float_as_uint(e0);
+              v[j + 1] = __float_as_uint(e1);
+              s0 += e0;
+              s1 += e1;
             }
-            v[j] = __float_as_uint(e0);
-            v[j + 1] = __float_as_uint(e1);
-            s0 += e0;
-            s1 += e1;
+            lloc += s0 + s1;
+            tmem_st_32cols(tmem_of(sub) + g * 64 + h * 32, v);
           }
-          lloc += s0 + s1;
-          tmem_st_32cols(lane_base + lc, v);
         }
         tmem_st_wait();
         const float2 tot = cluster_row_reduce<CN>(make_float2(mloc, lloc), kThreadCount, MergeMaxSumExp2(), s_pre, s_stats,
@@ -459,24 +595,29 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const float f = (mloc == -INFINITY || tot.y == 0.f) ? 0.f : ex2_approx(mloc - tot.x) / tot.y;
         // ---------------- pass C: scale, round once, store (zeros where masked)
 #pragma unroll
-        for (int c = 0; c < CHUNK_PAIRS; ++c) {
-          const int lc = (2 * c + h) * 32;
-          const int st = chunk_state(ncta0 + lc);
-          uint32_t pk[16];
-          if (st == 0) {
+        for (int sub = 0; sub < NSUB; ++sub) {
+          const int W = sub ? BNS1 : BNS0;
+          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          for (int g = 0; g < W / 64; ++g) {
+            const int col0 = n0 + g * 64 + h * 32;
+            const int st = live[sub] ? frag_state(col0) : 0;
+            uint32_t pk[16];
+            if (st == 0) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) pk[j] = 0u;
-          } else {
-            uint32_t v[32];
-            tmem_ld_32cols(lane_base + lc, v);
+              for (int j = 0; j < 16; ++j) pk[j] = 0u;
+            } else {
+              uint32_t v[32];
+              tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
+              for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
+            }
+            store_group(pk, n0 + g * 64, m0, b);
           }
-          if (valid) store_chunk_bf16(yrow + ncta0 + lc, pk);
+          release_accumulator(sub);
         }
-        release_accumulator();
       }
     }
+    if (store_thread) tma_store_wait_all();  // the staging buffers must outlive the last store's read
   }
 
   // -------------------------------------------------------------------------------------------- teardown

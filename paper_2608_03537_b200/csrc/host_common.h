@@ -27,16 +27,19 @@ void count_launch();
 bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
                          uint64_t stride2_bytes, uint32_t box_rows);
 
+// Tensor maps of one GEMM -> subgraph call: operands A [batch, M, K] and B [batch, K, N], residual R and output Y
+// [batch, M, N]; all bf16, 128-byte swizzle, boxes of 64 elements by 128 rows (A, R, Y) or 64 rows (B).
+struct GemmMaps {
+  CUtensorMap A, B, R, Y;
+};
+
 // Launchers implemented one per translation unit.  Each returns cudaSuccess or the launch error, and
 // cudaErrorInvalidValue if no instantiation covers (N, kind).  `supported_only` asks whether an instantiation
 // exists without launching.
-cudaError_t launch_fused_layernorm(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
-                                   bool supported_only);
-cudaError_t launch_fused_rmsnorm_max(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
-                                     bool supported_only);
-cudaError_t launch_fused_softmax(const CUtensorMap& tmA, const CUtensorMap& tmB, const FusedParams& p, cudaStream_t st,
-                                 bool supported_only);
-// Plain GEMM, Z = bf16(A.B), any N that is a multiple of 8.  Fills p.nblocks / p.total_tiles itself.
-cudaError_t launch_plain_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, FusedParams p, cudaStream_t st);
+cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+// Plain GEMM, Z = bf16(A.B) through maps.Y, any N that is a multiple of 8.
+cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 
 }  // namespace comfuse
