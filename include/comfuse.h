@@ -96,6 +96,31 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
                                        const comfuse_epilogue_args_t* args, void* workspace,
                                        size_t workspace_bytes, void* cuda_stream);
 
+/* GEMM -> subgraph through the UNFUSED path without a caller workspace.  (The paper has no counterpart of this
+ * entry point: it exists for callers of this library, not for the method.)
+ *
+ * Some callers cannot provide the workspace that comfuse_gemm_epilogue(fused = 0) needs, because they cannot
+ * allocate device memory where the call happens: code that runs while a stream is being captured or in a latency
+ * critical loop where cudaMalloc (which synchronises the device) is not allowed, plug-ins that receive tensors from
+ * a host framework but have no access to its allocator, or processes whose device memory is handed out entirely by
+ * another component.  For them the intermediate bf16 GEMM result is kept in a fixed array of
+ * COMFUSE_STATIC_SCRATCH_BYTES that is part of the library's device image; every GPU on which the library is loaded
+ * holds that array until the process exits.
+ *
+ * Semantics are those of comfuse_gemm_epilogue with desc->fused forced to 0; desc->fused is ignored.
+ *   - The call allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.
+ *   - batch * M * N * 2 bytes must fit in COMFUSE_STATIC_SCRATCH_BYTES; a larger problem is rejected with
+ *     COMFUSE_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address and configures the kernels it launches;
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  Nothing in it
+ *     needs clearing (each call overwrites the region it later reads), but two calls whose kernels can overlap on
+ *     the GPU -- different streams without an ordering between them -- race on it.  Order such calls on one stream
+ *     or with events. */
+#define COMFUSE_STATIC_SCRATCH_BYTES (16u << 20)
+comfuse_status_t comfuse_gemm_epilogue_static_scratch(const comfuse_gemm_desc_t* desc, const void* A, const void* B,
+                                                      void* Y, const comfuse_epilogue_args_t* args, void* cuda_stream);
+
 /* Back-to-back GEMM (Sec. 4, Eq. 2) with F = GELU_tanh(. + b1) and the tail
  *   O = LayerNorm(S.W2 + b2 + X) * gamma + beta,   S = F(X.W1),
  * X [M, K], W1 [K, N1], W2 [N1, N2], all dense row-major bf16, N2 == K.  In the fused path S (and P) never

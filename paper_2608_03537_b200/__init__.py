@@ -7,6 +7,7 @@ import of :func:`lib` fails loudly.
 
 Functions mirror the C entry points:
     gemm_epilogue(...)      -> comfuse_gemm_epilogue      (GEMM -> elementwise/reduction subgraph, Sec. 3)
+    gemm_epilogue_static_scratch(...) -> comfuse_gemm_epilogue_static_scratch (unfused path, no caller workspace)
     b2b_gemm(...)           -> comfuse_b2b_gemm           (GEMM -> F -> GEMM -> post-norm tail, Sec. 4)
     workspace_size(...)     -> comfuse_workspace_size
     b2b_workspace_size(...) -> comfuse_b2b_workspace_size
@@ -30,6 +31,7 @@ MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
     "comfuse_gemm_epilogue",
+    "comfuse_gemm_epilogue_static_scratch",
     "comfuse_b2b_workspace_size",
     "comfuse_b2b_gemm",
     "comfuse_last_device_status",
@@ -84,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.comfuse_gemm_epilogue.argtypes = [POINTER(GemmDesc), c_void_p, c_void_p, c_void_p, POINTER(EpilogueArgs),
                                             c_void_p, c_size_t, c_void_p]
         L.comfuse_gemm_epilogue.restype = c_int32
+        L.comfuse_gemm_epilogue_static_scratch.argtypes = [POINTER(GemmDesc), c_void_p, c_void_p, c_void_p, POINTER(EpilogueArgs), c_void_p]
+        L.comfuse_gemm_epilogue_static_scratch.restype = c_int32
         L.comfuse_b2b_workspace_size.argtypes = [POINTER(B2bDesc), POINTER(c_size_t)]
         L.comfuse_b2b_workspace_size.restype = c_int32
         L.comfuse_b2b_gemm.argtypes = [POINTER(B2bDesc)] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
@@ -146,6 +150,23 @@ def gemm_epilogue(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=N
     st = lib().comfuse_gemm_epilogue(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), ws_ptr, ws_bytes, _stream(stream))
     if st != OK:
         raise ComfuseError(st, "comfuse_gemm_epilogue")
+    return Y
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def gemm_epilogue_static_scratch(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=None, mask_tensor=None,
+                                 row_max=None, row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, stream=None):
+    """The unfused GEMM -> row-kernel path for callers that cannot allocate a workspace (for instance inside a stream
+    capture, or a plug-in without access to the host framework's allocator): the intermediate lives in a fixed
+    STATIC_SCRATCH_BYTES array inside the library.  batch*M*N*2 bytes must fit; calls that may overlap on the GPU race
+    on that array; make the first call on a device outside stream capture."""
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=False)
+    args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
+    st = lib().comfuse_gemm_epilogue_static_scratch(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_epilogue_static_scratch")
     return Y
 
 
