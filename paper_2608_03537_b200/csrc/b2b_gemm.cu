@@ -1,5 +1,495 @@
+// Fused back-to-back GEMM (Sec. 4):  P = X W1,  S = GELU_tanh(P + b1),  O' = S W2 + b2 + X,  O = LayerNorm(O').
+// Neither P nor S is written to global memory.
+//
+// Dataflow (Sec. 4.1, adapted): N1 is cut into 128-column chunks.  Instead of spreading the chunks over the CTAs of
+// a cluster and summing partial O tiles at the commit, one CTA pair walks all chunks of its 256 rows and accumulates
+// O in tensor memory, which keeps the sum deterministic and needs no cross-CTA reduction.
+//
+// Consumer schedule (Sec. 4.3, ML1 -> Epi1 -> ML2 -> Epi2 staggered by one stage): the UMMA lane issues
+//   ML1(0) ML1(1) | ML2(0) ML1(2) | ML2(1) ML1(3) | ML2(2) | ML2(3)
+// so that Epi1(j) (bias + GELU + bf16 rounding into a swizzled shared-memory A operand) overlaps ML1(j+1) and
+// ML2(j-1); P has two TMEM slots, S two shared-memory buffers, O two TMEM slots (Epi2 of tile t overlaps tile t+1).
+//
+// Producer (Sec. 4.2, unified circular buffer): X, the W1 chunks, the W2 chunks and the residual copy of X all flow
+// through ONE ring of 16 KB slots (a 128-row x 64-element bf16 box each), in the order the consumers need them.
+//
+// CTA pairs (cta_group::2): each CTA holds its own 128 rows of X / S and half (64 columns) of every weight chunk.
+#include <cuda_runtime.h>
+
 #include "b2b_params.h"
+#include "epilogue_common.cuh"
+#include "fused_pair.cuh"
+#include "host_common.h"
+#include "sm100_primitives.cuh"
+
 namespace comfuse {
-bool b2b_fused_supported(int, int, int) { return false; }
-cudaError_t launch_b2b_fused(const void*, const void*, const void*, B2bParams, cudaStream_t) { return cudaErrorInvalidValue; }
+
+namespace {
+
+constexpr int kB2bThreads = 320;
+constexpr int kSlotBytes = 128 * 64 * 2;  // one 128 x 64 bf16 box
+constexpr int kRingSlots = 8;
+constexpr int kMaxChunks = 4;             // N1 <= 512
+
+struct B2bSmem {
+  static constexpr int OFF_RING = 0;
+  static constexpr int OFF_S = kRingSlots * kSlotBytes;            // 2 buffers x 2 K blocks
+  static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // one output staging box
+  static constexpr int OFF_B1 = OFF_YBUF + kSlotBytes;             // fp32 [512]
+  static constexpr int OFF_VEC = OFF_B1 + kMaxChunks * 128 * 4;    // b2, gamma, beta fp32 [128] each
+  static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][2][128]
+  static constexpr int OFF_STATS = OFF_PRE + 2 * 2 * 128 * 8;      // float2 [2][1][128]
+  static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
+  // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats drain
+  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 2;
+  static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
+  static constexpr int BYTES = OFF_MISC + 16 + 1024;
+};
+static_assert(B2bSmem::BYTES <= 232448, "shared memory budget");
+
+// Ring items of one tile, in producer order (every role walks this sequence):
+//   X0 X1 | W1(0) W1(1) | { W2(j) W1(j+2) } for each chunk j | R0 R1      = 2 + 2*NC + 2 slots
+
+__global__ void __launch_bounds__(kB2bThreads, 1)
+b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
+                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  const uint32_t smem_base = smem_u32(smem);
+
+  float* s_b1 = reinterpret_cast<float*>(smem + B2bSmem::OFF_B1);
+  float* s_b2 = reinterpret_cast<float*>(smem + B2bSmem::OFF_VEC);
+  float* s_gamma = s_b2 + 128;
+  float* s_beta = s_gamma + 128;
+  float2* s_pre = reinterpret_cast<float2*>(smem + B2bSmem::OFF_PRE);
+  float2* s_stats = reinterpret_cast<float2*>(smem + B2bSmem::OFF_STATS);
+  const uint32_t bar_base = smem_base + B2bSmem::OFF_BAR;
+  auto bar_full = [&](int s) { return bar_base + 8u * s; };                        // weight / X slot landed (even CTA)
+  auto bar_empty = [&](int s) { return bar_base + 8u * (kRingSlots + s); };        // slot may be overwritten
+  auto bar_rfull = [&](int s) { return bar_base + 8u * (2 * kRingSlots + s); };    // residual slot landed (own CTA)
+  auto bar_pfull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + a); };    // P slot complete
+  auto bar_sfull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 2 + a); };   // S buffer written by both CTAs (even CTA)
+  auto bar_sempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 4 + a); };  // S buffer read by ML2
+  auto bar_ofull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 6 + a); };   // O slot complete
+  auto bar_oempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 8 + a); };  // O slot drained by both CTAs (even CTA)
+  const uint32_t bar_stats = bar_base + 8u * (3 * kRingSlots + 10);
+  const uint32_t bar_drain = bar_stats + 8u;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + B2bSmem::OFF_MISC);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + B2bSmem::OFF_MISC + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // cluster of exactly two CTAs
+  const uint32_t pm = rank & 1u;
+  const uint32_t leader = 0u, peer = rank ^ 1u;
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
+  const int NC = p.N1 / 128;
+  const WaitCtx w{s_abort, p.status, p.timeout_ns};
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRingSlots; ++s) {
+      mbar_init(bar_full(s), 2);
+      mbar_init(bar_empty(s), 1);
+      mbar_init(bar_rfull(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_pfull(a), 1);
+      mbar_init(bar_sfull(a), 2 * 256);
+      mbar_init(bar_sempty(a), 1);
+      mbar_init(bar_ofull(a), 1);
+      mbar_init(bar_oempty(a), 2 * 256);
+    }
+    mbar_init(bar_stats, 128);
+    mbar_init(bar_drain, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&tmX);
+    prefetch_tensormap(&tmW1);
+    prefetch_tensormap(&tmW2);
+    prefetch_tensormap(&tmO);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(s_tmem_base), 512);
+    tmem_relinquish_alloc_permit_pair();
+  }
+  for (int i = threadIdx.x; i < p.N1; i += kB2bThreads) s_b1[i] = p.b1 ? bf16_lo(p.b1[i]) : 0.f;
+  for (int i = threadIdx.x; i < 128; i += kB2bThreads) {
+    s_b2[i] = p.b2 ? bf16_lo(p.b2[i]) : 0.f;
+    s_gamma[i] = p.gamma ? bf16_lo(p.gamma[i]) : 1.f;
+    s_beta[i] = p.beta ? bf16_lo(p.beta[i]) : 0.f;
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  cluster_sync_all();
+  const uint32_t tmem_base = *s_tmem_base;
+  // TMEM columns: P slots at 0 and 128, O slots at 256 and 384
+  auto ring_addr = [&](int s) { return smem_base + B2bSmem::OFF_RING + s * kSlotBytes; };
+  auto s_addr = [&](int buf, int kb) { return smem_base + B2bSmem::OFF_S + (buf * 2 + kb) * kSlotBytes; };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      RingPos<kRingSlots> ring;
+      bool ok = true;
+      // one box into the current slot; kind 0: pair operand (signals the even CTA's full barrier), 1: residual
+      auto push = [&](const CUtensorMap* tm, int x, int y, int kind) {
+        if (!ok) return;
+        if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; return; }
+        if (kind == 0) {
+          const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
+          mbar_arrive_expect_tx_cluster(full, kSlotBytes);
+          tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, 0);
+        } else {
+          mbar_arrive_expect_tx(bar_rfull(ring.stage), kSlotBytes);
+          tma_load_3d(ring_addr(ring.stage), tm, bar_rfull(ring.stage), x, y, 0);
+        }
+        ring.advance();
+      };
+      const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
+      for (int tile = cluster_id; tile < p.mpairs && ok; tile += num_clusters) {
+        const int m0 = tile * 256 + static_cast<int>(pm) * 128;
+        push(&tmX, 0, m0, 0);
+        push(&tmX, 64, m0, 0);
+        push(&tmW1, 0 * 128 + wcol, 0, 0);
+        if (NC > 1) push(&tmW1, 1 * 128 + wcol, 0, 0);
+        for (int j = 0; j < NC; ++j) {
+          push(&tmW2, wcol, j * 128, 0);
+          if (j + 2 < NC) push(&tmW1, (j + 2) * 128 + wcol, 0, 0);
+        }
+        push(&tmX, 0, m0, 1);
+        push(&tmX, 64, m0, 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------------------------ UMMA issuer (even CTA)
+    if (lane == 0 && pm == 0) {
+      constexpr uint32_t idesc_ml1 = make_idesc_bf16(256, 128, false, true);
+      constexpr uint32_t idesc_ml2 = make_idesc_bf16(256, 128, false, true);
+      RingPos<kRingSlots> ring;
+      uint32_t full_bits = 0;
+      uint32_t sfull_uses[2] = {0, 0};
+      uint32_t tile_it = 0;
+      bool ok = true;
+      auto wait_slot = [&]() {  // the next ring item is a pair operand: wait until both halves have landed
+        if (!ok) return 0u;
+        if (!mbar_wait<false>(bar_full(ring.stage), (full_bits >> ring.stage) & 1u, w)) { ok = false; return 0u; }
+        full_bits ^= 1u << ring.stage;
+        tcgen05_fence_after_sync();
+        return ring_addr(ring.stage);
+      };
+      auto release_slot = [&](int stage) {
+        umma_commit_pair(bar_empty(stage));
+        umma_commit_pair(map_to_cta(bar_empty(stage), peer));
+      };
+      for (int tile = cluster_id; tile < p.mpairs && ok; tile += num_clusters, ++tile_it) {
+        const int obuf = tile_it & 1u;
+        const uint32_t d_o = tmem_base + 256 + obuf * 128;
+        // X: two K blocks
+        const int xs0 = ring.stage;
+        const uint32_t x0 = wait_slot();
+        ring.advance();
+        const int xs1 = ring.stage;
+        const uint32_t x1 = wait_slot();
+        ring.advance();
+        const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
+        const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
+        auto issue_ml1 = [&](int j) {
+          // P[j & 1] = X . W1[:, chunk j]
+          const int wstage = ring.stage;
+          const uint32_t wa = wait_slot();
+          ring.advance();
+          if (!ok) return;
+          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+          const uint32_t d_p = tmem_base + (j & 1) * 128;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            umma_bf16_ss_pair(d_p, (k < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((k & 3) * 2), wdesc + static_cast<uint64_t>(k * 128),
+                              idesc_ml1, k != 0 ? 1u : 0u);
+          release_slot(wstage);
+          umma_commit_pair(bar_pfull(j & 1));
+          umma_commit_pair(map_to_cta(bar_pfull(j & 1), peer));
+          if (j == NC - 1) {  // X is no longer needed by the tensor pipe
+            release_slot(xs0);
+            release_slot(xs1);
+          }
+        };
+        auto issue_ml2 = [&](int j) {
+          // O += S_j . W2[chunk j, :]
+          const int wstage = ring.stage;
+          const uint32_t wa = wait_slot();
+          ring.advance();
+          if (!ok) return;
+          const int sb = j & 1;
+          if (!mbar_wait<true>(bar_sfull(sb), sfull_uses[sb] & 1u, w)) { ok = false; return; }
+          ++sfull_uses[sb];
+          tcgen05_fence_after_sync();
+          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+          const uint64_t sdesc0 = make_smem_desc_sw128(s_addr(sb, 0), 16, 1024);
+          const uint64_t sdesc1 = make_smem_desc_sw128(s_addr(sb, 1), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            umma_bf16_ss_pair(d_o, (k < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((k & 3) * 2), wdesc + static_cast<uint64_t>(k * 128),
+                              idesc_ml2, (j | k) != 0 ? 1u : 0u);
+          release_slot(wstage);
+          umma_commit_pair(bar_sempty(sb));
+          umma_commit_pair(map_to_cta(bar_sempty(sb), peer));
+        };
+        // O slot must have been drained by Epi2 of the tile before the previous one
+        if (!mbar_wait<true>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        issue_ml1(0);
+        if (NC > 1) issue_ml1(1);
+        for (int j = 0; j < NC && ok; ++j) {
+          issue_ml2(j);
+          if (j + 2 < NC) issue_ml1(j + 2);
+        }
+        if (ok) {
+          umma_commit_pair(bar_ofull(obuf));
+          umma_commit_pair(map_to_cta(bar_ofull(obuf), peer));
+        }
+        ring.skip(2);  // the residual slots belong to the epilogue
+      }
+      umma_commit_pair(bar_drain);
+      mbar_wait<false>(bar_drain, 0, w);
+    }
+  } else {
+    // ------------------------------------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;
+    const int h = (warp - 2) >> 2;
+    const int row = q * 32 + lane;
+    const int epi_tid = threadIdx.x - 64;
+    const bool store_thread = epi_tid == 0;
+    const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
+    const uint32_t ybuf = smem_base + B2bSmem::OFF_YBUF;
+    const uint32_t sfull_leader = map_to_cta(bar_sfull(0), leader);
+    const uint32_t oempty_leader = map_to_cta(bar_oempty(0), leader);
+    RingPos<kRingSlots> ring;
+    uint32_t rfull_bits = 0;
+    uint32_t puses[2] = {0, 0}, suses[2] = {0, 0};
+    uint32_t tile_it = 0;
+    int xpar = 0;
+    uint32_t xphase = 0;
+
+    for (int tile = cluster_id; tile < p.mpairs; tile += num_clusters, ++tile_it) {
+      const int m0 = tile * 256 + static_cast<int>(pm) * 128;
+      const int obuf = tile_it & 1u;
+      // ---------------- Epi1(j): S_j = bf16(GELU(P_j + b1)) as the next UMMA's A operand
+      for (int j = 0; j < NC; ++j) {
+        const int pb = j & 1;
+        mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
+        ++puses[pb];
+        __syncwarp();
+        tcgen05_fence_after_sync();
+        // the S buffer is free once ML2 of chunk j-2 has read it
+        mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
+        ++suses[pb];
+        __syncwarp();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t v[32];
+          tmem_ld_32cols(tmem_base + lane_sel + pb * 128 + h * 64 + half * 32, v);
+          const float4* b4 = reinterpret_cast<const float4*>(s_b1 + j * 128 + h * 64 + half * 32);
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 bb = b4[i];
+            const float g0 = gelu_tanh_f32(__uint_as_float(v[4 * i]) + bb.x);
+            const float g1 = gelu_tanh_f32(__uint_as_float(v[4 * i + 1]) + bb.y);
+            const float g2 = gelu_tanh_f32(__uint_as_float(v[4 * i + 2]) + bb.z);
+            const float g3 = gelu_tanh_f32(__uint_as_float(v[4 * i + 3]) + bb.w);
+            pk[2 * i] = pack_bf16x2_rn(g0, g1);
+            pk[2 * i + 1] = pack_bf16x2_rn(g2, g3);
+          }
+          // this thread's 32 columns are 16-byte chunks half*4 .. half*4+3 of K block h of the S buffer
+          const uint32_t sb = s_addr(pb, h);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t a = sb + swz128(row, half * 4 + i);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                         "r"(pk[4 * i + 3])
+                         : "memory");
+          }
+        }
+        tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
+        fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
+        mbar_arrive_cluster(sfull_leader + 8u * pb);
+      }
+      ring.skip(2 + 2 * NC);  // X, W1 and W2 slots were the tensor pipe's
+      // ---------------- Epi2: O' = O + b2 + X, LayerNorm over the 128 columns, store
+      mbar_wait<false>(bar_ofull(obuf), (tile_it >> 1) & 1u, w);
+      __syncwarp();
+      tcgen05_fence_after_sync();
+      const int rstage = ring.stage + h >= kRingSlots ? ring.stage + h - kRingSlots : ring.stage + h;
+      // both residual slots are waited for by everybody (the phase bits must advance uniformly)
+      uint32_t r32[2][16];
+      {
+        const int s0 = ring.stage;
+        mbar_wait<false>(bar_rfull(s0), (rfull_bits >> s0) & 1u, w);
+        rfull_bits ^= 1u << s0;
+        const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
+        mbar_wait<false>(bar_rfull(s1), (rfull_bits >> s1) & 1u, w);
+        rfull_bits ^= 1u << s1;
+        __syncwarp();
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t a = ring_addr(rstage) + swz128(row, half * 4 + i);
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(r32[half][4 * i]), "=r"(r32[half][4 * i + 1]), "=r"(r32[half][4 * i + 2]), "=r"(r32[half][4 * i + 3])
+                       : "r"(a));
+        }
+      }
+      // hand the two residual slots back
+      __syncwarp();
+      named_barrier_sync(2, 256);
+      if (store_thread) {
+        mbar_arrive(bar_empty(ring.stage));
+        mbar_arrive(bar_empty(ring.stage + 1 == kRingSlots ? 0 : ring.stage + 1));
+      }
+      ring.skip(2);
+      // stage 1: x = O + b2 + X ; thread-local (mean, M2) over this thread's 64 columns
+      float x[2][32];
+      float2 part = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t v[32];
+        tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + h * 64 + half * 32, v);
+        const float4* b4 = reinterpret_cast<const float4*>(s_b2 + h * 64 + half * 32);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float4 bb = b4[i];
+          x[half][4 * i] = __uint_as_float(v[4 * i]) + bb.x + bf16_lo(r32[half][2 * i]);
+          x[half][4 * i + 1] = __uint_as_float(v[4 * i + 1]) + bb.y + bf16_hi(r32[half][2 * i]);
+          x[half][4 * i + 2] = __uint_as_float(v[4 * i + 2]) + bb.z + bf16_lo(r32[half][2 * i + 1]);
+          x[half][4 * i + 3] = __uint_as_float(v[4 * i + 3]) + bb.w + bf16_hi(r32[half][2 * i + 1]);
+          s0 += x[half][4 * i] + x[half][4 * i + 1];
+          s1 += x[half][4 * i + 2] + x[half][4 * i + 3];
+        }
+        const float cmean = (s0 + s1) * (1.f / 32.f);
+        float q0 = 0.f, q1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float d0 = x[half][i] - cmean, d1 = x[half][i + 1] - cmean;
+          q0 = fmaf(d0, d0, q0);
+          q1 = fmaf(d1, d1, q1);
+        }
+        const float2 cpart = make_float2(cmean, q0 + q1);
+        part = half == 0 ? cpart : MergeWelford()(part, 32.f, cpart, 32.f);
+      }
+      // the accumulator has been copied out: the O slot can be reused by the tile after the next one
+      tcgen05_fence_before_sync();
+      mbar_arrive_cluster(oempty_leader + 8u * obuf);
+      // reduce: the row lives in this CTA only (two half-row threads)
+      const float2 tot = cluster_row_reduce<1>(part, 64.f, MergeWelford(), s_pre, s_stats, bar_stats, row, h, 0u, xpar, xphase, w);
+      const float mu = tot.x;
+      const float rstd = rsqrtf(tot.y * (1.f / 128.f) + p.eps);
+      // stage 2: normalise, round once, stage one 128 x 64 box per half-row group and store it
+      uint32_t pk[2][16];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const float4* g4 = reinterpret_cast<const float4*>(s_gamma + h * 64 + half * 32);
+        const float4* be4 = reinterpret_cast<const float4*>(s_beta + h * 64 + half * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float4 gg = g4[i], be = be4[i];
+          const float y0 = fmaf((x[half][4 * i] - mu) * rstd, gg.x, be.x);
+          const float y1 = fmaf((x[half][4 * i + 1] - mu) * rstd, gg.y, be.y);
+          const float y2 = fmaf((x[half][4 * i + 2] - mu) * rstd, gg.z, be.z);
+          const float y3 = fmaf((x[half][4 * i + 3] - mu) * rstd, gg.w, be.w);
+          pk[half][2 * i] = pack_bf16x2_rn(y0, y1);
+          pk[half][2 * i + 1] = pack_bf16x2_rn(y2, y3);
+        }
+      }
+      // two boxes (columns 0..63 from the h = 0 threads, 64..127 from the h = 1 threads) through one staging buffer
+      for (int g = 0; g < 2; ++g) {
+        if (store_thread) tma_store_wait_read<0>();
+        named_barrier_sync(3, 256);
+        if (h == g) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t a = ybuf + swz128(row, half * 4 + i);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[half][4 * i]), "r"(pk[half][4 * i + 1]),
+                           "r"(pk[half][4 * i + 2]), "r"(pk[half][4 * i + 3])
+                           : "memory");
+            }
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(3, 256);
+        if (store_thread) {
+          tma_store_3d(&tmO, ybuf, g * 64, m0, 0);
+          tma_store_commit();
+        }
+      }
+    }
+    if (store_thread) tma_store_wait_all();
+  }
+
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool b2b_fused_supported(int K, int N1, int N2) {
+  return K == 128 && N2 == 128 && N1 >= 128 && N1 <= 128 * kMaxChunks && N1 % 128 == 0;
+}
+
+cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
+  const DeviceInfo* dev = current_device_info();
+  if (!dev) return cudaErrorInvalidDevice;
+  CUtensorMap tmX, tmW1, tmW2, tmO;
+  const uint64_t M = p.M, K = p.K, N1 = p.N1, N2 = p.N2;
+  // all boxes are 64 elements x 128 rows
+  if (!encode_tmap_bf16_3d(&tmX, X, K, M, 1, K * 2, M * K * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmW1, W1, N1, K, 1, N1 * 2, K * N1 * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmW2, W2, N2, N1, 1, N2 * 2, N1 * N2 * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmO, p.O, N2, M, 1, N2 * 2, M * N2 * 2, 128))
+    return cudaErrorInvalidValue;
+  p.mblocks = (p.M + 127) / 128;
+  p.mpairs = (p.mblocks + 1) / 2;
+
+  constexpr int kMaxDev = 64;
+  static int max_clusters[kMaxDev] = {0};
+  const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.blockDim = dim3(kB2bThreads, 1, 1);
+  cfg.dynamicSmemBytes = B2bSmem::BYTES;
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (max_clusters[di] == 0) {
+    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    if (e != cudaSuccess) return e;
+    int n = 0;
+    cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    if (n <= 0) return cudaErrorLaunchOutOfResources;
+    max_clusters[di] = n;
+  }
+  const int clusters = p.mpairs < max_clusters[di] ? p.mpairs : max_clusters[di];
+  cfg.gridDim = dim3(clusters * 2, 1, 1);
+  count_launch();
+  return cudaLaunchKernelEx(&cfg, b2b_pair_kernel, tmX, tmW1, tmW2, tmO, p);
+}
+
 }  // namespace comfuse

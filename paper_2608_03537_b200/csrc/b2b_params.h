@@ -8,7 +8,7 @@ namespace comfuse {
 
 struct B2bParams {
   int M, K, N1, N2;
-  int mblocks;
+  int mblocks, mpairs;  // 128-row blocks and pairs of them
   float eps;
   const uint16_t* X;  // also the residual of the tail
   const uint16_t* b1;

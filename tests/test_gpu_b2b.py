@@ -1,0 +1,68 @@
+"""GPU parity of the back-to-back GEMM: fused kernel (P and S never leave the chip) and the in-library unfused path
+(three bf16 intermediates) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_03537_b200 as cf
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # M, N1, affine
+    (256, 512, False),     # one row-block pair, all four N1 chunks
+    (300, 512, True),      # ragged: second pair has one partial block and one empty block
+    (1000, 256, True),     # two chunks
+    (130, 128, False),     # a single chunk: ML1 -> Epi1 -> ML2 with no overlap partner
+    (2048, 384, True),     # three chunks, several tiles per cluster on small grids
+]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,N1,affine", CASES)
+def test_b2b_mlp_layernorm(M, N1, affine, fused, cuda_device):
+    w = wl.b2b_mlp(M, 128, N1, 128, seed=M + N1, affine=affine)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"b2b M{M} N1{N1} fused={fused}")
+    assert cf.last_device_status() == cf.OK
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_config_b2b_mlp_full_size(fused, cuda_device):
+    """c5 at full size: sampled rows against the oracle; over every row, the un-normalised statistics property."""
+    w = wl.config(4)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    assert torch.isfinite(got["Y"].float()).all().item()
+    rows = wl.sample_rows(w.dims["M"], 512)
+    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c5 fused={fused}")
+    Y = got["Y"].float()          # gamma = 1, beta = 0: every row has mean ~0 and variance ~1
+    assert Y.mean(-1).abs().max().item() < 2e-2
+    assert (Y.var(-1, unbiased=False) - 1).abs().max().item() < 3e-2
+    print("c5", fused, res)
+
+
+def test_b2b_identity_second_weight(cuda_device):
+    """W2 = I, b2 = 0: the fused chain must reduce to LayerNorm(GELU(X W1 + b1) + X) (needs N1 = N2 = 128)."""
+    w = wl.b2b_mlp(384, 128, 128, 128, seed=7)
+    w.tensors["W2"] = wl.f32_to_bf16_bits(np.eye(128, dtype=np.float32))
+    w.tensors["b2"][:] = 0
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label="b2b identity W2")
+
+
+def test_b2b_bitwise_repeatable(cuda_device):
+    w = wl.b2b_mlp(2048, 128, 512, 128, seed=3)
+    T = P.dev_tensors(w)
+    a = P.run_gpu(w, T, fused=True)["Y"]
+    b = P.run_gpu(w, T, fused=True)["Y"]
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_b2b_unsupported_shapes_are_refused_for_the_fused_path(cuda_device):
+    d = cf.make_b2b_desc(256, 128, 640, 128, fused=True)      # N1 > 512
+    with pytest.raises(cf.ComfuseError) as e:
+        cf.b2b_workspace_size(d)
+    assert e.value.status == cf.ERR_UNSUPPORTED
+    assert cf.b2b_workspace_size(cf.make_b2b_desc(256, 128, 640, 128, fused=False)) == 256 * 640 * 2 + 256 * 128 * 2
