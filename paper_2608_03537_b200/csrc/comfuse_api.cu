@@ -104,7 +104,7 @@ bool make_gemm_maps(GemmMaps* maps, const void* A, const void* B, const void* R,
   };
   if (!encode_tmap_bf16_3d(&maps->A, A, K, M, batch, static_cast<uint64_t>(lda) * 2, bs(bsa, M, lda), 128)) return false;
   if (!encode_tmap_bf16_3d(&maps->B, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, K, ldb), 64)) return false;
-  if (!encode_tmap_bf16_3d(&maps->Y, Y, N, M, batch, static_cast<uint64_t>(ldy) * 2, bs(bsy, M, ldy), 128)) return false;
+  if (!encode_tmap_bf16_3d(&maps->Y, Y, N, M, batch, static_cast<uint64_t>(ldy) * 2, bs(bsy, M, ldy), 32)) return false;
   if (R && !encode_tmap_bf16_3d(&maps->R, R, N, M, batch, static_cast<uint64_t>(ldr) * 2, bs(bsr, M, ldr), 128)) return false;
   return true;
 }

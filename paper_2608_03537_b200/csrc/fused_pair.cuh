@@ -13,8 +13,10 @@
 // block pairs with a stride of the cluster count.
 //
 // Inside a CTA (10 warps): warp 0 = TMA producer, warp 1 = TMEM allocation and (even CTA only) UMMA issue,
-// warps 2-9 = epilogue (thread = one accumulator row; the two warps of a lane quarter split every 64-column
-// group into two 32-column fragments).
+// warps 2-9 = epilogue (thread = one accumulator row; the two warps of a lane quarter take alternate 64-column
+// groups).  Each epilogue warp is its own pipeline: it reads its 32 rows of the residual box, stages its 32 x 64
+// output box in a private shared-memory buffer and issues its own TMA store, so no CTA-wide barrier sits on the
+// per-group path.
 //
 // Pipelining (Sec. 3.3, PingPong at sub-tile grain).  The CTA's BN columns are one or two sub-tiles, each with its
 // own TMEM slot and full/empty barriers.  The MainLoop of sub-tile 1 runs while the epilogue's stage 1 works on
@@ -24,8 +26,8 @@
 // One circular shared-memory buffer feeds both consumers (the unified multi-stage buffer of Sec. 4.2, applied to
 // the epilogue operand): after the K blocks of a sub-tile the producer pushes that sub-tile's residual tile through
 // the same ring, 128 rows x 64 columns per TMA box, so the epilogue reads the residual from swizzled shared memory
-// instead of issuing one scattered global load per row.  Results leave the same way: 128 x 64 bf16 boxes are
-// written to a swizzled staging buffer and stored with TMA.
+// instead of issuing one scattered global load per row.  Results leave the same way: 32 x 64 bf16 boxes are
+// written to swizzled per-warp staging buffers and stored with TMA.
 #pragma once
 
 #include "epilogue_common.cuh"
@@ -48,7 +50,8 @@ struct PairCfg {
   static constexpr int ACC_COLS = NSUB == 2 ? BN : 2 * BNS0;              // two TMEM slots
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
-  static constexpr int YBUF_BYTES = 2 * GROUP_BYTES;
+  static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
+  static constexpr int YBUF_BYTES = 8 * WARP_BOX_BYTES;
   static constexpr int OFF_VEC = OFF_YBUF + YBUF_BYTES;
   static constexpr int VEC_BYTES = 3 * BN * 4;
   static constexpr int OFF_STATS = OFF_VEC + VEC_BYTES;
@@ -56,12 +59,13 @@ struct PairCfg {
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
   static constexpr int PRE_BYTES = 2 * 2 * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 3 * NSTAGES + 4 + 2;
+  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
   static_assert(BNS0 > 0 && ACC_COLS <= 512, "accumulators must fit the 512 TMEM columns");
   static_assert(NSTAGES <= 8, "per-stage phase bits are kept in one byte");
+  static_assert(GROUPS_PER_STAGE == 2, "a residual stage carries one even and one odd 64-column group");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
 };
@@ -106,9 +110,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto bar_full = [&](int s) { return bar_base + 8u * s; };                     // K-block stage landed (even CTA)
   auto bar_empty = [&](int s) { return bar_base + 8u * (NSTAGES + s); };        // stage may be overwritten
   auto bar_rfull = [&](int s) { return bar_base + 8u * (2 * NSTAGES + s); };    // residual stage landed (own CTA)
-  auto bar_tfull = [&](int a) { return bar_base + 8u * (3 * NSTAGES + a); };    // accumulator slot complete
-  auto bar_tempty = [&](int a) { return bar_base + 8u * (3 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
-  const uint32_t bar_stats = bar_base + 8u * (3 * NSTAGES + 4);
+  auto bar_rdone = [&](int s) { return bar_base + 8u * (3 * NSTAGES + s); };    // residual stage read by all 8 warps
+  auto bar_tfull = [&](int a) { return bar_base + 8u * (4 * NSTAGES + a); };    // accumulator slot complete
+  auto bar_tempty = [&](int a) { return bar_base + 8u * (4 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
+  const uint32_t bar_stats = bar_base + 8u * (4 * NSTAGES + 4);
   const uint32_t bar_drain = bar_stats + 8u;
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
@@ -131,8 +136,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(bar_full(s), 2);   // one arrive.expect_tx from each CTA of the pair
-      mbar_init(bar_empty(s), 1);  // one commit from the issuing CTA, or one arrive from the epilogue (residual stage)
+      mbar_init(bar_empty(s), 1);  // one commit from the issuing CTA
       mbar_init(bar_rfull(s), 1);
+      mbar_init(bar_rdone(s), 8);  // one arrive per epilogue warp
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull(a), 1);
@@ -187,6 +193,21 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (lane == 0) {
       RingPos<NSTAGES> ring;
       bool ok = true;
+      // A stage is handed back by the UMMA commit (K-block use) or by the eight epilogue warps (residual use); the two
+      // kinds have their own barriers, so the producer remembers each stage's last use and each barrier's phase.
+      uint32_t used = 0, last_res = 0, empty_bits = 0, rdone_bits = 0;
+      auto wait_stage_free = [&](int st) {
+        const uint32_t bit = 1u << st;
+        if (!(used & bit)) return true;
+        if (last_res & bit) {
+          if (!mbar_wait<false>(bar_rdone(st), (rdone_bits >> st) & 1u, w)) return false;
+          rdone_bits ^= bit;
+        } else {
+          if (!mbar_wait<false>(bar_empty(st), (empty_bits >> st) & 1u, w)) return false;
+          empty_bits ^= bit;
+        }
+        return true;
+      };
       for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
@@ -198,7 +219,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!ok || !unit_live(mpair0, n0)) continue;
           const uint32_t bytes = Cfg::A_BYTES + (W / 2) * 128;
           for (int kb = 0; kb < KB; ++kb) {
-            if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; break; }
+            if (!wait_stage_free(ring.stage)) { ok = false; break; }
+            used |= 1u << ring.stage;
+            last_res &= ~(1u << ring.stage);
             const uint32_t sa = smem_base + ring.stage * Cfg::STAGE_BYTES;
             const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
             mbar_arrive_expect_tx_cluster(full, bytes);
@@ -211,7 +234,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // the sub-tile's residual tile rides the same ring, right behind its last K block
             const int groups = W / 64;
             for (int g0 = 0; g0 < groups; g0 += GPS) {
-              if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; break; }
+              if (!wait_stage_free(ring.stage)) { ok = false; break; }
+              used |= 1u << ring.stage;
+              last_res |= 1u << ring.stage;
               const int ng = groups - g0 < GPS ? groups - g0 : GPS;
               const uint32_t sr = smem_base + ring.stage * Cfg::STAGE_BYTES;
               mbar_arrive_expect_tx(bar_rfull(ring.stage), ng * Cfg::GROUP_BYTES);
@@ -276,11 +301,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;
-    const int h = (warp - 2) >> 2;
+    const int q = warp & 3;         // TMEM lane quarter this warp may touch: rows 32q .. 32q+31 of the tile
+    const int h = (warp - 2) >> 2;  // this warp takes the 64-column groups of parity h
     const int row = q * 32 + lane;
-    const int epi_tid = threadIdx.x - 64;
-    const bool store_thread = epi_tid == 0;
     const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
     int xpar = 0;
     uint32_t xphase = 0;
@@ -289,36 +312,34 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     uint32_t rfull_bits = 0;
     uint32_t slot_uses[2] = {0, 0};
     uint32_t unit_count = 0;
-    uint32_t ygroup = 0;  // running count of output boxes: selects the staging buffer
-    constexpr float kThreadCount = static_cast<float>(BN / 2);
+    constexpr float kThreadCount = static_cast<float>(BN / 2);  // columns behind one thread's partial
     const uint32_t tempty_leader = map_to_cta(bar_tempty(0), leader);
-    const uint32_t ybuf = smem_base + Cfg::OFF_YBUF;
+    const uint32_t ybox = smem_base + Cfg::OFF_YBUF + (warp - 2) * Cfg::WARP_BOX_BYTES;  // this warp's staging box
 
-    // Stage one 128 x 64 box of packed bf16 (this thread: 32 columns of its row) and store it with TMA.
-    auto store_group = [&](const uint32_t (&pk)[16], int col0, int m0, int b) {
-      const uint32_t buf = ybuf + (ygroup & 1u) * Cfg::GROUP_BYTES;
-      ++ygroup;
-      if (store_thread) tma_store_wait_read<1>();  // the box that used this buffer two stores ago has been read out
-      named_barrier_sync(3, 256);
+    // Stage this thread's 64 packed columns (its row of the warp's 32 x 64 box) and store the box with TMA.
+    // pk[0..15] are columns 0..31 of the group, pk[16..31] columns 32..63.
+    auto store_box = [&](const uint32_t (&pk)[32], int col0, int m0, int b) {
+      if (lane == 0) tma_store_wait_read<0>();  // the previous box has been read out of the staging buffer
+      __syncwarp();
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t a = buf + swz128(row, h * 4 + i);
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t a = ybox + swz128(lane, i);
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
                      "r"(pk[4 * i + 3])
                      : "memory");
       }
       fence_proxy_async_smem();
-      named_barrier_sync(3, 256);
-      if (store_thread) {
-        tma_store_3d(&tmY, buf, col0, m0, b);
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_3d(&tmY, ybox, col0, m0 + q * 32, b);
         tma_store_commit();
       }
     };
-    // This thread's 32 residual values of group `g` of a residual stage, as 16 packed bf16 pairs.
-    auto load_residual = [&](uint32_t stage_addr, int g, uint32_t (&r32)[16]) {
+    // This thread's 64 residual values of box `gg` of a residual stage, as 32 packed bf16 pairs.
+    auto load_residual = [&](uint32_t stage_addr, int gg, uint32_t (&r32)[32]) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t a = stage_addr + g * Cfg::GROUP_BYTES + swz128(row, h * 4 + i);
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t a = stage_addr + gg * Cfg::GROUP_BYTES + swz128(row, i);
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                      : "=r"(r32[4 * i]), "=r"(r32[4 * i + 1]), "=r"(r32[4 * i + 2]), "=r"(r32[4 * i + 3])
                      : "r"(a));
@@ -365,14 +386,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           wait_accumulator(sub);
           const int W = sub ? BNS1 : BNS0;
           const int n0 = ncta0 + (sub ? BNS0 : 0);
-          for (int g = 0; g < W / 64; ++g) {
+          for (int g = h; g < W / 64; g += 2) {
             if (n0 + g * 64 >= p.N) break;
-            uint32_t v[32];
-            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
-            uint32_t pk[16];
+            uint32_t pk[32];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-            store_group(pk, n0 + g * 64, m0, b);
+            for (int half = 0; half < 2; ++half) {
+              uint32_t v[32];
+              tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            }
+            store_box(pk, n0 + g * 64, m0, b);
           }
           release_accumulator(sub);
         }
@@ -387,38 +412,37 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = sub ? BNS1 : BNS0;
           const int lsub = sub ? BNS0 : 0;  // first column of the sub-tile inside the CTA's column range
           const uint32_t taddr = tmem_of(sub);
-          for (int g0 = 0; g0 < W / 64; g0 += GPS) {
-            uint32_t stage_addr = 0;
+          for (int g = h; g < W / 64; g += 2) {
+            // groups (g - h, g - h + 1) share one residual stage; this warp reads box h of it
+            uint32_t r32[32];
             if (has_res) {
               mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
               rfull_bits ^= 1u << ring.stage;
               __syncwarp();
-              stage_addr = smem_base + ring.stage * Cfg::STAGE_BYTES;
+              load_residual(smem_base + ring.stage * Cfg::STAGE_BYTES, h, r32);
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_rdone(ring.stage));  // this warp is done with the stage
+              ring.advance();
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r32[j] = 0u;
             }
 #pragma unroll
-            for (int gg = 0; gg < GPS; ++gg) {
-              const int g = g0 + gg;
-              if (g >= W / 64) break;
-              const int lc = lsub + g * 64 + h * 32;
+            for (int half = 0; half < 2; ++half) {
+              const int lc = lsub + g * 64 + half * 32;
               uint32_t v[32];
-              tmem_ld_32cols(taddr + g * 64 + h * 32, v);
-              uint32_t r32[16];
-              if (has_res) {
-                load_residual(stage_addr, gg, r32);
-              } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) r32[j] = 0u;
-              }
+              tmem_ld_32cols(taddr + g * 64 + half * 32, v);
               const float4* bias4 = reinterpret_cast<const float4*>(s_bias + lc);
               if constexpr (EPI == EPI_LN) {
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 bb = bias4[j];
-                  const float x0 = fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x) + bf16_lo(r32[2 * j]);
-                  const float x1 = fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y) + bf16_hi(r32[2 * j]);
-                  const float x2 = fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z) + bf16_lo(r32[2 * j + 1]);
-                  const float x3 = fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w) + bf16_hi(r32[2 * j + 1]);
+                  const uint32_t ra = r32[half * 16 + 2 * j], rb = r32[half * 16 + 2 * j + 1];
+                  const float x0 = fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x) + bf16_lo(ra);
+                  const float x1 = fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y) + bf16_hi(ra);
+                  const float x2 = fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z) + bf16_lo(rb);
+                  const float x3 = fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w) + bf16_hi(rb);
                   v[4 * j] = __float_as_uint(x0); v[4 * j + 1] = __float_as_uint(x1);
                   v[4 * j + 2] = __float_as_uint(x2); v[4 * j + 3] = __float_as_uint(x3);
                   s0 += x0; s1 += x1; s2 += x2; s3 += x3;
@@ -439,24 +463,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 bb = bias4[j];
-                  const float h0 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x)) + bf16_lo(r32[2 * j]);
-                  const float h1 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y)) + bf16_hi(r32[2 * j]);
-                  const float h2 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z)) + bf16_lo(r32[2 * j + 1]);
-                  const float h3 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w)) + bf16_hi(r32[2 * j + 1]);
+                  const uint32_t ra = r32[half * 16 + 2 * j], rb = r32[half * 16 + 2 * j + 1];
+                  const float h0 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x)) + bf16_lo(ra);
+                  const float h1 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y)) + bf16_hi(ra);
+                  const float h2 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z)) + bf16_lo(rb);
+                  const float h3 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w)) + bf16_hi(rb);
                   v[4 * j] = __float_as_uint(h0); v[4 * j + 1] = __float_as_uint(h1);
                   v[4 * j + 2] = __float_as_uint(h2); v[4 * j + 3] = __float_as_uint(h3);
                   q0 = fmaf(h0, h0, q0); q1 = fmaf(h1, h1, q1); q2 = fmaf(h2, h2, q2); q3 = fmaf(h3, h3, q3);
                 }
                 part.x += (q0 + q1) + (q2 + q3);
               }
-              tmem_st_32cols(taddr + g * 64 + h * 32, v);
-            }
-            if (has_res) {
-              // all 256 threads are done with this residual stage: hand it back to the producer
-              __syncwarp();
-              named_barrier_sync(2, 256);
-              if (store_thread) mbar_arrive(bar_empty(ring.stage));
-              ring.advance();
+              tmem_st_32cols(taddr + g * 64 + half * 32, v);
             }
           }
         }
@@ -481,38 +499,41 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = sub ? BNS1 : BNS0;
           const int lsub = sub ? BNS0 : 0;
           const uint32_t taddr = tmem_of(sub);
-          for (int g = 0; g < W / 64; ++g) {
-            const int lc = lsub + g * 64 + h * 32;
-            uint32_t v[32];
-            tmem_ld_32cols(taddr + g * 64 + h * 32, v);
-            const float4* g4 = reinterpret_cast<const float4*>(s_gamma + lc);
-            const float4* b4 = reinterpret_cast<const float4*>(s_beta + lc);
-            uint32_t pk[16];
+          for (int g = h; g < W / 64; g += 2) {
+            uint32_t pk[32];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const float4 gg = g4[j];
-              float y0, y1, y2, y3;
-              if constexpr (EPI == EPI_LN) {
-                const float4 be = b4[j];
-                y0 = fmaf((__uint_as_float(v[4 * j]) - mu) * rstd, gg.x, be.x);
-                y1 = fmaf((__uint_as_float(v[4 * j + 1]) - mu) * rstd, gg.y, be.y);
-                y2 = fmaf((__uint_as_float(v[4 * j + 2]) - mu) * rstd, gg.z, be.z);
-                y3 = fmaf((__uint_as_float(v[4 * j + 3]) - mu) * rstd, gg.w, be.w);
-              } else {
-                y0 = __uint_as_float(v[4 * j]) * rstd * gg.x;
-                y1 = __uint_as_float(v[4 * j + 1]) * rstd * gg.y;
-                y2 = __uint_as_float(v[4 * j + 2]) * rstd * gg.z;
-                y3 = __uint_as_float(v[4 * j + 3]) * rstd * gg.w;
-                const int c = ncta0 + lc + 4 * j;
-                if (y0 > best) { best = y0; best_col = c; }
-                if (y1 > best) { best = y1; best_col = c + 1; }
-                if (y2 > best) { best = y2; best_col = c + 2; }
-                if (y3 > best) { best = y3; best_col = c + 3; }
+            for (int half = 0; half < 2; ++half) {
+              const int lc = lsub + g * 64 + half * 32;
+              uint32_t v[32];
+              tmem_ld_32cols(taddr + g * 64 + half * 32, v);
+              const float4* g4 = reinterpret_cast<const float4*>(s_gamma + lc);
+              const float4* b4 = reinterpret_cast<const float4*>(s_beta + lc);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float4 gg = g4[j];
+                float y0, y1, y2, y3;
+                if constexpr (EPI == EPI_LN) {
+                  const float4 be = b4[j];
+                  y0 = fmaf((__uint_as_float(v[4 * j]) - mu) * rstd, gg.x, be.x);
+                  y1 = fmaf((__uint_as_float(v[4 * j + 1]) - mu) * rstd, gg.y, be.y);
+                  y2 = fmaf((__uint_as_float(v[4 * j + 2]) - mu) * rstd, gg.z, be.z);
+                  y3 = fmaf((__uint_as_float(v[4 * j + 3]) - mu) * rstd, gg.w, be.w);
+                } else {
+                  y0 = __uint_as_float(v[4 * j]) * rstd * gg.x;
+                  y1 = __uint_as_float(v[4 * j + 1]) * rstd * gg.y;
+                  y2 = __uint_as_float(v[4 * j + 2]) * rstd * gg.z;
+                  y3 = __uint_as_float(v[4 * j + 3]) * rstd * gg.w;
+                  const int c = ncta0 + lc + 4 * j;
+                  if (y0 > best) { best = y0; best_col = c; }
+                  if (y1 > best) { best = y1; best_col = c + 1; }
+                  if (y2 > best) { best = y2; best_col = c + 2; }
+                  if (y3 > best) { best = y3; best_col = c + 3; }
+                }
+                pk[half * 16 + 2 * j] = pack_bf16x2_rn(y0, y1);
+                pk[half * 16 + 2 * j + 1] = pack_bf16x2_rn(y2, y3);
               }
-              pk[2 * j] = pack_bf16x2_rn(y0, y1);
-              pk[2 * j + 1] = pack_bf16x2_rn(y2, y3);
             }
-            store_group(pk, ncta0 + lsub + g * 64, m0, b);
+            store_box(pk, ncta0 + lsub + g * 64, m0, b);
           }
           release_accumulator(sub);
         }
@@ -541,20 +562,23 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!live[sub]) continue;
           const int W = sub ? BNS1 : BNS0;
           const int n0 = ncta0 + (sub ? BNS0 : 0);
-          for (int g = 0; g < W / 64; ++g) {
-            const int col0 = n0 + g * 64 + h * 32;
-            const int st = frag_state(col0);
-            if (st == 0) continue;
-            uint32_t v[32];
-            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
-            float m0v = -INFINITY, m1v = -INFINITY;
+          for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
-              if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
-              if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+            for (int half = 0; half < 2; ++half) {
+              const int col0 = n0 + g * 64 + half * 32;
+              const int st = frag_state(col0);
+              if (st == 0) continue;
+              uint32_t v[32];
+              tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              float m0v = -INFINITY, m1v = -INFINITY;
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
+                if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
+                if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+              }
+              mloc = fmaxf(mloc, fmaxf(m0v, m1v));
             }
-            mloc = fmaxf(mloc, fmaxf(m0v, m1v));
           }
         }
         // ---------------- pass B: e = 2^(t - mloc), thread-local sum, e written back over the scores
@@ -565,28 +589,31 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!live[sub]) continue;
           const int W = sub ? BNS1 : BNS0;
           const int n0 = ncta0 + (sub ? BNS0 : 0);
-          for (int g = 0; g < W / 64; ++g) {
-            const int col0 = n0 + g * 64 + h * 32;
-            const int st = frag_state(col0);
-            if (st == 0) continue;
-            uint32_t v[32];
-            tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
-            float s0 = 0.f, s1 = 0.f;
+          for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              float e0 = ex2_approx(fmaf(__uint_as_float(v[j]), sc, -msub));
-              float e1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), sc, -msub));
-              if (st != 2) {
-                if (col0 + j > grow) e0 = 0.f;
-                if (col0 + j + 1 > grow) e1 = 0.f;
+            for (int half = 0; half < 2; ++half) {
+              const int col0 = n0 + g * 64 + half * 32;
+              const int st = frag_state(col0);
+              if (st == 0) continue;
+              uint32_t v[32];
+              tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                float e0 = ex2_approx(fmaf(__uint_as_float(v[j]), sc, -msub));
+                float e1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), sc, -msub));
+                if (st != 2) {
+                  if (col0 + j > grow) e0 = 0.f;
+                  if (col0 + j + 1 > grow) e1 = 0.f;
+                }
+                v[j] = __float_as_uint(e0);
+                v[j + 1] = __float_as_uint(e1);
+                s0 += e0;
+                s1 += e1;
               }
-              v[j] = __float_as_uint(e0);
-              v[j + 1] = __float_as_uint(e1);
-              s0 += e0;
-              s1 += e1;
+              lloc += s0 + s1;
+              tmem_st_32cols(tmem_of(sub) + g * 64 + half * 32, v);
             }
-            lloc += s0 + s1;
-            tmem_st_32cols(tmem_of(sub) + g * 64 + h * 32, v);
           }
         }
         tmem_st_wait();
@@ -598,26 +625,30 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int sub = 0; sub < NSUB; ++sub) {
           const int W = sub ? BNS1 : BNS0;
           const int n0 = ncta0 + (sub ? BNS0 : 0);
-          for (int g = 0; g < W / 64; ++g) {
-            const int col0 = n0 + g * 64 + h * 32;
-            const int st = live[sub] ? frag_state(col0) : 0;
-            uint32_t pk[16];
-            if (st == 0) {
+          for (int g = h; g < W / 64; g += 2) {
+            uint32_t pk[32];
 #pragma unroll
-              for (int j = 0; j < 16; ++j) pk[j] = 0u;
-            } else {
-              uint32_t v[32];
-              tmem_ld_32cols(tmem_of(sub) + g * 64 + h * 32, v);
+            for (int half = 0; half < 2; ++half) {
+              const int col0 = n0 + g * 64 + half * 32;
+              const int st = live[sub] ? frag_state(col0) : 0;
+              if (st == 0) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = 0u;
+              } else {
+                uint32_t v[32];
+                tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
+              }
             }
-            store_group(pk, n0 + g * 64, m0, b);
+            store_box(pk, n0 + g * 64, m0, b);
           }
           release_accumulator(sub);
         }
       }
     }
-    if (store_thread) tma_store_wait_all();  // the staging buffers must outlive the last store's read
+    if (lane == 0) tma_store_wait_all();  // the staging buffer must outlive the last store's read
   }
 
   // -------------------------------------------------------------------------------------------- teardown

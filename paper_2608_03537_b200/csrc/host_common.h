@@ -28,7 +28,8 @@ bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t d0, uint64
                          uint64_t stride2_bytes, uint32_t box_rows);
 
 // Tensor maps of one GEMM -> subgraph call: operands A [batch, M, K] and B [batch, K, N], residual R and output Y
-// [batch, M, N]; all bf16, 128-byte swizzle, boxes of 64 elements by 128 rows (A, R, Y) or 64 rows (B).
+// [batch, M, N]; all bf16, 128-byte swizzle, boxes of 64 elements by 128 rows (A, R), 64 rows (B) or 32 rows (Y: one
+// epilogue warp's box).
 struct GemmMaps {
   CUtensorMap A, B, R, Y;
 };
