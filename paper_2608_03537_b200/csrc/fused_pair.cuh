@@ -51,7 +51,13 @@ struct PairCfg {
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
-  static constexpr int YBUF_BYTES = 8 * WARP_BOX_BYTES;
+  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * 2 * 128 * 8 + (4 * NSTAGES + 6) * 8 + 16 + 1024;
+  static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (8 * WARP_BOX_BYTES);
+  static constexpr int YBOXES = YBOX_ROOM >= 4 ? 4 : YBOX_ROOM;           // staging boxes per epilogue warp
+  static constexpr int YBUF_BYTES = YBOXES * 8 * WARP_BOX_BYTES;
+  // Softmax only: the CTA's 64-column groups are interleaved with its peers' (group g of column range c is global
+  // group g*CN + c), so that a causal mask leaves every CTA of the reduction group the same share of live columns.
+  static constexpr bool INTERLEAVE = EPI == EPI_SOFTMAX;
   static constexpr int OFF_VEC = OFF_YBUF + YBUF_BYTES;
   static constexpr int VEC_BYTES = 3 * BN * 4;
   static constexpr int OFF_STATS = OFF_VEC + VEC_BYTES;
@@ -67,6 +73,7 @@ struct PairCfg {
   static_assert(NSTAGES <= 8, "per-stage phase bits are kept in one byte");
   static_assert(GROUPS_PER_STAGE == 2, "a residual stage carries one even and one odd 64-column group");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+  static_assert(YBOXES >= 1, "at least one staging box per epilogue warp");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
 };
 
@@ -184,8 +191,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     mpair0 = mp * 256;
     ncta0 = (nb * CN + static_cast<int>(crank)) * BN;
   };
+  // First global column of this CTA's local 64-column group `lg` (0 .. BN/64-1).
+  auto group_col = [&](int ncta0, int lg) { return Cfg::INTERLEAVE ? (lg * CN + static_cast<int>(crank)) * 64 : ncta0 + lg * 64; };
   // A sub-tile is not computed when it lies past N, or when the causal mask removes it for BOTH row blocks of the
-  // pair.  Every role evaluates the same predicate.
+  // pair (its first group has the smallest columns).  Every role evaluates the same predicate.
   auto unit_live = [&](int mpair0, int n0) { return n0 < p.N && !(EPI == EPI_SOFTMAX && p.causal && n0 > mpair0 + 255); };
 
   if (warp == 0) {
@@ -215,7 +224,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int sub = 0; sub < NSUB; ++sub) {
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;  // first local 64-column group of the sub-tile
+          const int n0 = group_col(ncta0, lg0);
           if (!ok || !unit_live(mpair0, n0)) continue;
           const uint32_t bytes = Cfg::A_BYTES + (W / 2) * 128;
           for (int kb = 0; kb < KB; ++kb) {
@@ -227,7 +237,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             mbar_arrive_expect_tx_cluster(full, bytes);
             tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
             for (int j = 0; j < W / 128; ++j)
-              tma_load_3d_pair(sa + Cfg::A_BYTES + j * 8192, &tmB, full, n0 + static_cast<int>(pm) * (W / 2) + j * 64, kb * 64, b);
+              tma_load_3d_pair(sa + Cfg::A_BYTES + j * 8192, &tmB, full, group_col(ncta0, lg0 + static_cast<int>(pm) * (W / 128) + j), kb * 64, b);
             ring.advance();
           }
           if (ok && has_res) {
@@ -241,7 +251,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               const uint32_t sr = smem_base + ring.stage * Cfg::STAGE_BYTES;
               mbar_arrive_expect_tx(bar_rfull(ring.stage), ng * Cfg::GROUP_BYTES);
               for (int g = 0; g < ng; ++g)
-                tma_load_3d(sr + g * Cfg::GROUP_BYTES, &tmR, bar_rfull(ring.stage), n0 + (g0 + g) * 64, m0, b);
+                tma_load_3d(sr + g * Cfg::GROUP_BYTES, &tmR, bar_rfull(ring.stage), group_col(ncta0, lg0 + g0 + g), m0, b);
               ring.advance();
             }
           }
@@ -262,7 +272,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int sub = 0; sub < NSUB; ++sub) {
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;  // first local 64-column group of the sub-tile
+          const int n0 = group_col(ncta0, lg0);
           if (!ok || !unit_live(mpair0, n0)) continue;
           const int slot = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
           ++unit_count;
@@ -314,12 +325,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     uint32_t unit_count = 0;
     constexpr float kThreadCount = static_cast<float>(BN / 2);  // columns behind one thread's partial
     const uint32_t tempty_leader = map_to_cta(bar_tempty(0), leader);
-    const uint32_t ybox = smem_base + Cfg::OFF_YBUF + (warp - 2) * Cfg::WARP_BOX_BYTES;  // this warp's staging box
+    const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + (warp - 2) * Cfg::YBOXES * Cfg::WARP_BOX_BYTES;  // this warp's staging boxes
+    uint32_t ybox_sel = 0;
 
     // Stage this thread's 64 packed columns (its row of the warp's 32 x 64 box) and store the box with TMA.
     // pk[0..15] are columns 0..31 of the group, pk[16..31] columns 32..63.
     auto store_box = [&](const uint32_t (&pk)[32], int col0, int m0, int b) {
-      if (lane == 0) tma_store_wait_read<0>();  // the previous box has been read out of the staging buffer
+      const uint32_t ybox = ybox0 + ybox_sel * Cfg::WARP_BOX_BYTES;
+      if (++ybox_sel == Cfg::YBOXES) ybox_sel = 0;
+      if (lane == 0) tma_store_wait_read<Cfg::YBOXES - 1>();  // the last store that used this box has read it out
       __syncwarp();
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -358,7 +372,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       int slot[NSUB];
 #pragma unroll
       for (int sub = 0; sub < NSUB; ++sub) {
-        live[sub] = unit_live(mpair0, ncta0 + (sub ? BNS0 : 0));
+        live[sub] = unit_live(mpair0, group_col(ncta0, sub ? BNS0 / 64 : 0));
         slot[sub] = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
         if (live[sub]) ++unit_count;
       }
@@ -385,9 +399,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!live[sub]) continue;
           wait_accumulator(sub);
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;
           for (int g = h; g < W / 64; g += 2) {
-            if (n0 + g * 64 >= p.N) break;
+            if (group_col(ncta0, lg0 + g) >= p.N) break;
             uint32_t pk[32];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -397,7 +411,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               for (int j = 0; j < 16; ++j)
                 pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
             }
-            store_box(pk, n0 + g * 64, m0, b);
+            store_box(pk, group_col(ncta0, lg0 + g), m0, b);
           }
           release_accumulator(sub);
         }
@@ -561,11 +575,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           wait_accumulator(sub);
           if (!live[sub]) continue;
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;
           for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-              const int col0 = n0 + g * 64 + half * 32;
+              const int col0 = group_col(ncta0, lg0 + g) + half * 32;
               const int st = frag_state(col0);
               if (st == 0) continue;
               uint32_t v[32];
@@ -588,11 +602,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int sub = 0; sub < NSUB; ++sub) {
           if (!live[sub]) continue;
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;
           for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-              const int col0 = n0 + g * 64 + half * 32;
+              const int col0 = group_col(ncta0, lg0 + g) + half * 32;
               const int st = frag_state(col0);
               if (st == 0) continue;
               uint32_t v[32];
@@ -624,12 +638,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int sub = 0; sub < NSUB; ++sub) {
           const int W = sub ? BNS1 : BNS0;
-          const int n0 = ncta0 + (sub ? BNS0 : 0);
+          const int lg0 = sub ? BNS0 / 64 : 0;
           for (int g = h; g < W / 64; g += 2) {
             uint32_t pk[32];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-              const int col0 = n0 + g * 64 + half * 32;
+              const int col0 = group_col(ncta0, lg0 + g) + half * 32;
               const int st = live[sub] ? frag_state(col0) : 0;
               if (st == 0) {
 #pragma unroll
@@ -642,7 +656,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
               }
             }
-            store_box(pk, n0 + g * 64, m0, b);
+            store_box(pk, group_col(ncta0, lg0 + g), m0, b);
           }
           release_accumulator(sub);
         }

@@ -9,11 +9,11 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   case n:                                \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst>(maps, p, st);
   switch (p.N) {
-    COMFUSE_CASE(256, 256, 0, 1, 5)
-    COMFUSE_CASE(512, 256, 256, 1, 5)
-    COMFUSE_CASE(1024, 256, 256, 2, 5)
-    COMFUSE_CASE(2048, 256, 256, 4, 5)
-    COMFUSE_CASE(4096, 256, 256, 8, 5)
+    COMFUSE_CASE(256, 256, 0, 1, 3)
+    COMFUSE_CASE(512, 256, 256, 1, 3)
+    COMFUSE_CASE(1024, 256, 256, 2, 3)
+    COMFUSE_CASE(2048, 256, 256, 4, 3)
+    COMFUSE_CASE(4096, 256, 256, 8, 3)
     default:
       return cudaErrorInvalidValue;
   }
