@@ -43,6 +43,8 @@ def _newest_header_mtime() -> float:
 
 def _compile(src: str, obj: str, verbose: bool) -> None:
     cmd = [_nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+    if os.environ.get("COMFUSE_BUILD_TRACE"):   # phase-timestamp tracing build (see fused_params.h: trace)
+        cmd.insert(1, "-DCOMFUSE_TRACE")
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -255,6 +255,11 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
   p.status = dev->status_word;
   p.timeout_ns = timeout_ns();
+#ifdef COMFUSE_TRACE
+  // tracing build: COMFUSE_TRACE_PTR holds the device address of a uint64[64] buffer for phase timestamps
+  if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) p.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));
+  if (const char* tf = std::getenv("COMFUSE_TRACE_FLAGS")) p.trace_flags = std::atoi(tf);
+#endif
 
   cudaError_t e;
   if (desc->fused) {

@@ -8,10 +8,10 @@
 namespace comfuse {
 
 // One work item = a pair of adjacent 128-row blocks (times p.nblocks column blocks of CN*BN columns).
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES>
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0>
 cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream_t stream) {
-  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES>;
-  auto kern = fused_pair_kernel<EPI, BNS0, BNS1, CN, NSTAGES>;
+  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
+  auto kern = fused_pair_kernel<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
   const DeviceInfo* dev = current_device_info();
   if (!dev) return cudaErrorInvalidDevice;
   constexpr int kCluster = 2 * CN;

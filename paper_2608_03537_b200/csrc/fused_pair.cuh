@@ -16,7 +16,8 @@
 // warps 2-9 = epilogue (thread = one accumulator row; the two warps of a lane quarter take alternate 64-column
 // groups).  Each epilogue warp is its own pipeline: it reads its 32 rows of the residual box, stages its 32 x 64
 // output box in a private shared-memory buffer and issues its own TMA store, so no CTA-wide barrier sits on the
-// per-group path.
+// per-group path.  warp 10 = store warp: lane e waits for epilogue warp e's staged boxes and issues their TMA stores, so
+// the epilogue warps never stall on the store engine (about 40 GB/s per SM) and run ahead by the staging depth.
 //
 // Pipelining (Sec. 3.3, PingPong at sub-tile grain).  The CTA's BN columns are one or two sub-tiles, each with its
 // own TMEM slot and full/empty barriers.  The MainLoop of sub-tile 1 runs while the epilogue's stage 1 works on
@@ -36,22 +37,25 @@
 
 namespace comfuse {
 
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES>
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0>
 struct PairCfg {
-  static constexpr int kThreads = 320;
+  static constexpr int kThreads = 352;  // producer, UMMA, 8 epilogue warps, store warp
   static constexpr int kEpiThreads = 256;
   static constexpr int NSUB = BNS1 > 0 ? 2 : 1;
   static constexpr int BN = BNS0 + BNS1;
   static constexpr int BNSMAX = BNS0 > BNS1 ? BNS0 : BNS1;
   static constexpr int A_BYTES = 128 * 64 * 2;
   static constexpr int GROUP_BYTES = 128 * 64 * 2;                        // one 128 x 64 bf16 box
-  static constexpr int STAGE_BYTES = A_BYTES + (BNSMAX / 2) * 64 * 2;     // A tile + this CTA's half of the B tile
+  // LOCK = 1: both sub-tiles advance in lock step, one ring stage carries A and BOTH sub-tiles' B halves (A is fetched
+  // and read once per K block: less L2 -> shared-memory traffic, no overlap between the sub-tiles' epilogue and MainLoop).
+  static constexpr int STAGE_BYTES = A_BYTES + ((LOCK ? BN : BNSMAX) / 2) * 64 * 2;  // A tile + this CTA's half of the B tile(s)
   static constexpr int GROUPS_PER_STAGE = STAGE_BYTES / GROUP_BYTES;      // residual boxes one ring stage can carry
   static constexpr int ACC_COLS = NSUB == 2 ? BN : 2 * BNS0;              // two TMEM slots
+  static constexpr int ESUB = LOCK ? 1 : NSUB;                            // units the epilogue sees per tile
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
-  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * 2 * 128 * 8 + (4 * NSTAGES + 6) * 8 + 16 + 1024;
+  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * 2 * 128 * 8 + (4 * NSTAGES + 6 + 64) * 8 + 16 + 1024;
   static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (8 * WARP_BOX_BYTES);
   static constexpr int YBOXES = YBOX_ROOM >= 4 ? 4 : YBOX_ROOM;           // staging boxes per epilogue warp
   static constexpr int YBUF_BYTES = YBOXES * 8 * WARP_BOX_BYTES;
@@ -65,13 +69,14 @@ struct PairCfg {
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
   static constexpr int PRE_BYTES = 2 * 2 * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2;
+  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2 + 64;  // + staging-box full/free, 8 warps x up to 4 boxes each
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
   static_assert(BNS0 > 0 && ACC_COLS <= 512, "accumulators must fit the 512 TMEM columns");
   static_assert(NSTAGES <= 8, "per-stage phase bits are kept in one byte");
-  static_assert(GROUPS_PER_STAGE == 2, "a residual stage carries one even and one odd 64-column group");
+  static_assert(GROUPS_PER_STAGE >= 2, "a residual stage carries one even and one odd 64-column group");
+  static_assert(!LOCK || NSUB == 2, "lock step needs two sub-tiles");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
   static_assert(YBOXES >= 1, "at least one staging box per epilogue warp");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
@@ -94,14 +99,18 @@ struct RingPos {
 // 16-byte chunk `c` (0..7) of row `r` inside a 128-byte-swizzled 128 x 64 bf16 box.
 __device__ __forceinline__ uint32_t swz128(int r, int c) { return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES>
-__global__ void __launch_bounds__(320, 1)
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK>
+__global__ void __launch_bounds__(352, 1)
 fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
-  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES>;
+  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
   constexpr int BN = Cfg::BN;
   constexpr int NSUB = Cfg::NSUB;
-  constexpr int GPS = Cfg::GROUPS_PER_STAGE;
+  constexpr int ESUB = Cfg::ESUB;
+  constexpr int GPS = 2;  // residual boxes per ring stage: one even and one odd group
+  // what the epilogue (and the store warp) see as unit `sub` of a tile: its width and its first local 64-column group
+  auto unit_width = [](int sub) { return LOCK ? BN : (sub ? BNS1 : BNS0); };
+  auto unit_lg0 = [](int sub) { return LOCK ? 0 : (sub ? BNS0 / 64 : 0); };
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -122,6 +131,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto bar_tempty = [&](int a) { return bar_base + 8u * (4 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
   const uint32_t bar_stats = bar_base + 8u * (4 * NSTAGES + 4);
   const uint32_t bar_drain = bar_stats + 8u;
+  auto bar_yfull = [&](int e, int k) { return bar_drain + 8u + 8u * (e * 4 + k); };        // staging box written (epilogue warp e)
+  auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (32 + e * 4 + k); };   // staging box read out by its TMA store
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
 
@@ -153,6 +164,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     mbar_init(bar_stats, CN * 128);
     mbar_init(bar_drain, 1);
+    for (int e = 0; e < 8; ++e)
+      for (int k = 0; k < 4; ++k) {
+        mbar_init(bar_yfull(e, k), 1);
+        mbar_init(bar_yfree(e, k), 1);
+      }
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tensormap(&tmA);
@@ -222,9 +238,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         decode_tile(tile, b, mpair0, ncta0);
         const int m0 = mpair0 + static_cast<int>(pm) * 128;
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;  // first local 64-column group of the sub-tile
+        for (int sub = 0; sub < ESUB; ++sub) {
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);  // first local 64-column group of the unit
           const int n0 = group_col(ncta0, lg0);
           if (!ok || !unit_live(mpair0, n0)) continue;
           const uint32_t bytes = Cfg::A_BYTES + (W / 2) * 128;
@@ -236,8 +252,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
             mbar_arrive_expect_tx_cluster(full, bytes);
             tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
-            for (int j = 0; j < W / 128; ++j)
-              tma_load_3d_pair(sa + Cfg::A_BYTES + j * 8192, &tmB, full, group_col(ncta0, lg0 + static_cast<int>(pm) * (W / 128) + j), kb * 64, b);
+            // this CTA's half of each UMMA's B tile: boxes of 64 columns, 8 KB apart
+            auto load_b_half = [&](uint32_t dst, int first_group, int width) {
+              for (int j = 0; j < width / 128; ++j)
+                tma_load_3d_pair(dst + j * 8192, &tmB, full, group_col(ncta0, first_group + static_cast<int>(pm) * (width / 128) + j),
+                                 kb * 64, b);
+            };
+            if (LOCK) {
+              load_b_half(sa + Cfg::A_BYTES, 0, BNS0);
+              load_b_half(sa + Cfg::A_BYTES + (BNS0 / 2) * 128, BNS0 / 64, BNS1);
+            } else {
+              load_b_half(sa + Cfg::A_BYTES, lg0, W);
+            }
             ring.advance();
           }
           if (ok && has_res) {
@@ -270,18 +296,20 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;  // first local 64-column group of the sub-tile
+        for (int sub = 0; sub < ESUB; ++sub) {
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);  // first local 64-column group of the unit
           const int n0 = group_col(ncta0, lg0);
           if (!ok || !unit_live(mpair0, n0)) continue;
-          const int slot = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
+          const int slot = LOCK ? 0 : (NSUB == 2 ? sub : static_cast<int>(unit_count & 1u));
           ++unit_count;
           if (!mbar_wait<true>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; continue; }
           ++slot_uses[slot];
           tcgen05_fence_after_sync();
           const uint32_t d_tmem = tmem_base + (slot ? BNS0 : 0);
-          const uint32_t idesc = sub ? make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true) : make_idesc_bf16(256, BNS0, false, true);
+          constexpr uint32_t idesc0 = make_idesc_bf16(256, BNS0, false, true);
+          constexpr uint32_t idesc1 = make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true);
+          const uint32_t idesc = (!LOCK && sub) ? idesc1 : idesc0;
           for (int kb = 0; kb < KB; ++kb) {
             if (!mbar_wait<false>(bar_full(ring.stage), (full_bits >> ring.stage) & 1u, w)) { ok = false; break; }
             full_bits ^= 1u << ring.stage;
@@ -289,11 +317,14 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const uint32_t sa = smem_base + ring.stage * Cfg::STAGE_BYTES;
             const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
             const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
+            const uint64_t bdesc1 = make_smem_desc_sw128(sa + Cfg::A_BYTES + (BNS0 / 2) * 128, 8192, 1024);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               // K advances by 16 elements: 32 bytes inside A's swizzled row, 16 K-lines (2048 bytes) in B
-              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
-                                (kb | k) != 0 ? 1u : 0u);
+              const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc, acc);
+              if (LOCK)  // the second sub-tile reuses the A tile that is already in shared memory
+                umma_bf16_ss_pair(d_tmem + BNS0, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc1, acc);
             }
             // the stage is free in both CTAs once these UMMAs have read it
             umma_commit_pair(bar_empty(ring.stage));
@@ -309,6 +340,46 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
       mbar_wait<false>(bar_drain, 0, w);
+    }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------------------------------------ store warp
+    // Lane e mirrors epilogue warp e's sequence of output boxes: wait until the box is staged, store it with TMA, and
+    // hand the staging box back once the store has read it.  D stores stay in flight per lane.
+    if (lane < 8) {
+      const int e = lane;
+      const int q = (e + 2) & 3;
+      const int h = e >> 2;
+      constexpr int D = Cfg::YBOXES - 1;
+      const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + e * Cfg::YBOXES * Cfg::WARP_BOX_BYTES;
+      uint32_t n = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
+        int b, mpair0, ncta0;
+        decode_tile(tile, b, mpair0, ncta0);
+        const int m0 = mpair0 + static_cast<int>(pm) * 128;
+        for (int sub = 0; sub < ESUB && ok; ++sub) {
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);
+          if (EPI == EPI_NONE && !unit_live(mpair0, group_col(ncta0, lg0))) continue;
+          for (int g = h; g < W / 64; g += 2) {
+            const int col = group_col(ncta0, lg0 + g);
+            if (EPI == EPI_NONE && col >= p.N) break;
+            const uint32_t sel = n % Cfg::YBOXES;
+            if (!mbar_wait<false>(bar_yfull(e, sel), (n / Cfg::YBOXES) & 1u, w)) { ok = false; break; }
+#ifdef COMFUSE_TRACE
+            if (!(p.trace_flags & 1))
+#endif
+            tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, m0 + q * 32, b);
+            tma_store_commit();
+            if (n >= static_cast<uint32_t>(D)) {
+              tma_store_wait_read<D>();
+              mbar_arrive(bar_yfree(e, (n - D) % Cfg::YBOXES));
+            }
+            ++n;
+          }
+        }
+      }
+      tma_store_wait_all();  // the staging boxes must outlive the last stores' reads
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
@@ -330,10 +401,23 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     // Stage this thread's 64 packed columns (its row of the warp's 32 x 64 box) and store the box with TMA.
     // pk[0..15] are columns 0..31 of the group, pk[16..31] columns 32..63.
-    auto store_box = [&](const uint32_t (&pk)[32], int col0, int m0, int b) {
-      const uint32_t ybox = ybox0 + ybox_sel * Cfg::WARP_BOX_BYTES;
+    uint32_t ybox_count = 0;
+#ifdef COMFUSE_TRACE
+    int trace_ix = 0;
+#define COMFUSE_TRACE_POINT()                                                                          \
+  do {                                                                                                 \
+    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 64) p.trace[trace_ix++] = globaltimer_ns(); \
+  } while (0)
+#else
+#define COMFUSE_TRACE_POINT() do { } while (0)
+#endif
+    auto store_box = [&](const uint32_t (&pk)[32]) {
+      const uint32_t sel = ybox_sel;
+      const uint32_t ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
       if (++ybox_sel == Cfg::YBOXES) ybox_sel = 0;
-      if (lane == 0) tma_store_wait_read<Cfg::YBOXES - 1>();  // the last store that used this box has read it out
+      // the store of the box's previous contents has read it out
+      mbar_wait<false>(bar_yfree(warp - 2, sel), ((ybox_count / Cfg::YBOXES) & 1u) ^ 1u, w);
+      ++ybox_count;
       __syncwarp();
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -344,10 +428,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        tma_store_3d(&tmY, ybox, col0, m0 + q * 32, b);
-        tma_store_commit();
-      }
+      if (lane == 0) mbar_arrive(bar_yfull(warp - 2, sel));
     };
     // This thread's 64 residual values of box `gg` of a residual stage, as 32 packed bf16 pairs.
     auto load_residual = [&](uint32_t stage_addr, int gg, uint32_t (&r32)[32]) {
@@ -361,6 +442,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     };
 
     for (int tile = cluster_id; tile < p.total_tiles; tile += num_clusters) {
+      COMFUSE_TRACE_POINT();
       int b, mpair0, ncta0;
       decode_tile(tile, b, mpair0, ncta0);
       const int m0 = mpair0 + static_cast<int>(pm) * 128;
@@ -368,12 +450,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const bool valid = grow < p.M;
 
       // the slot of each sub-tile of this tile, and whether it is computed at all
-      bool live[NSUB];
-      int slot[NSUB];
+      bool live[ESUB];
+      int slot[ESUB];
 #pragma unroll
-      for (int sub = 0; sub < NSUB; ++sub) {
-        live[sub] = unit_live(mpair0, group_col(ncta0, sub ? BNS0 / 64 : 0));
-        slot[sub] = NSUB == 2 ? sub : static_cast<int>(unit_count & 1u);
+      for (int sub = 0; sub < ESUB; ++sub) {
+        live[sub] = unit_live(mpair0, group_col(ncta0, unit_lg0(sub)));
+        slot[sub] = LOCK ? 0 : (NSUB == 2 ? sub : static_cast<int>(unit_count & 1u));
         if (live[sub]) ++unit_count;
       }
       auto wait_accumulator = [&](int sub) {
@@ -395,11 +477,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
       if constexpr (EPI == EPI_NONE) {
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
+        for (int sub = 0; sub < ESUB; ++sub) {
           if (!live[sub]) continue;
           wait_accumulator(sub);
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);
           for (int g = h; g < W / 64; g += 2) {
             if (group_col(ncta0, lg0 + g) >= p.N) break;
             uint32_t pk[32];
@@ -411,7 +493,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               for (int j = 0; j < 16; ++j)
                 pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
             }
-            store_box(pk, group_col(ncta0, lg0 + g), m0, b);
+            store_box(pk);
           }
           release_accumulator(sub);
         }
@@ -420,11 +502,13 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // back over the accumulator in TMEM (the bypass path of Sec. 3.2)
         float2 part = make_float2(0.f, 0.f);
         float n_run = 0.f;
+        COMFUSE_TRACE_POINT();
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
+        for (int sub = 0; sub < ESUB; ++sub) {
           wait_accumulator(sub);
-          const int W = sub ? BNS1 : BNS0;
-          const int lsub = sub ? BNS0 : 0;  // first column of the sub-tile inside the CTA's column range
+          COMFUSE_TRACE_POINT();
+          const int W = unit_width(sub);
+          const int lsub = unit_lg0(sub) * 64;  // first column of the unit inside the CTA's column range
           const uint32_t taddr = tmem_of(sub);
           for (int g = h; g < W / 64; g += 2) {
             // groups (g - h, g - h + 1) share one residual stage; this warp reads box h of it
@@ -493,6 +577,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
         tmem_st_wait();
+        COMFUSE_TRACE_POINT();
         // ---------------- stage 1 (reduce): thread pair, then the CTAs that share these rows
         float2 tot;
         if constexpr (EPI == EPI_LN) {
@@ -502,6 +587,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tot = cluster_row_reduce<CN>(part, kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u,
                                        pm);
         }
+        COMFUSE_TRACE_POINT();
         const float mu = EPI == EPI_LN ? tot.x : 0.f;
         const float sq = EPI == EPI_LN ? tot.y : tot.x;
         const float rstd = rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
@@ -509,9 +595,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         float best = -INFINITY;
         int best_col = 0x7FFFFFFF;
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-          const int W = sub ? BNS1 : BNS0;
-          const int lsub = sub ? BNS0 : 0;
+        for (int sub = 0; sub < ESUB; ++sub) {
+          const int W = unit_width(sub);
+          const int lsub = unit_lg0(sub) * 64;
           const uint32_t taddr = tmem_of(sub);
           for (int g = h; g < W / 64; g += 2) {
             uint32_t pk[32];
@@ -547,7 +633,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 pk[half * 16 + 2 * j + 1] = pack_bf16x2_rn(y2, y3);
               }
             }
-            store_box(pk, ncta0 + lsub + g * 64, m0, b);
+            store_box(pk);
           }
           release_accumulator(sub);
         }
@@ -568,14 +654,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // loads stay convergent: 2 = all live, 1 = crosses the diagonal, 0 = all masked
         const int wrow0 = m0 + q * 32;
         auto frag_state = [&](int col0) { return !p.causal ? 2 : (col0 + 31 <= wrow0 ? 2 : (col0 > wrow0 + 31 ? 0 : 1)); };
+        COMFUSE_TRACE_POINT();
         // ---------------- pass A: thread-local row max
         float mloc = -INFINITY;
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
+        for (int sub = 0; sub < ESUB; ++sub) {
           wait_accumulator(sub);
           if (!live[sub]) continue;
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);
           for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -595,14 +682,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         }
+        COMFUSE_TRACE_POINT();
         // ---------------- pass B: e = 2^(t - mloc), thread-local sum, e written back over the scores
         float lloc = 0.f;
         const float msub = (mloc == -INFINITY) ? 0.f : mloc;
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
+        for (int sub = 0; sub < ESUB; ++sub) {
           if (!live[sub]) continue;
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);
           for (int g = h; g < W / 64; g += 2) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -631,14 +719,16 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
         tmem_st_wait();
+        COMFUSE_TRACE_POINT();
         const float2 tot = cluster_row_reduce<CN>(make_float2(mloc, lloc), kThreadCount, MergeMaxSumExp2(), s_pre, s_stats,
                                                   bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
         const float f = (mloc == -INFINITY || tot.y == 0.f) ? 0.f : ex2_approx(mloc - tot.x) / tot.y;
+        COMFUSE_TRACE_POINT();
         // ---------------- pass C: scale, round once, store (zeros where masked)
 #pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-          const int W = sub ? BNS1 : BNS0;
-          const int lg0 = sub ? BNS0 / 64 : 0;
+        for (int sub = 0; sub < ESUB; ++sub) {
+          const int W = unit_width(sub);
+          const int lg0 = unit_lg0(sub);
           for (int g = h; g < W / 64; g += 2) {
             uint32_t pk[32];
 #pragma unroll
@@ -656,13 +746,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
               }
             }
-            store_box(pk, group_col(ncta0, lg0 + g), m0, b);
+            store_box(pk);
           }
           release_accumulator(sub);
         }
       }
     }
-    if (lane == 0) tma_store_wait_all();  // the staging buffer must outlive the last store's read
   }
 
   // -------------------------------------------------------------------------------------------- teardown

@@ -26,6 +26,8 @@ struct FusedParams {
   int* row_argmax;
   unsigned int* status;
   unsigned long long timeout_ns;
+  unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null
+  int trace_flags;            // tracing builds: bit 0 = skip the output stores, bit 1 = skip the UMMAs
 };
 
 }  // namespace comfuse

@@ -5,16 +5,17 @@
 namespace comfuse {
 
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
-#define COMFUSE_CASE(n, b0, b1, cn, nst) \
-  case n:                                \
-    return supported_only ? cudaSuccess : launch_pair_instance<EPI_RMS_MAX, b0, b1, cn, nst>(maps, p, st);
+#define COMFUSE_CASE(n, b0, b1, cn, nst, lock) \
+  case n:                                      \
+    return supported_only ? cudaSuccess : launch_pair_instance<EPI_RMS_MAX, b0, b1, cn, nst, lock>(maps, p, st);
+  // Two sub-tiles advance in lock step (lock = 1): the A tile is fetched once per K block for both.
   switch (p.N) {
-    COMFUSE_CASE(256, 256, 0, 1, 5)
-    COMFUSE_CASE(512, 256, 256, 1, 5)
-    COMFUSE_CASE(768, 256, 128, 2, 5)
-    COMFUSE_CASE(1024, 256, 256, 2, 5)
-    COMFUSE_CASE(2048, 256, 256, 4, 5)
-    COMFUSE_CASE(4096, 256, 256, 8, 5)
+    COMFUSE_CASE(256, 256, 0, 1, 5, 0)
+    COMFUSE_CASE(512, 256, 256, 1, 3, 1)
+    COMFUSE_CASE(768, 256, 128, 2, 4, 1)
+    COMFUSE_CASE(1024, 256, 256, 2, 3, 1)
+    COMFUSE_CASE(2048, 256, 256, 4, 3, 1)
+    COMFUSE_CASE(4096, 256, 256, 8, 3, 1)
     default:
       return cudaErrorInvalidValue;
   }
