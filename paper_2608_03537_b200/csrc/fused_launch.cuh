@@ -2,6 +2,9 @@
 // non-portable size when above 8), persistent grid sized from the number of clusters the device can hold at once.
 #pragma once
 
+#include <cstdio>
+#include <cstdlib>
+
 #include "fused_pair.cuh"
 #include "host_common.h"
 
@@ -48,6 +51,9 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di] = n;
+    if (std::getenv("COMFUSE_VERBOSE"))
+      std::fprintf(stderr, "comfuse: kernel epi=%d bns=%d+%d cn=%d stages=%d lock=%d: cluster of %d CTAs, %d clusters fit, %d B smem, %d staging boxes/warp\n",
+                   EPI, BNS0, BNS1, CN, NSTAGES, LOCK, kCluster, n, Cfg::SMEM_BYTES, Cfg::YBOXES);
   }
   const int clusters = p.total_tiles < max_clusters[di] ? p.total_tiles : max_clusters[di];
   if (clusters <= 0) return cudaSuccess;

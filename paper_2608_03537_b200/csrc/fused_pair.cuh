@@ -634,6 +634,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               }
             }
             store_box(pk);
+            COMFUSE_TRACE_POINT();
           }
           release_accumulator(sub);
         }
