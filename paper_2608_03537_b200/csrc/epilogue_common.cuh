@@ -35,21 +35,22 @@ struct MergeArgmax {  // (value, column index bits); ties -> lower index
 };
 
 // The reduce phase above thread level.  All 256 epilogue threads of every CTA that shares the rows call this the
-// same number of times.  `per_thread_count` = elements behind each thread's partial (half of the CTA's columns).
+// same number of times.  `per_thread_count` = elements behind each thread's partial (1/NH of the CTA's columns).
 // `rank` is this CTA's index among the CN column ranges; the cluster rank of column range c is
 // c * rank_stride + rank_offset (CTA pairs interleave two row blocks in one cluster).
-template <int CN, class Merge>
+template <int CN, class Merge, int NH = 2>
 __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thread_count, Merge merge, float2* s_pre,
                                                      float2* s_stats, uint32_t stats_bar, int row, int h,
                                                      uint32_t rank, int& xpar, uint32_t& xphase, const WaitCtx& w,
                                                      uint32_t rank_stride = 1, uint32_t rank_offset = 0) {
-  // level 2: the two column-halves of the row, through shared memory
-  s_pre[(xpar * 2 + h) * 128 + row] = mine;
-  named_barrier_sync(1, 256);
-  const float2 cta_partial = merge(s_pre[(xpar * 2 + 0) * 128 + row], per_thread_count,
-                                   s_pre[(xpar * 2 + 1) * 128 + row], per_thread_count);
-  const float cta_count = 2.f * per_thread_count;
-  // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks of parity h
+  // level 2: the NH threads that share the row (one per epilogue warp of the lane quarter), through shared memory
+  s_pre[(xpar * NH + h) * 128 + row] = mine;
+  named_barrier_sync(1, 128 * NH);
+  float2 cta_partial = s_pre[(xpar * NH + 0) * 128 + row];
+#pragma unroll
+  for (int t = 1; t < NH; ++t) cta_partial = merge(cta_partial, per_thread_count * t, s_pre[(xpar * NH + t) * 128 + row], per_thread_count);
+  const float cta_count = static_cast<float>(NH) * per_thread_count;
+  // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks congruent to h mod NH
   float2* slot = s_stats + (xpar * CN + rank) * 128 + row;
   if constexpr (CN == 1) {
     if (h == 0) {
@@ -60,7 +61,7 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
     const uint32_t slot_addr = smem_u32(slot);
 #pragma unroll
     for (int dst = 0; dst < CN; ++dst) {
-      if ((dst & 1) == h) {
+      if ((dst % NH) == h) {
         const uint32_t peer = dst * rank_stride + rank_offset;
         st_cluster_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y);
         mbar_arrive_cluster(map_to_cta(stats_bar, peer));

@@ -11,10 +11,10 @@
 namespace comfuse {
 
 // One work item = a pair of adjacent 128-row blocks (times p.nblocks column blocks of CN*BN columns).
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0>
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0, int EPW = 2>
 cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream_t stream) {
-  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
-  auto kern = fused_pair_kernel<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
+  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW>;
+  auto kern = fused_pair_kernel<EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW>;
   const DeviceInfo* dev = current_device_info();
   if (!dev) return cudaErrorInvalidDevice;
   constexpr int kCluster = 2 * CN;
@@ -52,8 +52,8 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di] = n;
     if (std::getenv("COMFUSE_VERBOSE"))
-      std::fprintf(stderr, "comfuse: kernel epi=%d bns=%d+%d cn=%d stages=%d lock=%d: cluster of %d CTAs, %d clusters fit, %d B smem, %d staging boxes/warp\n",
-                   EPI, BNS0, BNS1, CN, NSTAGES, LOCK, kCluster, n, Cfg::SMEM_BYTES, Cfg::YBOXES);
+      std::fprintf(stderr, "comfuse: kernel epi=%d bns=%d+%d cn=%d stages=%d lock=%d epw=%d: cluster of %d CTAs, %d clusters fit, %d B smem, %d staging boxes/warp\n",
+                   EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW, kCluster, n, Cfg::SMEM_BYTES, Cfg::YBOXES);
   }
   const int clusters = p.total_tiles < max_clusters[di] ? p.total_tiles : max_clusters[di];
   if (clusters <= 0) return cudaSuccess;

@@ -37,10 +37,13 @@
 
 namespace comfuse {
 
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0>
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK = 0, int EPW = 2>
 struct PairCfg {
-  static constexpr int kThreads = 352;  // producer, UMMA, 8 epilogue warps, store warp
-  static constexpr int kEpiThreads = 256;
+  // EPW epilogue warps per TMEM lane quarter (2 or 4): they take the 64-column groups g with g % EPW == their index
+  static constexpr int kEpiWarps = 4 * EPW;
+  static constexpr int kEpiThreads = 32 * kEpiWarps;
+  static constexpr int kStoreWarp = 2 + kEpiWarps;
+  static constexpr int kThreads = 32 * (kStoreWarp + 1);  // producer, UMMA, epilogue warps, store warp
   static constexpr int NSUB = BNS1 > 0 ? 2 : 1;
   static constexpr int BN = BNS0 + BNS1;
   static constexpr int BNSMAX = BNS0 > BNS1 ? BNS0 : BNS1;
@@ -55,10 +58,10 @@ struct PairCfg {
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
-  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * 2 * 128 * 8 + (4 * NSTAGES + 6 + 64) * 8 + 16 + 1024;
-  static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (8 * WARP_BOX_BYTES);
+  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * EPW * 128 * 8 + (4 * NSTAGES + 6 + 128) * 8 + 16 + 1024;
+  static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (kEpiWarps * WARP_BOX_BYTES);
   static constexpr int YBOXES = YBOX_ROOM >= 4 ? 4 : YBOX_ROOM;           // staging boxes per epilogue warp
-  static constexpr int YBUF_BYTES = YBOXES * 8 * WARP_BOX_BYTES;
+  static constexpr int YBUF_BYTES = YBOXES * kEpiWarps * WARP_BOX_BYTES;
   // Softmax only: the CTA's 64-column groups are interleaved with its peers' (group g of column range c is global
   // group g*CN + c), so that a causal mask leaves every CTA of the reduction group the same share of live columns.
   static constexpr bool INTERLEAVE = EPI == EPI_SOFTMAX;
@@ -67,9 +70,9 @@ struct PairCfg {
   static constexpr int OFF_STATS = OFF_VEC + VEC_BYTES;
   static constexpr int STATS_BYTES = 2 * CN * 128 * 8;
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
-  static constexpr int PRE_BYTES = 2 * 2 * 128 * 8;
+  static constexpr int PRE_BYTES = 2 * EPW * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2 + 64;  // + staging-box full/free, 8 warps x up to 4 boxes each
+  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2 + 128;  // + staging-box full/free, up to 16 warps x 4 boxes each
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
@@ -77,6 +80,9 @@ struct PairCfg {
   static_assert(NSTAGES <= 8, "per-stage phase bits are kept in one byte");
   static_assert(GROUPS_PER_STAGE >= 2, "a residual stage carries one even and one odd 64-column group");
   static_assert(!LOCK || NSUB == 2, "lock step needs two sub-tiles");
+  static_assert(EPW == 2 || EPW == 4, "two or four epilogue warps per lane quarter");
+  static_assert((BNS0 / 64) % EPW == 0 && (BNS1 / 64) % EPW == 0, "every epilogue warp gets the same number of groups");
+  static_assert(EPW == 2 || EPI == EPI_SOFTMAX || EPI == EPI_NONE, "residual stages carry one group per warp pair");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
   static_assert(YBOXES >= 1, "at least one staging box per epilogue warp");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
@@ -99,11 +105,11 @@ struct RingPos {
 // 16-byte chunk `c` (0..7) of row `r` inside a 128-byte-swizzled 128 x 64 bf16 box.
 __device__ __forceinline__ uint32_t swz128(int r, int c) { return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK>
-__global__ void __launch_bounds__(352, 1)
+template <int EPI, int BNS0, int BNS1, int CN, int NSTAGES, int LOCK, int EPW>
+__global__ void __launch_bounds__(32 * (3 + 4 * EPW), 1)
 fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
-  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK>;
+  using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW>;
   constexpr int BN = Cfg::BN;
   constexpr int NSUB = Cfg::NSUB;
   constexpr int ESUB = Cfg::ESUB;
@@ -132,7 +138,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const uint32_t bar_stats = bar_base + 8u * (4 * NSTAGES + 4);
   const uint32_t bar_drain = bar_stats + 8u;
   auto bar_yfull = [&](int e, int k) { return bar_drain + 8u + 8u * (e * 4 + k); };        // staging box written (epilogue warp e)
-  auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (32 + e * 4 + k); };   // staging box read out by its TMA store
+  auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (64 + e * 4 + k); };   // staging box read out by its TMA store
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
 
@@ -164,7 +170,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     mbar_init(bar_stats, CN * 128);
     mbar_init(bar_drain, 1);
-    for (int e = 0; e < 8; ++e)
+    for (int e = 0; e < Cfg::kEpiWarps; ++e)
       for (int k = 0; k < 4; ++k) {
         mbar_init(bar_yfull(e, k), 1);
         mbar_init(bar_yfree(e, k), 1);
@@ -341,11 +347,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
       mbar_wait<false>(bar_drain, 0, w);
     }
-  } else if (warp == 10) {
+  } else if (warp == Cfg::kStoreWarp) {
     // ------------------------------------------------------------------------------------------ store warp
     // Lane e mirrors epilogue warp e's sequence of output boxes: wait until the box is staged, store it with TMA, and
     // hand the staging box back once the store has read it.  D stores stay in flight per lane.
-    if (lane < 8) {
+    if (lane < Cfg::kEpiWarps) {
       const int e = lane;
       const int q = (e + 2) & 3;
       const int h = e >> 2;
@@ -361,7 +367,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
           if (EPI == EPI_NONE && !unit_live(mpair0, group_col(ncta0, lg0))) continue;
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
             const int col = group_col(ncta0, lg0 + g);
             if (EPI == EPI_NONE && col >= p.N) break;
             const uint32_t sel = n % Cfg::YBOXES;
@@ -384,7 +390,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;         // TMEM lane quarter this warp may touch: rows 32q .. 32q+31 of the tile
-    const int h = (warp - 2) >> 2;  // this warp takes the 64-column groups of parity h
+    const int h = (warp - 2) >> 2;  // this warp takes the 64-column groups g with g % EPW == h
     const int row = q * 32 + lane;
     const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
     int xpar = 0;
@@ -394,7 +400,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     uint32_t rfull_bits = 0;
     uint32_t slot_uses[2] = {0, 0};
     uint32_t unit_count = 0;
-    constexpr float kThreadCount = static_cast<float>(BN / 2);  // columns behind one thread's partial
+    constexpr float kThreadCount = static_cast<float>(BN / EPW);  // columns behind one thread's partial
     const uint32_t tempty_leader = map_to_cta(bar_tempty(0), leader);
     const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + (warp - 2) * Cfg::YBOXES * Cfg::WARP_BOX_BYTES;  // this warp's staging boxes
     uint32_t ybox_sel = 0;
@@ -482,7 +488,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           wait_accumulator(sub);
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
             if (group_col(ncta0, lg0 + g) >= p.N) break;
             uint32_t pk[32];
 #pragma unroll
@@ -510,7 +516,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = unit_width(sub);
           const int lsub = unit_lg0(sub) * 64;  // first column of the unit inside the CTA's column range
           const uint32_t taddr = tmem_of(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
             // groups (g - h, g - h + 1) share one residual stage; this warp reads box h of it
             uint32_t r32[32];
             if (has_res) {
@@ -581,10 +587,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // ---------------- stage 1 (reduce): thread pair, then the CTAs that share these rows
         float2 tot;
         if constexpr (EPI == EPI_LN) {
-          tot = cluster_row_reduce<CN>(part, kThreadCount, MergeWelford(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w,
+          tot = cluster_row_reduce<CN, MergeWelford, EPW>(part, kThreadCount, MergeWelford(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w,
                                        2u, pm);
         } else {
-          tot = cluster_row_reduce<CN>(part, kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u,
+          tot = cluster_row_reduce<CN, MergeSum, EPW>(part, kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u,
                                        pm);
         }
         COMFUSE_TRACE_POINT();
@@ -599,7 +605,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = unit_width(sub);
           const int lsub = unit_lg0(sub) * 64;
           const uint32_t taddr = tmem_of(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
             uint32_t pk[32];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -640,7 +646,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         if constexpr (EPI == EPI_RMS_MAX) {
           // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
-          const float2 mx = cluster_row_reduce<CN>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
+          const float2 mx = cluster_row_reduce<CN, MergeArgmax, EPW>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
                                                    s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
           if (crank == 0 && h == 0 && valid) {
             const long long o = static_cast<long long>(b) * p.M + grow;
@@ -664,7 +670,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!live[sub]) continue;
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               const int col0 = group_col(ncta0, lg0 + g) + half * 32;
@@ -692,7 +698,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!live[sub]) continue;
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               const int col0 = group_col(ncta0, lg0 + g) + half * 32;
@@ -721,7 +727,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         tmem_st_wait();
         COMFUSE_TRACE_POINT();
-        const float2 tot = cluster_row_reduce<CN>(make_float2(mloc, lloc), kThreadCount, MergeMaxSumExp2(), s_pre, s_stats,
+        const float2 tot = cluster_row_reduce<CN, MergeMaxSumExp2, EPW>(make_float2(mloc, lloc), kThreadCount, MergeMaxSumExp2(), s_pre, s_stats,
                                                   bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
         const float f = (mloc == -INFINITY || tot.y == 0.f) ? 0.f : ex2_approx(mloc - tot.x) / tot.y;
         COMFUSE_TRACE_POINT();
@@ -730,7 +736,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int sub = 0; sub < ESUB; ++sub) {
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
-          for (int g = h; g < W / 64; g += 2) {
+          for (int g = h; g < W / 64; g += EPW) {
             uint32_t pk[32];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {

@@ -5,15 +5,16 @@
 namespace comfuse {
 
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
-#define COMFUSE_CASE(n, b0, b1, cn, nst) \
-  case n:                                \
-    return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst>(maps, p, st);
+#define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
+  case n:                                     \
+    return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, 0, epw>(maps, p, st);
+  // The softmax passes are latency-bound on few warps and need few registers: four epilogue warps per lane quarter.
   switch (p.N) {
-    COMFUSE_CASE(256, 256, 0, 1, 3)
-    COMFUSE_CASE(512, 256, 256, 1, 3)
-    COMFUSE_CASE(1024, 256, 256, 2, 3)
-    COMFUSE_CASE(2048, 256, 256, 4, 3)
-    COMFUSE_CASE(4096, 256, 256, 8, 3)
+    COMFUSE_CASE(256, 256, 0, 1, 3, 4)
+    COMFUSE_CASE(512, 256, 256, 1, 2, 4)
+    COMFUSE_CASE(1024, 256, 256, 2, 2, 4)
+    COMFUSE_CASE(2048, 256, 256, 4, 2, 4)
+    COMFUSE_CASE(4096, 256, 256, 8, 2, 4)
     default:
       return cudaErrorInvalidValue;
   }
