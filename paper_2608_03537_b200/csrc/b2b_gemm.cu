@@ -272,8 +272,18 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     uint32_t tile_it = 0;
     int xpar = 0;
     uint32_t xphase = 0;
+#ifdef COMFUSE_TRACE
+    int trace_ix = 0;
+#define B2B_TRACE_POINT()                                                                                \
+  do {                                                                                                   \
+    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 64) p.trace[trace_ix++] = globaltimer_ns(); \
+  } while (0)
+#else
+#define B2B_TRACE_POINT() do { } while (0)
+#endif
 
     for (int tile = cluster_id; tile < p.mpairs; tile += num_clusters, ++tile_it) {
+      B2B_TRACE_POINT();
       const int m0 = tile * 256 + static_cast<int>(pm) * 128;
       const int obuf = tile_it & 1u;
       // ---------------- Epi1(j): S_j = bf16(GELU(P_j + b1)) as the next UMMA's A operand
@@ -283,6 +293,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ++puses[pb];
         __syncwarp();
         tcgen05_fence_after_sync();
+        B2B_TRACE_POINT();
         // the S buffer is free once ML2 of chunk j-2 has read it
         mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
         ++suses[pb];
@@ -296,12 +307,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float4 bb = b4[i];
-            const float g0 = gelu_tanh_f32(__uint_as_float(v[4 * i]) + bb.x);
-            const float g1 = gelu_tanh_f32(__uint_as_float(v[4 * i + 1]) + bb.y);
-            const float g2 = gelu_tanh_f32(__uint_as_float(v[4 * i + 2]) + bb.z);
-            const float g3 = gelu_tanh_f32(__uint_as_float(v[4 * i + 3]) + bb.w);
-            pk[2 * i] = pack_bf16x2_rn(g0, g1);
-            pk[2 * i + 1] = pack_bf16x2_rn(g2, g3);
+            const float2 g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
+            const float2 g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
+            pk[2 * i] = pack_bf16x2_rn(g01);
+            pk[2 * i + 1] = pack_bf16x2_rn(g23);
           }
           // this thread's 32 columns are 16-byte chunks half*4 .. half*4+3 of K block h of the S buffer
           const uint32_t sb = s_addr(pb, h);
@@ -316,12 +325,14 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
         fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
         mbar_arrive_cluster(sfull_leader + 8u * pb);
+        B2B_TRACE_POINT();
       }
       ring.skip(2 + 2 * NC);  // X, W1 and W2 slots were the tensor pipe's
       // ---------------- Epi2: O' = O + b2 + X, LayerNorm over the 128 columns, store
       mbar_wait<false>(bar_ofull(obuf), (tile_it >> 1) & 1u, w);
       __syncwarp();
       tcgen05_fence_after_sync();
+      B2B_TRACE_POINT();
       const int rstage = ring.stage + h >= kRingSlots ? ring.stage + h - kRingSlots : ring.stage + h;
       // both residual slots are waited for by everybody (the phase bits must advance uniformly)
       uint32_t r32[2][16];
@@ -387,6 +398,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       mbar_arrive_cluster(oempty_leader + 8u * obuf);
       // reduce: the row lives in this CTA only (two half-row threads)
       const float2 tot = cluster_row_reduce<1>(part, 64.f, MergeWelford(), s_pre, s_stats, bar_stats, row, h, 0u, xpar, xphase, w);
+      B2B_TRACE_POINT();
       const float mu = tot.x;
       const float rstd = rsqrtf(tot.y * (1.f / 128.f) + p.eps);
       // stage 2: normalise, round once, stage one 128 x 64 box per half-row group and store it

@@ -18,6 +18,7 @@ struct B2bParams {
   uint16_t* O;
   unsigned int* status;
   unsigned long long timeout_ns;
+  unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null
 };
 
 bool b2b_fused_supported(int K, int N1, int N2);

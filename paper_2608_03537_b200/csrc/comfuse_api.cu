@@ -355,6 +355,9 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     bp.O = static_cast<uint16_t*>(O);
     bp.status = dev->status_word;
     bp.timeout_ns = timeout_ns();
+#ifdef COMFUSE_TRACE
+    if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) bp.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));
+#endif
     cudaError_t e = launch_b2b_fused(X, W1, W2, bp, st);
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }

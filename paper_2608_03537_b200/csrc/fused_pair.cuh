@@ -538,44 +538,50 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tmem_ld_32cols(taddr + g * 64 + half * 32, v);
               const float4* bias4 = reinterpret_cast<const float4*>(s_bias + lc);
               if constexpr (EPI == EPI_LN) {
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                float2 s01 = splat2(0.f), s23 = splat2(0.f);
+                const float2 al = splat2(p.alpha);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 bb = bias4[j];
-                  const uint32_t ra = r32[half * 16 + 2 * j], rb = r32[half * 16 + 2 * j + 1];
-                  const float x0 = fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x) + bf16_lo(ra);
-                  const float x1 = fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y) + bf16_hi(ra);
-                  const float x2 = fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z) + bf16_lo(rb);
-                  const float x3 = fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w) + bf16_hi(rb);
-                  v[4 * j] = __float_as_uint(x0); v[4 * j + 1] = __float_as_uint(x1);
-                  v[4 * j + 2] = __float_as_uint(x2); v[4 * j + 3] = __float_as_uint(x3);
-                  s0 += x0; s1 += x1; s2 += x2; s3 += x3;
+                  const float2 x01 = add2(fma2(al, f2_from_bits(v[4 * j], v[4 * j + 1]), make_float2(bb.x, bb.y)),
+                                          bf16x2_to_f2(r32[half * 16 + 2 * j]));
+                  const float2 x23 = add2(fma2(al, f2_from_bits(v[4 * j + 2], v[4 * j + 3]), make_float2(bb.z, bb.w)),
+                                          bf16x2_to_f2(r32[half * 16 + 2 * j + 1]));
+                  v[4 * j] = __float_as_uint(x01.x); v[4 * j + 1] = __float_as_uint(x01.y);
+                  v[4 * j + 2] = __float_as_uint(x23.x); v[4 * j + 3] = __float_as_uint(x23.y);
+                  s01 = add2(s01, x01);
+                  s23 = add2(s23, x23);
                 }
-                const float cmean = ((s0 + s1) + (s2 + s3)) * (1.f / 32.f);
-                float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+                const float cmean = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32.f);
+                const float2 nm = splat2(-cmean);
+                float2 q01 = splat2(0.f), q23 = splat2(0.f);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                  const float d0 = __uint_as_float(v[4 * j]) - cmean, d1 = __uint_as_float(v[4 * j + 1]) - cmean;
-                  const float d2 = __uint_as_float(v[4 * j + 2]) - cmean, d3 = __uint_as_float(v[4 * j + 3]) - cmean;
-                  q0 = fmaf(d0, d0, q0); q1 = fmaf(d1, d1, q1); q2 = fmaf(d2, d2, q2); q3 = fmaf(d3, d3, q3);
+                  const float2 d01 = add2(f2_from_bits(v[4 * j], v[4 * j + 1]), nm);
+                  const float2 d23 = add2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), nm);
+                  q01 = fma2(d01, d01, q01);
+                  q23 = fma2(d23, d23, q23);
                 }
+                const float q0 = q01.x, q1 = q01.y, q2 = q23.x, q3 = q23.y;
                 const float2 cpart = make_float2(cmean, (q0 + q1) + (q2 + q3));
                 part = (n_run == 0.f) ? cpart : MergeWelford()(part, n_run, cpart, 32.f);
                 n_run += 32.f;
               } else {
-                float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+                float2 q01 = splat2(0.f), q23 = splat2(0.f);
+                const float2 al = splat2(p.alpha);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 bb = bias4[j];
-                  const uint32_t ra = r32[half * 16 + 2 * j], rb = r32[half * 16 + 2 * j + 1];
-                  const float h0 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j]), bb.x)) + bf16_lo(ra);
-                  const float h1 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 1]), bb.y)) + bf16_hi(ra);
-                  const float h2 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 2]), bb.z)) + bf16_lo(rb);
-                  const float h3 = gelu_tanh_f32(fmaf(p.alpha, __uint_as_float(v[4 * j + 3]), bb.w)) + bf16_hi(rb);
-                  v[4 * j] = __float_as_uint(h0); v[4 * j + 1] = __float_as_uint(h1);
-                  v[4 * j + 2] = __float_as_uint(h2); v[4 * j + 3] = __float_as_uint(h3);
-                  q0 = fmaf(h0, h0, q0); q1 = fmaf(h1, h1, q1); q2 = fmaf(h2, h2, q2); q3 = fmaf(h3, h3, q3);
+                  const float2 h01 = add2(gelu_tanh_f32x2(fma2(al, f2_from_bits(v[4 * j], v[4 * j + 1]), make_float2(bb.x, bb.y))),
+                                          bf16x2_to_f2(r32[half * 16 + 2 * j]));
+                  const float2 h23 = add2(gelu_tanh_f32x2(fma2(al, f2_from_bits(v[4 * j + 2], v[4 * j + 3]), make_float2(bb.z, bb.w))),
+                                          bf16x2_to_f2(r32[half * 16 + 2 * j + 1]));
+                  v[4 * j] = __float_as_uint(h01.x); v[4 * j + 1] = __float_as_uint(h01.y);
+                  v[4 * j + 2] = __float_as_uint(h23.x); v[4 * j + 3] = __float_as_uint(h23.y);
+                  q01 = fma2(h01, h01, q01);
+                  q23 = fma2(h23, h23, q23);
                 }
+                const float q0 = q01.x, q1 = q01.y, q2 = q23.x, q3 = q23.y;
                 part.x += (q0 + q1) + (q2 + q3);
               }
               tmem_st_32cols(taddr + g * 64 + half * 32, v);
@@ -619,16 +625,17 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const float4 gg = g4[j];
                 float y0, y1, y2, y3;
                 if constexpr (EPI == EPI_LN) {
+                  // y = (x - mu) * rstd * gamma + beta as two packed FMAs: n = x * rstd + (-mu * rstd), y = n * gamma + beta
                   const float4 be = b4[j];
-                  y0 = fmaf((__uint_as_float(v[4 * j]) - mu) * rstd, gg.x, be.x);
-                  y1 = fmaf((__uint_as_float(v[4 * j + 1]) - mu) * rstd, gg.y, be.y);
-                  y2 = fmaf((__uint_as_float(v[4 * j + 2]) - mu) * rstd, gg.z, be.z);
-                  y3 = fmaf((__uint_as_float(v[4 * j + 3]) - mu) * rstd, gg.w, be.w);
+                  const float2 n01 = fma2(f2_from_bits(v[4 * j], v[4 * j + 1]), splat2(rstd), splat2(-mu * rstd));
+                  const float2 n23 = fma2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd), splat2(-mu * rstd));
+                  const float2 y01 = fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y));
+                  const float2 y23 = fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w));
+                  y0 = y01.x; y1 = y01.y; y2 = y23.x; y3 = y23.y;
                 } else {
-                  y0 = __uint_as_float(v[4 * j]) * rstd * gg.x;
-                  y1 = __uint_as_float(v[4 * j + 1]) * rstd * gg.y;
-                  y2 = __uint_as_float(v[4 * j + 2]) * rstd * gg.z;
-                  y3 = __uint_as_float(v[4 * j + 3]) * rstd * gg.w;
+                  const float2 y01 = mul2(mul2(f2_from_bits(v[4 * j], v[4 * j + 1]), splat2(rstd)), make_float2(gg.x, gg.y));
+                  const float2 y23 = mul2(mul2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd)), make_float2(gg.z, gg.w));
+                  y0 = y01.x; y1 = y01.y; y2 = y23.x; y3 = y23.y;
                   const int c = ncta0 + lc + 4 * j;
                   if (y0 > best) { best = y0; best_col = c; }
                   if (y1 > best) { best = y1; best_col = c + 1; }
@@ -709,8 +716,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               float s0 = 0.f, s1 = 0.f;
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
-                float e0 = ex2_approx(fmaf(__uint_as_float(v[j]), sc, -msub));
-                float e1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), sc, -msub));
+                const float2 t01 = fma2(f2_from_bits(v[j], v[j + 1]), splat2(sc), splat2(-msub));
+                float e0 = ex2_approx(t01.x);
+                float e1 = ex2_approx(t01.y);
                 if (st != 2) {
                   if (col0 + j > grow) e0 = 0.f;
                   if (col0 + j + 1 > grow) e1 = 0.f;
@@ -749,8 +757,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 uint32_t v[32];
                 tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                  pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]) * f, __uint_as_float(v[2 * j + 1]) * f);
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(f)));
               }
             }
             store_box(pk);

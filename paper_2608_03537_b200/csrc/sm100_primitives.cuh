@@ -276,6 +276,24 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed fp32x2 arithmetic (one instruction for two lanes of a float2): halves the issue slots of the epilogue math.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 splat2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 f2_from_bits(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
+// the two bf16 halves of a packed word, widened exactly
+__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t u) { return make_float2(bf16_lo(u), bf16_hi(u)); }
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float2 v) { return pack_bf16x2_rn(v.x, v.y); }
+// GELU, tanh form, on a pair: six packed instructions and two MUFU.TANH
+__device__ __forceinline__ float2 gelu_tanh_f32x2(float2 z) {
+  const float2 c0 = splat2(0.7978845608028654f);
+  const float2 c1 = splat2(0.7978845608028654f * 0.044715f);
+  const float2 u = mul2(z, fma2(c1, mul2(z, z), c0));
+  const float2 t = make_float2(tanh_approx(u.x), tanh_approx(u.y));
+  const float2 hz = mul2(splat2(0.5f), z);
+  return fma2(hz, t, hz);
+}
 // GELU, tanh form: 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).
 __device__ __forceinline__ float gelu_tanh_f32(float x) {
   const float c0 = 0.7978845608028654f;
