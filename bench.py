@@ -180,6 +180,24 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------------------ multi-process helpers
+def max_over_ranks(ms: float, device=None) -> float:
+    """The slowest rank's time (every rank gets it).  Works on any initialised process group (nccl or gloo)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes `units_per_rank` per step; the job's rate is all ranks' units over the
+    slowest rank's time."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------------ CUDA arm
 def run_comfuse(args):
     import torch
@@ -266,12 +284,7 @@ def run_comfuse(args):
             fn(i)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev)
 
     # ---- warm-up, then the timed region.  The K steps are replayed from a CUDA graph that holds one launch per
     # buffer set (the paper's protocol, Sec. 6 Setup: capture and replay to take host launch cost out of the device
@@ -306,11 +319,7 @@ def run_comfuse(args):
     run_steps(args.steps, lambda i: step(sets[i % nsets]))
     e1.record()
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dev)
     clocks = sampler.stop()
     launches = cf.launch_count() - launches0
     if graph is not None:   # replayed launches do not pass through the library's host code: count them from the graph
@@ -322,7 +331,7 @@ def run_comfuse(args):
     ms_step = ms_total / args.steps
     flops = w.gemm_flops()
     bytes_min = w.min_hbm_bytes()
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(flops, world, ms_step) / 1e12
 
     # ---- roofline of the dominant kernel (the fused kernel; one launch per step)
     t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
@@ -386,7 +395,7 @@ def run_comfuse(args):
     for i in range(2):
         e2e_step(i)
     ms_e2e = timed(n_e2e, e2e_step) / n_e2e
-    e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+    e2e = {"value": whole_job_value(flops, world, ms_e2e) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e}
 
     # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only, on a bounded sample

@@ -1,0 +1,116 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every function that include/comfuse.h
+declares, and rejects bad arguments before it touches CUDA."""
+import ctypes
+import os
+import re
+
+import paper_2608_03537_b200 as cf
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+FAKE = ctypes.c_void_p(4096)       # 16-byte aligned, never dereferenced: validation comes first
+ODD = ctypes.c_void_p(4096 + 2)    # misaligned
+
+
+def _desc(**kw):
+    d = cf.GemmDesc()
+    d.batch, d.M, d.N, d.K = 1, 256, 768, 512
+    d.lda, d.ldb, d.ldr, d.ldy = 512, 768, 768, 768
+    d.batch_stride_a = d.batch_stride_b = d.batch_stride_r = d.batch_stride_y = 0
+    d.kind, d.mask, d.alpha, d.eps, d.fused, d.reserved = cf.EPI_BIAS_RES_LAYERNORM, cf.MASK_NONE, 1.0, 1e-5, 1, 0
+    for k, v in kw.items():
+        setattr(d, k, v)
+    return d
+
+
+def _ws(d):
+    n = ctypes.c_size_t(12345)
+    return cf.lib().comfuse_workspace_size(ctypes.byref(d), ctypes.byref(n)), n.value
+
+
+def test_library_exports_every_declared_function():
+    header = open(os.path.join(ROOT, "include", "comfuse.h")).read()
+    declared = set(re.findall(r"\b(comfuse_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(cf.EXPORTED_SYMBOLS), declared ^ set(cf.EXPORTED_SYMBOLS)
+    L = cf.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_status_strings_and_launch_counter():
+    L = cf.lib()
+    texts = [L.comfuse_status_string(i).decode() for i in range(8)]
+    assert texts[0] == "ok" and len(set(texts)) == 8
+    assert "unknown" in L.comfuse_status_string(99).decode()
+    assert cf.launch_count() >= 0
+
+
+def test_workspace_size_rules():
+    assert _ws(_desc()) == (cf.OK, 0)                                      # fused: no workspace
+    assert _ws(_desc(fused=0)) == (cf.OK, 256 * 768 * 2)                   # unfused: dense bf16 Z
+    assert _ws(_desc(fused=0, batch=3, batch_stride_a=256 * 512, batch_stride_b=512 * 768, batch_stride_y=256 * 768,
+                     batch_stride_r=256 * 768)) == (cf.OK, 3 * 256 * 768 * 2)
+    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776))[0] == cf.ERR_UNSUPPORTED      # no fused instantiation for N = 776
+    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776, fused=0))[0] == cf.OK          # ... but the unfused path takes it
+    assert _ws(_desc(N=770, ldb=776, ldr=776, ldy=776))[0] == cf.ERR_ALIGNMENT        # N must be a multiple of 8
+    assert _ws(_desc(lda=516))[0] == cf.ERR_ALIGNMENT                                  # leading dims too
+    assert _ws(_desc(lda=256))[0] == cf.ERR_INVALID_ARG                                # lda < K
+    assert _ws(_desc(M=0))[0] == cf.ERR_INVALID_ARG
+    assert _ws(_desc(kind=7))[0] == cf.ERR_INVALID_ARG
+    assert _ws(_desc(reserved=1))[0] == cf.ERR_INVALID_ARG
+    assert _ws(_desc(mask=cf.MASK_CAUSAL))[0] == cf.ERR_INVALID_ARG                    # masks belong to the softmax kind
+    sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldb=2048, ldr=2048, ldy=2048)
+    assert _ws(_desc(**sm, mask=cf.MASK_CAUSAL))[0] == cf.ERR_UNSUPPORTED              # causal needs M == N
+    assert _ws(_desc(**sm, M=2048, mask=cf.MASK_CAUSAL))[0] == cf.OK
+    assert _ws(_desc(**sm, mask=cf.MASK_ADDITIVE))[0] == cf.ERR_UNSUPPORTED            # additive mask: unfused only
+    assert _ws(_desc(**sm, mask=cf.MASK_ADDITIVE, fused=0))[0] == cf.OK
+    assert cf.lib().comfuse_workspace_size(None, None) == cf.ERR_INVALID_ARG
+
+
+def test_gemm_epilogue_rejects_bad_arguments_before_any_launch():
+    L = cf.lib()
+    d = _desc()
+    args = cf.EpilogueArgs(None, None, None, None, None, None, None)
+    call = lambda dd, A, B, Y, a, ws, n: L.comfuse_gemm_epilogue(ctypes.byref(dd), A, B, Y, ctypes.byref(a), ws, n, None)
+    before = cf.launch_count()
+    assert call(d, None, FAKE, FAKE, args, None, 0) == cf.ERR_INVALID_ARG              # NULL operand
+    assert call(d, ODD, FAKE, FAKE, args, None, 0) == cf.ERR_ALIGNMENT                 # misaligned operand
+    bad = cf.EpilogueArgs(ODD, None, None, None, None, None, None)
+    assert call(d, FAKE, FAKE, FAKE, bad, None, 0) == cf.ERR_ALIGNMENT                 # misaligned bias vector
+    rms = _desc(kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX)
+    assert call(rms, FAKE, FAKE, FAKE, args, None, 0) == cf.ERR_INVALID_ARG            # row_max / row_argmax missing
+    un = _desc(fused=0)
+    assert call(un, FAKE, FAKE, FAKE, args, None, 0) == cf.ERR_WORKSPACE               # unfused without workspace
+    assert call(un, FAKE, FAKE, FAKE, args, FAKE, 100) == cf.ERR_WORKSPACE             # ... or with too little
+    assert cf.launch_count() == before
+
+
+def test_b2b_validation():
+    L = cf.lib()
+    n = ctypes.c_size_t(0)
+    ok = cf.make_b2b_desc(1024, 128, 512, 128, fused=True)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(ok), ctypes.byref(n)) == cf.OK and n.value == 0
+    un = cf.make_b2b_desc(1024, 128, 512, 128, fused=False)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(un), ctypes.byref(n)) == cf.OK
+    assert n.value == (1024 * 512 + 1024 * 128) * 2
+    for bad, code in [(cf.make_b2b_desc(1024, 128, 512, 256), cf.ERR_INVALID_ARG),      # residual needs N2 == K
+                      (cf.make_b2b_desc(1024, 256, 512, 256), cf.ERR_UNSUPPORTED),      # fused kernel: K = N2 = 128
+                      (cf.make_b2b_desc(1024, 128, 1024, 128), cf.ERR_UNSUPPORTED),     # N1 <= 512
+                      (cf.make_b2b_desc(1024, 128, 516, 128), cf.ERR_ALIGNMENT),
+                      (cf.make_b2b_desc(0, 128, 512, 128), cf.ERR_INVALID_ARG)]:
+        assert L.comfuse_b2b_workspace_size(ctypes.byref(bad), ctypes.byref(n)) == code
+    assert L.comfuse_b2b_gemm(ctypes.byref(ok), None, FAKE, FAKE, FAKE, FAKE, None, None, FAKE, None, 0, None) == cf.ERR_INVALID_ARG
+    assert L.comfuse_b2b_gemm(ctypes.byref(ok), ODD, FAKE, FAKE, FAKE, FAKE, None, None, FAKE, None, 0, None) == cf.ERR_ALIGNMENT
+
+
+def test_valid_call_without_a_usable_gpu_fails_cleanly():
+    """On a machine with no CUDA device a well-formed call must come back with an error code, not crash and not fall
+    back to anything else."""
+    import torch
+    if torch.cuda.is_available():
+        return
+    L = cf.lib()
+    d = _desc()
+    args = cf.EpilogueArgs(None, None, None, None, None, None, None)
+    st = L.comfuse_gemm_epilogue(ctypes.byref(d), FAKE, FAKE, FAKE, ctypes.byref(args), None, 0, None)
+    assert st in (cf.ERR_CUDA, cf.ERR_ARCH)
+    assert cf.lib().comfuse_last_device_status(None) in (cf.ERR_CUDA, cf.ERR_ARCH)
