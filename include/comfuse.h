@@ -144,6 +144,13 @@ comfuse_status_t comfuse_last_device_status(void* cuda_stream);
 /* Number of kernels this library has launched in this process since it was loaded (for accounting). */
 uint64_t comfuse_launch_count(void);
 
+/* Failure-detection self-test (the paper has no counterpart).  Launches one small kernel whose threads wait on a barrier
+ * that nothing signals, with a limit of `timeout_ms` (1..1000).  The waits must expire: the kernel ends normally, the
+ * device status word then reads COMFUSE_ERR_TIMEOUT (see comfuse_last_device_status) and the CUDA context stays usable.
+ * If `expired_waits` (a HOST pointer) is not NULL the call synchronises the stream and stores how many threads saw an
+ * expired or aborted wait (all 64). */
+comfuse_status_t comfuse_selftest_bounded_wait(uint32_t timeout_ms, void* cuda_stream, uint32_t* expired_waits);
+
 const char* comfuse_status_string(comfuse_status_t status);
 
 #ifdef __cplusplus

@@ -12,6 +12,7 @@ Functions mirror the C entry points:
     workspace_size(...)     -> comfuse_workspace_size
     b2b_workspace_size(...) -> comfuse_b2b_workspace_size
     last_device_status()    -> comfuse_last_device_status
+    selftest_bounded_wait() -> comfuse_selftest_bounded_wait
     launch_count()          -> comfuse_launch_count
 """
 from __future__ import annotations
@@ -36,6 +37,7 @@ EXPORTED_SYMBOLS = (
     "comfuse_b2b_gemm",
     "comfuse_last_device_status",
     "comfuse_launch_count",
+    "comfuse_selftest_bounded_wait",
     "comfuse_status_string",
 )
 
@@ -94,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.comfuse_b2b_gemm.restype = c_int32
         L.comfuse_last_device_status.argtypes = [c_void_p]
         L.comfuse_last_device_status.restype = c_int32
+        L.comfuse_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, POINTER(ctypes.c_uint32)]
+        L.comfuse_selftest_bounded_wait.restype = c_int32
         L.comfuse_launch_count.argtypes = []
         L.comfuse_launch_count.restype = c_uint64
         L.comfuse_status_string.argtypes = [c_int32]
@@ -200,6 +204,16 @@ def b2b_gemm(X, W1, b1, W2, b2, O, *, gamma=None, beta=None, eps=1e-5, fused=Tru
 def last_device_status(stream=None) -> int:
     """Synchronise the stream and return (and clear) the device status word: OK or ERR_TIMEOUT."""
     return int(lib().comfuse_last_device_status(_stream(stream)))
+
+
+def selftest_bounded_wait(timeout_ms: int = 20, stream=None) -> int:
+    """Run the bounded-wait self-test kernel; returns how many of its 64 threads saw an expired or aborted wait.  The
+    device status word reads ERR_TIMEOUT afterwards (last_device_status() returns and clears it)."""
+    n = ctypes.c_uint32(0)
+    st = lib().comfuse_selftest_bounded_wait(int(timeout_ms), _stream(stream), byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_selftest_bounded_wait")
+    return int(n.value)
 
 
 def launch_count() -> int:
