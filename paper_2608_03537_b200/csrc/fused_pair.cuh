@@ -527,6 +527,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               __syncwarp();
               if (lane == 0) mbar_arrive(bar_rdone(ring.stage));  // this warp is done with the stage
               ring.advance();
+              COMFUSE_TRACE_POINT();
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j) r32[j] = 0u;
@@ -586,6 +587,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               }
               tmem_st_32cols(taddr + g * 64 + half * 32, v);
             }
+            COMFUSE_TRACE_POINT();
           }
         }
         tmem_st_wait();
