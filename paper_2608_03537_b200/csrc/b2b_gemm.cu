@@ -26,7 +26,9 @@ namespace comfuse {
 
 namespace {
 
-constexpr int kB2bThreads = 320;
+constexpr int kB2bEpiWarps = 16;                       // four per TMEM lane quarter, 32 columns of a 128-column chunk each
+constexpr int kB2bEpiThreads = 32 * kB2bEpiWarps;
+constexpr int kB2bThreads = 32 * (2 + kB2bEpiWarps);  // producer, UMMA, epilogue warps
 constexpr int kSlotBytes = 128 * 64 * 2;  // one 128 x 64 bf16 box
 constexpr int kRingSlots = 8;
 constexpr int kMaxChunks = 4;             // N1 <= 512
@@ -37,8 +39,8 @@ struct B2bSmem {
   static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // one output staging box
   static constexpr int OFF_B1 = OFF_YBUF + kSlotBytes;             // fp32 [512]
   static constexpr int OFF_VEC = OFF_B1 + kMaxChunks * 128 * 4;    // b2, gamma, beta fp32 [128] each
-  static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][2][128]
-  static constexpr int OFF_STATS = OFF_PRE + 2 * 2 * 128 * 8;      // float2 [2][1][128]
+  static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][4][128]
+  static constexpr int OFF_STATS = OFF_PRE + 2 * 4 * 128 * 8;      // float2 [2][1][128]
   static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
   // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats drain
   static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 2;
@@ -96,12 +98,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_pfull(a), 1);
-      mbar_init(bar_sfull(a), 2 * 256);
+      mbar_init(bar_sfull(a), 2 * kB2bEpiWarps);   // one arrival per epilogue warp of both CTAs
       mbar_init(bar_sempty(a), 1);
       mbar_init(bar_ofull(a), 1);
-      mbar_init(bar_oempty(a), 2 * 256);
+      mbar_init(bar_oempty(a), 2 * kB2bEpiWarps);
     }
-    mbar_init(bar_stats, 128);
+    mbar_init(bar_stats, 4);
     mbar_init(bar_drain, 1);
     *s_abort = 0;
     fence_mbar_init();
@@ -257,8 +259,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;
-    const int h = (warp - 2) >> 2;
+    const int q = warp & 3;          // TMEM lane quarter: rows 32q .. 32q+31
+    const int hh = (warp - 2) >> 2;  // which 32 columns of every 128-column chunk / of the 128 output columns
     const int row = q * 32 + lane;
     const int epi_tid = threadIdx.x - 64;
     const bool store_thread = epi_tid == 0;
@@ -266,6 +268,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const uint32_t ybuf = smem_base + B2bSmem::OFF_YBUF;
     const uint32_t sfull_leader = map_to_cta(bar_sfull(0), leader);
     const uint32_t oempty_leader = map_to_cta(bar_oempty(0), leader);
+    const int kblk = hh >> 1;            // K block of S (and residual box) this thread's columns fall into
+    const int chunk0 = (hh & 1) * 4;     // first of its four 16-byte chunks inside that 128-byte row
     RingPos<kRingSlots> ring;
     uint32_t rfull_bits = 0;
     uint32_t puses[2] = {0, 0}, suses[2] = {0, 0};
@@ -298,33 +302,30 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
         ++suses[pb];
         __syncwarp();
+        uint32_t v[32];
+        tmem_ld_32cols(tmem_base + lane_sel + pb * 128 + hh * 32, v);
+        const float4* b4 = reinterpret_cast<const float4*>(s_b1 + j * 128 + hh * 32);
+        uint32_t pk[16];
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t v[32];
-          tmem_ld_32cols(tmem_base + lane_sel + pb * 128 + h * 64 + half * 32, v);
-          const float4* b4 = reinterpret_cast<const float4*>(s_b1 + j * 128 + h * 64 + half * 32);
-          uint32_t pk[16];
+        for (int i = 0; i < 8; ++i) {
+          const float4 bb = b4[i];
+          const float2 g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
+          const float2 g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
+          pk[2 * i] = pack_bf16x2_rn(g01);
+          pk[2 * i + 1] = pack_bf16x2_rn(g23);
+        }
+        const uint32_t sb = s_addr(pb, kblk);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float4 bb = b4[i];
-            const float2 g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
-            const float2 g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
-            pk[2 * i] = pack_bf16x2_rn(g01);
-            pk[2 * i + 1] = pack_bf16x2_rn(g23);
-          }
-          // this thread's 32 columns are 16-byte chunks half*4 .. half*4+3 of K block h of the S buffer
-          const uint32_t sb = s_addr(pb, h);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t a = sb + swz128(row, half * 4 + i);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                         "r"(pk[4 * i + 3])
-                         : "memory");
-          }
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t a = sb + swz128(row, chunk0 + i);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                       "r"(pk[4 * i + 3])
+                       : "memory");
         }
         tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
         fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
-        mbar_arrive_cluster(sfull_leader + 8u * pb);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(sfull_leader + 8u * pb);
         B2B_TRACE_POINT();
       }
       ring.skip(2 + 2 * NC);  // X, W1 and W2 slots were the tensor pipe's
@@ -333,108 +334,103 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       __syncwarp();
       tcgen05_fence_after_sync();
       B2B_TRACE_POINT();
-      const int rstage = ring.stage + h >= kRingSlots ? ring.stage + h - kRingSlots : ring.stage + h;
+      const int s0 = ring.stage;
+      const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
       // both residual slots are waited for by everybody (the phase bits must advance uniformly)
-      uint32_t r32[2][16];
-      {
-        const int s0 = ring.stage;
-        mbar_wait<false>(bar_rfull(s0), (rfull_bits >> s0) & 1u, w);
-        rfull_bits ^= 1u << s0;
-        const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
-        mbar_wait<false>(bar_rfull(s1), (rfull_bits >> s1) & 1u, w);
-        rfull_bits ^= 1u << s1;
-        __syncwarp();
-      }
+      mbar_wait<false>(bar_rfull(s0), (rfull_bits >> s0) & 1u, w);
+      rfull_bits ^= 1u << s0;
+      mbar_wait<false>(bar_rfull(s1), (rfull_bits >> s1) & 1u, w);
+      rfull_bits ^= 1u << s1;
+      __syncwarp();
+      uint32_t r32[16];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t a = ring_addr(rstage) + swz128(row, half * 4 + i);
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(r32[half][4 * i]), "=r"(r32[half][4 * i + 1]), "=r"(r32[half][4 * i + 2]), "=r"(r32[half][4 * i + 3])
-                       : "r"(a));
-        }
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t a = ring_addr(kblk ? s1 : s0) + swz128(row, chunk0 + i);
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(r32[4 * i]), "=r"(r32[4 * i + 1]), "=r"(r32[4 * i + 2]), "=r"(r32[4 * i + 3])
+                     : "r"(a));
       }
       // hand the two residual slots back
       __syncwarp();
-      named_barrier_sync(2, 256);
+      named_barrier_sync(2, kB2bEpiThreads);
       if (store_thread) {
-        mbar_arrive(bar_empty(ring.stage));
-        mbar_arrive(bar_empty(ring.stage + 1 == kRingSlots ? 0 : ring.stage + 1));
+        mbar_arrive(bar_empty(s0));
+        mbar_arrive(bar_empty(s1));
       }
       ring.skip(2);
-      // stage 1: x = O + b2 + X ; thread-local (mean, M2) over this thread's 64 columns
-      float x[2][32];
-      float2 part = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      // stage 1: x = O + b2 + X ; thread-local (mean, M2) over this thread's 32 columns; x goes back into TMEM
+      const uint32_t o_addr = tmem_base + lane_sel + 256 + obuf * 128 + hh * 32;
+      float2 part;
+      {
         uint32_t v[32];
-        tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + h * 64 + half * 32, v);
-        const float4* b4 = reinterpret_cast<const float4*>(s_b2 + h * 64 + half * 32);
-        float s0 = 0.f, s1 = 0.f;
+        tmem_ld_32cols(o_addr, v);
+        const float4* b4 = reinterpret_cast<const float4*>(s_b2 + hh * 32);
+        float2 s01 = splat2(0.f), s23 = splat2(0.f);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float4 bb = b4[i];
-          x[half][4 * i] = __uint_as_float(v[4 * i]) + bb.x + bf16_lo(r32[half][2 * i]);
-          x[half][4 * i + 1] = __uint_as_float(v[4 * i + 1]) + bb.y + bf16_hi(r32[half][2 * i]);
-          x[half][4 * i + 2] = __uint_as_float(v[4 * i + 2]) + bb.z + bf16_lo(r32[half][2 * i + 1]);
-          x[half][4 * i + 3] = __uint_as_float(v[4 * i + 3]) + bb.w + bf16_hi(r32[half][2 * i + 1]);
-          s0 += x[half][4 * i] + x[half][4 * i + 1];
-          s1 += x[half][4 * i + 2] + x[half][4 * i + 3];
+          const float2 x01 = add2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)), bf16x2_to_f2(r32[2 * i]));
+          const float2 x23 = add2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)), bf16x2_to_f2(r32[2 * i + 1]));
+          v[4 * i] = __float_as_uint(x01.x); v[4 * i + 1] = __float_as_uint(x01.y);
+          v[4 * i + 2] = __float_as_uint(x23.x); v[4 * i + 3] = __float_as_uint(x23.y);
+          s01 = add2(s01, x01);
+          s23 = add2(s23, x23);
         }
-        const float cmean = (s0 + s1) * (1.f / 32.f);
-        float q0 = 0.f, q1 = 0.f;
+        const float cmean = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32.f);
+        const float2 nm = splat2(-cmean);
+        float2 q01 = splat2(0.f), q23 = splat2(0.f);
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float d0 = x[half][i] - cmean, d1 = x[half][i + 1] - cmean;
-          q0 = fmaf(d0, d0, q0);
-          q1 = fmaf(d1, d1, q1);
+        for (int i = 0; i < 8; ++i) {
+          const float2 d01 = add2(f2_from_bits(v[4 * i], v[4 * i + 1]), nm);
+          const float2 d23 = add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), nm);
+          q01 = fma2(d01, d01, q01);
+          q23 = fma2(d23, d23, q23);
         }
-        const float2 cpart = make_float2(cmean, q0 + q1);
-        part = half == 0 ? cpart : MergeWelford()(part, 32.f, cpart, 32.f);
+        part = make_float2(cmean, (q01.x + q01.y) + (q23.x + q23.y));
+        tmem_st_32cols(o_addr, v);
+        tmem_st_wait();
       }
-      // the accumulator has been copied out: the O slot can be reused by the tile after the next one
-      tcgen05_fence_before_sync();
-      mbar_arrive_cluster(oempty_leader + 8u * obuf);
-      // reduce: the row lives in this CTA only (two half-row threads)
-      const float2 tot = cluster_row_reduce<1>(part, 64.f, MergeWelford(), s_pre, s_stats, bar_stats, row, h, 0u, xpar, xphase, w);
+      // reduce: the row lives in this CTA only (four quarter-row threads)
+      const float2 tot =
+          cluster_row_reduce<1, MergeWelford, 4>(part, 32.f, MergeWelford(), s_pre, s_stats, bar_stats, row, hh, 0u, xpar, xphase, w);
       B2B_TRACE_POINT();
       const float mu = tot.x;
       const float rstd = rsqrtf(tot.y * (1.f / 128.f) + p.eps);
-      // stage 2: normalise, round once, stage one 128 x 64 box per half-row group and store it
-      uint32_t pk[2][16];
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const float4* g4 = reinterpret_cast<const float4*>(s_gamma + h * 64 + half * 32);
-        const float4* be4 = reinterpret_cast<const float4*>(s_beta + h * 64 + half * 32);
+      // stage 2: normalise the resident x, round once
+      uint32_t pk[16];
+      {
+        uint32_t v[32];
+        tmem_ld_32cols(o_addr, v);
+        const float4* g4 = reinterpret_cast<const float4*>(s_gamma + hh * 32);
+        const float4* be4 = reinterpret_cast<const float4*>(s_beta + hh * 32);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float4 gg = g4[i], be = be4[i];
-          const float y0 = fmaf((x[half][4 * i] - mu) * rstd, gg.x, be.x);
-          const float y1 = fmaf((x[half][4 * i + 1] - mu) * rstd, gg.y, be.y);
-          const float y2 = fmaf((x[half][4 * i + 2] - mu) * rstd, gg.z, be.z);
-          const float y3 = fmaf((x[half][4 * i + 3] - mu) * rstd, gg.w, be.w);
-          pk[half][2 * i] = pack_bf16x2_rn(y0, y1);
-          pk[half][2 * i + 1] = pack_bf16x2_rn(y2, y3);
+          const float2 n01 = fma2(f2_from_bits(v[4 * i], v[4 * i + 1]), splat2(rstd), splat2(-mu * rstd));
+          const float2 n23 = fma2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), splat2(rstd), splat2(-mu * rstd));
+          pk[2 * i] = pack_bf16x2_rn(fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y)));
+          pk[2 * i + 1] = pack_bf16x2_rn(fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w)));
         }
       }
-      // two boxes (columns 0..63 from the h = 0 threads, 64..127 from the h = 1 threads) through one staging buffer
+      // the accumulator has been read for the last time: the O slot can be reused by the tile after the next one
+      tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(oempty_leader + 8u * obuf);
+      // two 128 x 64 boxes (columns 0..63 from the hh = 0, 1 warps, 64..127 from hh = 2, 3) through one staging buffer
       for (int g = 0; g < 2; ++g) {
         if (store_thread) tma_store_wait_read<0>();
-        named_barrier_sync(3, 256);
-        if (h == g) {
+        named_barrier_sync(3, kB2bEpiThreads);
+        if (kblk == g) {
 #pragma unroll
-          for (int half = 0; half < 2; ++half)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t a = ybuf + swz128(row, half * 4 + i);
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[half][4 * i]), "r"(pk[half][4 * i + 1]),
-                           "r"(pk[half][4 * i + 2]), "r"(pk[half][4 * i + 3])
-                           : "memory");
-            }
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t a = ybuf + swz128(row, chunk0 + i);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                         "r"(pk[4 * i + 3])
+                         : "memory");
+          }
         }
         fence_proxy_async_smem();
-        named_barrier_sync(3, 256);
+        named_barrier_sync(3, kB2bEpiThreads);
         if (store_thread) {
           tma_store_3d(&tmO, ybuf, g * 64, m0, 0);
           tma_store_commit();

@@ -51,11 +51,15 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
   for (int t = 1; t < NH; ++t) cta_partial = merge(cta_partial, per_thread_count * t, s_pre[(xpar * NH + t) * 128 + row], per_thread_count);
   const float cta_count = static_cast<float>(NH) * per_thread_count;
   // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks congruent to h mod NH
+  // Arrivals are per warp (lane 0, after a warp barrier that orders the other lanes' stores before it): the barrier
+  // expects 4 arrivals per source CTA, one from each lane quarter's sending warp.
+  const bool lane0 = (threadIdx.x & 31) == 0;
   float2* slot = s_stats + (xpar * CN + rank) * 128 + row;
   if constexpr (CN == 1) {
     if (h == 0) {
       *slot = cta_partial;
-      mbar_arrive(stats_bar);
+      __syncwarp();
+      if (lane0) mbar_arrive(stats_bar);
     }
   } else {
     const uint32_t slot_addr = smem_u32(slot);
@@ -64,8 +68,13 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
       if ((dst % NH) == h) {
         const uint32_t peer = dst * rank_stride + rank_offset;
         st_cluster_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y);
-        mbar_arrive_cluster(map_to_cta(stats_bar, peer));
       }
+    }
+    __syncwarp();
+    if (lane0) {
+#pragma unroll
+      for (int dst = 0; dst < CN; ++dst)
+        if ((dst % NH) == h) mbar_arrive_cluster(map_to_cta(stats_bar, dst * rank_stride + rank_offset));
     }
   }
   if constexpr (CN == 1) {

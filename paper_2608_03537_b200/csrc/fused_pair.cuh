@@ -3,8 +3,8 @@
 // Why pairs: one SM's shared memory delivers 128 B/clk, and a 128 x 256 x 16 bf16 UMMA that reads both operands
 // from shared memory already needs 96 B/clk before TMA has written the next tiles.  With cta_group::2 two CTAs
 // multiply 256 rows at once: each holds its own 128 rows of A and only HALF of the B tile, so the per-SM operand
-// traffic (and the L2 -> shared-memory fill) of the weight operand halves.  No multicast copies are used: each
-// CTA fetches its own half with ordinary TMA loads that signal the issuing (even) CTA's barrier.
+// traffic (and the L2 -> shared-memory fill) of the weight operand halves.  Every CTA fetches its
+// own half with ordinary (single-destination) TMA loads that signal the issuing (even) CTA's barrier.
 //
 // Work decomposition (Sec. 3.1, cluster-granular scheduling with a secondary mapping by CTA rank): a cluster has
 // 2*CN CTAs; cluster rank r works on row block (r & 1) of a pair of adjacent 128-row blocks and on column range
@@ -166,9 +166,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull(a), 1);
-      mbar_init(bar_tempty(a), 2 * Cfg::kEpiThreads);  // both CTAs' epilogue threads
+      mbar_init(bar_tempty(a), 2 * Cfg::kEpiWarps);  // one arrival per epilogue warp of both CTAs
     }
-    mbar_init(bar_stats, CN * 128);
+    mbar_init(bar_stats, CN * 4);  // per source CTA: one arrival from each lane quarter's sending warp
     mbar_init(bar_drain, 1);
     for (int e = 0; e < Cfg::kEpiWarps; ++e)
       for (int k = 0; k < 4; ++k) {
@@ -476,7 +476,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       auto release_accumulator = [&](int sub) {
         if (live[sub]) {
           tcgen05_fence_before_sync();
-          mbar_arrive_cluster(tempty_leader + 8u * slot[sub]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * slot[sub]);
         }
       };
       auto tmem_of = [&](int sub) { return tmem_base + lane_sel + (slot[sub] ? BNS0 : 0); };
