@@ -43,7 +43,7 @@ struct B2bSmem {
   static constexpr int OFF_STATS = OFF_PRE + 2 * 4 * 128 * 8;      // float2 [2][1][128]
   static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
   // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats drain
-  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 2;
+  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 3;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
@@ -76,7 +76,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   auto bar_ofull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 6 + a); };   // O slot complete
   auto bar_oempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 8 + a); };  // O slot drained by both CTAs (even CTA)
   const uint32_t bar_stats = bar_base + 8u * (3 * kRingSlots + 10);
-  const uint32_t bar_drain = bar_stats + 8u;
+  const uint32_t bar_drain = bar_stats + 16u;
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + B2bSmem::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + B2bSmem::OFF_MISC + 4);
 
@@ -104,6 +104,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       mbar_init(bar_oempty(a), 2 * kB2bEpiWarps);
     }
     mbar_init(bar_stats, 4);
+    mbar_init(bar_stats + 8u, 4);
     mbar_init(bar_drain, 1);
     *s_abort = 0;
     fence_mbar_init();
@@ -225,7 +226,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ring.advance();
           if (!ok) return;
           const int sb = j & 1;
-          if (!mbar_wait<true>(bar_sfull(sb), sfull_uses[sb] & 1u, w)) { ok = false; return; }
+          if (!mbar_wait<false>(bar_sfull(sb), sfull_uses[sb] & 1u, w)) { ok = false; return; }
           ++sfull_uses[sb];
           tcgen05_fence_after_sync();
           const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
@@ -240,7 +241,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           umma_commit_pair(map_to_cta(bar_sempty(sb), peer));
         };
         // O slot must have been drained by Epi2 of the tile before the previous one
-        if (!mbar_wait<true>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
+        if (!mbar_wait<false>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
         tcgen05_fence_after_sync();
         issue_ml1(0);
         if (NC > 1) issue_ml1(1);
@@ -302,19 +303,32 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
         ++suses[pb];
         __syncwarp();
+        B2B_TRACE_POINT();
         uint32_t v[32];
         tmem_ld_32cols(tmem_base + lane_sel + pb * 128 + hh * 32, v);
         const float4* b4 = reinterpret_cast<const float4*>(s_b1 + j * 128 + hh * 32);
         uint32_t pk[16];
+#ifdef COMFUSE_TRACE
+        const int tf = p.trace_flags;
+#else
+        constexpr int tf = 0;
+#endif
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float4 bb = b4[i];
-          const float2 g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
-          const float2 g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
+          float2 g01, g23;
+          if (tf & 1) {  // experiment: no transcendental
+            g01 = add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y));
+            g23 = add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w));
+          } else {
+            g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
+            g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
+          }
           pk[2 * i] = pack_bf16x2_rn(g01);
           pk[2 * i + 1] = pack_bf16x2_rn(g23);
         }
         const uint32_t sb = s_addr(pb, kblk);
+        if (!(tf & 2)) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint32_t a = sb + swz128(row, chunk0 + i);
@@ -322,10 +336,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
                        "r"(pk[4 * i + 3])
                        : "memory");
         }
+        }
+        B2B_TRACE_POINT();
         tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
-        fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
+        if (!(tf & 4)) fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(sfull_leader + 8u * pb);
+        if (lane == 0) mbar_arrive_cluster_noflush(sfull_leader + 8u * pb);
         B2B_TRACE_POINT();
       }
       ring.skip(2 + 2 * NC);  // X, W1 and W2 slots were the tensor pipe's
@@ -415,7 +431,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       // the accumulator has been read for the last time: the O slot can be reused by the tile after the next one
       tcgen05_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(oempty_leader + 8u * obuf);
+      if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
       // two 128 x 64 boxes (columns 0..63 from the hh = 0, 1 warps, 64..127 from hh = 2, 3) through one staging buffer
       for (int g = 0; g < 2; ++g) {
         if (store_thread) tma_store_wait_read<0>();

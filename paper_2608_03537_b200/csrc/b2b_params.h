@@ -19,6 +19,7 @@ struct B2bParams {
   unsigned int* status;
   unsigned long long timeout_ns;
   unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null
+  int trace_flags;            // tracing builds: experiment switches
 };
 
 bool b2b_fused_supported(int K, int N1, int N2);

@@ -357,6 +357,7 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     bp.timeout_ns = timeout_ns();
 #ifdef COMFUSE_TRACE
     if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) bp.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));
+    if (const char* tf = std::getenv("COMFUSE_TRACE_FLAGS")) bp.trace_flags = std::atoi(tf);
 #endif
     cudaError_t e = launch_b2b_fused(X, W1, W2, bp, st);
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;

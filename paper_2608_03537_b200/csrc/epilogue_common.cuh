@@ -34,10 +34,14 @@ struct MergeArgmax {  // (value, column index bits); ties -> lower index
   }
 };
 
-// The reduce phase above thread level.  All 256 epilogue threads of every CTA that shares the rows call this the
-// same number of times.  `per_thread_count` = elements behind each thread's partial (1/NH of the CTA's columns).
+// The reduce phase above thread level.  All epilogue threads of every CTA that shares the rows call this the same
+// number of times.  `per_thread_count` = elements behind each thread's partial (1/NH of the CTA's columns).
 // `rank` is this CTA's index among the CN column ranges; the cluster rank of column range c is
 // c * rank_stride + rank_offset (CTA pairs interleave two row blocks in one cluster).
+// Exchanges alternate between two buffers AND two barriers (`stats_bar`, `stats_bar + 8`): a CTA that has passed
+// exchange e may start sending exchange e + 1 while a slow peer's exchange-e message to some third CTA is still in
+// flight; with one barrier that early message could complete the third CTA's phase e in place of the late one.
+// `xpar` = buffer / barrier of the next exchange, `xphase` = one phase bit per barrier.
 template <int CN, class Merge, int NH = 2>
 __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thread_count, Merge merge, float2* s_pre,
                                                      float2* s_stats, uint32_t stats_bar, int row, int h,
@@ -51,42 +55,37 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
   for (int t = 1; t < NH; ++t) cta_partial = merge(cta_partial, per_thread_count * t, s_pre[(xpar * NH + t) * 128 + row], per_thread_count);
   const float cta_count = static_cast<float>(NH) * per_thread_count;
   // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks congruent to h mod NH
-  // Arrivals are per warp (lane 0, after a warp barrier that orders the other lanes' stores before it): the barrier
-  // expects 4 arrivals per source CTA, one from each lane quarter's sending warp.
-  const bool lane0 = (threadIdx.x & 31) == 0;
+  const uint32_t bar = stats_bar + 8u * xpar;
+  const uint32_t phase = (xphase >> xpar) & 1u;
   float2* slot = s_stats + (xpar * CN + rank) * 128 + row;
   if constexpr (CN == 1) {
+    // one CTA: plain stores, one arrival per lane quarter (lane 0, after a warp barrier that orders the other lanes'
+    // stores before it); the barrier expects 4 arrivals
     if (h == 0) {
       *slot = cta_partial;
       __syncwarp();
-      if (lane0) mbar_arrive(stats_bar);
+      if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
     }
+    mbar_wait<false>(bar, phase, w);
   } else {
+    // each partial travels as an asynchronous 8-byte store that is counted on the destination's barrier; one local
+    // thread arms the barrier with the byte count of the whole exchange (CN peers x 128 rows x 8 bytes)
+    if (h == 0 && row == 0) mbar_arrive_expect_tx(bar, CN * 128 * 8);
     const uint32_t slot_addr = smem_u32(slot);
 #pragma unroll
     for (int dst = 0; dst < CN; ++dst) {
       if ((dst % NH) == h) {
         const uint32_t peer = dst * rank_stride + rank_offset;
-        st_cluster_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y);
+        st_async_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y, map_to_cta(bar, peer));
       }
     }
-    __syncwarp();
-    if (lane0) {
-#pragma unroll
-      for (int dst = 0; dst < CN; ++dst)
-        if ((dst % NH) == h) mbar_arrive_cluster(map_to_cta(stats_bar, dst * rank_stride + rank_offset));
-    }
-  }
-  if constexpr (CN == 1) {
-    mbar_wait<false>(stats_bar, xphase, w);
-  } else {
-    mbar_wait<true>(stats_bar, xphase, w);
+    mbar_wait<true>(bar, phase, w);
   }
   float2 acc = s_stats[(xpar * CN + 0) * 128 + row];
 #pragma unroll
   for (int c = 1; c < CN; ++c) acc = merge(acc, cta_count * c, s_stats[(xpar * CN + c) * 128 + row], cta_count);
+  xphase ^= 1u << xpar;
   xpar ^= 1;
-  xphase ^= 1;
   __syncwarp();
   return acc;
 }

@@ -58,7 +58,7 @@ struct PairCfg {
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
-  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * EPW * 128 * 8 + (4 * NSTAGES + 6 + 128) * 8 + 16 + 1024;
+  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * EPW * 128 * 8 + (4 * NSTAGES + 7 + 128) * 8 + 16 + 1024;
   static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (kEpiWarps * WARP_BOX_BYTES);
   static constexpr int YBOXES = YBOX_ROOM >= 4 ? 4 : YBOX_ROOM;           // staging boxes per epilogue warp
   static constexpr int YBUF_BYTES = YBOXES * kEpiWarps * WARP_BOX_BYTES;
@@ -72,7 +72,7 @@ struct PairCfg {
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
   static constexpr int PRE_BYTES = 2 * EPW * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 2 + 128;  // + staging-box full/free, up to 16 warps x 4 boxes each
+  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 3 + 128;  // + staging-box full/free, up to 16 warps x 4 boxes each
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
@@ -136,7 +136,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto bar_tfull = [&](int a) { return bar_base + 8u * (4 * NSTAGES + a); };    // accumulator slot complete
   auto bar_tempty = [&](int a) { return bar_base + 8u * (4 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
   const uint32_t bar_stats = bar_base + 8u * (4 * NSTAGES + 4);
-  const uint32_t bar_drain = bar_stats + 8u;
+  const uint32_t bar_drain = bar_stats + 16u;  // two statistics barriers (one per exchange parity)
   auto bar_yfull = [&](int e, int k) { return bar_drain + 8u + 8u * (e * 4 + k); };        // staging box written (epilogue warp e)
   auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (64 + e * 4 + k); };   // staging box read out by its TMA store
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
@@ -168,7 +168,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       mbar_init(bar_tfull(a), 1);
       mbar_init(bar_tempty(a), 2 * Cfg::kEpiWarps);  // one arrival per epilogue warp of both CTAs
     }
-    mbar_init(bar_stats, CN * 4);  // per source CTA: one arrival from each lane quarter's sending warp
+    mbar_init(bar_stats, CN == 1 ? 4 : 1);       // one CTA: an arrival per lane quarter; else one arming arrive + bytes
+    mbar_init(bar_stats + 8u, CN == 1 ? 4 : 1);
     mbar_init(bar_drain, 1);
     for (int e = 0; e < Cfg::kEpiWarps; ++e)
       for (int k = 0; k < 4; ++k) {
@@ -309,7 +310,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!ok || !unit_live(mpair0, n0)) continue;
           const int slot = LOCK ? 0 : (NSUB == 2 ? sub : static_cast<int>(unit_count & 1u));
           ++unit_count;
-          if (!mbar_wait<true>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; continue; }
+          if (!mbar_wait<false>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; continue; }
           ++slot_uses[slot];
           tcgen05_fence_after_sync();
           const uint32_t d_tmem = tmem_base + (slot ? BNS0 : 0);
@@ -477,7 +478,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (live[sub]) {
           tcgen05_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * slot[sub]);
+          if (lane == 0) mbar_arrive_cluster_noflush(tempty_leader + 8u * slot[sub]);
         }
       };
       auto tmem_of = [&](int sub) { return tmem_base + lane_sel + (slot[sub] ? BNS0 : 0); };

@@ -54,6 +54,14 @@ __device__ __forceinline__ void st_cluster_f32x2(uint32_t cluster_addr, float a,
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(cluster_addr), "f"(a), "f"(b) : "memory");
 }
 
+// Store 8 bytes into a peer CTA's shared memory and count them on a barrier of that CTA in one asynchronous operation:
+// the data is visible to whoever observes the barrier's phase complete, so the sender needs no release fence.
+__device__ __forceinline__ void st_async_f32x2(uint32_t cluster_addr, float a, float b, uint32_t cluster_mbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(cluster_addr),
+               "f"(a), "f"(b), "r"(cluster_mbar)
+               : "memory");
+}
+
 // ----------------------------------------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -69,6 +77,13 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 // Arrive on a barrier in another CTA of the cluster; releases this thread's earlier (remote) stores.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Arrive on a barrier that may live in another CTA of the cluster, with the default (CTA-scope) release: enough when
+// the barrier orders tensor-memory reads or async-proxy (UMMA / TMA) accesses, which have their own fences, and far
+// cheaper than the cluster-scope release (about 0.5 us per arrive on this part), which is only needed when ordinary
+// shared-memory data written by this thread must become visible to threads of the other CTA.
+__device__ __forceinline__ void mbar_arrive_cluster_noflush(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
