@@ -126,7 +126,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
-  cluster_sync_all();
+  cluster_sync_after_init();  // every CTA's barriers exist before any peer signals them
   const uint32_t tmem_base = *s_tmem_base;
   // TMEM columns: P slots at 0 and 128, O slots at 256 and 384
   auto ring_addr = [&](int s) { return smem_base + B2bSmem::OFF_RING + s * kSlotBytes; };
@@ -453,7 +453,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
     }
-    if (store_thread) tma_store_wait_all();
+    if (store_thread) tma_store_wait_read<0>();  // the staging buffer must outlive the last store's read
   }
 
   tcgen05_fence_before_sync();

@@ -156,6 +156,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const bool has_res = (EPI == EPI_LN || EPI == EPI_RMS_MAX) && p.residual != nullptr;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
 
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[62] = globaltimer_ns();  // kernel entry
+#endif
   // -------------------------------------------------------------------------------------------- set-up
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
@@ -201,7 +204,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
-  cluster_sync_all();  // every CTA's barriers exist before any peer signals them
+  cluster_sync_after_init();  // every CTA's barriers exist before any peer signals them
   const uint32_t tmem_base = *s_tmem_base;
 
   // tile -> (batch, first row of the pair, first column of this CTA)
@@ -386,7 +389,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
       }
-      tma_store_wait_all();  // the staging boxes must outlive the last stores' reads
+      tma_store_wait_read<0>();  // the staging boxes must outlive the last stores' reads (the stores themselves complete at kernel end)
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
@@ -413,7 +416,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int trace_ix = 0;
 #define COMFUSE_TRACE_POINT()                                                                          \
   do {                                                                                                 \
-    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 64) p.trace[trace_ix++] = globaltimer_ns(); \
+    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 60) p.trace[trace_ix++] = globaltimer_ns(); \
   } while (0)
 #else
 #define COMFUSE_TRACE_POINT() do { } while (0)
@@ -773,6 +776,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   }
 
   // -------------------------------------------------------------------------------------------- teardown
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[61] = globaltimer_ns();  // epilogue warps done
+#endif
   tcgen05_fence_before_sync();
   __syncthreads();
   cluster_sync_all();  // no peer may still signal this CTA's barriers, write its shared memory or its TMEM
@@ -781,6 +787,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tcgen05_fence_after_sync();
     tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
   }
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[63] = globaltimer_ns();  // kernel exit
+#endif
 }
 
 }  // namespace comfuse
