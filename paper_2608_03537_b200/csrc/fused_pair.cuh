@@ -58,7 +58,7 @@ struct PairCfg {
   static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
   static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;                      // one warp's 32 x 64 bf16 output box
-  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * EPW * 128 * 8 + (4 * NSTAGES + 7 + 128) * 8 + 16 + 1024;
+  static constexpr int FIXED_BYTES = 3 * BN * 4 + 2 * CN * 128 * 8 + 2 * EPW * 128 * 8 + (4 * NSTAGES + 7 + 192) * 8 + 16 + 1024;
   static constexpr int YBOX_ROOM = (232448 - NSTAGES * STAGE_BYTES - FIXED_BYTES) / (kEpiWarps * WARP_BOX_BYTES);
   static constexpr int YBOXES = YBOX_ROOM >= 4 ? 4 : YBOX_ROOM;           // staging boxes per epilogue warp
   static constexpr int YBUF_BYTES = YBOXES * kEpiWarps * WARP_BOX_BYTES;
@@ -72,7 +72,12 @@ struct PairCfg {
   static constexpr int OFF_PRE = OFF_STATS + STATS_BYTES;
   static constexpr int PRE_BYTES = 2 * EPW * 128 * 8;
   static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
-  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 3 + 128;  // + staging-box full/free, up to 16 warps x 4 boxes each
+  static constexpr int NUM_BARS = 4 * NSTAGES + 4 + 3 + 192;  // + staging-box full/free/last-tile, up to 16 warps x 4 boxes each
+  // A CTA's LAST tile has the whole circular buffer to itself once its accumulator is complete (nothing is loaded after
+  // it), so every output box of that tile gets a staging box of its own there and no epilogue warp waits for a store.
+  static constexpr int BOXES_PER_WARP = BN / 64 / EPW;
+  static constexpr bool RING_STAGING = EPI != EPI_SOFTMAX && ESUB == 1 && BOXES_PER_WARP <= 4 &&
+                                       kEpiWarps * BOXES_PER_WARP * WARP_BOX_BYTES <= NSTAGES * STAGE_BYTES;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
   static_assert(BNS0 % 128 == 0 && BNS0 <= 256 && BNS1 % 128 == 0 && BNS1 <= 256, "each CTA's half must be whole 64-column boxes");
@@ -139,6 +144,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const uint32_t bar_drain = bar_stats + 16u;  // two statistics barriers (one per exchange parity)
   auto bar_yfull = [&](int e, int k) { return bar_drain + 8u + 8u * (e * 4 + k); };        // staging box written (epilogue warp e)
   auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (64 + e * 4 + k); };   // staging box read out by its TMA store
+  auto bar_ylast = [&](int e, int k) { return bar_drain + 8u + 8u * (128 + e * 4 + k); };  // last tile: box k of warp e staged in the ring
+  auto ring_box = [&](int e, int k) { return smem_base + static_cast<uint32_t>((e * Cfg::BOXES_PER_WARP + k) * Cfg::WARP_BOX_BYTES); };
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
 
@@ -178,6 +185,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (int k = 0; k < 4; ++k) {
         mbar_init(bar_yfull(e, k), 1);
         mbar_init(bar_yfree(e, k), 1);
+        mbar_init(bar_ylast(e, k), 1);
       }
     *s_abort = 0;
     fence_mbar_init();
@@ -367,6 +375,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
         const int m0 = mpair0 + static_cast<int>(pm) * 128;
+        const bool in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles;
+        int kk = 0;  // box of this tile
         for (int sub = 0; sub < ESUB && ok; ++sub) {
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
@@ -374,6 +384,16 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           for (int g = h; g < W / 64; g += EPW) {
             const int col = group_col(ncta0, lg0 + g);
             if (EPI == EPI_NONE && col >= p.N) break;
+            if (in_ring) {
+              if (!mbar_wait<false>(bar_ylast(e, kk), 0, w)) { ok = false; break; }
+#ifdef COMFUSE_TRACE
+              if (!(p.trace_flags & 1))
+#endif
+              tma_store_3d(&tmY, ring_box(e, kk), col, m0 + q * 32, b);
+              tma_store_commit();
+              ++kk;
+              continue;
+            }
             const uint32_t sel = n % Cfg::YBOXES;
             if (!mbar_wait<false>(bar_yfull(e, sel), (n / Cfg::YBOXES) & 1u, w)) { ok = false; break; }
 #ifdef COMFUSE_TRACE
@@ -421,13 +441,23 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #else
 #define COMFUSE_TRACE_POINT() do { } while (0)
 #endif
+    bool in_ring = false;  // this tile's boxes are staged in the (idle) circular buffer
+    int ring_k = 0;
     auto store_box = [&](const uint32_t (&pk)[32]) {
-      const uint32_t sel = ybox_sel;
-      const uint32_t ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
-      if (++ybox_sel == Cfg::YBOXES) ybox_sel = 0;
-      // the store of the box's previous contents has read it out
-      mbar_wait<false>(bar_yfree(warp - 2, sel), ((ybox_count / Cfg::YBOXES) & 1u) ^ 1u, w);
-      ++ybox_count;
+      uint32_t ybox, ybar;
+      if (Cfg::RING_STAGING && in_ring) {
+        ybox = ring_box(warp - 2, ring_k);
+        ybar = bar_ylast(warp - 2, ring_k);
+        ++ring_k;
+      } else {
+        const uint32_t sel = ybox_sel;
+        ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
+        ybar = bar_yfull(warp - 2, sel);
+        if (++ybox_sel == Cfg::YBOXES) ybox_sel = 0;
+        // the store of the box's previous contents has read it out
+        mbar_wait<false>(bar_yfree(warp - 2, sel), ((ybox_count / Cfg::YBOXES) & 1u) ^ 1u, w);
+        ++ybox_count;
+      }
       __syncwarp();
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -438,7 +468,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_yfull(warp - 2, sel));
+      if (lane == 0) mbar_arrive(ybar);
     };
     // This thread's 64 residual values of box `gg` of a residual stage, as 32 packed bf16 pairs.
     auto load_residual = [&](uint32_t stage_addr, int gg, uint32_t (&r32)[32]) {
@@ -457,6 +487,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       decode_tile(tile, b, mpair0, ncta0);
       const int m0 = mpair0 + static_cast<int>(pm) * 128;
       const int grow = m0 + row;
+      in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles;
       const bool valid = grow < p.M;
 
       // the slot of each sub-tile of this tile, and whether it is computed at all
