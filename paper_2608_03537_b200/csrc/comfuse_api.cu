@@ -151,7 +151,9 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
 comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
   if (d->mask == COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
+  p.M = d->M;
   p.N = d->N;
+  p.K = d->K;
   GemmMaps dummy;
   std::memset(&dummy, 0, sizeof(dummy));
   cudaError_t e = cudaErrorInvalidValue;

@@ -5,6 +5,10 @@
 namespace comfuse {
 
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
+  // Short K: recomputing a score chunk is cheaper than keeping the row block on-chip across a cluster.
+  // COMFUSE_SOFTMAX_CLUSTER=1 forces the cluster kernel where it has an instantiation (for comparisons).
+  static const bool force_cluster = std::getenv("COMFUSE_SOFTMAX_CLUSTER") != nullptr;
+  if (softmax_rows_supported(p) && !force_cluster) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
 #define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
   case n:                                     \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, 0, epw>(maps, p, st);

@@ -40,6 +40,9 @@ struct GemmMaps {
 cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+// Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).
+bool softmax_rows_supported(const FusedParams& p);
+cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 // Plain GEMM, Z = bf16(A.B) through maps.Y, any N that is a multiple of 8.
 cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 

@@ -1,0 +1,399 @@
+// Row softmax behind a SHORT-K GEMM:  P = softmax(alpha * A.B + mask)  over the last dimension, for K so small that
+// computing a score tile twice is cheaper than moving it (the attention-score pattern of Sec. 6.1: K = head size).
+//
+// Stage-Stream view (Sec. 3): the row reduction (max, sum of exponentials) is the stage boundary.  The general kernel
+// keeps a whole row block on-chip by spreading its columns over a cluster and aggregating the partial statistics
+// through distributed shared memory (Sec. 3.2).  With K <= 256 the producer stage is so cheap that this kernel takes
+// the other side of the same trade: one CTA pair owns 256 complete rows, streams the row through tensor memory in
+// 256-column chunks TWICE (MainLoop re-run instead of on-chip residency), and needs no cross-CTA exchange at all:
+//
+//   pass 0   for every live chunk:  S = A.B_chunk (UMMA, cta_group::2)  ->  online (max, sum) per thread
+//   merge    the four threads that share a row combine their partials through shared memory
+//   pass 1   for every live chunk:  S again  ->  P = 2^(S*alpha*log2e - (max + log2 sum))  ->  bf16 box -> TMA store
+//
+// Clusters are pairs, so all SMs are used (wider clusters leave SMs idle), any N fits, and the accumulator slots
+// alternate so that the UMMAs of chunk u+1 run under the epilogue of chunk u.  Under a causal mask, chunks above the
+// diagonal are neither computed nor staged: the store warp writes them from one constant zero box, early, while the
+// epilogue warps are busy with pass 0.
+//
+// Warp roles as in the general kernel: warp 0 TMA producer, warp 1 TMEM allocation + UMMA issue (even CTA),
+// 16 epilogue warps (thread = row; warp e takes lane quarter e % 4 and 64-column group e / 4 of each chunk), last warp
+// issues the TMA stores.  Every wait is bounded.
+#pragma once
+
+#include "fused_params.h"
+#include "sm100_primitives.cuh"
+
+namespace comfuse {
+
+template <int NSTAGES, int YBOXES>
+struct RowSoftmaxCfg {
+  static constexpr int kEpiWarps = 16;
+  static constexpr int kStoreWarp = 2 + kEpiWarps;
+  static constexpr int kThreads = 32 * (kStoreWarp + 1);
+  static constexpr int CHUNK = 256;                          // columns per UMMA and per accumulator slot
+  static constexpr int A_BYTES = 128 * 64 * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + (CHUNK / 2) * 64 * 2;  // A block + this CTA's half of the B chunk
+  static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;
+  static constexpr int OFF_YBUF = NSTAGES * STAGE_BYTES;
+  static constexpr int YBUF_BYTES = kEpiWarps * YBOXES * WARP_BOX_BYTES;
+  static constexpr int OFF_ZERO = OFF_YBUF + YBUF_BYTES;     // constant zero box
+  static constexpr int OFF_PRE = OFF_ZERO + WARP_BOX_BYTES;  // per-row partials of the 4 column groups, two tile parities
+  static constexpr int PRE_BYTES = 2 * 4 * 128 * 8;
+  static constexpr int OFF_BAR = OFF_PRE + PRE_BYTES;
+  static constexpr int NUM_BARS = 2 * NSTAGES + 4 + 1 + 2 * kEpiWarps * YBOXES;
+  static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
+  static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
+  static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+  static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
+  static_assert(NSTAGES >= 2 && NSTAGES <= 8 && YBOXES >= 1 && YBOXES <= 4, "ring and staging depths");
+};
+
+template <int NSTAGES, int YBOXES>
+__global__ void __launch_bounds__(32 * 19, 1)
+softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
+  using Cfg = RowSoftmaxCfg<NSTAGES, YBOXES>;
+  constexpr int CHUNK = Cfg::CHUNK;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  const uint32_t smem_base = smem_u32(smem);
+
+  float2* s_pre = reinterpret_cast<float2*>(smem + Cfg::OFF_PRE);
+  const uint32_t bar_base = smem_base + Cfg::OFF_BAR;
+  auto bar_full = [&](int s) { return bar_base + 8u * s; };                     // K-block stage landed (even CTA)
+  auto bar_empty = [&](int s) { return bar_base + 8u * (NSTAGES + s); };        // stage may be overwritten
+  auto bar_tfull = [&](int a) { return bar_base + 8u * (2 * NSTAGES + a); };    // accumulator slot complete
+  auto bar_tempty = [&](int a) { return bar_base + 8u * (2 * NSTAGES + 2 + a); };  // slot drained by both CTAs (even CTA)
+  const uint32_t bar_drain = bar_base + 8u * (2 * NSTAGES + 4);
+  auto bar_yfull = [&](int e, int k) { return bar_drain + 8u + 8u * (e * YBOXES + k); };
+  auto bar_yfree = [&](int e, int k) { return bar_drain + 8u + 8u * (Cfg::kEpiWarps * YBOXES + e * YBOXES + k); };
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Cfg::OFF_MISC);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::OFF_MISC + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t pm = cluster_ctarank();  // which 128-row block of the pair; rank 0 issues the UMMAs
+  const uint32_t peer = pm ^ 1u;
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
+  const int KB = (p.K + 63) >> 6;
+  const int nch = (p.N + CHUNK - 1) / CHUNK;
+  const int rounds = (p.total_tiles + num_clusters - 1) / num_clusters;
+  const WaitCtx w{s_abort, p.status, p.timeout_ns};
+
+  // -------------------------------------------------------------------------------------------- set-up
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NSTAGES; ++s) {
+      mbar_init(bar_full(s), 2);   // one arrive.expect_tx from each CTA of the pair
+      mbar_init(bar_empty(s), 1);  // one commit from the issuing CTA
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull(a), 1);
+      mbar_init(bar_tempty(a), 2 * Cfg::kEpiWarps);  // one arrival per epilogue warp of both CTAs
+    }
+    mbar_init(bar_drain, 1);
+    for (int e = 0; e < Cfg::kEpiWarps; ++e)
+      for (int k = 0; k < YBOXES; ++k) {
+        mbar_init(bar_yfull(e, k), 1);
+        mbar_init(bar_yfree(e, k), 1);
+      }
+    *s_abort = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(&tmB);
+    prefetch_tensormap(&tmY);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(s_tmem_base), 2 * CHUNK);
+    tmem_relinquish_alloc_permit_pair();
+  }
+  for (int i = threadIdx.x; i < Cfg::WARP_BOX_BYTES / 4; i += Cfg::kThreads) reinterpret_cast<uint32_t*>(smem + Cfg::OFF_ZERO)[i] = 0u;
+  fence_proxy_async_smem();  // the zero box is read by TMA stores
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  cluster_sync_after_init();  // both CTAs' barriers exist before the peer signals them
+  const uint32_t tmem_base = *s_tmem_base;
+
+  // Tile of this cluster in round r.  Tiles are ordered by falling cost (under a causal mask a lower row block has
+  // more live chunks) and dealt to the clusters in alternating direction, so the clusters' sums stay close.
+  auto tile_at = [&](int r, int& b, int& mpair0, int& live_chunks) {
+    const int pos = r * num_clusters + ((r & 1) ? num_clusters - 1 - cluster_id : cluster_id);
+    if (pos >= p.total_tiles) return false;
+    const int mp = p.mpairs - 1 - pos / p.batch;
+    b = pos - (pos / p.batch) * p.batch;
+    mpair0 = mp * 256;
+    live_chunks = p.causal ? (mp + 1 < nch ? mp + 1 : nch) : nch;  // chunk c is live iff c*256 <= mpair0 + 255
+    return true;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int r = 0; r < rounds && ok; ++r) {
+        int b, mpair0, L;
+        if (!tile_at(r, b, mpair0, L)) continue;
+        const int m0 = mpair0 + static_cast<int>(pm) * 128;
+        for (int u = 0; u < 2 * L && ok; ++u) {
+          const int c = u < L ? u : u - L;
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!mbar_wait<false>(bar_empty(stage), phase ^ 1u, w)) { ok = false; break; }  // passes on a fresh barrier
+            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+            const uint32_t full = map_to_cta(bar_full(stage), 0);
+            mbar_arrive_expect_tx_cluster(full, Cfg::STAGE_BYTES);
+            tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
+            // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
+            const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
+            tma_load_3d_pair(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b);
+            tma_load_3d_pair(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b);
+            if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------------------------ UMMA issuer (even CTA)
+    if (lane == 0 && pm == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t slot_uses[2] = {0, 0};
+      uint32_t unit = 0;
+      bool ok = true;
+      constexpr uint32_t idesc = make_idesc_bf16(256, CHUNK, false, true);
+      for (int r = 0; r < rounds && ok; ++r) {
+        int b, mpair0, L;
+        if (!tile_at(r, b, mpair0, L)) continue;
+        for (int u = 0; u < 2 * L && ok; ++u, ++unit) {
+          const int slot = static_cast<int>(unit & 1u);
+          if (!mbar_wait<false>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; break; }
+          ++slot_uses[slot];
+          tcgen05_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + slot * CHUNK;
+          for (int kb = 0; kb < KB; ++kb) {
+            if (!mbar_wait<false>(bar_full(stage), phase, w)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+            const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
+            const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside A's swizzled row, 2048 bytes in B
+              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
+                                (kb | k) != 0 ? 1u : 0u);
+            umma_commit_pair(bar_empty(stage));
+            umma_commit_pair(map_to_cta(bar_empty(stage), peer));
+            if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) {
+            umma_commit_pair(bar_tfull(slot));
+            umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
+          }
+        }
+      }
+      umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
+      mbar_wait<false>(bar_drain, 0, w);
+    }
+  } else if (warp == Cfg::kStoreWarp) {
+    // ------------------------------------------------------------------------------------------ store warp
+    // Lane e mirrors epilogue warp e: zero boxes of the tile's dead chunks first (no hand-shake: the zero box is
+    // constant), then, per live chunk, wait until the box is staged, store it, hand the staging box back.
+    if (lane < Cfg::kEpiWarps) {
+      const int e = lane;
+      const int q = (e + 2) & 3;
+      const int h = e >> 2;
+      constexpr int D = YBOXES - 1;
+      const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + e * YBOXES * Cfg::WARP_BOX_BYTES;
+      uint32_t n = 0;
+      bool ok = true;
+      for (int r = 0; r < rounds && ok; ++r) {
+        int b, mpair0, L;
+        if (!tile_at(r, b, mpair0, L)) continue;
+        const int y0 = mpair0 + static_cast<int>(pm) * 128 + q * 32;
+        for (int c = L; c < nch; ++c) {
+          const int col = c * CHUNK + h * 64;
+          if (col < p.N) tma_store_3d(&tmY, smem_base + Cfg::OFF_ZERO, col, y0, b);
+        }
+        for (int c = 0; c < L; ++c) {
+          const int col = c * CHUNK + h * 64;
+          if (col >= p.N) break;
+          const uint32_t sel = n % YBOXES;
+          if (!mbar_wait<false>(bar_yfull(e, sel), (n / YBOXES) & 1u, w)) { ok = false; break; }
+          tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, y0, b);
+          tma_store_commit();
+          if (n >= static_cast<uint32_t>(D)) {
+            tma_store_wait_read<D>();
+            mbar_arrive(bar_yfree(e, (n - D) % YBOXES));
+          }
+          ++n;
+        }
+      }
+      tma_store_commit();
+      tma_store_wait_read<0>();  // shared memory must outlive the last stores' reads (the stores complete at kernel end)
+    }
+  } else {
+    // ------------------------------------------------------------------------------------------ epilogue warps
+    const int e = warp - 2;
+    const int q = warp & 3;  // TMEM lane quarter this warp may touch: rows 32q .. 32q+31 of the CTA's row block
+    const int h = e >> 2;    // the 64-column group of every chunk this warp takes
+    const int row = q * 32 + lane;
+    const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
+    const uint32_t tempty_leader = map_to_cta(bar_tempty(0), 0);
+    const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + e * YBOXES * Cfg::WARP_BOX_BYTES;
+    uint32_t slot_uses[2] = {0, 0};
+    uint32_t unit = 0, nbox = 0, tile_par = 0;
+    // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
+    const float sc = p.alpha * 1.4426950408889634f;
+
+    auto wait_slot = [&](int slot) {
+      mbar_wait<false>(bar_tfull(slot), slot_uses[slot] & 1u, w);
+      ++slot_uses[slot];
+      __syncwarp();
+      tcgen05_fence_after_sync();
+    };
+    auto release_slot = [&](int slot) {
+      tcgen05_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster_noflush(tempty_leader + 8u * slot);
+    };
+
+    for (int r = 0; r < rounds; ++r) {
+      int b, mpair0, L;
+      if (!tile_at(r, b, mpair0, L)) continue;
+      const int m0 = mpair0 + static_cast<int>(pm) * 128;
+      const int grow = m0 + row;
+      // last live column of this thread's row, and of the warp's first / last row (fragment classification must be
+      // uniform over the warp so that the warp-wide TMEM loads stay convergent)
+      const int lim = p.causal ? (grow < p.N - 1 ? grow : p.N - 1) : p.N - 1;
+      const int wrow0 = m0 + q * 32;
+      const int lim_lo = p.causal ? (wrow0 < p.N - 1 ? wrow0 : p.N - 1) : p.N - 1;
+      const int lim_hi = p.causal ? (wrow0 + 31 < p.N - 1 ? wrow0 + 31 : p.N - 1) : p.N - 1;
+      // 2 = all 32 columns live for all 32 rows, 0 = none live for any row, 1 = mixed
+      auto frag_state = [&](int col0) { return col0 + 31 <= lim_lo ? 2 : (col0 > lim_hi ? 0 : 1); };
+
+      // ---------------- pass 0: online (max, sum of 2^(t - max)) over this thread's columns of every live chunk
+      float m_run = -INFINITY, s_run = 0.f;
+      for (int c = 0; c < L; ++c, ++unit) {
+        const int slot = static_cast<int>(unit & 1u);
+        wait_slot(slot);
+        const uint32_t taddr = tmem_base + lane_sel + slot * CHUNK + h * 64;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int col0 = c * CHUNK + h * 64 + half * 32;
+          const int st = frag_state(col0);
+          if (st == 0) continue;
+          uint32_t v[32];
+          tmem_ld_32cols(taddr + half * 32, v);
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
+            if (st != 2) {
+              if (col0 + j > lim) t0 = -INFINITY;
+              if (col0 + j + 1 > lim) t1 = -INFINITY;
+            }
+            v[j] = __float_as_uint(t0);
+            v[j + 1] = __float_as_uint(t1);
+            mx0 = fmaxf(mx0, t0);
+            mx1 = fmaxf(mx1, t1);
+          }
+          const float m_new = fmaxf(m_run, fmaxf(mx0, mx1));
+          if (m_new != -INFINITY) {  // else every column seen so far is masked for this row
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              s0 += ex2_approx(__uint_as_float(v[j]) - m_new);
+              s1 += ex2_approx(__uint_as_float(v[j + 1]) - m_new);
+            }
+            s_run = s_run * ex2_approx(m_run - m_new) + (s0 + s1);
+            m_run = m_new;
+          }
+        }
+        release_slot(slot);
+      }
+      // ---------------- merge the four column groups of the row (they live in the four warps of this lane quarter)
+      float2* pre = s_pre + tile_par * 512;
+      tile_par ^= 1u;
+      pre[h * 128 + row] = make_float2(m_run, s_run);
+      named_barrier_sync(1 + q, 128);
+      float m_row = -INFINITY, s_row = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 o = pre[i * 128 + row];
+        const float m_new = fmaxf(m_row, o.x);
+        if (m_new != -INFINITY) {
+          s_row = s_row * ex2_approx(m_row - m_new) + o.y * ex2_approx(o.x - m_new);
+          m_row = m_new;
+        }
+      }
+      // P = 2^(t - off); a row without a live column (cannot happen under the causal mask) is all zero: 2^(-inf)
+      const float off = s_row > 0.f ? m_row + __log2f(s_row) : INFINITY;
+
+      // ---------------- pass 1: the scores again, normalised, rounded once, staged and stored
+      for (int c = 0; c < L; ++c, ++unit) {
+        const int slot = static_cast<int>(unit & 1u);
+        wait_slot(slot);
+        const uint32_t taddr = tmem_base + lane_sel + slot * CHUNK + h * 64;
+        const int colg = c * CHUNK + h * 64;
+        uint32_t pk[32];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int col0 = colg + half * 32;
+          const int st = frag_state(col0);
+          if (st == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[half * 16 + j] = 0u;
+          } else {
+            uint32_t v[32];
+            tmem_ld_32cols(taddr + half * 32, v);
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              const float2 t01 = fma2(f2_from_bits(v[j], v[j + 1]), splat2(sc), splat2(-off));
+              float e0 = ex2_approx(t01.x), e1 = ex2_approx(t01.y);
+              if (st != 2) {
+                if (col0 + j > lim) e0 = 0.f;
+                if (col0 + j + 1 > lim) e1 = 0.f;
+              }
+              pk[half * 16 + j / 2] = pack_bf16x2_rn(e0, e1);
+            }
+          }
+        }
+        release_slot(slot);
+        if (colg < p.N) {
+          const uint32_t sel = nbox % YBOXES;
+          const uint32_t ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
+          // the store of the box's previous contents has read it out
+          mbar_wait<false>(bar_yfree(e, sel), ((nbox / YBOXES) & 1u) ^ 1u, w);
+          ++nbox;
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t a = ybox + static_cast<uint32_t>(lane * 128 + ((i ^ (lane & 7)) << 4));  // 128-byte swizzle
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                         "r"(pk[4 * i + 3])
+                         : "memory");
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_yfull(e, sel));
+        }
+      }
+    }
+  }
+
+  // -------------------------------------------------------------------------------------------- teardown
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();  // the peer may no longer signal this CTA's barriers or write its TMEM
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, 2 * CHUNK);
+  }
+}
+
+}  // namespace comfuse

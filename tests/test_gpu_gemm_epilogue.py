@@ -114,10 +114,22 @@ SOFTMAX_CASES = [
     (2, 256, 256, 64, True),
     (3, 512, 512, 64, True),
     (2, 1024, 1024, 32, True),
-    (2, 2048, 2048, 64, True),     # the 8-CTA cluster instantiation of the attention-score configuration
+    (2, 2048, 2048, 64, True),     # the attention-score configuration (short K: row kernel, chunks computed twice)
     (1, 300, 512, 64, False),      # no mask, ragged M
     (2, 200, 2048, 40, False),
     (1, 4096, 4096, 16, True),
+    (1, 1000, 1000, 64, True),     # row kernel: N not a multiple of the 64-column box, diagonal inside a chunk
+    (2, 136, 1096, 128, False),    # row kernel: two K blocks, ragged last chunk
+    (1, 384, 8192, 256, False),    # row kernel: N beyond what one cluster can hold, four K blocks, odd row-block count
+    (37, 256, 256, 8, True),       # row kernel: more tiles than one round, minimal K
+    # K > 256: the cluster kernel (row block resident on-chip, statistics exchanged through distributed shared memory)
+    (2, 256, 256, 320, True),
+    (3, 512, 512, 320, True),
+    (2, 1024, 1024, 264, True),
+    (2, 2048, 2048, 320, True),
+    (1, 300, 512, 320, False),
+    (2, 200, 2048, 272, False),
+    (1, 4096, 4096, 264, True),
 ]
 
 
