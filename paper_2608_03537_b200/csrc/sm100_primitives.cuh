@@ -153,6 +153,10 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src
                "r"(x), "r"(y), "r"(z)
                : "memory");
 }
+// Untiled bulk copy shared -> global (both addresses 16-byte aligned, size a multiple of 16); joins the thread's bulk group.
+__device__ __forceinline__ void bulk_store_1d(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int kPending>
 __device__ __forceinline__ void tma_store_wait_read() {
@@ -295,6 +299,12 @@ __device__ __forceinline__ float tanh_approx(float x) {
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Three-input maximum (one instruction on sm_100).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
 // Packed fp32x2 arithmetic (one instruction for two lanes of a float2): halves the issue slots of the epilogue math.

@@ -13,12 +13,12 @@
 //
 // Clusters are pairs, so all SMs are used (wider clusters leave SMs idle), any N fits, and the accumulator slots
 // alternate so that the UMMAs of chunk u+1 run under the epilogue of chunk u.  Under a causal mask, chunks above the
-// diagonal are neither computed nor staged: the store warp writes them from one constant zero box, early, while the
-// epilogue warps are busy with pass 0.
+// diagonal are neither computed nor staged: the epilogue warps write their zeros with plain stores, a few rows after
+// every chunk pass, from a cursor that runs through the cluster's tiles on its own.
 //
 // Warp roles as in the general kernel: warp 0 TMA producer, warp 1 TMEM allocation + UMMA issue (even CTA),
 // 16 epilogue warps (thread = row; warp e takes lane quarter e % 4 and 64-column group e / 4 of each chunk), last warp
-// issues the TMA stores.  Every wait is bounded.
+// issues the TMA stores of the staged boxes.  Every wait is bounded.
 #pragma once
 
 #include "fused_params.h"
@@ -30,7 +30,9 @@ template <int NSTAGES, int YBOXES>
 struct RowSoftmaxCfg {
   static constexpr int kEpiWarps = 16;
   static constexpr int kStoreWarp = 2 + kEpiWarps;
-  static constexpr int kThreads = 32 * (kStoreWarp + 1);
+  static constexpr int kZeroWarp = kStoreWarp + 1;
+  static constexpr int kThreads = 32 * (kZeroWarp + 1);
+  static constexpr int ZERO_TMA_LANES = 8;                   // zero boxes in flight per SM
   static constexpr int CHUNK = 256;                          // columns per UMMA and per accumulator slot
   static constexpr int A_BYTES = 128 * 64 * 2;
   static constexpr int STAGE_BYTES = A_BYTES + (CHUNK / 2) * 64 * 2;  // A block + this CTA's half of the B chunk
@@ -50,7 +52,7 @@ struct RowSoftmaxCfg {
 };
 
 template <int NSTAGES, int YBOXES>
-__global__ void __launch_bounds__(32 * 19, 1)
+__global__ void __launch_bounds__(32 * 20, 1)
 softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
   using Cfg = RowSoftmaxCfg<NSTAGES, YBOXES>;
@@ -141,19 +143,19 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!tile_at(r, b, mpair0, L)) continue;
         const int m0 = mpair0 + static_cast<int>(pm) * 128;
         for (int u = 0; u < 2 * L && ok; ++u) {
-          const int c = u < L ? u : u - L;
-          for (int kb = 0; kb < KB; ++kb) {
-            if (!mbar_wait<false>(bar_empty(stage), phase ^ 1u, w)) { ok = false; break; }  // passes on a fresh barrier
-            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
-            const uint32_t full = map_to_cta(bar_full(stage), 0);
-            mbar_arrive_expect_tx_cluster(full, Cfg::STAGE_BYTES);
-            tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
-            // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
-            const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
-            tma_load_3d_pair(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b);
-            tma_load_3d_pair(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b);
-            if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
-          }
+        const int c = u < L ? u : u - L;  // pass 0 over the live chunks, then pass 1
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait<false>(bar_empty(stage), phase ^ 1u, w)) { ok = false; break; }  // passes on a fresh barrier
+          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+          const uint32_t full = map_to_cta(bar_full(stage), 0);
+          mbar_arrive_expect_tx_cluster(full, Cfg::STAGE_BYTES);
+          tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
+          // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
+          const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
+          tma_load_3d_pair(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b);
+          tma_load_3d_pair(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b);
+          if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
+        }
         }
       }
     }
@@ -164,44 +166,44 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t phase = 0;
       uint32_t slot_uses[2] = {0, 0};
       uint32_t unit = 0;
-      bool ok = true;
       constexpr uint32_t idesc = make_idesc_bf16(256, CHUNK, false, true);
-      for (int r = 0; r < rounds && ok; ++r) {
+      bool ok = true;
+      uint32_t total_units = 0;
+      for (int r = 0; r < rounds; ++r) {
         int b, mpair0, L;
-        if (!tile_at(r, b, mpair0, L)) continue;
-        for (int u = 0; u < 2 * L && ok; ++u, ++unit) {
-          const int slot = static_cast<int>(unit & 1u);
-          if (!mbar_wait<false>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) { ok = false; break; }
-          ++slot_uses[slot];
+        if (tile_at(r, b, mpair0, L)) total_units += 2u * L;
+      }
+      while (ok && unit < total_units) {
+        const int slot = static_cast<int>(unit & 1u);
+        ++unit;
+        if (!mbar_wait<false>(bar_tempty(slot), (slot_uses[slot] & 1u) ^ 1u, w)) break;
+        ++slot_uses[slot];
+        tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + slot * CHUNK;
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait<false>(bar_full(stage), phase, w)) { ok = false; break; }
           tcgen05_fence_after_sync();
-          const uint32_t d_tmem = tmem_base + slot * CHUNK;
-          for (int kb = 0; kb < KB; ++kb) {
-            if (!mbar_wait<false>(bar_full(stage), phase, w)) { ok = false; break; }
-            tcgen05_fence_after_sync();
-            const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
-            const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
-            const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
+          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+          const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
+          const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside A's swizzled row, 2048 bytes in B
-              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
-                                (kb | k) != 0 ? 1u : 0u);
-            umma_commit_pair(bar_empty(stage));
-            umma_commit_pair(map_to_cta(bar_empty(stage), peer));
-            if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
-          }
-          if (ok) {
-            umma_commit_pair(bar_tfull(slot));
-            umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
-          }
+          for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside A's swizzled row, 2048 bytes in B
+            umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
+                              (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(bar_empty(stage));
+          umma_commit_pair(map_to_cta(bar_empty(stage), peer));
+          if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
         }
+        if (!ok) break;
+        umma_commit_pair(bar_tfull(slot));
+        umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
       }
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
       mbar_wait<false>(bar_drain, 0, w);
     }
   } else if (warp == Cfg::kStoreWarp) {
     // ------------------------------------------------------------------------------------------ store warp
-    // Lane e mirrors epilogue warp e: zero boxes of the tile's dead chunks first (no hand-shake: the zero box is
-    // constant), then, per live chunk, wait until the box is staged, store it, hand the staging box back.
+    // Lane e mirrors epilogue warp e: per live chunk, wait until the box is staged, store it, hand the staging box back.
     if (lane < Cfg::kEpiWarps) {
       const int e = lane;
       const int q = (e + 2) & 3;
@@ -213,27 +215,51 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int r = 0; r < rounds && ok; ++r) {
         int b, mpair0, L;
         if (!tile_at(r, b, mpair0, L)) continue;
-        const int y0 = mpair0 + static_cast<int>(pm) * 128 + q * 32;
-        for (int c = L; c < nch; ++c) {
-          const int col = c * CHUNK + h * 64;
-          if (col < p.N) tma_store_3d(&tmY, smem_base + Cfg::OFF_ZERO, col, y0, b);
-        }
         for (int c = 0; c < L; ++c) {
-          const int col = c * CHUNK + h * 64;
-          if (col >= p.N) break;
-          const uint32_t sel = n % YBOXES;
-          if (!mbar_wait<false>(bar_yfull(e, sel), (n / YBOXES) & 1u, w)) { ok = false; break; }
-          tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, y0, b);
-          tma_store_commit();
-          if (n >= static_cast<uint32_t>(D)) {
-            tma_store_wait_read<D>();
-            mbar_arrive(bar_yfree(e, (n - D) % YBOXES));
-          }
-          ++n;
+        const int col = c * CHUNK + h * 64;
+        if (col >= p.N) break;
+        const uint32_t sel = n % YBOXES;
+        if (!mbar_wait<false>(bar_yfull(e, sel), (n / YBOXES) & 1u, w)) { ok = false; break; }
+#ifdef COMFUSE_TRACE
+        if (!(p.trace_flags & 1))
+#endif
+        tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, mpair0 + static_cast<int>(pm) * 128 + q * 32, b);
+        tma_store_commit();
+        if (n >= static_cast<uint32_t>(D)) {
+          tma_store_wait_read<D>();
+          mbar_arrive(bar_yfree(e, (n - D) % YBOXES));
+        }
+        ++n;
         }
       }
-      tma_store_commit();
       tma_store_wait_read<0>();  // shared memory must outlive the last stores' reads (the stores complete at kernel end)
+    }
+  } else if (warp == Cfg::kZeroWarp) {
+    // ------------------------------------------------------------------------------------------ zero-box warp
+    // The chunks above the causal diagonal hold zeros and depend on nothing.  A few lanes, each with one TMA store of a
+    // constant zero box in flight, walk them with a cursor of their own, independent of the epilogue (asynchronous
+    // stores: plain stores would share the SM's memory-instruction queue with the epilogue's exponentials and
+    // shared-memory traffic).  Few boxes in flight, so that a staged box never queues far behind zeros.
+    if (lane < Cfg::ZERO_TMA_LANES && p.causal) {
+      uint32_t k = 0;
+      for (int r = 0; r < rounds; ++r) {
+        int b, mpair0, L;
+        if (!tile_at(r, b, mpair0, L)) continue;
+        const int y0 = mpair0 + static_cast<int>(pm) * 128;
+        for (int c = L; c < nch; ++c)
+          for (int i = 0; i < 16; ++i, ++k) {
+            if (k % Cfg::ZERO_TMA_LANES != static_cast<uint32_t>(lane)) continue;
+            const int col = c * CHUNK + (i >> 2) * 64;
+            if (col >= p.N) continue;
+            tma_store_wait_all();
+#ifdef COMFUSE_TRACE
+            if (!(p.trace_flags & 4))
+#endif
+            tma_store_3d(&tmY, smem_base + Cfg::OFF_ZERO, col, y0 + (i & 3) * 32, b);
+            tma_store_commit();
+          }
+      }
+      tma_store_wait_read<0>();
     }
   } else {
     // ------------------------------------------------------------------------------------------ epilogue warps
@@ -249,11 +275,22 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
     const float sc = p.alpha * 1.4426950408889634f;
 
+#ifdef COMFUSE_TRACE
+    int trace_ix = 0;
+#define ROWS_TRACE_POINT()                                                                             \
+  do {                                                                                                 \
+    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 60) p.trace[trace_ix++] = globaltimer_ns(); \
+  } while (0)
+#else
+#define ROWS_TRACE_POINT() do { } while (0)
+#endif
     auto wait_slot = [&](int slot) {
+      ROWS_TRACE_POINT();
       mbar_wait<false>(bar_tfull(slot), slot_uses[slot] & 1u, w);
       ++slot_uses[slot];
       __syncwarp();
       tcgen05_fence_after_sync();
+      ROWS_TRACE_POINT();
     };
     auto release_slot = [&](int slot) {
       tcgen05_fence_before_sync();
@@ -264,122 +301,138 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int r = 0; r < rounds; ++r) {
       int b, mpair0, L;
       if (!tile_at(r, b, mpair0, L)) continue;
-      const int m0 = mpair0 + static_cast<int>(pm) * 128;
-      const int grow = m0 + row;
-      // last live column of this thread's row, and of the warp's first / last row (fragment classification must be
-      // uniform over the warp so that the warp-wide TMEM loads stay convergent)
-      const int lim = p.causal ? (grow < p.N - 1 ? grow : p.N - 1) : p.N - 1;
-      const int wrow0 = m0 + q * 32;
-      const int lim_lo = p.causal ? (wrow0 < p.N - 1 ? wrow0 : p.N - 1) : p.N - 1;
-      const int lim_hi = p.causal ? (wrow0 + 31 < p.N - 1 ? wrow0 + 31 : p.N - 1) : p.N - 1;
-      // 2 = all 32 columns live for all 32 rows, 0 = none live for any row, 1 = mixed
-      auto frag_state = [&](int col0) { return col0 + 31 <= lim_lo ? 2 : (col0 > lim_hi ? 0 : 1); };
+      float m_run = -INFINITY, s_run = 0.f;  // pass 0: this thread's running maximum and sum of 2^(t - max)
+      float off = INFINITY;                  // pass 1: P = 2^(t - off)
+      for (int u = 0; u < 2 * L; ++u) {
+        {
+          const int pass = u < L ? 0 : 1, c = u < L ? u : u - L;
+          const int m0 = mpair0 + static_cast<int>(pm) * 128;
+          const int grow = m0 + row;
+          // last live column of this thread's row, and of the warp's first / last row (fragment classification must be
+          // uniform over the warp so that the warp-wide TMEM loads stay convergent)
+          const int lim = p.causal ? (grow < p.N - 1 ? grow : p.N - 1) : p.N - 1;
+          const int wrow0 = m0 + q * 32;
+          const int lim_lo = p.causal ? (wrow0 < p.N - 1 ? wrow0 : p.N - 1) : p.N - 1;
+          const int lim_hi = p.causal ? (wrow0 + 31 < p.N - 1 ? wrow0 + 31 : p.N - 1) : p.N - 1;
+          // 2 = all 32 columns live for all 32 rows, 0 = none live for any row, 1 = mixed
+          auto frag_state = [&](int col0) { return col0 + 31 <= lim_lo ? 2 : (col0 > lim_hi ? 0 : 1); };
 
-      // ---------------- pass 0: online (max, sum of 2^(t - max)) over this thread's columns of every live chunk
-      float m_run = -INFINITY, s_run = 0.f;
-      for (int c = 0; c < L; ++c, ++unit) {
-        const int slot = static_cast<int>(unit & 1u);
-        wait_slot(slot);
-        const uint32_t taddr = tmem_base + lane_sel + slot * CHUNK + h * 64;
+          const int slot = static_cast<int>(unit & 1u);
+          ++unit;
+          wait_slot(slot);
+          const uint32_t taddr = tmem_base + lane_sel + slot * CHUNK + h * 64;
+          const int colg = c * CHUNK + h * 64;
+          if (pass == 0) {
+            // ---------------- pass 0: online (max, sum of 2^(t - max)) over this thread's columns of the chunk
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int col0 = c * CHUNK + h * 64 + half * 32;
-          const int st = frag_state(col0);
-          if (st == 0) continue;
-          uint32_t v[32];
-          tmem_ld_32cols(taddr + half * 32, v);
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+            for (int half = 0; half < 2; ++half) {
+              const int col0 = colg + half * 32;
+              const int st = frag_state(col0);
+              if (st == 0) continue;
+              uint32_t v[32];
+              tmem_ld_32cols(taddr + half * 32, v);
+              float2 tv[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
-            if (st != 2) {
-              if (col0 + j > lim) t0 = -INFINITY;
-              if (col0 + j + 1 > lim) t1 = -INFINITY;
-            }
-            v[j] = __float_as_uint(t0);
-            v[j + 1] = __float_as_uint(t1);
-            mx0 = fmaxf(mx0, t0);
-            mx1 = fmaxf(mx1, t1);
-          }
-          const float m_new = fmaxf(m_run, fmaxf(mx0, mx1));
-          if (m_new != -INFINITY) {  // else every column seen so far is masked for this row
-            float s0 = 0.f, s1 = 0.f;
+              for (int j = 0; j < 16; ++j) tv[j] = mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc));
+              if (st != 2) {  // the fragment crosses the diagonal (or the end of the row): rare, kept out of the main path
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              s0 += ex2_approx(__uint_as_float(v[j]) - m_new);
-              s1 += ex2_approx(__uint_as_float(v[j + 1]) - m_new);
-            }
-            s_run = s_run * ex2_approx(m_run - m_new) + (s0 + s1);
-            m_run = m_new;
-          }
-        }
-        release_slot(slot);
-      }
-      // ---------------- merge the four column groups of the row (they live in the four warps of this lane quarter)
-      float2* pre = s_pre + tile_par * 512;
-      tile_par ^= 1u;
-      pre[h * 128 + row] = make_float2(m_run, s_run);
-      named_barrier_sync(1 + q, 128);
-      float m_row = -INFINITY, s_row = 0.f;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 o = pre[i * 128 + row];
-        const float m_new = fmaxf(m_row, o.x);
-        if (m_new != -INFINITY) {
-          s_row = s_row * ex2_approx(m_row - m_new) + o.y * ex2_approx(o.x - m_new);
-          m_row = m_new;
-        }
-      }
-      // P = 2^(t - off); a row without a live column (cannot happen under the causal mask) is all zero: 2^(-inf)
-      const float off = s_row > 0.f ? m_row + __log2f(s_row) : INFINITY;
-
-      // ---------------- pass 1: the scores again, normalised, rounded once, staged and stored
-      for (int c = 0; c < L; ++c, ++unit) {
-        const int slot = static_cast<int>(unit & 1u);
-        wait_slot(slot);
-        const uint32_t taddr = tmem_base + lane_sel + slot * CHUNK + h * 64;
-        const int colg = c * CHUNK + h * 64;
-        uint32_t pk[32];
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int col0 = colg + half * 32;
-          const int st = frag_state(col0);
-          if (st == 0) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) pk[half * 16 + j] = 0u;
-          } else {
-            uint32_t v[32];
-            tmem_ld_32cols(taddr + half * 32, v);
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              const float2 t01 = fma2(f2_from_bits(v[j], v[j + 1]), splat2(sc), splat2(-off));
-              float e0 = ex2_approx(t01.x), e1 = ex2_approx(t01.y);
-              if (st != 2) {
-                if (col0 + j > lim) e0 = 0.f;
-                if (col0 + j + 1 > lim) e1 = 0.f;
+                for (int j = 0; j < 16; ++j) {
+                  if (col0 + 2 * j > lim) tv[j].x = -INFINITY;
+                  if (col0 + 2 * j + 1 > lim) tv[j].y = -INFINITY;
+                }
               }
-              pk[half * 16 + j / 2] = pack_bf16x2_rn(e0, e1);
+              float mx0 = m_run, mx1 = -INFINITY;
+#pragma unroll
+              for (int j = 0; j < 16; j += 2) {
+                mx0 = max3(mx0, tv[j].x, tv[j].y);
+                mx1 = max3(mx1, tv[j + 1].x, tv[j + 1].y);
+              }
+              const float m_new = fmaxf(mx0, mx1);
+              if (st == 2 || m_new != -INFINITY) {  // else every column seen so far is masked for this row
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                const float2 neg_m = splat2(-m_new);
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                  const float2 d0 = add2(tv[j], neg_m), d1 = add2(tv[j + 1], neg_m);
+                  acc0 = add2(acc0, make_float2(ex2_approx(d0.x), ex2_approx(d0.y)));
+                  acc1 = add2(acc1, make_float2(ex2_approx(d1.x), ex2_approx(d1.y)));
+                }
+                const float2 acc = add2(acc0, acc1);
+                s_run = fmaf(s_run, ex2_approx(m_run - m_new), acc.x + acc.y);
+                m_run = m_new;
+              }
+            }
+            release_slot(slot);
+          } else {
+            // ---------------- pass 1: the scores again, normalised, rounded once, staged and stored
+            uint32_t pk[32];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const int col0 = colg + half * 32;
+              const int st = frag_state(col0);
+              if (st == 0) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = 0u;
+              } else {
+                uint32_t v[32];
+                tmem_ld_32cols(taddr + half * 32, v);
+                float2 ev[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), splat2(-off));
+                  ev[j] = make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
+                }
+                if (st != 2) {  // crosses the diagonal (or the end of the row)
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) {
+                    if (col0 + 2 * j > lim) ev[j].x = 0.f;
+                    if (col0 + 2 * j + 1 > lim) ev[j].y = 0.f;
+                  }
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_bf16x2_rn(ev[j]);
+              }
+            }
+            release_slot(slot);
+            if (colg < p.N) {
+              const uint32_t sel = nbox % YBOXES;
+              const uint32_t ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
+              // the store of the box's previous contents has read it out
+              mbar_wait<false>(bar_yfree(e, sel), ((nbox / YBOXES) & 1u) ^ 1u, w);
+              ++nbox;
+              __syncwarp();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const uint32_t a = ybox + static_cast<uint32_t>(lane * 128 + ((i ^ (lane & 7)) << 4));  // 128-byte swizzle
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]),
+                             "r"(pk[4 * i + 2]), "r"(pk[4 * i + 3])
+                             : "memory");
+              }
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_yfull(e, sel));
             }
           }
         }
-        release_slot(slot);
-        if (colg < p.N) {
-          const uint32_t sel = nbox % YBOXES;
-          const uint32_t ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
-          // the store of the box's previous contents has read it out
-          mbar_wait<false>(bar_yfree(e, sel), ((nbox / YBOXES) & 1u) ^ 1u, w);
-          ++nbox;
-          __syncwarp();
+        if (u == L - 1) {
+          // ---------------- pass 0 of the tile is complete: merge the four column groups of the row (they live in the
+          // four warps of this lane quarter); the result serves the tile's pass 1, which starts with the next unit
+          float2* pre = s_pre + tile_par * 512;
+          tile_par ^= 1u;
+          pre[h * 128 + row] = make_float2(m_run, s_run);
+          named_barrier_sync(1 + q, 128);
+          float m_row = -INFINITY, s_row = 0.f;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint32_t a = ybox + static_cast<uint32_t>(lane * 128 + ((i ^ (lane & 7)) << 4));  // 128-byte swizzle
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                         "r"(pk[4 * i + 3])
-                         : "memory");
+          for (int i = 0; i < 4; ++i) {
+            const float2 o = pre[i * 128 + row];
+            const float m_new = fmaxf(m_row, o.x);
+            if (m_new != -INFINITY) {
+              s_row = s_row * ex2_approx(m_row - m_new) + o.y * ex2_approx(o.x - m_new);
+              m_row = m_new;
+            }
           }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_yfull(e, sel));
+          // a row without a live column (cannot happen under the causal mask) is all zero: 2^(-inf)
+          off = s_row > 0.f ? m_row + __log2f(s_row) : INFINITY;
         }
       }
     }
