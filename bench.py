@@ -34,7 +34,7 @@ METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
 WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
 # captures summarised under profiles/, in bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 69_471_744, "c3": None, "c4": None, "c5": 8_726_528}
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": 69_505_280, "c3": 270_358_528, "c4": 550_356_992, "c5": 8_714_496}
 
 
 def load_peaks():
@@ -343,7 +343,12 @@ def run_comfuse(args):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
     roof["peak_source"] = f"of {peaks['source']} (burst figure, kernel timed alone)"
-    roof["kernel"] = "fused_gemm_kernel" if w.kind != wl.KIND_B2B_MLP_LAYERNORM else "b2b_gemm_kernel"
+    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        roof["kernel"] = "b2b_pair_kernel"
+    elif w.kind == wl.KIND_SCALE_MASK_SOFTMAX and d["K"] <= 256:
+        roof["kernel"] = "softmax_rows_kernel"      # short K: score chunks computed twice, no cluster exchange
+    else:
+        roof["kernel"] = "fused_pair_kernel"
     roof["algorithmic_flops_per_launch"] = flops
     roof["algorithmic_bytes_per_launch"] = bytes_min
     roof["roofline_us"] = max(t_tensor, t_hbm) * 1e6
