@@ -88,7 +88,12 @@ typedef struct {
   int32_t* row_argmax;
 } comfuse_epilogue_args_t;
 
-/* Bytes of caller-provided workspace the described call needs (0 for fused calls). */
+/* Bytes of caller-provided workspace the described call needs.  Fused calls need none, except LayerNorm / RMSNorm rows
+ * wider than the largest cluster can hold on-chip (N > 4096; supported for N a multiple of 4096 up to 65536).  Those run as
+ * two kernels: the fused kernel finishes stage 1 per 4096-column block, stores the un-normalised row (rounded to bf16) in
+ * Y and one partial statistic per row and block in the workspace (batch * M * N/4096 * 8 bytes); a second kernel merges the
+ * partials and rescales the row in place (the un-normalised values are materialised because they no longer fit on-chip,
+ * Sec. 2.2).  Their results carry one extra bf16 rounding, like those of the unfused path. */
 comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes);
 
 /* GEMM -> subgraph (Sec. 3).  A, B inputs; Y output [batch, M, N] bf16, rounded once, at the store. */

@@ -147,7 +147,8 @@ def workspace_size(desc: GemmDesc) -> int:
 def gemm_epilogue(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=None, mask_tensor=None, row_max=None,
                   row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, workspace=None, stream=None):
     """Enqueue Y = subgraph(alpha * A.B) on the current (or given) stream.  Tensors are CUDA bf16 (row_max fp32,
-    row_argmax int32).  ``workspace`` is a CUDA uint8 tensor of at least workspace_size(desc) bytes (unfused path)."""
+    row_argmax int32).  ``workspace`` is a CUDA uint8 tensor of at least workspace_size(desc) bytes (unfused path, and fused LayerNorm /
+    RMSNorm rows wider than 4096 columns)."""
     d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused)
     args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())

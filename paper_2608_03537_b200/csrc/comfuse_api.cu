@@ -154,6 +154,7 @@ comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
   p.M = d->M;
   p.N = d->N;
   p.K = d->K;
+  p.wide = wide_row_blocks(kind_to_epi(d->kind), d->N) > 0;
   GemmMaps dummy;
   std::memset(&dummy, 0, sizeof(dummy));
   cudaError_t e = cudaErrorInvalidValue;
@@ -196,7 +197,8 @@ comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t*
   if (desc->fused) {
     s = fused_supported(desc);
     if (s != COMFUSE_OK) return s;
-    *bytes = 0;
+    // rows wider than one cluster: one partial statistic (8 bytes) per row and 4096-column block
+    *bytes = static_cast<size_t>(wide_row_blocks(kind_to_epi(desc->kind), desc->N)) * desc->batch * desc->M * sizeof(float2);
   } else {
     if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
     *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
@@ -273,10 +275,29 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
     p.Y = static_cast<uint16_t*>(Y);
     p.ldy = desc->ldy; p.batch_stride_y = bsy;
     p.row_max = a.row_max; p.row_argmax = a.row_argmax;
+    const int wide_blocks = wide_row_blocks(epi, desc->N);
+    if (wide_blocks) {  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace
+      p.wide = 1;
+      p.nblocks = wide_blocks;
+      p.wide_partials = static_cast<float2*>(workspace);
+      p.gamma = nullptr;
+      p.beta = nullptr;
+    }
     switch (epi) {
       case EPI_LN: e = launch_fused_layernorm(maps, p, st, false); break;
       case EPI_RMS_MAX: e = launch_fused_rmsnorm_max(maps, p, st, false); break;
       default: e = launch_fused_softmax(maps, p, st, false); break;
+    }
+    if (e == cudaSuccess && wide_blocks) {  // second kernel: merge the blocks' statistics, rescale the row in place
+      RowParams r = {};
+      r.batch = desc->batch; r.M = desc->M; r.N = desc->N;
+      r.gamma = static_cast<const uint16_t*>(a.gamma);
+      r.beta = static_cast<const uint16_t*>(a.beta);
+      r.eps = desc->eps;
+      r.Y = static_cast<uint16_t*>(Y);
+      r.ldy = desc->ldy; r.batch_stride_y = bsy;
+      r.row_max = a.row_max; r.row_argmax = a.row_argmax;
+      e = launch_wide_row_finish(epi, r, p.wide_partials, wide_blocks, st);
     }
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }

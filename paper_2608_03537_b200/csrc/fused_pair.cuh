@@ -200,11 +200,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   }
   if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
     // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once
+    // (wide rows: the bias of the tile's column block is loaded per tile by the epilogue warps, gamma/beta are identity)
     const int c0 = crank * BN;
     for (int i = threadIdx.x; i < BN; i += Cfg::kThreads) {
       const int c = c0 + i;
       const bool in = c < p.N;
-      s_bias[i] = (p.bias && in) ? bf16_lo(p.bias[c]) : 0.f;
+      s_bias[i] = (p.bias && in && !p.wide) ? bf16_lo(p.bias[c]) : 0.f;
       s_gamma[i] = (p.gamma && in) ? bf16_lo(p.gamma[c]) : 1.f;
       s_beta[i] = (p.beta && in) ? bf16_lo(p.beta[c]) : 0.f;
     }
@@ -544,6 +545,13 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // back over the accumulator in TMEM (the bypass path of Sec. 3.2)
         float2 part = make_float2(0.f, 0.f);
         float n_run = 0.f;
+        if (p.wide) {
+          // this tile's column block differs from the previous tile's: fetch its bias (every epilogue thread of the CTA
+          // has left stage 1 of the previous tile, the cluster-wide reduce there waits for all rows)
+          if (p.bias)
+            for (int i = threadIdx.x - 64; i < BN; i += Cfg::kEpiThreads) s_bias[i] = ncta0 + i < p.N ? bf16_lo(p.bias[ncta0 + i]) : 0.f;
+          named_barrier_sync(3, Cfg::kEpiThreads);
+        }
         COMFUSE_TRACE_POINT();
 #pragma unroll
         for (int sub = 0; sub < ESUB; ++sub) {
@@ -638,9 +646,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                        pm);
         }
         COMFUSE_TRACE_POINT();
-        const float mu = EPI == EPI_LN ? tot.x : 0.f;
+        // wide rows: the statistic covers this column block only; store x as it is (gamma = 1, beta = 0 were loaded) and
+        // leave the normalisation to the second kernel
+        const float mu = (EPI == EPI_LN && !p.wide) ? tot.x : 0.f;
         const float sq = EPI == EPI_LN ? tot.y : tot.x;
-        const float rstd = rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
+        const float rstd = p.wide ? 1.f : rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
+        if (p.wide && crank == 0 && h == 0 && valid) {
+          const int nb = (ncta0 / (CN * BN));
+          p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
+        }
         // ---------------- stage 2 (PostOp): normalise the resident x, round once, store
         float best = -INFINITY;
         int best_col = 0x7FFFFFFF;
@@ -689,7 +703,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           release_accumulator(sub);
         }
-        if constexpr (EPI == EPI_RMS_MAX) {
+        if (EPI == EPI_RMS_MAX && !p.wide) {
           // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
           const float2 mx = cluster_row_reduce<CN, MergeArgmax, EPW>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
                                                    s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);

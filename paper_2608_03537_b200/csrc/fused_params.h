@@ -1,6 +1,7 @@
 // Kernel parameter block of the GEMM -> subgraph kernels (plain data, shared by host and device code).
 #pragma once
 
+#include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace comfuse {
@@ -24,6 +25,11 @@ struct FusedParams {
   long long ldy, batch_stride_y;
   float* row_max;
   int* row_argmax;
+  // Rows wider than one cluster (nblocks > 1 with a normalising epilogue): every cluster finishes stage 1 for its
+  // column block only, stores the un-normalised values and writes the block's partial statistic of each row to
+  // wide_partials[(batch * M + row) * nblocks + block]; a second kernel merges the partials and rescales in place.
+  int wide;
+  float2* wide_partials;
   unsigned int* status;
   unsigned long long timeout_ns;
   unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null

@@ -39,6 +39,12 @@ struct GemmMaps {
 // exists without launching.
 cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+// Rows wider than the largest cluster (16 CTAs x 256 columns): LayerNorm / RMSNorm kinds run per 4096-column block and a
+// second kernel merges the blocks' statistics (the wide-row fallback).  Returns the number of blocks, 0 = not a wide row.
+constexpr int kWideRowBlock = 4096;
+inline int wide_row_blocks(int epi, int N) {
+  return ((epi == EPI_LN || epi == EPI_RMS_MAX) && N > kWideRowBlock && N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? N / kWideRowBlock : 0;
+}
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).
 bool softmax_rows_supported(const FusedParams& p);

@@ -206,6 +206,66 @@ __global__ void __launch_bounds__(256) row_epilogue_kernel(const RowParams p) {
   }
 }
 
+// Second kernel of the wide-row path: the fused kernel stored the un-normalised x (bf16) in Y and one partial statistic
+// per row and column block; merge the partials in block order, rescale the row in place, and (RMSNorm kind) take the row
+// maximum / lowest argmax of the normalised values.  One block per row.
+template <int KIND>
+__global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p, const float2* partials, int nblocks) {
+  __shared__ float s_red[8];
+  __shared__ int s_idx[8];
+  const long long r = blockIdx.x;  // row over batch * M
+  const int b = static_cast<int>(r / p.M);
+  const int i = static_cast<int>(r - static_cast<long long>(b) * p.M);
+  uint16_t* y = p.Y + static_cast<long long>(b) * p.batch_stride_y + static_cast<long long>(i) * p.ldy;
+  const float2* q = partials + r * nblocks;
+  const float wb = static_cast<float>(p.N / nblocks);  // columns per block (equal by construction)
+  float mu = 0.f, rstd;
+  if constexpr (KIND == EPI_LN) {
+    // equal-count Chan merge: mean of the block means, M2 = sum M2_b + wb * sum (mean_b - mean)^2
+    float ms = 0.f;
+    for (int k = 0; k < nblocks; ++k) ms += q[k].x;
+    mu = ms / static_cast<float>(nblocks);
+    float m2 = 0.f;
+    for (int k = 0; k < nblocks; ++k) {
+      const float d = q[k].x - mu;
+      m2 += q[k].y + wb * d * d;
+    }
+    rstd = rsqrtf(m2 / static_cast<float>(p.N) + p.eps);
+  } else {
+    float ss = 0.f;
+    for (int k = 0; k < nblocks; ++k) ss += q[k].x;
+    rstd = rsqrtf(ss / static_cast<float>(p.N) + p.eps);
+  }
+  float best = -INFINITY;
+  int best_col = 0x7FFFFFFF;
+  const int nvec = p.N >> 3;
+  for (int vi = threadIdx.x; vi < nvec; vi += 256) {
+    float xf[8], gf[8], bf[8];
+    const uint4 one = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+    unpack8(reinterpret_cast<const uint4*>(y)[vi], xf);
+    unpack8(p.gamma ? __ldg(reinterpret_cast<const uint4*>(p.gamma) + vi) : one, gf);
+    unpack8((KIND == EPI_LN && p.beta) ? __ldg(reinterpret_cast<const uint4*>(p.beta) + vi) : make_uint4(0, 0, 0, 0), bf);
+    float o[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if constexpr (KIND == EPI_LN) {
+        o[j] = fmaf((xf[j] - mu) * rstd, gf[j], bf[j]);
+      } else {
+        o[j] = xf[j] * rstd * gf[j];
+        if (o[j] > best) { best = o[j]; best_col = vi * 8 + j; }
+      }
+    }
+    reinterpret_cast<uint4*>(y)[vi] = make_uint4(pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
+  }
+  if constexpr (KIND == EPI_RMS_MAX) {
+    row_argmax_reduce<256>(best, best_col, s_red, s_idx);
+    if (threadIdx.x == 0) {
+      p.row_max[r] = best;
+      p.row_argmax[r] = best_col;
+    }
+  }
+}
+
 // S = bf16(GELU_tanh(P + b1)), in place over a dense [rows, n] bf16 matrix (unfused B2B: the intermediate epilogue).
 __global__ void __launch_bounds__(256) bias_gelu_kernel(uint16_t* P, const uint16_t* bias, long long nvec_total, int nvec_row) {
   const long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -251,6 +311,15 @@ cudaError_t launch_row_epilogue(int kind, const RowParams& p, cudaStream_t st) {
     case EPI_SOFTMAX: return dispatch_rows<EPI_SOFTMAX>(p, st);
     default: return cudaErrorInvalidValue;
   }
+}
+
+cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, cudaStream_t st) {
+  const unsigned rows = static_cast<unsigned>(static_cast<long long>(p.batch) * p.M);
+  count_launch();
+  if (kind == EPI_LN) wide_row_finish_kernel<EPI_LN><<<rows, 256, 0, st>>>(p, partials, nblocks);
+  else if (kind == EPI_RMS_MAX) wide_row_finish_kernel<EPI_RMS_MAX><<<rows, 256, 0, st>>>(p, partials, nblocks);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_bias_gelu(uint16_t* P, const uint16_t* bias, long long rows, int n, cudaStream_t st) {

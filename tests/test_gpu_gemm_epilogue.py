@@ -69,6 +69,40 @@ def test_gelu_rmsnorm_max_epilogue(M, N, K, fused, cuda_device):
                     rowmax_tol=5e-3 if fused else 3e-2)
 
 
+WIDE_SHAPES = [(300, 8192, 72), (129, 12288, 64)]   # rows wider than the largest cluster (16 CTAs x 256 columns)
+
+
+@pytest.mark.parametrize("M,N,K", WIDE_SHAPES)
+def test_layernorm_wide_rows_two_kernel_path(M, N, K, cuda_device):
+    """fused = 1 with N > 4096: per-4096-column-block stage 1 with partial statistics, then the rescaling kernel.  The row
+    passes through bf16 once before it is normalised, like the unfused path's intermediate, so it gets that path's budget."""
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(M, N, K, seed=N + K, affine=True)
+    T = P.dev_tensors(w)
+    desc = cf.make_gemm_desc(T["A"], T["B"], torch.empty(M, N, dtype=torch.bfloat16, device=T["A"].device),
+                             cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=True)
+    assert cf.workspace_size(desc) == M * (N // 4096) * 8      # one (mean, M2) pair per row and block
+    got = P.run_gpu(w, T, fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN wide {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("M,N,K", WIDE_SHAPES)
+def test_gelu_rmsnorm_max_wide_rows_two_kernel_path(M, N, K, cuda_device):
+    w = wl.complex_subgraph(M, N, K, seed=M + N)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"RMS wide {M}x{N}x{K}", rowmax_tol=3e-2)
+
+
+def test_wide_rows_need_their_workspace(cuda_device):
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(128, 8192, 64, seed=3, affine=False)
+    T = P.dev_tensors(w)
+    Y = torch.empty(128, 8192, dtype=torch.bfloat16, device=T["A"].device)
+    with pytest.raises(cf.ComfuseError) as ei:
+        cf.gemm_epilogue(T["A"], T["B"], Y, cf.EPI_BIAS_RES_LAYERNORM, bias=T["bias"], residual=T["residual"], fused=True)
+    assert ei.value.status == cf.ERR_WORKSPACE
+
+
 def test_argmax_planted_spike(cuda_device):
     """A residual spike pins the arg max of chosen rows, in every CTA of the cluster and at the chunk borders."""
     M, N, K = 128, 768, 64
