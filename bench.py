@@ -352,6 +352,14 @@ def run_comfuse(args):
     roof["algorithmic_flops_per_launch"] = flops
     roof["algorithmic_bytes_per_launch"] = bytes_min
     roof["roofline_us"] = max(t_tensor, t_hbm) * 1e6
+    # the same fraction against the nominal figures (2250 TFLOP/s dense bf16, 8 TB/s), for context
+    nominal = 2250.0 if roof["bound"] == "tensor" else 8000.0
+    roof["frac_of_nominal"] = roof["achieved"] / nominal
+    roof["nominal_peak"] = nominal
+    if w.kind == wl.KIND_SCALE_MASK_SOFTMAX and w.scalars.get("causal"):
+        # GEMM flops of the 128 x 128 score tiles the causal mask leaves (value counts all tiles, as a dense GEMM would)
+        t = -(-d["M"] // 128)
+        roof["flops_causal_tiles_only"] = flops * (t * (t + 1) / 2) / (t * t)
 
     extra = {}
     if not args.kernel_only:
@@ -374,6 +382,27 @@ def run_comfuse(args):
             del ws2
         except cf.ComfuseError as e:
             extra["unfused_error"] = str(e)
+        # ---- context: the same step with its inputs and outputs resident in L2 (one buffer set, back to back), and the
+        # GEMM(s) alone through the vendor library, so that "residual" = what the subgraph costs on top of the GEMM
+        # (Sec. 6.2 reports fusion benefit this way)
+        n3 = max(3, min(args.steps, 50))
+        for i in range(3):
+            step(sets[0])
+        extra["warm_l2_ms_per_step"] = timed(n3, lambda i: step(sets[0])) / n3
+
+        def gemm_only(sx):
+            if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+                return torch.matmul(torch.matmul(sx["X"], sx["W1"]), sx["W2"])
+            return torch.matmul(sx["A"], sx["B"])
+        for i in range(3):
+            gemm_only(sets[i % nsets])
+        ms_gemm = timed(n3, lambda i: gemm_only(sets[i % nsets])) / n3
+        extra["gemm_only_ms_per_step"] = ms_gemm
+        extra["gemm_only_impl"] = "torch.matmul (vendor library), bf16 output"
+        fused_ms = ms_step if fused else extra.get("fused_ms_per_step")
+        unfused_ms = extra.get("unfused_ms_per_step") if fused else ms_step
+        extra["residual_ms"] = {"fused": None if fused_ms is None else fused_ms - ms_gemm,
+                                "unfused": None if unfused_ms is None else unfused_ms - ms_gemm}
 
     # ---- end to end: activations from pinned host memory, result back to pinned host memory, every step
     if args.kernel_only:
