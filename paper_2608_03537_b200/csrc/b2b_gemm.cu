@@ -89,6 +89,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int num_clusters = gridDim.x >> 1;
   const int NC = p.N1 / 128;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
+  griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRingSlots; ++s) {
@@ -117,17 +118,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     tmem_alloc_pair(smem_u32(s_tmem_base), 512);
     tmem_relinquish_alloc_permit_pair();
   }
-  for (int i = threadIdx.x; i < p.N1; i += kB2bThreads) s_b1[i] = p.b1 ? bf16_lo(p.b1[i]) : 0.f;
-  for (int i = threadIdx.x; i < 128; i += kB2bThreads) {
-    s_b2[i] = p.b2 ? bf16_lo(p.b2[i]) : 0.f;
-    s_gamma[i] = p.gamma ? bf16_lo(p.gamma[i]) : 1.f;
-    s_beta[i] = p.beta ? bf16_lo(p.beta[i]) : 0.f;
-  }
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   cluster_sync_after_init();  // every CTA's barriers exist before any peer signals them
   const uint32_t tmem_base = *s_tmem_base;
+  griddep_wait();  // the set-up above may overlap the previous kernel's tail; global memory is touched only below
   // TMEM columns: P slots at 0 and 128, O slots at 256 and 384
   auto ring_addr = [&](int s) { return smem_base + B2bSmem::OFF_RING + s * kSlotBytes; };
   auto s_addr = [&](int buf, int kb) { return smem_base + B2bSmem::OFF_S + (buf * 2 + kb) * kSlotBytes; };
@@ -265,6 +261,14 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int row = q * 32 + lane;
     const int epi_tid = threadIdx.x - 64;
     const bool store_thread = epi_tid == 0;
+    // the row vectors, widened to fp32 once, by the epilogue warps (idle until the first P chunk is complete)
+    for (int i = epi_tid; i < p.N1; i += kB2bEpiThreads) s_b1[i] = p.b1 ? bf16_lo(p.b1[i]) : 0.f;
+    for (int i = epi_tid; i < 128; i += kB2bEpiThreads) {
+      s_b2[i] = p.b2 ? bf16_lo(p.b2[i]) : 0.f;
+      s_gamma[i] = p.gamma ? bf16_lo(p.gamma[i]) : 1.f;
+      s_beta[i] = p.beta ? bf16_lo(p.beta[i]) : 0.f;
+    }
+    named_barrier_sync(2, kB2bEpiThreads);
     const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
     const uint32_t ybuf = smem_base + B2bSmem::OFF_YBUF;
     const uint32_t sfull_leader = map_to_cta(bar_sfull(0), leader);
@@ -490,7 +494,7 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   static int max_clusters[kMaxDev] = {0};
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(kB2bThreads, 1, 1);
   cfg.dynamicSmemBytes = B2bSmem::BYTES;
   cfg.stream = st;
@@ -498,8 +502,10 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   if (max_clusters[di] == 0) {
     cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;

@@ -57,6 +57,14 @@ bool mult8(long long v) { return (v & 7) == 0; }
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+bool programmatic_launch_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("COMFUSE_PDL");
+    return !(e && e[0] == '0');
+  }();
+  return on;
+}
+
 const DeviceInfo* current_device_info() {
   int d = -1;
   if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDev) return nullptr;

@@ -162,6 +162,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int KB = (p.K + 63) >> 6;
   const bool has_res = (EPI == EPI_LN || EPI == EPI_RMS_MAX) && p.residual != nullptr;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
+  griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
 #ifdef COMFUSE_TRACE
   if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[62] = globaltimer_ns();  // kernel entry
@@ -198,23 +199,14 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tmem_alloc_pair(smem_u32(s_tmem_base), Cfg::TMEM_COLS);
     tmem_relinquish_alloc_permit_pair();
   }
-  if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
-    // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once
-    // (wide rows: the bias of the tile's column block is loaded per tile by the epilogue warps, gamma/beta are identity)
-    const int c0 = crank * BN;
-    for (int i = threadIdx.x; i < BN; i += Cfg::kThreads) {
-      const int c = c0 + i;
-      const bool in = c < p.N;
-      s_bias[i] = (p.bias && in && !p.wide) ? bf16_lo(p.bias[c]) : 0.f;
-      s_gamma[i] = (p.gamma && in) ? bf16_lo(p.gamma[c]) : 1.f;
-      s_beta[i] = (p.beta && in) ? bf16_lo(p.beta[c]) : 0.f;
-    }
-  }
   tcgen05_fence_before_sync();
   __syncthreads();
   tcgen05_fence_after_sync();
   cluster_sync_after_init();  // every CTA's barriers exist before any peer signals them
   const uint32_t tmem_base = *s_tmem_base;
+  // Everything above touched no global memory and may overlap the previous kernel's tail; everything below may read what
+  // that kernel wrote (or overwrite what it still reads).
+  griddep_wait();
 
   // tile -> (batch, first row of the pair, first column of this CTA)
   auto decode_tile = [&](int tile, int& b, int& mpair0, int& ncta0) {
@@ -421,6 +413,20 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int xpar = 0;
     uint32_t xphase = 0;
     (void)xpar; (void)xphase; (void)s_pre; (void)s_stats; (void)s_bias; (void)s_gamma; (void)s_beta;
+    if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
+      // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once, by the epilogue warps
+      // (they have nothing else to do until the first accumulator is complete); wide rows: the bias of the tile's column
+      // block is loaded per tile instead, gamma/beta are identity
+      const int c0 = crank * BN;
+      for (int i = threadIdx.x - 64; i < BN; i += Cfg::kEpiThreads) {
+        const int c = c0 + i;
+        const bool in = c < p.N;
+        s_bias[i] = (p.bias && in && !p.wide) ? bf16_lo(p.bias[c]) : 0.f;
+        s_gamma[i] = (p.gamma && in) ? bf16_lo(p.gamma[c]) : 1.f;
+        s_beta[i] = (p.beta && in) ? bf16_lo(p.beta[c]) : 0.f;
+      }
+      named_barrier_sync(3, Cfg::kEpiThreads);
+    }
     RingPos<NSTAGES> ring;
     uint32_t rfull_bits = 0;
     uint32_t slot_uses[2] = {0, 0};

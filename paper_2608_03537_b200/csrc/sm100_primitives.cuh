@@ -45,6 +45,13 @@ __device__ __forceinline__ void cluster_sync_after_init() {
   asm volatile("barrier.cluster.arrive.relaxed;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
 }
 
+// Programmatic dependent launch.  launch_dependents: the next kernel in the stream (if it was launched with programmatic
+// stream serialization) may be scheduled once every CTA of this grid has issued it or exited, i.e. its set-up overlaps
+// this kernel's tail.  wait: returns when the kernel this grid depends on has completed and its memory is visible; a
+// kernel must execute it before its first access to global memory.  Both are no-ops without such a dependency.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }

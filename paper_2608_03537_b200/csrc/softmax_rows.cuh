@@ -85,6 +85,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int nch = (p.N + CHUNK - 1) / CHUNK;
   const int rounds = (p.total_tiles + num_clusters - 1) / num_clusters;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
+  griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
   // -------------------------------------------------------------------------------------------- set-up
   if (threadIdx.x == 0) {
@@ -119,6 +120,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   tcgen05_fence_after_sync();
   cluster_sync_after_init();  // both CTAs' barriers exist before the peer signals them
   const uint32_t tmem_base = *s_tmem_base;
+  griddep_wait();  // the set-up above may overlap the previous kernel's tail; global memory is touched only below
 
   // Tile of this cluster in round r.  Tiles are ordered by falling cost (under a causal mask a lower row block has
   // more live chunks) and dealt to the clusters in alternating direction, so the clusters' sums stay close.

@@ -217,3 +217,34 @@ def test_fused_and_unfused_runs_are_bitwise_repeatable(cuda_device):
 def test_no_timeout_recorded(cuda_device):
     import paper_2608_03537_b200 as cf
     assert cf.last_device_status() == cf.OK
+
+
+def test_back_to_back_dependent_launches_see_each_others_results(cuda_device):
+    """Kernels are launched with programmatic stream serialization: the set-up of a kernel overlaps the tail of the previous
+    one, and it waits for that kernel before it touches global memory.  A chain in which every call consumes the previous
+    call's output, enqueued without any synchronisation, must give bit-for-bit what the same chain gives with a
+    synchronisation after every call."""
+    import paper_2608_03537_b200 as cf
+    M, N, K = 512, 256, 256
+    w = wl.post_norm(M, N, K, seed=11, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+
+    def chain(sync):
+        x = T["A"].clone()                       # [M, 256]; N == K so the output can feed the next call
+        bufs = [torch.empty(M, N, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        for i in range(12):
+            y = bufs[i & 1]                      # ping-pong: a call overwrites what the call before the previous one wrote
+            cf.gemm_epilogue(x, T["B"], y, cf.EPI_BIAS_RES_LAYERNORM, bias=T["bias"], residual=T["residual"],
+                             gamma=T["gamma"], beta=T["beta"], fused=True)
+            if sync:
+                torch.cuda.synchronize()
+            x = y
+        torch.cuda.synchronize()
+        return x.clone()
+
+    a = chain(sync=True)
+    for _ in range(3):
+        b = chain(sync=False)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert cf.last_device_status() == cf.OK
