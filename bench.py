@@ -412,25 +412,44 @@ def run_comfuse(args):
         if world > 1:
             dist.destroy_process_group()
         return
+    # One call of the library's host-buffer entry point per step: it copies the step's activations from pinned host
+    # memory into a device staging buffer, runs the same kernels, and copies the result back to pinned host memory.
     host_in = {k: torch.from_numpy(np.ascontiguousarray(w.tensors[k]).view(np.int16)).view(torch.bfloat16).pin_memory()
                for k in w.tensors if k in act_names}
     host_out = torch.empty(out_shape, dtype=torch.bfloat16).pin_memory()
     h2d = sum(t.numel() * 2 for t in host_in.values())
     d2h = host_out.numel() * 2
+    s0 = sets[0]
+    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        bdesc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused)
+        staging = torch.empty(cf.b2b_host_staging_size(bdesc), dtype=torch.uint8, device=dev)
 
-    def e2e_step(i):
-        s = sets[i % nsets]
-        for k, t in host_in.items():
-            s[k].copy_(t, non_blocking=True)
-        step(s)
-        host_out.copy_(s["Y"], non_blocking=True)
+        def e2e_step(i):
+            cf.b2b_gemm_host(host_in["X"], s0["W1"], s0["b1"], s0["W2"], s0["b2"], host_out, staging=staging,
+                             gamma=s0.get("gamma"), beta=s0.get("beta"), eps=w.scalars["eps"], fused=fused, workspace=ws)
+    else:
+        hmask = cf.HOST_A | cf.HOST_Y | (cf.HOST_B if "B" in host_in else 0) | (cf.HOST_RESIDUAL if "residual" in host_in else 0)
+        hB = host_in.get("B", s0["B"])
+        hdesc = cf.make_gemm_desc(host_in["A"], hB, host_out, kind, residual=host_in.get("residual"), mask=mask, fused=fused)
+        staging = torch.empty(cf.host_staging_size(hdesc, hmask), dtype=torch.uint8, device=dev)
+        ekw = dict(alpha=w.scalars["alpha"], mask=mask, fused=fused, workspace=ws, staging=staging, host_mask=hmask)
+        if w.kind != wl.KIND_SCALE_MASK_SOFTMAX:
+            ekw.update(bias=s0.get("bias"), residual=host_in.get("residual"), gamma=s0.get("gamma"), eps=w.scalars["eps"])
+        if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+            ekw.update(beta=s0.get("beta"))
+        if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+            ekw.update(row_max=s0["row_max"], row_argmax=s0["row_argmax"])
+
+        def e2e_step(i):
+            cf.gemm_epilogue_host(host_in["A"], hB, host_out, kind, **ekw)
 
     n_e2e = max(3, min(args.steps, 20))
     for i in range(2):
         e2e_step(i)
     ms_e2e = timed(n_e2e, e2e_step) / n_e2e
     e2e = {"value": whole_job_value(flops, world, ms_e2e) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e}
+           "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e,
+           "call": "comfuse_b2b_gemm_host" if w.kind == wl.KIND_B2B_MLP_LAYERNORM else "comfuse_gemm_epilogue_host"}
 
     # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only, on a bounded sample
     cpu = None

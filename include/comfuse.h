@@ -142,6 +142,29 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
                                   const void* W2, const void* b2, const void* gamma, const void* beta, void* O,
                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Host-buffer forms (the paper has no counterpart: it measures kernels on resident tensors).  The per-step tensors
+ * selected by `host_mask` are HOST pointers (pinned memory if the copies are to be asynchronous); everything else stays a
+ * device pointer as above.  The call enqueues, on `cuda_stream`: one host -> device copy per selected input into
+ * `staging` (DEVICE memory owned by the caller, at least comfuse_host_staging_size() bytes, 16-byte aligned), the same
+ * kernels as comfuse_gemm_epilogue, and, if COMFUSE_HOST_Y is set, one device -> host copy of the result.  Each copy moves
+ * the tensor's whole strided extent ((batch-1)*batch_stride + (rows-1)*ld + cols elements), pad columns included.  Nothing
+ * is allocated and nothing synchronises; the host buffers must stay valid until the stream has passed the call.
+ * Errors: as comfuse_gemm_epilogue; COMFUSE_ERR_WORKSPACE also when `staging` is NULL or too small. */
+#define COMFUSE_HOST_A 1u
+#define COMFUSE_HOST_B 2u
+#define COMFUSE_HOST_RESIDUAL 4u /* args->residual is a host pointer */
+#define COMFUSE_HOST_Y 8u
+comfuse_status_t comfuse_host_staging_size(const comfuse_gemm_desc_t* desc, uint32_t host_mask, size_t* bytes);
+comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t* desc, const void* A, const void* B, void* Y,
+                                            const comfuse_epilogue_args_t* args, uint32_t host_mask, void* staging,
+                                            size_t staging_bytes, void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* The same for the back-to-back GEMM: X and O are host pointers (dense), the weights and vectors device pointers. */
+comfuse_status_t comfuse_b2b_host_staging_size(const comfuse_b2b_desc_t* desc, size_t* bytes);
+comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc, const void* X, const void* W1, const void* b1,
+                                       const void* W2, const void* b2, const void* gamma, const void* beta, void* O,
+                                       void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word of the current device:
  * COMFUSE_OK, COMFUSE_ERR_TIMEOUT, or COMFUSE_ERR_CUDA if the stream reports an error. */
 comfuse_status_t comfuse_last_device_status(void* cuda_stream);

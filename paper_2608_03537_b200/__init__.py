@@ -8,6 +8,8 @@ import of :func:`lib` fails loudly.
 Functions mirror the C entry points:
     gemm_epilogue(...)      -> comfuse_gemm_epilogue      (GEMM -> elementwise/reduction subgraph, Sec. 3)
     gemm_epilogue_static_scratch(...) -> comfuse_gemm_epilogue_static_scratch (unfused path, no caller workspace)
+    gemm_epilogue_host(...) -> comfuse_gemm_epilogue_host (per-step tensors in host memory, staged through a device buffer)
+    b2b_gemm_host(...)      -> comfuse_b2b_gemm_host
     b2b_gemm(...)           -> comfuse_b2b_gemm           (GEMM -> F -> GEMM -> post-norm tail, Sec. 4)
     workspace_size(...)     -> comfuse_workspace_size
     b2b_workspace_size(...) -> comfuse_b2b_workspace_size
@@ -28,6 +30,7 @@ LIB_PATH = os.path.join(_PKG_DIR, "libcomfuse.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
 EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 0, 1, 2
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
+HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
 
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
@@ -35,6 +38,10 @@ EXPORTED_SYMBOLS = (
     "comfuse_gemm_epilogue_static_scratch",
     "comfuse_b2b_workspace_size",
     "comfuse_b2b_gemm",
+    "comfuse_host_staging_size",
+    "comfuse_gemm_epilogue_host",
+    "comfuse_b2b_host_staging_size",
+    "comfuse_b2b_gemm_host",
     "comfuse_last_device_status",
     "comfuse_launch_count",
     "comfuse_selftest_bounded_wait",
@@ -94,6 +101,15 @@ def lib() -> ctypes.CDLL:
         L.comfuse_b2b_workspace_size.restype = c_int32
         L.comfuse_b2b_gemm.argtypes = [POINTER(B2bDesc)] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
         L.comfuse_b2b_gemm.restype = c_int32
+        L.comfuse_host_staging_size.argtypes = [POINTER(GemmDesc), ctypes.c_uint32, POINTER(c_size_t)]
+        L.comfuse_host_staging_size.restype = c_int32
+        L.comfuse_gemm_epilogue_host.argtypes = [POINTER(GemmDesc), c_void_p, c_void_p, c_void_p, POINTER(EpilogueArgs),
+                                                 ctypes.c_uint32, c_void_p, c_size_t, c_void_p, c_size_t, c_void_p]
+        L.comfuse_gemm_epilogue_host.restype = c_int32
+        L.comfuse_b2b_host_staging_size.argtypes = [POINTER(B2bDesc), POINTER(c_size_t)]
+        L.comfuse_b2b_host_staging_size.restype = c_int32
+        L.comfuse_b2b_gemm_host.argtypes = [POINTER(B2bDesc)] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p, c_size_t, c_void_p]
+        L.comfuse_b2b_gemm_host.restype = c_int32
         L.comfuse_last_device_status.argtypes = [c_void_p]
         L.comfuse_last_device_status.restype = c_int32
         L.comfuse_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, POINTER(ctypes.c_uint32)]
@@ -179,6 +195,31 @@ def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True) -> B2bDesc:
     return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)))
 
 
+def host_staging_size(desc: GemmDesc, host_mask: int) -> int:
+    n = c_size_t(0)
+    st = lib().comfuse_host_staging_size(byref(desc), int(host_mask), byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_host_staging_size")
+    return int(n.value)
+
+
+def gemm_epilogue_host(A, B, Y, kind, *, staging, host_mask, bias=None, residual=None, gamma=None, beta=None,
+                       mask_tensor=None, row_max=None, row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True,
+                       workspace=None, stream=None):
+    """gemm_epilogue with the tensors named in ``host_mask`` (HOST_A | HOST_B | HOST_RESIDUAL | HOST_Y) living in host
+    memory (CPU tensors, pinned for asynchronous copies); ``staging`` is a CUDA uint8 tensor of at least
+    host_staging_size(desc, host_mask) bytes.  Copies and kernels are enqueued on the stream; nothing synchronises."""
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused)
+    args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_gemm_epilogue_host(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), int(host_mask),
+                                          c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),
+                                          ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_epilogue_host")
+    return Y
+
+
 def b2b_workspace_size(desc: B2bDesc) -> int:
     n = c_size_t(0)
     st = lib().comfuse_b2b_workspace_size(byref(desc), byref(n))
@@ -199,6 +240,31 @@ def b2b_gemm(X, W1, b1, W2, b2, O, *, gamma=None, beta=None, eps=1e-5, fused=Tru
                                 ws_ptr, ws_bytes, _stream(stream))
     if st != OK:
         raise ComfuseError(st, "comfuse_b2b_gemm")
+    return O
+
+
+def b2b_host_staging_size(desc: B2bDesc) -> int:
+    n = c_size_t(0)
+    st = lib().comfuse_b2b_host_staging_size(byref(desc), byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_host_staging_size")
+    return int(n.value)
+
+
+def b2b_gemm_host(X, W1, b1, W2, b2, O, *, staging, gamma=None, beta=None, eps=1e-5, fused=True, workspace=None, stream=None):
+    """b2b_gemm with X and O in host memory (dense CPU tensors, pinned for asynchronous copies); weights and vectors are
+    CUDA tensors; ``staging`` is a CUDA uint8 tensor of at least b2b_host_staging_size(desc) bytes."""
+    M, K = X.shape
+    N1, N2 = W1.shape[1], W2.shape[1]
+    for t in (X, W1, W2, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, eps, fused)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm_host(byref(d), _ptr(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gamma), _ptr(beta), _ptr(O),
+                                     c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),
+                                     ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm_host")
     return O
 
 

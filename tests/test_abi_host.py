@@ -66,6 +66,24 @@ def test_workspace_size_rules():
     assert cf.lib().comfuse_workspace_size(None, None) == cf.ERR_INVALID_ARG
 
 
+def test_wide_row_and_host_staging_sizes():
+    wide = dict(N=8192, ldb=8192, ldr=8192, ldy=8192)
+    assert _ws(_desc(**wide)) == (cf.OK, 256 * 2 * 8)                      # fused wide rows: (mean, M2) per row and 4096-column block
+    assert _ws(_desc(**wide, kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX)) == (cf.OK, 256 * 2 * 8)
+    assert _ws(_desc(N=8200, ldb=8200, ldr=8200, ldy=8200))[0] == cf.ERR_UNSUPPORTED   # wide rows come in whole 4096-column blocks
+    d = _desc()                                                            # A [256, 512], B [512, 768], R, Y [256, 768], dense
+    n = ctypes.c_size_t(0)
+    L = cf.lib()
+    assert L.comfuse_host_staging_size(ctypes.byref(d), cf.HOST_A | cf.HOST_RESIDUAL | cf.HOST_Y, ctypes.byref(n)) == cf.OK
+    assert n.value == 256 * 512 * 2 + 2 * 256 * 768 * 2                    # already multiples of the 256-byte slot alignment
+    assert L.comfuse_host_staging_size(ctypes.byref(d), 0, ctypes.byref(n)) == cf.OK and n.value == 0
+    assert L.comfuse_host_staging_size(ctypes.byref(d), 16, ctypes.byref(n)) == cf.ERR_INVALID_ARG      # unknown mask bit
+    assert L.comfuse_host_staging_size(None, 1, ctypes.byref(n)) == cf.ERR_INVALID_ARG
+    b = cf.make_b2b_desc(1000, 128, 512, 128, 1e-5, True)
+    assert L.comfuse_b2b_host_staging_size(ctypes.byref(b), ctypes.byref(n)) == cf.OK
+    assert n.value == 2 * 1000 * 128 * 2
+
+
 def test_gemm_epilogue_rejects_bad_arguments_before_any_launch():
     L = cf.lib()
     d = _desc()

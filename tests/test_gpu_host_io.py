@@ -1,0 +1,82 @@
+"""GPU: the host-buffer forms of the entry points (per-step tensors in pinned host memory, staged through a caller-provided
+device buffer) give bit for bit what the device-pointer forms give, and reject a staging buffer that is too small."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _pinned(t):
+    return t.cpu().pin_memory()
+
+
+def test_layernorm_host_buffers_match_device_buffers(cuda_device):
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(300, 768, 200, seed=17, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hA, hR = _pinned(T["A"]), _pinned(T["residual"])
+    hY = torch.empty(300, 768, dtype=torch.bfloat16).pin_memory()
+    mask = cf.HOST_A | cf.HOST_RESIDUAL | cf.HOST_Y
+    desc = cf.make_gemm_desc(hA, T["B"], hY, cf.EPI_BIAS_RES_LAYERNORM, residual=hR, fused=True)
+    staging = torch.empty(cf.host_staging_size(desc, mask), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        hY.fill_(7.0)
+        cf.gemm_epilogue_host(hA, T["B"], hY, cf.EPI_BIAS_RES_LAYERNORM, staging=staging, host_mask=mask, bias=T["bias"],
+                              residual=hR, gamma=T["gamma"], beta=T["beta"], alpha=w.scalars["alpha"], eps=w.scalars["eps"])
+        torch.cuda.synchronize()
+        assert torch.equal(hY.view(torch.int16), ref.cpu().view(torch.int16))
+    # against the oracle as well
+    err = np.abs(wl.bf16_to_f64(hY.view(torch.int16).numpy().view(np.uint16)) - P.run_oracle(w)["Y"])
+    assert err.max() <= P.TOL_NORM_MAX and err.mean() <= P.TOL_NORM_MEAN
+
+
+def test_softmax_host_buffers_batched(cuda_device):
+    import paper_2608_03537_b200 as cf
+    w = wl.scaled_masked_softmax(3, 256, 256, 64, seed=5, causal=True)
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hA, hB = _pinned(T["A"]), _pinned(T["B"])
+    hY = torch.empty(3, 256, 256, dtype=torch.bfloat16).pin_memory()
+    mask = cf.HOST_A | cf.HOST_B | cf.HOST_Y
+    desc = cf.make_gemm_desc(hA, hB, hY, cf.EPI_SCALE_MASK_SOFTMAX, mask=cf.MASK_CAUSAL, fused=True)
+    staging = torch.empty(cf.host_staging_size(desc, mask), dtype=torch.uint8, device=dev)
+    cf.gemm_epilogue_host(hA, hB, hY, cf.EPI_SCALE_MASK_SOFTMAX, staging=staging, host_mask=mask, alpha=w.scalars["alpha"],
+                          mask=cf.MASK_CAUSAL)
+    torch.cuda.synchronize()
+    assert torch.equal(hY.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_b2b_host_buffers_match_device_buffers(cuda_device):
+    import paper_2608_03537_b200 as cf
+    w = wl.b2b_mlp(M=600, K=128, N1=512, N2=128, seed=8, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["X"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hX = _pinned(T["X"])
+    hO = torch.empty(600, 128, dtype=torch.bfloat16).pin_memory()
+    desc = cf.make_b2b_desc(600, 128, 512, 128, w.scalars["eps"], True)
+    staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=dev)
+    cf.b2b_gemm_host(hX, T["W1"], T["b1"], T["W2"], T["b2"], hO, staging=staging, gamma=T.get("gamma"), beta=T.get("beta"),
+                     eps=w.scalars["eps"])
+    torch.cuda.synchronize()
+    assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_host_form_rejects_small_staging(cuda_device):
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(256, 256, 64, seed=2, affine=False)
+    T = P.dev_tensors(w)
+    hA = _pinned(T["A"])
+    hY = torch.empty(256, 256, dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(1024, dtype=torch.uint8, device=T["B"].device)
+    with pytest.raises(cf.ComfuseError) as ei:
+        cf.gemm_epilogue_host(hA, T["B"], hY, cf.EPI_BIAS_RES_LAYERNORM, staging=staging, host_mask=cf.HOST_A | cf.HOST_Y,
+                              bias=T["bias"], residual=T["residual"])
+    assert ei.value.status == cf.ERR_WORKSPACE
