@@ -321,6 +321,23 @@ __device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a
 __device__ __forceinline__ float2 splat2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 f2_from_bits(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
 // the two bf16 halves of a packed word, widened exactly
+// 2^x for two values on the FMA pipe, without the MUFU unit (which the ex2 instruction shares with shared-memory and
+// global stores through the SM's memory-instruction queue): x = n + f with n = round(x), |f| <= 0.5; 2^f by a degree-4
+// minimax polynomial (relative error 4.2e-6); the exponent is added to the float's bit pattern.  x is clamped at -126
+// (results below 2^-126 come out as 2^-126); meant for x <= 0.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 r = add2(x, splat2(12582912.f));  // 1.5 * 2^23: the low mantissa bits of r hold n in two's complement
+  const float2 n = add2(r, splat2(-12582912.f));
+  const float2 f = fma2(n, splat2(-1.f), x);
+  float2 q = fma2(splat2(0.009689519181847572f), f, splat2(0.055905185639858246f));
+  q = fma2(q, f, splat2(0.24021807312965393f));
+  q = fma2(q, f, splat2(0.6931246519088745f));
+  q = fma2(q, f, splat2(1.f));
+  return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(r.x) << 23)),
+                     __int_as_float(__float_as_int(q.y) + (__float_as_int(r.y) << 23)));
+}
 __device__ __forceinline__ float2 bf16x2_to_f2(uint32_t u) { return make_float2(bf16_lo(u), bf16_hi(u)); }
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float2 v) { return pack_bf16x2_rn(v.x, v.y); }
 // GELU, tanh form, on a pair: six packed instructions and two MUFU.TANH

@@ -34,6 +34,10 @@ struct RowSoftmaxCfg {
   static constexpr int kThreads = 32 * (kZeroWarp + 1);
   static constexpr int ZERO_TMA_LANES = 8;                   // zero boxes in flight per SM
   static constexpr int CHUNK = 256;                          // columns per UMMA and per accumulator slot
+  // Which of a 32-column fragment's 16 column pairs take 2^x from the FMA-pipe polynomial instead of the MUFU unit
+  // (bit j = pair j).  The MUFU unit delivers 16 results per clock per SM and is this kernel's busiest pipe; the
+  // polynomial costs about six issue slots per value, so a bit over a third of the pairs balances the two.
+  static constexpr uint32_t POLY_PAIRS = 0x5252u;            // pairs 1, 4, 6, 9, 12, 14
   static constexpr int A_BYTES = 128 * 64 * 2;
   static constexpr int STAGE_BYTES = A_BYTES + (CHUNK / 2) * 64 * 2;  // A block + this CTA's half of the B chunk
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;
@@ -276,6 +280,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     uint32_t unit = 0, nbox = 0, tile_par = 0;
     // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
     const float sc = p.alpha * 1.4426950408889634f;
+    constexpr uint32_t poly_pairs = Cfg::POLY_PAIRS;
 
 #ifdef COMFUSE_TRACE
     int trace_ix = 0;
@@ -356,8 +361,8 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                 for (int j = 0; j < 16; j += 2) {
                   const float2 d0 = add2(tv[j], neg_m), d1 = add2(tv[j + 1], neg_m);
-                  acc0 = add2(acc0, make_float2(ex2_approx(d0.x), ex2_approx(d0.y)));
-                  acc1 = add2(acc1, make_float2(ex2_approx(d1.x), ex2_approx(d1.y)));
+                  acc0 = add2(acc0, ((poly_pairs >> j) & 1u) ? ex2_poly2(d0) : make_float2(ex2_approx(d0.x), ex2_approx(d0.y)));
+                  acc1 = add2(acc1, ((poly_pairs >> (j + 1)) & 1u) ? ex2_poly2(d1) : make_float2(ex2_approx(d1.x), ex2_approx(d1.y)));
                 }
                 const float2 acc = add2(acc0, acc1);
                 s_run = fmaf(s_run, ex2_approx(m_run - m_new), acc.x + acc.y);
@@ -382,7 +387,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), splat2(-off));
-                  ev[j] = make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
+                  ev[j] = ((poly_pairs >> j) & 1u) ? ex2_poly2(t01) : make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
                 }
                 if (st != 2) {  // crosses the diagonal (or the end of the row)
 #pragma unroll
