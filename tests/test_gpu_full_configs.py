@@ -72,3 +72,38 @@ def test_config_tiny_post_norm_full(cuda_device):
     for fused in (True, False):
         got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
         print("c1", fused, P.check_outputs(w, got, P.run_oracle(w), label=f"c1 fused={fused}"))
+
+
+@pytest.mark.parametrize("cfg", [1, 3, 4])
+def test_cuda_graph_replay_matches_direct_launches(cfg, cuda_device):
+    """The benchmark replays its steps from a CUDA graph (one launch per buffer set, launched with programmatic stream
+    serialization so consecutive launches overlap at their edges).  The replayed launches must write, bit for bit, what a
+    direct launch writes; the direct launch is what the tests above compare with the oracle."""
+    import paper_2608_03537_b200 as cf
+    w = wl.config(cfg)
+    T = P.dev_tensors(w)
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    outs = [torch.full_like(ref, float("nan")) for _ in range(3)]
+
+    def launch(Y):
+        if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+            cf.b2b_gemm(T["X"], T["W1"], T["b1"], T["W2"], T["b2"], Y, gamma=T.get("gamma"), beta=T.get("beta"), eps=w.scalars["eps"])
+        elif w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+            cf.gemm_epilogue(T["A"], T["B"], Y, cf.EPI_BIAS_RES_LAYERNORM, bias=T["bias"], residual=T["residual"], gamma=T["gamma"],
+                             beta=T["beta"], alpha=w.scalars["alpha"], eps=w.scalars["eps"])
+        else:
+            cf.gemm_epilogue(T["A"], T["B"], Y, cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"], mask=cf.MASK_CAUSAL)
+
+    launch(outs[0])                      # first use outside the capture (configures the kernel)
+    torch.cuda.synchronize()
+    outs[0].fill_(float("nan"))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for Y in outs:
+            launch(Y)
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    for Y in outs:
+        assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
+    assert cf.last_device_status() == cf.OK
