@@ -113,25 +113,28 @@ def causal_mask(M: int, N: int, rows=None) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- the three GEMM -> subgraph op lists
-def bias_res_layernorm(A, B, bias=None, residual=None, gamma=None, beta=None, alpha=1.0, eps=1e-5):
+def bias_res_layernorm(A, B, bias=None, residual=None, gamma=None, beta=None, alpha=1.0, eps=1e-5, relu=False):
     """Y = LayerNorm(alpha * A.B + bias + R) * gamma + beta   (post-norm pattern; Sec. 3.2's worked example
-    x = alpha * Acc + Bias with the mean / x - mean stages)."""
+    x = alpha * Acc + Bias with the mean / x - mean stages).  ``relu``: Y = max(Y, 0) after the affine step, the
+    MatMul-BiasAdd-LayerNorm-ReLU pattern of Sec. 6.2."""
     H = alpha * gemm(A, B)
     if bias is not None:
         H = H + np.asarray(bias, dtype=np.float64)
     if residual is not None:
         H = H + np.asarray(residual, dtype=np.float64)
-    return layernorm_rows(H, gamma, beta, eps)
+    Y = layernorm_rows(H, gamma, beta, eps)
+    return np.maximum(Y, 0.0) if relu else Y
 
 
-def bias_gelu_res_rmsnorm_max(A, B, bias=None, residual=None, g=None, alpha=1.0, eps=1e-5):
+def bias_gelu_res_rmsnorm_max(A, B, bias=None, residual=None, g=None, alpha=1.0, eps=1e-5, activation=True):
     """Z = alpha * A.B + bias; H = GELU_tanh(Z) + R; Y = RMSNorm(H) * g; then a second, chained
     reduction over Y (Sec. 3.2: multiple reduction stages): row max and argmax.
-    Returns (Y, rowmax, argmax)."""
+    ``activation=False`` leaves the GELU out (H = Z + R): with no residual that is the MatMul-BiasAdd-RMSNorm
+    pattern of Sec. 6.2.  Returns (Y, rowmax, argmax)."""
     Z = alpha * gemm(A, B)
     if bias is not None:
         Z = Z + np.asarray(bias, dtype=np.float64)
-    H = gelu_tanh(Z)
+    H = gelu_tanh(Z) if activation else Z
     if residual is not None:
         H = H + np.asarray(residual, dtype=np.float64)
     Y = rmsnorm_rows(H, g, eps)
@@ -139,10 +142,13 @@ def bias_gelu_res_rmsnorm_max(A, B, bias=None, residual=None, g=None, alpha=1.0,
     return Y, mx, am
 
 
-def scale_mask_softmax(A, B, alpha=1.0, mask=None):
+def scale_mask_softmax(A, B, alpha=1.0, mask=None, softcap=0.0):
     """P = softmax(alpha * A.B + mask) over the last dim (the attention-score normalisation pattern of
-    Sec. 6.1 with an additive mask in place of the soft-cap).  ``mask`` broadcasts over leading dims."""
+    Sec. 6.1).  ``mask`` broadcasts over leading dims.  ``softcap`` > 0: the scaled scores pass through
+    softcap * tanh(. / softcap) before the mask, the MatMul-Scale-TanhSoftcap-Softmax pattern of Sec. 6.2."""
     T = alpha * gemm(A, B)
+    if softcap and softcap > 0.0:
+        T = softcap * np.tanh(T / softcap)
     if mask is not None:
         T = T + mask
     return softmax_rows(T)

@@ -92,11 +92,13 @@ def run_oracle(w: wl.Workload, rows=None, batches=None):
         return {"Y": Y}
     if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
         Y = orc.bias_res_layernorm(f64(w, "A", rows), f64(w, "B"), f64(w, "bias"), f64(w, "residual", rows),
-                                   f64(w, "gamma"), f64(w, "beta"), w.scalars["alpha"], w.scalars["eps"])
+                                   f64(w, "gamma"), f64(w, "beta"), w.scalars["alpha"], w.scalars["eps"],
+                                   relu=w.scalars.get("relu", False))
         return {"Y": Y}
     if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
         Y, mx, am = orc.bias_gelu_res_rmsnorm_max(f64(w, "A", rows), f64(w, "B"), f64(w, "bias"), f64(w, "residual", rows),
-                                                  f64(w, "gamma"), w.scalars["alpha"], w.scalars["eps"])
+                                                  f64(w, "gamma"), w.scalars["alpha"], w.scalars["eps"],
+                                                  activation=w.scalars.get("activation", True))
         return {"Y": Y, "row_max": mx, "row_argmax": am}
     # softmax
     bsel = list(range(d["batch"])) if batches is None else list(batches)
@@ -110,7 +112,7 @@ def run_oracle(w: wl.Workload, rows=None, batches=None):
     if "mask" in w.tensors:
         m = wl.bf16_to_f64(w.tensors["mask"])
         mask = m if rows is None else m[rows]
-    P = orc.scale_mask_softmax(wl.bf16_to_f64(A), wl.bf16_to_f64(B), w.scalars["alpha"], mask)
+    P = orc.scale_mask_softmax(wl.bf16_to_f64(A), wl.bf16_to_f64(B), w.scalars["alpha"], mask, softcap=w.scalars.get("softcap", 0.0))
     return {"Y": P}
 
 

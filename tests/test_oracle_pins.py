@@ -332,3 +332,68 @@ def test_softmax_merge_any_split(splits):
     P = orc.softmax_rows(x)
     with np.errstate(invalid="ignore"):
         np.testing.assert_allclose(np.where(np.isneginf(x), 0.0, np.exp(x - m[:, None])) / l[:, None], P, rtol=0, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- the Sec. 6.2 pattern variants
+def test_layernorm_relu_variant_brute_force_and_sign():
+    """MatMul-BiasAdd-LayerNorm-ReLU: scalar-loop brute force; every output is >= 0 and equals the plain result where
+    that is positive (so the ReLU sits after the affine step, not before the normalisation)."""
+    r = _rng(40)
+    A, B = r.standard_normal((5, 7)), r.standard_normal((7, 6))
+    bias, gamma, beta = r.standard_normal(6), r.standard_normal(6), r.standard_normal(6)
+    eps = 1e-5
+    want = np.zeros((5, 6))
+    for i in range(5):
+        h = [sum(A[i, k] * B[k, j] for k in range(7)) + bias[j] for j in range(6)]
+        mu = sum(h) / 6
+        var = sum((x - mu) ** 2 for x in h) / 6
+        for j in range(6):
+            y = (h[j] - mu) / math.sqrt(var + eps) * gamma[j] + beta[j]
+            want[i, j] = y if y > 0 else 0.0
+    got = orc.bias_res_layernorm(A, B, bias, None, gamma, beta, 1.0, eps, relu=True)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    plain = orc.bias_res_layernorm(A, B, bias, None, gamma, beta, 1.0, eps)
+    assert (got >= 0).all() and (got[plain > 0] == plain[plain > 0]).all() and (got[plain <= 0] == 0).all()
+    assert (plain < 0).any()          # the case actually exercises the clamp
+
+
+def test_rmsnorm_without_activation_is_bias_rmsnorm():
+    """MatMul-BiasAdd-RMSNorm: with the activation off and no residual the op list is RMSNorm(A.B + bias) * g:
+    brute force, and the identity sum_j (Y_j / g_j)^2 = N * ms / (ms + eps)."""
+    r = _rng(41)
+    A, B, bias, g = r.standard_normal((4, 9)), r.standard_normal((9, 8)), r.standard_normal(8), r.uniform(0.5, 1.5, 8)
+    eps = 1e-3
+    Y, mx, am = orc.bias_gelu_res_rmsnorm_max(A, B, bias, None, g, 1.0, eps, activation=False)
+    for i in range(4):
+        z = [sum(A[i, k] * B[k, j] for k in range(9)) + bias[j] for j in range(8)]
+        ms = sum(x * x for x in z) / 8
+        row = [z[j] / math.sqrt(ms + eps) * g[j] for j in range(8)]
+        np.testing.assert_allclose(Y[i], row, rtol=0, atol=1e-12)
+        assert abs(sum((row[j] / g[j]) ** 2 for j in range(8)) - 8 * ms / (ms + eps)) < 1e-12
+        assert mx[i] == max(row) and am[i] == row.index(max(row))
+    with_act = orc.bias_gelu_res_rmsnorm_max(A, B, bias, None, g, 1.0, eps)[0]
+    assert np.abs(with_act - Y).max() > 1e-2      # the switch does something
+
+
+def test_softcap_softmax_bounds_limit_and_library():
+    """MatMul-Scale-TanhSoftcap-Softmax.  (1) brute force with math.tanh / math.exp; (2) the capped scores lie in
+    (-c, c), so no two probabilities of a row differ by more than a factor e^(2c); (3) c -> infinity recovers the
+    plain softmax; (4) library cross-check in fp64; (5) the mask applies after the cap: masked entries are exactly 0."""
+    r = _rng(42)
+    A, B = 3.0 * r.standard_normal((6, 5)), 3.0 * r.standard_normal((5, 7))
+    alpha, c = 0.7, 2.0
+    P = orc.scale_mask_softmax(A, B, alpha, None, softcap=c)
+    for i in range(6):
+        t = [c * math.tanh(alpha * sum(A[i, k] * B[k, j] for k in range(5)) / c) for j in range(7)]
+        m = max(t)
+        e = [math.exp(x - m) for x in t]
+        np.testing.assert_allclose(P[i], [x / sum(e) for x in e], rtol=0, atol=1e-14)
+    assert (P.max(-1) / P.min(-1) < math.exp(2 * c)).all()
+    plain = orc.scale_mask_softmax(A, B, alpha, None)
+    assert (plain.max(-1) / plain.min(-1)).max() > math.exp(2 * c)        # uncapped rows exceed the bound: the cap matters
+    np.testing.assert_allclose(orc.scale_mask_softmax(A, B, alpha, None, softcap=1e9), plain, rtol=0, atol=1e-12)
+    Z = torch.from_numpy(A) @ torch.from_numpy(B) * alpha
+    lib = torch.softmax(c * torch.tanh(Z / c), dim=-1).numpy()
+    np.testing.assert_allclose(P, lib, rtol=0, atol=1e-14)
+    Pm = orc.scale_mask_softmax(A[:, :5], B[:, :6], alpha, orc.causal_mask(6, 6), softcap=c)
+    assert (Pm[np.triu_indices(6, 1)] == 0).all() and np.allclose(Pm.sum(-1), 1.0, atol=1e-12) and Pm[0, 0] == 1.0

@@ -124,7 +124,7 @@ class Workload:
         return total
 
 
-def _gemm_epilogue_ln(name, seed, M, N, K, affine):
+def _gemm_epilogue_ln(name, seed, M, N, K, affine, relu=False):
     t = {
         "A": normal_bf16(seed, 0, (M, K)),
         "B": normal_bf16(seed, 1, (K, N), std=1.0 / math.sqrt(K)),
@@ -135,16 +135,17 @@ def _gemm_epilogue_ln(name, seed, M, N, K, affine):
         t["gamma"] = normal_bf16(seed, 4, (N,), mean=1.0, std=0.02)
         t["beta"] = normal_bf16(seed, 5, (N,), mean=0.0, std=0.02)
     return Workload(name, KIND_BIAS_RES_LAYERNORM, {"M": M, "N": N, "K": K},
-                    {"alpha": 1.0, "eps": 1e-5}, t)
+                    {"alpha": 1.0, "eps": 1e-5, "relu": bool(relu)}, t)
 
 
-def post_norm(M=256, N=256, K=256, seed=0, affine=False, name=None) -> Workload:
-    """Y = LayerNorm(X.W + b + R).  X,R ~ N(0,1); W ~ N(0, var 1/K); b ~ U(-0.1, 0.1)."""
-    return _gemm_epilogue_ln(name or f"post_norm_{M}x{N}x{K}", seed, M, N, K, affine)
+def post_norm(M=256, N=256, K=256, seed=0, affine=False, name=None, relu=False) -> Workload:
+    """Y = LayerNorm(X.W + b + R) (then ReLU if ``relu``).  X,R ~ N(0,1); W ~ N(0, var 1/K); b ~ U(-0.1, 0.1)."""
+    return _gemm_epilogue_ln(name or f"post_norm_{M}x{N}x{K}", seed, M, N, K, affine, relu)
 
 
-def complex_subgraph(M=8192, N=4096, K=4096, seed=2, name=None) -> Workload:
-    """Z = X.W + b; H = GELU_tanh(Z) + R; Y = RMSNorm(H).g; row max / argmax of Y."""
+def complex_subgraph(M=8192, N=4096, K=4096, seed=2, name=None, activation=True, residual=True) -> Workload:
+    """Z = X.W + b; H = GELU_tanh(Z) + R; Y = RMSNorm(H).g; row max / argmax of Y.  Without the activation and the
+    residual this is the plain bias + RMSNorm pattern."""
     t = {
         "A": normal_bf16(seed, 0, (M, K)),
         "B": normal_bf16(seed, 1, (K, N), std=1.0 / math.sqrt(K)),
@@ -152,19 +153,22 @@ def complex_subgraph(M=8192, N=4096, K=4096, seed=2, name=None) -> Workload:
         "residual": normal_bf16(seed, 3, (M, N)),
         "gamma": normal_bf16(seed, 4, (N,), mean=1.0, std=0.02),
     }
+    if not residual:
+        del t["residual"]
     return Workload(name or f"complex_subgraph_{M}x{N}x{K}", KIND_BIAS_GELU_RES_RMSNORM_MAX,
-                    {"M": M, "N": N, "K": K}, {"alpha": 1.0, "eps": 1e-5}, t)
+                    {"M": M, "N": N, "K": K}, {"alpha": 1.0, "eps": 1e-5, "activation": bool(activation)}, t)
 
 
-def scaled_masked_softmax(batch=64, M=2048, N=2048, K=64, seed=3, causal=True, name=None) -> Workload:
-    """P = softmax(alpha * A.B + mask) per batch; alpha = 1/sqrt(K); causal 0 / -inf mask."""
+def scaled_masked_softmax(batch=64, M=2048, N=2048, K=64, seed=3, causal=True, name=None, softcap=0.0) -> Workload:
+    """P = softmax(alpha * A.B + mask) per batch; alpha = 1/sqrt(K); causal 0 / -inf mask; ``softcap`` > 0 passes the
+    scaled scores through softcap * tanh(. / softcap) first."""
     t = {
         "A": normal_bf16(seed, 0, (batch, M, K)),
         "B": normal_bf16(seed, 1, (batch, K, N)),
     }
     return Workload(name or f"softmax_{batch}x{M}x{N}x{K}", KIND_SCALE_MASK_SOFTMAX,
                     {"batch": batch, "M": M, "N": N, "K": K},
-                    {"alpha": 1.0 / math.sqrt(K), "causal": bool(causal)}, t)
+                    {"alpha": 1.0 / math.sqrt(K), "causal": bool(causal), "softcap": float(softcap)}, t)
 
 
 def b2b_mlp(M=32768, K=128, N1=512, N2=128, seed=4, affine=False, name=None) -> Workload:
