@@ -72,8 +72,16 @@ typedef struct {
   float alpha;              /* scales the accumulator before anything else */
   float eps;                /* added to the variance / mean square inside the square root */
   int32_t fused;            /* 1 = fused kernel, 0 = in-library unfused path */
+  uint32_t flags;           /* COMFUSE_FLAG_* bits, 0 for the op lists exactly as described at the enum */
+  float softcap;            /* SOFTMAX kind: if > 0, the scaled scores become softcap * tanh(alpha*A.B / softcap) before
+                               the mask is added (Sec. 6.2, MatMul-Scale-TanhSoftcap-Softmax); must be 0 for other kinds */
   int32_t reserved;         /* must be 0 */
 } comfuse_gemm_desc_t;
+
+/* Variants of the op lists (the three evaluation patterns of Sec. 6.2 are LAYERNORM + POST_RELU, RMSNORM_MAX +
+ * NO_ACTIVATION without a residual, and SOFTMAX with softcap > 0). */
+#define COMFUSE_FLAG_POST_RELU 1u      /* BIAS_RES_LAYERNORM kind only: Y = max(Y, 0) after the affine step            */
+#define COMFUSE_FLAG_NO_ACTIVATION 2u  /* BIAS_GELU_RES_RMSNORM_MAX kind only: H = alpha*A.B + bias + R, no GELU       */
 
 /* Runtime-parameter table of the op list.  bf16 device vectors of length N; NULL means absent
  * (bias, residual: 0; gamma: 1; beta: 0).  row_max / row_argmax: [batch*M] outputs of the

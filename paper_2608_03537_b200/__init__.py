@@ -31,6 +31,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ER
 EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 0, 1, 2
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
+FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2
 
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
@@ -55,7 +56,7 @@ class GemmDesc(Structure):
         ("lda", c_int64), ("ldb", c_int64), ("ldr", c_int64), ("ldy", c_int64),
         ("batch_stride_a", c_int64), ("batch_stride_b", c_int64), ("batch_stride_r", c_int64), ("batch_stride_y", c_int64),
         ("kind", c_int32), ("mask", c_int32), ("alpha", c_float), ("eps", c_float),
-        ("fused", c_int32), ("reserved", c_int32),
+        ("fused", c_int32), ("flags", ctypes.c_uint32), ("softcap", c_float), ("reserved", c_int32),
     ]
 
 
@@ -132,7 +133,8 @@ def _stream(stream=None):
     return c_void_p(s.cuda_stream)
 
 
-def make_gemm_desc(A, B, Y, kind, *, residual=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True) -> GemmDesc:
+def make_gemm_desc(A, B, Y, kind, *, residual=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, flags=0,
+                   softcap=0.0) -> GemmDesc:
     """Describe A [b, M, K] (or [M, K]), B [b, K, N] (or [K, N]), Y [b, M, N] from torch tensors' shapes and strides."""
     batched = A.dim() == 3
     batch = A.shape[0] if batched else 1
@@ -149,6 +151,7 @@ def make_gemm_desc(A, B, Y, kind, *, residual=None, alpha=1.0, eps=1e-5, mask=MA
     d.batch_stride_y = Y.stride(0) if batched else M * d.ldy
     d.batch_stride_r = (residual.stride(0) if batched else M * d.ldr) if residual is not None else M * N
     d.kind, d.mask, d.alpha, d.eps, d.fused, d.reserved = int(kind), int(mask), float(alpha), float(eps), int(bool(fused)), 0
+    d.flags, d.softcap = int(flags), float(softcap)
     return d
 
 
@@ -161,11 +164,12 @@ def workspace_size(desc: GemmDesc) -> int:
 
 
 def gemm_epilogue(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=None, mask_tensor=None, row_max=None,
-                  row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, workspace=None, stream=None):
+                  row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, workspace=None, stream=None, flags=0,
+                  softcap=0.0):
     """Enqueue Y = subgraph(alpha * A.B) on the current (or given) stream.  Tensors are CUDA bf16 (row_max fp32,
     row_argmax int32).  ``workspace`` is a CUDA uint8 tensor of at least workspace_size(desc) bytes (unfused path, and fused LayerNorm /
     RMSNorm rows wider than 4096 columns)."""
-    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused)
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused, flags=flags, softcap=softcap)
     args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
     st = lib().comfuse_gemm_epilogue(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), ws_ptr, ws_bytes, _stream(stream))

@@ -141,6 +141,10 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
   if (d->mask < COMFUSE_MASK_NONE || d->mask > COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_INVALID_ARG;
   if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
   if (d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->flags & ~(COMFUSE_FLAG_POST_RELU | COMFUSE_FLAG_NO_ACTIVATION)) return COMFUSE_ERR_INVALID_ARG;
+  if ((d->flags & COMFUSE_FLAG_POST_RELU) && d->kind != COMFUSE_EPI_BIAS_RES_LAYERNORM) return COMFUSE_ERR_INVALID_ARG;
+  if ((d->flags & COMFUSE_FLAG_NO_ACTIVATION) && d->kind != COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX) return COMFUSE_ERR_INVALID_ARG;
+  if (!(d->softcap >= 0.f) || (d->softcap > 0.f && d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX)) return COMFUSE_ERR_INVALID_ARG;
   if (d->lda < d->K || d->ldb < d->N || d->ldy < d->N) return COMFUSE_ERR_INVALID_ARG;
   if (d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && d->mask != COMFUSE_MASK_NONE) return COMFUSE_ERR_INVALID_ARG;
   if (!mult8(d->N) || !mult8(d->K)) return COMFUSE_ERR_ALIGNMENT;
@@ -265,6 +269,9 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.total_tiles = p.batch * p.mblocks;
   p.alpha = desc->alpha; p.eps = desc->eps;
   p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
+  p.post_relu = (desc->flags & COMFUSE_FLAG_POST_RELU) ? 1 : 0;
+  p.no_activation = (desc->flags & COMFUSE_FLAG_NO_ACTIVATION) ? 1 : 0;
+  p.softcap = desc->softcap;
   p.status = dev->status_word;
   p.timeout_ns = timeout_ns();
 #ifdef COMFUSE_TRACE
@@ -302,6 +309,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
       r.gamma = static_cast<const uint16_t*>(a.gamma);
       r.beta = static_cast<const uint16_t*>(a.beta);
       r.eps = desc->eps;
+      r.post_relu = p.post_relu;
       r.Y = static_cast<uint16_t*>(Y);
       r.ldy = desc->ldy; r.batch_stride_y = bsy;
       r.row_max = a.row_max; r.row_argmax = a.row_argmax;
@@ -328,6 +336,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   r.mask = desc->mask == COMFUSE_MASK_ADDITIVE ? static_cast<const uint16_t*>(a.mask) : nullptr;
   r.causal = p.causal;
   r.alpha = desc->alpha; r.eps = desc->eps;
+  r.post_relu = p.post_relu; r.no_activation = p.no_activation; r.softcap = desc->softcap;
   r.Y = static_cast<uint16_t*>(Y);
   r.ldy = desc->ldy; r.batch_stride_y = bsy;
   r.row_max = a.row_max; r.row_argmax = a.row_argmax;

@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(32 * (3 + 4 * EPW), 1)
 fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
   using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW>;
+  constexpr bool kIsRms = EPI == EPI_RMS_MAX || EPI == EPI_RMS_MAX_LINEAR;  // the latter: no GELU in stage 1
   constexpr int BN = Cfg::BN;
   constexpr int NSUB = Cfg::NSUB;
   constexpr int ESUB = Cfg::ESUB;
@@ -160,7 +161,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int cluster_id = blockIdx.x / CLUSTER;
   const int num_clusters = gridDim.x / CLUSTER;
   const int KB = (p.K + 63) >> 6;
-  const bool has_res = (EPI == EPI_LN || EPI == EPI_RMS_MAX) && p.residual != nullptr;
+  const bool has_res = (EPI == EPI_LN || kIsRms) && p.residual != nullptr;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
@@ -413,7 +414,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int xpar = 0;
     uint32_t xphase = 0;
     (void)xpar; (void)xphase; (void)s_pre; (void)s_stats; (void)s_bias; (void)s_gamma; (void)s_beta;
-    if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
+    if constexpr (EPI == EPI_LN || kIsRms) {
       // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once, by the epilogue warps
       // (they have nothing else to do until the first accumulator is complete); wide rows: the bias of the tile's column
       // block is loaded per tile instead, gamma/beta are identity
@@ -546,7 +547,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           release_accumulator(sub);
         }
-      } else if constexpr (EPI == EPI_LN || EPI == EPI_RMS_MAX) {
+      } else if constexpr (EPI == EPI_LN || kIsRms) {
         // ---------------- stage 1 (compute): x = f(alpha*Acc + bias, R); thread-local partial statistic; x is written
         // back over the accumulator in TMEM (the bypass path of Sec. 3.2)
         float2 part = make_float2(0.f, 0.f);
@@ -623,10 +624,14 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 bb = bias4[j];
-                  const float2 h01 = add2(gelu_tanh_f32x2(fma2(al, f2_from_bits(v[4 * j], v[4 * j + 1]), make_float2(bb.x, bb.y))),
-                                          bf16x2_to_f2(r32[half * 16 + 2 * j]));
-                  const float2 h23 = add2(gelu_tanh_f32x2(fma2(al, f2_from_bits(v[4 * j + 2], v[4 * j + 3]), make_float2(bb.z, bb.w))),
-                                          bf16x2_to_f2(r32[half * 16 + 2 * j + 1]));
+                  float2 z01 = fma2(al, f2_from_bits(v[4 * j], v[4 * j + 1]), make_float2(bb.x, bb.y));
+                  float2 z23 = fma2(al, f2_from_bits(v[4 * j + 2], v[4 * j + 3]), make_float2(bb.z, bb.w));
+                  if constexpr (EPI == EPI_RMS_MAX) {
+                    z01 = gelu_tanh_f32x2(z01);
+                    z23 = gelu_tanh_f32x2(z23);
+                  }
+                  const float2 h01 = add2(z01, bf16x2_to_f2(r32[half * 16 + 2 * j]));
+                  const float2 h23 = add2(z23, bf16x2_to_f2(r32[half * 16 + 2 * j + 1]));
                   v[4 * j] = __float_as_uint(h01.x); v[4 * j + 1] = __float_as_uint(h01.y);
                   v[4 * j + 2] = __float_as_uint(h23.x); v[4 * j + 3] = __float_as_uint(h23.y);
                   q01 = fma2(h01, h01, q01);
@@ -662,6 +667,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
         }
         // ---------------- stage 2 (PostOp): normalise the resident x, round once, store
+        const float relu_floor = (p.post_relu && !p.wide) ? 0.f : -INFINITY;  // wide rows: the second kernel applies it
+        (void)relu_floor;
         float best = -INFINITY;
         int best_col = 0x7FFFFFFF;
 #pragma unroll
@@ -689,7 +696,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const float2 n23 = fma2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd), splat2(-mu * rstd));
                   const float2 y01 = fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y));
                   const float2 y23 = fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w));
-                  y0 = y01.x; y1 = y01.y; y2 = y23.x; y3 = y23.y;
+                  // relu_floor is 0 for the LayerNorm-ReLU pattern, -inf otherwise
+                  y0 = fmaxf(y01.x, relu_floor); y1 = fmaxf(y01.y, relu_floor); y2 = fmaxf(y23.x, relu_floor); y3 = fmaxf(y23.y, relu_floor);
                 } else {
                   const float2 y01 = mul2(mul2(f2_from_bits(v[4 * j], v[4 * j + 1]), splat2(rstd)), make_float2(gg.x, gg.y));
                   const float2 y23 = mul2(mul2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd)), make_float2(gg.z, gg.w));
@@ -709,7 +717,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
           release_accumulator(sub);
         }
-        if (EPI == EPI_RMS_MAX && !p.wide) {
+        if (kIsRms && !p.wide) {
           // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
           const float2 mx = cluster_row_reduce<CN, MergeArgmax, EPW>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
                                                    s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
@@ -721,7 +729,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
       } else {  // EPI_SOFTMAX
         // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
-        const float sc = p.alpha * 1.4426950408889634f;
+        // with a soft-cap the accumulators are mapped to capped log2-domain scores right after they are loaded, and sc = 1
+        const bool capped = p.softcap > 0.f;
+        const SoftcapLog2 cap_fn(p.alpha, capped ? p.softcap : 1.f);
+        const float sc = capped ? 1.f : p.alpha * 1.4426950408889634f;
         // fragment classification under the causal mask, uniform over the warp's 32 rows so that the warp-wide TMEM
         // loads stay convergent: 2 = all live, 1 = crosses the diagonal, 0 = all masked
         const int wrow0 = m0 + q * 32;
@@ -743,6 +754,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (st == 0) continue;
               uint32_t v[32];
               tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              if (capped) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
+              }
               float m0v = -INFINITY, m1v = -INFINITY;
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
@@ -771,6 +786,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (st == 0) continue;
               uint32_t v[32];
               tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              if (capped) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
+              }
               float s0 = 0.f, s1 = 0.f;
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {

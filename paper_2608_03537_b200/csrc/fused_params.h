@@ -6,7 +6,8 @@
 
 namespace comfuse {
 
-enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3 };
+// EPI_RMS_MAX_LINEAR: the RMSNorm op list without its GELU (a kernel instantiation of its own, chosen by FusedParams::no_activation)
+enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3, EPI_RMS_MAX_LINEAR = 4 };
 
 struct FusedParams {
   int M, N, K, batch;
@@ -16,6 +17,9 @@ struct FusedParams {
   int total_tiles;  // batch * mblocks * nblocks
   float alpha, eps;
   int causal;
+  int post_relu;      // LayerNorm kind: Y = max(Y, 0) after the affine step
+  int no_activation;  // RMSNorm kind: no GELU in stage 1
+  float softcap;      // softmax kind: > 0 = scaled scores pass through softcap * tanh(. / softcap)
   const uint16_t* bias;
   const uint16_t* gamma;
   const uint16_t* beta;

@@ -7,7 +7,9 @@ namespace comfuse {
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
 #define COMFUSE_CASE(n, b0, b1, cn, nst, lock) \
   case n:                                      \
-    return supported_only ? cudaSuccess : launch_pair_instance<EPI_RMS_MAX, b0, b1, cn, nst, lock>(maps, p, st);
+    return supported_only   ? cudaSuccess                                                                        \
+           : p.no_activation ? launch_pair_instance<EPI_RMS_MAX_LINEAR, b0, b1, cn, nst, lock>(maps, p, st)        \
+                             : launch_pair_instance<EPI_RMS_MAX, b0, b1, cn, nst, lock>(maps, p, st);
   // Two sub-tiles advance in lock step (lock = 1): the A tile is fetched once per K block for both.
   // Wide rows (p.wide): every cluster covers one 4096-column block of the row, p.nblocks blocks per row.
   switch (p.wide ? kWideRowBlock : p.N) {

@@ -107,9 +107,12 @@ __global__ void __launch_bounds__(256) row_epilogue_kernel(const RowParams p) {
       if constexpr (KIND == EPI_LN) {
         x[v][j] = ok ? fmaf(p.alpha, zf[j], bf[j]) + rf[j] : 0.f;
       } else if constexpr (KIND == EPI_RMS_MAX) {
-        x[v][j] = ok ? gelu_tanh_ref(fmaf(p.alpha, zf[j], bf[j])) + rf[j] : 0.f;
+        const float z = fmaf(p.alpha, zf[j], bf[j]);
+        x[v][j] = ok ? (p.no_activation ? z : gelu_tanh_ref(z)) + rf[j] : 0.f;
       } else {
-        float tv = p.alpha * zf[j] + mf[j];
+        float tv = p.alpha * zf[j];
+        if (p.softcap > 0.f) tv = p.softcap * tanhf(tv / p.softcap);
+        tv += mf[j];
         if (p.causal && col > i) tv = -INFINITY;
         x[v][j] = ok ? tv : -INFINITY;
       }
@@ -144,7 +147,10 @@ __global__ void __launch_bounds__(256) row_epilogue_kernel(const RowParams p) {
       unpack8(p.beta ? __ldg(reinterpret_cast<const uint4*>(p.beta) + vi) : make_uint4(0, 0, 0, 0), bf);
       float o[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) o[j] = fmaf((x[v][j] - mu) * rstd, gf[j], bf[j]);
+      for (int j = 0; j < 8; ++j) {
+        o[j] = fmaf((x[v][j] - mu) * rstd, gf[j], bf[j]);
+        if (p.post_relu) o[j] = fmaxf(o[j], 0.f);
+      }
       reinterpret_cast<uint4*>(y)[vi] = make_uint4(pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
     }
   } else if constexpr (KIND == EPI_RMS_MAX) {
@@ -250,6 +256,7 @@ __global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p,
     for (int j = 0; j < 8; ++j) {
       if constexpr (KIND == EPI_LN) {
         o[j] = fmaf((xf[j] - mu) * rstd, gf[j], bf[j]);
+        if (p.post_relu) o[j] = fmaxf(o[j], 0.f);
       } else {
         o[j] = xf[j] * rstd * gf[j];
         if (o[j] > best) { best = o[j]; best_col = vi * 8 + j; }

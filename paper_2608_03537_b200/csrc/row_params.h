@@ -18,6 +18,8 @@ struct RowParams {
   const uint16_t* mask;  // additive [M, N] bf16 or nullptr
   int causal;
   float alpha, eps;
+  int post_relu, no_activation;  // variants of the LayerNorm / RMSNorm op lists (see FusedParams)
+  float softcap;                 // softmax: soft-cap of the scaled scores, 0 = none
   uint16_t* Y;
   long long ldy, batch_stride_y;
   float* row_max;

@@ -314,6 +314,23 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Tanh soft-cap of an attention score, result in the log2 domain the softmax kernels work in:
+//   t = log2(e) * cap * tanh(alpha * acc / cap) = c1 - 2 * c1 / (1 + 2^(acc * c3)),  c1 = cap * log2 e,  c3 = 2 * alpha * log2 e / cap.
+// Built from ex2 and rcp (absolute error of tanh about 1e-7) rather than tanh.approx, whose 2^-11 relative error times
+// the cap would move the probabilities by more than their rounding.
+struct SoftcapLog2 {
+  float c1, c3;
+  __device__ __forceinline__ SoftcapLog2(float alpha, float cap)
+      : c1(cap * 1.4426950408889634f), c3(2.f * alpha * 1.4426950408889634f / cap) {}
+  __device__ __forceinline__ float operator()(float acc) const {
+    return fmaf(-2.f * c1, rcp_approx(1.f + ex2_approx(acc * c3)), c1);
+  }
+};
 // Packed fp32x2 arithmetic (one instruction for two lanes of a float2): halves the issue slots of the epilogue math.
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }

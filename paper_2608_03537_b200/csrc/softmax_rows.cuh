@@ -279,7 +279,10 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     uint32_t slot_uses[2] = {0, 0};
     uint32_t unit = 0, nbox = 0, tile_par = 0;
     // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
-    const float sc = p.alpha * 1.4426950408889634f;
+    // with a soft-cap the accumulators are mapped to capped log2-domain scores right after they are loaded, and sc = 1
+    const bool capped = p.softcap > 0.f;
+    const SoftcapLog2 cap_fn(p.alpha, capped ? p.softcap : 1.f);
+    const float sc = capped ? 1.f : p.alpha * 1.4426950408889634f;
     constexpr uint32_t poly_pairs = Cfg::POLY_PAIRS;
 
 #ifdef COMFUSE_TRACE
@@ -338,6 +341,10 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               if (st == 0) continue;
               uint32_t v[32];
               tmem_ld_32cols(taddr + half * 32, v);
+              if (capped) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
+              }
               float2 tv[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) tv[j] = mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc));
@@ -383,6 +390,10 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               } else {
                 uint32_t v[32];
                 tmem_ld_32cols(taddr + half * 32, v);
+                if (capped) {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
+                }
                 float2 ev[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {

@@ -75,8 +75,11 @@ def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
         kw = dict(alpha=w.scalars["alpha"], mask=cf.MASK_CAUSAL if w.scalars.get("causal") else cf.MASK_NONE)
         if "mask" in T:
             kw.update(mask=cf.MASK_ADDITIVE, mask_tensor=T["mask"])
+    flags = (cf.FLAG_POST_RELU if w.scalars.get("relu") else 0) | (0 if w.scalars.get("activation", True) else cf.FLAG_NO_ACTIVATION)
+    kw.update(flags=flags, softcap=w.scalars.get("softcap", 0.0))
     desc = cf.make_gemm_desc(T["A"], T["B"], Y, kind, residual=kw.get("residual"), alpha=kw.get("alpha", 1.0),
-                             eps=kw.get("eps", 1e-5), mask=kw.get("mask", cf.MASK_NONE), fused=fused)
+                             eps=kw.get("eps", 1e-5), mask=kw.get("mask", cf.MASK_NONE), fused=fused, flags=flags,
+                             softcap=kw["softcap"])
     ws = torch.empty(max(cf.workspace_size(desc), 16), dtype=torch.uint8, device=dev)
     cf.gemm_epilogue(T["A"], T["B"], Y, kind, fused=fused, workspace=ws, **kw)
     return out

@@ -84,6 +84,19 @@ def test_wide_row_and_host_staging_sizes():
     assert n.value == 2 * 1000 * 128 * 2
 
 
+def test_pattern_variant_flags_are_checked():
+    assert _ws(_desc(flags=cf.FLAG_POST_RELU))[0] == cf.OK                                  # LayerNorm + ReLU
+    assert _ws(_desc(flags=cf.FLAG_NO_ACTIVATION))[0] == cf.ERR_INVALID_ARG                 # belongs to the RMSNorm kind
+    assert _ws(_desc(kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, flags=cf.FLAG_NO_ACTIVATION))[0] == cf.OK
+    assert _ws(_desc(kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, flags=cf.FLAG_POST_RELU))[0] == cf.ERR_INVALID_ARG
+    assert _ws(_desc(flags=4))[0] == cf.ERR_INVALID_ARG                                     # unknown bit
+    assert _ws(_desc(softcap=30.0))[0] == cf.ERR_INVALID_ARG                                # soft-cap belongs to the softmax kind
+    sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldb=2048, ldr=2048, ldy=2048)
+    assert _ws(_desc(**sm, softcap=30.0))[0] == cf.OK
+    assert _ws(_desc(**sm, softcap=-1.0))[0] == cf.ERR_INVALID_ARG
+    assert _ws(_desc(**sm, softcap=float("nan")))[0] == cf.ERR_INVALID_ARG
+
+
 def test_gemm_epilogue_rejects_bad_arguments_before_any_launch():
     L = cf.lib()
     d = _desc()

@@ -248,3 +248,44 @@ def test_back_to_back_dependent_launches_see_each_others_results(cuda_device):
         b = chain(sync=False)
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
     assert cf.last_device_status() == cf.OK
+
+
+# --------------------------------------------------------------------------------------------- the Sec. 6.2 patterns
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,N,K", [(300, 768, 200), (200, 4096, 128), (300, 8192, 72)])
+def test_matmul_bias_layernorm_relu_pattern(M, N, K, fused, cuda_device):
+    w = wl.post_norm(M, N, K, seed=M + N + K + 1, affine=True, relu=True)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN+ReLU {M}x{N}x{K} fused={fused}")
+    Y = got["Y"].float()
+    assert (Y >= 0).all().item() and (Y == 0).float().mean().item() > 0.3     # about half the values are clamped
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,N,K", [(140, 768, 64), (150, 4096, 128), (129, 8192, 64)])
+def test_matmul_bias_rmsnorm_pattern(M, N, K, fused, cuda_device):
+    """RMSNorm(A.B + bias) * g: no activation, no residual (the row max / argmax outputs are still produced)."""
+    w = wl.complex_subgraph(M, N, K, seed=M + N + 2, activation=False, residual=False)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"bias+RMS {M}x{N}x{K} fused={fused}",
+                    rowmax_tol=5e-3 if (fused and N <= 4096) else 3e-2)
+
+
+SOFTCAP_CASES = [
+    # batch, M, N, K, causal, softcap
+    (2, 512, 512, 64, True, 5.0),      # row kernel (short K), strong cap
+    (1, 300, 1000, 64, False, 30.0),   # row kernel, ragged N, mild cap
+    (2, 256, 2048, 320, False, 5.0),   # cluster kernel (K > 256)
+    (1, 1024, 1024, 264, True, 2.0),   # cluster kernel, causal
+]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M,N,K,causal,cap", SOFTCAP_CASES)
+def test_matmul_scale_tanh_softcap_softmax_pattern(batch, M, N, K, causal, cap, fused, cuda_device):
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=N + K + 7, causal=causal, softcap=cap)
+    # make the cap bite: scores of standard deviation ~4 instead of ~1
+    w.scalars["alpha"] *= 4.0
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"softcap {cap} b{batch} {M}x{N}x{K} causal={causal} fused={fused}",
+                    softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
