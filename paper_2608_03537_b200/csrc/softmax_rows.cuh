@@ -144,6 +144,9 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // every operand chunk is read twice per tile and the K matrix by every tile of its batch, while 16 times as many
+      // output bytes stream through the L2: ask it to keep the operands
+      const uint64_t keep = l2_policy_evict_last();
       for (int r = 0; r < rounds && ok; ++r) {
         int b, mpair0, L;
         if (!tile_at(r, b, mpair0, L)) continue;
@@ -155,11 +158,11 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint32_t full = map_to_cta(bar_full(stage), 0);
           mbar_arrive_expect_tx_cluster(full, Cfg::STAGE_BYTES);
-          tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
+          tma_load_3d_pair_hint(sa, &tmA, full, kb * 64, m0, b, keep);
           // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
           const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
-          tma_load_3d_pair(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b);
-          tma_load_3d_pair(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b);
+          tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b, keep);
+          tma_load_3d_pair_hint(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b, keep);
           if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
         }
         }
@@ -216,6 +219,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int h = e >> 2;
       constexpr int D = YBOXES - 1;
       const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + e * YBOXES * Cfg::WARP_BOX_BYTES;
+      const uint64_t stream_out = l2_policy_evict_first();  // the output is never read again
       uint32_t n = 0;
       bool ok = true;
       for (int r = 0; r < rounds && ok; ++r) {
@@ -229,7 +233,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #ifdef COMFUSE_TRACE
         if (!(p.trace_flags & 1))
 #endif
-        tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, mpair0 + static_cast<int>(pm) * 128 + q * 32, b);
+        tma_store_3d_hint(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, mpair0 + static_cast<int>(pm) * 128 + q * 32, b, stream_out);
         tma_store_commit();
         if (n >= static_cast<uint32_t>(D)) {
           tma_store_wait_read<D>();
@@ -247,6 +251,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // stores: plain stores would share the SM's memory-instruction queue with the epilogue's exponentials and
     // shared-memory traffic).  Few boxes in flight, so that a staged box never queues far behind zeros.
     if (lane < Cfg::ZERO_TMA_LANES && p.causal) {
+      const uint64_t stream_out = l2_policy_evict_first();
       uint32_t k = 0;
       for (int r = 0; r < rounds; ++r) {
         int b, mpair0, L;
@@ -261,7 +266,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #ifdef COMFUSE_TRACE
             if (!(p.trace_flags & 4))
 #endif
-            tma_store_3d(&tmY, smem_base + Cfg::OFF_ZERO, col, y0 + (i & 3) * 32, b);
+            tma_store_3d_hint(&tmY, smem_base + Cfg::OFF_ZERO, col, y0 + (i & 3) * 32, b, stream_out);
             tma_store_commit();
           }
       }
