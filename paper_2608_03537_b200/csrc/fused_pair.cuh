@@ -233,6 +233,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // A stage is handed back by the UMMA commit (K-block use) or by the eight epilogue warps (residual use); the two
       // kinds have their own barriers, so the producer remembers each stage's last use and each barrier's phase.
       uint32_t used = 0, last_res = 0, empty_bits = 0, rdone_bits = 0;
+      // L2 priorities: the B operand (weights) is re-read by every row block, the residual is read exactly once
+      const uint64_t once = l2_policy_evict_first();
       auto wait_stage_free = [&](int st) {
         const uint32_t bit = 1u << st;
         if (!(used & bit)) return true;
@@ -289,7 +291,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               const uint32_t sr = smem_base + ring.stage * Cfg::STAGE_BYTES;
               mbar_arrive_expect_tx(bar_rfull(ring.stage), ng * Cfg::GROUP_BYTES);
               for (int g = 0; g < ng; ++g)
-                tma_load_3d(sr + g * Cfg::GROUP_BYTES, &tmR, bar_rfull(ring.stage), group_col(ncta0, lg0 + g0 + g), m0, b);
+                tma_load_3d_hint(sr + g * Cfg::GROUP_BYTES, &tmR, bar_rfull(ring.stage), group_col(ncta0, lg0 + g0 + g), m0, b, once);
               ring.advance();
             }
           }
@@ -363,6 +365,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int h = e >> 2;
       constexpr int D = Cfg::YBOXES - 1;
       const uint32_t ybox0 = smem_base + Cfg::OFF_YBUF + e * Cfg::YBOXES * Cfg::WARP_BOX_BYTES;
+      const uint64_t once = l2_policy_evict_first();  // the output is not read again by this kernel
       uint32_t n = 0;
       bool ok = true;
       for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
@@ -383,7 +386,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
               if (!(p.trace_flags & 1))
 #endif
-              tma_store_3d(&tmY, ring_box(e, kk), col, m0 + q * 32, b);
+              tma_store_3d_hint(&tmY, ring_box(e, kk), col, m0 + q * 32, b, once);
               tma_store_commit();
               ++kk;
               continue;
@@ -393,7 +396,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
             if (!(p.trace_flags & 1))
 #endif
-            tma_store_3d(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, m0 + q * 32, b);
+            tma_store_3d_hint(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, m0 + q * 32, b, once);
             tma_store_commit();
             if (n >= static_cast<uint32_t>(D)) {
               tma_store_wait_read<D>();
