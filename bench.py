@@ -34,7 +34,7 @@ METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
 WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
 # captures summarised under profiles/, in bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 69_505_280, "c3": 270_358_528, "c4": 550_356_992, "c5": 8_714_496}
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": 70_144_768, "c3": 221_126_912, "c4": 513_010_432, "c5": 8_714_240}
 
 
 def load_peaks():
