@@ -176,6 +176,13 @@ def b2b_from_intermediate(S, X, W2, b2, gamma=None, beta=None, eps=1e-5):
     return layernorm_rows(O, gamma, beta, eps)
 
 
+def b2b_softmax_attention(Q, Kt, V, alpha=1.0):
+    """Sec. 4, Eq. 2 with F = row softmax (the attention-form instance the paper evaluates as Target-Attention,
+    Sec. 6.3):  P = alpha * Q Kt,  S = softmax(P) over the source positions,  O = S V.
+    Q [.., M, d], Kt [.., d, S] (the keys already transposed: a plain row-major second operand), V [.., S, d2]."""
+    return gemm(softmax_rows(alpha * gemm(Q, Kt)), V)
+
+
 # --------------------------------------------------------------------------- partial-statistics merges
 # The fused kernels combine per-tile partial statistics (Sec. 3.1: thread-local aggregation, then
 # hierarchical aggregation up to the inter-CTA level).  The merges below are the textbook pairwise

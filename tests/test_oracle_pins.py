@@ -397,3 +397,33 @@ def test_softcap_softmax_bounds_limit_and_library():
     np.testing.assert_allclose(P, lib, rtol=0, atol=1e-14)
     Pm = orc.scale_mask_softmax(A[:, :5], B[:, :6], alpha, orc.causal_mask(6, 6), softcap=c)
     assert (Pm[np.triu_indices(6, 1)] == 0).all() and np.allclose(Pm.sum(-1), 1.0, atol=1e-12) and Pm[0, 0] == 1.0
+
+
+# ----------------------------------------------------------------------------- B2B with a reduction as F (attention form)
+def test_b2b_softmax_attention_brute_force_and_properties():
+    """Scalar-loop brute force; zero queries attend uniformly (every output row is the mean of the value rows); every output
+    lies inside the per-column range of V (rows of softmax are convex weights); a key that dominates one query's scores
+    makes that query's output its value row; batched call equals per-batch calls; library cross-check in fp64."""
+    r = _rng(50)
+    Q, Kt, V = r.standard_normal((5, 4)), r.standard_normal((4, 6)), r.standard_normal((6, 3))
+    alpha = 0.5
+    O = orc.b2b_softmax_attention(Q, Kt, V, alpha)
+    for i in range(5):
+        s = [alpha * sum(Q[i, k] * Kt[k, j] for k in range(4)) for j in range(6)]
+        m = max(s)
+        e = [math.exp(x - m) for x in s]
+        pr = [x / sum(e) for x in e]
+        for c in range(3):
+            assert abs(O[i, c] - sum(pr[j] * V[j, c] for j in range(6))) < 1e-13
+    np.testing.assert_allclose(orc.b2b_softmax_attention(np.zeros((2, 4)), Kt, V, alpha), np.tile(V.mean(0), (2, 1)), atol=1e-14)
+    assert (O >= V.min(0) - 1e-12).all() and (O <= V.max(0) + 1e-12).all()
+    Kd = Kt.copy()
+    Kd[:, 2] = 50.0 * Q[1] / np.dot(Q[1], Q[1])          # query 1 . key 2 = 50 / alpha-scaled: dominates that row
+    Od = orc.b2b_softmax_attention(Q, Kd, V, 1.0)
+    np.testing.assert_allclose(Od[1], V[2], atol=1e-9)
+    Qb, Kb, Vb = r.standard_normal((3, 5, 4)), r.standard_normal((3, 4, 6)), r.standard_normal((3, 6, 3))
+    Ob = orc.b2b_softmax_attention(Qb, Kb, Vb, alpha)
+    for b in range(3):
+        np.testing.assert_allclose(Ob[b], orc.b2b_softmax_attention(Qb[b], Kb[b], Vb[b], alpha), atol=1e-14)
+    lib = torch.softmax(torch.from_numpy(Q) @ torch.from_numpy(Kt) * alpha, dim=-1) @ torch.from_numpy(V)
+    np.testing.assert_allclose(O, lib.numpy(), atol=1e-13)

@@ -88,6 +88,7 @@ KIND_BIAS_RES_LAYERNORM = "bias_res_layernorm"
 KIND_BIAS_GELU_RES_RMSNORM_MAX = "bias_gelu_res_rmsnorm_max"
 KIND_SCALE_MASK_SOFTMAX = "scale_mask_softmax"
 KIND_B2B_MLP_LAYERNORM = "b2b_mlp_layernorm"
+KIND_B2B_SOFTMAX_ATTENTION = "b2b_softmax_attention"
 
 
 @dataclass
@@ -102,13 +103,15 @@ class Workload:
 
     def gemm_flops(self) -> float:
         d = self.dims
-        if self.kind == KIND_B2B_MLP_LAYERNORM:
-            return 2.0 * d["M"] * d["K"] * d["N1"] + 2.0 * d["M"] * d["N1"] * d["N2"]
+        if self.kind in (KIND_B2B_MLP_LAYERNORM, KIND_B2B_SOFTMAX_ATTENTION):
+            return d.get("batch", 1) * (2.0 * d["M"] * d["K"] * d["N1"] + 2.0 * d["M"] * d["N1"] * d["N2"])
         return 2.0 * d.get("batch", 1) * d["M"] * d["N"] * d["K"]
 
     def min_hbm_bytes(self) -> float:
         """Every operand read once and every output written once, nothing else."""
         d = self.dims
+        if self.kind == KIND_B2B_SOFTMAX_ATTENTION:
+            return 2.0 * d["batch"] * (d["M"] * d["K"] + d["K"] * d["N1"] + d["N1"] * d["N2"] + d["M"] * d["N2"])
         if self.kind == KIND_B2B_MLP_LAYERNORM:
             M, K, N1, N2 = d["M"], d["K"], d["N1"], d["N2"]
             return 2.0 * (M * K + K * N1 + N1 * N2 + N1 + N2 + M * N2) + (
@@ -189,6 +192,18 @@ def b2b_mlp(M=32768, K=128, N1=512, N2=128, seed=4, affine=False, name=None) -> 
 
 
 # The five named configurations (index = position in the benchmark's config list).
+def target_attention(batch=32, M=4096, S=256, d=128, seed=5, name=None) -> Workload:
+    """O = softmax(Q.Kt / sqrt(d)).V per batch: M target positions attend to S source positions (the paper's
+    Target-Attention shape is M = 4096, S = 256).  Q, Kt, V ~ N(0, 1)."""
+    t = {
+        "X": normal_bf16(seed, 0, (batch, M, d)),
+        "W1": normal_bf16(seed, 1, (batch, d, S)),
+        "W2": normal_bf16(seed, 2, (batch, S, d)),
+    }
+    return Workload(name or f"target_attention_{batch}x{M}x{S}x{d}", KIND_B2B_SOFTMAX_ATTENTION,
+                    {"batch": batch, "M": M, "K": d, "N1": S, "N2": d}, {"alpha": 1.0 / math.sqrt(d)}, t)
+
+
 def config(index: int) -> Workload:
     if index == 0:   # post-norm tiny, gamma = 1, beta = 0, seed 0
         return post_norm(256, 256, 256, seed=0, affine=False, name="c1_post_norm_tiny")
@@ -200,6 +215,8 @@ def config(index: int) -> Workload:
         return scaled_masked_softmax(64, 2048, 2048, 64, seed=3, name="c4_scaled_causal_softmax")
     if index == 4:   # back-to-back GEMM MLP with post-norm
         return b2b_mlp(32768, 128, 512, 128, seed=4, name="c5_b2b_mlp")
+    if index == 5:   # beyond the five named configurations: B2B with a reduction as F (attention form)
+        return target_attention(32, 4096, 256, 128, seed=5, name="a1_target_attention")
     raise IndexError(index)
 
 
