@@ -384,7 +384,7 @@ def run_comfuse(args):
             extra["unfused_error"] = str(e)
         # ---- context: the same step with its inputs and outputs resident in L2 (one buffer set, back to back), and the
         # GEMM(s) alone through the vendor library, so that "residual" = what the subgraph costs on top of the GEMM
-        # (Sec. 6.2 reports fusion benefit this way)
+        # (Sec. 6.1 reports fusion benefit this way: residual time)
         n3 = max(3, min(args.steps, 50))
         for i in range(3):
             step(sets[0])

@@ -74,11 +74,11 @@ typedef struct {
   int32_t fused;            /* 1 = fused kernel, 0 = in-library unfused path */
   uint32_t flags;           /* COMFUSE_FLAG_* bits, 0 for the op lists exactly as described at the enum */
   float softcap;            /* SOFTMAX kind: if > 0, the scaled scores become softcap * tanh(alpha*A.B / softcap) before
-                               the mask is added (Sec. 6.2, MatMul-Scale-TanhSoftcap-Softmax); must be 0 for other kinds */
+                               the mask is added (Sec. 6.1, MatMul-Scale-TanhSoftcap-Softmax); must be 0 for other kinds */
   int32_t reserved;         /* must be 0 */
 } comfuse_gemm_desc_t;
 
-/* Variants of the op lists (the three evaluation patterns of Sec. 6.2 are LAYERNORM + POST_RELU, RMSNORM_MAX +
+/* Variants of the op lists (the three evaluation patterns of Sec. 6.1 are LAYERNORM + POST_RELU, RMSNORM_MAX +
  * NO_ACTIVATION without a residual, and SOFTMAX with softcap > 0). */
 #define COMFUSE_FLAG_POST_RELU 1u      /* BIAS_RES_LAYERNORM kind only: Y = max(Y, 0) after the affine step            */
 #define COMFUSE_FLAG_NO_ACTIVATION 2u  /* BIAS_GELU_RES_RMSNORM_MAX kind only: H = alpha*A.B + bias + R, no GELU       */

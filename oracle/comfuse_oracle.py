@@ -116,7 +116,7 @@ def causal_mask(M: int, N: int, rows=None) -> np.ndarray:
 def bias_res_layernorm(A, B, bias=None, residual=None, gamma=None, beta=None, alpha=1.0, eps=1e-5, relu=False):
     """Y = LayerNorm(alpha * A.B + bias + R) * gamma + beta   (post-norm pattern; Sec. 3.2's worked example
     x = alpha * Acc + Bias with the mean / x - mean stages).  ``relu``: Y = max(Y, 0) after the affine step, the
-    MatMul-BiasAdd-LayerNorm-ReLU pattern of Sec. 6.2."""
+    MatMul-BiasAdd-LayerNorm-ReLU pattern of Sec. 6.1."""
     H = alpha * gemm(A, B)
     if bias is not None:
         H = H + np.asarray(bias, dtype=np.float64)
@@ -130,7 +130,7 @@ def bias_gelu_res_rmsnorm_max(A, B, bias=None, residual=None, g=None, alpha=1.0,
     """Z = alpha * A.B + bias; H = GELU_tanh(Z) + R; Y = RMSNorm(H) * g; then a second, chained
     reduction over Y (Sec. 3.2: multiple reduction stages): row max and argmax.
     ``activation=False`` leaves the GELU out (H = Z + R): with no residual that is the MatMul-BiasAdd-RMSNorm
-    pattern of Sec. 6.2.  Returns (Y, rowmax, argmax)."""
+    pattern of Sec. 6.1.  Returns (Y, rowmax, argmax)."""
     Z = alpha * gemm(A, B)
     if bias is not None:
         Z = Z + np.asarray(bias, dtype=np.float64)
@@ -145,7 +145,7 @@ def bias_gelu_res_rmsnorm_max(A, B, bias=None, residual=None, g=None, alpha=1.0,
 def scale_mask_softmax(A, B, alpha=1.0, mask=None, softcap=0.0):
     """P = softmax(alpha * A.B + mask) over the last dim (the attention-score normalisation pattern of
     Sec. 6.1).  ``mask`` broadcasts over leading dims.  ``softcap`` > 0: the scaled scores pass through
-    softcap * tanh(. / softcap) before the mask, the MatMul-Scale-TanhSoftcap-Softmax pattern of Sec. 6.2."""
+    softcap * tanh(. / softcap) before the mask, the MatMul-Scale-TanhSoftcap-Softmax pattern of Sec. 6.1."""
     T = alpha * gemm(A, B)
     if softcap and softcap > 0.0:
         T = softcap * np.tanh(T / softcap)
@@ -178,7 +178,7 @@ def b2b_from_intermediate(S, X, W2, b2, gamma=None, beta=None, eps=1e-5):
 
 def b2b_softmax_attention(Q, Kt, V, alpha=1.0):
     """Sec. 4, Eq. 2 with F = row softmax (the attention-form instance the paper evaluates as Target-Attention,
-    Sec. 6.3):  P = alpha * Q Kt,  S = softmax(P) over the source positions,  O = S V.
+    Sec. 6.2, Table II):  P = alpha * Q Kt,  S = softmax(P) over the source positions,  O = S V.
     Q [.., M, d], Kt [.., d, S] (the keys already transposed: a plain row-major second operand), V [.., S, d2]."""
     return gemm(softmax_rows(alpha * gemm(Q, Kt)), V)
 

@@ -250,7 +250,7 @@ def test_back_to_back_dependent_launches_see_each_others_results(cuda_device):
     assert cf.last_device_status() == cf.OK
 
 
-# --------------------------------------------------------------------------------------------- the Sec. 6.2 patterns
+# --------------------------------------------------------------------------------------------- the Sec. 6.1 patterns
 @pytest.mark.parametrize("fused", [True, False])
 @pytest.mark.parametrize("M,N,K", [(300, 768, 200), (200, 4096, 128), (300, 8192, 72)])
 def test_matmul_bias_layernorm_relu_pattern(M, N, K, fused, cuda_device):

@@ -334,7 +334,7 @@ def test_softmax_merge_any_split(splits):
         np.testing.assert_allclose(np.where(np.isneginf(x), 0.0, np.exp(x - m[:, None])) / l[:, None], P, rtol=0, atol=1e-13)
 
 
-# ----------------------------------------------------------------------------- the Sec. 6.2 pattern variants
+# ----------------------------------------------------------------------------- the Sec. 6.1 pattern variants
 def test_layernorm_relu_variant_brute_force_and_sign():
     """MatMul-BiasAdd-LayerNorm-ReLU: scalar-loop brute force; every output is >= 0 and equals the plain result where
     that is positive (so the ReLU sits after the affine step, not before the normalisation)."""
