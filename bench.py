@@ -31,10 +31,10 @@ sys.path.insert(0, ROOT)
 import workloads as wl  # noqa: E402
 
 METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
-WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4}
+WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "a1": 5}   # a1: target attention, beyond the five named configurations
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
 # captures summarised under profiles/, in bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": 70_144_768, "c3": 221_126_912, "c4": 513_010_432, "c5": 8_714_240}
+NCU_TRAFFIC_BYTES = {"a1": None, "c1": None, "c2": 70_144_768, "c3": 221_126_912, "c4": 513_010_432, "c5": 8_714_240}
 
 
 def load_peaks():
@@ -105,6 +105,8 @@ def oracle_call(w, rows):
     """One evaluation of the fp64 oracle on `rows` of workload `w` (inputs already widened to fp64)."""
     from oracle import comfuse_oracle as orc
     t = w._f64
+    if w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION:
+        return orc.b2b_softmax_attention(t["X"][0][rows], t["W1"][0], t["W2"][0], w.scalars["alpha"])
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
         return orc.b2b_mlp_layernorm(t["X"][rows], t["W1"], t["b1"], t["W2"], t["b2"], t.get("gamma"), t.get("beta"), w.scalars["eps"])
     if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
@@ -120,14 +122,14 @@ def oracle_call(w, rows):
 def widen_for_oracle(w, softmax_batches=1):
     w._f64 = {}
     for k, v in w.tensors.items():
-        if w.kind == wl.KIND_SCALE_MASK_SOFTMAX:
+        if w.kind in (wl.KIND_SCALE_MASK_SOFTMAX, wl.KIND_B2B_SOFTMAX_ATTENTION):
             v = v[:softmax_batches]
         w._f64[k] = wl.bf16_to_f64(v)
 
 
 def sample_flops(w, nrows):
     d = w.dims
-    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+    if w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION):
         return 2.0 * nrows * (d["K"] * d["N1"] + d["N1"] * d["N2"])
     return 2.0 * nrows * d["N"] * d["K"]
 
@@ -225,11 +227,13 @@ def run_comfuse(args):
 
     # ---- buffer sets: per-step activations (inputs read once per step and the outputs) are replicated until the
     # rotation exceeds 3x the L2 capacity; weights and row vectors are shared (they are meant to be L2 resident)
-    act_names = {"A", "residual", "X"} if w.kind != wl.KIND_SCALE_MASK_SOFTMAX else {"A", "B"}
+    attention = w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION
+    b2b = w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION)
+    act_names = {"A", "B"} if w.kind == wl.KIND_SCALE_MASK_SOFTMAX else ({"X", "W1", "W2"} if attention else {"A", "residual", "X"})
     base = {k: to_dev(v) for k, v in w.tensors.items()}
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
     d = w.dims
-    out_shape = (d["batch"], d["M"], d["N"]) if "batch" in d else (d["M"], d.get("N", d.get("N2")))
+    out_shape = (d["batch"], d["M"], d.get("N", d.get("N2"))) if "batch" in d else (d["M"], d.get("N", d.get("N2")))
     per_set = sum(base[k].numel() * 2 for k in base if k in act_names) + int(np.prod(out_shape)) * 2
     nsets = int(max(2, min(16, -(-3 * l2_bytes // per_set))))
     sets = []
@@ -242,8 +246,13 @@ def run_comfuse(args):
         sets.append(s)
 
     # workspace (unfused path only)
-    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
-        ws_bytes = cf.b2b_workspace_size(cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused))
+    def b2b_desc(use_fused):
+        if attention:
+            return cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, use_fused, cf.B2B_SOFTMAX_ATTENTION, d["batch"], w.scalars["alpha"])
+        return cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], use_fused)
+
+    if b2b:
+        ws_bytes = cf.b2b_workspace_size(b2b_desc(fused))
     else:
         kind = {wl.KIND_BIAS_RES_LAYERNORM: cf.EPI_BIAS_RES_LAYERNORM,
                 wl.KIND_BIAS_GELU_RES_RMSNORM_MAX: cf.EPI_BIAS_GELU_RES_RMSNORM_MAX,
@@ -254,7 +263,9 @@ def run_comfuse(args):
     ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
 
     def step(s, use_fused=fused, workspace=ws):
-        if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+        if attention:
+            cf.b2b_attention(s["X"], s["W1"], s["W2"], s["Y"], alpha=w.scalars["alpha"], fused=use_fused, workspace=workspace)
+        elif w.kind == wl.KIND_B2B_MLP_LAYERNORM:
             cf.b2b_gemm(s["X"], s["W1"], s["b1"], s["W2"], s["b2"], s["Y"], gamma=s.get("gamma"), beta=s.get("beta"),
                         eps=w.scalars["eps"], fused=use_fused, workspace=workspace)
         elif w.kind == wl.KIND_BIAS_RES_LAYERNORM:
@@ -343,7 +354,7 @@ def run_comfuse(args):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
     roof["peak_source"] = f"of {peaks['source']} (burst figure, kernel timed alone)"
-    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+    if b2b:
         roof["kernel"] = "b2b_pair_kernel"
     elif w.kind == wl.KIND_SCALE_MASK_SOFTMAX and d["K"] <= 256:
         roof["kernel"] = "softmax_rows_kernel"      # short K: score chunks computed twice, no cluster exchange
@@ -366,8 +377,8 @@ def run_comfuse(args):
         # ---- the in-library unfused path on the same buffers (context: speedup of fusion)
         try:
             other = not fused
-            if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
-                ob = cf.b2b_workspace_size(cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], other))
+            if b2b:
+                ob = cf.b2b_workspace_size(b2b_desc(other))
             else:
                 desc.fused = int(other)
                 ob = cf.workspace_size(desc)
@@ -391,7 +402,7 @@ def run_comfuse(args):
         extra["warm_l2_ms_per_step"] = timed(n3, lambda i: step(sets[0])) / n3
 
         def gemm_only(sx):
-            if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+            if b2b:
                 return torch.matmul(torch.matmul(sx["X"], sx["W1"]), sx["W2"])
             return torch.matmul(sx["A"], sx["B"])
         for i in range(3):
@@ -420,13 +431,17 @@ def run_comfuse(args):
     h2d = sum(t.numel() * 2 for t in host_in.values())
     d2h = host_out.numel() * 2
     s0 = sets[0]
-    if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
-        bdesc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused)
+    if b2b:
+        bdesc = b2b_desc(fused)
         staging = torch.empty(cf.b2b_host_staging_size(bdesc), dtype=torch.uint8, device=dev)
 
         def e2e_step(i):
-            cf.b2b_gemm_host(host_in["X"], s0["W1"], s0["b1"], s0["W2"], s0["b2"], host_out, staging=staging,
-                             gamma=s0.get("gamma"), beta=s0.get("beta"), eps=w.scalars["eps"], fused=fused, workspace=ws)
+            if attention:
+                cf.b2b_attention_host(host_in["X"], host_in["W1"], host_in["W2"], host_out, staging=staging,
+                                      alpha=w.scalars["alpha"], fused=fused, workspace=ws)
+            else:
+                cf.b2b_gemm_host(host_in["X"], s0["W1"], s0["b1"], s0["W2"], s0["b2"], host_out, staging=staging,
+                                 gamma=s0.get("gamma"), beta=s0.get("beta"), eps=w.scalars["eps"], fused=fused, workspace=ws)
     else:
         hmask = cf.HOST_A | cf.HOST_Y | (cf.HOST_B if "B" in host_in else 0) | (cf.HOST_RESIDUAL if "residual" in host_in else 0)
         hB = host_in.get("B", s0["B"])
@@ -449,7 +464,7 @@ def run_comfuse(args):
     ms_e2e = timed(n_e2e, e2e_step) / n_e2e
     e2e = {"value": whole_job_value(flops, world, ms_e2e) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e,
-           "call": "comfuse_b2b_gemm_host" if w.kind == wl.KIND_B2B_MLP_LAYERNORM else "comfuse_gemm_epilogue_host"}
+           "call": "comfuse_b2b_gemm_host" if b2b else "comfuse_gemm_epilogue_host"}
 
     # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only, on a bounded sample
     cpu = None

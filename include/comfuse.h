@@ -138,10 +138,24 @@ comfuse_status_t comfuse_gemm_epilogue_static_scratch(const comfuse_gemm_desc_t*
  *   O = LayerNorm(S.W2 + b2 + X) * gamma + beta,   S = F(X.W1),
  * X [M, K], W1 [K, N1], W2 [N1, N2], all dense row-major bf16, N2 == K.  In the fused path S (and P) never
  * leave the chip: S is rounded to bf16 as the second GEMM's tensor-core operand. */
+typedef enum {
+  COMFUSE_B2B_MLP_GELU_LAYERNORM = 0, /* as above                                                                   */
+  /* Attention form (Sec. 4, Eq. 2 with a row reduction as F; the Target-Attention workload of Sec. 6.2):
+   *   O = softmax(alpha * X.W1) . W2   per batch,  softmax over the N1 source positions,
+   * X [batch, M, K] queries, W1 [batch, K, N1] keys (already transposed), W2 [batch, N1, N2] values, O [batch, M, N2],
+   * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128, N1 = 256 (a whole score row fits the
+   * accumulators of one CTA pair); the probabilities are rounded to bf16 as the second GEMM's operand.             */
+  COMFUSE_B2B_SOFTMAX_ATTENTION = 1
+} comfuse_b2b_kind_t;
+
 typedef struct {
   int32_t M, K, N1, N2;
   float eps;
   int32_t fused;
+  int32_t kind;   /* comfuse_b2b_kind_t */
+  int32_t batch;  /* >= 1; must be 1 for the MLP kind (its weights are shared by all rows) */
+  float alpha;    /* attention kind: scale of the scores; ignored by the MLP kind */
+  int32_t reserved; /* must be 0 */
 } comfuse_b2b_desc_t;
 
 comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size_t* bytes);
@@ -166,7 +180,8 @@ comfuse_status_t comfuse_host_staging_size(const comfuse_gemm_desc_t* desc, uint
 comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t* desc, const void* A, const void* B, void* Y,
                                             const comfuse_epilogue_args_t* args, uint32_t host_mask, void* staging,
                                             size_t staging_bytes, void* workspace, size_t workspace_bytes, void* cuda_stream);
-/* The same for the back-to-back GEMM: X and O are host pointers (dense), the weights and vectors device pointers. */
+/* The same for the back-to-back GEMM: X and O are host pointers (dense), the weights and vectors device pointers; for
+ * the attention kind W1 (keys) and W2 (values) are per-step tensors too and are host pointers as well. */
 comfuse_status_t comfuse_b2b_host_staging_size(const comfuse_b2b_desc_t* desc, size_t* bytes);
 comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc, const void* X, const void* W1, const void* b1,
                                        const void* W2, const void* b2, const void* gamma, const void* beta, void* O,

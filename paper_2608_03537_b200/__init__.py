@@ -32,6 +32,7 @@ EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
 FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2
+B2B_MLP_GELU_LAYERNORM, B2B_SOFTMAX_ATTENTION = 0, 1
 
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
@@ -68,7 +69,8 @@ class EpilogueArgs(Structure):
 
 
 class B2bDesc(Structure):
-    _fields_ = [("M", c_int32), ("K", c_int32), ("N1", c_int32), ("N2", c_int32), ("eps", c_float), ("fused", c_int32)]
+    _fields_ = [("M", c_int32), ("K", c_int32), ("N1", c_int32), ("N2", c_int32), ("eps", c_float), ("fused", c_int32),
+                ("kind", c_int32), ("batch", c_int32), ("alpha", c_float), ("reserved", c_int32)]
 
 
 class ComfuseError(RuntimeError):
@@ -195,8 +197,24 @@ def gemm_epilogue_static_scratch(A, B, Y, kind, *, bias=None, residual=None, gam
     return Y
 
 
-def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True) -> B2bDesc:
-    return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)))
+def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True, kind=B2B_MLP_GELU_LAYERNORM, batch=1, alpha=1.0) -> B2bDesc:
+    return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)), int(kind), int(batch), float(alpha), 0)
+
+
+def b2b_attention(Q, Kt, V, O, *, alpha, fused=True, workspace=None, stream=None):
+    """Enqueue O = softmax(alpha * Q.Kt).V per batch (the attention form of the back-to-back GEMM).  Dense CUDA bf16
+    tensors Q [b, M, d], Kt [b, d, S] (keys already transposed), V [b, S, d2], O [b, M, d2]."""
+    nb, M, K = Q.shape
+    N1, N2 = Kt.shape[2], V.shape[2]
+    assert Kt.shape == (nb, K, N1) and V.shape == (nb, N1, N2) and O.shape == (nb, M, N2)
+    for t in (Q, Kt, V, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm(byref(d), _ptr(Q), _ptr(Kt), None, _ptr(V), None, None, None, _ptr(O), ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm")
+    return O
 
 
 def host_staging_size(desc: GemmDesc, host_mask: int) -> int:
@@ -265,6 +283,23 @@ def b2b_gemm_host(X, W1, b1, W2, b2, O, *, staging, gamma=None, beta=None, eps=1
     d = make_b2b_desc(M, K, N1, N2, eps, fused)
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
     st = lib().comfuse_b2b_gemm_host(byref(d), _ptr(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gamma), _ptr(beta), _ptr(O),
+                                     c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),
+                                     ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm_host")
+    return O
+
+
+def b2b_attention_host(Q, Kt, V, O, *, staging, alpha, fused=True, workspace=None, stream=None):
+    """b2b_attention with Q, Kt, V and O in host memory (dense CPU tensors, pinned for asynchronous copies); ``staging`` is a
+    CUDA uint8 tensor of at least b2b_host_staging_size(desc) bytes."""
+    nb, M, K = Q.shape
+    N1, N2 = Kt.shape[2], V.shape[2]
+    for t in (Q, Kt, V, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm_host(byref(d), _ptr(Q), _ptr(Kt), None, _ptr(V), None, None, None, _ptr(O),
                                      c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),
                                      ws_ptr, ws_bytes, _stream(stream))
     if st != OK:

@@ -52,6 +52,8 @@ static_assert(B2bSmem::BYTES <= 232448, "shared memory budget");
 // Ring items of one tile, in producer order (every role walks this sequence):
 //   X0 X1 | W1(0) W1(1) | { W2(j) W1(j+2) } for each chunk j | R0 R1      = 2 + 2*NC + 2 slots
 
+// MODE 0: MLP form (F = GELU(. + b1), tail = + b2 + X, LayerNorm); MODE 1: attention form (F = row softmax, no tail).
+template <int MODE>
 __global__ void __launch_bounds__(kB2bThreads, 1)
 b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                 const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
@@ -88,6 +90,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
   const int NC = p.N1 / 128;
+  const int total_tiles = p.batch * p.mpairs;
+  constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
@@ -134,22 +138,24 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       RingPos<kRingSlots> ring;
       bool ok = true;
       // one box into the current slot; kind 0: pair operand (signals the even CTA's full barrier), 1: residual
+      int bz = 0;  // batch coordinate of the current tile
       auto push = [&](const CUtensorMap* tm, int x, int y, int kind) {
         if (!ok) return;
         if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; return; }
         if (kind == 0) {
           const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
           mbar_arrive_expect_tx_cluster(full, kSlotBytes);
-          tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, 0);
+          tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, bz);
         } else {
           mbar_arrive_expect_tx(bar_rfull(ring.stage), kSlotBytes);
-          tma_load_3d(ring_addr(ring.stage), tm, bar_rfull(ring.stage), x, y, 0);
+          tma_load_3d(ring_addr(ring.stage), tm, bar_rfull(ring.stage), x, y, bz);
         }
         ring.advance();
       };
       const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
-      for (int tile = cluster_id; tile < p.mpairs && ok; tile += num_clusters) {
-        const int m0 = tile * 256 + static_cast<int>(pm) * 128;
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
+        bz = tile / p.mpairs;
+        const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
         push(&tmX, 0, m0, 0);
         push(&tmX, 64, m0, 0);
         push(&tmW1, 0 * 128 + wcol, 0, 0);
@@ -158,8 +164,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           push(&tmW2, wcol, j * 128, 0);
           if (j + 2 < NC) push(&tmW1, (j + 2) * 128 + wcol, 0, 0);
         }
-        push(&tmX, 0, m0, 1);
-        push(&tmX, 64, m0, 1);
+        if (has_tail_residual) {
+          push(&tmX, 0, m0, 1);
+          push(&tmX, 64, m0, 1);
+        }
       }
     }
   } else if (warp == 1) {
@@ -183,7 +191,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         umma_commit_pair(bar_empty(stage));
         umma_commit_pair(map_to_cta(bar_empty(stage), peer));
       };
-      for (int tile = cluster_id; tile < p.mpairs && ok; tile += num_clusters, ++tile_it) {
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
         const int obuf = tile_it & 1u;
         const uint32_t d_o = tmem_base + 256 + obuf * 128;
         // X: two K blocks
@@ -249,7 +257,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           umma_commit_pair(bar_ofull(obuf));
           umma_commit_pair(map_to_cta(bar_ofull(obuf), peer));
         }
-        ring.skip(2);  // the residual slots belong to the epilogue
+        if (has_tail_residual) ring.skip(2);  // the residual slots belong to the epilogue
       }
       umma_commit_pair(bar_drain);
       mbar_wait<false>(bar_drain, 0, w);
@@ -291,12 +299,77 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #define B2B_TRACE_POINT() do { } while (0)
 #endif
 
-    for (int tile = cluster_id; tile < p.mpairs; tile += num_clusters, ++tile_it) {
+    for (int tile = cluster_id; tile < total_tiles; tile += num_clusters, ++tile_it) {
       B2B_TRACE_POINT();
-      const int m0 = tile * 256 + static_cast<int>(pm) * 128;
+      const int bz = tile / p.mpairs;
+      const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
       const int obuf = tile_it & 1u;
+      float inv_l = 0.f;  // attention form: 1 / (row sum of the exponentials)
+      if constexpr (MODE == 1) {
+        // ---------------- Epi1, attention form (N1 = 256: both P chunks hold one whole score row): row max and sum of
+        // exponentials across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next
+        // UMMAs' A operand; the division by the sum waits for Epi2 (O = (S.V) / sum)
+        for (int pb = 0; pb < 2; ++pb) {
+          mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
+          ++puses[pb];
+          mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
+          ++suses[pb];
+        }
+        __syncwarp();
+        tcgen05_fence_after_sync();
+        const float sc = p.alpha * 1.4426950408889634f;  // log2 domain
+        uint32_t v0[32], v1[32];
+        tmem_ld_32cols(tmem_base + lane_sel + 0 * 128 + hh * 32, v0);
+        tmem_ld_32cols(tmem_base + lane_sel + 1 * 128 + hh * 32, v1);
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          mx0 = max3(mx0, __uint_as_float(v0[i]), __uint_as_float(v0[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(v1[i]), __uint_as_float(v1[i + 1]));
+        }
+        // sc > 0 is required (checked by the host): the maximum of the scaled scores is the scaled maximum
+        const float mloc = fmaxf(mx0, mx1) * sc;
+        float2 a0 = splat2(0.f), a1 = splat2(0.f);
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float2 d0 = fma2(f2_from_bits(v0[i], v0[i + 1]), splat2(sc), splat2(-mloc));
+          const float2 d1 = fma2(f2_from_bits(v1[i], v1[i + 1]), splat2(sc), splat2(-mloc));
+          const float2 e0 = make_float2(ex2_approx(d0.x), ex2_approx(d0.y)), e1 = make_float2(ex2_approx(d1.x), ex2_approx(d1.y));
+          v0[i] = __float_as_uint(e0.x); v0[i + 1] = __float_as_uint(e0.y);
+          v1[i] = __float_as_uint(e1.x); v1[i + 1] = __float_as_uint(e1.y);
+          a0 = add2(a0, e0);
+          a1 = add2(a1, e1);
+        }
+        const float lloc = (a0.x + a0.y) + (a1.x + a1.y);
+        const float2 tot = cluster_row_reduce<1, MergeMaxSumExp2, 4>(make_float2(mloc, lloc), 64.f, MergeMaxSumExp2(), s_pre, s_stats,
+                                                                     bar_stats, row, hh, 0u, xpar, xphase, w);
+        const float f = ex2_approx(mloc - tot.x);  // this thread's exponentials are relative to its own maximum
+        inv_l = tot.y > 0.f ? 1.f / tot.y : 0.f;
+#pragma unroll
+        for (int pb = 0; pb < 2; ++pb) {
+          const uint32_t(&vv)[32] = pb ? v1 : v0;
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(vv[2 * i], vv[2 * i + 1]), splat2(f)));
+          const uint32_t sb = s_addr(pb, kblk);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t a = sb + swz128(row, chunk0 + i);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                         "r"(pk[4 * i + 3])
+                         : "memory");
+          }
+        }
+        tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
+        fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster_noflush(sfull_leader);
+          mbar_arrive_cluster_noflush(sfull_leader + 8u);
+        }
+      }
       // ---------------- Epi1(j): S_j = bf16(GELU(P_j + b1)) as the next UMMA's A operand
-      for (int j = 0; j < NC; ++j) {
+      for (int j = 0; j < (MODE == 0 ? NC : 0); ++j) {
         const int pb = j & 1;
         mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
         ++puses[pb];
@@ -354,6 +427,15 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       __syncwarp();
       tcgen05_fence_after_sync();
       B2B_TRACE_POINT();
+      const uint32_t o_addr = tmem_base + lane_sel + 256 + obuf * 128 + hh * 32;
+      uint32_t pk[16];
+      if constexpr (MODE == 1) {
+        // attention form: O = (S.V) / (row sum), rounded once
+        uint32_t v[32];
+        tmem_ld_32cols(o_addr, v);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * i], v[2 * i + 1]), splat2(inv_l)));
+      } else {
       const int s0 = ring.stage;
       const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
       // both residual slots are waited for by everybody (the phase bits must advance uniformly)
@@ -379,7 +461,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
       ring.skip(2);
       // stage 1: x = O + b2 + X ; thread-local (mean, M2) over this thread's 32 columns; x goes back into TMEM
-      const uint32_t o_addr = tmem_base + lane_sel + 256 + obuf * 128 + hh * 32;
       float2 part;
       {
         uint32_t v[32];
@@ -417,7 +498,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const float mu = tot.x;
       const float rstd = rsqrtf(tot.y * (1.f / 128.f) + p.eps);
       // stage 2: normalise the resident x, round once
-      uint32_t pk[16];
       {
         uint32_t v[32];
         tmem_ld_32cols(o_addr, v);
@@ -432,6 +512,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           pk[2 * i + 1] = pack_bf16x2_rn(fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w)));
         }
       }
+      }  // MLP form
       // the accumulator has been read for the last time: the O slot can be reused by the tile after the next one
       tcgen05_fence_before_sync();
       __syncwarp();
@@ -452,7 +533,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         fence_proxy_async_smem();
         named_barrier_sync(3, kB2bEpiThreads);
         if (store_thread) {
-          tma_store_3d(&tmO, ybuf, g * 64, m0, 0);
+          tma_store_3d(&tmO, ybuf, g * 64, m0, bz);
           tma_store_commit();
         }
       }
@@ -472,7 +553,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
 }  // namespace
 
-bool b2b_fused_supported(int K, int N1, int N2) {
+bool b2b_fused_supported(int K, int N1, int N2, int mode) {
+  if (mode == 1) return K == 128 && N2 == 128 && N1 == 256;  // attention form: one whole score row in the two P slots
   return K == 128 && N2 == 128 && N1 >= 128 && N1 <= 128 * kMaxChunks && N1 % 128 == 0;
 }
 
@@ -481,11 +563,13 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   if (!dev) return cudaErrorInvalidDevice;
   CUtensorMap tmX, tmW1, tmW2, tmO;
   const uint64_t M = p.M, K = p.K, N1 = p.N1, N2 = p.N2;
+  if (p.batch < 1) p.batch = 1;
+  const uint64_t nb = static_cast<uint64_t>(p.batch);  // dense [batch, rows, cols] tensors (the MLP form has batch = 1)
   // all boxes are 64 elements x 128 rows
-  if (!encode_tmap_bf16_3d(&tmX, X, K, M, 1, K * 2, M * K * 2, 128) ||
-      !encode_tmap_bf16_3d(&tmW1, W1, N1, K, 1, N1 * 2, K * N1 * 2, 128) ||
-      !encode_tmap_bf16_3d(&tmW2, W2, N2, N1, 1, N2 * 2, N1 * N2 * 2, 128) ||
-      !encode_tmap_bf16_3d(&tmO, p.O, N2, M, 1, N2 * 2, M * N2 * 2, 128))
+  if (!encode_tmap_bf16_3d(&tmX, X, K, M, nb, K * 2, M * K * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmW1, W1, N1, K, nb, N1 * 2, K * N1 * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmW2, W2, N2, N1, nb, N2 * 2, N1 * N2 * 2, 128) ||
+      !encode_tmap_bf16_3d(&tmO, p.O, N2, M, nb, N2 * 2, M * N2 * 2, 128))
     return cudaErrorInvalidValue;
   p.mblocks = (p.M + 127) / 128;
   p.mpairs = (p.mblocks + 1) / 2;
@@ -507,19 +591,23 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   if (max_clusters[di] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(b2b_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
-    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<0>, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di] = n;
   }
-  const int clusters = p.mpairs < max_clusters[di] ? p.mpairs : max_clusters[di];
+  const int tiles = p.batch * p.mpairs;
+  const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
-  return cudaLaunchKernelEx(&cfg, b2b_pair_kernel, tmX, tmW1, tmW2, tmO, p);
+  return p.mode == 1 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1>, tmX, tmW1, tmW2, tmO, p)
+                     : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<0>, tmX, tmW1, tmW2, tmO, p);
 }
 
 }  // namespace comfuse

@@ -8,7 +8,10 @@ namespace comfuse {
 
 struct B2bParams {
   int M, K, N1, N2;
-  int mblocks, mpairs;  // 128-row blocks and pairs of them
+  int mblocks, mpairs;  // 128-row blocks and pairs of them (per batch)
+  int batch;            // attention form: X, W1, W2, O are [batch, ., .]; MLP form: 1
+  int mode;             // 0: F = GELU(. + b1), tail = + b2 + X, LayerNorm; 1: F = softmax(alpha * .), tail = none
+  float alpha;          // attention form: scale of the scores
   float eps;
   const uint16_t* X;  // also the residual of the tail
   const uint16_t* b1;
@@ -22,7 +25,7 @@ struct B2bParams {
   int trace_flags;            // tracing builds: experiment switches
 };
 
-bool b2b_fused_supported(int K, int N1, int N2);
+bool b2b_fused_supported(int K, int N1, int N2, int mode);
 cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
 
 }  // namespace comfuse

@@ -348,10 +348,17 @@ static comfuse_status_t validate_b2b_desc(const comfuse_b2b_desc_t* d) {
   if (!d) return COMFUSE_ERR_INVALID_ARG;
   if (d->M < 1 || d->K < 1 || d->N1 < 1 || d->N2 < 1) return COMFUSE_ERR_INVALID_ARG;
   if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
-  if (d->N2 != d->K) return COMFUSE_ERR_INVALID_ARG;  // the residual is X itself
+  if (d->kind != COMFUSE_B2B_MLP_GELU_LAYERNORM && d->kind != COMFUSE_B2B_SOFTMAX_ATTENTION) return COMFUSE_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->kind == COMFUSE_B2B_MLP_GELU_LAYERNORM) {
+    if (d->batch != 1) return COMFUSE_ERR_INVALID_ARG;
+    if (d->N2 != d->K) return COMFUSE_ERR_INVALID_ARG;  // the residual is X itself
+  } else if (!(d->alpha > 0.f)) {
+    return COMFUSE_ERR_INVALID_ARG;
+  }
   if (!mult8(d->K) || !mult8(d->N1) || !mult8(d->N2)) return COMFUSE_ERR_ALIGNMENT;
-  if (d->fused && !b2b_fused_supported(d->K, d->N1, d->N2)) return COMFUSE_ERR_UNSUPPORTED;
-  if (!d->fused && d->N2 > 8192) return COMFUSE_ERR_UNSUPPORTED;
+  if (d->fused && !b2b_fused_supported(d->K, d->N1, d->N2, d->kind)) return COMFUSE_ERR_UNSUPPORTED;
+  if (!d->fused && (d->kind == COMFUSE_B2B_MLP_GELU_LAYERNORM ? d->N2 : d->N1) > 8192) return COMFUSE_ERR_UNSUPPORTED;
   return COMFUSE_OK;
 }
 
@@ -359,7 +366,10 @@ comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size
   if (!bytes) return COMFUSE_ERR_INVALID_ARG;
   comfuse_status_t s = validate_b2b_desc(desc);
   if (s != COMFUSE_OK) return s;
-  *bytes = desc->fused ? 0 : (static_cast<size_t>(desc->M) * desc->N1 + static_cast<size_t>(desc->M) * desc->N2) * 2;
+  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1]
+    *bytes = desc->fused ? 0 : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2;
+  else
+    *bytes = desc->fused ? 0 : (static_cast<size_t>(desc->M) * desc->N1 + static_cast<size_t>(desc->M) * desc->N2) * 2;
   return COMFUSE_OK;
 }
 
@@ -369,6 +379,8 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
   comfuse_status_t s = validate_b2b_desc(desc);
   if (s != COMFUSE_OK) return s;
   if (!X || !W1 || !W2 || !O) return COMFUSE_ERR_INVALID_ARG;
+  const bool attention = desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION;
+  if (attention && (b1 || b2 || gamma || beta)) return COMFUSE_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W1) || !aligned16(W2) || !aligned16(O) || !aligned16(b1) || !aligned16(b2) ||
       !aligned16(gamma) || !aligned16(beta))
     return COMFUSE_ERR_ALIGNMENT;
@@ -386,6 +398,7 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
   if (desc->fused) {
     B2bParams bp = {};
     bp.M = M; bp.K = K; bp.N1 = N1; bp.N2 = N2;
+    bp.batch = desc->batch; bp.mode = attention ? 1 : 0; bp.alpha = desc->alpha;
     bp.eps = desc->eps;
     bp.X = static_cast<const uint16_t*>(X);
     bp.b1 = static_cast<const uint16_t*>(b1);
@@ -401,6 +414,32 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
 #endif
     cudaError_t e = launch_b2b_fused(X, W1, W2, bp, st);
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+  }
+
+  if (attention) {
+    // unfused: P = X.W1 (bf16, workspace) -> row softmax of alpha * P in place -> O = P.W2, batched
+    uint16_t* P = static_cast<uint16_t*>(workspace);
+    const int nb = desc->batch;
+    GemmMaps maps;
+    FusedParams p = {};
+    p.batch = nb; p.mblocks = (M + 127) / 128; p.alpha = 1.f;
+    p.status = dev->status_word; p.timeout_ns = timeout_ns();
+    if (!make_gemm_maps(&maps, X, W1, nullptr, P, nb, M, N1, K, K, N1, 0, N1, static_cast<long long>(M) * K,
+                        static_cast<long long>(K) * N1, 0, static_cast<long long>(M) * N1))
+      return COMFUSE_ERR_CUDA;
+    p.M = M; p.N = N1; p.K = K; p.Y = P; p.ldy = N1; p.batch_stride_y = static_cast<long long>(M) * N1;
+    if (launch_plain_gemm(maps, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    RowParams r = {};
+    r.batch = 1; r.M = nb * M; r.N = N1;  // the rows of all batches, dense
+    r.Z = P; r.ldz = N1;
+    r.alpha = desc->alpha;
+    r.Y = P; r.ldy = N1;
+    if (launch_row_epilogue(EPI_SOFTMAX, r, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    if (!make_gemm_maps(&maps, P, W2, nullptr, O, nb, M, N2, N1, N1, N2, 0, N2, static_cast<long long>(M) * N1,
+                        static_cast<long long>(N1) * N2, 0, static_cast<long long>(M) * N2))
+      return COMFUSE_ERR_CUDA;
+    p.N = N2; p.K = N1; p.Y = static_cast<uint16_t*>(O); p.ldy = N2; p.batch_stride_y = static_cast<long long>(M) * N2;
+    return launch_plain_gemm(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }
 
   // unfused: P = X.W1 -> S = GELU(P + b1) in place -> O' = S.W2 -> LayerNorm(O' + b2 + X)

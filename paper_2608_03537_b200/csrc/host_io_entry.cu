@@ -84,7 +84,10 @@ extern "C" comfuse_status_t comfuse_b2b_host_staging_size(const comfuse_b2b_desc
   size_t ws = 0;
   const comfuse_status_t s = comfuse_b2b_workspace_size(desc, &ws);  // validates the description
   if (s != COMFUSE_OK) return s;
-  *bytes = round_up(static_cast<size_t>(desc->M) * desc->K * 2) + round_up(static_cast<size_t>(desc->M) * desc->N2 * 2);
+  const size_t nb = static_cast<size_t>(desc->batch);
+  *bytes = round_up(nb * desc->M * desc->K * 2) + round_up(nb * desc->M * desc->N2 * 2);
+  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // keys and values are per-step tensors too
+    *bytes += round_up(nb * desc->K * desc->N1 * 2) + round_up(nb * desc->N1 * desc->N2 * 2);
   return COMFUSE_OK;
 }
 
@@ -99,10 +102,21 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
   if (!staging || staging_bytes < need) return COMFUSE_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(staging) & 15u) return COMFUSE_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t xb = static_cast<size_t>(desc->M) * desc->K * 2, ob = static_cast<size_t>(desc->M) * desc->N2 * 2;
+  const size_t nb = static_cast<size_t>(desc->batch);
+  const size_t xb = nb * desc->M * desc->K * 2, ob = nb * desc->M * desc->N2 * 2;
   unsigned char* dX = static_cast<unsigned char*>(staging);
   unsigned char* dO = dX + round_up(xb);
   if (cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION) {  // W1 (keys) and W2 (values) are host pointers as well
+    if (!W1 || !W2) return COMFUSE_ERR_INVALID_ARG;
+    const size_t w1b = nb * desc->K * desc->N1 * 2, w2b = nb * desc->N1 * desc->N2 * 2;
+    unsigned char* dW1 = dO + round_up(ob);
+    unsigned char* dW2 = dW1 + round_up(w1b);
+    if (cudaMemcpyAsync(dW1, W1, w1b, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    if (cudaMemcpyAsync(dW2, W2, w2b, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    W1 = dW1;
+    W2 = dW2;
+  }
   s = comfuse_b2b_gemm(desc, dX, W1, b1, W2, b2, gamma, beta, dO, workspace, workspace_bytes, cuda_stream);
   if (s != COMFUSE_OK) return s;
   if (cudaMemcpyAsync(O, dO, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess) return COMFUSE_ERR_CUDA;

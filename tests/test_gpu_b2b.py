@@ -66,3 +66,36 @@ def test_b2b_unsupported_shapes_are_refused_for_the_fused_path(cuda_device):
         cf.b2b_workspace_size(d)
     assert e.value.status == cf.ERR_UNSUPPORTED
     assert cf.b2b_workspace_size(cf.make_b2b_desc(256, 128, 640, 128, fused=False)) == 256 * 640 * 2 + 256 * 128 * 2
+
+
+# --------------------------------------------------------------------------------------------- attention form (F = softmax)
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M", [(2, 256), (3, 600), (37, 128), (1, 1)])
+def test_b2b_softmax_attention(batch, M, fused, cuda_device):
+    """O = softmax(Q.Kt / sqrt(d)).V with 256 source positions and head size 128: several tiles, ragged M, more tiles than
+    one round of CTA pairs, the one-row edge."""
+    w = wl.target_attention(batch, M, 256, 128, seed=batch + M)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"attention b{batch} M{M} fused={fused}")
+
+
+def test_b2b_softmax_attention_sharp_and_flat_rows(cuda_device):
+    """Large scores (one key dominates: the output is that value row; no overflow) and zero queries (uniform weights: the
+    output is the mean of the value rows)."""
+    w = wl.target_attention(2, 256, 256, 128, seed=9)
+    w.scalars["alpha"] = 4.0                       # scores of standard deviation ~45
+    w.tensors["X"][1, 128:] = 0                    # zero queries in the second half of batch 1 (bf16 bits 0 = 0.0)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    ref = P.run_oracle(w)
+    P.check_outputs(w, got, ref, label="attention sharp/flat")
+    V1 = wl.bf16_to_f64(w.tensors["W2"][1])
+    assert np.abs(P.to_f64(got["Y"][1, 128:]) - V1.mean(0)).max() < 2e-3
+
+
+def test_b2b_attention_full_size_sampled(cuda_device):
+    w = wl.config(5)                               # 32 x (4096 x 128 -> 256 -> 128)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    assert torch.isfinite(got["Y"].float()).all().item()
+    rows = wl.sample_rows(w.dims["M"], 64)
+    batches = [0, 13, 31]
+    P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches, label="a1 target attention")
