@@ -131,6 +131,22 @@ def test_b2b_validation():
         assert L.comfuse_b2b_workspace_size(ctypes.byref(bad), ctypes.byref(n)) == code
     assert L.comfuse_b2b_gemm(ctypes.byref(ok), None, FAKE, FAKE, FAKE, FAKE, None, None, FAKE, None, 0, None) == cf.ERR_INVALID_ARG
     assert L.comfuse_b2b_gemm(ctypes.byref(ok), ODD, FAKE, FAKE, FAKE, FAKE, None, None, FAKE, None, 0, None) == cf.ERR_ALIGNMENT
+    # attention form
+    A = cf.B2B_SOFTMAX_ATTENTION
+    att = cf.make_b2b_desc(4096, 128, 256, 128, 0.0, True, A, 32, 0.088)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK and n.value == 0
+    attu = cf.make_b2b_desc(4096, 128, 256, 128, 0.0, False, A, 32, 0.088)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(attu), ctypes.byref(n)) == cf.OK and n.value == 32 * 4096 * 256 * 2
+    for bad, code in [(cf.make_b2b_desc(4096, 128, 512, 128, 0.0, True, A, 2, 0.1), cf.ERR_UNSUPPORTED),   # fused: N1 = 256 only
+                      (cf.make_b2b_desc(4096, 128, 512, 128, 0.0, False, A, 2, 0.1), cf.OK),               # unfused takes it
+                      (cf.make_b2b_desc(4096, 64, 256, 64, 0.0, False, A, 2, 0.1), cf.OK),                  # N2 != K is fine here
+                      (cf.make_b2b_desc(4096, 128, 256, 128, 0.0, True, A, 2, 0.0), cf.ERR_INVALID_ARG),   # alpha must be > 0
+                      (cf.make_b2b_desc(4096, 128, 256, 128, 0.0, True, A, 0, 0.1), cf.ERR_INVALID_ARG),   # batch >= 1
+                      (cf.make_b2b_desc(4096, 128, 256, 128, 0.0, True, 7, 1, 0.1), cf.ERR_INVALID_ARG),   # unknown kind
+                      (cf.make_b2b_desc(1024, 128, 512, 128, 1e-5, True, cf.B2B_MLP_GELU_LAYERNORM, 2, 1.0), cf.ERR_INVALID_ARG)]:
+        assert L.comfuse_b2b_workspace_size(ctypes.byref(bad), ctypes.byref(n)) == code
+    # the attention form has no bias / affine vectors
+    assert L.comfuse_b2b_gemm(ctypes.byref(att), FAKE, FAKE, FAKE, FAKE, None, None, None, FAKE, None, 0, None) == cf.ERR_INVALID_ARG
 
 
 def test_valid_call_without_a_usable_gpu_fails_cleanly():
