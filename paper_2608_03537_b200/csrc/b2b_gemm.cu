@@ -42,8 +42,8 @@ struct B2bSmem {
   static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][4][128]
   static constexpr int OFF_STATS = OFF_PRE + 2 * 4 * 128 * 8;      // float2 [2][1][128]
   static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
-  // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats drain
-  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 3;
+  // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats[2] drain pfree
+  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 4;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
@@ -79,6 +79,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   auto bar_oempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 8 + a); };  // O slot drained by both CTAs (even CTA)
   const uint32_t bar_stats = bar_base + 8u * (3 * kRingSlots + 10);
   const uint32_t bar_drain = bar_stats + 16u;
+  const uint32_t bar_pfree = bar_drain + 8u;  // attention form: both P slots read by every epilogue warp (even CTA)
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + B2bSmem::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + B2bSmem::OFF_MISC + 4);
 
@@ -111,6 +112,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     mbar_init(bar_stats, 4);
     mbar_init(bar_stats + 8u, 4);
     mbar_init(bar_drain, 1);
+    mbar_init(bar_pfree, 2 * kB2bEpiWarps);
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tensormap(&tmX);
@@ -153,7 +155,25 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ring.advance();
       };
       const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
+      if constexpr (MODE == 1) {
+        // attention form, software-pipelined over tiles (see the UMMA lane): Q and K of tile t+1 go in before V of tile t
+        auto push_qk = [&](int tile) {
+          bz = tile / p.mpairs;
+          const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
+          push(&tmX, 0, m0, 0);
+          push(&tmX, 64, m0, 0);
+          push(&tmW1, 0 * 128 + wcol, 0, 0);
+          push(&tmW1, 1 * 128 + wcol, 0, 0);
+        };
+        if (cluster_id < total_tiles) push_qk(cluster_id);
+        for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
+          if (tile + num_clusters < total_tiles) push_qk(tile + num_clusters);
+          bz = tile / p.mpairs;
+          push(&tmW2, wcol, 0 * 128, 0);
+          push(&tmW2, wcol, 1 * 128, 0);
+        }
+      }
+      for (int tile = cluster_id; MODE == 0 && tile < total_tiles && ok; tile += num_clusters) {
         bz = tile / p.mpairs;
         const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
         push(&tmX, 0, m0, 0);
@@ -191,7 +211,75 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         umma_commit_pair(bar_empty(stage));
         umma_commit_pair(map_to_cta(bar_empty(stage), peer));
       };
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
+      if constexpr (MODE == 1) {
+        // Attention form, software-pipelined over the cluster's tiles: the scores of tile t+1 (ML1) are issued as soon
+        // as the epilogue has read the scores of tile t out of the P slots, BEFORE S.V of tile t (ML2), so that the
+        // epilogue can go from the softmax of tile t straight to the softmax of tile t+1 while ML2(t) runs, and finds
+        // O(t) complete when it comes back for the normalisation.
+        auto ml1 = [&]() {  // P[0], P[1] = Q . Kt chunks 0, 1 of the next tile in the ring
+          const int xs0 = ring.stage;
+          const uint32_t x0 = wait_slot();
+          ring.advance();
+          const int xs1 = ring.stage;
+          const uint32_t x1 = wait_slot();
+          ring.advance();
+          const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
+          const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
+          for (int j = 0; j < 2 && ok; ++j) {
+            const int wstage = ring.stage;
+            const uint32_t wa = wait_slot();
+            ring.advance();
+            if (!ok) return;
+            const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
+                                wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
+            release_slot(wstage);
+            umma_commit_pair(bar_pfull(j));
+            umma_commit_pair(map_to_cta(bar_pfull(j), peer));
+          }
+          release_slot(xs0);
+          release_slot(xs1);
+        };
+        if (cluster_id < total_tiles) ml1();
+        for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
+          const int obuf = tile_it & 1u;
+          const uint32_t d_o = tmem_base + 256 + obuf * 128;
+          if (tile + num_clusters < total_tiles) {
+            if (!mbar_wait<false>(bar_pfree, tile_it & 1u, w)) { ok = false; break; }  // the epilogue holds tile t's scores in registers
+            tcgen05_fence_after_sync();
+            ml1();
+            if (!ok) break;
+          }
+          if (!mbar_wait<false>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          for (int j = 0; j < 2 && ok; ++j) {  // O = S . V, two K halves of 128 source positions
+            const int wstage = ring.stage;
+            const uint32_t wa = wait_slot();
+            ring.advance();
+            if (!ok) break;
+            if (!mbar_wait<false>(bar_sfull(j), sfull_uses[j] & 1u, w)) { ok = false; break; }
+            ++sfull_uses[j];
+            tcgen05_fence_after_sync();
+            const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+            const uint64_t sdesc0 = make_smem_desc_sw128(s_addr(j, 0), 16, 1024);
+            const uint64_t sdesc1 = make_smem_desc_sw128(s_addr(j, 1), 16, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              umma_bf16_ss_pair(d_o, (kk < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((kk & 3) * 2), wdesc + static_cast<uint64_t>(kk * 128),
+                                idesc_ml2, (j | kk) != 0 ? 1u : 0u);
+            release_slot(wstage);
+            umma_commit_pair(bar_sempty(j));
+            umma_commit_pair(map_to_cta(bar_sempty(j), peer));
+          }
+          if (ok) {
+            umma_commit_pair(bar_ofull(obuf));
+            umma_commit_pair(map_to_cta(bar_ofull(obuf), peer));
+          }
+        }
+      }
+      for (int tile = cluster_id; MODE == 0 && tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
         const int obuf = tile_it & 1u;
         const uint32_t d_o = tmem_base + 256 + obuf * 128;
         // X: two K blocks
@@ -299,21 +387,18 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #define B2B_TRACE_POINT() do { } while (0)
 #endif
 
-    for (int tile = cluster_id; tile < total_tiles; tile += num_clusters, ++tile_it) {
-      B2B_TRACE_POINT();
-      const int bz = tile / p.mpairs;
-      const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
-      const int obuf = tile_it & 1u;
-      float inv_l = 0.f;  // attention form: 1 / (row sum of the exponentials)
-      if constexpr (MODE == 1) {
-        // ---------------- Epi1, attention form (N1 = 256: both P chunks hold one whole score row): row max and sum of
-        // exponentials across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next
-        // UMMAs' A operand; the division by the sum waits for Epi2 (O = (S.V) / sum)
+    if constexpr (MODE == 1) {
+      // ================= attention form, software-pipelined over the cluster's tiles:
+      //   softmax(t0) | softmax(t1) finish(t0) | softmax(t2) finish(t1) | ... | finish(last)
+      // so that S.V of tile t (ML2) runs under the softmax of tile t+1 and the UMMA lane never waits for this epilogue
+      // longer than one softmax.
+      // ---------------- Epi1 (N1 = 256: the two P slots hold one whole score row): row max and sum of exponentials
+      // across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next UMMAs' A operand;
+      // returns 1 / (row sum), applied in the tile's finish step (O = (S.V) / sum)
+      auto softmax_tile = [&]() -> float {
         for (int pb = 0; pb < 2; ++pb) {
           mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
           ++puses[pb];
-          mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
-          ++suses[pb];
         }
         __syncwarp();
         tcgen05_fence_after_sync();
@@ -321,6 +406,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         uint32_t v0[32], v1[32];
         tmem_ld_32cols(tmem_base + lane_sel + 0 * 128 + hh * 32, v0);
         tmem_ld_32cols(tmem_base + lane_sel + 1 * 128 + hh * 32, v1);
+        // the scores are in registers: the P slots may take the next tile's scores
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster_noflush(map_to_cta(bar_pfree, leader));
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
@@ -344,7 +433,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const float2 tot = cluster_row_reduce<1, MergeMaxSumExp2, 4>(make_float2(mloc, lloc), 64.f, MergeMaxSumExp2(), s_pre, s_stats,
                                                                      bar_stats, row, hh, 0u, xpar, xphase, w);
         const float f = ex2_approx(mloc - tot.x);  // this thread's exponentials are relative to its own maximum
-        inv_l = tot.y > 0.f ? 1.f / tot.y : 0.f;
+        // the S buffers are free once ML2 of the previous tile has read them
+        for (int pb = 0; pb < 2; ++pb) {
+          mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
+          ++suses[pb];
+        }
+        __syncwarp();
 #pragma unroll
         for (int pb = 0; pb < 2; ++pb) {
           const uint32_t(&vv)[32] = pb ? v1 : v0;
@@ -360,16 +454,67 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
                          : "memory");
           }
         }
-        tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
-        fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
+        fence_proxy_async_smem();  // S writes are visible to the tensor core's shared-memory reads
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_cluster_noflush(sfull_leader);
           mbar_arrive_cluster_noflush(sfull_leader + 8u);
         }
+        return tot.y > 0.f ? 1.f / tot.y : 0.f;
+      };
+      // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes through one staging buffer
+      auto finish_tile = [&](int tile, uint32_t it, float inv_l) {
+        const int bz = tile / p.mpairs;
+        const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
+        const int obuf = it & 1u;
+        mbar_wait<false>(bar_ofull(obuf), (it >> 1) & 1u, w);
+        __syncwarp();
+        tcgen05_fence_after_sync();
+        uint32_t pk[16];
+        {
+          uint32_t v[32];
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + hh * 32, v);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * i], v[2 * i + 1]), splat2(inv_l)));
+        }
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
+        for (int g = 0; g < 2; ++g) {
+          if (store_thread) tma_store_wait_read<0>();
+          named_barrier_sync(3, kB2bEpiThreads);
+          if (kblk == g) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t a = ybuf + swz128(row, chunk0 + i);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                           "r"(pk[4 * i + 3])
+                           : "memory");
+            }
+          }
+          fence_proxy_async_smem();
+          named_barrier_sync(3, kB2bEpiThreads);
+          if (store_thread) {
+            tma_store_3d(&tmO, ybuf, g * 64, m0, bz);
+            tma_store_commit();
+          }
+        }
+      };
+      float inv_next = 0.f;
+      if (cluster_id < total_tiles) inv_next = softmax_tile();
+      for (int tile = cluster_id; tile < total_tiles; tile += num_clusters, ++tile_it) {
+        const float inv_cur = inv_next;
+        if (tile + num_clusters < total_tiles) inv_next = softmax_tile();
+        finish_tile(tile, tile_it, inv_cur);
       }
+    }
+    for (int tile = cluster_id; MODE == 0 && tile < total_tiles; tile += num_clusters, ++tile_it) {
+      B2B_TRACE_POINT();
+      const int bz = tile / p.mpairs;
+      const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
+      const int obuf = tile_it & 1u;
       // ---------------- Epi1(j): S_j = bf16(GELU(P_j + b1)) as the next UMMA's A operand
-      for (int j = 0; j < (MODE == 0 ? NC : 0); ++j) {
+      for (int j = 0; j < NC; ++j) {
         const int pb = j & 1;
         mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
         ++puses[pb];
@@ -429,13 +574,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       B2B_TRACE_POINT();
       const uint32_t o_addr = tmem_base + lane_sel + 256 + obuf * 128 + hh * 32;
       uint32_t pk[16];
-      if constexpr (MODE == 1) {
-        // attention form: O = (S.V) / (row sum), rounded once
-        uint32_t v[32];
-        tmem_ld_32cols(o_addr, v);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * i], v[2 * i + 1]), splat2(inv_l)));
-      } else {
+      {
       const int s0 = ring.stage;
       const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
       // both residual slots are waited for by everybody (the phase bits must advance uniformly)
