@@ -95,6 +95,9 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[62] = globaltimer_ns();  // kernel entry
+#endif
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kRingSlots; ++s) {
@@ -381,7 +384,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     int trace_ix = 0;
 #define B2B_TRACE_POINT()                                                                                \
   do {                                                                                                   \
-    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 64) p.trace[trace_ix++] = globaltimer_ns(); \
+    if (p.trace && blockIdx.x == 0 && warp == 2 && lane == 0 && trace_ix < 60) p.trace[trace_ix++] = globaltimer_ns(); \
   } while (0)
 #else
 #define B2B_TRACE_POINT() do { } while (0)
@@ -680,6 +683,9 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     if (store_thread) tma_store_wait_read<0>();  // the staging buffer must outlive the last store's read
   }
 
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[61] = globaltimer_ns();  // epilogue warps done
+#endif
   tcgen05_fence_before_sync();
   __syncthreads();
   cluster_sync_all();
@@ -688,6 +694,9 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     tcgen05_fence_after_sync();
     tmem_dealloc_pair(tmem_base, 512);
   }
+#ifdef COMFUSE_TRACE
+  if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[63] = globaltimer_ns();  // kernel exit
+#endif
 }
 
 }  // namespace
