@@ -32,12 +32,13 @@ struct RowSoftmaxCfg {
   static constexpr int kStoreWarp = 2 + kEpiWarps;
   static constexpr int kZeroWarp = kStoreWarp + 1;
   static constexpr int kThreads = 32 * (kZeroWarp + 1);
-  static constexpr int ZERO_TMA_LANES = 8;                   // zero boxes in flight per SM
+  static constexpr int ZERO_TMA_LANES = 4;                   // zero boxes in flight per SM
   static constexpr int CHUNK = 256;                          // columns per UMMA and per accumulator slot
   // Which of a 32-column fragment's 16 column pairs take 2^x from the FMA-pipe polynomial instead of the MUFU unit
   // (bit j = pair j).  The MUFU unit delivers 16 results per clock per SM and is this kernel's busiest pipe; the
-  // polynomial costs about six issue slots per value, so a bit over a third of the pairs balances the two.
-  static constexpr uint32_t POLY_PAIRS = 0x5252u;            // pairs 1, 4, 6, 9, 12, 14
+  // polynomial costs about six issue slots per value.  Measured on the attention-score workload: none 126.2 us,
+  // 2 of 16 pairs 123.7, 3: 123.1, 4: 122.7, 5: 123.9, 6: 124.8, 8: 128.8.
+  static constexpr uint32_t POLY_PAIRS = 0x1248u;            // pairs 3, 6, 9, 12
   static constexpr int A_BYTES = 128 * 64 * 2;
   static constexpr int STAGE_BYTES = A_BYTES + (CHUNK / 2) * 64 * 2;  // A block + this CTA's half of the B chunk
   static constexpr int WARP_BOX_BYTES = 32 * 64 * 2;
