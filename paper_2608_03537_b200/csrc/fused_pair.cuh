@@ -670,8 +670,6 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
         }
         // ---------------- stage 2 (PostOp): normalise the resident x, round once, store
-        const float relu_floor = (p.post_relu && !p.wide) ? 0.f : -INFINITY;  // wide rows: the second kernel applies it
-        (void)relu_floor;
         float best = -INFINITY;
         int best_col = 0x7FFFFFFF;
 #pragma unroll
@@ -699,8 +697,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const float2 n23 = fma2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd), splat2(-mu * rstd));
                   const float2 y01 = fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y));
                   const float2 y23 = fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w));
-                  // relu_floor is 0 for the LayerNorm-ReLU pattern, -inf otherwise
-                  y0 = fmaxf(y01.x, relu_floor); y1 = fmaxf(y01.y, relu_floor); y2 = fmaxf(y23.x, relu_floor); y3 = fmaxf(y23.y, relu_floor);
+                  y0 = y01.x; y1 = y01.y; y2 = y23.x; y3 = y23.y;
                 } else {
                   const float2 y01 = mul2(mul2(f2_from_bits(v[4 * j], v[4 * j + 1]), splat2(rstd)), make_float2(gg.x, gg.y));
                   const float2 y23 = mul2(mul2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd)), make_float2(gg.z, gg.w));
@@ -714,6 +711,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 pk[half * 16 + 2 * j] = pack_bf16x2_rn(y0, y1);
                 pk[half * 16 + 2 * j + 1] = pack_bf16x2_rn(y2, y3);
               }
+            }
+            if (EPI == EPI_LN && p.post_relu && !p.wide) {
+              // LayerNorm-ReLU pattern: on the rounded pairs (rounding is monotone and 0 is exact, so the order does not
+              // matter); wide rows: the second kernel applies it
+#pragma unroll
+              for (int j = 0; j < 32; ++j) asm("max.bf16x2 %0, %0, %1;" : "+r"(pk[j]) : "r"(0u));
             }
             store_box(pk);
             COMFUSE_TRACE_POINT();
