@@ -230,3 +230,107 @@ def sample_rows(M: int, count: int, seed: int = 12345) -> np.ndarray:
     pool = g.choice(M, size=min(M, extra), replace=False)
     rows = sorted(fixed.union(int(r) for r in pool))
     return np.asarray(rows[:max(count, len(fixed))], dtype=np.int64)
+
+
+# ----------------------------------------------------------------------------
+# epilogue programs as data (node lists; no arithmetic here, only the lists)
+# ----------------------------------------------------------------------------
+# A node is (op, in0, in1, param, imm): op is a name of the Fusion-Spec vocabulary (Sec. 5.2: accumulator entry,
+# broadcasts, element-wise computations, reductions), in0/in1 index earlier nodes, param indexes the call's parameter
+# table, imm is the value of a "const" node.
+
+
+class _Prog:
+    def __init__(self):
+        self.nodes = []
+
+    def add(self, op, a=-1, b=-1, param=-1, imm=0.0):
+        self.nodes.append((op, int(a), int(b), int(param), float(imm)))
+        return len(self.nodes) - 1
+
+
+@dataclass
+class SpecProgram:
+    """An epilogue program: ordered nodes, the terminal node stored as Y, per-row outputs, and what each parameter slot
+    holds ("rowvec" [N] / "tensor" [M, N])."""
+    nodes: list
+    terminal: int
+    row_outputs: tuple = ()
+    param_kinds: tuple = ()
+
+
+def spec_layernorm(eps=1e-5, bias=True, residual=True, affine=True, relu=False) -> SpecProgram:
+    """MatMul-BiasAdd(-Residual)-LayerNorm(-ReLU) spelled with primitive nodes: two mean reductions (Sec. 3.2, Fig. 3;
+    the MBLR pattern of Sec. 6.1 with relu=True).  Parameter slots in order: bias, residual, gamma, beta (those present)."""
+    g = _Prog()
+    kinds = []
+    x = g.add("acc")
+    if bias:
+        kinds.append("rowvec")
+        x = g.add("add", x, g.add("rowvec", param=len(kinds) - 1))
+    if residual:
+        kinds.append("tensor")
+        x = g.add("add", x, g.add("tensor", param=len(kinds) - 1))
+    mean = g.add("mean", x)
+    d = g.add("sub", x, mean)
+    var = g.add("mean", g.add("square", d))
+    rstd = g.add("rsqrt", g.add("add", var, g.add("const", imm=eps)))
+    y = g.add("mul", d, rstd)
+    if affine:
+        kinds.append("rowvec")
+        y = g.add("mul", y, g.add("rowvec", param=len(kinds) - 1))
+        kinds.append("rowvec")
+        y = g.add("add", y, g.add("rowvec", param=len(kinds) - 1))
+    if relu:
+        y = g.add("relu", y)
+    return SpecProgram(g.nodes, y, (), tuple(kinds))
+
+
+def spec_rmsnorm_max(eps=1e-5, activation=True, residual=True) -> SpecProgram:
+    """MatMul-BiasAdd(-GELU)(-Residual)-RMSNorm, then the chained row max / arg max (Sec. 3.2 chaining; the MBR pattern
+    of Sec. 6.1 with activation=False, residual=False).  Parameter slots: bias, [residual], gain."""
+    g = _Prog()
+    kinds = ["rowvec"]
+    x = g.add("add", g.add("acc"), g.add("rowvec", param=0))
+    if activation:
+        x = g.add("gelu_tanh", x)
+    if residual:
+        kinds.append("tensor")
+        x = g.add("add", x, g.add("tensor", param=len(kinds) - 1))
+    ms = g.add("mean", g.add("square", x))
+    rstd = g.add("rsqrt", g.add("add", ms, g.add("const", imm=eps)))
+    kinds.append("rowvec")
+    y = g.add("mul", g.add("mul", x, rstd), g.add("rowvec", param=len(kinds) - 1))
+    mx = g.add("rmax", y)
+    am = g.add("argmax", y)
+    return SpecProgram(g.nodes, y, (mx, am), tuple(kinds))
+
+
+def spec_softmax(alpha=1.0, causal=False, softcap=0.0) -> SpecProgram:
+    """MatMul-Scale(-TanhSoftcap)(-Mask)-Softmax spelled with primitive nodes (the MSTS pattern of Sec. 6.1): a max and a
+    sum reduction."""
+    g = _Prog()
+    t = g.add("mul", g.add("acc"), g.add("const", imm=alpha))
+    if softcap > 0.0:
+        t = g.add("mul", g.add("tanh", g.add("mul", t, g.add("const", imm=1.0 / softcap))), g.add("const", imm=softcap))
+    if causal:
+        t = g.add("add", t, g.add("causal_mask"))
+    e = g.add("exp", g.add("sub", t, g.add("rmax", t)))
+    y = g.add("div", e, g.add("sum", e))
+    return SpecProgram(g.nodes, y, (), ())
+
+
+def spec_gated_minmax() -> SpecProgram:
+    """A program outside the compiled patterns: a gate x * sigmoid(x) spelled with two uses of x (a DAG, not a chain),
+    rescaled to the row's range with a min and a max reduction, plus the row product of the gate's sigmoid as a
+    per-row output (exercises the min / max / prod reduction operators of Sec. 5).  Parameter slot 0: bias."""
+    g = _Prog()
+    x = g.add("add", g.add("acc"), g.add("rowvec", param=0))
+    sg = g.add("sigmoid", x)
+    s = g.add("mul", x, sg)
+    lo = g.add("rmin", s)
+    hi = g.add("rmax", s)
+    rng = g.add("add", g.add("sub", hi, lo), g.add("const", imm=1e-3))
+    y = g.add("div", g.add("sub", s, lo), rng)
+    pr = g.add("prod", g.add("add", g.add("mul", sg, g.add("const", imm=0.01)), g.add("const", imm=0.995)))
+    return SpecProgram(g.nodes, y, (lo, hi, pr), ("rowvec",))
