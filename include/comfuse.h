@@ -204,6 +204,105 @@ comfuse_status_t comfuse_selftest_bounded_wait(uint32_t timeout_ms, void* cuda_s
 
 const char* comfuse_status_string(comfuse_status_t status);
 
+/* ------------------------------------------------------------------------------------------------------------
+ * Epilogue given as DATA (Sec. 5.2 Fusion Spec IR, Sec. 5.3 reduction subgraph splitting, Sec. 5.4 backend mapping).
+ *
+ * The memory-intensive subgraph is a topologically ordered list of nodes of four categories -- accumulator entry,
+ * broadcast, element-wise computation, reduction over the last dimension N -- with edges to EARLIER nodes, one
+ * terminal node (its value is stored to Y as bf16, rounded once) and a table of runtime parameters.  A reduction
+ * yields one value per row that later element-wise nodes may use (broadcast along the row); that is how LayerNorm,
+ * RMSNorm and Softmax are spelled with primitive nodes.  All arithmetic is fp32.
+ *
+ * What the library does with a program (the two mappings of Sec. 5):
+ *   1. checks it (closure: a node outside this vocabulary, a forward edge, a mistyped parameter is rejected with
+ *      COMFUSE_ERR_INVALID_ARG, nothing is dropped silently), types every node (tensor / per-row / constant) and
+ *      splits it into stages at the reduction nodes: stage(node) = max over its inputs of stage(input), plus one
+ *      behind a reduction;
+ *   2. lowers it: a program whose stages have the shape of a compiled fused instantiation (affine entry
+ *      [activation] [+ residual] -> LayerNorm | RMSNorm [-> max/argmax] | softmax, in any spelling the canonicaliser
+ *      recognises: operand order of commutative nodes, optional nodes absent) runs as that ONE fused kernel
+ *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); any other valid program runs on the standard pathway
+ *      (COMFUSE_SPEC_PATH_ROW_PROGRAM): the GEMM kernel writes bf16 Z to the workspace and one row-program kernel
+ *      evaluates the node list per row with the row resident in shared memory, one pass per stage.
+ */
+typedef enum {
+  COMFUSE_OP_ACC = 0,          /* accumulator entry: (A.B)[i, j]                                      */
+  COMFUSE_OP_CONST = 1,        /* scalar broadcast of `imm`                                           */
+  COMFUSE_OP_ROWVEC = 2,       /* row-vector broadcast: params[param][j], bf16 [N]                    */
+  COMFUSE_OP_TENSOR = 3,       /* full tensor: params[param][i, j], bf16 [batch, M, N], ld = param_ld */
+  COMFUSE_OP_CAUSAL_MASK = 4,  /* 0 where j <= i, -inf above the diagonal                             */
+  COMFUSE_OP_NEG = 16, COMFUSE_OP_ABS = 17, COMFUSE_OP_SQUARE = 18, COMFUSE_OP_SQRT = 19, COMFUSE_OP_RSQRT = 20,
+  COMFUSE_OP_RECIP = 21, COMFUSE_OP_EXP = 22, COMFUSE_OP_LOG = 23, COMFUSE_OP_TANH = 24, COMFUSE_OP_RELU = 25,
+  COMFUSE_OP_GELU_TANH = 26, COMFUSE_OP_SIGMOID = 27,                                    /* unary: in0       */
+  COMFUSE_OP_ADD = 32, COMFUSE_OP_SUB = 33, COMFUSE_OP_MUL = 34, COMFUSE_OP_DIV = 35,
+  COMFUSE_OP_MAX = 36, COMFUSE_OP_MIN = 37,                                              /* binary: in0, in1 */
+  /* reductions of in0 over the row (ReduceOp sum / prod / max / min and ReduceMode mean of the StreamReduction
+   * node, Sec. 5); ARGMAX = lowest column attaining the row maximum, as a number */
+  COMFUSE_OP_RED_SUM = 48, COMFUSE_OP_RED_MEAN = 49, COMFUSE_OP_RED_MAX = 50, COMFUSE_OP_RED_MIN = 51,
+  COMFUSE_OP_RED_PROD = 52, COMFUSE_OP_RED_ARGMAX = 53
+} comfuse_op_t;
+
+typedef struct {
+  int32_t op;        /* comfuse_op_t */
+  int32_t in0, in1;  /* indices of earlier nodes, -1 where the op takes no such input */
+  int32_t param;     /* ROWVEC / TENSOR: index into the parameter table, else -1 */
+  float imm;         /* CONST: the value */
+} comfuse_spec_node_t;
+
+#define COMFUSE_SPEC_MAX_NODES 128
+#define COMFUSE_SPEC_MAX_PARAMS 12
+#define COMFUSE_SPEC_MAX_ROW_OUTPUTS 8
+
+typedef struct {
+  int32_t n_nodes;                   /* 1 .. COMFUSE_SPEC_MAX_NODES */
+  const comfuse_spec_node_t* nodes;  /* HOST array, read during the call only */
+  int32_t terminal;                  /* node whose value is Y */
+  int32_t n_params;                  /* entries of the parameter table, 0 .. COMFUSE_SPEC_MAX_PARAMS */
+  int32_t n_row_outputs;             /* 0 .. COMFUSE_SPEC_MAX_ROW_OUTPUTS */
+  const int32_t* row_outputs;        /* HOST array of per-row valued nodes; output k is written to row_out[k]:
+                                        fp32 [batch*M], or int32 [batch*M] when the node is a RED_ARGMAX */
+} comfuse_fusion_spec_t;
+
+typedef struct {
+  int32_t batch, M, N, K;
+  int64_t lda, ldb, ldy;
+  int64_t batch_stride_a, batch_stride_b, batch_stride_y;  /* used when batch > 1 */
+} comfuse_gemm_shape_t;
+
+typedef enum { COMFUSE_SPEC_PATH_FUSED_KERNEL = 0, COMFUSE_SPEC_PATH_ROW_PROGRAM = 1 } comfuse_spec_path_t;
+
+/* What the library will do with a program on a given shape (host-side analysis only; no device is touched). */
+typedef struct {
+  int32_t n_stages;       /* 1 + number of reductions on the longest dependency chain                    */
+  int32_t n_reductions;   /* live reduction nodes                                                       */
+  int32_t n_live_nodes;   /* nodes the terminal or a row output depends on                              */
+  int32_t path;           /* comfuse_spec_path_t chosen when `fused` = 1                                */
+  int32_t fused_kind;     /* FUSED_KERNEL: the comfuse_epilogue_kind_t it lowers to, else -1            */
+  uint32_t fused_flags;   /* FUSED_KERNEL: COMFUSE_FLAG_* bits                                          */
+  float alpha, eps, softcap;  /* FUSED_KERNEL: recovered constants                                      */
+  int32_t causal;         /* FUSED_KERNEL: 1 if the program adds the causal mask                        */
+  int32_t n_instructions; /* ROW_PROGRAM: computed nodes the row kernel executes                        */
+  int32_t n_slots;        /* ROW_PROGRAM: row-sized fp32 buffers held in shared memory at the same time */
+} comfuse_spec_plan_t;
+
+/* Analyse a program: OK and *plan filled, INVALID_ARG for a malformed program (see above), UNSUPPORTED if it is valid
+ * but cannot run on this shape (the row program's buffers exceed shared memory and no fused kernel matches). */
+comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape,
+                                   comfuse_spec_plan_t* plan);
+
+/* Workspace comfuse_gemm_spec needs (bytes): 0 or row scratch for the fused kernel, batch*M*N*2 for the row program. */
+comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape,
+                                                  int32_t fused, size_t* bytes);
+
+/* Y = program(A . B).  `params`: HOST array of spec->n_params DEVICE pointers (bf16; ROWVEC [N], TENSOR [batch, M, N]
+ * with leading dimension param_ld[k], 0 = N); `param_ld` may be NULL.  `row_out`: HOST array of n_row_outputs DEVICE
+ * pointers.  `fused` = 1: take the fused kernel when the program lowers to one; 0: always the row-program pathway.
+ * Asynchronous on `cuda_stream`; the host arrays are not read after the call returns. */
+comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A,
+                                   const void* B, void* Y, const void* const* params, const int64_t* param_ld,
+                                   void* const* row_out, int32_t fused, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -44,6 +44,9 @@ EXPORTED_SYMBOLS = (
     "comfuse_gemm_epilogue_host",
     "comfuse_b2b_host_staging_size",
     "comfuse_b2b_gemm_host",
+    "comfuse_spec_plan",
+    "comfuse_gemm_spec_workspace_size",
+    "comfuse_gemm_spec",
     "comfuse_last_device_status",
     "comfuse_launch_count",
     "comfuse_selftest_bounded_wait",
@@ -71,6 +74,39 @@ class EpilogueArgs(Structure):
 class B2bDesc(Structure):
     _fields_ = [("M", c_int32), ("K", c_int32), ("N1", c_int32), ("N2", c_int32), ("eps", c_float), ("fused", c_int32),
                 ("kind", c_int32), ("batch", c_int32), ("alpha", c_float), ("reserved", c_int32)]
+
+
+# Epilogue programs as data: the node vocabulary (comfuse_op_t), by name
+OPS = {
+    "acc": 0, "const": 1, "rowvec": 2, "tensor": 3, "causal_mask": 4,
+    "neg": 16, "abs": 17, "square": 18, "sqrt": 19, "rsqrt": 20, "recip": 21, "exp": 22, "log": 23, "tanh": 24,
+    "relu": 25, "gelu_tanh": 26, "sigmoid": 27,
+    "add": 32, "sub": 33, "mul": 34, "div": 35, "max": 36, "min": 37,
+    "sum": 48, "mean": 49, "rmax": 50, "rmin": 51, "prod": 52, "argmax": 53,
+}
+SPEC_PATH_FUSED_KERNEL = 0
+SPEC_PATH_ROW_PROGRAM = 1
+
+
+class SpecNode(Structure):
+    _fields_ = [("op", c_int32), ("in0", c_int32), ("in1", c_int32), ("param", c_int32), ("imm", c_float)]
+
+
+class FusionSpec(Structure):
+    _fields_ = [("n_nodes", c_int32), ("nodes", POINTER(SpecNode)), ("terminal", c_int32), ("n_params", c_int32),
+                ("n_row_outputs", c_int32), ("row_outputs", POINTER(c_int32))]
+
+
+class GemmShape(Structure):
+    _fields_ = [("batch", c_int32), ("M", c_int32), ("N", c_int32), ("K", c_int32),
+                ("lda", c_int64), ("ldb", c_int64), ("ldy", c_int64),
+                ("batch_stride_a", c_int64), ("batch_stride_b", c_int64), ("batch_stride_y", c_int64)]
+
+
+class SpecPlan(Structure):
+    _fields_ = [("n_stages", c_int32), ("n_reductions", c_int32), ("n_live_nodes", c_int32), ("path", c_int32),
+                ("fused_kind", c_int32), ("fused_flags", ctypes.c_uint32), ("alpha", c_float), ("eps", c_float),
+                ("softcap", c_float), ("causal", c_int32), ("n_instructions", c_int32), ("n_slots", c_int32)]
 
 
 class ComfuseError(RuntimeError):
@@ -113,6 +149,13 @@ def lib() -> ctypes.CDLL:
         L.comfuse_b2b_host_staging_size.restype = c_int32
         L.comfuse_b2b_gemm_host.argtypes = [POINTER(B2bDesc)] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p, c_size_t, c_void_p]
         L.comfuse_b2b_gemm_host.restype = c_int32
+        L.comfuse_spec_plan.argtypes = [POINTER(FusionSpec), POINTER(GemmShape), POINTER(SpecPlan)]
+        L.comfuse_spec_plan.restype = c_int32
+        L.comfuse_gemm_spec_workspace_size.argtypes = [POINTER(FusionSpec), POINTER(GemmShape), c_int32, POINTER(c_size_t)]
+        L.comfuse_gemm_spec_workspace_size.restype = c_int32
+        L.comfuse_gemm_spec.argtypes = [POINTER(FusionSpec), POINTER(GemmShape), c_void_p, c_void_p, c_void_p, POINTER(c_void_p),
+                                        POINTER(c_int64), POINTER(c_void_p), c_int32, c_void_p, c_size_t, c_void_p]
+        L.comfuse_gemm_spec.restype = c_int32
         L.comfuse_last_device_status.argtypes = [c_void_p]
         L.comfuse_last_device_status.restype = c_int32
         L.comfuse_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, POINTER(ctypes.c_uint32)]
@@ -305,6 +348,63 @@ def b2b_attention_host(Q, Kt, V, O, *, staging, alpha, fused=True, workspace=Non
     if st != OK:
         raise ComfuseError(st, "comfuse_b2b_gemm_host")
     return O
+
+
+def make_spec(nodes, terminal, n_params=0, row_outputs=()) -> FusionSpec:
+    """Pack a node list ``[(op name or code, in0, in1, param, imm), ...]`` into the C structure (host arrays are kept
+    alive by the returned object)."""
+    arr = (SpecNode * len(nodes))()
+    for k, (op, a, b, prm, imm) in enumerate(nodes):
+        arr[k] = SpecNode(OPS[op] if isinstance(op, str) else int(op), int(a), int(b), int(prm), float(imm))
+    ro = (c_int32 * max(1, len(row_outputs)))(*[int(r) for r in row_outputs])
+    spec = FusionSpec(len(nodes), ctypes.cast(arr, POINTER(SpecNode)), int(terminal), int(n_params), len(row_outputs),
+                      ctypes.cast(ro, POINTER(c_int32)))
+    spec._keep = (arr, ro)
+    return spec
+
+
+def make_gemm_shape(batch, M, N, K, lda=None, ldb=None, ldy=None, batch_stride_a=None, batch_stride_b=None,
+                    batch_stride_y=None) -> GemmShape:
+    lda, ldb, ldy = lda or K, ldb or N, ldy or N
+    return GemmShape(batch, M, N, K, lda, ldb, ldy, batch_stride_a or M * lda, batch_stride_b or K * ldb, batch_stride_y or M * ldy)
+
+
+def spec_plan(spec: FusionSpec, shape: GemmShape) -> SpecPlan:
+    """Host-side analysis of a program on a shape (needs no GPU): stages, path, recovered constants."""
+    plan = SpecPlan()
+    st = lib().comfuse_spec_plan(byref(spec), byref(shape), byref(plan))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_spec_plan")
+    return plan
+
+
+def gemm_spec_workspace_size(spec: FusionSpec, shape: GemmShape, fused=True) -> int:
+    n = c_size_t(0)
+    st = lib().comfuse_gemm_spec_workspace_size(byref(spec), byref(shape), 1 if fused else 0, byref(n))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_spec_workspace_size")
+    return int(n.value)
+
+
+def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, workspace=None, stream=None):
+    """Enqueue Y = program(A.B): ``spec`` from make_spec, ``params`` the CUDA bf16 tensors of the parameter table
+    (row vectors [N], tensors [batch, M, N]), ``row_out`` the per-row output tensors (fp32, int32 for an arg max)."""
+    batched = A.dim() == 3
+    batch = A.shape[0] if batched else 1
+    M, K = A.shape[-2], A.shape[-1]
+    N = B.shape[-1]
+    shape = make_gemm_shape(batch, M, N, K, A.stride(-2), B.stride(-2), Y.stride(-2),
+                            A.stride(0) if batched else None, B.stride(0) if batched else None, Y.stride(0) if batched else None)
+    n = max(1, len(params))
+    pp = (c_void_p * n)(*[None if t is None else t.data_ptr() for t in params])
+    ld = (c_int64 * n)(*[0 if (t is None or t.dim() < 2) else t.stride(-2) for t in params])
+    ro = (c_void_p * max(1, len(row_out)))(*[t.data_ptr() for t in row_out])
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_gemm_spec(byref(spec), byref(shape), _ptr(A), _ptr(B), _ptr(Y), pp, ld, ro, 1 if fused else 0,
+                                 ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_spec")
+    return Y
 
 
 def last_device_status(stream=None) -> int:

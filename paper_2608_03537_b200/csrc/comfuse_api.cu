@@ -180,6 +180,30 @@ comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
 }
 
 }  // namespace
+
+comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
+                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st) {
+  const DeviceInfo* dev = nullptr;
+  comfuse_status_t s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  GemmMaps maps;
+  if (!make_gemm_maps(&maps, A, B, nullptr, Z, batch, M, N, K, lda, ldb, 0, N, batch_stride_a, batch_stride_b, 0,
+                      static_cast<long long>(M) * N))
+    return COMFUSE_ERR_CUDA;
+  FusedParams p = {};
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.mblocks = (M + 127) / 128;
+  p.nblocks = 1;
+  p.total_tiles = batch * p.mblocks;
+  p.alpha = 1.f;
+  p.status = dev->status_word;
+  p.timeout_ns = timeout_ns();
+  p.Y = static_cast<uint16_t*>(Z);
+  p.ldy = N;
+  p.batch_stride_y = static_cast<long long>(M) * N;
+  return launch_plain_gemm(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
 }  // namespace comfuse
 
 using namespace comfuse;

@@ -1,0 +1,609 @@
+// Epilogue programs given as data: host-side analysis and lowering (Sec. 5.2 frontend mapping, Sec. 5.3 reduction
+// subgraph splitting, Sec. 5.4 backend mapping) and the entry points that run them.
+//
+//   analyse():  checks the node list (closed vocabulary, edges to earlier nodes only, consistent parameter use), types
+//               every node (tensor / per-row / constant), folds constants, marks what the terminal and the row outputs
+//               depend on, and numbers the stages: a reduction's result belongs to the stage after its input's.
+//   match_*():  canonicalisation onto the compiled fused instantiations.  The matchers walk the DAG from the terminal
+//               node and accept any operand order of commutative nodes and any subset of the optional nodes.
+//   lower_row_program(): the standard pathway -- one instruction per live computed node, shared-memory slots assigned
+//               by liveness (a node's buffer is released at its last use and may be overwritten in place).
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "comfuse.h"
+#include "fusion_spec.h"
+#include "host_common.h"
+
+namespace comfuse {
+
+namespace {
+
+enum NodeType : uint8_t { T_TENSOR = 0, T_ROW = 1, T_CONST = 2 };
+
+bool is_unary(int op) { return op >= COMFUSE_OP_NEG && op <= COMFUSE_OP_SIGMOID; }
+bool is_binary(int op) { return op >= COMFUSE_OP_ADD && op <= COMFUSE_OP_MIN; }
+bool is_reduce(int op) { return op >= COMFUSE_OP_RED_SUM && op <= COMFUSE_OP_RED_ARGMAX; }
+bool is_leaf(int op) { return op >= COMFUSE_OP_ACC && op <= COMFUSE_OP_CAUSAL_MASK; }
+
+float fold_unary(int op, float a) {
+  switch (op) {
+    case COMFUSE_OP_NEG: return -a;
+    case COMFUSE_OP_ABS: return std::fabs(a);
+    case COMFUSE_OP_SQUARE: return a * a;
+    case COMFUSE_OP_SQRT: return std::sqrt(a);
+    case COMFUSE_OP_RSQRT: return 1.f / std::sqrt(a);
+    case COMFUSE_OP_RECIP: return 1.f / a;
+    case COMFUSE_OP_EXP: return std::exp(a);
+    case COMFUSE_OP_LOG: return std::log(a);
+    case COMFUSE_OP_TANH: return std::tanh(a);
+    case COMFUSE_OP_RELU: return a > 0.f ? a : 0.f;
+    case COMFUSE_OP_GELU_TANH: return 0.5f * a * (1.f + std::tanh(0.7978845608028654f * (a + 0.044715f * a * a * a)));
+    case COMFUSE_OP_SIGMOID: return 1.f / (1.f + std::exp(-a));
+    default: return a;
+  }
+}
+
+float fold_binary(int op, float a, float b) {
+  switch (op) {
+    case COMFUSE_OP_ADD: return a + b;
+    case COMFUSE_OP_SUB: return a - b;
+    case COMFUSE_OP_MUL: return a * b;
+    case COMFUSE_OP_DIV: return a / b;
+    case COMFUSE_OP_MAX: return a > b ? a : b;
+    case COMFUSE_OP_MIN: return a < b ? a : b;
+    default: return a;
+  }
+}
+
+struct Analysis {
+  int n = 0;
+  std::vector<comfuse_spec_node_t> nodes;
+  std::vector<uint8_t> type;     // NodeType
+  std::vector<float> cval;       // value of T_CONST nodes (given or folded)
+  std::vector<uint8_t> live;
+  std::vector<int> stage;
+  int param_kind[COMFUSE_SPEC_MAX_PARAMS];  // 0 unused, COMFUSE_OP_ROWVEC or COMFUSE_OP_TENSOR
+  int terminal = 0;
+  std::vector<int> row_outputs;
+  int n_stages = 1, n_reductions = 0, n_live = 0;
+};
+
+comfuse_status_t analyse(const comfuse_fusion_spec_t* spec, Analysis& an) {
+  if (!spec || !spec->nodes) return COMFUSE_ERR_INVALID_ARG;
+  if (spec->n_nodes < 1 || spec->n_nodes > COMFUSE_SPEC_MAX_NODES) return COMFUSE_ERR_INVALID_ARG;
+  if (spec->n_params < 0 || spec->n_params > COMFUSE_SPEC_MAX_PARAMS) return COMFUSE_ERR_INVALID_ARG;
+  if (spec->n_row_outputs < 0 || spec->n_row_outputs > COMFUSE_SPEC_MAX_ROW_OUTPUTS) return COMFUSE_ERR_INVALID_ARG;
+  if (spec->n_row_outputs > 0 && !spec->row_outputs) return COMFUSE_ERR_INVALID_ARG;
+  if (spec->terminal < 0 || spec->terminal >= spec->n_nodes) return COMFUSE_ERR_INVALID_ARG;
+  const int n = spec->n_nodes;
+  an.n = n;
+  an.nodes.assign(spec->nodes, spec->nodes + n);
+  an.type.assign(n, T_TENSOR);
+  an.cval.assign(n, 0.f);
+  an.live.assign(n, 0);
+  an.stage.assign(n, 0);
+  an.terminal = spec->terminal;
+  std::memset(an.param_kind, 0, sizeof(an.param_kind));
+  for (int k = 0; k < n; ++k) {
+    const comfuse_spec_node_t& nd = an.nodes[k];
+    const int op = nd.op;
+    auto edge_ok = [&](int e) { return e >= 0 && e < k; };
+    if (is_leaf(op)) {
+      if (nd.in0 != -1 || nd.in1 != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (op == COMFUSE_OP_ROWVEC || op == COMFUSE_OP_TENSOR) {
+        if (nd.param < 0 || nd.param >= spec->n_params) return COMFUSE_ERR_INVALID_ARG;
+        if (an.param_kind[nd.param] != 0 && an.param_kind[nd.param] != op) return COMFUSE_ERR_INVALID_ARG;  // one slot, two shapes
+        an.param_kind[nd.param] = op;
+      } else if (nd.param != -1) {
+        return COMFUSE_ERR_INVALID_ARG;
+      }
+      if (op == COMFUSE_OP_CONST) {
+        an.type[k] = T_CONST;
+        an.cval[k] = nd.imm;
+      }
+    } else if (is_unary(op) || is_reduce(op)) {
+      if (!edge_ok(nd.in0) || nd.in1 != -1 || nd.param != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (is_reduce(op)) {
+        an.type[k] = T_ROW;
+        an.stage[k] = an.stage[nd.in0] + 1;
+      } else {
+        an.type[k] = an.type[nd.in0];
+        an.stage[k] = an.stage[nd.in0];
+        if (an.type[k] == T_CONST) an.cval[k] = fold_unary(op, an.cval[nd.in0]);
+      }
+    } else if (is_binary(op)) {
+      if (!edge_ok(nd.in0) || !edge_ok(nd.in1) || nd.param != -1) return COMFUSE_ERR_INVALID_ARG;
+      const uint8_t ta = an.type[nd.in0], tb = an.type[nd.in1];
+      an.type[k] = (ta == T_TENSOR || tb == T_TENSOR) ? T_TENSOR : (ta == T_ROW || tb == T_ROW) ? T_ROW : T_CONST;
+      an.stage[k] = an.stage[nd.in0] > an.stage[nd.in1] ? an.stage[nd.in0] : an.stage[nd.in1];
+      if (an.type[k] == T_CONST) an.cval[k] = fold_binary(op, an.cval[nd.in0], an.cval[nd.in1]);
+    } else {
+      return COMFUSE_ERR_INVALID_ARG;  // outside the vocabulary: rejected, never dropped
+    }
+  }
+  an.row_outputs.assign(spec->row_outputs, spec->row_outputs + spec->n_row_outputs);
+  for (int r : an.row_outputs) {
+    if (r < 0 || r >= n) return COMFUSE_ERR_INVALID_ARG;
+    if (an.type[r] == T_TENSOR) return COMFUSE_ERR_INVALID_ARG;  // a row output is one value per row
+  }
+  // liveness: what the terminal and the row outputs depend on (constants that were folded need no inputs)
+  an.live[an.terminal] = 1;
+  for (int r : an.row_outputs) an.live[r] = 1;
+  for (int k = n - 1; k >= 0; --k) {
+    if (!an.live[k] || an.type[k] == T_CONST) continue;
+    if (an.nodes[k].in0 >= 0) an.live[an.nodes[k].in0] = 1;
+    if (an.nodes[k].in1 >= 0) an.live[an.nodes[k].in1] = 1;
+  }
+  int max_stage = 0;
+  for (int k = 0; k < n; ++k) {
+    if (!an.live[k]) continue;
+    ++an.n_live;
+    if (is_reduce(an.nodes[k].op)) ++an.n_reductions;
+    if (an.stage[k] > max_stage) max_stage = an.stage[k];
+  }
+  an.n_stages = max_stage + 1;
+  return COMFUSE_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ canonicalisation
+struct FusedMatch {
+  int kind = -1;
+  uint32_t flags = 0;
+  float alpha = 1.f, eps = 0.f, softcap = 0.f;
+  int causal = 0;
+  int bias = -1, residual = -1, gamma = -1, beta = -1;  // parameter slots, -1 = absent
+  int row_max_out = -1, row_argmax_out = -1;            // positions in row_outputs, -1 = not asked for
+};
+
+struct Matcher {
+  const Analysis& an;
+  std::vector<uint8_t> used;
+  explicit Matcher(const Analysis& a) : an(a), used(a.n, 0) {}
+  const comfuse_spec_node_t& nd(int k) const { return an.nodes[k]; }
+  bool is(int k, int op) const { return k >= 0 && an.type[k] != T_CONST && nd(k).op == op; }
+  bool is_const(int k) const { return k >= 0 && an.type[k] == T_CONST; }
+  void use(int k) { used[k] = 1; }
+  // binary node `k` of kind `op` with one operand satisfying `pred`: returns the OTHER operand and the matching one
+  template <class Pred>
+  bool split(int k, int op, Pred pred, int& other, int& hit) const {
+    if (!is(k, op)) return false;
+    const int a = nd(k).in0, b = nd(k).in1;
+    if (pred(b)) { other = a; hit = b; return true; }
+    if (op != COMFUSE_OP_SUB && op != COMFUSE_OP_DIV && pred(a)) { other = b; hit = a; return true; }
+    return false;
+  }
+  bool all_live_used() const {
+    for (int k = 0; k < an.n; ++k)
+      if (an.live[k] && !used[k] && an.type[k] != T_CONST) return false;
+    return true;
+  }
+
+  // x = [act](alpha * acc [+ bias]) [+ residual], peeled from the outside; without an activation the bias and the
+  // residual may come in either order (with one, gelu_entry_order_ok() checks the order afterwards)
+  bool entry(int k, bool allow_act, FusedMatch& m, bool& had_act) {
+    had_act = false;
+    int other, hit;
+    for (int guard = 0; guard < 4; ++guard) {
+      if (m.residual < 0 && split(k, COMFUSE_OP_ADD, [&](int t) { return is(t, COMFUSE_OP_TENSOR); }, other, hit)) {
+        m.residual = nd(hit).param; use(k); use(hit); k = other;
+      } else if (!had_act && allow_act && is(k, COMFUSE_OP_GELU_TANH)) {
+        had_act = true; use(k); k = nd(k).in0;
+      } else if (m.bias < 0 && split(k, COMFUSE_OP_ADD, [&](int t) { return is(t, COMFUSE_OP_ROWVEC); }, other, hit)) {
+        m.bias = nd(hit).param; use(k); use(hit); k = other;
+      } else {
+        break;
+      }
+    }
+    if (split(k, COMFUSE_OP_MUL, [&](int t) { return is_const(t); }, other, hit)) {
+      m.alpha = an.cval[hit]; use(k); k = other;
+    }
+    if (!is(k, COMFUSE_OP_ACC)) return false;
+    use(k);
+    return true;
+  }
+};
+
+// Order check for the GELU entry: residual outside the activation, bias inside (entry() peels greedily).
+bool gelu_entry_order_ok(const Analysis& an, int x) {
+  // chain from x down to acc: ops seen in order
+  int k = x;
+  bool seen_act = false;
+  for (int guard = 0; guard < 8; ++guard) {
+    const comfuse_spec_node_t& nd = an.nodes[k];
+    if (nd.op == COMFUSE_OP_ACC) return true;
+    if (nd.op == COMFUSE_OP_GELU_TANH) { seen_act = true; k = nd.in0; continue; }
+    if (nd.op == COMFUSE_OP_ADD || nd.op == COMFUSE_OP_MUL) {
+      const int a = nd.in0, b = nd.in1;
+      const bool a_leaf = is_leaf(an.nodes[a].op) && an.nodes[a].op != COMFUSE_OP_ACC, b_leaf = is_leaf(an.nodes[b].op) && an.nodes[b].op != COMFUSE_OP_ACC;
+      const int leaf = b_leaf ? b : a_leaf ? a : -1;
+      if (leaf < 0) return false;
+      const int lop = an.nodes[leaf].op;
+      if (lop == COMFUSE_OP_TENSOR && seen_act) return false;   // residual inside the activation
+      if (lop == COMFUSE_OP_ROWVEC && !seen_act) return false;  // bias outside the activation
+      k = leaf == b ? a : b;
+      continue;
+    }
+    return false;
+  }
+  return false;
+}
+
+bool match_layernorm(const Analysis& an, FusedMatch& m) {
+  if (!an.row_outputs.empty()) return false;
+  Matcher t(an);
+  int k = an.terminal, other, hit;
+  if (t.is(k, COMFUSE_OP_RELU)) { m.flags |= COMFUSE_FLAG_POST_RELU; t.use(k); k = t.nd(k).in0; }
+  if (t.split(k, COMFUSE_OP_ADD, [&](int q) { return t.is(q, COMFUSE_OP_ROWVEC); }, other, hit)) {
+    m.beta = t.nd(hit).param; t.use(k); t.use(hit); k = other;
+  }
+  if (t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is(q, COMFUSE_OP_ROWVEC); }, other, hit)) {
+    m.gamma = t.nd(hit).param; t.use(k); t.use(hit); k = other;
+  }
+  // (x - mean(x)) * rsqrt(mean((x - mean(x))^2) + eps)
+  int d, rstd;
+  if (!t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is(q, COMFUSE_OP_RSQRT); }, d, rstd)) return false;
+  t.use(k); t.use(rstd);
+  int var, epsn;
+  if (!t.split(t.nd(rstd).in0, COMFUSE_OP_ADD, [&](int q) { return t.is_const(q); }, var, epsn)) return false;
+  t.use(t.nd(rstd).in0);
+  m.eps = an.cval[epsn];
+  if (!t.is(var, COMFUSE_OP_RED_MEAN)) return false;
+  t.use(var);
+  const int sq = t.nd(var).in0;
+  const bool squared = t.is(sq, COMFUSE_OP_SQUARE) ? t.nd(sq).in0 == d : (t.is(sq, COMFUSE_OP_MUL) && t.nd(sq).in0 == d && t.nd(sq).in1 == d);
+  if (!squared) return false;
+  t.use(sq);
+  if (!t.is(d, COMFUSE_OP_SUB)) return false;
+  t.use(d);
+  const int x = t.nd(d).in0, mean = t.nd(d).in1;
+  if (!t.is(mean, COMFUSE_OP_RED_MEAN) || t.nd(mean).in0 != x) return false;
+  t.use(mean);
+  bool had_act;
+  if (!t.entry(x, false, m, had_act)) return false;
+  if (!t.all_live_used()) return false;
+  m.kind = COMFUSE_EPI_BIAS_RES_LAYERNORM;
+  return m.eps >= 0.f;
+}
+
+bool match_rmsnorm(const Analysis& an, FusedMatch& m) {
+  Matcher t(an);
+  int k = an.terminal, other, hit;
+  const int y = k;
+  if (t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is(q, COMFUSE_OP_ROWVEC); }, other, hit)) {
+    m.gamma = t.nd(hit).param; t.use(k); t.use(hit); k = other;
+  }
+  int x, rstd;
+  if (!t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is(q, COMFUSE_OP_RSQRT); }, x, rstd)) return false;
+  t.use(k); t.use(rstd);
+  int ms, epsn;
+  if (!t.split(t.nd(rstd).in0, COMFUSE_OP_ADD, [&](int q) { return t.is_const(q); }, ms, epsn)) return false;
+  t.use(t.nd(rstd).in0);
+  m.eps = an.cval[epsn];
+  if (!t.is(ms, COMFUSE_OP_RED_MEAN)) return false;
+  t.use(ms);
+  const int sq = t.nd(ms).in0;
+  const bool squared = t.is(sq, COMFUSE_OP_SQUARE) ? t.nd(sq).in0 == x : (t.is(sq, COMFUSE_OP_MUL) && t.nd(sq).in0 == x && t.nd(sq).in1 == x);
+  if (!squared) return false;
+  t.use(sq);
+  bool had_act;
+  if (!t.entry(x, true, m, had_act)) return false;
+  if (had_act ? !gelu_entry_order_ok(an, x) : false) return false;
+  if (!had_act) m.flags |= COMFUSE_FLAG_NO_ACTIVATION;
+  // the chained second reduction: row outputs may be the max and/or the arg max of Y
+  for (size_t r = 0; r < an.row_outputs.size(); ++r) {
+    const int q = an.row_outputs[r];
+    if (t.is(q, COMFUSE_OP_RED_MAX) && t.nd(q).in0 == y && m.row_max_out < 0) { m.row_max_out = static_cast<int>(r); t.use(q); }
+    else if (t.is(q, COMFUSE_OP_RED_ARGMAX) && t.nd(q).in0 == y && m.row_argmax_out < 0) { m.row_argmax_out = static_cast<int>(r); t.use(q); }
+    else return false;
+  }
+  if (!t.all_live_used()) return false;
+  m.kind = COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX;
+  return m.eps >= 0.f;
+}
+
+bool match_softmax(const Analysis& an, FusedMatch& m) {
+  if (!an.row_outputs.empty()) return false;
+  Matcher t(an);
+  const int k = an.terminal;
+  int e, sum;
+  if (t.is(k, COMFUSE_OP_DIV)) {
+    e = t.nd(k).in0; sum = t.nd(k).in1;
+  } else {
+    int rc;
+    if (!t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is(q, COMFUSE_OP_RECIP); }, e, rc)) return false;
+    t.use(rc);
+    sum = t.nd(rc).in0;
+  }
+  t.use(k);
+  if (!t.is(sum, COMFUSE_OP_RED_SUM) || t.nd(sum).in0 != e || !t.is(e, COMFUSE_OP_EXP)) return false;
+  t.use(sum); t.use(e);
+  const int d = t.nd(e).in0;
+  if (!t.is(d, COMFUSE_OP_SUB)) return false;
+  t.use(d);
+  int s = t.nd(d).in0;
+  const int mx = t.nd(d).in1;
+  if (!t.is(mx, COMFUSE_OP_RED_MAX) || t.nd(mx).in0 != s) return false;
+  t.use(mx);
+  int other, hit;
+  if (t.split(s, COMFUSE_OP_ADD, [&](int q) { return t.is(q, COMFUSE_OP_CAUSAL_MASK); }, other, hit)) {
+    m.causal = 1; t.use(s); t.use(hit); s = other;
+  }
+  // soft-cap: c2 * tanh(c1 * u) with c1 * c2 = 1
+  int th, c2;
+  if (t.split(s, COMFUSE_OP_MUL, [&](int q) { return t.is_const(q); }, th, c2) && t.is(th, COMFUSE_OP_TANH)) {
+    int u, c1;
+    if (!t.split(t.nd(th).in0, COMFUSE_OP_MUL, [&](int q) { return t.is_const(q); }, u, c1)) return false;
+    const float cap = an.cval[c2];
+    if (!(cap > 0.f) || std::fabs(an.cval[c1] * cap - 1.f) > 1e-5f) return false;
+    m.softcap = cap;
+    t.use(s); t.use(th); t.use(t.nd(th).in0);
+    s = u;
+  }
+  if (t.split(s, COMFUSE_OP_MUL, [&](int q) { return t.is_const(q); }, other, hit)) {
+    m.alpha = an.cval[hit]; t.use(s); s = other;
+  }
+  if (!t.is(s, COMFUSE_OP_ACC)) return false;
+  t.use(s);
+  if (!t.all_live_used()) return false;
+  m.kind = COMFUSE_EPI_SCALE_MASK_SOFTMAX;
+  return true;
+}
+
+bool match_fused(const Analysis& an, FusedMatch& m) {
+  { FusedMatch t; if (match_layernorm(an, t)) { m = t; return true; } }
+  { FusedMatch t; if (match_rmsnorm(an, t)) { m = t; return true; } }
+  { FusedMatch t; if (match_softmax(an, t)) { m = t; return true; } }
+  return false;
+}
+
+// ------------------------------------------------------------------------------------------------ row program
+comfuse_status_t lower_row_program(const Analysis& an, int N, RowProgram& P, int& n_instr, int& n_slots) {
+  const int n = an.n;
+  std::vector<int> last_use(n, -1);
+  for (int k = 0; k < n; ++k) {
+    if (!an.live[k] || an.type[k] == T_CONST) continue;
+    if (an.nodes[k].in0 >= 0) last_use[an.nodes[k].in0] = k;
+    if (an.nodes[k].in1 >= 0) last_use[an.nodes[k].in1] = k;
+  }
+  last_use[an.terminal] = n;
+  for (int r : an.row_outputs) last_use[r] = n;
+  std::vector<Operand> ref(n, Operand{OPK_NONE, 0, 0, 0.f});
+  std::vector<int> free_slots;
+  int slots = 0, scalars = 0, ni = 0;
+  for (int k = 0; k < n; ++k) {
+    if (!an.live[k]) continue;
+    const comfuse_spec_node_t& nd = an.nodes[k];
+    if (an.type[k] == T_CONST) { ref[k] = Operand{OPK_CONST, 0, 0, an.cval[k]}; continue; }
+    switch (nd.op) {
+      case COMFUSE_OP_ACC: ref[k] = Operand{OPK_ACC, 0, 0, 0.f}; continue;
+      case COMFUSE_OP_ROWVEC: ref[k] = Operand{OPK_ROWVEC, 0, static_cast<int16_t>(nd.param), 0.f}; continue;
+      case COMFUSE_OP_TENSOR: ref[k] = Operand{OPK_TENSOR, 0, static_cast<int16_t>(nd.param), 0.f}; continue;
+      case COMFUSE_OP_CAUSAL_MASK: ref[k] = Operand{OPK_MASK, 0, 0, 0.f}; continue;
+      default: break;
+    }
+    if (ni >= kRowMaxInstr) return COMFUSE_ERR_UNSUPPORTED;
+    RowInstr& in = P.ins[ni++];
+    in.op = static_cast<uint8_t>(nd.op);
+    in.a = ref[nd.in0];
+    in.b = nd.in1 >= 0 ? ref[nd.in1] : Operand{OPK_NONE, 0, 0, 0.f};
+    if (an.type[k] == T_ROW) {
+      if (scalars >= kRowMaxScalars) return COMFUSE_ERR_UNSUPPORTED;
+      in.dst_scalar = 1;
+      in.dst = static_cast<int16_t>(scalars);
+      ref[k] = Operand{OPK_SCALAR, 0, static_cast<int16_t>(scalars), 0.f};
+      ++scalars;
+    } else {
+      in.dst_scalar = 0;
+      // overwrite an operand's buffer in place if this is its last use, else take a free buffer, else a new one
+      int slot = -1;
+      for (int e : {nd.in0, nd.in1})
+        if (slot < 0 && e >= 0 && ref[e].kind == OPK_SLOT && last_use[e] == k) slot = ref[e].index;
+      if (slot < 0) {
+        if (!free_slots.empty()) { slot = free_slots.back(); free_slots.pop_back(); }
+        else slot = slots++;
+      }
+      in.dst = static_cast<int16_t>(slot);
+      ref[k] = Operand{OPK_SLOT, 0, static_cast<int16_t>(slot), 0.f};
+    }
+    // release the buffers whose last reader this was (unless just taken over)
+    for (int e : {nd.in0, nd.in1}) {
+      if (e < 0 || ref[e].kind != OPK_SLOT || last_use[e] != k) continue;
+      if (ref[k].kind == OPK_SLOT && ref[k].index == ref[e].index) continue;
+      bool already = false;
+      for (int f : free_slots) already |= f == ref[e].index;
+      if (!already) free_slots.push_back(ref[e].index);
+    }
+  }
+  if (static_cast<size_t>(slots) * N * sizeof(float) > kRowMaxSlotBytes) return COMFUSE_ERR_UNSUPPORTED;
+  P.terminal = ref[an.terminal];
+  P.n_row_out = static_cast<int>(an.row_outputs.size());
+  for (int r = 0; r < P.n_row_out; ++r) {
+    P.row_out_src[r] = ref[an.row_outputs[r]];
+    P.row_out_int[r] = an.nodes[an.row_outputs[r]].op == COMFUSE_OP_RED_ARGMAX && an.type[an.row_outputs[r]] == T_ROW;
+  }
+  P.n_instr = ni;
+  P.n_slots = slots;
+  n_instr = ni;
+  n_slots = slots;
+  return COMFUSE_OK;
+}
+
+comfuse_status_t validate_shape(const comfuse_gemm_shape_t* s) {
+  if (!s) return COMFUSE_ERR_INVALID_ARG;
+  if (s->batch < 1 || s->M < 1 || s->N < 1 || s->K < 1) return COMFUSE_ERR_INVALID_ARG;
+  if (s->lda < s->K || s->ldb < s->N || s->ldy < s->N) return COMFUSE_ERR_INVALID_ARG;
+  if ((s->N & 7) || (s->K & 7) || (s->lda & 7) || (s->ldb & 7) || (s->ldy & 7)) return COMFUSE_ERR_ALIGNMENT;
+  if (s->batch > 1) {
+    if (s->batch_stride_a < static_cast<long long>(s->M - 1) * s->lda + s->K) return COMFUSE_ERR_INVALID_ARG;
+    if (s->batch_stride_b < static_cast<long long>(s->K - 1) * s->ldb + s->N) return COMFUSE_ERR_INVALID_ARG;
+    if (s->batch_stride_y < static_cast<long long>(s->M - 1) * s->ldy + s->N) return COMFUSE_ERR_INVALID_ARG;
+    if ((s->batch_stride_a & 7) || (s->batch_stride_b & 7) || (s->batch_stride_y & 7)) return COMFUSE_ERR_ALIGNMENT;
+  }
+  return COMFUSE_OK;
+}
+
+// The descriptor of the fused instantiation a matched program lowers to.
+comfuse_gemm_desc_t fused_desc(const comfuse_gemm_shape_t& s, const FusedMatch& m, long long ldr) {
+  comfuse_gemm_desc_t d;
+  std::memset(&d, 0, sizeof(d));
+  d.batch = s.batch; d.M = s.M; d.N = s.N; d.K = s.K;
+  d.lda = s.lda; d.ldb = s.ldb; d.ldy = s.ldy; d.ldr = ldr;
+  d.batch_stride_a = s.batch_stride_a; d.batch_stride_b = s.batch_stride_b; d.batch_stride_y = s.batch_stride_y;
+  d.batch_stride_r = static_cast<long long>(s.M) * ldr;
+  d.kind = m.kind;
+  d.mask = m.causal ? COMFUSE_MASK_CAUSAL : COMFUSE_MASK_NONE;
+  d.alpha = m.alpha; d.eps = m.eps; d.fused = 1; d.flags = m.flags; d.softcap = m.softcap;
+  return d;
+}
+
+struct Decision {
+  Analysis an;
+  FusedMatch match;
+  bool fused = false;
+  size_t fused_inner_ws = 0;  // what the fused entry point itself needs
+  size_t fused_scratch = 0;   // row max / arg max the caller did not ask for
+};
+
+comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int want_fused, Decision& dc) {
+  comfuse_status_t s = validate_shape(shape);
+  if (s != COMFUSE_OK) return s;
+  s = analyse(spec, dc.an);
+  if (s != COMFUSE_OK) return s;
+  if (want_fused && match_fused(dc.an, dc.match)) {
+    const comfuse_gemm_desc_t d = fused_desc(*shape, dc.match, shape->N);
+    size_t ws = 0;
+    if (comfuse_workspace_size(&d, &ws) == COMFUSE_OK) {
+      dc.fused = true;
+      dc.fused_inner_ws = (ws + 255) & ~static_cast<size_t>(255);
+      if (dc.match.kind == COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX && (dc.match.row_max_out < 0 || dc.match.row_argmax_out < 0))
+        dc.fused_scratch = 2 * static_cast<size_t>(shape->batch) * shape->M * 4;
+    }
+  }
+  return COMFUSE_OK;
+}
+
+}  // namespace
+}  // namespace comfuse
+
+using namespace comfuse;
+
+extern "C" {
+
+comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, comfuse_spec_plan_t* plan) {
+  if (!plan) return COMFUSE_ERR_INVALID_ARG;
+  Decision dc;
+  comfuse_status_t s = decide(spec, shape, 1, dc);
+  if (s != COMFUSE_OK) return s;
+  std::memset(plan, 0, sizeof(*plan));
+  plan->n_stages = dc.an.n_stages;
+  plan->n_reductions = dc.an.n_reductions;
+  plan->n_live_nodes = dc.an.n_live;
+  plan->fused_kind = -1;
+  if (dc.fused) {
+    plan->path = COMFUSE_SPEC_PATH_FUSED_KERNEL;
+    plan->fused_kind = dc.match.kind;
+    plan->fused_flags = dc.match.flags;
+    plan->alpha = dc.match.alpha; plan->eps = dc.match.eps; plan->softcap = dc.match.softcap;
+    plan->causal = dc.match.causal;
+    return COMFUSE_OK;
+  }
+  plan->path = COMFUSE_SPEC_PATH_ROW_PROGRAM;
+  RowProgram P;
+  std::memset(&P, 0, sizeof(P));
+  return lower_row_program(dc.an, shape->N, P, plan->n_instructions, plan->n_slots);
+}
+
+comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused,
+                                                  size_t* bytes) {
+  if (!bytes || (fused != 0 && fused != 1)) return COMFUSE_ERR_INVALID_ARG;
+  Decision dc;
+  comfuse_status_t s = decide(spec, shape, fused, dc);
+  if (s != COMFUSE_OK) return s;
+  if (dc.fused) {
+    *bytes = dc.fused_inner_ws + dc.fused_scratch;
+    return COMFUSE_OK;
+  }
+  RowProgram P;
+  std::memset(&P, 0, sizeof(P));
+  int ni, ns;
+  s = lower_row_program(dc.an, shape->N, P, ni, ns);
+  if (s != COMFUSE_OK) return s;
+  *bytes = static_cast<size_t>(shape->batch) * shape->M * shape->N * 2;
+  return COMFUSE_OK;
+}
+
+comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A, const void* B,
+                                   void* Y, const void* const* params, const int64_t* param_ld, void* const* row_out, int32_t fused,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (fused != 0 && fused != 1) return COMFUSE_ERR_INVALID_ARG;
+  Decision dc;
+  comfuse_status_t s = decide(spec, shape, fused, dc);
+  if (s != COMFUSE_OK) return s;
+  if (!A || !B || !Y) return COMFUSE_ERR_INVALID_ARG;
+  const Analysis& an = dc.an;
+  // the parameter table: every slot a live node reads must be there, aligned, with a usable leading dimension
+  long long ld[COMFUSE_SPEC_MAX_PARAMS] = {0};
+  for (int k = 0; k < an.n; ++k) {
+    if (!an.live[k]) continue;
+    const int op = an.nodes[k].op;
+    if (op != COMFUSE_OP_ROWVEC && op != COMFUSE_OP_TENSOR) continue;
+    const int q = an.nodes[k].param;
+    if (!params || !params[q]) return COMFUSE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(params[q]) & 15u) return COMFUSE_ERR_ALIGNMENT;
+    if (op == COMFUSE_OP_TENSOR) {
+      ld[q] = (param_ld && param_ld[q] > 0) ? param_ld[q] : shape->N;
+      if (ld[q] < shape->N) return COMFUSE_ERR_INVALID_ARG;
+      if (ld[q] & 7) return COMFUSE_ERR_ALIGNMENT;
+    }
+  }
+  for (size_t r = 0; r < an.row_outputs.size(); ++r)
+    if (!row_out || !row_out[r]) return COMFUSE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(Y)) & 15u) return COMFUSE_ERR_ALIGNMENT;
+  size_t need = 0;
+  s = comfuse_gemm_spec_workspace_size(spec, shape, fused, &need);
+  if (s != COMFUSE_OK) return s;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return COMFUSE_ERR_WORKSPACE;
+  if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return COMFUSE_ERR_ALIGNMENT;
+
+  if (dc.fused) {
+    const FusedMatch& m = dc.match;
+    const comfuse_gemm_desc_t d = fused_desc(*shape, m, m.residual >= 0 ? ld[m.residual] : shape->N);
+    comfuse_epilogue_args_t a;
+    std::memset(&a, 0, sizeof(a));
+    auto prm = [&](int q) { return q >= 0 ? params[q] : nullptr; };
+    a.bias = prm(m.bias); a.residual = prm(m.residual); a.gamma = prm(m.gamma); a.beta = prm(m.beta);
+    if (m.kind == COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX) {
+      char* scratch = static_cast<char*>(workspace) + dc.fused_inner_ws;
+      const size_t rows = static_cast<size_t>(shape->batch) * shape->M;
+      a.row_max = m.row_max_out >= 0 ? static_cast<float*>(row_out[m.row_max_out]) : reinterpret_cast<float*>(scratch);
+      a.row_argmax = m.row_argmax_out >= 0 ? static_cast<int32_t*>(row_out[m.row_argmax_out]) : reinterpret_cast<int32_t*>(scratch + rows * 4);
+    }
+    return comfuse_gemm_epilogue(&d, A, B, Y, &a, workspace, dc.fused_inner_ws, cuda_stream);
+  }
+
+  // standard pathway: GEMM -> bf16 Z in the workspace -> row program
+  RowProgram P;
+  std::memset(&P, 0, sizeof(P));
+  int ni, ns;
+  s = lower_row_program(an, shape->N, P, ni, ns);
+  if (s != COMFUSE_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  s = gemm_to_bf16(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->batch_stride_a, shape->batch_stride_b, A, B,
+                   workspace, st);
+  if (s != COMFUSE_OK) return s;
+  P.batch = shape->batch; P.M = shape->M; P.N = shape->N;
+  P.Z = static_cast<const uint16_t*>(workspace);
+  P.Y = static_cast<uint16_t*>(Y);
+  P.ldy = shape->ldy;
+  P.batch_stride_y = shape->batch > 1 ? shape->batch_stride_y : 0;
+  for (int q = 0; q < spec->n_params; ++q) {
+    P.params[q] = params ? static_cast<const uint16_t*>(params[q]) : nullptr;
+    P.param_ld[q] = ld[q];
+  }
+  for (int r = 0; r < P.n_row_out; ++r) P.row_out[r] = row_out[r];
+  return launch_row_program(P, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -56,3 +56,12 @@ cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_
 cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 
 }  // namespace comfuse
+
+#include "comfuse.h"
+
+namespace comfuse {
+// Z = bf16(A . B), dense [batch, M, N] (ld = N), with the plain tensor-core GEMM kernel; arguments already validated.
+comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
+                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st);
+
+}  // namespace comfuse

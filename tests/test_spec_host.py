@@ -1,0 +1,130 @@
+"""Host-side analysis of epilogue programs (no GPU): validation, typing, stage numbering at the reductions (Sec. 5.3),
+canonicalisation onto the fused instantiations in any operand order (Sec. 5.4), liveness-based buffer assignment of
+the row program."""
+import pytest
+
+import paper_2608_03537_b200 as cf
+import workloads as wl
+
+SHAPE = cf.make_gemm_shape(1, 512, 1024, 256)
+
+
+def _plan(nodes, terminal, n_params=0, row_outputs=(), shape=SHAPE):
+    return cf.spec_plan(cf.make_spec(nodes, terminal, n_params, row_outputs), shape)
+
+
+def _status(nodes, terminal, n_params=0, row_outputs=(), shape=SHAPE):
+    with pytest.raises(cf.ComfuseError) as e:
+        _plan(nodes, terminal, n_params, row_outputs, shape)
+    return e.value.status
+
+
+N_ = ("acc", -1, -1, -1, 0.0)
+
+
+def test_stage_numbering_follows_the_reductions():
+    assert _plan([N_], 0).n_stages == 1
+    assert _plan([N_, ("relu", 0, -1, -1, 0)], 1).n_stages == 1
+    p = wl.spec_layernorm()
+    assert _plan(p.nodes, p.terminal, 4).n_stages == 3          # x | x - mean | normalise
+    p = wl.spec_softmax(0.5)
+    assert _plan(p.nodes, p.terminal).n_stages == 3             # max | sum of exp | scale
+    p = wl.spec_rmsnorm_max()
+    pl = _plan(p.nodes, p.terminal, 3, p.row_outputs)
+    assert pl.n_stages == 3 and pl.n_reductions == 3            # mean square | max and arg max of Y (same stage)
+    p = wl.spec_gated_minmax()
+    pl = _plan(p.nodes, p.terminal, 1, p.row_outputs)
+    assert pl.n_stages == 2 and pl.n_reductions == 3            # three independent reductions share one boundary
+
+
+def test_dead_nodes_are_not_counted():
+    nodes = [N_, ("exp", 0, -1, -1, 0), ("sum", 1, -1, -1, 0), ("relu", 0, -1, -1, 0)]
+    pl = _plan(nodes, 3)
+    assert pl.n_live_nodes == 2 and pl.n_reductions == 0 and pl.n_stages == 1 and pl.n_instructions == 1
+
+
+def test_constants_are_folded_on_the_host():
+    # y = acc * (1 / sqrt(4))  ->  one instruction, no per-row arithmetic
+    nodes = [N_, ("const", -1, -1, -1, 4.0), ("rsqrt", 1, -1, -1, 0), ("mul", 0, 2, -1, 0)]
+    pl = _plan(nodes, 3)
+    assert pl.n_instructions == 1 and pl.n_slots == 1
+
+
+@pytest.mark.parametrize("prog,n_params,kind,flags", [
+    (wl.spec_layernorm(), 4, cf.EPI_BIAS_RES_LAYERNORM, 0),
+    (wl.spec_layernorm(relu=True, residual=False), 3, cf.EPI_BIAS_RES_LAYERNORM, cf.FLAG_POST_RELU),
+    (wl.spec_layernorm(bias=False, residual=False, affine=False), 0, cf.EPI_BIAS_RES_LAYERNORM, 0),
+    (wl.spec_rmsnorm_max(), 3, cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, 0),
+    (wl.spec_rmsnorm_max(activation=False, residual=False), 2, cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, cf.FLAG_NO_ACTIVATION),
+    (wl.spec_softmax(0.125), 0, cf.EPI_SCALE_MASK_SOFTMAX, 0),
+])
+def test_primitive_spellings_lower_to_the_fused_kernels(prog, n_params, kind, flags):
+    pl = _plan(prog.nodes, prog.terminal, n_params, prog.row_outputs)
+    assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.fused_kind == kind and pl.fused_flags == flags
+
+
+def _swap_commutative(nodes):
+    return [(op, b, a, p, i) if op in ("add", "mul") else (op, a, b, p, i) for (op, a, b, p, i) in nodes]
+
+
+@pytest.mark.parametrize("prog,n_params", [(wl.spec_layernorm(relu=True), 4), (wl.spec_rmsnorm_max(), 3), (wl.spec_softmax(0.3, False, 5.0), 0)])
+def test_operand_order_of_commutative_nodes_does_not_matter(prog, n_params):
+    a = _plan(prog.nodes, prog.terminal, n_params, prog.row_outputs)
+    b = _plan(_swap_commutative(prog.nodes), prog.terminal, n_params, prog.row_outputs)
+    assert a.path == b.path == cf.SPEC_PATH_FUSED_KERNEL and a.fused_kind == b.fused_kind and a.fused_flags == b.fused_flags
+
+
+def test_recovered_constants():
+    p = wl.spec_softmax(alpha=0.125, causal=True, softcap=30.0)
+    pl = _plan(p.nodes, p.terminal, shape=cf.make_gemm_shape(4, 1024, 1024, 64))
+    assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.causal == 1
+    assert pl.alpha == pytest.approx(0.125) and pl.softcap == pytest.approx(30.0)
+    p = wl.spec_layernorm(eps=3e-4)
+    assert _plan(p.nodes, p.terminal, 4).eps == pytest.approx(3e-4)
+
+
+def test_near_misses_take_the_row_program():
+    # residual added INSIDE the activation: not the compiled RMSNorm entry
+    g = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("tensor", -1, -1, 1, 0), ("add", 2, 3, -1, 0), ("gelu_tanh", 4, -1, -1, 0),
+         ("square", 5, -1, -1, 0), ("mean", 6, -1, -1, 0), ("const", -1, -1, -1, 1e-5), ("add", 7, 8, -1, 0), ("rsqrt", 9, -1, -1, 0),
+         ("mul", 5, 10, -1, 0)]
+    assert _plan(g, 11, 2).path == cf.SPEC_PATH_ROW_PROGRAM
+    # soft-cap whose two constants are not reciprocal
+    p = wl.spec_softmax(0.5, False, 2.0)
+    nodes = [(op, a, b, q, 0.7 if (op == "const" and abs(i - 0.5) < 1e-9 and k > 1) else i) for k, (op, a, b, q, i) in enumerate(p.nodes)]
+    assert _plan(nodes, p.terminal).path == cf.SPEC_PATH_ROW_PROGRAM
+    # LayerNorm with an extra row output
+    p = wl.spec_layernorm()
+    assert _plan(p.nodes, p.terminal, 4, (p.nodes.index(("mean", 4, -1, -1, 0.0)),)).path == cf.SPEC_PATH_ROW_PROGRAM
+    # causal softmax on a non-square problem: no fused instantiation
+    p = wl.spec_softmax(0.5, True)
+    assert _plan(p.nodes, p.terminal, shape=cf.make_gemm_shape(1, 256, 512, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
+    # a fused pattern on a row length without an instantiation
+    p = wl.spec_layernorm()
+    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
+
+
+def test_row_program_reuses_buffers_by_liveness():
+    p = wl.spec_layernorm(relu=True)
+    spec = cf.make_spec(p.nodes, p.terminal, 4)
+    # forced row program: x, x - mean and its square are the only tensors alive together
+    assert cf.gemm_spec_workspace_size(spec, SHAPE, fused=False) == 512 * 1024 * 2
+    chain = [N_] + [("relu", k, -1, -1, 0) for k in range(20)]
+    pl = _plan(chain, 20)
+    assert pl.n_instructions == 20 and pl.n_slots == 1           # a chain runs in place
+    p = wl.spec_gated_minmax()
+    assert _plan(p.nodes, p.terminal, 1, p.row_outputs).n_slots == 2
+
+
+def test_malformed_programs_are_rejected():
+    INV = cf.ERR_INVALID_ARG
+    assert _status([N_, ("add", 0, 2, -1, 0), ("const", -1, -1, -1, 1.0)], 1) == INV          # forward edge
+    assert _status([N_, ("add", 0, -1, -1, 0)], 1) == INV                                      # missing operand
+    assert _status([N_, (99, 0, -1, -1, 0)], 1) == INV                                         # outside the vocabulary
+    assert _status([N_, ("relu", 0, 0, -1, 0)], 1) == INV                                      # unary with two inputs
+    assert _status([N_, ("rowvec", -1, -1, 0, 0)], 1, n_params=0) == INV                       # parameter slot out of range
+    assert _status([N_, ("rowvec", -1, -1, 0, 0), ("tensor", -1, -1, 0, 0), ("add", 1, 2, -1, 0)], 3, n_params=1) == INV  # one slot, two shapes
+    assert _status([N_], 1) == INV                                                             # terminal out of range
+    assert _status([N_, ("relu", 0, -1, -1, 0)], 1, row_outputs=(1,)) == INV                   # row output must be per-row
+    assert _status([N_], 0, shape=cf.make_gemm_shape(1, 64, 100, 64)) == cf.ERR_ALIGNMENT      # N not a multiple of 8
+    assert _status([("acc", 0, -1, -1, 0)], 0) == INV                                          # entry node with an input
