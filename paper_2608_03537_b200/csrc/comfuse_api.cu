@@ -57,6 +57,15 @@ bool mult8(long long v) { return (v & 7) == 0; }
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+// COMFUSE_REDUCE_MODE=leader selects leader-follower aggregation of the row statistics, anything else all-to-all.
+bool leader_reduce_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("COMFUSE_REDUCE_MODE");
+    return e && std::strcmp(e, "leader") == 0;
+  }();
+  return on;
+}
+
 bool programmatic_launch_enabled() {
   static const bool on = [] {
     const char* e = std::getenv("COMFUSE_PDL");
@@ -298,6 +307,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.softcap = desc->softcap;
   p.status = dev->status_word;
   p.timeout_ns = timeout_ns();
+  p.leader_reduce = leader_reduce_enabled() ? 1 : 0;
 #ifdef COMFUSE_TRACE
   // tracing build: COMFUSE_TRACE_PTR holds the device address of a uint64[64] buffer for phase timestamps
   if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) p.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));

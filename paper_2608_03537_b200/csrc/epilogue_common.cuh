@@ -46,7 +46,7 @@ template <int CN, class Merge, int NH = 2>
 __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thread_count, Merge merge, float2* s_pre,
                                                      float2* s_stats, uint32_t stats_bar, int row, int h,
                                                      uint32_t rank, int& xpar, uint32_t& xphase, const WaitCtx& w,
-                                                     uint32_t rank_stride = 1, uint32_t rank_offset = 0) {
+                                                     uint32_t rank_stride = 1, uint32_t rank_offset = 0, bool leader_mode = false) {
   // level 2: the NH threads that share the row (one per epilogue warp of the lane quarter), through shared memory
   s_pre[(xpar * NH + h) * 128 + row] = mine;
   named_barrier_sync(1, 128 * NH);
@@ -70,16 +70,49 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
   } else {
     // each partial travels as an asynchronous 8-byte store that is counted on the destination's barrier; one local
     // thread arms the barrier with the byte count of the whole exchange (CN peers x 128 rows x 8 bytes)
-    if (h == 0 && row == 0) mbar_arrive_expect_tx(bar, CN * 128 * 8);
     const uint32_t slot_addr = smem_u32(slot);
+    if (!leader_mode) {
+      if (h == 0 && row == 0) mbar_arrive_expect_tx(bar, CN * 128 * 8);
 #pragma unroll
-    for (int dst = 0; dst < CN; ++dst) {
-      if ((dst % NH) == h) {
-        const uint32_t peer = dst * rank_stride + rank_offset;
-        st_async_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y, map_to_cta(bar, peer));
+      for (int dst = 0; dst < CN; ++dst) {
+        if ((dst % NH) == h) {
+          const uint32_t peer = dst * rank_stride + rank_offset;
+          st_async_f32x2(map_to_cta(slot_addr, peer), cta_partial.x, cta_partial.y, map_to_cta(bar, peer));
+        }
       }
+      mbar_wait<true>(bar, phase, w);
+    } else {
+      // leader-follower aggregation (Sec. 3.1, the mode for large CN): every CTA sends its partial to column range 0
+      // only (CN messages per row instead of CN^2); that CTA merges in the same rank order and sends the result back.
+      // The followers' barrier counts the one returning message, the leader's the CN partials.
+      const uint32_t lead = rank_offset;
+      if (h == 0 && row == 0) mbar_arrive_expect_tx(bar, (rank == 0 ? CN : 1) * 128 * 8);
+      if (h == 0) st_async_f32x2(map_to_cta(slot_addr, lead), cta_partial.x, cta_partial.y, map_to_cta(bar, lead));
+      mbar_wait<true>(bar, phase, w);
+      if (rank == 0) {
+        float2 acc = s_stats[(xpar * CN + 0) * 128 + row];
+#pragma unroll
+        for (int c = 1; c < CN; ++c) acc = merge(acc, cta_count * c, s_stats[(xpar * CN + c) * 128 + row], cta_count);
+        // slot 0 of every follower receives the merged value (thread h serves the followers congruent to h mod NH)
+        const uint32_t res_addr = smem_u32(s_stats + (xpar * CN + 0) * 128 + row);
+#pragma unroll
+        for (int dst = 1; dst < CN; ++dst) {
+          if ((dst % NH) == h) {
+            const uint32_t peer = dst * rank_stride + rank_offset;
+            st_async_f32x2(map_to_cta(res_addr, peer), acc.x, acc.y, map_to_cta(bar, peer));
+          }
+        }
+        xphase ^= 1u << xpar;
+        xpar ^= 1;
+        __syncwarp();
+        return acc;
+      }
+      const float2 acc = s_stats[(xpar * CN + 0) * 128 + row];
+      xphase ^= 1u << xpar;
+      xpar ^= 1;
+      __syncwarp();
+      return acc;
     }
-    mbar_wait<true>(bar, phase, w);
   }
   float2 acc = s_stats[(xpar * CN + 0) * 128 + row];
 #pragma unroll

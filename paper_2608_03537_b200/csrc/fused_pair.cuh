@@ -654,10 +654,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         float2 tot;
         if constexpr (EPI == EPI_LN) {
           tot = cluster_row_reduce<CN, MergeWelford, EPW>(part, kThreadCount, MergeWelford(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w,
-                                       2u, pm);
+                                       2u, pm, p.leader_reduce != 0);
         } else {
           tot = cluster_row_reduce<CN, MergeSum, EPW>(part, kThreadCount, MergeSum(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u,
-                                       pm);
+                                       pm, p.leader_reduce != 0);
         }
         COMFUSE_TRACE_POINT();
         // wide rows: the statistic covers this column block only; store x as it is (gamma = 1, beta = 0 were loaded) and
@@ -726,7 +726,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (kIsRms && !p.wide) {
           // ---------------- stage 3: the second, chained reduction reuses the exchange buffers (Sec. 3.2)
           const float2 mx = cluster_row_reduce<CN, MergeArgmax, EPW>(make_float2(best, __int_as_float(best_col)), kThreadCount, MergeArgmax(), s_pre,
-                                                   s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
+                                                   s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm, p.leader_reduce != 0);
           if (crank == 0 && h == 0 && valid) {
             const long long o = static_cast<long long>(b) * p.M + grow;
             p.row_max[o] = mx.x;
@@ -819,7 +819,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tmem_st_wait();
         COMFUSE_TRACE_POINT();
         const float2 tot = cluster_row_reduce<CN, MergeMaxSumExp2, EPW>(make_float2(mloc, lloc), kThreadCount, MergeMaxSumExp2(), s_pre, s_stats,
-                                                  bar_stats, row, h, crank, xpar, xphase, w, 2u, pm);
+                                                  bar_stats, row, h, crank, xpar, xphase, w, 2u, pm, p.leader_reduce != 0);
         const float f = (mloc == -INFINITY || tot.y == 0.f) ? 0.f : ex2_approx(mloc - tot.x) / tot.y;
         COMFUSE_TRACE_POINT();
         // ---------------- pass C: scale, round once, store (zeros where masked)

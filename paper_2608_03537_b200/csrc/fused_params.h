@@ -34,6 +34,10 @@ struct FusedParams {
   // wide_partials[(batch * M + row) * nblocks + block]; a second kernel merges the partials and rescales in place.
   int wide;
   float2* wide_partials;
+  // Cross-CTA aggregation of the row statistics (Sec. 3.1): 0 = all-to-all (every CTA sends its partial to every peer),
+  // 1 = leader-follower (partials go to column range 0, which merges and sends the result back).  Same merge order,
+  // hence the same bits, either way.
+  int leader_reduce;
   unsigned int* status;
   unsigned long long timeout_ns;
   unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null

@@ -24,6 +24,8 @@ void count_launch();
 // Kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail; they
 // wait for that kernel before touching global memory) unless COMFUSE_PDL=0.
 bool programmatic_launch_enabled();
+// Cross-CTA aggregation mode of the row statistics: COMFUSE_REDUCE_MODE=leader, default all-to-all.
+bool leader_reduce_enabled();
 
 // Encode a 3-D bf16 tiled tensor map with 128-byte swizzle: dims/strides innermost first; strides in BYTES for
 // dims 1 and 2; box = {64, box_rows, 1}.
