@@ -36,6 +36,7 @@ BROADCAST_OPS = ("const", "rowvec", "tensor", "causal_mask")
 UNARY_OPS = ("neg", "abs", "square", "sqrt", "rsqrt", "recip", "exp", "log", "tanh", "relu", "gelu_tanh", "sigmoid")
 BINARY_OPS = ("add", "sub", "mul", "div", "max", "min")
 REDUCE_OPS = ("sum", "mean", "rmax", "rmin", "prod", "argmax")
+TOPK_OPS = ("topk_values", "topk_indices")  # K is the node's ``param``; the value is [M, K] and can only be a row output
 
 
 def _unary(op: str, a: np.ndarray) -> np.ndarray:
@@ -138,6 +139,10 @@ def eval_nodes(nodes, Z: np.ndarray, params=(), row0: int = 0):
             if a.shape[0] != M:
                 a = np.broadcast_to(a, (M, N))
             v = _reduce(op, a, N)
+        elif op in TOPK_OPS:
+            a = np.broadcast_to(np.asarray(vals[in0]), (M, N))
+            tv, ti = topk_rows(a, param)
+            v = tv if op == "topk_values" else ti.astype(np.float64)
         else:
             raise ValueError(f"node {k}: unknown op {op!r}")
         vals.append(v)
@@ -146,12 +151,17 @@ def eval_nodes(nodes, Z: np.ndarray, params=(), row0: int = 0):
 
 def gemm_spec(A, B, nodes, terminal: int, params=(), row_outputs=()):
     """Y = value of node ``terminal`` of the program evaluated on Z = A B, as [M, N]; plus the per-row values of the
-    nodes listed in ``row_outputs`` (each [M])  (Sec. 5.2: terminal node, parameter table; Sec. 3: Y = epilogue(A B))."""
+    nodes listed in ``row_outputs`` (each [M]; [M, K] for a Top-K node)  (Sec. 5.2: terminal node, parameter table; Sec. 3: Y = epilogue(A B))."""
     Z = np.matmul(np.asarray(A, dtype=np.float64), np.asarray(B, dtype=np.float64))
     M, N = Z.shape
     vals = eval_nodes(nodes, Z, params)
     Y = np.broadcast_to(np.asarray(vals[terminal], dtype=np.float64), (M, N)).copy()
-    rows = [np.broadcast_to(np.asarray(vals[r], dtype=np.float64), (M, 1))[:, 0].copy() for r in row_outputs]
+    rows = []
+    for r in row_outputs:
+        if nodes[r][0] in TOPK_OPS:
+            rows.append(np.asarray(vals[r], dtype=np.float64).copy())  # [M, K]
+        else:
+            rows.append(np.broadcast_to(np.asarray(vals[r], dtype=np.float64), (M, 1))[:, 0].copy())
     return Y, rows
 
 

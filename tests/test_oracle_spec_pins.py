@@ -107,6 +107,25 @@ def test_topk_rows_hand_computed_with_ties():
     np.testing.assert_array_equal(c, [[1, 2, 0], [0, 2, 3]])
 
 
+def test_topk_nodes_hand_computed_through_the_program_evaluator():
+    # top-2 of relu(z): rows [0 5 0 5 1] -> (5, 5) at columns (1, 3); [2 0 0 0 3] -> (3, 2) at (4, 0)
+    Z = np.array([[-1.0, 5.0, -3.0, 5.0, 1.0], [2.0, -7.0, -7.0, -1.0, 3.0]])
+    nodes = [("acc", -1, -1, -1, 0.0), ("relu", 0, -1, -1, 0.0), ("topk_values", 1, -1, 2, 0.0), ("topk_indices", 1, -1, 2, 0.0)]
+    Y, (tv, ti) = spo.gemm_spec(np.eye(2), Z, nodes, 1, (), (2, 3))
+    np.testing.assert_array_equal(Y, np.maximum(Z, 0.0))
+    np.testing.assert_array_equal(tv, [[5.0, 5.0], [3.0, 2.0]])
+    np.testing.assert_array_equal(ti, [[1, 3], [4, 0]])
+
+
+def test_topk_agrees_with_the_library_sort_on_distinct_values():
+    g = _rng(21)
+    Yv = g.permutation(200).astype(np.float64).reshape(4, 50)  # all distinct: no tie rule involved
+    v, c = spo.topk_rows(Yv, 7)
+    tv, tc = torch.topk(torch.from_numpy(Yv), 7, dim=1)
+    np.testing.assert_array_equal(v, tv.numpy())
+    np.testing.assert_array_equal(c, tc.numpy())
+
+
 def test_row_scalar_and_constant_operands_broadcast():
     # y = (z - min z) / 2 + 1, per-row value fed back into an element-wise node, constants on either side
     Z = np.array([[1.0, 5.0, 3.0], [-2.0, -6.0, 0.0]])
