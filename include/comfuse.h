@@ -239,13 +239,17 @@ typedef enum {
   /* reductions of in0 over the row (ReduceOp sum / prod / max / min and ReduceMode mean of the StreamReduction
    * node, Sec. 5); ARGMAX = lowest column attaining the row maximum, as a number */
   COMFUSE_OP_RED_SUM = 48, COMFUSE_OP_RED_MEAN = 49, COMFUSE_OP_RED_MAX = 50, COMFUSE_OP_RED_MIN = 51,
-  COMFUSE_OP_RED_PROD = 52, COMFUSE_OP_RED_ARGMAX = 53
+  COMFUSE_OP_RED_PROD = 52, COMFUSE_OP_RED_ARGMAX = 53,
+  /* Top-K reduction (the StreamReduction node's hyper-parameter K, Sec. 5): `param` = K (1 .. 64, <= N).  The K largest
+   * values of in0 per row in falling order, equal values in rising column order (VALUES), and their columns (INDICES).
+   * K values per row: such a node can only be a row output (fp32 resp. int32 [batch*M, K]), not an input. */
+  COMFUSE_OP_RED_TOPK_VALUES = 54, COMFUSE_OP_RED_TOPK_INDICES = 55
 } comfuse_op_t;
 
 typedef struct {
   int32_t op;        /* comfuse_op_t */
   int32_t in0, in1;  /* indices of earlier nodes, -1 where the op takes no such input */
-  int32_t param;     /* ROWVEC / TENSOR: index into the parameter table, else -1 */
+  int32_t param;     /* ROWVEC / TENSOR: index into the parameter table; RED_TOPK_*: K; else -1 */
   float imm;         /* CONST: the value */
 } comfuse_spec_node_t;
 
@@ -260,7 +264,8 @@ typedef struct {
   int32_t n_params;                  /* entries of the parameter table, 0 .. COMFUSE_SPEC_MAX_PARAMS */
   int32_t n_row_outputs;             /* 0 .. COMFUSE_SPEC_MAX_ROW_OUTPUTS */
   const int32_t* row_outputs;        /* HOST array of per-row valued nodes; output k is written to row_out[k]:
-                                        fp32 [batch*M], or int32 [batch*M] when the node is a RED_ARGMAX */
+                                        fp32 [batch*M], or int32 [batch*M] when the node is a RED_ARGMAX;
+                                        [batch*M, K] for the RED_TOPK_* nodes */
 } comfuse_fusion_spec_t;
 
 typedef struct {

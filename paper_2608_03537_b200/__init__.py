@@ -82,7 +82,7 @@ OPS = {
     "neg": 16, "abs": 17, "square": 18, "sqrt": 19, "rsqrt": 20, "recip": 21, "exp": 22, "log": 23, "tanh": 24,
     "relu": 25, "gelu_tanh": 26, "sigmoid": 27,
     "add": 32, "sub": 33, "mul": 34, "div": 35, "max": 36, "min": 37,
-    "sum": 48, "mean": 49, "rmax": 50, "rmin": 51, "prod": 52, "argmax": 53,
+    "sum": 48, "mean": 49, "rmax": 50, "rmin": 51, "prod": 52, "argmax": 53, "topk_values": 54, "topk_indices": 55,
 }
 SPEC_PATH_FUSED_KERNEL = 0
 SPEC_PATH_ROW_PROGRAM = 1

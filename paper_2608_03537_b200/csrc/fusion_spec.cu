@@ -24,7 +24,8 @@ enum NodeType : uint8_t { T_TENSOR = 0, T_ROW = 1, T_CONST = 2 };
 
 bool is_unary(int op) { return op >= COMFUSE_OP_NEG && op <= COMFUSE_OP_SIGMOID; }
 bool is_binary(int op) { return op >= COMFUSE_OP_ADD && op <= COMFUSE_OP_MIN; }
-bool is_reduce(int op) { return op >= COMFUSE_OP_RED_SUM && op <= COMFUSE_OP_RED_ARGMAX; }
+bool is_reduce(int op) { return op >= COMFUSE_OP_RED_SUM && op <= COMFUSE_OP_RED_TOPK_INDICES; }
+bool is_topk(int op) { return op == COMFUSE_OP_RED_TOPK_VALUES || op == COMFUSE_OP_RED_TOPK_INDICES; }
 bool is_leaf(int op) { return op >= COMFUSE_OP_ACC && op <= COMFUSE_OP_CAUSAL_MASK; }
 
 float fold_unary(int op, float a) {
@@ -77,6 +78,7 @@ comfuse_status_t analyse(const comfuse_fusion_spec_t* spec, Analysis& an) {
   if (spec->n_row_outputs < 0 || spec->n_row_outputs > COMFUSE_SPEC_MAX_ROW_OUTPUTS) return COMFUSE_ERR_INVALID_ARG;
   if (spec->n_row_outputs > 0 && !spec->row_outputs) return COMFUSE_ERR_INVALID_ARG;
   if (spec->terminal < 0 || spec->terminal >= spec->n_nodes) return COMFUSE_ERR_INVALID_ARG;
+  if (is_topk(spec->nodes[spec->terminal].op)) return COMFUSE_ERR_INVALID_ARG;
   const int n = spec->n_nodes;
   an.n = n;
   an.nodes.assign(spec->nodes, spec->nodes + n);
@@ -104,7 +106,9 @@ comfuse_status_t analyse(const comfuse_fusion_spec_t* spec, Analysis& an) {
         an.cval[k] = nd.imm;
       }
     } else if (is_unary(op) || is_reduce(op)) {
-      if (!edge_ok(nd.in0) || nd.in1 != -1 || nd.param != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (!edge_ok(nd.in0) || nd.in1 != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (is_topk(op) ? (nd.param < 1 || nd.param > 64) : nd.param != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (is_topk(an.nodes[nd.in0].op)) return COMFUSE_ERR_INVALID_ARG;  // K values per row: a row output only
       if (is_reduce(op)) {
         an.type[k] = T_ROW;
         an.stage[k] = an.stage[nd.in0] + 1;
@@ -115,6 +119,7 @@ comfuse_status_t analyse(const comfuse_fusion_spec_t* spec, Analysis& an) {
       }
     } else if (is_binary(op)) {
       if (!edge_ok(nd.in0) || !edge_ok(nd.in1) || nd.param != -1) return COMFUSE_ERR_INVALID_ARG;
+      if (is_topk(an.nodes[nd.in0].op) || is_topk(an.nodes[nd.in1].op)) return COMFUSE_ERR_INVALID_ARG;
       const uint8_t ta = an.type[nd.in0], tb = an.type[nd.in1];
       an.type[k] = (ta == T_TENSOR || tb == T_TENSOR) ? T_TENSOR : (ta == T_ROW || tb == T_ROW) ? T_ROW : T_CONST;
       an.stage[k] = an.stage[nd.in0] > an.stage[nd.in1] ? an.stage[nd.in0] : an.stage[nd.in1];
@@ -388,7 +393,17 @@ comfuse_status_t lower_row_program(const Analysis& an, int N, RowProgram& P, int
     in.op = static_cast<uint8_t>(nd.op);
     in.a = ref[nd.in0];
     in.b = nd.in1 >= 0 ? ref[nd.in1] : Operand{OPK_NONE, 0, 0, 0.f};
-    if (an.type[k] == T_ROW) {
+    if (is_topk(nd.op)) {
+      // written straight to its row output, K values per row: dst = position in the row-output list, b.index = K
+      if (nd.param > N) return COMFUSE_ERR_INVALID_ARG;
+      int pos = -1;
+      for (size_t r = 0; r < an.row_outputs.size(); ++r)
+        if (an.row_outputs[r] == k) { pos = static_cast<int>(r); break; }
+      in.dst_scalar = 1;
+      in.dst = static_cast<int16_t>(pos);
+      in.b = Operand{OPK_NONE, 0, static_cast<int16_t>(nd.param), 0.f};
+      ref[k] = Operand{OPK_NONE, 0, 0, 0.f};
+    } else if (an.type[k] == T_ROW) {
       if (scalars >= kRowMaxScalars) return COMFUSE_ERR_UNSUPPORTED;
       in.dst_scalar = 1;
       in.dst = static_cast<int16_t>(scalars);

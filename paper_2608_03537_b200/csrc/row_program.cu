@@ -115,7 +115,41 @@ __global__ void __launch_bounds__(256) row_program_kernel(const __grid_constant_
   for (int k = 0; k < P.n_instr; ++k) {
     const RowInstr& in = P.ins[k];
     const int op = in.op;
-    if (op >= COMFUSE_OP_RED_SUM) {
+    if (op == COMFUSE_OP_RED_TOPK_VALUES || op == COMFUSE_OP_RED_TOPK_INDICES) {
+      // ---- Top-K: K rounds of a block arg max over the elements that rank after the previous pick in the order
+      // (value falling, column rising); round r's pick goes straight to the row output
+      const int K = in.b.index;
+      float last_v = CUDART_INF_F;
+      int last_i = -1;
+      for (int r = 0; r < K; ++r) {
+        float acc = -CUDART_INF_F;
+        int idx = 0x7FFFFFFF;
+        for (int j = tid; j < pairs; j += T) {
+          const float2 v = fetch(c, in.a, j);
+          const float e[2] = {v.x, v.y};
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int col = 2 * j + u;
+            const bool eligible = e[u] < last_v || (e[u] == last_v && col > last_i);
+            if (eligible && (e[u] > acc || (e[u] == acc && col < idx))) { acc = e[u]; idx = col; }
+          }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) argmax_merge(acc, idx, __shfl_xor_sync(0xFFFFFFFFu, acc, off), __shfl_xor_sync(0xFFFFFFFFu, idx, off));
+        if (lane == 0) { s_red[wid] = acc; s_redi[wid] = idx; }
+        __syncthreads();
+        float rv = s_red[0];
+        int ri = s_redi[0];
+        for (int w = 1; w < nwarps; ++w) argmax_merge(rv, ri, s_red[w], s_redi[w]);
+        __syncthreads();  // everyone has read the partials before the next round overwrites them
+        last_v = rv;
+        last_i = ri;
+        if (tid == 0 && in.dst >= 0) {
+          if (op == COMFUSE_OP_RED_TOPK_INDICES) static_cast<int*>(P.row_out[in.dst])[row_lin * K + r] = ri;
+          else static_cast<float*>(P.row_out[in.dst])[row_lin * K + r] = rv;
+        }
+      }
+    } else if (op >= COMFUSE_OP_RED_SUM) {
       // ---- stage boundary: block-wide reduction of operand a over the row
       const bool is_max = op == COMFUSE_OP_RED_MAX || op == COMFUSE_OP_RED_ARGMAX;
       float acc = op == COMFUSE_OP_RED_PROD ? 1.f : is_max ? -CUDART_INF_F : op == COMFUSE_OP_RED_MIN ? CUDART_INF_F : 0.f;
@@ -201,6 +235,7 @@ __global__ void __launch_bounds__(256) row_program_kernel(const __grid_constant_
   }
   if (tid == 0) {
     for (int r = 0; r < P.n_row_out; ++r) {
+      if (P.row_out_src[r].kind == OPK_NONE) continue;  // a Top-K node: already written
       const float v = scalar_of(c, P.row_out_src[r]);
       if (P.row_out_int[r]) static_cast<int*>(P.row_out[r])[row_lin] = static_cast<int>(v);
       else static_cast<float*>(P.row_out[r])[row_lin] = v;

@@ -142,3 +142,53 @@ def test_row_program_rejects_rows_that_do_not_fit_shared_memory():
     with pytest.raises(cf.ComfuseError) as e:
         cf.spec_plan(spec, cf.make_gemm_shape(1, 128, 65536, 64))
     assert e.value.status == cf.ERR_UNSUPPORTED
+
+
+def _topk_prog(k):
+    nodes = [("acc", -1, -1, -1, 0.0), ("rowvec", -1, -1, 0, 0.0), ("add", 0, 1, -1, 0.0), ("relu", 2, -1, -1, 0.0),
+             ("topk_values", 3, -1, k, 0.0), ("topk_indices", 3, -1, k, 0.0)]
+    return wl.SpecProgram(nodes, 3, (4, 5), ("rowvec",))
+
+
+def _run_topk(A, B, bias, k):
+    prog = _topk_prog(k)
+    M, N = A.shape[0], B.shape[1]
+    spec = cf.make_spec(prog.nodes, prog.terminal, 1, prog.row_outputs)
+    shape = cf.make_gemm_shape(1, M, N, A.shape[1])
+    dev = "cuda:0"
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    tv = torch.full((M, k), float("nan"), dtype=torch.float32, device=dev)
+    ti = torch.full((M, k), -1, dtype=torch.int32, device=dev)
+    ws = torch.empty(cf.gemm_spec_workspace_size(spec, shape), dtype=torch.uint8, device=dev)
+    cf.gemm_spec(to_dev(A), to_dev(B), Y, spec, params=[to_dev(bias)], row_out=[tv, ti], workspace=ws)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK
+    f = wl.bf16_to_f64
+    Yref, (rv, ri) = spo.gemm_spec(f(A), f(B), prog.nodes, prog.terminal, [f(bias)], prog.row_outputs)
+    return Y, tv.cpu().numpy(), ti.cpu().numpy(), Yref, rv, ri
+
+
+def test_topk_row_outputs_exact_on_integer_data_with_ties():
+    # small integers: the GEMM result is exact in bf16, so values AND columns must equal the oracle's, ties included
+    g = np.random.default_rng(5)
+    M, N, K = 70, 264, 16
+    A = wl.f32_to_bf16_bits(g.integers(-1, 2, size=(M, K)).astype(np.float32))
+    B = wl.f32_to_bf16_bits(g.integers(-2, 3, size=(K, N)).astype(np.float32))
+    bias = wl.f32_to_bf16_bits(np.zeros(N, dtype=np.float32))
+    Y, tv, ti, Yref, rv, ri = _run_topk(A, B, bias, 9)
+    np.testing.assert_array_equal(to_f64(Y), Yref)
+    np.testing.assert_array_equal(tv.astype(np.float64), rv)
+    np.testing.assert_array_equal(ti.astype(np.int64), ri.astype(np.int64))
+    assert (rv[:, :-1] == rv[:, 1:]).any()  # the data does contain ties
+
+
+def test_topk_row_outputs_on_gaussian_data():
+    M, N, K, k = 300, 1024, 136, 5
+    A, B, (bias,) = _inputs(41, 1, M, N, K, ("rowvec",))
+    Y, tv, ti, Yref, rv, ri = _run_topk(A, B, bias, k)
+    assert np.abs(to_f64(Y) - Yref).max() <= 3e-2
+    np.testing.assert_allclose(tv, rv, atol=3e-2)
+    assert np.all(np.diff(tv, axis=1) <= 0)                       # falling order
+    assert np.all((ti >= 0) & (ti < N)) and all(len(set(r)) == k for r in ti.tolist())
+    np.testing.assert_allclose(np.take_along_axis(Yref, ti.astype(np.int64), axis=1), tv, atol=3e-2)  # the picked columns hold those values
+    assert np.mean(ti == ri.astype(np.int64)) > 0.9

@@ -128,3 +128,15 @@ def test_malformed_programs_are_rejected():
     assert _status([N_, ("relu", 0, -1, -1, 0)], 1, row_outputs=(1,)) == INV                   # row output must be per-row
     assert _status([N_], 0, shape=cf.make_gemm_shape(1, 64, 100, 64)) == cf.ERR_ALIGNMENT      # N not a multiple of 8
     assert _status([("acc", 0, -1, -1, 0)], 0) == INV                                          # entry node with an input
+
+
+def test_topk_nodes_are_row_outputs_only():
+    INV = cf.ERR_INVALID_ARG
+    tk = ("topk_values", 0, -1, 4, 0.0)
+    assert _plan([N_, tk], 0, row_outputs=(1,)).path == cf.SPEC_PATH_ROW_PROGRAM
+    assert _plan([N_, tk], 0, row_outputs=(1,)).n_stages == 2
+    assert _status([N_, tk], 1) == INV                                           # cannot be the terminal
+    assert _status([N_, tk, ("relu", 1, -1, -1, 0)], 2) == INV                   # cannot feed a node
+    assert _status([N_, ("topk_values", 0, -1, 0, 0.0)], 0, row_outputs=(1,)) == INV    # K >= 1
+    assert _status([N_, ("topk_indices", 0, -1, 65, 0.0)], 0, row_outputs=(1,)) == INV  # K <= 64
+    assert _status([N_, ("topk_values", 0, -1, 40, 0.0)], 0, row_outputs=(1,), shape=cf.make_gemm_shape(1, 64, 32, 64)) == INV  # K <= N
