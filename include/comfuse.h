@@ -221,7 +221,12 @@ const char* comfuse_status_string(comfuse_status_t status);
  *   2. lowers it: a program whose stages have the shape of a compiled fused instantiation (affine entry
  *      [activation] [+ residual] -> LayerNorm | RMSNorm [-> max/argmax] | softmax, in any spelling the canonicaliser
  *      recognises: operand order of commutative nodes, optional nodes absent) runs as that ONE fused kernel
- *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); any other valid program runs on the standard pathway
+ *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); a program in which ONE tensor stays resident across the reductions and
+ *      every tensor-valued expression is a chain on it (element-wise nodes whose other operand is a constant, a per-row
+ *      value, a row vector, the causal mask or -- before the first reduction -- one full tensor; at most 3 row vectors,
+ *      6 reductions, 6 row outputs, 4 passes) runs as ONE fused kernel whose epilogue interprets the stages over the on-chip
+ *      accumulator (COMFUSE_SPEC_PATH_FUSED_PROGRAM; N in {256, 512, 768, 1024, 2048, 4096}: the reductions sum, mean,
+ *      max, min, prod, argmax merge across the cluster); any other valid program runs on the standard pathway
  *      (COMFUSE_SPEC_PATH_ROW_PROGRAM): the GEMM kernel writes bf16 Z to the workspace and one row-program kernel
  *      evaluates the node list per row with the row resident in shared memory, one pass per stage.
  */
@@ -274,7 +279,11 @@ typedef struct {
   int64_t batch_stride_a, batch_stride_b, batch_stride_y;  /* used when batch > 1 */
 } comfuse_gemm_shape_t;
 
-typedef enum { COMFUSE_SPEC_PATH_FUSED_KERNEL = 0, COMFUSE_SPEC_PATH_ROW_PROGRAM = 1 } comfuse_spec_path_t;
+typedef enum {
+  COMFUSE_SPEC_PATH_FUSED_KERNEL = 0,  /* a compiled fused instantiation (the enum kinds)                              */
+  COMFUSE_SPEC_PATH_ROW_PROGRAM = 1,   /* GEMM kernel, bf16 Z, row-program kernel                                      */
+  COMFUSE_SPEC_PATH_FUSED_PROGRAM = 2  /* ONE fused kernel whose epilogue interprets the program on-chip, stage by stage */
+} comfuse_spec_path_t;
 
 /* What the library will do with a program on a given shape (host-side analysis only; no device is touched). */
 typedef struct {
@@ -282,12 +291,14 @@ typedef struct {
   int32_t n_reductions;   /* live reduction nodes                                                       */
   int32_t n_live_nodes;   /* nodes the terminal or a row output depends on                              */
   int32_t path;           /* comfuse_spec_path_t chosen when `fused` = 1                                */
+  int32_t program_path;   /* the path when `fused` = 2 (compiled kinds skipped): FUSED_PROGRAM or ROW_PROGRAM */
+  int32_t n_passes;       /* FUSED_PROGRAM: passes over the resident tensor                             */
   int32_t fused_kind;     /* FUSED_KERNEL: the comfuse_epilogue_kind_t it lowers to, else -1            */
   uint32_t fused_flags;   /* FUSED_KERNEL: COMFUSE_FLAG_* bits                                          */
   float alpha, eps, softcap;  /* FUSED_KERNEL: recovered constants                                      */
   int32_t causal;         /* FUSED_KERNEL: 1 if the program adds the causal mask                        */
-  int32_t n_instructions; /* ROW_PROGRAM: computed nodes the row kernel executes                        */
-  int32_t n_slots;        /* ROW_PROGRAM: row-sized fp32 buffers held in shared memory at the same time */
+  int32_t n_instructions; /* the row program (`fused` = 0): computed nodes the row kernel executes      */
+  int32_t n_slots;        /* the row program: row-sized fp32 buffers held in shared memory at once      */
 } comfuse_spec_plan_t;
 
 /* Analyse a program: OK and *plan filled, INVALID_ARG for a malformed program (see above), UNSUPPORTED if it is valid
@@ -301,7 +312,8 @@ comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* s
 
 /* Y = program(A . B).  `params`: HOST array of spec->n_params DEVICE pointers (bf16; ROWVEC [N], TENSOR [batch, M, N]
  * with leading dimension param_ld[k], 0 = N); `param_ld` may be NULL.  `row_out`: HOST array of n_row_outputs DEVICE
- * pointers.  `fused` = 1: take the fused kernel when the program lowers to one; 0: always the row-program pathway.
+ * pointers.  `fused` = 1: the best path (compiled fused kind, else on-chip interpreter, else row program); 2: skip the
+ * compiled kinds (on-chip interpreter, else row program); 0: always the row-program pathway.
  * Asynchronous on `cuda_stream`; the host arrays are not read after the call returns. */
 comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A,
                                    const void* B, void* Y, const void* const* params, const int64_t* param_ld,

@@ -86,6 +86,7 @@ OPS = {
 }
 SPEC_PATH_FUSED_KERNEL = 0
 SPEC_PATH_ROW_PROGRAM = 1
+SPEC_PATH_FUSED_PROGRAM = 2
 
 
 class SpecNode(Structure):
@@ -105,6 +106,7 @@ class GemmShape(Structure):
 
 class SpecPlan(Structure):
     _fields_ = [("n_stages", c_int32), ("n_reductions", c_int32), ("n_live_nodes", c_int32), ("path", c_int32),
+                ("program_path", c_int32), ("n_passes", c_int32),
                 ("fused_kind", c_int32), ("fused_flags", ctypes.c_uint32), ("alpha", c_float), ("eps", c_float),
                 ("softcap", c_float), ("causal", c_int32), ("n_instructions", c_int32), ("n_slots", c_int32)]
 
@@ -380,7 +382,7 @@ def spec_plan(spec: FusionSpec, shape: GemmShape) -> SpecPlan:
 
 def gemm_spec_workspace_size(spec: FusionSpec, shape: GemmShape, fused=True) -> int:
     n = c_size_t(0)
-    st = lib().comfuse_gemm_spec_workspace_size(byref(spec), byref(shape), 1 if fused else 0, byref(n))
+    st = lib().comfuse_gemm_spec_workspace_size(byref(spec), byref(shape), int(fused), byref(n))
     if st != OK:
         raise ComfuseError(st, "comfuse_gemm_spec_workspace_size")
     return int(n.value)
@@ -400,7 +402,7 @@ def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, w
     ld = (c_int64 * n)(*[0 if (t is None or t.dim() < 2) else t.stride(-2) for t in params])
     ro = (c_void_p * max(1, len(row_out)))(*[t.data_ptr() for t in row_out])
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
-    st = lib().comfuse_gemm_spec(byref(spec), byref(shape), _ptr(A), _ptr(B), _ptr(Y), pp, ld, ro, 1 if fused else 0,
+    st = lib().comfuse_gemm_spec(byref(spec), byref(shape), _ptr(A), _ptr(B), _ptr(Y), pp, ld, ro, int(fused),
                                  ws_ptr, ws_bytes, _stream(stream))
     if st != OK:
         raise ComfuseError(st, "comfuse_gemm_spec")

@@ -213,6 +213,42 @@ comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, lon
   return launch_plain_gemm(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
 }
 
+comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
+                                   long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
+                                   const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
+                                   cudaStream_t st, bool query_only) {
+  FusedParams p = {};
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  GemmMaps maps;
+  if (query_only) {
+    std::memset(&maps, 0, sizeof(maps));
+    return launch_fused_program(maps, p, nullptr, true) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
+  }
+  const DeviceInfo* dev = nullptr;
+  comfuse_status_t s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  const long long bsr = static_cast<long long>(M) * ldr;
+  if (!make_gemm_maps(&maps, A, B, residual, Y, batch, M, N, K, lda, ldb, ldr, ldy, batch_stride_a, batch_stride_b, bsr,
+                      batch > 1 ? batch_stride_y : 0))
+    return COMFUSE_ERR_CUDA;
+  p.mblocks = (M + 127) / 128;
+  p.nblocks = 1;
+  p.total_tiles = batch * p.mblocks;
+  p.alpha = 1.f;
+  p.status = dev->status_word;
+  p.timeout_ns = timeout_ns();
+  p.leader_reduce = leader_reduce_enabled() ? 1 : 0;
+  p.bias = static_cast<const uint16_t*>(vecs[0]);
+  p.gamma = static_cast<const uint16_t*>(vecs[1]);
+  p.beta = static_cast<const uint16_t*>(vecs[2]);
+  p.residual = static_cast<const uint16_t*>(residual);
+  p.ldr = ldr; p.batch_stride_r = bsr;
+  p.Y = static_cast<uint16_t*>(Y);
+  p.ldy = ldy; p.batch_stride_y = batch > 1 ? batch_stride_y : 0;
+  p.program = prog;
+  return launch_fused_program(maps, p, st, false) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
 }  // namespace comfuse
 
 using namespace comfuse;

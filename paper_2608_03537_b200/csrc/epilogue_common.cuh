@@ -26,6 +26,19 @@ struct MergeMaxSumExp2 {  // (max, sum of 2^(t - max)); a partial with max = -in
     return make_float2(m, a.y * fa + b.y * fb);
   }
 };
+struct MergeByOp {  // (value, unused) under a run-time reduction operator: comfuse_op_t sum / mean / max / min / prod
+  int op;
+  __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const {
+    float r;
+    switch (op) {
+      case 50: r = fmaxf(a.x, b.x); break;  // COMFUSE_OP_RED_MAX
+      case 51: r = fminf(a.x, b.x); break;  // COMFUSE_OP_RED_MIN
+      case 52: r = a.x * b.x; break;        // COMFUSE_OP_RED_PROD
+      default: r = a.x + b.x; break;        // sum, mean
+    }
+    return make_float2(r, 0.f);
+  }
+};
 struct MergeArgmax {  // (value, column index bits); ties -> lower index
   __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const {
     const int ia = __float_as_int(a.y), ib = __float_as_int(b.y);

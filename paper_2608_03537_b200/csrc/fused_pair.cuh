@@ -31,6 +31,7 @@
 // written to swizzled per-warp staging buffers and stored with TMA.
 #pragma once
 
+#include "comfuse.h"
 #include "epilogue_common.cuh"
 #include "fused_params.h"
 #include "sm100_primitives.cuh"
@@ -161,7 +162,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int cluster_id = blockIdx.x / CLUSTER;
   const int num_clusters = gridDim.x / CLUSTER;
   const int KB = (p.K + 63) >> 6;
-  const bool has_res = (EPI == EPI_LN || kIsRms) && p.residual != nullptr;
+  const bool has_res = (EPI == EPI_LN || kIsRms || EPI == EPI_PROGRAM) && p.residual != nullptr;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
@@ -417,7 +418,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int xpar = 0;
     uint32_t xphase = 0;
     (void)xpar; (void)xphase; (void)s_pre; (void)s_stats; (void)s_bias; (void)s_gamma; (void)s_beta;
-    if constexpr (EPI == EPI_LN || kIsRms) {
+    if constexpr (EPI == EPI_LN || kIsRms || EPI == EPI_PROGRAM) {
       // row-vector broadcasts (Sec. 5.2: 1-D parameters) of this CTA's columns, widened to fp32 once, by the epilogue warps
       // (they have nothing else to do until the first accumulator is complete); wide rows: the bias of the tile's column
       // block is loaded per tile instead, gamma/beta are identity
@@ -731,6 +732,328 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const long long o = static_cast<long long>(b) * p.M + grow;
             p.row_max[o] = mx.x;
             p.row_argmax[o] = __float_as_int(mx.y);
+          }
+        }
+      } else if constexpr (EPI == EPI_PROGRAM) {
+        // ---------------- epilogue given as data: the stage program's passes over the TMEM-resident x (Sec. 3, Sec. 5.3)
+        const StageProgram& sp = p.program;
+        float sc[kStageMaxScalars];  // this row's scalars (reduction results and arithmetic on them)
+#pragma unroll
+        for (int i = 0; i < kStageMaxScalars; ++i) sc[i] = 0.f;
+        const float* vecs[3] = {s_bias, s_gamma, s_beta};
+        // one chain instruction on a 32-column fragment; col0 = first global column, lc = first CTA-local column
+        auto run_chain = [&](const ChainInstr* code, int n, float (&v)[32], int lc, int col0, const uint32_t* res16) {
+          for (int i = 0; i < n; ++i) {
+            const ChainInstr ci = code[i];
+            const int op = ci.op;
+            if (op < COMFUSE_OP_ADD) {  // unary
+              switch (op) {
+                case COMFUSE_OP_NEG:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = -v[j];
+                  break;
+                case COMFUSE_OP_ABS:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = fabsf(v[j]);
+                  break;
+                case COMFUSE_OP_SQUARE:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = v[j] * v[j];
+                  break;
+                case COMFUSE_OP_SQRT:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = sqrtf(v[j]);
+                  break;
+                case COMFUSE_OP_RSQRT:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = rsqrtf(v[j]);
+                  break;
+                case COMFUSE_OP_RECIP:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = __frcp_rn(v[j]);
+                  break;
+                case COMFUSE_OP_EXP:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = ex2_approx(v[j] * 1.4426950408889634f);
+                  break;
+                case COMFUSE_OP_LOG:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = __logf(v[j]);
+                  break;
+                case COMFUSE_OP_TANH:  // 1 - 2 / (1 + e^(2x)): absolute error about 1e-7 (tanh.approx has 2^-11 relative)
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = 1.f - 2.f * __frcp_rn(1.f + ex2_approx(2.8853900817779268f * v[j]));
+                  break;
+                case COMFUSE_OP_RELU:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+                  break;
+                case COMFUSE_OP_GELU_TANH:
+#pragma unroll
+                  for (int j = 0; j < 32; j += 2) {
+                    const float2 gz = gelu_tanh_f32x2(make_float2(v[j], v[j + 1]));
+                    v[j] = gz.x; v[j + 1] = gz.y;
+                  }
+                  break;
+                default:  // COMFUSE_OP_SIGMOID
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) v[j] = __frcp_rn(1.f + ex2_approx(-1.4426950408889634f * v[j]));
+                  break;
+              }
+              continue;
+            }
+            // binary: materialise the operand fragment, then apply
+            float o[32];
+            switch (ci.operand) {
+              case CHO_SCALAR: {
+                float sv = 0.f;
+#pragma unroll
+                for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ci.index) ? sc[q] : sv;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = sv;
+                break;
+              }
+              case CHO_ROWVEC: {
+                const float4* v4 = reinterpret_cast<const float4*>(vecs[ci.index] + lc);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 t4 = v4[j];
+                  o[4 * j] = t4.x; o[4 * j + 1] = t4.y; o[4 * j + 2] = t4.z; o[4 * j + 3] = t4.w;
+                }
+                break;
+              }
+              case CHO_RESIDUAL:
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const float2 t2 = bf16x2_to_f2(res16[j]);
+                  o[2 * j] = t2.x; o[2 * j + 1] = t2.y;
+                }
+                break;
+              case CHO_MASK:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;
+                break;
+              default:  // CHO_CONST
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = ci.imm;
+                break;
+            }
+            switch (op) {
+              case COMFUSE_OP_ADD:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = v[j] + o[j];
+                break;
+              case COMFUSE_OP_SUB:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = v[j] - o[j];
+                break;
+              case COMFUSE_OP_MUL:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = v[j] * o[j];
+                break;
+              case COMFUSE_OP_DIV:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __fdividef(v[j], o[j]);
+                break;
+              case COMFUSE_OP_MAX:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], o[j]);
+                break;
+              case COMFUSE_OP_MIN:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = fminf(v[j], o[j]);
+                break;
+              case kChainRsub:
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = o[j] - v[j];
+                break;
+              default:  // kChainRdiv
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __fdividef(o[j], v[j]);
+                break;
+            }
+          }
+        };
+        // thread-local partials of the reductions (value; column for an arg max); indexed at run time (local memory)
+        float racc[kStageMaxRed];
+        int ridx[kStageMaxRed];
+        auto red_init = [&](int r) {
+          const int op = r < sp.n_red ? sp.red[r].op : COMFUSE_OP_RED_SUM;
+          racc[r] = op == COMFUSE_OP_RED_PROD ? 1.f : (op == COMFUSE_OP_RED_MAX || op == COMFUSE_OP_RED_ARGMAX) ? -INFINITY
+                    : op == COMFUSE_OP_RED_MIN ? INFINITY : 0.f;
+          ridx[r] = 0x7FFFFFFF;
+        };
+        auto red_accumulate = [&](int r, const float (&u)[32], int col0) {
+          float a = racc[r];
+          switch (sp.red[r].op) {
+            case COMFUSE_OP_RED_SUM:
+            case COMFUSE_OP_RED_MEAN: {
+              float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) { t0 += u[j]; t1 += u[j + 1]; t2 += u[j + 2]; t3 += u[j + 3]; }
+              a += (t0 + t1) + (t2 + t3);
+              break;
+            }
+            case COMFUSE_OP_RED_MAX:
+#pragma unroll
+              for (int j = 0; j < 32; ++j) a = fmaxf(a, u[j]);
+              break;
+            case COMFUSE_OP_RED_MIN:
+#pragma unroll
+              for (int j = 0; j < 32; ++j) a = fminf(a, u[j]);
+              break;
+            case COMFUSE_OP_RED_PROD:
+#pragma unroll
+              for (int j = 0; j < 32; ++j) a *= u[j];
+              break;
+            default: {  // arg max: columns rise, a strict compare keeps the lowest
+              int ix = ridx[r];
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (u[j] > a) { a = u[j]; ix = col0 + j; }
+              ridx[r] = ix;
+              break;
+            }
+          }
+          racc[r] = a;
+        };
+        // cluster-wide merge of reduction r; the result becomes scalar sp.red[r].dst
+        auto red_merge = [&](int r) {
+          const int op = sp.red[r].op;
+          float2 tot;
+          const float2 mine = make_float2(racc[r], __int_as_float(ridx[r]));
+          if (op == COMFUSE_OP_RED_ARGMAX)
+            tot = cluster_row_reduce<CN, MergeArgmax, EPW>(mine, kThreadCount, MergeArgmax(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
+                                                          w, 2u, pm, p.leader_reduce != 0);
+          else
+            tot = cluster_row_reduce<CN, MergeByOp, EPW>(mine, kThreadCount, MergeByOp{op}, s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
+                                                        w, 2u, pm, p.leader_reduce != 0);
+          float val = op == COMFUSE_OP_RED_ARGMAX ? static_cast<float>(__float_as_int(tot.y)) : tot.x;
+          if (op == COMFUSE_OP_RED_MEAN) val *= 1.f / static_cast<float>(CN * BN);
+#pragma unroll
+          for (int q = 0; q < kStageMaxScalars; ++q)
+            if (q == sp.red[r].dst) sc[q] = val;
+        };
+        auto scalar_get = [&](int kind, int ix, float imm) {
+          float sv = imm;
+          if (kind == CHO_SCALAR) {
+#pragma unroll
+            for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ix) ? sc[q] : sv;
+          }
+          return sv;
+        };
+        auto boundary = [&](int pass) {
+          // merges of the pass's reductions in program order (every CTA of the group makes the same calls), then the
+          // per-row arithmetic that depends on them
+#pragma unroll 1
+          for (int r = 0; r < sp.n_red; ++r)
+            if (sp.red[r].pass == pass) red_merge(r);
+          for (int i = 0; i < sp.n_scalar_instr; ++i) {
+            const ScalarInstr si = sp.sc[i];
+            if (si.after_pass != pass) continue;
+            const float a = scalar_get(si.a_kind, si.a, si.a_imm);
+            const float bq = scalar_get(si.b_kind, si.b, si.b_imm);
+            float rv;
+            switch (si.op) {
+              case COMFUSE_OP_NEG: rv = -a; break;
+              case COMFUSE_OP_ABS: rv = fabsf(a); break;
+              case COMFUSE_OP_SQUARE: rv = a * a; break;
+              case COMFUSE_OP_SQRT: rv = sqrtf(a); break;
+              case COMFUSE_OP_RSQRT: rv = rsqrtf(a); break;
+              case COMFUSE_OP_RECIP: rv = 1.f / a; break;
+              case COMFUSE_OP_EXP: rv = expf(a); break;
+              case COMFUSE_OP_LOG: rv = logf(a); break;
+              case COMFUSE_OP_TANH: rv = tanhf(a); break;
+              case COMFUSE_OP_RELU: rv = fmaxf(a, 0.f); break;
+              case COMFUSE_OP_GELU_TANH: rv = 0.5f * a * (1.f + tanhf(0.7978845608028654f * (a + 0.044715f * a * a * a))); break;
+              case COMFUSE_OP_SIGMOID: rv = 1.f / (1.f + expf(-a)); break;
+              case COMFUSE_OP_ADD: rv = a + bq; break;
+              case COMFUSE_OP_SUB: rv = a - bq; break;
+              case COMFUSE_OP_MUL: rv = a * bq; break;
+              case COMFUSE_OP_DIV: rv = a / bq; break;
+              case COMFUSE_OP_MAX: rv = fmaxf(a, bq); break;
+              default: rv = fminf(a, bq); break;
+            }
+#pragma unroll
+            for (int q = 0; q < kStageMaxScalars; ++q)
+              if (q == si.dst) sc[q] = rv;
+          }
+        };
+#pragma unroll 1
+        for (int r = 0; r < kStageMaxRed; ++r) red_init(r);
+
+        for (int pass = 0; pass < sp.n_passes; ++pass) {
+          const bool is_terminal = pass == sp.terminal_pass;
+#pragma unroll
+          for (int sub = 0; sub < ESUB; ++sub) {
+            if (pass == 0) wait_accumulator(sub);
+            const int W = unit_width(sub);
+            const int lsub = unit_lg0(sub) * 64;
+            const uint32_t taddr = tmem_of(sub);
+            for (int g = h; g < W / 64; g += EPW) {
+              uint32_t r32[32];
+              if (pass == 0) {
+                if (has_res) {
+                  mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
+                  rfull_bits ^= 1u << ring.stage;
+                  __syncwarp();
+                  load_residual(smem_base + ring.stage * Cfg::STAGE_BYTES, h, r32);
+                  __syncwarp();
+                  if (lane == 0) mbar_arrive(bar_rdone(ring.stage));
+                  ring.advance();
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) r32[j] = 0u;
+                }
+              }
+              uint32_t pk[32];
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                const int lc = lsub + g * 64 + half * 32;
+                const int col0 = ncta0 + lc;
+                uint32_t vb[32];
+                tmem_ld_32cols(taddr + g * 64 + half * 32, vb);
+                float x[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(vb[j]);
+                if (pass == 0) {
+                  run_chain(sp.entry, sp.n_entry, x, lc, col0, r32 + half * 16);
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) vb[j] = __float_as_uint(x[j]);
+                  if (sp.n_passes > 1 || !is_terminal) tmem_st_32cols(taddr + g * 64 + half * 32, vb);
+                }
+#pragma unroll 1
+                for (int r = 0; r < sp.n_red; ++r) {
+                  if (sp.red[r].pass == pass && !sp.red[r].on_terminal) {
+                    float u[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) u[j] = x[j];
+                    run_chain(sp.chains + sp.red[r].chain_off, sp.red[r].chain_len, u, lc, col0, nullptr);
+                    red_accumulate(r, u, col0);
+                  }
+                }
+                if (is_terminal) {
+                  run_chain(sp.fin, sp.n_final, x, lc, col0, nullptr);
+#pragma unroll 1
+                  for (int r = 0; r < sp.n_red; ++r)
+                    if (sp.red[r].on_terminal) red_accumulate(r, x, col0);
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_bf16x2_rn(x[2 * j], x[2 * j + 1]);
+                }
+              }
+              if (is_terminal) store_box(pk);
+            }
+            if (pass == sp.n_passes - 1) release_accumulator(sub);
+          }
+          if (pass == 0) tmem_st_wait();
+          boundary(pass);
+        }
+        if (crank == 0 && h == 0 && valid) {
+          const long long o = static_cast<long long>(b) * p.M + grow;
+          for (int r = 0; r < sp.n_row_out; ++r) {
+            const float val = scalar_get(CHO_SCALAR, sp.out[r].scalar, 0.f);
+            if (sp.out[r].is_int) static_cast<int*>(sp.out[r].ptr)[o] = static_cast<int>(val);
+            else static_cast<float*>(sp.out[r].ptr)[o] = val;
           }
         }
       } else {  // EPI_SOFTMAX

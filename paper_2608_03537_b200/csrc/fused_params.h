@@ -7,7 +7,76 @@
 namespace comfuse {
 
 // EPI_RMS_MAX_LINEAR: the RMSNorm op list without its GELU (a kernel instantiation of its own, chosen by FusedParams::no_activation)
-enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3, EPI_RMS_MAX_LINEAR = 4 };
+enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3, EPI_RMS_MAX_LINEAR = 4, EPI_PROGRAM = 5 };
+
+// ---------------------------------------------------------------------------------------------------------------
+// Stage program: an epilogue given as data, lowered for the on-chip interpreter of the fused kernel (EPI_PROGRAM).
+// The Stage-Stream model (Sec. 3) with ONE resident tensor x (the accumulator's TMEM columns) and per-row scalars:
+//   pass 0:   v = entry(acc)            -> x (written back to TMEM); reductions whose input is available in pass 0
+//   pass s:   for every reduction of pass s: u = chain_r(x) -> thread partial -> cluster merge -> scalar
+//             then the per-row scalar instructions of that boundary
+//   the pass the terminal belongs to also computes y = final(x), rounds and stores it, and accumulates the
+//   reductions that take y itself as input (the chained second reduction of Sec. 3.2).
+// Chains are accumulator-machine code on a 32-column fragment: v = op(v) or v = v (op) operand.
+enum ChainOperand : uint8_t {
+  CHO_NONE = 0,
+  CHO_CONST,     // imm
+  CHO_SCALAR,    // per-row scalar `index`
+  CHO_ROWVEC,    // row-vector parameter staged in shared memory, `index` = 0..2
+  CHO_RESIDUAL,  // the full-tensor parameter (entry chain only; delivered through the operand ring)
+  CHO_MASK       // causal mask: 0 where column <= row, -inf above the diagonal
+};
+// chain opcodes: the comfuse_op_t values of the unary / binary nodes, plus the reversed non-commutative forms
+constexpr int kChainRsub = 64;  // v = operand - v
+constexpr int kChainRdiv = 65;  // v = operand / v
+
+struct ChainInstr {
+  uint8_t op;
+  uint8_t operand;  // ChainOperand
+  int16_t index;
+  float imm;
+};
+
+struct StageReduction {
+  uint8_t pass;        // the pass in which its input is available
+  uint8_t op;          // comfuse_op_t of the reduction (sum, mean, max, min, prod, argmax)
+  uint8_t chain_off;   // its input chain: chains[chain_off .. chain_off + chain_len), applied to x
+  uint8_t chain_len;
+  uint8_t on_terminal; // input is y itself: accumulated in the terminal's pass from the unrounded y
+  uint8_t dst;         // per-row scalar it defines
+  uint8_t pad[2];
+};
+
+struct ScalarInstr {   // per-row arithmetic at a stage boundary: s[dst] = op(a, b)
+  uint8_t after_pass;  // runs after the merges of this pass
+  uint8_t op;
+  uint8_t dst;
+  uint8_t a_kind, b_kind;  // CHO_CONST or CHO_SCALAR
+  uint8_t a, b;
+  uint8_t pad;
+  float a_imm, b_imm;
+};
+
+struct StageRowOutput {
+  void* ptr;        // fp32 [batch * M], int32 for an arg max
+  uint8_t scalar;
+  uint8_t is_int;
+  uint8_t pad[6];
+};
+
+constexpr int kStageMaxEntry = 12, kStageMaxFinal = 16, kStageMaxChains = 24, kStageMaxRed = 6, kStageMaxScalarInstr = 12,
+              kStageMaxScalars = 16, kStageMaxRowOut = 6, kStageMaxPasses = 4;
+
+struct StageProgram {
+  uint8_t n_entry, n_final, n_red, n_scalar_instr;
+  uint8_t n_passes, terminal_pass, n_row_out, pad;
+  ChainInstr entry[kStageMaxEntry];
+  ChainInstr fin[kStageMaxFinal];
+  ChainInstr chains[kStageMaxChains];
+  StageReduction red[kStageMaxRed];
+  ScalarInstr sc[kStageMaxScalarInstr];
+  StageRowOutput out[kStageMaxRowOut];
+};
 
 struct FusedParams {
   int M, N, K, batch;
@@ -38,6 +107,7 @@ struct FusedParams {
   // 1 = leader-follower (partials go to column range 0, which merges and sends the result back).  Same merge order,
   // hence the same bits, either way.
   int leader_reduce;
+  StageProgram program;  // EPI_PROGRAM only
   unsigned int* status;
   unsigned long long timeout_ns;
   unsigned long long* trace;  // phase timestamps of CTA 0 (builds with -DCOMFUSE_TRACE only), else null

@@ -363,6 +363,187 @@ bool match_fused(const Analysis& an, FusedMatch& m) {
   return false;
 }
 
+// ------------------------------------------------------------------------------------------------ stage program
+// Lowering for the on-chip interpreter (fused_params.h: StageProgram): possible when ONE tensor stays resident
+// across the stage boundaries (Sec. 5.3: the reduction's statistics and the passed-through original tensor are the
+// two entry points of the nested sub-program) and every tensor-valued expression is a chain on it.
+struct StageBinding {
+  int rowvec_param[3] = {-1, -1, -1};
+  int n_rowvec = 0;
+  int tensor_param = -1;
+  int row_out_pos[kStageMaxRowOut] = {};  // StageProgram::out[r] is row output number row_out_pos[r]
+};
+
+struct StageLowering {
+  const Analysis& an;
+  StageBinding& bind;
+  std::vector<int> scalar_of;  // per node: its per-row scalar index, -1 = none
+  int x_root = -1;
+  explicit StageLowering(const Analysis& a, StageBinding& b) : an(a), bind(b), scalar_of(a.n, -1) {}
+
+  bool tensor(int k) const { return an.type[k] == T_TENSOR; }
+  // can node k be the right-hand operand of a chain instruction?
+  bool operand(int k, bool entry_mode, ChainInstr& ci) {
+    ci.operand = CHO_NONE; ci.index = 0; ci.imm = 0.f;
+    if (an.type[k] == T_CONST) { ci.operand = CHO_CONST; ci.imm = an.cval[k]; return true; }
+    if (an.type[k] == T_ROW) {
+      if (scalar_of[k] < 0) return false;
+      ci.operand = CHO_SCALAR; ci.index = static_cast<int16_t>(scalar_of[k]);
+      return true;
+    }
+    switch (an.nodes[k].op) {
+      case COMFUSE_OP_ROWVEC: {
+        const int q = an.nodes[k].param;
+        int slot = -1;
+        for (int i = 0; i < bind.n_rowvec; ++i) if (bind.rowvec_param[i] == q) slot = i;
+        if (slot < 0) {
+          if (bind.n_rowvec == 3) return false;
+          slot = bind.n_rowvec++;
+          bind.rowvec_param[slot] = q;
+        }
+        ci.operand = CHO_ROWVEC; ci.index = static_cast<int16_t>(slot);
+        return true;
+      }
+      case COMFUSE_OP_TENSOR:
+        if (!entry_mode) return false;  // the operand ring delivers it once, in pass 0
+        if (bind.tensor_param >= 0 && bind.tensor_param != an.nodes[k].param) return false;
+        bind.tensor_param = an.nodes[k].param;
+        ci.operand = CHO_RESIDUAL;
+        return true;
+      case COMFUSE_OP_CAUSAL_MASK: ci.operand = CHO_MASK; return true;
+      default: return false;
+    }
+  }
+  bool is_root(int k, bool entry_mode) const { return entry_mode ? an.nodes[k].op == COMFUSE_OP_ACC : k == x_root; }
+  // code that turns the root's value into node k's value
+  bool chain(int k, bool entry_mode, std::vector<ChainInstr>& out) {
+    if (is_root(k, entry_mode)) return true;
+    if (!tensor(k)) return false;
+    const comfuse_spec_node_t& nd = an.nodes[k];
+    if (is_unary(nd.op)) {
+      if (!chain(nd.in0, entry_mode, out)) return false;
+      out.push_back(ChainInstr{static_cast<uint8_t>(nd.op), CHO_NONE, 0, 0.f});
+      return true;
+    }
+    if (!is_binary(nd.op)) return false;  // a tensor leaf that is not the root cannot start a chain
+    const int a = nd.in0, b = nd.in1;
+    ChainInstr ci;
+    auto carrier = [&](int q) { return is_root(q, entry_mode) || (tensor(q) && !is_leaf(an.nodes[q].op)); };
+    if (a == b && nd.op == COMFUSE_OP_MUL && carrier(a)) {
+      if (!chain(a, entry_mode, out)) return false;
+      out.push_back(ChainInstr{COMFUSE_OP_SQUARE, CHO_NONE, 0, 0.f});
+      return true;
+    }
+    if (carrier(a) && !carrier(b) && operand(b, entry_mode, ci)) {
+      if (!chain(a, entry_mode, out)) return false;
+      ci.op = static_cast<uint8_t>(nd.op);
+      out.push_back(ci);
+      return true;
+    }
+    if (carrier(b) && !carrier(a) && operand(a, entry_mode, ci)) {
+      if (!chain(b, entry_mode, out)) return false;
+      ci.op = static_cast<uint8_t>(nd.op == COMFUSE_OP_SUB ? kChainRsub : nd.op == COMFUSE_OP_DIV ? kChainRdiv : nd.op);
+      out.push_back(ci);
+      return true;
+    }
+    return false;  // two computed tensors (needs a second resident tensor), or two broadcasts
+  }
+};
+
+bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bind) {
+  std::memset(&sp, 0, sizeof(sp));
+  if (!an.row_outputs.empty() && an.row_outputs.size() > static_cast<size_t>(kStageMaxRowOut)) return false;
+  if (an.type[an.terminal] != T_TENSOR) return false;
+  StageLowering L(an, bind);
+  const int n = an.n;
+  // the resident tensor: the one stage-0 tensor that later stages read
+  int first_acc = -1;
+  std::vector<int> cand;
+  for (int k = 0; k < n; ++k) {
+    if (!an.live[k]) continue;
+    if (an.nodes[k].op == COMFUSE_OP_ACC && first_acc < 0) first_acc = k;
+    if (an.type[k] != T_TENSOR || an.stage[k] < 1 || is_reduce(an.nodes[k].op)) continue;
+    for (int e : {an.nodes[k].in0, an.nodes[k].in1}) {
+      if (e < 0 || an.type[e] != T_TENSOR || an.stage[e] != 0) continue;
+      const int eop = an.nodes[e].op;
+      if (is_leaf(eop) && eop != COMFUSE_OP_ACC) continue;  // broadcasts are re-read, not resident
+      bool seen = false;
+      for (int c : cand) seen |= c == e;
+      if (!seen) cand.push_back(e);
+    }
+  }
+  if (cand.size() > 1) return false;
+  if (first_acc < 0) return false;
+  L.x_root = cand.size() == 1 ? cand[0] : (an.stage[an.terminal] == 0 ? an.terminal : first_acc);
+  // stage 0: acc -> x
+  std::vector<ChainInstr> code;
+  if (!L.chain(L.x_root, true, code) || code.size() > static_cast<size_t>(kStageMaxEntry)) return false;
+  sp.n_entry = static_cast<uint8_t>(code.size());
+  for (size_t i = 0; i < code.size(); ++i) sp.entry[i] = code[i];
+  // reductions and per-row arithmetic, in node order
+  int scalars = 0, pool = 0, max_pass = an.stage[an.terminal];
+  for (int k = 0; k < n; ++k) {
+    if (!an.live[k] || an.type[k] != T_ROW) continue;
+    const comfuse_spec_node_t& nd = an.nodes[k];
+    if (scalars >= kStageMaxScalars) return false;
+    if (is_reduce(nd.op)) {
+      if (is_topk(nd.op) || sp.n_red >= kStageMaxRed) return false;
+      const int e = nd.in0;
+      if (an.type[e] != T_TENSOR) return false;
+      StageReduction& r = sp.red[sp.n_red];
+      r.op = static_cast<uint8_t>(nd.op);
+      r.pass = static_cast<uint8_t>(an.stage[e]);
+      r.dst = static_cast<uint8_t>(scalars);
+      if (e == an.terminal) {
+        r.on_terminal = 1;
+      } else {
+        code.clear();
+        if (!L.chain(e, false, code) || pool + code.size() > static_cast<size_t>(kStageMaxChains)) return false;
+        r.chain_off = static_cast<uint8_t>(pool);
+        r.chain_len = static_cast<uint8_t>(code.size());
+        for (const ChainInstr& c : code) sp.chains[pool++] = c;
+      }
+      if (r.pass > max_pass) max_pass = r.pass;
+      ++sp.n_red;
+    } else {
+      if (sp.n_scalar_instr >= kStageMaxScalarInstr || an.stage[k] < 1) return false;
+      ScalarInstr& si = sp.sc[sp.n_scalar_instr++];
+      si.after_pass = static_cast<uint8_t>(an.stage[k] - 1);
+      si.op = static_cast<uint8_t>(nd.op);
+      si.dst = static_cast<uint8_t>(scalars);
+      auto set = [&](int e, uint8_t& kind, uint8_t& ix, float& imm) {
+        if (e < 0) { kind = CHO_CONST; ix = 0; imm = 0.f; return true; }
+        if (an.type[e] == T_CONST) { kind = CHO_CONST; ix = 0; imm = an.cval[e]; return true; }
+        if (an.type[e] != T_ROW || L.scalar_of[e] < 0) return false;
+        kind = CHO_SCALAR; ix = static_cast<uint8_t>(L.scalar_of[e]); imm = 0.f;
+        return true;
+      };
+      if (!set(nd.in0, si.a_kind, si.a, si.a_imm) || !set(nd.in1, si.b_kind, si.b, si.b_imm)) return false;
+    }
+    L.scalar_of[k] = scalars++;
+  }
+  // the terminal: x -> y
+  code.clear();
+  if (!L.chain(an.terminal, false, code) || code.size() > static_cast<size_t>(kStageMaxFinal)) return false;
+  sp.n_final = static_cast<uint8_t>(code.size());
+  for (size_t i = 0; i < code.size(); ++i) sp.fin[i] = code[i];
+  sp.terminal_pass = static_cast<uint8_t>(an.stage[an.terminal]);
+  if (max_pass + 1 > kStageMaxPasses) return false;
+  sp.n_passes = static_cast<uint8_t>(max_pass + 1);
+  // a reduction on y is accumulated in the terminal's pass; anything the terminal needs must be merged before it
+  for (int r = 0; r < sp.n_red; ++r)
+    if (sp.red[r].on_terminal) sp.red[r].pass = sp.terminal_pass;
+  for (size_t r = 0; r < an.row_outputs.size(); ++r) {
+    const int q = an.row_outputs[r];
+    if (an.type[q] != T_ROW || L.scalar_of[q] < 0) return false;
+    sp.out[r].scalar = static_cast<uint8_t>(L.scalar_of[q]);
+    sp.out[r].is_int = an.nodes[q].op == COMFUSE_OP_RED_ARGMAX;
+    bind.row_out_pos[r] = static_cast<int>(r);
+  }
+  sp.n_row_out = static_cast<uint8_t>(an.row_outputs.size());
+  return true;
+}
+
 // ------------------------------------------------------------------------------------------------ row program
 comfuse_status_t lower_row_program(const Analysis& an, int N, RowProgram& P, int& n_instr, int& n_slots) {
   const int n = an.n;
@@ -476,7 +657,10 @@ comfuse_gemm_desc_t fused_desc(const comfuse_gemm_shape_t& s, const FusedMatch& 
 struct Decision {
   Analysis an;
   FusedMatch match;
-  bool fused = false;
+  bool fused = false;       // a compiled fused kind
+  bool on_chip = false;     // the on-chip stage-program interpreter
+  StageProgram stage_prog;
+  StageBinding stage_bind;
   size_t fused_inner_ws = 0;  // what the fused entry point itself needs
   size_t fused_scratch = 0;   // row max / arg max the caller did not ask for
 };
@@ -486,7 +670,7 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
   if (s != COMFUSE_OK) return s;
   s = analyse(spec, dc.an);
   if (s != COMFUSE_OK) return s;
-  if (want_fused && match_fused(dc.an, dc.match)) {
+  if (want_fused == 1 && match_fused(dc.an, dc.match)) {
     const comfuse_gemm_desc_t d = fused_desc(*shape, dc.match, shape->N);
     size_t ws = 0;
     if (comfuse_workspace_size(&d, &ws) == COMFUSE_OK) {
@@ -495,6 +679,11 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
       if (dc.match.kind == COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX && (dc.match.row_max_out < 0 || dc.match.row_argmax_out < 0))
         dc.fused_scratch = 2 * static_cast<size_t>(shape->batch) * shape->M * 4;
     }
+  }
+  if (want_fused && !dc.fused && lower_stage_program(dc.an, dc.stage_prog, dc.stage_bind)) {
+    const void* none[3] = {nullptr, nullptr, nullptr};
+    dc.on_chip = run_fused_program(shape->batch, shape->M, shape->N, shape->K, 0, 0, 0, 0, 0, 0, nullptr, nullptr, nullptr, dc.stage_prog,
+                                   none, nullptr, 0, nullptr, true) == COMFUSE_OK;
   }
   return COMFUSE_OK;
 }
@@ -522,22 +711,34 @@ comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comf
     plan->fused_flags = dc.match.flags;
     plan->alpha = dc.match.alpha; plan->eps = dc.match.eps; plan->softcap = dc.match.softcap;
     plan->causal = dc.match.causal;
-    return COMFUSE_OK;
   }
-  plan->path = COMFUSE_SPEC_PATH_ROW_PROGRAM;
+  // what `fused` = 2 would take (the compiled kinds skipped)
+  Decision d2;
+  s = decide(spec, shape, 2, d2);
+  if (s != COMFUSE_OK) return s;
+  plan->program_path = d2.on_chip ? COMFUSE_SPEC_PATH_FUSED_PROGRAM : COMFUSE_SPEC_PATH_ROW_PROGRAM;
+  if (d2.on_chip) plan->n_passes = d2.stage_prog.n_passes;
+  if (!dc.fused) plan->path = plan->program_path;
+  // the row program (what `fused` = 0 runs) is described in any case
   RowProgram P;
   std::memset(&P, 0, sizeof(P));
-  return lower_row_program(dc.an, shape->N, P, plan->n_instructions, plan->n_slots);
+  s = lower_row_program(dc.an, shape->N, P, plan->n_instructions, plan->n_slots);
+  // where another path exists, the row program's limits are no error
+  return (plan->path == COMFUSE_SPEC_PATH_ROW_PROGRAM) ? s : COMFUSE_OK;
 }
 
 comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused,
                                                   size_t* bytes) {
-  if (!bytes || (fused != 0 && fused != 1)) return COMFUSE_ERR_INVALID_ARG;
+  if (!bytes || fused < 0 || fused > 2) return COMFUSE_ERR_INVALID_ARG;
   Decision dc;
   comfuse_status_t s = decide(spec, shape, fused, dc);
   if (s != COMFUSE_OK) return s;
   if (dc.fused) {
     *bytes = dc.fused_inner_ws + dc.fused_scratch;
+    return COMFUSE_OK;
+  }
+  if (dc.on_chip) {
+    *bytes = 0;
     return COMFUSE_OK;
   }
   RowProgram P;
@@ -552,7 +753,7 @@ comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* s
 comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A, const void* B,
                                    void* Y, const void* const* params, const int64_t* param_ld, void* const* row_out, int32_t fused,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  if (fused != 0 && fused != 1) return COMFUSE_ERR_INVALID_ARG;
+  if (fused < 0 || fused > 2) return COMFUSE_ERR_INVALID_ARG;
   Decision dc;
   comfuse_status_t s = decide(spec, shape, fused, dc);
   if (s != COMFUSE_OK) return s;
@@ -598,13 +799,26 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
     return comfuse_gemm_epilogue(&d, A, B, Y, &a, workspace, dc.fused_inner_ws, cuda_stream);
   }
 
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (dc.on_chip) {
+    // ONE fused kernel, the program's stages interpreted over the on-chip accumulator
+    const StageBinding& bd = dc.stage_bind;
+    const void* vecs[3] = {nullptr, nullptr, nullptr};
+    for (int i = 0; i < bd.n_rowvec; ++i) vecs[i] = params[bd.rowvec_param[i]];
+    StageProgram sp = dc.stage_prog;
+    for (int r = 0; r < sp.n_row_out; ++r) sp.out[r].ptr = row_out[bd.row_out_pos[r]];
+    const void* res = bd.tensor_param >= 0 ? params[bd.tensor_param] : nullptr;
+    return run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
+                             shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res,
+                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false);
+  }
+
   // standard pathway: GEMM -> bf16 Z in the workspace -> row program
   RowProgram P;
   std::memset(&P, 0, sizeof(P));
   int ni, ns;
   s = lower_row_program(an, shape->N, P, ni, ns);
   if (s != COMFUSE_OK) return s;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   s = gemm_to_bf16(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->batch_stride_a, shape->batch_stride_b, A, B,
                    workspace, st);
   if (s != COMFUSE_OK) return s;

@@ -44,6 +44,8 @@ struct GemmMaps {
 // exists without launching.
 cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+// Epilogue = the stage program in p.program, interpreted on-chip (N in {256, 512, 768, 1024, 2048, 4096}).
+cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Rows wider than the largest cluster (16 CTAs x 256 columns): LayerNorm / RMSNorm kinds run per 4096-column block and a
 // second kernel merges the blocks' statistics (the wide-row fallback).  Returns the number of blocks, 0 = not a wide row.
 constexpr int kWideRowBlock = 4096;
@@ -62,6 +64,13 @@ cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t 
 #include "comfuse.h"
 
 namespace comfuse {
+// Y = stage program(A . B) with the on-chip interpreter (EPI_PROGRAM).  `vecs` = the up to three row-vector parameters
+// the program's CHO_ROWVEC operands index, `residual` = its full-tensor parameter or null.  `query_only`: just say
+// whether an instantiation exists for N (no device is touched).
+comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
+                                   long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
+                                   const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
+                                   cudaStream_t st, bool query_only);
 // Z = bf16(A . B), dense [batch, M, N] (ld = N), with the plain tensor-core GEMM kernel; arguments already validated.
 comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
                               long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st);

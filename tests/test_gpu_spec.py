@@ -27,6 +27,7 @@ def _inputs(seed, batch, M, N, K, kinds):
 
 
 def _run(prog, A, B, params, fused, batch, M, N):
+    fused = int(fused)
     dev = "cuda:0"
     spec = cf.make_spec(prog.nodes, prog.terminal, len(prog.param_kinds), prog.row_outputs)
     dA, dB = to_dev(A), to_dev(B)
@@ -108,6 +109,54 @@ def test_same_program_on_the_row_program_pathway(name):
     tmax = TOL_SOFTMAX_UNFUSED if kind == cf.EPI_SCALE_MASK_SOFTMAX else tmax
     assert np.isfinite(err).all() and err.max() <= tmax and err.mean() <= tmean, (err.max(), err.mean())
     _check_rows(prog, ro, Rref, Yref, tol=2e-2)
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_same_program_on_the_on_chip_interpreter(name):
+    prog, batch, M, N, K, kind, tmax, tmean = CASES[name]
+    A, B, params = _inputs(35, batch, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, 2, batch, M, N)
+    assert plan.program_path == cf.SPEC_PATH_FUSED_PROGRAM and launches == 1
+    Yref, Rref = _oracle(prog, A, B, params, batch)
+    err = np.abs(to_f64(Y) - Yref)
+    assert np.isfinite(err).all() and err.max() <= tmax and err.mean() <= tmean, (err.max(), err.mean())
+    _check_rows(prog, ro, Rref, Yref)
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 1024, 136), (520, 4096, 72), (129, 256, 64), (260, 768, 264)])
+def test_chain_program_outside_the_compiled_patterns_runs_on_chip(M, N, K):
+    prog = wl.spec_range_normalise()
+    A, B, params = _inputs(36, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, True, 1, M, N)
+    assert plan.path == cf.SPEC_PATH_FUSED_PROGRAM and plan.n_passes == 2 and launches == 1
+    Yref, Rref = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    assert np.isfinite(err).all() and err.max() <= 4e-3 and err.mean() <= 1e-3, (err.max(), err.mean())
+    lo, hi, pr, sm, am = [t.cpu().numpy() for t in ro]
+    np.testing.assert_allclose(lo, Rref[0], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(hi, Rref[1], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(pr, Rref[2], rtol=1e-4)
+    np.testing.assert_allclose(sm, Rref[3], rtol=1e-4)
+    # y's maximum is attained where x's is; the gap to the runner-up is far above fp32 rounding for Gaussian rows
+    assert np.mean(am == Rref[4].astype(np.int64)) > 0.995
+    chosen = Yref[np.arange(M), am.astype(np.int64)]
+    assert np.all(chosen >= Yref.max(axis=1) - 1e-5)
+
+
+def test_near_miss_of_a_compiled_kind_runs_on_chip():
+    # residual inside the activation (the compiled RMSNorm kind has it outside), no row outputs
+    N_ = ("acc", -1, -1, -1, 0.0)
+    nodes = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("tensor", -1, -1, 1, 0), ("add", 2, 3, -1, 0), ("gelu_tanh", 4, -1, -1, 0),
+             ("square", 5, -1, -1, 0), ("mean", 6, -1, -1, 0), ("const", -1, -1, -1, 1e-5), ("add", 7, 8, -1, 0), ("rsqrt", 9, -1, -1, 0),
+             ("mul", 5, 10, -1, 0)]
+    prog = wl.SpecProgram(nodes, 11, (), ("rowvec", "tensor"))
+    M, N, K = 392, 2048, 136
+    A, B, params = _inputs(37, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, True, 1, M, N)
+    assert plan.path == cf.SPEC_PATH_FUSED_PROGRAM and launches == 1
+    Yref, _ = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    assert np.isfinite(err).all() and err.max() <= TOL_NORM_MAX and err.mean() <= TOL_NORM_MEAN, (err.max(), err.mean())
 
 
 def test_fused_lowering_equals_the_enum_entry_point_bit_for_bit():

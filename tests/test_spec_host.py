@@ -83,25 +83,51 @@ def test_recovered_constants():
     assert _plan(p.nodes, p.terminal, 4).eps == pytest.approx(3e-4)
 
 
-def test_near_misses_take_the_row_program():
-    # residual added INSIDE the activation: not the compiled RMSNorm entry
+def test_near_misses_do_not_take_a_compiled_kind():
+    PROG, ROW = cf.SPEC_PATH_FUSED_PROGRAM, cf.SPEC_PATH_ROW_PROGRAM
+    # residual added INSIDE the activation: not the compiled RMSNorm entry, but still one resident tensor -> on-chip interpreter
     g = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("tensor", -1, -1, 1, 0), ("add", 2, 3, -1, 0), ("gelu_tanh", 4, -1, -1, 0),
          ("square", 5, -1, -1, 0), ("mean", 6, -1, -1, 0), ("const", -1, -1, -1, 1e-5), ("add", 7, 8, -1, 0), ("rsqrt", 9, -1, -1, 0),
          ("mul", 5, 10, -1, 0)]
-    assert _plan(g, 11, 2).path == cf.SPEC_PATH_ROW_PROGRAM
+    assert _plan(g, 11, 2).path == PROG
     # soft-cap whose two constants are not reciprocal
     p = wl.spec_softmax(0.5, False, 2.0)
     nodes = [(op, a, b, q, 0.7 if (op == "const" and abs(i - 0.5) < 1e-9 and k > 1) else i) for k, (op, a, b, q, i) in enumerate(p.nodes)]
-    assert _plan(nodes, p.terminal).path == cf.SPEC_PATH_ROW_PROGRAM
+    assert _plan(nodes, p.terminal).path == PROG
     # LayerNorm with an extra row output
     p = wl.spec_layernorm()
-    assert _plan(p.nodes, p.terminal, 4, (p.nodes.index(("mean", 4, -1, -1, 0.0)),)).path == cf.SPEC_PATH_ROW_PROGRAM
-    # causal softmax on a non-square problem: no fused instantiation
+    assert _plan(p.nodes, p.terminal, 4, (p.nodes.index(("mean", 4, -1, -1, 0.0)),)).path == PROG
+    # causal softmax on a non-square problem: no compiled softmax kind, the interpreter takes any M
     p = wl.spec_softmax(0.5, True)
-    assert _plan(p.nodes, p.terminal, shape=cf.make_gemm_shape(1, 256, 512, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
-    # a fused pattern on a row length without an instantiation
+    assert _plan(p.nodes, p.terminal, shape=cf.make_gemm_shape(1, 256, 512, 64)).path == PROG
+    # a row length without any fused instantiation
     p = wl.spec_layernorm()
-    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
+    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == ROW
+
+
+def test_on_chip_lowering_needs_one_resident_tensor():
+    PROG, ROW = cf.SPEC_PATH_FUSED_PROGRAM, cf.SPEC_PATH_ROW_PROGRAM
+    # compiled kinds are also expressible on-chip (what `fused` = 2 runs), with one pass per stage that reads x
+    for prog, n_params, passes in ((wl.spec_layernorm(relu=True), 4, 3), (wl.spec_rmsnorm_max(), 3, 2), (wl.spec_softmax(0.2, True, 3.0), 0, 3)):
+        pl = _plan(prog.nodes, prog.terminal, n_params, prog.row_outputs, shape=cf.make_gemm_shape(1, 1024, 1024, 64))
+        assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.program_path == PROG and pl.n_passes == passes
+    # x * sigmoid(x): two computed tensors meet in one node -> needs a second resident tensor -> row program
+    p = wl.spec_gated_minmax()
+    pl = _plan(p.nodes, p.terminal, 1, p.row_outputs)
+    assert pl.path == ROW and pl.program_path == ROW
+    # no reduction at all: a single pass
+    pl = _plan([N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0)], 3, 1)
+    assert pl.path == PROG and pl.n_passes == 1
+    # a reduction of something below the resident tensor (max of the raw accumulator while x = acc + bias is kept)
+    nodes = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("rmax", 0, -1, -1, 0), ("mean", 2, -1, -1, 0), ("sub", 2, 4, -1, 0),
+             ("mul", 5, 3, -1, 0)]
+    assert _plan(nodes, 6, 1).path == ROW
+    # four row vectors: more than the kernel stages in shared memory
+    nodes = [N_] + [("rowvec", -1, -1, q, 0) for q in range(4)] + [("add", 0, 1, -1, 0), ("mul", 5, 2, -1, 0), ("add", 6, 3, -1, 0), ("mul", 7, 4, -1, 0)]
+    assert _plan(nodes, 8, 4).path == ROW
+    # a full tensor used after a reduction (the operand ring delivers it in pass 0 only)
+    nodes = [N_, ("mean", 0, -1, -1, 0), ("sub", 0, 1, -1, 0), ("tensor", -1, -1, 0, 0), ("add", 2, 3, -1, 0)]
+    assert _plan(nodes, 4, 1).path == ROW
 
 
 def test_row_program_reuses_buffers_by_liveness():

@@ -334,3 +334,19 @@ def spec_gated_minmax() -> SpecProgram:
     y = g.add("div", g.add("sub", s, lo), rng)
     pr = g.add("prod", g.add("add", g.add("mul", sg, g.add("const", imm=0.01)), g.add("const", imm=0.995)))
     return SpecProgram(g.nodes, y, (lo, hi, pr), ("rowvec",))
+
+
+def spec_range_normalise() -> SpecProgram:
+    """A chain program outside the compiled patterns that keeps ONE tensor resident: x = acc + bias, rescaled to the row's
+    range with a min and a max reduction (same stage boundary), then chained reductions on the result (sum, arg max) and a
+    product reduction of a function of x (the sum / prod / max / min operators of Sec. 5).  Parameter slot 0: bias."""
+    g = _Prog()
+    x = g.add("add", g.add("acc"), g.add("rowvec", param=0))
+    lo = g.add("rmin", x)
+    hi = g.add("rmax", x)
+    rng = g.add("add", g.add("sub", hi, lo), g.add("const", imm=1e-3))
+    y = g.add("div", g.add("sub", x, lo), rng)
+    pr = g.add("prod", g.add("add", g.add("mul", g.add("sigmoid", x), g.add("const", imm=0.01)), g.add("const", imm=0.995)))
+    sm = g.add("sum", y)
+    am = g.add("argmax", y)
+    return SpecProgram(g.nodes, y, (lo, hi, pr, sm, am), ("rowvec",))
