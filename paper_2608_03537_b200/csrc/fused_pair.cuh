@@ -735,18 +735,145 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
       } else if constexpr (EPI == EPI_PROGRAM) {
-        // ---------------- epilogue given as data: the stage program's passes over the TMEM-resident x (Sec. 3, Sec. 5.3)
+        // ---------------- epilogue given as data: the stage program's passes over the TMEM-resident x (Sec. 3, Sec. 5.3).
+        // ONE interpreter loop (one copy of every operation's code: the kernel is instruction-fetch bound otherwise)
+        // runs the pass's micro-instruction stream on each 32-column fragment: v is the working fragment, x the resident one.
+        static_assert(ESUB == 1, "stage programs run on single-unit tiles");
         const StageProgram& sp = p.program;
         float sc[kStageMaxScalars];  // this row's scalars (reduction results and arithmetic on them)
 #pragma unroll
         for (int i = 0; i < kStageMaxScalars; ++i) sc[i] = 0.f;
         const float* vecs[3] = {s_bias, s_gamma, s_beta};
-        // one chain instruction on a 32-column fragment; col0 = first global column, lc = first CTA-local column
-        auto run_chain = [&](const ChainInstr* code, int n, float (&v)[32], int lc, int col0, const uint32_t* res16) {
-          for (int i = 0; i < n; ++i) {
-            const ChainInstr ci = code[i];
-            const int op = ci.op;
-            if (op < COMFUSE_OP_ADD) {  // unary
+        float racc[kStageMaxRed];  // thread-local partials (value; column for an arg max); indexed at run time
+        int ridx[kStageMaxRed];
+#pragma unroll 1
+        for (int r = 0; r < kStageMaxRed; ++r) {
+          const int op = r < sp.n_red ? sp.red[r].op : COMFUSE_OP_RED_SUM;
+          racc[r] = op == COMFUSE_OP_RED_PROD ? 1.f : (op == COMFUSE_OP_RED_MAX || op == COMFUSE_OP_RED_ARGMAX) ? -INFINITY
+                    : op == COMFUSE_OP_RED_MIN ? INFINITY : 0.f;
+          ridx[r] = 0x7FFFFFFF;
+        }
+        auto scalar_get = [&](int kind, int ix, float imm) {
+          float sv = imm;
+          if (kind == CHO_SCALAR) {
+#pragma unroll
+            for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ix) ? sc[q] : sv;
+          }
+          return sv;
+        };
+        auto scalar_set = [&](int ix, float val) {
+#pragma unroll
+          for (int q = 0; q < kStageMaxScalars; ++q)
+            if (q == ix) sc[q] = val;
+        };
+        wait_accumulator(0);
+        const uint32_t taddr = tmem_of(0);
+        constexpr int kFrags = 2 * (BN / 64) / EPW;  // this thread's 32-column fragments of the tile
+        uint32_t r32[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r32[j] = 0u;
+        uint32_t ybox = 0, ybar = 0;
+
+#pragma unroll 1
+        for (int pass = 0; pass < sp.n_passes; ++pass) {
+          const int i0 = sp.pass_off[pass], i1 = sp.pass_off[pass + 1];
+#pragma unroll 1
+          for (int f = 0; f < kFrags; ++f) {
+            const int g = h + EPW * (f >> 1), half = f & 1;
+            const int lc = g * 64 + half * 32;  // first CTA-local column of the fragment
+            const int col0 = ncta0 + lc;
+            if (pass == 0 && half == 0 && has_res) {
+              // the residual box of this group rides the operand ring (one stage per warp pair and group)
+              mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
+              rfull_bits ^= 1u << ring.stage;
+              __syncwarp();
+              load_residual(smem_base + ring.stage * Cfg::STAGE_BYTES, h, r32);
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_rdone(ring.stage));
+              ring.advance();
+            }
+            float v[32], x[32];
+            {
+              uint32_t vb[32];
+              tmem_ld_32cols(taddr + lc, vb);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(vb[j]); x[j] = v[j]; }
+            }
+#pragma unroll 1
+            for (int i = i0; i < i1; ++i) {
+              const ChainInstr ci = sp.code[i];
+              const int op = ci.op;
+              if (op >= COMFUSE_OP_ADD && op <= kChainRdiv) {
+                // ---- binary: materialise the operand of the fragment, then apply
+                float o[32];
+                switch (ci.operand) {
+                  case CHO_SCALAR: {
+                    const float sv = scalar_get(CHO_SCALAR, ci.index, 0.f);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = sv;
+                    break;
+                  }
+                  case CHO_ROWVEC: {
+                    const float4* v4 = reinterpret_cast<const float4*>(vecs[ci.index] + lc);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                      const float4 t4 = v4[j];
+                      o[4 * j] = t4.x; o[4 * j + 1] = t4.y; o[4 * j + 2] = t4.z; o[4 * j + 3] = t4.w;
+                    }
+                    break;
+                  }
+                  case CHO_RESIDUAL:
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                      const float2 t2 = bf16x2_to_f2(half ? r32[16 + j] : r32[j]);
+                      o[2 * j] = t2.x; o[2 * j + 1] = t2.y;
+                    }
+                    break;
+                  case CHO_MASK:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;
+                    break;
+                  default:  // CHO_CONST
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = ci.imm;
+                    break;
+                }
+                switch (op) {
+                  case COMFUSE_OP_ADD:
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) { const float2 t = add2(make_float2(v[j], v[j + 1]), make_float2(o[j], o[j + 1])); v[j] = t.x; v[j + 1] = t.y; }
+                    break;
+                  case COMFUSE_OP_SUB:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = v[j] - o[j];
+                    break;
+                  case COMFUSE_OP_MUL:
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) { const float2 t = mul2(make_float2(v[j], v[j + 1]), make_float2(o[j], o[j + 1])); v[j] = t.x; v[j + 1] = t.y; }
+                    break;
+                  case COMFUSE_OP_DIV:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __fdividef(v[j], o[j]);
+                    break;
+                  case COMFUSE_OP_MAX:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], o[j]);
+                    break;
+                  case COMFUSE_OP_MIN:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = fminf(v[j], o[j]);
+                    break;
+                  case kChainRsub:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = o[j] - v[j];
+                    break;
+                  default:  // kChainRdiv
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __fdividef(o[j], v[j]);
+                    break;
+                }
+                continue;
+              }
               switch (op) {
                 case COMFUSE_OP_NEG:
 #pragma unroll
@@ -758,11 +885,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   break;
                 case COMFUSE_OP_SQUARE:
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) v[j] = v[j] * v[j];
+                  for (int j = 0; j < 32; j += 2) { const float2 t = mul2(make_float2(v[j], v[j + 1]), make_float2(v[j], v[j + 1])); v[j] = t.x; v[j + 1] = t.y; }
                   break;
                 case COMFUSE_OP_SQRT:
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) v[j] = sqrtf(v[j]);
+                  for (int j = 0; j < 32; ++j) v[j] = __fsqrt_rn(v[j]);
                   break;
                 case COMFUSE_OP_RSQRT:
 #pragma unroll
@@ -770,7 +897,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   break;
                 case COMFUSE_OP_RECIP:
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) v[j] = __frcp_rn(v[j]);
+                  for (int j = 0; j < 32; ++j) v[j] = __fdividef(1.f, v[j]);
                   break;
                 case COMFUSE_OP_EXP:
 #pragma unroll
@@ -782,7 +909,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   break;
                 case COMFUSE_OP_TANH:  // 1 - 2 / (1 + e^(2x)): absolute error about 1e-7 (tanh.approx has 2^-11 relative)
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) v[j] = 1.f - 2.f * __frcp_rn(1.f + ex2_approx(2.8853900817779268f * v[j]));
+                  for (int j = 0; j < 32; ++j) v[j] = 1.f - 2.f * __fdividef(1.f, 1.f + ex2_approx(2.8853900817779268f * v[j]));
                   break;
                 case COMFUSE_OP_RELU:
 #pragma unroll
@@ -795,159 +922,129 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     v[j] = gz.x; v[j + 1] = gz.y;
                   }
                   break;
-                default:  // COMFUSE_OP_SIGMOID
+                case COMFUSE_OP_SIGMOID:
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) v[j] = __frcp_rn(1.f + ex2_approx(-1.4426950408889634f * v[j]));
+                  for (int j = 0; j < 32; ++j) v[j] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * v[j]));
                   break;
-              }
-              continue;
-            }
-            // binary: materialise the operand fragment, then apply
-            float o[32];
-            switch (ci.operand) {
-              case CHO_SCALAR: {
-                float sv = 0.f;
+                case kChainXsave: {  // x = v; written back over the accumulator when a later pass reads it
 #pragma unroll
-                for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ci.index) ? sc[q] : sv;
+                  for (int j = 0; j < 32; ++j) x[j] = v[j];
+                  if (sp.n_passes > 1) {
+                    uint32_t vb[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) o[j] = sv;
-                break;
-              }
-              case CHO_ROWVEC: {
-                const float4* v4 = reinterpret_cast<const float4*>(vecs[ci.index] + lc);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float4 t4 = v4[j];
-                  o[4 * j] = t4.x; o[4 * j + 1] = t4.y; o[4 * j + 2] = t4.z; o[4 * j + 3] = t4.w;
+                    for (int j = 0; j < 32; ++j) vb[j] = __float_as_uint(v[j]);
+                    tmem_st_32cols(taddr + lc, vb);
+                  }
+                  break;
                 }
-                break;
-              }
-              case CHO_RESIDUAL:
+                case kChainXload:
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  const float2 t2 = bf16x2_to_f2(res16[j]);
-                  o[2 * j] = t2.x; o[2 * j + 1] = t2.y;
+                  for (int j = 0; j < 32; ++j) v[j] = x[j];
+                  break;
+                case kChainAcc: {  // thread-local partial of reduction ci.index over v
+                  const int r = ci.index;
+                  float a = racc[r];
+                  switch (sp.red[r].op) {
+                    case COMFUSE_OP_RED_SUM:
+                    case COMFUSE_OP_RED_MEAN: {
+                      float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+#pragma unroll
+                      for (int j = 0; j < 32; j += 4) { t0 += v[j]; t1 += v[j + 1]; t2 += v[j + 2]; t3 += v[j + 3]; }
+                      a += (t0 + t1) + (t2 + t3);
+                      break;
+                    }
+                    case COMFUSE_OP_RED_MIN: {
+                      float t0 = v[0], t1 = v[1], t2 = v[2], t3 = v[3];
+#pragma unroll
+                      for (int j = 4; j < 32; j += 4) { t0 = fminf(t0, v[j]); t1 = fminf(t1, v[j + 1]); t2 = fminf(t2, v[j + 2]); t3 = fminf(t3, v[j + 3]); }
+                      a = fminf(a, fminf(fminf(t0, t1), fminf(t2, t3)));
+                      break;
+                    }
+                    case COMFUSE_OP_RED_PROD: {
+                      float t0 = 1.f, t1 = 1.f, t2 = 1.f, t3 = 1.f;
+#pragma unroll
+                      for (int j = 0; j < 32; j += 4) { t0 *= v[j]; t1 *= v[j + 1]; t2 *= v[j + 2]; t3 *= v[j + 3]; }
+                      a *= (t0 * t1) * (t2 * t3);
+                      break;
+                    }
+                    default: {  // max and arg max: the fragment's maximum by a tree; for the arg max its first column
+                      // (columns rise from fragment to fragment, a strict compare against the running best keeps the lowest)
+                      float t0 = v[0], t1 = v[1];
+#pragma unroll
+                      for (int j = 2; j < 30; j += 4) { t0 = max3(t0, v[j], v[j + 1]); t1 = max3(t1, v[j + 2], v[j + 3]); }
+                      const float fm = max3(t0, t1, fmaxf(v[30], v[31]));
+                      if (sp.red[r].op == COMFUSE_OP_RED_ARGMAX) {
+                        if (fm > a) {
+                          int ix = 31;
+#pragma unroll
+                          for (int j = 30; j >= 0; --j) ix = (v[j] == fm) ? j : ix;
+                          ridx[r] = col0 + ix;
+                          a = fm;
+                        }
+                      } else {
+                        a = fmaxf(a, fm);
+                      }
+                      break;
+                    }
+                  }
+                  racc[r] = a;
+                  break;
                 }
-                break;
-              case CHO_MASK:
+                default: {  // kChainEmit: round v once and put this half of the row into the warp's staging box
+                  if (half == 0) {
+                    if (Cfg::RING_STAGING && in_ring) {
+                      ybox = ring_box(warp - 2, ring_k);
+                      ybar = bar_ylast(warp - 2, ring_k);
+                      ++ring_k;
+                    } else {
+                      const uint32_t sel = ybox_sel;
+                      ybox = ybox0 + sel * Cfg::WARP_BOX_BYTES;
+                      ybar = bar_yfull(warp - 2, sel);
+                      if (++ybox_sel == Cfg::YBOXES) ybox_sel = 0;
+                      mbar_wait<false>(bar_yfree(warp - 2, sel), ((ybox_count / Cfg::YBOXES) & 1u) ^ 1u, w);
+                      ++ybox_count;
+                    }
+                    __syncwarp();
+                  }
 #pragma unroll
-                for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;
-                break;
-              default:  // CHO_CONST
-#pragma unroll
-                for (int j = 0; j < 32; ++j) o[j] = ci.imm;
-                break;
-            }
-            switch (op) {
-              case COMFUSE_OP_ADD:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = v[j] + o[j];
-                break;
-              case COMFUSE_OP_SUB:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = v[j] - o[j];
-                break;
-              case COMFUSE_OP_MUL:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = v[j] * o[j];
-                break;
-              case COMFUSE_OP_DIV:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __fdividef(v[j], o[j]);
-                break;
-              case COMFUSE_OP_MAX:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], o[j]);
-                break;
-              case COMFUSE_OP_MIN:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = fminf(v[j], o[j]);
-                break;
-              case kChainRsub:
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = o[j] - v[j];
-                break;
-              default:  // kChainRdiv
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __fdividef(o[j], v[j]);
-                break;
+                  for (int q = 0; q < 4; ++q) {
+                    const uint32_t a = ybox + swz128(lane, half * 4 + q);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pack_bf16x2_rn(v[8 * q], v[8 * q + 1])),
+                                 "r"(pack_bf16x2_rn(v[8 * q + 2], v[8 * q + 3])), "r"(pack_bf16x2_rn(v[8 * q + 4], v[8 * q + 5])),
+                                 "r"(pack_bf16x2_rn(v[8 * q + 6], v[8 * q + 7]))
+                                 : "memory");
+                  }
+                  if (half == 1) {
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(ybar);
+                  }
+                  break;
+                }
+              }
             }
           }
-        };
-        // thread-local partials of the reductions (value; column for an arg max); indexed at run time (local memory)
-        float racc[kStageMaxRed];
-        int ridx[kStageMaxRed];
-        auto red_init = [&](int r) {
-          const int op = r < sp.n_red ? sp.red[r].op : COMFUSE_OP_RED_SUM;
-          racc[r] = op == COMFUSE_OP_RED_PROD ? 1.f : (op == COMFUSE_OP_RED_MAX || op == COMFUSE_OP_RED_ARGMAX) ? -INFINITY
-                    : op == COMFUSE_OP_RED_MIN ? INFINITY : 0.f;
-          ridx[r] = 0x7FFFFFFF;
-        };
-        auto red_accumulate = [&](int r, const float (&u)[32], int col0) {
-          float a = racc[r];
-          switch (sp.red[r].op) {
-            case COMFUSE_OP_RED_SUM:
-            case COMFUSE_OP_RED_MEAN: {
-              float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) { t0 += u[j]; t1 += u[j + 1]; t2 += u[j + 2]; t3 += u[j + 3]; }
-              a += (t0 + t1) + (t2 + t3);
-              break;
-            }
-            case COMFUSE_OP_RED_MAX:
-#pragma unroll
-              for (int j = 0; j < 32; ++j) a = fmaxf(a, u[j]);
-              break;
-            case COMFUSE_OP_RED_MIN:
-#pragma unroll
-              for (int j = 0; j < 32; ++j) a = fminf(a, u[j]);
-              break;
-            case COMFUSE_OP_RED_PROD:
-#pragma unroll
-              for (int j = 0; j < 32; ++j) a *= u[j];
-              break;
-            default: {  // arg max: columns rise, a strict compare keeps the lowest
-              int ix = ridx[r];
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (u[j] > a) { a = u[j]; ix = col0 + j; }
-              ridx[r] = ix;
-              break;
-            }
-          }
-          racc[r] = a;
-        };
-        // cluster-wide merge of reduction r; the result becomes scalar sp.red[r].dst
-        auto red_merge = [&](int r) {
-          const int op = sp.red[r].op;
-          float2 tot;
-          const float2 mine = make_float2(racc[r], __int_as_float(ridx[r]));
-          if (op == COMFUSE_OP_RED_ARGMAX)
-            tot = cluster_row_reduce<CN, MergeArgmax, EPW>(mine, kThreadCount, MergeArgmax(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
-                                                          w, 2u, pm, p.leader_reduce != 0);
-          else
-            tot = cluster_row_reduce<CN, MergeByOp, EPW>(mine, kThreadCount, MergeByOp{op}, s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
-                                                        w, 2u, pm, p.leader_reduce != 0);
-          float val = op == COMFUSE_OP_RED_ARGMAX ? static_cast<float>(__float_as_int(tot.y)) : tot.x;
-          if (op == COMFUSE_OP_RED_MEAN) val *= 1.f / static_cast<float>(CN * BN);
-#pragma unroll
-          for (int q = 0; q < kStageMaxScalars; ++q)
-            if (q == sp.red[r].dst) sc[q] = val;
-        };
-        auto scalar_get = [&](int kind, int ix, float imm) {
-          float sv = imm;
-          if (kind == CHO_SCALAR) {
-#pragma unroll
-            for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ix) ? sc[q] : sv;
-          }
-          return sv;
-        };
-        auto boundary = [&](int pass) {
-          // merges of the pass's reductions in program order (every CTA of the group makes the same calls), then the
-          // per-row arithmetic that depends on them
+          if (pass == 0) tmem_st_wait();
+          if (pass == sp.n_passes - 1) release_accumulator(0);
+          // ---- stage boundary: merges of the pass's reductions in program order (every CTA of the group makes the same
+          // calls), then the per-row arithmetic that depends on them
 #pragma unroll 1
-          for (int r = 0; r < sp.n_red; ++r)
-            if (sp.red[r].pass == pass) red_merge(r);
+          for (int r = 0; r < sp.n_red; ++r) {
+            if (sp.red[r].pass != pass) continue;
+            const int op = sp.red[r].op;
+            float2 tot;
+            const float2 mine = make_float2(racc[r], __int_as_float(ridx[r]));
+            if (op == COMFUSE_OP_RED_ARGMAX)
+              tot = cluster_row_reduce<CN, MergeArgmax, EPW>(mine, kThreadCount, MergeArgmax(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
+                                                            w, 2u, pm, p.leader_reduce != 0);
+            else
+              tot = cluster_row_reduce<CN, MergeByOp, EPW>(mine, kThreadCount, MergeByOp{op}, s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
+                                                          w, 2u, pm, p.leader_reduce != 0);
+            float val = op == COMFUSE_OP_RED_ARGMAX ? static_cast<float>(__float_as_int(tot.y)) : tot.x;
+            if (op == COMFUSE_OP_RED_MEAN) val *= 1.f / static_cast<float>(CN * BN);
+            scalar_set(sp.red[r].dst, val);
+          }
+#pragma unroll 1
           for (int i = 0; i < sp.n_scalar_instr; ++i) {
             const ScalarInstr si = sp.sc[i];
             if (si.after_pass != pass) continue;
@@ -974,79 +1071,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               case COMFUSE_OP_MAX: rv = fmaxf(a, bq); break;
               default: rv = fminf(a, bq); break;
             }
-#pragma unroll
-            for (int q = 0; q < kStageMaxScalars; ++q)
-              if (q == si.dst) sc[q] = rv;
+            scalar_set(si.dst, rv);
           }
-        };
-#pragma unroll 1
-        for (int r = 0; r < kStageMaxRed; ++r) red_init(r);
-
-        for (int pass = 0; pass < sp.n_passes; ++pass) {
-          const bool is_terminal = pass == sp.terminal_pass;
-#pragma unroll
-          for (int sub = 0; sub < ESUB; ++sub) {
-            if (pass == 0) wait_accumulator(sub);
-            const int W = unit_width(sub);
-            const int lsub = unit_lg0(sub) * 64;
-            const uint32_t taddr = tmem_of(sub);
-            for (int g = h; g < W / 64; g += EPW) {
-              uint32_t r32[32];
-              if (pass == 0) {
-                if (has_res) {
-                  mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
-                  rfull_bits ^= 1u << ring.stage;
-                  __syncwarp();
-                  load_residual(smem_base + ring.stage * Cfg::STAGE_BYTES, h, r32);
-                  __syncwarp();
-                  if (lane == 0) mbar_arrive(bar_rdone(ring.stage));
-                  ring.advance();
-                } else {
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) r32[j] = 0u;
-                }
-              }
-              uint32_t pk[32];
-#pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const int lc = lsub + g * 64 + half * 32;
-                const int col0 = ncta0 + lc;
-                uint32_t vb[32];
-                tmem_ld_32cols(taddr + g * 64 + half * 32, vb);
-                float x[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(vb[j]);
-                if (pass == 0) {
-                  run_chain(sp.entry, sp.n_entry, x, lc, col0, r32 + half * 16);
-#pragma unroll
-                  for (int j = 0; j < 32; ++j) vb[j] = __float_as_uint(x[j]);
-                  if (sp.n_passes > 1 || !is_terminal) tmem_st_32cols(taddr + g * 64 + half * 32, vb);
-                }
-#pragma unroll 1
-                for (int r = 0; r < sp.n_red; ++r) {
-                  if (sp.red[r].pass == pass && !sp.red[r].on_terminal) {
-                    float u[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) u[j] = x[j];
-                    run_chain(sp.chains + sp.red[r].chain_off, sp.red[r].chain_len, u, lc, col0, nullptr);
-                    red_accumulate(r, u, col0);
-                  }
-                }
-                if (is_terminal) {
-                  run_chain(sp.fin, sp.n_final, x, lc, col0, nullptr);
-#pragma unroll 1
-                  for (int r = 0; r < sp.n_red; ++r)
-                    if (sp.red[r].on_terminal) red_accumulate(r, x, col0);
-#pragma unroll
-                  for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_bf16x2_rn(x[2 * j], x[2 * j + 1]);
-                }
-              }
-              if (is_terminal) store_box(pk);
-            }
-            if (pass == sp.n_passes - 1) release_accumulator(sub);
-          }
-          if (pass == 0) tmem_st_wait();
-          boundary(pass);
         }
         if (crank == 0 && h == 0 && valid) {
           const long long o = static_cast<long long>(b) * p.M + grow;

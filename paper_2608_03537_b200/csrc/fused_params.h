@@ -27,8 +27,13 @@ enum ChainOperand : uint8_t {
   CHO_MASK       // causal mask: 0 where column <= row, -inf above the diagonal
 };
 // chain opcodes: the comfuse_op_t values of the unary / binary nodes, plus the reversed non-commutative forms
-constexpr int kChainRsub = 64;  // v = operand - v
-constexpr int kChainRdiv = 65;  // v = operand / v
+constexpr int kChainRsub = 38;  // v = operand - v
+constexpr int kChainRdiv = 39;  // v = operand / v
+// micro-instructions of a pass's stream (besides the chain operations)
+constexpr int kChainXsave = 66;  // x = v (pass 0, after the entry chain)
+constexpr int kChainXload = 67;  // v = x
+constexpr int kChainAcc = 68;    // accumulate v into the thread-local partial of reduction `index`
+constexpr int kChainEmit = 69;   // round v and stage it for the output store
 
 struct ChainInstr {
   uint8_t op;
@@ -40,11 +45,8 @@ struct ChainInstr {
 struct StageReduction {
   uint8_t pass;        // the pass in which its input is available
   uint8_t op;          // comfuse_op_t of the reduction (sum, mean, max, min, prod, argmax)
-  uint8_t chain_off;   // its input chain: chains[chain_off .. chain_off + chain_len), applied to x
-  uint8_t chain_len;
   uint8_t on_terminal; // input is y itself: accumulated in the terminal's pass from the unrounded y
   uint8_t dst;         // per-row scalar it defines
-  uint8_t pad[2];
 };
 
 struct ScalarInstr {   // per-row arithmetic at a stage boundary: s[dst] = op(a, b)
@@ -64,15 +66,18 @@ struct StageRowOutput {
   uint8_t pad[6];
 };
 
-constexpr int kStageMaxEntry = 12, kStageMaxFinal = 16, kStageMaxChains = 24, kStageMaxRed = 6, kStageMaxScalarInstr = 12,
-              kStageMaxScalars = 16, kStageMaxRowOut = 6, kStageMaxPasses = 4;
+constexpr int kStageMaxCode = 80, kStageMaxRed = 6, kStageMaxScalarInstr = 12, kStageMaxScalars = 16, kStageMaxRowOut = 6,
+              kStageMaxPasses = 4;
 
 struct StageProgram {
-  uint8_t n_entry, n_final, n_red, n_scalar_instr;
-  uint8_t n_passes, terminal_pass, n_row_out, pad;
-  ChainInstr entry[kStageMaxEntry];
-  ChainInstr fin[kStageMaxFinal];
-  ChainInstr chains[kStageMaxChains];
+  uint8_t n_red, n_scalar_instr, n_passes, terminal_pass;
+  uint8_t n_row_out, pad[3];
+  // per pass, the micro-instruction stream run on every 32-column fragment: code[pass_off[s] .. pass_off[s + 1]).
+  // pass 0: entry chain, XSAVE; every pass: per reduction of the pass (XLOAD if v was changed,) its chain, ACC; the
+  // terminal's pass: (XLOAD,) final chain, ACC of the reductions on y, EMIT.
+  uint8_t pass_off[kStageMaxPasses + 1];
+  uint8_t pad2[3];
+  ChainInstr code[kStageMaxCode];
   StageReduction red[kStageMaxRed];
   ScalarInstr sc[kStageMaxScalarInstr];
   StageRowOutput out[kStageMaxRowOut];

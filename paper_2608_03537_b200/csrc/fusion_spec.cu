@@ -378,8 +378,30 @@ struct StageLowering {
   const Analysis& an;
   StageBinding& bind;
   std::vector<int> scalar_of;  // per node: its per-row scalar index, -1 = none
+  std::vector<int> recip_of;   // per node: the scalar holding its reciprocal, -1 = not needed yet
   int x_root = -1;
-  explicit StageLowering(const Analysis& a, StageBinding& b) : an(a), bind(b), scalar_of(a.n, -1) {}
+  int scalars = 0;             // per-row scalars allocated so far
+  StageProgram* sp = nullptr;
+  explicit StageLowering(const Analysis& a, StageBinding& b) : an(a), bind(b), scalar_of(a.n, -1), recip_of(a.n, -1) {}
+
+  // v / s with s a per-row value (or constant) becomes v * (1 / s): one reciprocal per row instead of one per element
+  bool divide_by(int k, ChainInstr& ci) {
+    if (ci.operand == CHO_CONST) { ci.op = COMFUSE_OP_MUL; ci.imm = 1.f / ci.imm; return true; }
+    if (ci.operand != CHO_SCALAR) { ci.op = COMFUSE_OP_DIV; return true; }
+    if (recip_of[k] < 0) {
+      if (scalars >= kStageMaxScalars || sp->n_scalar_instr >= kStageMaxScalarInstr || an.stage[k] < 1) return false;
+      ScalarInstr& si = sp->sc[sp->n_scalar_instr++];
+      si.after_pass = static_cast<uint8_t>(an.stage[k] - 1);
+      si.op = COMFUSE_OP_RECIP;
+      si.dst = static_cast<uint8_t>(scalars);
+      si.a_kind = CHO_SCALAR; si.a = static_cast<uint8_t>(scalar_of[k]); si.a_imm = 0.f;
+      si.b_kind = CHO_CONST; si.b = 0; si.b_imm = 0.f;
+      recip_of[k] = scalars++;
+    }
+    ci.op = COMFUSE_OP_MUL;
+    ci.index = static_cast<int16_t>(recip_of[k]);
+    return true;
+  }
 
   bool tensor(int k) const { return an.type[k] == T_TENSOR; }
   // can node k be the right-hand operand of a chain instruction?
@@ -437,6 +459,7 @@ struct StageLowering {
     if (carrier(a) && !carrier(b) && operand(b, entry_mode, ci)) {
       if (!chain(a, entry_mode, out)) return false;
       ci.op = static_cast<uint8_t>(nd.op);
+      if (nd.op == COMFUSE_OP_DIV && !divide_by(b, ci)) return false;
       out.push_back(ci);
       return true;
     }
@@ -455,6 +478,7 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
   if (!an.row_outputs.empty() && an.row_outputs.size() > static_cast<size_t>(kStageMaxRowOut)) return false;
   if (an.type[an.terminal] != T_TENSOR) return false;
   StageLowering L(an, bind);
+  L.sp = &sp;
   const int n = an.n;
   // the resident tensor: the one stage-0 tensor that later stages read
   int first_acc = -1;
@@ -476,16 +500,17 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
   if (first_acc < 0) return false;
   L.x_root = cand.size() == 1 ? cand[0] : (an.stage[an.terminal] == 0 ? an.terminal : first_acc);
   // stage 0: acc -> x
-  std::vector<ChainInstr> code;
-  if (!L.chain(L.x_root, true, code) || code.size() > static_cast<size_t>(kStageMaxEntry)) return false;
-  sp.n_entry = static_cast<uint8_t>(code.size());
-  for (size_t i = 0; i < code.size(); ++i) sp.entry[i] = code[i];
+  std::vector<ChainInstr> entry, fin;
+  std::vector<std::vector<ChainInstr>> red_chain;
+  if (!L.chain(L.x_root, true, entry)) return false;
   // reductions and per-row arithmetic, in node order
-  int scalars = 0, pool = 0, max_pass = an.stage[an.terminal];
+  int max_pass = an.stage[an.terminal];
+  int& scalars = L.scalars;
   for (int k = 0; k < n; ++k) {
     if (!an.live[k] || an.type[k] != T_ROW) continue;
     const comfuse_spec_node_t& nd = an.nodes[k];
     if (scalars >= kStageMaxScalars) return false;
+    const int my = scalars++;  // before the chains below, which may allocate reciprocals
     if (is_reduce(nd.op)) {
       if (is_topk(nd.op) || sp.n_red >= kStageMaxRed) return false;
       const int e = nd.in0;
@@ -493,16 +518,10 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
       StageReduction& r = sp.red[sp.n_red];
       r.op = static_cast<uint8_t>(nd.op);
       r.pass = static_cast<uint8_t>(an.stage[e]);
-      r.dst = static_cast<uint8_t>(scalars);
-      if (e == an.terminal) {
-        r.on_terminal = 1;
-      } else {
-        code.clear();
-        if (!L.chain(e, false, code) || pool + code.size() > static_cast<size_t>(kStageMaxChains)) return false;
-        r.chain_off = static_cast<uint8_t>(pool);
-        r.chain_len = static_cast<uint8_t>(code.size());
-        for (const ChainInstr& c : code) sp.chains[pool++] = c;
-      }
+      r.dst = static_cast<uint8_t>(my);
+      red_chain.emplace_back();
+      if (e == an.terminal) r.on_terminal = 1;
+      else if (!L.chain(e, false, red_chain.back())) return false;
       if (r.pass > max_pass) max_pass = r.pass;
       ++sp.n_red;
     } else {
@@ -510,7 +529,7 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
       ScalarInstr& si = sp.sc[sp.n_scalar_instr++];
       si.after_pass = static_cast<uint8_t>(an.stage[k] - 1);
       si.op = static_cast<uint8_t>(nd.op);
-      si.dst = static_cast<uint8_t>(scalars);
+      si.dst = static_cast<uint8_t>(my);
       auto set = [&](int e, uint8_t& kind, uint8_t& ix, float& imm) {
         if (e < 0) { kind = CHO_CONST; ix = 0; imm = 0.f; return true; }
         if (an.type[e] == T_CONST) { kind = CHO_CONST; ix = 0; imm = an.cval[e]; return true; }
@@ -520,19 +539,45 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
       };
       if (!set(nd.in0, si.a_kind, si.a, si.a_imm) || !set(nd.in1, si.b_kind, si.b, si.b_imm)) return false;
     }
-    L.scalar_of[k] = scalars++;
+    L.scalar_of[k] = my;
   }
   // the terminal: x -> y
-  code.clear();
-  if (!L.chain(an.terminal, false, code) || code.size() > static_cast<size_t>(kStageMaxFinal)) return false;
-  sp.n_final = static_cast<uint8_t>(code.size());
-  for (size_t i = 0; i < code.size(); ++i) sp.fin[i] = code[i];
+  if (!L.chain(an.terminal, false, fin)) return false;
   sp.terminal_pass = static_cast<uint8_t>(an.stage[an.terminal]);
   if (max_pass + 1 > kStageMaxPasses) return false;
   sp.n_passes = static_cast<uint8_t>(max_pass + 1);
-  // a reduction on y is accumulated in the terminal's pass; anything the terminal needs must be merged before it
+  // a reduction on y is accumulated in the terminal's pass
   for (int r = 0; r < sp.n_red; ++r)
     if (sp.red[r].on_terminal) sp.red[r].pass = sp.terminal_pass;
+  // the micro-instruction stream of every pass
+  int nc = 0;
+  bool ok = true;
+  auto emit = [&](ChainInstr c) { if (nc < kStageMaxCode) sp.code[nc++] = c; else ok = false; };
+  auto micro = [&](int op, int index = 0) { emit(ChainInstr{static_cast<uint8_t>(op), CHO_NONE, static_cast<int16_t>(index), 0.f}); };
+  for (int pass = 0; pass < sp.n_passes; ++pass) {
+    sp.pass_off[pass] = static_cast<uint8_t>(nc);
+    bool v_is_x = true;  // at the start of a later pass v = x as loaded from TMEM
+    if (pass == 0) {
+      for (const ChainInstr& c : entry) emit(c);
+      micro(kChainXsave);
+    }
+    for (int r = 0; r < sp.n_red; ++r) {
+      if (sp.red[r].pass != pass || sp.red[r].on_terminal) continue;
+      if (!v_is_x) micro(kChainXload);
+      for (const ChainInstr& c : red_chain[r]) emit(c);
+      v_is_x = red_chain[r].empty();
+      micro(kChainAcc, r);
+    }
+    if (pass == sp.terminal_pass) {
+      if (!v_is_x) micro(kChainXload);
+      for (const ChainInstr& c : fin) emit(c);
+      for (int r = 0; r < sp.n_red; ++r)
+        if (sp.red[r].on_terminal) micro(kChainAcc, r);
+      micro(kChainEmit);
+    }
+  }
+  sp.pass_off[sp.n_passes] = static_cast<uint8_t>(nc);
+  if (!ok) return false;
   for (size_t r = 0; r < an.row_outputs.size(); ++r) {
     const int q = an.row_outputs[r];
     if (an.type[q] != T_ROW || L.scalar_of[q] < 0) return false;
@@ -654,6 +699,29 @@ comfuse_gemm_desc_t fused_desc(const comfuse_gemm_shape_t& s, const FusedMatch& 
   return d;
 }
 
+// Which interpreter for a program both can run?  Both cost roughly a fixed time per element and executed instruction
+// (measured on four programs on one B200: about 0.36 ns per micro-instruction on-chip -- 8 epilogue warps per SM, the
+// chains re-run in every pass, transcendental operations counted three times -- against 0.9 ns per instruction plus 0.6 ns for
+// the bf16 round trip of Z in the row program, which has every SM's full occupancy).  A coarse model, good enough to send
+// exponential-heavy three-pass programs to the row program and the rest on-chip.
+bool on_chip_is_cheaper(const Analysis& an, const StageProgram& sp, int N) {
+  RowProgram P;
+  std::memset(&P, 0, sizeof(P));
+  int ni = 0, ns = 0;
+  if (lower_row_program(an, N, P, ni, ns) != COMFUSE_OK) return true;  // the row program cannot run it at all
+  float units = 0.f;
+  for (int pass = 0; pass < sp.n_passes; ++pass) {
+    units += 2.f;  // fragment load, loop overhead
+    for (int i = sp.pass_off[pass]; i < sp.pass_off[pass + 1]; ++i) {
+      const int op = sp.code[i].op;
+      const bool transcendental = op == COMFUSE_OP_EXP || op == COMFUSE_OP_LOG || op == COMFUSE_OP_TANH || op == COMFUSE_OP_GELU_TANH ||
+                                  op == COMFUSE_OP_SIGMOID || op == COMFUSE_OP_DIV || op == kChainRdiv || op == COMFUSE_OP_RECIP;
+      units += transcendental ? 3.f : 1.f;
+    }
+  }
+  return 0.36f * units <= 0.9f * static_cast<float>(ni) + 0.6f;
+}
+
 struct Decision {
   Analysis an;
   FusedMatch match;
@@ -684,6 +752,7 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
     const void* none[3] = {nullptr, nullptr, nullptr};
     dc.on_chip = run_fused_program(shape->batch, shape->M, shape->N, shape->K, 0, 0, 0, 0, 0, 0, nullptr, nullptr, nullptr, dc.stage_prog,
                                    none, nullptr, 0, nullptr, true) == COMFUSE_OK;
+    if (dc.on_chip && want_fused == 1 && !on_chip_is_cheaper(dc.an, dc.stage_prog, shape->N)) dc.on_chip = false;
   }
   return COMFUSE_OK;
 }
@@ -718,7 +787,7 @@ comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comf
   if (s != COMFUSE_OK) return s;
   plan->program_path = d2.on_chip ? COMFUSE_SPEC_PATH_FUSED_PROGRAM : COMFUSE_SPEC_PATH_ROW_PROGRAM;
   if (d2.on_chip) plan->n_passes = d2.stage_prog.n_passes;
-  if (!dc.fused) plan->path = plan->program_path;
+  if (!dc.fused) plan->path = dc.on_chip ? COMFUSE_SPEC_PATH_FUSED_PROGRAM : COMFUSE_SPEC_PATH_ROW_PROGRAM;
   // the row program (what `fused` = 0 runs) is described in any case
   RowProgram P;
   std::memset(&P, 0, sizeof(P));
