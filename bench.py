@@ -31,10 +31,11 @@ sys.path.insert(0, ROOT)
 import workloads as wl  # noqa: E402
 
 METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
-WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "a1": 5}   # a1: target attention, beyond the five named configurations
+# a1 (target attention) and p1 (an epilogue given as data, on-chip interpreter) lie beyond the five named configurations
+WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "a1": 5, "p1": 6}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
 # captures summarised under profiles/, in bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {"a1": 39_304_448, "c1": None, "c2": 70_159_872, "c3": 217_753_600, "c4": 512_653_312, "c5": 8_714_240}
+NCU_TRAFFIC_BYTES = {"p1": None, "a1": 39_304_448, "c1": None, "c2": 70_159_872, "c3": 217_753_600, "c4": 512_653_312, "c5": 8_714_240}
 
 
 def load_peaks():
@@ -105,6 +106,11 @@ def oracle_call(w, rows):
     """One evaluation of the fp64 oracle on `rows` of workload `w` (inputs already widened to fp64)."""
     from oracle import comfuse_oracle as orc
     t = w._f64
+    if w.kind == wl.KIND_GEMM_PROGRAM:
+        from oracle import fusion_spec_oracle as spo
+        pr = w.program
+        params = [t[f"p{k}"] if kd == "rowvec" else t[f"p{k}"][rows] for k, kd in enumerate(pr.param_kinds)]
+        return spo.gemm_spec(t["A"][rows], t["B"], pr.nodes, pr.terminal, params, pr.row_outputs)
     if w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION:
         return orc.b2b_softmax_attention(t["X"][0][rows], t["W1"][0], t["W2"][0], w.scalars["alpha"])
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
@@ -229,6 +235,11 @@ def run_comfuse(args):
     # rotation exceeds 3x the L2 capacity; weights and row vectors are shared (they are meant to be L2 resident)
     attention = w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION
     b2b = w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION)
+    program = w.kind == wl.KIND_GEMM_PROGRAM
+    if program:
+        spec = cf.make_spec(w.program.nodes, w.program.terminal, len(w.program.param_kinds), w.program.row_outputs)
+        pshape = cf.make_gemm_shape(1, w.dims["M"], w.dims["N"], w.dims["K"])
+        plan = cf.spec_plan(spec, pshape)
     act_names = {"A", "B"} if w.kind == wl.KIND_SCALE_MASK_SOFTMAX else ({"X", "W1", "W2"} if attention else {"A", "residual", "X"})
     base = {k: to_dev(v) for k, v in w.tensors.items()}
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
@@ -243,6 +254,9 @@ def run_comfuse(args):
         if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
             s["row_max"] = torch.zeros(out_shape[:-1], dtype=torch.float32, device=dev)
             s["row_argmax"] = torch.zeros(out_shape[:-1], dtype=torch.int32, device=dev)
+        if program:
+            s["row_out"] = [torch.zeros(d["M"], dtype=torch.int32 if w.program.nodes[r][0] == "argmax" else torch.float32, device=dev)
+                            for r in w.program.row_outputs]
         sets.append(s)
 
     # workspace (unfused path only)
@@ -253,6 +267,8 @@ def run_comfuse(args):
 
     if b2b:
         ws_bytes = cf.b2b_workspace_size(b2b_desc(fused))
+    elif program:
+        ws_bytes = cf.gemm_spec_workspace_size(spec, pshape, fused)
     else:
         kind = {wl.KIND_BIAS_RES_LAYERNORM: cf.EPI_BIAS_RES_LAYERNORM,
                 wl.KIND_BIAS_GELU_RES_RMSNORM_MAX: cf.EPI_BIAS_GELU_RES_RMSNORM_MAX,
@@ -263,7 +279,10 @@ def run_comfuse(args):
     ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
 
     def step(s, use_fused=fused, workspace=ws):
-        if attention:
+        if program:
+            cf.gemm_spec(s["A"], s["B"], s["Y"], spec, params=[s[f"p{k}"] for k in range(len(w.program.param_kinds))],
+                         row_out=s["row_out"], fused=use_fused, workspace=workspace)
+        elif attention:
             cf.b2b_attention(s["X"], s["W1"], s["W2"], s["Y"], alpha=w.scalars["alpha"], fused=use_fused, workspace=workspace)
         elif w.kind == wl.KIND_B2B_MLP_LAYERNORM:
             cf.b2b_gemm(s["X"], s["W1"], s["b1"], s["W2"], s["b2"], s["Y"], gamma=s.get("gamma"), beta=s.get("beta"),
@@ -354,7 +373,10 @@ def run_comfuse(args):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(name)
     roof["peak_source"] = f"of {peaks['source']} (burst figure, kernel timed alone)"
-    if b2b:
+    if program:
+        roof["kernel"] = {cf.SPEC_PATH_FUSED_KERNEL: "fused_pair_kernel (compiled kind)", cf.SPEC_PATH_FUSED_PROGRAM: "fused_pair_kernel<EPI_PROGRAM> (on-chip interpreter)",
+                          cf.SPEC_PATH_ROW_PROGRAM: "fused_pair_kernel<EPI_NONE> + row_program_kernel"}[plan.path if fused else cf.SPEC_PATH_ROW_PROGRAM]
+    elif b2b:
         roof["kernel"] = "b2b_pair_kernel"
     elif w.kind == wl.KIND_SCALE_MASK_SOFTMAX and d["K"] <= 256:
         roof["kernel"] = "softmax_rows_kernel"      # short K: score chunks computed twice, no cluster exchange
@@ -379,6 +401,8 @@ def run_comfuse(args):
             other = not fused
             if b2b:
                 ob = cf.b2b_workspace_size(b2b_desc(other))
+            elif program:
+                ob = cf.gemm_spec_workspace_size(spec, pshape, other)
             else:
                 desc.fused = int(other)
                 ob = cf.workspace_size(desc)
@@ -431,7 +455,17 @@ def run_comfuse(args):
     h2d = sum(t.numel() * 2 for t in host_in.values())
     d2h = host_out.numel() * 2
     s0 = sets[0]
-    if b2b:
+    if program:
+        # no host-buffer form of the program entry point: the step's activations are copied from pinned memory with
+        # stream copies around the same call, all inside the timed region
+        dA = torch.empty_like(s0["A"])
+
+        def e2e_step(i):
+            dA.copy_(host_in["A"], non_blocking=True)
+            cf.gemm_spec(dA, s0["B"], s0["Y"], spec, params=[s0[f"p{k}"] for k in range(len(w.program.param_kinds))],
+                         row_out=s0["row_out"], fused=fused, workspace=ws)
+            host_out.copy_(s0["Y"], non_blocking=True)
+    elif b2b:
         bdesc = b2b_desc(fused)
         staging = torch.empty(cf.b2b_host_staging_size(bdesc), dtype=torch.uint8, device=dev)
 
@@ -464,7 +498,8 @@ def run_comfuse(args):
     ms_e2e = timed(n_e2e, e2e_step) / n_e2e
     e2e = {"value": whole_job_value(flops, world, ms_e2e) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e,
-           "call": "comfuse_b2b_gemm_host" if b2b else "comfuse_gemm_epilogue_host"}
+           "call": "comfuse_gemm_spec between stream copies from / to pinned memory" if program
+                   else ("comfuse_b2b_gemm_host" if b2b else "comfuse_gemm_epilogue_host")}
 
     # ---- CPU baseline: the oracle as it stands, on rank 0 at N = 1 only, on a bounded sample
     cpu = None

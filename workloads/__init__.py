@@ -89,6 +89,7 @@ KIND_BIAS_GELU_RES_RMSNORM_MAX = "bias_gelu_res_rmsnorm_max"
 KIND_SCALE_MASK_SOFTMAX = "scale_mask_softmax"
 KIND_B2B_MLP_LAYERNORM = "b2b_mlp_layernorm"
 KIND_B2B_SOFTMAX_ATTENTION = "b2b_softmax_attention"
+KIND_GEMM_PROGRAM = "gemm_program"   # epilogue given as a node list (Workload.program)
 
 
 @dataclass
@@ -100,6 +101,7 @@ class Workload:
     dims: dict
     scalars: dict
     tensors: dict = field(default_factory=dict)
+    program: object = None  # SpecProgram for KIND_GEMM_PROGRAM; its parameter slot k is tensors[f"p{k}"]
 
     def gemm_flops(self) -> float:
         d = self.dims
@@ -119,6 +121,9 @@ class Workload:
             )
         b, M, N, K = d.get("batch", 1), d["M"], d["N"], d["K"]
         total = 2.0 * b * (M * K + K * N + M * N)
+        if self.kind == KIND_GEMM_PROGRAM:
+            total += sum(2.0 * v.size for k, v in self.tensors.items() if k.startswith("p"))
+            total += 4.0 * M * len(self.program.row_outputs)
         if self.kind == KIND_BIAS_RES_LAYERNORM:
             total += 2.0 * (M * N + N)  # residual, bias
             total += 2.0 * 2 * N if "gamma" in self.tensors else 0.0
@@ -217,6 +222,8 @@ def config(index: int) -> Workload:
         return b2b_mlp(32768, 128, 512, 128, seed=4, name="c5_b2b_mlp")
     if index == 5:   # beyond the five named configurations: B2B with a reduction as F (attention form)
         return target_attention(32, 4096, 256, 128, seed=5, name="a1_target_attention")
+    if index == 6:   # beyond the five: an epilogue given as data that no compiled kind covers
+        return program_range_normalise(8192, 1024, 1024, seed=6, name="p1_program_range_normalise")
     raise IndexError(index)
 
 
@@ -350,3 +357,14 @@ def spec_range_normalise() -> SpecProgram:
     sm = g.add("sum", y)
     am = g.add("argmax", y)
     return SpecProgram(g.nodes, y, (lo, hi, pr, sm, am), ("rowvec",))
+
+
+def program_range_normalise(M=8192, N=1024, K=1024, seed=6, name=None) -> Workload:
+    """GEMM followed by the range-normalising chain program (spec_range_normalise): inputs as for the post-norm pattern."""
+    t = {
+        "A": normal_bf16(seed, 0, (M, K)),
+        "B": normal_bf16(seed, 1, (K, N), std=1.0 / math.sqrt(K)),
+        "p0": uniform_bf16(seed, 2, (N,), -0.1, 0.1),
+    }
+    return Workload(name or f"program_range_normalise_{M}x{N}x{K}", KIND_GEMM_PROGRAM, {"M": M, "N": N, "K": K}, {}, t,
+                    program=spec_range_normalise())
