@@ -804,15 +804,51 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               const ChainInstr ci = sp.code[i];
               const int op = ci.op;
               if (op >= COMFUSE_OP_ADD && op <= kChainRdiv) {
-                // ---- binary: materialise the operand of the fragment, then apply
+                // ---- binary with a row-uniform operand (constant or per-row scalar): applied directly
+                if (ci.operand == CHO_SCALAR || ci.operand == CHO_CONST) {
+                  const float sv = scalar_get(ci.operand, ci.index, ci.imm);
+                  const float2 s2 = make_float2(sv, sv);
+                  switch (op) {
+                    case COMFUSE_OP_ADD:
+#pragma unroll
+                      for (int j = 0; j < 32; j += 2) { const float2 t = add2(make_float2(v[j], v[j + 1]), s2); v[j] = t.x; v[j + 1] = t.y; }
+                      break;
+                    case COMFUSE_OP_SUB: {
+                      const float2 n2 = make_float2(-sv, -sv);
+#pragma unroll
+                      for (int j = 0; j < 32; j += 2) { const float2 t = add2(make_float2(v[j], v[j + 1]), n2); v[j] = t.x; v[j + 1] = t.y; }
+                      break;
+                    }
+                    case COMFUSE_OP_MUL:
+#pragma unroll
+                      for (int j = 0; j < 32; j += 2) { const float2 t = mul2(make_float2(v[j], v[j + 1]), s2); v[j] = t.x; v[j + 1] = t.y; }
+                      break;
+                    case COMFUSE_OP_DIV:
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = __fdividef(v[j], sv);
+                      break;
+                    case COMFUSE_OP_MAX:
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], sv);
+                      break;
+                    case COMFUSE_OP_MIN:
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = fminf(v[j], sv);
+                      break;
+                    case kChainRsub:
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = sv - v[j];
+                      break;
+                    default:  // kChainRdiv
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = __fdividef(sv, v[j]);
+                      break;
+                  }
+                  continue;
+                }
+                // ---- binary with a per-column operand: materialise the operand of the fragment, then apply
                 float o[32];
                 switch (ci.operand) {
-                  case CHO_SCALAR: {
-                    const float sv = scalar_get(CHO_SCALAR, ci.index, 0.f);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) o[j] = sv;
-                    break;
-                  }
                   case CHO_ROWVEC: {
                     const float4* v4 = reinterpret_cast<const float4*>(vecs[ci.index] + lc);
 #pragma unroll
@@ -829,13 +865,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                       o[2 * j] = t2.x; o[2 * j + 1] = t2.y;
                     }
                     break;
-                  case CHO_MASK:
+                  default:  // CHO_MASK
 #pragma unroll
                     for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;
-                    break;
-                  default:  // CHO_CONST
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) o[j] = ci.imm;
                     break;
                 }
                 switch (op) {
