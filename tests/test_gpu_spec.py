@@ -241,3 +241,57 @@ def test_topk_row_outputs_on_gaussian_data():
     assert np.all((ti >= 0) & (ti < N)) and all(len(set(r)) == k for r in ti.tolist())
     np.testing.assert_allclose(np.take_along_axis(Yref, ti.astype(np.int64), axis=1), tv, atol=3e-2)  # the picked columns hold those values
     assert np.mean(ti == ri.astype(np.int64)) > 0.9
+
+
+def test_program_workload_at_bench_size_sampled_rows_and_graph_replay():
+    """p1 at the size bench.py times, launched the way it launches it (captured once, replayed): sampled rows against the
+    oracle, properties that hold for every row, and replay = direct launch bit for bit."""
+    w = wl.config(6)
+    prog, d = w.program, w.dims
+    M, N, K = d["M"], d["N"], d["K"]
+    dev = "cuda:0"
+    spec = cf.make_spec(prog.nodes, prog.terminal, len(prog.param_kinds), prog.row_outputs)
+    shape = cf.make_gemm_shape(1, M, N, K)
+    assert cf.spec_plan(spec, shape).path == cf.SPEC_PATH_FUSED_PROGRAM
+    A, B, p0 = to_dev(w.tensors["A"]), to_dev(w.tensors["B"]), to_dev(w.tensors["p0"])
+
+    def outputs():
+        Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev)
+        ro = [torch.full((M,), -7, dtype=torch.int32 if prog.nodes[r][0] == "argmax" else torch.float32, device=dev) for r in prog.row_outputs]
+        return Y, ro
+
+    Y, ro = outputs()
+    cf.gemm_spec(A, B, Y, spec, params=[p0], row_out=ro)
+    torch.cuda.synchronize()
+    Yg, rog = outputs()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        cf.gemm_spec(A, B, Yg, spec, params=[p0], row_out=rog)   # warm-up on the capture stream
+        torch.cuda.synchronize()
+        Yg.fill_(float("nan"))
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            cf.gemm_spec(A, B, Yg, spec, params=[p0], row_out=rog)
+    g.replay()
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK
+    assert torch.equal(Y.view(torch.int16), Yg.view(torch.int16))
+    for a, b in zip(ro, rog):
+        assert torch.equal(a, b)
+    # sampled rows against the oracle
+    rows = wl.sample_rows(M, 128)
+    f = wl.bf16_to_f64
+    Yref, Rref = spo.gemm_spec(f(w.tensors["A"][rows]), f(w.tensors["B"]), prog.nodes, prog.terminal, [f(w.tensors["p0"])], prog.row_outputs)
+    err = np.abs(to_f64(Y[torch.from_numpy(rows).to(dev)]) - Yref)
+    assert err.max() <= 4e-3 and err.mean() <= 1e-3, (err.max(), err.mean())
+    got_rows = [t.cpu().numpy()[rows] for t in ro]
+    np.testing.assert_allclose(got_rows[0], Rref[0], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(got_rows[1], Rref[1], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(got_rows[2], Rref[2], rtol=1e-4)
+    np.testing.assert_allclose(got_rows[3], Rref[3], rtol=1e-4)
+    # every row: y lies in [0, 1), is 0 at the row minimum, attains its maximum at the reported column
+    Yf = Y.float()
+    assert torch.isfinite(Yf).all().item() and Yf.min().item() == 0.0 and Yf.max().item() <= 1.0
+    assert torch.equal(Yf.min(-1).values, torch.zeros(M, device=dev))
+    picked = Yf.gather(-1, ro[4].long()[:, None])[:, 0]
+    assert torch.equal(picked, Yf.max(-1).values)
