@@ -753,19 +753,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     : op == COMFUSE_OP_RED_MIN ? INFINITY : 0.f;
           ridx[r] = 0x7FFFFFFF;
         }
-        auto scalar_get = [&](int kind, int ix, float imm) {
-          float sv = imm;
-          if (kind == CHO_SCALAR) {
-#pragma unroll
-            for (int q = 0; q < kStageMaxScalars; ++q) sv = (q == ix) ? sc[q] : sv;
-          }
-          return sv;
-        };
-        auto scalar_set = [&](int ix, float val) {
-#pragma unroll
-          for (int q = 0; q < kStageMaxScalars; ++q)
-            if (q == ix) sc[q] = val;
-        };
+        // indexed at run time (a small local-memory array: one load instead of a chain of selects)
+        auto scalar_get = [&](int kind, int ix, float imm) { return kind == CHO_SCALAR ? sc[ix & (kStageMaxScalars - 1)] : imm; };
+        auto scalar_set = [&](int ix, float val) { sc[ix & (kStageMaxScalars - 1)] = val; };
         wait_accumulator(0);
         const uint32_t taddr = tmem_of(0);
         constexpr int kFrags = 2 * (BN / 64) / EPW;  // this thread's 32-column fragments of the tile
