@@ -248,11 +248,16 @@ __global__ void __launch_bounds__(256) row_program_kernel(const __grid_constant_
 cudaError_t launch_row_program(const RowProgram& prog, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(prog.n_slots) * prog.N * sizeof(float);
   if (smem > kRowMaxSlotBytes) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the shared-memory opt-in is a per-device attribute of the kernel
+  constexpr int kMaxDev = 64;
+  static bool attr_set[kMaxDev] = {};
+  const DeviceInfo* dev = current_device_info();
+  if (!dev) return cudaErrorInvalidDevice;
+  const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
+  if (!attr_set[di] || dev->device >= kMaxDev) {
     cudaError_t e = cudaFuncSetAttribute(row_program_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kRowMaxSlotBytes));
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[di] = true;
   }
   const int threads = prog.N >= 1024 ? 256 : prog.N >= 256 ? 128 : 64;
   const long long rows = static_cast<long long>(prog.batch) * prog.M;
