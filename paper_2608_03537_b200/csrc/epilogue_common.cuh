@@ -67,20 +67,17 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
 #pragma unroll
   for (int t = 1; t < NH; ++t) cta_partial = merge(cta_partial, per_thread_count * t, s_pre[(xpar * NH + t) * 128 + row], per_thread_count);
   const float cta_count = static_cast<float>(NH) * per_thread_count;
+  if constexpr (CN == 1) {
+    // one CTA owns the whole row: the level-2 merge is already the result.  The next call uses the other level-2
+    // buffer, and the one after that comes behind the next call's named barrier, which every reader of this one passes first.
+    xpar ^= 1;
+    return cta_partial;
+  }
   // level 3: all-to-all over distributed shared memory; thread h serves the destination ranks congruent to h mod NH
   const uint32_t bar = stats_bar + 8u * xpar;
   const uint32_t phase = (xphase >> xpar) & 1u;
   float2* slot = s_stats + (xpar * CN + rank) * 128 + row;
-  if constexpr (CN == 1) {
-    // one CTA: plain stores, one arrival per lane quarter (lane 0, after a warp barrier that orders the other lanes'
-    // stores before it); the barrier expects 4 arrivals
-    if (h == 0) {
-      *slot = cta_partial;
-      __syncwarp();
-      if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
-    }
-    mbar_wait<false>(bar, phase, w);
-  } else {
+  {
     // each partial travels as an asynchronous 8-byte store that is counted on the destination's barrier; one local
     // thread arms the barrier with the byte count of the whole exchange (CN peers x 128 rows x 8 bytes)
     const uint32_t slot_addr = smem_u32(slot);
