@@ -123,7 +123,8 @@ def test_same_program_on_the_on_chip_interpreter(name):
     _check_rows(prog, ro, Rref, Yref)
 
 
-@pytest.mark.parametrize("M,N,K", [(300, 1024, 136), (520, 4096, 72), (129, 256, 64), (260, 768, 264)])
+# the last two shapes give every cluster several tiles (persistent walk, staging boxes reused, last tile staged in the ring)
+@pytest.mark.parametrize("M,N,K", [(300, 1024, 136), (520, 4096, 72), (129, 256, 64), (260, 768, 264), (4000, 4096, 64), (9000, 256, 64)])
 def test_chain_program_outside_the_compiled_patterns_runs_on_chip(M, N, K):
     prog = wl.spec_range_normalise()
     A, B, params = _inputs(36, 1, M, N, K, prog.param_kinds)
@@ -141,6 +142,18 @@ def test_chain_program_outside_the_compiled_patterns_runs_on_chip(M, N, K):
     assert np.mean(am == Rref[4].astype(np.int64)) > 0.995
     chosen = Yref[np.arange(M), am.astype(np.int64)]
     assert np.all(chosen >= Yref.max(axis=1) - 1e-5)
+
+
+def test_interpreter_with_residual_over_several_tiles_per_cluster():
+    # LayerNorm-ReLU in primitives forced onto the interpreter: the residual rides the operand ring tile after tile
+    prog = wl.spec_layernorm(relu=True)
+    M, N, K = 5000, 2048, 72
+    A, B, params = _inputs(38, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, 2, 1, M, N)
+    assert plan.program_path == cf.SPEC_PATH_FUSED_PROGRAM and launches == 1
+    Yref, _ = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    assert np.isfinite(err).all() and err.max() <= TOL_NORM_MAX and err.mean() <= TOL_NORM_MEAN, (err.max(), err.mean())
 
 
 def test_near_miss_of_a_compiled_kind_runs_on_chip():
