@@ -99,3 +99,16 @@ def test_b2b_attention_full_size_sampled(cuda_device):
     rows = wl.sample_rows(w.dims["M"], 64)
     batches = [0, 13, 31]
     P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches, label="a1 target attention")
+
+
+@pytest.mark.parametrize("batch,M,S,d", [(4, 512, 512, 128), (2, 300, 1000, 64)])
+def test_b2b_softmax_attention_other_shapes_unfused_path(batch, M, S, d, cuda_device):
+    """Shapes without a fused instantiation (the Self-Attention 512 x 512 shape of Sec. 6.2, Table II; a ragged one): the
+    fused call says UNSUPPORTED, the in-library unfused path (batched GEMM, row softmax, batched GEMM) matches the oracle."""
+    import paper_2608_03537_b200 as cf
+    w = wl.target_attention(batch, M, S, d, seed=S + d)
+    with pytest.raises(cf.ComfuseError) as e:
+        P.run_gpu(w, P.dev_tensors(w), fused=True)
+    assert e.value.status == cf.ERR_UNSUPPORTED
+    got = P.run_gpu(w, P.dev_tensors(w), fused=False)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"attention {batch}x{M}x{S}x{d} unfused")
