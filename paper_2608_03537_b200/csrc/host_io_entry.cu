@@ -5,10 +5,49 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstdlib>
+#include <mutex>
 
 #include "../../include/comfuse.h"
 
 namespace {
+
+// Row-chunk pipelining of the host-buffer GEMM call: rows are independent, so the call is cut into up to kPipeChunks row
+// ranges; range c's inputs are copied on a copy-in stream while range c-1 computes on the caller's stream and range c-2's
+// result goes back on a copy-out stream (both copy engines and the SMs busy at once).  The two helper streams and the
+// events are created once per device and reused; the caller's stream forks into them at the start of the call and joins
+// them at its end, so the call keeps its stream-ordered semantics.  COMFUSE_HOST_PIPELINE=0 turns it off.
+constexpr int kPipeChunks = 8;
+constexpr int kMaxDevPipe = 64;
+struct Pipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, copied[kPipeChunks] = {}, computed[kPipeChunks] = {};
+};
+Pipe g_pipe[kMaxDevPipe];
+std::mutex g_pipe_mutex;
+
+Pipe* pipe_for_current_device() {
+  static const bool enabled = [] {
+    const char* e = std::getenv("COMFUSE_HOST_PIPELINE");
+    return !(e && e[0] == '0');
+  }();
+  int d = -1;
+  if (!enabled || cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevPipe) return nullptr;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  Pipe& p = g_pipe[d];
+  if (p.ready) return &p;
+  bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming) == cudaSuccess;
+  for (int c = 0; ok && c < kPipeChunks; ++c)
+    ok = cudaEventCreateWithFlags(&p.copied[c], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&p.computed[c], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) return nullptr;
+  p.ready = true;
+  return &p;
+}
 
 constexpr size_t kAlign = 256;
 size_t round_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -69,6 +108,66 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
     cur += round_up(bytes);
     return err == cudaSuccess;
   };
+  // ---- pipelined form: one row range after the other (row-independent op lists, one batch, A and Y in host memory)
+  const int rows_per_chunk = ((desc->M + kPipeChunks - 1) / kPipeChunks + 255) / 256 * 256;
+  Pipe* pipe = (desc->batch == 1 && desc->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && (host_mask & COMFUSE_HOST_A) &&
+                (host_mask & COMFUSE_HOST_Y) && desc->M >= 2 * rows_per_chunk)
+                   ? pipe_for_current_device() : nullptr;
+  if (pipe) {
+    unsigned char* sA = cur;
+    cur += round_up(e.a);
+    unsigned char* sB = cur;
+    cur += round_up(e.b);
+    unsigned char* sR = cur;
+    cur += round_up(e.r);
+    unsigned char* sY = cur;
+    if ((host_mask & COMFUSE_HOST_B)) {
+      if (cudaMemcpyAsync(sB, B, e.b, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+      dB = sB;
+    }
+    const bool host_r = (host_mask & COMFUSE_HOST_RESIDUAL) != 0;
+    const unsigned char* hA = static_cast<const unsigned char*>(A);
+    const unsigned char* hR = host_r ? static_cast<const unsigned char*>(args->residual) : nullptr;
+    const unsigned char* dR = host_r ? sR : static_cast<const unsigned char*>(a.residual);
+    unsigned char* hY = static_cast<unsigned char*>(Y);
+    size_t ws_rows_bytes = 0;  // workspace bytes per row (dense Z of the unfused path, or the wide rows' partials)
+    {
+      size_t ws_all = 0;
+      if (comfuse_workspace_size(desc, &ws_all) != COMFUSE_OK) return COMFUSE_ERR_INVALID_ARG;
+      ws_rows_bytes = ws_all / static_cast<size_t>(desc->M);
+      if (ws_all > 0 && (!workspace || workspace_bytes < ws_all)) return COMFUSE_ERR_WORKSPACE;
+    }
+    if (cudaEventRecord(pipe->fork, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    if (cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    if (cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    int c = 0;
+    for (int r0 = 0; r0 < desc->M; r0 += rows_per_chunk, ++c) {
+      const int rows = desc->M - r0 < rows_per_chunk ? desc->M - r0 : rows_per_chunk;
+      const size_t offA = static_cast<size_t>(r0) * desc->lda * 2, offR = static_cast<size_t>(r0) * desc->ldr * 2,
+                   offY = static_cast<size_t>(r0) * desc->ldy * 2;
+      if (cudaMemcpyAsync(sA + offA, hA + offA, extent_bytes(1, rows, desc->K, desc->lda, 0), cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      if (host_r && cudaMemcpyAsync(sR + offR, hR + offR, extent_bytes(1, rows, desc->N, desc->ldr, 0), cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      if (cudaEventRecord(pipe->copied[c], pipe->in) != cudaSuccess || cudaStreamWaitEvent(st, pipe->copied[c], 0) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      comfuse_gemm_desc_t dc = *desc;
+      dc.M = rows;
+      comfuse_epilogue_args_t ac = a;
+      if (dR) ac.residual = dR + offR;
+      if (ac.row_max) ac.row_max += r0;
+      if (ac.row_argmax) ac.row_argmax += r0;
+      unsigned char* wsc = workspace ? static_cast<unsigned char*>(workspace) + static_cast<size_t>(r0) * ws_rows_bytes : nullptr;
+      s = comfuse_gemm_epilogue(&dc, sA + offA, dB, sY + offY, &ac, wsc, wsc ? workspace_bytes - static_cast<size_t>(r0) * ws_rows_bytes : 0, cuda_stream);
+      if (s != COMFUSE_OK) return s;
+      if (cudaEventRecord(pipe->computed[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->out, pipe->computed[c], 0) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      if (cudaMemcpyAsync(hY + offY, sY + offY, extent_bytes(1, rows, desc->N, desc->ldy, 0), cudaMemcpyDeviceToHost, pipe->out) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+    }
+    if (cudaEventRecord(pipe->join, pipe->out) != cudaSuccess || cudaStreamWaitEvent(st, pipe->join, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    return COMFUSE_OK;
+  }
   if ((host_mask & COMFUSE_HOST_A) && !stage_in(A, e.a, &dA)) return COMFUSE_ERR_CUDA;
   if ((host_mask & COMFUSE_HOST_B) && !stage_in(B, e.b, &dB)) return COMFUSE_ERR_CUDA;
   if ((host_mask & COMFUSE_HOST_RESIDUAL) && !stage_in(args->residual, e.r, &a.residual)) return COMFUSE_ERR_CUDA;

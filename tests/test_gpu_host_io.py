@@ -80,3 +80,48 @@ def test_host_form_rejects_small_staging(cuda_device):
         cf.gemm_epilogue_host(hA, T["B"], hY, cf.EPI_BIAS_RES_LAYERNORM, staging=staging, host_mask=cf.HOST_A | cf.HOST_Y,
                               bias=T["bias"], residual=T["residual"])
     assert ei.value.status == cf.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("case", ["layernorm_fused", "layernorm_unfused", "rmsnorm_max", "layernorm_wide_rows"])
+def test_pipelined_host_form_over_row_chunks_matches_device_form(case, cuda_device):
+    """Enough rows for the host form to run as a pipeline of row ranges (copy-in, compute and copy-out streams): results,
+    row outputs included, are bit for bit those of the device-pointer call; repeated calls on one stream reuse the staging
+    buffer safely; an event recorded after the call on the caller's stream covers the whole call."""
+    import paper_2608_03537_b200 as cf
+    if case == "rmsnorm_max":
+        w = wl.complex_subgraph(2100, 1024, 136, seed=23)
+        kind = cf.EPI_BIAS_GELU_RES_RMSNORM_MAX
+    elif case == "layernorm_wide_rows":
+        w = wl.post_norm(1100, 8192, 72, seed=24, affine=True)
+        kind = cf.EPI_BIAS_RES_LAYERNORM
+    else:
+        w = wl.post_norm(2100, 768, 200, seed=22, affine=True)
+        kind = cf.EPI_BIAS_RES_LAYERNORM
+    fused = case != "layernorm_unfused"
+    M, N = w.dims["M"], w.dims["N"]
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+    ref = P.run_gpu(w, T, fused=fused)
+    hA, hR = _pinned(T["A"]), _pinned(T["residual"])
+    hY = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+    mask = cf.HOST_A | cf.HOST_RESIDUAL | cf.HOST_Y
+    desc = cf.make_gemm_desc(hA, T["B"], hY, kind, residual=hR, fused=fused)
+    staging = torch.empty(cf.host_staging_size(desc, mask), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(16, cf.workspace_size(desc)), dtype=torch.uint8, device=dev)
+    kw = dict(staging=staging, host_mask=mask, bias=T["bias"], residual=hR, gamma=T["gamma"], alpha=w.scalars["alpha"],
+              eps=w.scalars["eps"], fused=fused, workspace=ws)
+    if kind == cf.EPI_BIAS_RES_LAYERNORM:
+        kw["beta"] = T["beta"]
+    else:
+        kw["row_max"] = torch.zeros(M, dtype=torch.float32, device=dev)
+        kw["row_argmax"] = torch.zeros(M, dtype=torch.int32, device=dev)
+    done = torch.cuda.Event()
+    for it in range(3):
+        hY.fill_(7.0)
+        cf.gemm_epilogue_host(hA, T["B"], hY, kind, **kw)
+        # an event recorded behind the call on the caller's stream covers the helper streams' copies as well
+        done.record()
+        done.synchronize()
+        assert torch.equal(hY.view(torch.int16), ref["Y"].cpu().view(torch.int16)), (case, it)
+    if "row_max" in kw:
+        assert torch.equal(kw["row_max"], ref["row_max"]) and torch.equal(kw["row_argmax"], ref["row_argmax"])
