@@ -171,8 +171,8 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
  * kernels as comfuse_gemm_epilogue, and, if COMFUSE_HOST_Y is set, one device -> host copy of the result.  Each copy moves
  * the tensor's whole strided extent ((batch-1)*batch_stride + (rows-1)*ld + cols elements), pad columns included.  Nothing
  * is allocated and nothing synchronises; the host buffers must stay valid until the stream has passed the call.
- * With one batch, A and Y in host memory, a LayerNorm / RMSNorm kind and at least 512 rows the call runs as a pipeline of
- * up to eight row ranges (rows are independent): range c is copied in on a library-owned copy stream while range c-1
+ * With one batch, A and Y in host memory, a LayerNorm / RMSNorm kind and at least 8 MB of activations the call runs as a
+ * pipeline of up to eight row ranges of at least 4 MB each (rows are independent): range c is copied in on a library-owned copy stream while range c-1
  * computes on `cuda_stream` and range c-2's result is copied out on a second library-owned stream.  `cuda_stream` forks
  * into the two helper streams at the start of the call and joins them at its end, so work enqueued on it afterwards (an
  * event, the next call) is ordered behind the whole call; results are bit for bit those of the unpipelined form.  The

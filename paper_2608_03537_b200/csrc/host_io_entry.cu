@@ -18,6 +18,13 @@ namespace {
 // events are created once per device and reused; the caller's stream forks into them at the start of the call and joins
 // them at its end, so the call keeps its stream-ordered semantics.  COMFUSE_HOST_PIPELINE=0 turns it off.
 constexpr int kPipeChunks = 8;
+// Every range costs host time (tensor-map encodes, launches, event records): cut only into ranges whose host -> device
+// traffic is worth it.
+constexpr size_t kPipeMinChunkBytes = 4u << 20;
+int pipe_chunks(size_t h2d_bytes) {
+  const size_t n = h2d_bytes / kPipeMinChunkBytes;
+  return n >= static_cast<size_t>(kPipeChunks) ? kPipeChunks : static_cast<int>(n);
+}
 constexpr int kMaxDevPipe = 64;
 struct Pipe {
   bool ready = false;
@@ -109,8 +116,9 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
     return err == cudaSuccess;
   };
   // ---- pipelined form: one row range after the other (row-independent op lists, one batch, A and Y in host memory)
-  const int rows_per_chunk = ((desc->M + kPipeChunks - 1) / kPipeChunks + 255) / 256 * 256;
-  Pipe* pipe = (desc->batch == 1 && desc->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && (host_mask & COMFUSE_HOST_A) &&
+  const int nchunks = pipe_chunks(e.a + e.r);
+  const int rows_per_chunk = nchunks >= 2 ? ((desc->M + nchunks - 1) / nchunks + 255) / 256 * 256 : desc->M;
+  Pipe* pipe = (nchunks >= 2 && desc->batch == 1 && desc->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && (host_mask & COMFUSE_HOST_A) &&
                 (host_mask & COMFUSE_HOST_Y) && desc->M >= 2 * rows_per_chunk)
                    ? pipe_for_current_device() : nullptr;
   if (pipe) {
@@ -205,6 +213,56 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
   const size_t xb = nb * desc->M * desc->K * 2, ob = nb * desc->M * desc->N2 * 2;
   unsigned char* dX = static_cast<unsigned char*>(staging);
   unsigned char* dO = dX + round_up(xb);
+  // ---- pipelined form: row ranges (MLP kind) or batch ranges (attention kind) flow through copy-in, compute and copy-out
+  // streams like the GEMM form above
+  const bool attn = desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION;
+  const long long units = attn ? desc->batch : desc->M;                     // what is cut: batches or rows
+  const long long grain = attn ? 1 : 256;
+  const int nchunks = pipe_chunks(xb + (attn ? nb * (static_cast<size_t>(desc->K) * desc->N1 + static_cast<size_t>(desc->N1) * desc->N2) * 2 : 0));
+  const long long per_chunk = nchunks >= 2 ? ((units + nchunks - 1) / nchunks + grain - 1) / grain * grain : units;
+  Pipe* pipe = (nchunks >= 2 && units >= 2 * per_chunk && (!attn || (W1 && W2))) ? pipe_for_current_device() : nullptr;
+  if (pipe) {
+    const size_t w1b = nb * desc->K * desc->N1 * 2, w2b = nb * desc->N1 * desc->N2 * 2;
+    unsigned char* dW1 = dO + round_up(ob);
+    unsigned char* dW2 = dW1 + round_up(w1b);
+    size_t ws_all = 0;
+    if (comfuse_b2b_workspace_size(desc, &ws_all) != COMFUSE_OK) return COMFUSE_ERR_INVALID_ARG;
+    if (ws_all > 0 && (!workspace || workspace_bytes < ws_all)) return COMFUSE_ERR_WORKSPACE;
+    const size_t ws_unit = ws_all / static_cast<size_t>(units);
+    // bytes per unit (row or batch) of each per-step tensor
+    const size_t ux = static_cast<size_t>(attn ? desc->M : 1) * desc->K * 2, uo = static_cast<size_t>(attn ? desc->M : 1) * desc->N2 * 2;
+    const size_t u1 = static_cast<size_t>(desc->K) * desc->N1 * 2, u2 = static_cast<size_t>(desc->N1) * desc->N2 * 2;
+    if (cudaEventRecord(pipe->fork, st) != cudaSuccess || cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess)
+      return COMFUSE_ERR_CUDA;
+    int c = 0;
+    for (long long u0 = 0; u0 < units; u0 += per_chunk, ++c) {
+      const long long n = units - u0 < per_chunk ? units - u0 : per_chunk;
+      const unsigned char* hX = static_cast<const unsigned char*>(X) + u0 * ux;
+      if (cudaMemcpyAsync(dX + u0 * ux, hX, n * ux, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess) return COMFUSE_ERR_CUDA;
+      if (attn) {
+        if (cudaMemcpyAsync(dW1 + u0 * u1, static_cast<const unsigned char*>(W1) + u0 * u1, n * u1, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess ||
+            cudaMemcpyAsync(dW2 + u0 * u2, static_cast<const unsigned char*>(W2) + u0 * u2, n * u2, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
+          return COMFUSE_ERR_CUDA;
+      }
+      if (cudaEventRecord(pipe->copied[c], pipe->in) != cudaSuccess || cudaStreamWaitEvent(st, pipe->copied[c], 0) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      comfuse_b2b_desc_t dc = *desc;
+      if (attn) dc.batch = static_cast<int32_t>(n);
+      else dc.M = static_cast<int32_t>(n);
+      unsigned char* wsc = workspace ? static_cast<unsigned char*>(workspace) + u0 * ws_unit : nullptr;
+      s = comfuse_b2b_gemm(&dc, dX + u0 * ux, attn ? static_cast<const void*>(dW1 + u0 * u1) : W1, b1,
+                           attn ? static_cast<const void*>(dW2 + u0 * u2) : W2, b2, gamma, beta, dO + u0 * uo, wsc,
+                           wsc ? workspace_bytes - u0 * ws_unit : 0, cuda_stream);
+      if (s != COMFUSE_OK) return s;
+      if (cudaEventRecord(pipe->computed[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->out, pipe->computed[c], 0) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      if (cudaMemcpyAsync(static_cast<unsigned char*>(O) + u0 * uo, dO + u0 * uo, n * uo, cudaMemcpyDeviceToHost, pipe->out) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+    }
+    if (cudaEventRecord(pipe->join, pipe->out) != cudaSuccess || cudaStreamWaitEvent(st, pipe->join, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    return COMFUSE_OK;
+  }
   if (cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
   if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION) {  // W1 (keys) and W2 (values) are host pointers as well
     if (!W1 || !W2) return COMFUSE_ERR_INVALID_ARG;

@@ -89,13 +89,13 @@ def test_pipelined_host_form_over_row_chunks_matches_device_form(case, cuda_devi
     buffer safely; an event recorded after the call on the caller's stream covers the whole call."""
     import paper_2608_03537_b200 as cf
     if case == "rmsnorm_max":
-        w = wl.complex_subgraph(2100, 1024, 136, seed=23)
+        w = wl.complex_subgraph(2100, 1024, 2048, seed=23)     # 8.6 MB of A + 4.3 MB of residual: three row ranges
         kind = cf.EPI_BIAS_GELU_RES_RMSNORM_MAX
     elif case == "layernorm_wide_rows":
-        w = wl.post_norm(1100, 8192, 72, seed=24, affine=True)
+        w = wl.post_norm(1100, 8192, 72, seed=24, affine=True)   # 18 MB of residual: four row ranges
         kind = cf.EPI_BIAS_RES_LAYERNORM
     else:
-        w = wl.post_norm(2100, 768, 200, seed=22, affine=True)
+        w = wl.post_norm(4200, 768, 1024, seed=22, affine=True)  # 8.6 MB of A + 6.5 MB of residual: three row ranges
         kind = cf.EPI_BIAS_RES_LAYERNORM
     fused = case != "layernorm_unfused"
     M, N = w.dims["M"], w.dims["N"]
@@ -125,3 +125,39 @@ def test_pipelined_host_form_over_row_chunks_matches_device_form(case, cuda_devi
         assert torch.equal(hY.view(torch.int16), ref["Y"].cpu().view(torch.int16)), (case, it)
     if "row_max" in kw:
         assert torch.equal(kw["row_max"], ref["row_max"]) and torch.equal(kw["row_argmax"], ref["row_argmax"])
+
+
+def test_pipelined_b2b_host_forms_match_device_forms(cuda_device):
+    """Large enough for the B2B host forms to run as pipelines (row ranges for the MLP kind, batch ranges for the attention
+    kind): bit for bit the device-pointer results, and within tolerance of the oracle on sampled rows."""
+    import paper_2608_03537_b200 as cf
+    # MLP kind: 40000 rows, X = 10 MB -> two row ranges
+    w = wl.b2b_mlp(M=40000, K=128, N1=512, N2=128, seed=31, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["X"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hX = _pinned(T["X"])
+    hO = torch.empty(40000, 128, dtype=torch.bfloat16).pin_memory()
+    desc = cf.make_b2b_desc(40000, 128, 512, 128, w.scalars["eps"], True)
+    staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        hO.fill_(3.0)
+        cf.b2b_gemm_host(hX, T["W1"], T["b1"], T["W2"], T["b2"], hO, staging=staging, gamma=T.get("gamma"), beta=T.get("beta"),
+                         eps=w.scalars["eps"])
+        torch.cuda.synchronize()
+        assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+    rows = wl.sample_rows(40000, 64)
+    P.check_outputs(w, {"Y": ref}, P.run_oracle(w, rows=rows), rows=rows, label="b2b host pipelined")
+    # attention kind: 20 batches, Q = 10.5 MB -> batch ranges
+    w = wl.target_attention(20, 2048, 256, 128, seed=32)
+    T = P.dev_tensors(w)
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hQ, hK, hV = _pinned(T["X"]), _pinned(T["W1"]), _pinned(T["W2"])
+    hO = torch.empty(20, 2048, 128, dtype=torch.bfloat16).pin_memory()
+    desc = cf.make_b2b_desc(2048, 128, 256, 128, 0.0, True, cf.B2B_SOFTMAX_ATTENTION, 20, w.scalars["alpha"])
+    staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        hO.fill_(3.0)
+        cf.b2b_attention_host(hQ, hK, hV, hO, staging=staging, alpha=w.scalars["alpha"])
+        torch.cuda.synchronize()
+        assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
