@@ -143,8 +143,9 @@ typedef enum {
   /* Attention form (Sec. 4, Eq. 2 with a row reduction as F; the Target-Attention workload of Sec. 6.2):
    *   O = softmax(alpha * X.W1) . W2   per batch,  softmax over the N1 source positions,
    * X [batch, M, K] queries, W1 [batch, K, N1] keys (already transposed), W2 [batch, N1, N2] values, O [batch, M, N2],
-   * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128, N1 = 256 (a whole score row fits the
-   * accumulators of one CTA pair); the probabilities are rounded to bf16 as the second GEMM's operand.             */
+   * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128 and N1 = 256 (a whole score row fits the
+   * accumulators of one CTA pair) or N1 = 512 (two sub-tiles of 256 source positions, each exponentiated against its own
+   * row maximum, combined when O is normalised); the probabilities are rounded to bf16 as the second GEMM's operand. */
   COMFUSE_B2B_SOFTMAX_ATTENTION = 1
 } comfuse_b2b_kind_t;
 

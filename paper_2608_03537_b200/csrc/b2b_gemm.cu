@@ -92,6 +92,11 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int num_clusters = gridDim.x >> 1;
   const int NC = p.N1 / 128;
   const int total_tiles = p.batch * p.mpairs;
+  // attention form: a score row of 512 source positions is processed as two sub-tiles of 256 (each with its own maximum
+  // and its own O slot) that the normalisation step combines; nsub = sub-tiles this cluster walks
+  const int nhalf = MODE == 1 ? p.N1 / 256 : 1;
+  const int my_tiles = cluster_id < total_tiles ? (total_tiles - cluster_id + num_clusters - 1) / num_clusters : 0;
+  const int nsub = my_tiles * nhalf;
   constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
@@ -160,20 +165,23 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
       if constexpr (MODE == 1) {
         // attention form, software-pipelined over tiles (see the UMMA lane): Q and K of tile t+1 go in before V of tile t
-        auto push_qk = [&](int tile) {
+        // sub-tile k of this cluster = 256 source positions (`half`) of its (k / nhalf)-th row tile
+        auto push_qk = [&](int k) {
+          const int tile = cluster_id + (k / nhalf) * num_clusters, half = k % nhalf;
           bz = tile / p.mpairs;
           const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
           push(&tmX, 0, m0, 0);
           push(&tmX, 64, m0, 0);
-          push(&tmW1, 0 * 128 + wcol, 0, 0);
-          push(&tmW1, 1 * 128 + wcol, 0, 0);
+          push(&tmW1, half * 256 + 0 * 128 + wcol, 0, 0);
+          push(&tmW1, half * 256 + 1 * 128 + wcol, 0, 0);
         };
-        if (cluster_id < total_tiles) push_qk(cluster_id);
-        for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters) {
-          if (tile + num_clusters < total_tiles) push_qk(tile + num_clusters);
+        if (nsub > 0) push_qk(0);
+        for (int k = 0; k < nsub && ok; ++k) {
+          if (k + 1 < nsub) push_qk(k + 1);
+          const int tile = cluster_id + (k / nhalf) * num_clusters, half = k % nhalf;
           bz = tile / p.mpairs;
-          push(&tmW2, wcol, 0 * 128, 0);
-          push(&tmW2, wcol, 1 * 128, 0);
+          push(&tmW2, wcol, half * 256 + 0 * 128, 0);
+          push(&tmW2, wcol, half * 256 + 1 * 128, 0);
         }
       }
       for (int tile = cluster_id; MODE == 0 && tile < total_tiles && ok; tile += num_clusters) {
@@ -245,11 +253,11 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           release_slot(xs0);
           release_slot(xs1);
         };
-        if (cluster_id < total_tiles) ml1();
-        for (int tile = cluster_id; tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
+        if (nsub > 0) ml1();
+        for (int k = 0; k < nsub && ok; ++k, ++tile_it) {
           const int obuf = tile_it & 1u;
           const uint32_t d_o = tmem_base + 256 + obuf * 128;
-          if (tile + num_clusters < total_tiles) {
+          if (k + 1 < nsub) {
             if (!mbar_wait<false>(bar_pfree, tile_it & 1u, w)) { ok = false; break; }  // the epilogue holds tile t's scores in registers
             tcgen05_fence_after_sync();
             ml1();
@@ -398,7 +406,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       // ---------------- Epi1 (N1 = 256: the two P slots hold one whole score row): row max and sum of exponentials
       // across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next UMMAs' A operand;
       // returns 1 / (row sum), applied in the tile's finish step (O = (S.V) / sum)
-      auto softmax_tile = [&]() -> float {
+      auto softmax_tile = [&]() -> float2 {
         for (int pb = 0; pb < 2; ++pb) {
           mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
           ++puses[pb];
@@ -463,26 +471,51 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           mbar_arrive_cluster_noflush(sfull_leader);
           mbar_arrive_cluster_noflush(sfull_leader + 8u);
         }
-        return tot.y > 0.f ? 1.f / tot.y : 0.f;
+        return tot;  // (row maximum in the log2 domain, sum of 2^(t - maximum)) of this sub-tile
       };
       // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes through one staging buffer
-      auto finish_tile = [&](int tile, uint32_t it, float inv_l) {
+      // `it` = number of the row tile's first sub-tile; ml0 / ml1 = (maximum, sum) of its one or two sub-tiles
+      auto finish_tile = [&](int tile, uint32_t it, float2 ml0, float2 ml1) {
         const int bz = tile / p.mpairs;
         const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
-        const int obuf = it & 1u;
-        mbar_wait<false>(bar_ofull(obuf), (it >> 1) & 1u, w);
-        __syncwarp();
-        tcgen05_fence_after_sync();
         uint32_t pk[16];
-        {
+        if (nhalf == 1) {
+          const int obuf = it & 1u;
+          const float inv_l = ml0.y > 0.f ? 1.f / ml0.y : 0.f;
+          mbar_wait<false>(bar_ofull(obuf), (it >> 1) & 1u, w);
+          __syncwarp();
+          tcgen05_fence_after_sync();
           uint32_t v[32];
           tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + hh * 32, v);
 #pragma unroll
           for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * i], v[2 * i + 1]), splat2(inv_l)));
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
+        } else {
+          // two sub-tiles, each exponentiated against its own maximum: O = (O0 2^(m0-m) + O1 2^(m1-m)) / (l0 2^(m0-m) + l1 2^(m1-m))
+          const float mm = fmaxf(ml0.x, ml1.x);
+          const float f0 = ml0.x == -INFINITY ? 0.f : ex2_approx(ml0.x - mm), f1 = ml1.x == -INFINITY ? 0.f : ex2_approx(ml1.x - mm);
+          const float l = ml0.y * f0 + ml1.y * f1;
+          const float inv_l = l > 0.f ? 1.f / l : 0.f;
+          const float2 w0 = splat2(f0 * inv_l), w1 = splat2(f1 * inv_l);
+          mbar_wait<false>(bar_ofull(0), (it >> 1) & 1u, w);  // `it` is even: slot 0 holds the first sub-tile's S.V, slot 1 the second's
+          mbar_wait<false>(bar_ofull(1), (it >> 1) & 1u, w);
+          __syncwarp();
+          tcgen05_fence_after_sync();
+          uint32_t v0[32], v1[32];
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + 0 * 128 + hh * 32, v0);
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + 1 * 128 + hh * 32, v1);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            pk[i] = pack_bf16x2_rn(fma2(f2_from_bits(v1[2 * i], v1[2 * i + 1]), w1, mul2(f2_from_bits(v0[2 * i], v0[2 * i + 1]), w0)));
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive_cluster_noflush(oempty_leader);
+            mbar_arrive_cluster_noflush(oempty_leader + 8u);
+          }
         }
-        tcgen05_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
         for (int g = 0; g < 2; ++g) {
           if (store_thread) tma_store_wait_read<0>();
           named_barrier_sync(3, kB2bEpiThreads);
@@ -503,12 +536,26 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           }
         }
       };
-      float inv_next = 0.f;
-      if (cluster_id < total_tiles) inv_next = softmax_tile();
-      for (int tile = cluster_id; tile < total_tiles; tile += num_clusters, ++tile_it) {
-        const float inv_cur = inv_next;
-        if (tile + num_clusters < total_tiles) inv_next = softmax_tile();
-        finish_tile(tile, tile_it, inv_cur);
+      // Order (the S buffers and the O slots are handed back by the steps named behind the arrows):
+      //   one sub-tile per row tile:   softmax(0) | softmax(t+1), finish(t) ...
+      //   two sub-tiles per row tile:  softmax(0), softmax(1) | softmax(2t+2), finish(t), softmax(2t+3) ...
+      // (S.V of sub-tile 2t+2 needs O slot 0, which finish(t) releases; the softmax of 2t+3 needs the S buffers that
+      // S.V of 2t+2 releases, so it must come behind finish(t).)
+      float2 ml_a = make_float2(-INFINITY, 0.f), ml_b = ml_a;
+      if (nsub > 0) ml_a = softmax_tile();
+      if (nhalf == 2 && nsub > 1) ml_b = softmax_tile();
+      for (int i = 0; i < my_tiles; ++i) {
+        const int tile = cluster_id + i * num_clusters;
+        const int first = i * nhalf;
+        const float2 c0 = ml_a, c1 = ml_b;
+        if (nhalf == 1) {
+          if (first + 1 < nsub) ml_a = softmax_tile();
+          finish_tile(tile, static_cast<uint32_t>(first), c0, c0);
+        } else {
+          if (first + 2 < nsub) ml_a = softmax_tile();
+          finish_tile(tile, static_cast<uint32_t>(first), c0, c1);
+          if (first + 3 < nsub) ml_b = softmax_tile();
+        }
       }
     }
     for (int tile = cluster_id; MODE == 0 && tile < total_tiles; tile += num_clusters, ++tile_it) {
@@ -702,7 +749,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 }  // namespace
 
 bool b2b_fused_supported(int K, int N1, int N2, int mode) {
-  if (mode == 1) return K == 128 && N2 == 128 && N1 == 256;  // attention form: one whole score row in the two P slots
+  // attention form: 256 source positions fill the two P slots; 512 run as two sub-tiles combined at the normalisation
+  if (mode == 1) return K == 128 && N2 == 128 && (N1 == 256 || N1 == 512);
   return K == 128 && N2 == 128 && N1 >= 128 && N1 <= 128 * kMaxChunks && N1 % 128 == 0;
 }
 

@@ -101,10 +101,30 @@ def test_b2b_attention_full_size_sampled(cuda_device):
     P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches, label="a1 target attention")
 
 
-@pytest.mark.parametrize("batch,M,S,d", [(4, 512, 512, 128), (2, 300, 1000, 64)])
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M", [(4, 512), (3, 600), (40, 256), (100, 512), (1, 1)])
+def test_b2b_softmax_attention_512_source_positions(batch, M, fused, cuda_device):
+    """The Self-Attention 512 x 512 shape of Sec. 6.2 (Table II) and neighbours: a score row of 512 runs as two sub-tiles of
+    256 with their own maxima, combined at the normalisation; ragged M, up to three row tiles (six sub-tiles) per CTA pair, the
+    one-row edge."""
+    w = wl.target_attention(batch, M, 512, 128, seed=batch + M + 1)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"attention S=512 b{batch} M{M} fused={fused}")
+
+
+def test_b2b_softmax_attention_512_sharp_rows_in_either_half(cuda_device):
+    """Large scores: the dominant key lies in the first half for some rows and in the second half for others, so the two
+    sub-tiles' maxima differ by tens of units either way; no overflow, the output is the dominant value row."""
+    w = wl.target_attention(2, 256, 512, 128, seed=77)
+    w.scalars["alpha"] = 4.0
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label="attention S=512 sharp")
+
+
+@pytest.mark.parametrize("batch,M,S,d", [(4, 512, 1024, 128), (2, 300, 1000, 64)])
 def test_b2b_softmax_attention_other_shapes_unfused_path(batch, M, S, d, cuda_device):
-    """Shapes without a fused instantiation (the Self-Attention 512 x 512 shape of Sec. 6.2, Table II; a ragged one): the
-    fused call says UNSUPPORTED, the in-library unfused path (batched GEMM, row softmax, batched GEMM) matches the oracle."""
+    """Shapes without a fused instantiation: the fused call says UNSUPPORTED, the in-library unfused path (batched GEMM, row
+    softmax, batched GEMM) matches the oracle."""
     import paper_2608_03537_b200 as cf
     w = wl.target_attention(batch, M, S, d, seed=S + d)
     with pytest.raises(cf.ComfuseError) as e:
