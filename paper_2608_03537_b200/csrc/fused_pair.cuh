@@ -163,6 +163,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int num_clusters = gridDim.x / CLUSTER;
   const int KB = (p.K + 63) >> 6;
   const bool has_res = (EPI == EPI_LN || kIsRms || EPI == EPI_PROGRAM) && p.residual != nullptr;
+  // The last tile's output boxes may be staged in the circular buffer only if nothing is still arriving there when they
+  // are written: a stage program that stores in its first pass does so while the residual boxes are still coming in.
+  const bool ring_idle_at_store = !(EPI == EPI_PROGRAM && has_res && p.program.terminal_pass == 0);
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
@@ -373,7 +376,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
         const int m0 = mpair0 + static_cast<int>(pm) * 128;
-        const bool in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles;
+        const bool in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles && ring_idle_at_store;
         int kk = 0;  // box of this tile
         for (int sub = 0; sub < ESUB && ok; ++sub) {
           const int W = unit_width(sub);
@@ -499,7 +502,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       decode_tile(tile, b, mpair0, ncta0);
       const int m0 = mpair0 + static_cast<int>(pm) * 128;
       const int grow = m0 + row;
-      in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles;
+      in_ring = Cfg::RING_STAGING && tile + num_clusters >= p.total_tiles && ring_idle_at_store;
       const bool valid = grow < p.M;
 
       // the slot of each sub-tile of this tile, and whether it is computed at all

@@ -473,19 +473,16 @@ struct StageLowering {
   }
 };
 
+bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, StageBinding& bind);
+
 bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bind) {
-  std::memset(&sp, 0, sizeof(sp));
   if (!an.row_outputs.empty() && an.row_outputs.size() > static_cast<size_t>(kStageMaxRowOut)) return false;
   if (an.type[an.terminal] != T_TENSOR) return false;
-  StageLowering L(an, bind);
-  L.sp = &sp;
   const int n = an.n;
   // the resident tensor: the one stage-0 tensor that later stages read
-  int first_acc = -1;
   std::vector<int> cand;
   for (int k = 0; k < n; ++k) {
     if (!an.live[k]) continue;
-    if (an.nodes[k].op == COMFUSE_OP_ACC && first_acc < 0) first_acc = k;
     if (an.type[k] != T_TENSOR || an.stage[k] < 1 || is_reduce(an.nodes[k].op)) continue;
     for (int e : {an.nodes[k].in0, an.nodes[k].in1}) {
       if (e < 0 || an.type[e] != T_TENSOR || an.stage[e] != 0) continue;
@@ -497,8 +494,24 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
     }
   }
   if (cand.size() > 1) return false;
-  if (first_acc < 0) return false;
-  L.x_root = cand.size() == 1 ? cand[0] : (an.stage[an.terminal] == 0 ? an.terminal : first_acc);
+  if (cand.size() == 1) return lower_stage_program_from(an, cand[0], sp, bind);
+  // no later stage reads a stage-0 tensor (the reductions only feed row outputs): any stage-0 tensor from which the
+  // terminal and every reduction input can be reached by chains will do; try them from the last to the first
+  for (int k = n - 1; k >= 0; --k) {
+    if (!an.live[k] || an.type[k] != T_TENSOR || an.stage[k] != 0) continue;
+    if (is_leaf(an.nodes[k].op) && an.nodes[k].op != COMFUSE_OP_ACC) continue;
+    StageBinding b2;
+    if (lower_stage_program_from(an, k, sp, b2)) { bind = b2; return true; }
+  }
+  return false;
+}
+
+bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, StageBinding& bind) {
+  std::memset(&sp, 0, sizeof(sp));
+  StageLowering L(an, bind);
+  L.sp = &sp;
+  L.x_root = x_root;
+  const int n = an.n;
   // stage 0: acc -> x
   std::vector<ChainInstr> entry, fin;
   std::vector<std::vector<ChainInstr>> red_chain;
