@@ -133,14 +133,15 @@ def run_oracle(w: wl.Workload, rows=None, batches=None):
 
 
 # --------------------------------------------------------------------------------------------- comparison
-def check_outputs(w: wl.Workload, got: dict, ref: dict, rows=None, batches=None, label="", rowmax_tol=5e-3, softmax_tol=TOL_SOFTMAX_MAX):
+def check_outputs(w: wl.Workload, got: dict, ref: dict, rows=None, batches=None, label="", rowmax_tol=5e-3, softmax_tol=TOL_SOFTMAX_MAX,
+                  norm_tol=TOL_NORM_MAX):
     """Element-by-element comparison against the oracle with the stated tolerances; returns the error figures.
     `rowmax_tol`: absolute tolerance of the fp32 row maximum (and the slack within which a reported arg max column
     must reach the oracle's maximum).  The fused path keeps fp32 up to that point (5e-3 covers tanh.approx); the
     unfused path has rounded the GEMM result to bf16 first, so it gets the normalised-tensor tolerance 3e-2.
     `softmax_tol`: 2e-3 for the fused kernel; the unfused path exponentiates bf16-rounded scores (relative error
     2^-9 on |score| up to ~4 after scaling), which alone moves a probability near 0.5 by up to ~4e-3, so the tests
-    give it 1e-2 and say so."""
+    give it 1e-2 and say so.  `norm_tol`: max-abs bound of normalised outputs (3e-2 unless a caller says otherwise)."""
     Y = got["Y"]
     if batches is not None:
         Y = Y[list(batches)]
@@ -156,7 +157,7 @@ def check_outputs(w: wl.Workload, got: dict, ref: dict, rows=None, batches=None,
         dead = ref["Y"] == 0.0
         assert (Yg[dead] == 0.0).all(), f"{label}: masked entries must be exactly zero"
     else:
-        assert res["max_abs"] <= TOL_NORM_MAX, f"{label}: max-abs {res['max_abs']:.3e}"
+        assert res["max_abs"] <= norm_tol, f"{label}: max-abs {res['max_abs']:.3e}"
         assert res["mean_abs"] <= TOL_NORM_MEAN, f"{label}: mean-abs {res['mean_abs']:.3e}"
     if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
         rm, am = got["row_max"], got["row_argmax"]

@@ -1,0 +1,59 @@
+"""Randomised sweep of the compiled op lists: seeded random shapes (ragged M, K not a multiple of the 64-wide K block,
+every row length with a fused instantiation, batches for the softmax), optional operands left out at random, the pattern
+flags, fused and unfused, each against the fp64 oracle with the stated tolerances."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+ROW_LENGTHS = [256, 512, 768, 1024, 2048, 4096]
+
+
+def _case(seed):
+    g = np.random.default_rng(seed)
+    kind = ["ln", "rms", "softmax"][int(g.integers(3))]
+    K = int(g.integers(1, 66)) * 8                      # 8 .. 520: partial K blocks included
+    M = int(g.integers(1, 700))
+    fused = bool(g.random() < 0.7)
+    if kind == "ln":
+        N = ROW_LENGTHS[int(g.integers(len(ROW_LENGTHS)))]
+        w = wl.post_norm(M, N, K, seed=seed, affine=bool(g.random() < 0.6), relu=bool(g.random() < 0.4))
+        for name in ("bias", "residual"):
+            if g.random() < 0.3:
+                del w.tensors[name]
+    elif kind == "rms":
+        N = ROW_LENGTHS[int(g.integers(len(ROW_LENGTHS)))]
+        w = wl.complex_subgraph(M, N, K, seed=seed, activation=bool(g.random() < 0.6), residual=bool(g.random() < 0.6))
+        if g.random() < 0.3:
+            del w.tensors["bias"]
+    else:
+        batch = int(g.integers(1, 4))
+        causal = bool(g.random() < 0.4)
+        softcap = float(np.round(g.uniform(1.0, 8.0), 2)) if g.random() < 0.3 else 0.0
+        if K <= 256:
+            N = int(g.integers(8, 160)) * 8               # any row length for the short-K kernel: 64 .. 1272
+        else:
+            N = [256, 512, 1024, 2048][int(g.integers(4))]   # the cluster kernel's instantiations
+        if causal:
+            M = N
+        w = wl.scaled_masked_softmax(batch, M, N, K, seed=seed, causal=causal, softcap=softcap)
+    return w, fused
+
+
+@pytest.mark.parametrize("seed", range(200))
+def test_random_shape_and_operands(seed, cuda_device):
+    w, fused = _case(7000 + seed)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    kw = {}
+    if w.kind == wl.KIND_SCALE_MASK_SOFTMAX:
+        kw["softmax_tol"] = P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED
+    if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+        kw["rowmax_tol"] = 5e-3 if fused else 3e-2
+    if not fused and w.kind != wl.KIND_SCALE_MASK_SOFTMAX:
+        # the unfused baseline normalises the bf16-rounded GEMM result: on outputs of magnitude 4 .. 8 (half-ulp 1.56e-2) an
+        # occasional element lands just above 3e-2 (seen: 3.03e-2); the fused kernels are held to 3e-2
+        kw["norm_tol"] = 4e-2
+    P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused} {sorted(w.tensors)} {w.scalars}", **kw)
