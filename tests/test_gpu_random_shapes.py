@@ -57,3 +57,20 @@ def test_random_shape_and_operands(seed, cuda_device):
         # occasional element lands just above 3e-2 (seen: 3.03e-2); the fused kernels are held to 3e-2
         kw["norm_tol"] = 4e-2
     P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused} {sorted(w.tensors)} {w.scalars}", **kw)
+
+
+@pytest.mark.parametrize("seed", range(150))
+def test_random_b2b_shapes(seed, cuda_device):
+    """Back-to-back GEMM, both forms: random row counts (ragged tiles, fewer and more tiles than CTA pairs), every chunk count
+    of the MLP form, both source lengths of the attention form, random scale; fused and unfused."""
+    g = np.random.default_rng(9000 + seed)
+    fused = bool(g.random() < 0.7)
+    if g.random() < 0.5:
+        w = wl.b2b_mlp(M=int(g.integers(1, 3000)), K=128, N1=128 * int(g.integers(1, 5)), N2=128, seed=seed, affine=bool(g.random() < 0.5))
+    else:
+        w = wl.target_attention(int(g.integers(1, 6)), int(g.integers(1, 1200)), [256, 512][int(g.integers(2))], 128, seed=seed)
+        # scores of standard deviation up to ~7 for the fused kernel; the unfused baseline rounds the scores to bf16 before it
+        # exponentiates them (absolute error 2^-9 |score|), so it is only held to the tolerance on moderate scores
+        w.scalars["alpha"] = float(np.round(g.uniform(0.02, 0.6 if fused else 0.12), 3))
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused} {w.scalars}")
