@@ -169,3 +169,47 @@ def test_topk_nodes_are_row_outputs_only():
     assert _status([N_, ("topk_values", 0, -1, 0, 0.0)], 0, row_outputs=(1,)) == INV    # K >= 1
     assert _status([N_, ("topk_indices", 0, -1, 65, 0.0)], 0, row_outputs=(1,)) == INV  # K <= 64
     assert _status([N_, ("topk_values", 0, -1, 40, 0.0)], 0, row_outputs=(1,), shape=cf.make_gemm_shape(1, 64, 32, 64)) == INV  # K <= N
+
+
+def test_random_node_lists_never_crash_the_analysis():
+    """Fuzz: arbitrary op codes, edges, parameter indices and terminals are either accepted or rejected with a status --
+    and whatever is accepted can be planned on every pathway selector and sized."""
+    import ctypes
+    import numpy as np
+    g = np.random.default_rng(123)
+    codes = sorted(cf.OPS.values()) + [5, 15, 28, 31, 38, 47, 56, 99, -1]
+    L = cf.lib()
+    accepted = 0
+    for _ in range(3000):
+        n = int(g.integers(1, 20))
+        nodes = [(0, -1, -1, -1, 0.0)]
+        for k in range(1, n):
+            op = int(g.choice(sorted(cf.OPS.values())))
+            a = int(g.integers(0, k)) if op >= 16 else -1
+            b = int(g.integers(0, k)) if 32 <= op <= 37 else -1
+            prm = int(g.integers(0, 3)) if op in (2, 3) else (int(g.integers(1, 9)) if op in (54, 55) else -1)
+            nodes.append((op, a, b, prm, float(g.normal())))
+        if g.random() < 0.4:   # corrupt one field of one node
+            k = int(g.integers(0, n))
+            f = list(nodes[k])
+            f[int(g.integers(0, 4))] = int(g.choice(codes)) if g.random() < 0.5 else int(g.integers(-3, n + 3))
+            nodes[k] = tuple(f)
+        n_params = int(g.integers(2, 5))
+        terminal = int(g.integers(-1, n + 1)) if g.random() < 0.2 else int(g.integers(0, n))
+        ro = tuple(int(x) for x in g.integers(0, n, size=int(g.integers(0, 3))))
+        spec = cf.make_spec(nodes, terminal, n_params, ro)
+        shape = cf.make_gemm_shape(1, int(g.integers(1, 600)), int(g.choice([64, 256, 768, 1000, 4096, 12])), int(g.integers(1, 40)) * 8)
+        plan = cf.SpecPlan()
+        st = L.comfuse_spec_plan(ctypes.byref(spec), ctypes.byref(shape), ctypes.byref(plan))
+        assert st in (cf.OK, cf.ERR_INVALID_ARG, cf.ERR_UNSUPPORTED, cf.ERR_ALIGNMENT), st
+        for fused in (0, 1, 2):
+            nbytes = ctypes.c_size_t(0)
+            st2 = L.comfuse_gemm_spec_workspace_size(ctypes.byref(spec), ctypes.byref(shape), fused, ctypes.byref(nbytes))
+            assert st2 in (cf.OK, cf.ERR_INVALID_ARG, cf.ERR_UNSUPPORTED, cf.ERR_ALIGNMENT), st2
+            if st in (cf.ERR_INVALID_ARG, cf.ERR_ALIGNMENT):
+                assert st2 == st
+        if st == cf.OK:
+            accepted += 1
+            assert plan.n_stages >= 1 and plan.n_live_nodes >= 1
+            assert plan.path in (cf.SPEC_PATH_FUSED_KERNEL, cf.SPEC_PATH_ROW_PROGRAM, cf.SPEC_PATH_FUSED_PROGRAM)
+    assert accepted > 20
