@@ -222,6 +222,8 @@ def config(index: int) -> Workload:
         return b2b_mlp(32768, 128, 512, 128, seed=4, name="c5_b2b_mlp")
     if index == 5:   # beyond the five named configurations: B2B with a reduction as F (attention form)
         return target_attention(32, 4096, 256, 128, seed=5, name="a1_target_attention")
+    if index == 7:   # beyond the five: the Self-Attention 512 x 512 shape of Sec. 6.2 (two sub-tiles of 256 source positions)
+        return target_attention(256, 512, 512, 128, seed=7, name="a2_self_attention_512")
     if index == 6:   # beyond the five: an epilogue given as data that no compiled kind covers
         return program_range_normalise(8192, 1024, 1024, seed=6, name="p1_program_range_normalise")
     raise IndexError(index)
