@@ -310,6 +310,7 @@ def run_comfuse(args):
         """K steps bracketed by barrier + synchronize; device time from CUDA events on the launching stream."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
+        torch.cuda._sleep(400_000)  # see the main timed region
         e0.record()
         for i in range(nsteps):
             fn(i)
@@ -331,21 +332,40 @@ def run_comfuse(args):
             for s in sets:
                 step(s)
         graph_launches = cf.launch_count() - c0
-        graph.replay()
+        # untimed replays on top of the requested warm-up steps: a short timed region right after capture otherwise
+        # measures clock ramp-up and first-replay costs (20 timed steps read 6 % slower than 200)
+        for _ in range(max(1, -(-60 // nsets))):
+            graph.replay()
+        torch.cuda.synchronize()
+
+    # steps that do not fill a whole graph are replayed from a second, shorter graph (direct launches would add host time)
+    rest_graph = None
+    if graph is not None and args.steps % nsets:
+        rest_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(rest_graph):
+            for s in sets[:args.steps % nsets]:
+                step(s)
+        rest_graph.replay()
         torch.cuda.synchronize()
 
     def run_steps(n, fn):
         full, rest = (n // nsets, n % nsets) if graph is not None else (0, n)
         for _ in range(full):
             graph.replay()
-        for i in range(rest):
-            fn(i)
+        if rest and rest_graph is not None and rest == args.steps % nsets:
+            rest_graph.replay()
+        else:
+            for i in range(rest):
+                fn(i)
 
     sampler = ClockSampler(local)
     launches0 = cf.launch_count()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    # a short busy-wait kernel in front of the start event: the host enqueues the K steps while it runs, so the timed
+    # region holds the steps' device time and not the latency of the first launch into an idle stream
+    torch.cuda._sleep(400_000)
     e0.record()
     run_steps(args.steps, lambda i: step(sets[i % nsets]))
     e1.record()
@@ -356,6 +376,8 @@ def run_comfuse(args):
     if graph is not None:   # replayed launches do not pass through the library's host code: count them from the graph
         per_graph = graph_launches
         launches += (args.steps // nsets) * per_graph
+        if rest_graph is not None:
+            launches += (args.steps % nsets) * (per_graph // nsets)
     status = cf.last_device_status()
     if status != cf.OK:
         raise SystemExit(f"device status {status} after the timed region")
