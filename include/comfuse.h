@@ -52,7 +52,11 @@ typedef enum {
    * reduction: row_max[i] = max_j Y, row_argmax[i] = lowest such j  -- Sec. 2.2 (MatMul + RMSNorm), Sec. 3.2 */
   COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX = 1,
   /* P = softmax(alpha*A.B + mask) over the last dim  -- Sec. 5 (ReduceMode softmax), Sec. 6.1 (attention scores) */
-  COMFUSE_EPI_SCALE_MASK_SOFTMAX = 2
+  COMFUSE_EPI_SCALE_MASK_SOFTMAX = 2,
+  /* Y = act(alpha*A.B + bias), act in {none, ReLU, GELU_tanh, tanh, sigmoid}: a reduction-free epilogue (any N that is a
+   * multiple of 8, the plain GEMM's tiling).  Reported by comfuse_spec_plan for programs that lower to it and run by
+   * comfuse_gemm_spec; comfuse_gemm_epilogue does not take this kind (INVALID_ARG). */
+  COMFUSE_EPI_BIAS_ACTIVATION = 3
 } comfuse_epilogue_kind_t;
 
 typedef enum {
@@ -226,8 +230,9 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      splits it into stages at the reduction nodes: stage(node) = max over its inputs of stage(input), plus one
  *      behind a reduction;
  *   2. lowers it: a program whose stages have the shape of a compiled fused instantiation (affine entry
- *      [activation] [+ residual] -> LayerNorm | RMSNorm [-> max/argmax] | softmax, in any spelling the canonicaliser
- *      recognises: operand order of commutative nodes, optional nodes absent) runs as that ONE fused kernel
+ *      [activation] [+ residual] -> LayerNorm | RMSNorm [-> max/argmax] | softmax, or a reduction-free act(alpha*acc + bias),
+ *      in any spelling the canonicaliser recognises: operand order of commutative nodes, optional nodes absent) runs as
+ *      that ONE fused kernel
  *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); a program in which ONE tensor stays resident across the reductions and
  *      every tensor-valued expression is a chain on it (element-wise nodes whose other operand is a constant, a per-row
  *      value, a row vector, the causal mask or -- before the first reduction -- one full tensor; at most 3 row vectors,

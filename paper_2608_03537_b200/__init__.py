@@ -29,6 +29,7 @@ LIB_PATH = os.path.join(_PKG_DIR, "libcomfuse.so")
 # status codes / enums of include/comfuse.h
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
 EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 0, 1, 2
+EPI_BIAS_ACTIVATION = 3   # reduction-free epilogue; reached through gemm_spec only
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
 FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2

@@ -213,6 +213,32 @@ comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, lon
   return launch_plain_gemm(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
 }
 
+comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
+                                      long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
+                                      const void* bias, float alpha, int activation, cudaStream_t st) {
+  const DeviceInfo* dev = nullptr;
+  comfuse_status_t s = check_device(&dev);
+  if (s != COMFUSE_OK) return s;
+  GemmMaps maps;
+  if (!make_gemm_maps(&maps, A, B, nullptr, Y, batch, M, N, K, lda, ldb, 0, ldy, batch_stride_a, batch_stride_b, 0,
+                      batch > 1 ? batch_stride_y : 0))
+    return COMFUSE_ERR_CUDA;
+  FusedParams p = {};
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.mblocks = (M + 127) / 128;
+  p.nblocks = 1;
+  p.total_tiles = batch * p.mblocks;
+  p.alpha = alpha;
+  p.activation = activation;
+  p.bias = static_cast<const uint16_t*>(bias);
+  p.status = dev->status_word;
+  p.timeout_ns = timeout_ns();
+  p.Y = static_cast<uint16_t*>(Y);
+  p.ldy = ldy;
+  p.batch_stride_y = batch > 1 ? batch_stride_y : 0;
+  return launch_gemm_elementwise(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
 comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,

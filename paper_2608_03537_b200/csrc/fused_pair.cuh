@@ -88,7 +88,7 @@ struct PairCfg {
   static_assert(!LOCK || NSUB == 2, "lock step needs two sub-tiles");
   static_assert(EPW == 2 || EPW == 4, "two or four epilogue warps per lane quarter");
   static_assert((BNS0 / 64) % EPW == 0 && (BNS1 / 64) % EPW == 0, "every epilogue warp gets the same number of groups");
-  static_assert(EPW == 2 || EPI == EPI_SOFTMAX || EPI == EPI_NONE, "residual stages carry one group per warp pair");
+  static_assert(EPW == 2 || EPI == EPI_SOFTMAX || EPI == EPI_NONE || EPI == EPI_ELEMENTWISE, "residual stages carry one group per warp pair");
   static_assert(SMEM_BYTES <= 232448, "shared memory budget");
   static_assert(YBOXES >= 1, "at least one staging box per epilogue warp");
   static_assert(SMEM_BYTES > 116 * 1024, "one CTA per SM is assumed (TMEM allocation never waits for a co-resident CTA)");
@@ -117,6 +117,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
   using Cfg = PairCfg<EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW>;
   constexpr bool kIsRms = EPI == EPI_RMS_MAX || EPI == EPI_RMS_MAX_LINEAR;  // the latter: no GELU in stage 1
+  constexpr bool kIsPlain = EPI == EPI_NONE || EPI == EPI_ELEMENTWISE;      // no reduction: column blocks are independent
   constexpr int BN = Cfg::BN;
   constexpr int NSUB = Cfg::NSUB;
   constexpr int ESUB = Cfg::ESUB;
@@ -381,10 +382,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int sub = 0; sub < ESUB && ok; ++sub) {
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
-          if (EPI == EPI_NONE && !unit_live(mpair0, group_col(ncta0, lg0))) continue;
+          if (kIsPlain && !unit_live(mpair0, group_col(ncta0, lg0))) continue;
           for (int g = h; g < W / 64; g += EPW) {
             const int col = group_col(ncta0, lg0 + g);
-            if (EPI == EPI_NONE && col >= p.N) break;
+            if (kIsPlain && col >= p.N) break;
             if (in_ring) {
               if (!mbar_wait<false>(bar_ylast(e, kk), 0, w)) { ok = false; break; }
 #ifdef COMFUSE_TRACE
@@ -532,7 +533,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       };
       auto tmem_of = [&](int sub) { return tmem_base + lane_sel + (slot[sub] ? BNS0 : 0); };
 
-      if constexpr (EPI == EPI_NONE) {
+      if constexpr (kIsPlain) {
 #pragma unroll
         for (int sub = 0; sub < ESUB; ++sub) {
           if (!live[sub]) continue;
@@ -540,15 +541,43 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const int W = unit_width(sub);
           const int lg0 = unit_lg0(sub);
           for (int g = h; g < W / 64; g += EPW) {
-            if (group_col(ncta0, lg0 + g) >= p.N) break;
+            const int gcol = group_col(ncta0, lg0 + g);
+            if (gcol >= p.N) break;
             uint32_t pk[32];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               uint32_t v[32];
               tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              if constexpr (EPI == EPI_ELEMENTWISE) {
+                // y = act(alpha * acc + bias): the bias of these 32 columns straight from global memory (bf16 pairs; the
+                // column block differs from tile to tile, N is a multiple of 8 and the group starts on a multiple of 64)
+                const int c0 = gcol + half * 32;
+                const float2 al = splat2(p.alpha);
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                for (int j = 0; j < 16; ++j) {
+                  float2 bb = splat2(0.f);
+                  if (p.bias && c0 + 2 * j < p.N) bb = bf16x2_to_f2(__ldg(reinterpret_cast<const uint32_t*>(p.bias + c0) + j));
+                  float2 z = fma2(al, f2_from_bits(v[2 * j], v[2 * j + 1]), bb);
+                  switch (p.activation) {
+                    case COMFUSE_OP_RELU: z = make_float2(fmaxf(z.x, 0.f), fmaxf(z.y, 0.f)); break;
+                    case COMFUSE_OP_GELU_TANH: z = gelu_tanh_f32x2(z); break;
+                    case COMFUSE_OP_TANH:
+                      z = make_float2(1.f - 2.f * __fdividef(1.f, 1.f + ex2_approx(2.8853900817779268f * z.x)),
+                                      1.f - 2.f * __fdividef(1.f, 1.f + ex2_approx(2.8853900817779268f * z.y)));
+                      break;
+                    case COMFUSE_OP_SIGMOID:
+                      z = make_float2(__fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z.x)),
+                                      __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * z.y)));
+                      break;
+                    default: break;
+                  }
+                  pk[half * 16 + j] = pack_bf16x2_rn(z.x, z.y);
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              }
             }
             store_box(pk);
           }

@@ -7,7 +7,9 @@
 namespace comfuse {
 
 // EPI_RMS_MAX_LINEAR: the RMSNorm op list without its GELU (a kernel instantiation of its own, chosen by FusedParams::no_activation)
-enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3, EPI_RMS_MAX_LINEAR = 4, EPI_PROGRAM = 5 };
+// EPI_ELEMENTWISE: Y = act(alpha * Acc + bias), no reduction: the plain GEMM's tiling (any N, all SMs, two accumulator
+// slots) with the activation in its store epilogue; FusedParams::activation is the comfuse_op_t of the unary node (0 = none)
+enum : int { EPI_NONE = 0, EPI_LN = 1, EPI_RMS_MAX = 2, EPI_SOFTMAX = 3, EPI_RMS_MAX_LINEAR = 4, EPI_PROGRAM = 5, EPI_ELEMENTWISE = 6 };
 
 // ---------------------------------------------------------------------------------------------------------------
 // Stage program: an epilogue given as data, lowered for the on-chip interpreter of the fused kernel (EPI_PROGRAM).
@@ -94,6 +96,7 @@ struct FusedParams {
   int post_relu;      // LayerNorm kind: Y = max(Y, 0) after the affine step
   int no_activation;  // RMSNorm kind: no GELU in stage 1
   float softcap;      // softmax kind: > 0 = scaled scores pass through softcap * tanh(. / softcap)
+  int activation;     // EPI_ELEMENTWISE: relu / gelu_tanh / tanh / sigmoid as comfuse_op_t, 0 = none
   const uint16_t* bias;
   const uint16_t* gamma;
   const uint16_t* beta;

@@ -160,6 +160,7 @@ struct FusedMatch {
   int causal = 0;
   int bias = -1, residual = -1, gamma = -1, beta = -1;  // parameter slots, -1 = absent
   int row_max_out = -1, row_argmax_out = -1;            // positions in row_outputs, -1 = not asked for
+  int activation = 0;                                   // BIAS_ACTIVATION kind: comfuse_op_t of the unary node, 0 = none
 };
 
 struct Matcher {
@@ -356,7 +357,28 @@ bool match_softmax(const Analysis& an, FusedMatch& m) {
   return true;
 }
 
+// act(alpha * acc + bias) with nothing else alive: no reduction, no row output
+bool match_elementwise(const Analysis& an, FusedMatch& m) {
+  if (!an.row_outputs.empty() || an.n_reductions != 0) return false;
+  Matcher t(an);
+  int k = an.terminal, other, hit;
+  for (int op : {COMFUSE_OP_RELU, COMFUSE_OP_GELU_TANH, COMFUSE_OP_TANH, COMFUSE_OP_SIGMOID})
+    if (m.activation == 0 && t.is(k, op)) { m.activation = op; t.use(k); k = t.nd(k).in0; }
+  if (t.split(k, COMFUSE_OP_ADD, [&](int q) { return t.is(q, COMFUSE_OP_ROWVEC); }, other, hit)) {
+    m.bias = t.nd(hit).param; t.use(k); t.use(hit); k = other;
+  }
+  if (t.split(k, COMFUSE_OP_MUL, [&](int q) { return t.is_const(q); }, other, hit)) {
+    m.alpha = an.cval[hit]; t.use(k); k = other;
+  }
+  if (!t.is(k, COMFUSE_OP_ACC)) return false;
+  t.use(k);
+  if (!t.all_live_used()) return false;
+  m.kind = COMFUSE_EPI_BIAS_ACTIVATION;
+  return true;
+}
+
 bool match_fused(const Analysis& an, FusedMatch& m) {
+  { FusedMatch t; if (match_elementwise(an, t)) { m = t; return true; } }
   { FusedMatch t; if (match_layernorm(an, t)) { m = t; return true; } }
   { FusedMatch t; if (match_rmsnorm(an, t)) { m = t; return true; } }
   { FusedMatch t; if (match_softmax(an, t)) { m = t; return true; } }
@@ -754,7 +776,9 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
   if (want_fused == 1 && match_fused(dc.an, dc.match)) {
     const comfuse_gemm_desc_t d = fused_desc(*shape, dc.match, shape->N);
     size_t ws = 0;
-    if (comfuse_workspace_size(&d, &ws) == COMFUSE_OK) {
+    if (dc.match.kind == COMFUSE_EPI_BIAS_ACTIVATION) {
+      dc.fused = true;  // the plain GEMM's tiling takes any shape the validation let through
+    } else if (comfuse_workspace_size(&d, &ws) == COMFUSE_OK) {
       dc.fused = true;
       dc.fused_inner_ws = (ws + 255) & ~static_cast<size_t>(255);
       if (dc.match.kind == COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX && (dc.match.row_max_out < 0 || dc.match.row_argmax_out < 0))
@@ -865,6 +889,12 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
   if (need > 0 && (!workspace || workspace_bytes < need)) return COMFUSE_ERR_WORKSPACE;
   if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return COMFUSE_ERR_ALIGNMENT;
 
+  if (dc.fused && dc.match.kind == COMFUSE_EPI_BIAS_ACTIVATION) {
+    const FusedMatch& m = dc.match;
+    return run_gemm_elementwise(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
+                                shape->batch_stride_b, shape->batch_stride_y, A, B, Y, m.bias >= 0 ? params[m.bias] : nullptr, m.alpha,
+                                m.activation, static_cast<cudaStream_t>(cuda_stream));
+  }
   if (dc.fused) {
     const FusedMatch& m = dc.match;
     const comfuse_gemm_desc_t d = fused_desc(*shape, m, m.residual >= 0 ? ld[m.residual] : shape->N);

@@ -58,6 +58,8 @@ bool softmax_rows_supported(const FusedParams& p);
 cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 // Plain GEMM, Z = bf16(A.B) through maps.Y, any N that is a multiple of 8.
 cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t st);
+// Y = act(alpha * A.B + bias) with the plain GEMM's tiling; p.activation = comfuse_op_t of the unary node, 0 = none.
+cudaError_t launch_gemm_elementwise(const GemmMaps& maps, FusedParams p, cudaStream_t st);
 
 }  // namespace comfuse
 
@@ -71,6 +73,10 @@ comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
                                    cudaStream_t st, bool query_only);
+// Y = act(alpha * A . B + bias) (reduction-free epilogue), any N that is a multiple of 8; bias may be null.
+comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
+                                      long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
+                                      const void* bias, float alpha, int activation, cudaStream_t st);
 // Z = bf16(A . B), dense [batch, M, N] (ld = N), with the plain tensor-core GEMM kernel; arguments already validated.
 comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
                               long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st);

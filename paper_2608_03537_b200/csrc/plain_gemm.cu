@@ -11,4 +11,11 @@ cudaError_t launch_plain_gemm(const GemmMaps& maps, FusedParams p, cudaStream_t 
   return launch_pair_instance<EPI_NONE, 256, 0, 1, 5>(maps, p, st);
 }
 
+// Y = act(alpha * A.B + bias): the same tiling with the activation in the store epilogue (reduction-free epilogues).
+cudaError_t launch_gemm_elementwise(const GemmMaps& maps, FusedParams p, cudaStream_t st) {
+  constexpr int BN = 256;
+  p.nblocks = (p.N + BN - 1) / BN;
+  return launch_pair_instance<EPI_ELEMENTWISE, 256, 0, 1, 5>(maps, p, st);
+}
+
 }  // namespace comfuse

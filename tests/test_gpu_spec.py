@@ -308,3 +308,44 @@ def test_program_workload_at_bench_size_sampled_rows_and_graph_replay():
     assert torch.equal(Yf.min(-1).values, torch.zeros(M, device=dev))
     picked = Yf.gather(-1, ro[4].long()[:, None])[:, 0]
     assert torch.equal(picked, Yf.max(-1).values)
+
+
+@pytest.mark.parametrize("act", [None, "relu", "gelu_tanh", "tanh", "sigmoid"])
+@pytest.mark.parametrize("M,N,K", [(300, 1000, 136), (520, 128, 1024), (64, 4096, 64)])
+def test_reduction_free_program_runs_on_the_plain_tiling(act, M, N, K):
+    """act(alpha * acc + bias) lowers to the GEMM kernel with the activation in its store epilogue: one launch, any N."""
+    nodes = [("acc", -1, -1, -1, 0.0), ("const", -1, -1, -1, 0.75), ("mul", 0, 1, -1, 0.0), ("rowvec", -1, -1, 0, 0.0), ("add", 3, 2, -1, 0.0)]
+    if act:
+        nodes.append((act, 4, -1, -1, 0.0))
+    prog = wl.SpecProgram(nodes, len(nodes) - 1, (), ("rowvec",))
+    A, B, params = _inputs(51, 1, M, N, K, prog.param_kinds)
+    Y, _, plan, launches = _run(prog, A, B, params, True, 1, M, N)
+    assert plan.path == cf.SPEC_PATH_FUSED_KERNEL and plan.fused_kind == cf.EPI_BIAS_ACTIVATION and launches == 1
+    assert plan.alpha == pytest.approx(0.75)
+    Yref, _ = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    scale = max(1.0, float(np.abs(Yref).max()))
+    assert np.isfinite(err).all() and err.max() <= 2.0 ** -8 * scale, (err.max(), scale)   # bf16 output rounding + approximations
+
+
+def test_two_layer_mlp_of_the_dlrm_shape_as_two_program_calls():
+    """1024 -> 512 -> 128 with ReLU after each layer (the DLRM shape of Sec. 6.2, Table II, which has no fused B2B kernel
+    here): two reduction-free program calls, the bf16 hidden layer goes through global memory."""
+    M = 1000
+    g = 61
+    X = wl.normal_bf16(g, 0, (M, 1024))
+    W1 = wl.normal_bf16(g, 1, (1024, 512), std=1024 ** -0.5)
+    W2 = wl.normal_bf16(g, 2, (512, 128), std=512 ** -0.5)
+    b1 = wl.uniform_bf16(g, 3, (512,), -0.1, 0.1)
+    b2 = wl.uniform_bf16(g, 4, (128,), -0.1, 0.1)
+    layer = wl.SpecProgram([("acc", -1, -1, -1, 0.0), ("rowvec", -1, -1, 0, 0.0), ("add", 0, 1, -1, 0.0), ("relu", 2, -1, -1, 0.0)], 3, (), ("rowvec",))
+    H, _, plan1, l1 = _run(layer, X, W1, [b1], True, 1, M, 512)
+    Hbits = H.view(torch.int16).cpu().numpy().view(np.uint16)
+    O, _, plan2, l2 = _run(layer, Hbits, W2, [b2], True, 1, M, 128)
+    assert plan1.fused_kind == plan2.fused_kind == cf.EPI_BIAS_ACTIVATION and l1 == l2 == 1
+    f = wl.bf16_to_f64
+    Href = np.maximum(f(X) @ f(W1) + f(b1), 0.0)
+    Oref = np.maximum(Href @ f(W2) + f(b2), 0.0)
+    assert np.abs(to_f64(H) - Href).max() <= 2.0 ** -8 * max(1.0, np.abs(Href).max())
+    # the second layer sees the bf16-rounded hidden activations
+    assert np.abs(to_f64(O) - Oref).max() <= 3e-2 and np.abs(to_f64(O) - Oref).mean() <= 3e-3

@@ -118,8 +118,14 @@ def test_on_chip_lowering_needs_one_resident_tensor():
     p = wl.spec_gated_minmax()
     pl = _plan(p.nodes, p.terminal, 1, p.row_outputs)
     assert pl.path == ROW and pl.program_path == ROW
-    # no reduction at all: a single pass
+    # no reduction at all: act(acc + bias) is a compiled reduction-free kind (the plain GEMM's tiling, any N); on the
+    # interpreter it is a single pass
     pl = _plan([N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0)], 3, 1)
+    assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.fused_kind == cf.EPI_BIAS_ACTIVATION and pl.program_path == PROG and pl.n_passes == 1
+    pl = _plan([N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0)], 3, 1, shape=cf.make_gemm_shape(1, 300, 1000, 72))
+    assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.program_path == ROW          # any row length
+    # two element-wise steps behind the bias: not that kind, still one resident tensor
+    pl = _plan([N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0), ("square", 3, -1, -1, 0)], 4, 1)
     assert pl.path == PROG and pl.n_passes == 1
     # a reduction of something below the resident tensor (max of the raw accumulator while x = acc + bias is kept)
     nodes = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("rmax", 0, -1, -1, 0), ("mean", 2, -1, -1, 0), ("sub", 2, 4, -1, 0),
