@@ -289,3 +289,13 @@ def test_matmul_scale_tanh_softcap_softmax_pattern(batch, M, N, K, causal, cap, 
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     P.check_outputs(w, got, P.run_oracle(w), label=f"softcap {cap} b{batch} {M}x{N}x{K} causal={causal} fused={fused}",
                     softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_layernorm_with_a_large_common_offset(fused, cuda_device):
+    """Rows whose mean is ~60 times their standard deviation: the statistics must not cancel (chunk-centred partial sums
+    merged with the pairwise update, not sum and sum of squares)."""
+    w = wl.post_norm(300, 1024, 136, seed=91, affine=True)
+    w.tensors["bias"] = wl.f32_to_bf16_bits(np.full(1024, 64.0, dtype=np.float32))
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"large offset fused={fused}")
