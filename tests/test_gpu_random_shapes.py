@@ -9,6 +9,12 @@ from tests import parity as P
 
 pytestmark = pytest.mark.gpu
 
+
+def _N(default):
+    """Seeds per test; COMFUSE_FUZZ_SEEDS scales the sweep for a longer soak."""
+    import os
+    return range(int(os.environ.get("COMFUSE_FUZZ_SEEDS", default)))
+
 ROW_LENGTHS = [256, 512, 768, 1024, 2048, 4096]
 
 
@@ -43,7 +49,7 @@ def _case(seed):
     return w, fused
 
 
-@pytest.mark.parametrize("seed", range(200))
+@pytest.mark.parametrize("seed", _N(200))
 def test_random_shape_and_operands(seed, cuda_device):
     w, fused = _case(7000 + seed)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
@@ -56,10 +62,15 @@ def test_random_shape_and_operands(seed, cuda_device):
         # the unfused baseline normalises the bf16-rounded GEMM result: on outputs of magnitude 4 .. 8 (half-ulp 1.56e-2) an
         # occasional element lands just above 3e-2 (seen: 3.03e-2); the fused kernels are held to 3e-2
         kw["norm_tol"] = 4e-2
-    P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused} {sorted(w.tensors)} {w.scalars}", **kw)
+    ref = P.run_oracle(w)
+    if w.kind != wl.KIND_SCALE_MASK_SOFTMAX:
+        # the stated bound assumes outputs below 8 in magnitude (bf16 half-ulp 1.56e-2 on [4, 8)); the RMSNorm of GELU values
+        # without a residual reaches beyond that, where rounding alone is 3.1e-2: there the bound follows the magnitude
+        kw["norm_tol"] = max(kw.get("norm_tol", P.TOL_NORM_MAX), 2.0 ** -7 * float(np.abs(ref["Y"]).max()))
+    P.check_outputs(w, got, ref, label=f"{w.name} fused={fused} {sorted(w.tensors)} {w.scalars}", **kw)
 
 
-@pytest.mark.parametrize("seed", range(150))
+@pytest.mark.parametrize("seed", _N(150))
 def test_random_b2b_shapes(seed, cuda_device):
     """Back-to-back GEMM, both forms: random row counts (ragged tiles, fewer and more tiles than CTA pairs), every chunk count
     of the MLP form, both source lengths of the attention form, random scale; fused and unfused."""

@@ -13,9 +13,28 @@ from tests.parity import to_dev, to_f64
 
 pytestmark = pytest.mark.gpu
 
+
+def _N(default):
+    """Seeds per test; COMFUSE_FUZZ_SEEDS scales the sweep for a longer soak."""
+    import os
+    return range(int(os.environ.get("COMFUSE_FUZZ_SEEDS", default)))
+
 UNARY = ["neg", "abs", "square", "tanh", "relu", "sigmoid", "gelu_tanh", "exp"]
 BINARY = ["add", "sub", "mul", "max", "min", "div"]
 REDUCE = ["sum", "mean", "rmax", "rmin"]
+
+
+def _reference_on_rounded_z(A, B, nodes, terminal, params, row_outputs):
+    """The oracle evaluated behind the GEMM result rounded to bf16 (fp32 accumulate, round to nearest even): what the
+    row-program pathway is defined to compute."""
+    f = wl.bf16_to_f64
+    Z = (f(A) @ f(B)).astype(np.float32)
+    Zb = wl.bf16_to_f64(wl.f32_to_bf16_bits(Z))
+    vals = spo.eval_nodes(nodes, Zb, [f(p) for p in params])
+    M, N = Zb.shape
+    Y = np.broadcast_to(np.asarray(vals[terminal], dtype=np.float64), (M, N)).copy()
+    rows = [np.broadcast_to(np.asarray(vals[r], dtype=np.float64), (M, 1))[:, 0].copy() for r in row_outputs]
+    return Y, rows
 
 
 def _random_program(seed):
@@ -60,7 +79,7 @@ def _random_program(seed):
     return nodes, terminal, row_outputs, n_params
 
 
-@pytest.mark.parametrize("seed", range(64))
+@pytest.mark.parametrize("seed", _N(64))
 def test_random_program_matches_the_oracle_on_every_pathway(seed):
     M, N, K = 130, 256, 64
     nodes, terminal, row_outputs, n_params = _random_program(1000 + seed)
@@ -72,15 +91,20 @@ def test_random_program_matches_the_oracle_on_every_pathway(seed):
     big = max(float(np.max(np.abs(np.asarray(v)))) if np.all(np.isfinite(np.asarray(v))) else np.inf for v in vals)
     if not np.isfinite(big) or big > 1e3:
         pytest.skip("program leaves the bounded range")
-    Yref, Rref = spo.gemm_spec(f(A), f(B), nodes, terminal, [f(p) for p in params], row_outputs)
+    ref_exact = spo.gemm_spec(f(A), f(B), nodes, terminal, [f(p) for p in params], row_outputs)
+    ref_rounded = _reference_on_rounded_z(A, B, nodes, terminal, params, row_outputs)
     spec = cf.make_spec(nodes, terminal, n_params, row_outputs)
     shape = cf.make_gemm_shape(1, M, N, K)
     plan = cf.spec_plan(spec, shape)
     dev = "cuda:0"
     dA, dB, dP = to_dev(A), to_dev(B), [to_dev(p) for p in params]
-    scale = max(1.0, float(np.abs(Yref).max()))
     seen = set()
     for fused in (1, 2, 0):
+        path = plan.path if fused == 1 else (plan.program_path if fused == 2 else cf.SPEC_PATH_ROW_PROGRAM)
+        # the row-program pathway is defined on the bf16-rounded GEMM result: random programs can be arbitrarily sensitive
+        # to that rounding (tanh of a row sum near zero), so it is compared with the oracle evaluated on the rounded Z
+        Yref, Rref = ref_rounded if path == cf.SPEC_PATH_ROW_PROGRAM else ref_exact
+        scale = max(1.0, float(np.abs(Yref).max()))
         Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev)
         ro = [torch.full((M,), float("nan"), dtype=torch.float32, device=dev) for _ in row_outputs]
         ws = torch.empty(max(16, cf.gemm_spec_workspace_size(spec, shape, fused)), dtype=torch.uint8, device=dev)
@@ -92,7 +116,7 @@ def test_random_program_matches_the_oracle_on_every_pathway(seed):
         for got, ref in zip(ro, Rref):
             rs = max(1.0, float(np.abs(ref).max()))
             assert np.abs(got.cpu().numpy().astype(np.float64) - ref).max() <= 3e-2 * rs, (seed, fused, "row output")
-        seen.add(plan.path if fused == 1 else (plan.program_path if fused == 2 else cf.SPEC_PATH_ROW_PROGRAM))
+        seen.add(path)
     assert cf.SPEC_PATH_ROW_PROGRAM in seen
 
 
@@ -160,7 +184,7 @@ def _random_chain_program(seed):
     return nodes, y, tuple(outs), n_params
 
 
-@pytest.mark.parametrize("seed", range(160))
+@pytest.mark.parametrize("seed", _N(160))
 def test_random_chain_program_on_the_on_chip_interpreter(seed):
     M, N, K = (300, 1024, 72) if seed % 2 else (130, 256, 64)
     nodes, terminal, row_outputs, n_params = _random_chain_program(5000 + seed)
@@ -175,7 +199,8 @@ def test_random_chain_program_on_the_on_chip_interpreter(seed):
     big = max(float(np.max(np.abs(np.asarray(v)))) if np.all(np.isfinite(np.asarray(v))) else np.inf for v in vals)
     if not np.isfinite(big) or big > 1e3 * N:
         pytest.skip("program leaves the bounded range")
-    Yref, Rref = spo.gemm_spec(f(A), f(B), nodes, terminal, [f(p) for p in params], row_outputs)
+    ref_exact = spo.gemm_spec(f(A), f(B), nodes, terminal, [f(p) for p in params], row_outputs)
+    ref_rounded = _reference_on_rounded_z(A, B, nodes, terminal, params, row_outputs)
     spec = cf.make_spec(nodes, terminal, n_params, row_outputs)
     shape = cf.make_gemm_shape(1, M, N, K)
     plan = cf.spec_plan(spec, shape)
@@ -183,8 +208,9 @@ def test_random_chain_program_on_the_on_chip_interpreter(seed):
         pytest.skip("beyond the interpreter's limits")
     dev = "cuda:0"
     dA, dB, dP = to_dev(A), to_dev(B), [to_dev(p) for p in params]
-    scale = max(1.0, float(np.abs(Yref).max()))
     for fused in (2, 0):
+        Yref, Rref = ref_exact if fused == 2 else ref_rounded
+        scale = max(1.0, float(np.abs(Yref).max()))
         Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev)
         ro = [torch.full((M,), -1, dtype=torch.int32 if nodes[r][0] == "argmax" else torch.float32, device=dev) for r in row_outputs]
         ws = torch.empty(max(16, cf.gemm_spec_workspace_size(spec, shape, fused)), dtype=torch.uint8, device=dev)
