@@ -85,3 +85,21 @@ def test_random_b2b_shapes(seed, cuda_device):
         w.scalars["alpha"] = float(np.round(g.uniform(0.02, 0.6 if fused else 0.12), 3))
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused} {w.scalars}")
+
+
+@pytest.mark.parametrize("seed", _N(24))
+def test_random_wide_rows(seed, cuda_device):
+    """Rows wider than one cluster (two-kernel path): N = k x 4096, random M and K, LayerNorm / RMSNorm with their flags."""
+    g = np.random.default_rng(11000 + seed)
+    N = 4096 * int(g.integers(2, 6))
+    M, K = int(g.integers(1, 400)), int(g.integers(1, 20)) * 8
+    if g.random() < 0.5:
+        w = wl.post_norm(M, N, K, seed=seed, affine=bool(g.random() < 0.6), relu=bool(g.random() < 0.4))
+    else:
+        w = wl.complex_subgraph(M, N, K, seed=seed, activation=bool(g.random() < 0.6), residual=bool(g.random() < 0.7))
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    ref = P.run_oracle(w)
+    kw = {"norm_tol": max(4e-2, 2.0 ** -7 * float(np.abs(ref["Y"]).max()))}   # the un-normalised row passes through bf16 once
+    if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+        kw["rowmax_tol"] = 3e-2
+    P.check_outputs(w, got, ref, label=f"{w.name} wide {sorted(w.tensors)} {w.scalars}", **kw)
