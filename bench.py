@@ -457,6 +457,39 @@ def run_comfuse(args):
         ms_gemm = timed(n3, lambda i: gemm_only(sets[i % nsets])) / n3
         extra["gemm_only_ms_per_step"] = ms_gemm
         extra["gemm_only_impl"] = "torch.matmul (vendor library), bf16 output"
+        # ---- context: the same subgraph as framework library calls on the same buffers (vendor GEMM, vendor / framework
+        # element-wise, normalisation, softmax and attention kernels), each op its own launch(es)
+        import torch.nn.functional as F
+
+        def eager(sx):
+            if program:
+                return None
+            if attention:   # keys in the layout the library call wants ([S, d], made once, outside the timed region)
+                if "K_rows" not in sx:
+                    sx["K_rows"] = sx["W1"].transpose(1, 2).contiguous()
+                return F.scaled_dot_product_attention(sx["X"].unsqueeze(0), sx["K_rows"].unsqueeze(0), sx["W2"].unsqueeze(0), scale=w.scalars["alpha"])
+            if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
+                hid = F.gelu(torch.addmm(sx["b1"], sx["X"], sx["W1"]), approximate="tanh")
+                return F.layer_norm(torch.addmm(sx["b2"], hid, sx["W2"]) + sx["X"], (d["N2"],), sx.get("gamma"), sx.get("beta"), w.scalars["eps"])
+            if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+                return F.layer_norm(torch.addmm(sx["bias"], sx["A"], sx["B"]) + sx["residual"], (d["N"],), sx.get("gamma"), sx.get("beta"), w.scalars["eps"])
+            if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
+                y = F.rms_norm(F.gelu(torch.addmm(sx["bias"], sx["A"], sx["B"]), approximate="tanh") + sx["residual"], (d["N"],), sx["gamma"], w.scalars["eps"])
+                return y.max(dim=-1)
+            t = torch.bmm(sx["A"], sx["B"]) * w.scalars["alpha"]
+            if w.scalars.get("causal"):
+                t = t.masked_fill(causal_mask, float("-inf"))
+            return torch.softmax(t, dim=-1)
+        if not program:
+            causal_mask = torch.ones(d["M"], d.get("N", 1), dtype=torch.bool, device=dev).triu(1) if w.scalars.get("causal") else None
+            try:
+                for i in range(max(3, nsets)):
+                    eager(sets[i % nsets])
+                extra["torch_eager_ms_per_step"] = timed(n3, lambda i: eager(sets[i % nsets])) / n3
+                extra["torch_eager_impl"] = ("F.scaled_dot_product_attention" if attention else
+                                             "torch.addmm / bmm + framework element-wise, normalisation and softmax kernels") + ", bf16"
+            except Exception as ex:  # an op missing from this torch build is no reason to lose the bench line
+                extra["torch_eager_error"] = repr(ex)[:200]
         fused_ms = ms_step if fused else extra.get("fused_ms_per_step")
         unfused_ms = extra.get("unfused_ms_per_step") if fused else ms_step
         extra["residual_ms"] = {"fused": None if fused_ms is None else fused_ms - ms_gemm,
