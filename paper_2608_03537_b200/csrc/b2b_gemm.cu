@@ -99,6 +99,9 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int my_tiles = cluster_id < total_tiles ? (total_tiles - cluster_id + num_clusters - 1) / num_clusters : 0;
   const int nsub = my_tiles * nhalf;
   constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
+  // The attention form's epilogue, not its loads, sets the pace: it walks seven of the eight ring slots and uses the
+  // eighth as a second output staging box, so that both 64-column halves of a tile are staged and stored together.
+  constexpr int RING = MODE == 1 ? kRingSlots - 1 : kRingSlots;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 #ifdef COMFUSE_TRACE
@@ -146,7 +149,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      RingPos<kRingSlots> ring;
+      RingPos<RING> ring;
       bool ok = true;
       // one box into the current slot; kind 0: pair operand (signals the even CTA's full barrier), 1: residual
       int bz = 0;  // batch coordinate of the current tile
@@ -207,7 +210,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     if (lane == 0 && pm == 0) {
       constexpr uint32_t idesc_ml1 = make_idesc_bf16(256, 128, false, true);
       constexpr uint32_t idesc_ml2 = make_idesc_bf16(256, 128, false, true);
-      RingPos<kRingSlots> ring;
+      RingPos<RING> ring;
       uint32_t full_bits = 0;
       uint32_t sfull_uses[2] = {0, 0};
       uint32_t tile_it = 0;
@@ -383,7 +386,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const uint32_t oempty_leader = map_to_cta(bar_oempty(0), leader);
     const int kblk = hh >> 1;            // K block of S (and residual box) this thread's columns fall into
     const int chunk0 = (hh & 1) * 4;     // first of its four 16-byte chunks inside that 128-byte row
-    RingPos<kRingSlots> ring;
+    RingPos<RING> ring;
     uint32_t rfull_bits = 0;
     uint32_t puses[2] = {0, 0}, suses[2] = {0, 0};
     uint32_t tile_it = 0;
@@ -414,6 +417,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
         __syncwarp();
         tcgen05_fence_after_sync();
+        B2B_TRACE_POINT();  // scores of the sub-tile complete
         const float sc = p.alpha * 1.4426950408889634f;  // log2 domain
         uint32_t v0[32], v1[32];
         tmem_ld_32cols(tmem_base + lane_sel + 0 * 128 + hh * 32, v0);
@@ -447,6 +451,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         const float lloc = (a0.x + a0.y) + (a1.x + a1.y);
         const float2 tot = cluster_row_reduce<1, MergeMaxSumExp2, 4>(make_float2(mloc, lloc), 64.f, MergeMaxSumExp2(), s_pre, s_stats,
                                                                      bar_stats, row, hh, 0u, xpar, xphase, w);
+        B2B_TRACE_POINT();  // exponentials done, row statistics merged
         const float f = ex2_approx(mloc - tot.x);  // this thread's exponentials are relative to its own maximum
         // the S buffers are free once ML2 of the previous tile has read them
         for (int pb = 0; pb < 2; ++pb) {
@@ -454,6 +459,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           ++suses[pb];
         }
         __syncwarp();
+        B2B_TRACE_POINT();  // S buffers free
 #pragma unroll
         for (int pb = 0; pb < 2; ++pb) {
           const uint32_t(&vv)[32] = pb ? v1 : v0;
@@ -475,6 +481,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           mbar_arrive_cluster_noflush(sfull_leader);
           mbar_arrive_cluster_noflush(sfull_leader + 8u);
         }
+        B2B_TRACE_POINT();  // S handed to the tensor pipe
         return tot;  // (row maximum in the log2 domain, sum of 2^(t - maximum)) of this sub-tile
       };
       // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes through one staging buffer
@@ -489,6 +496,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           mbar_wait<false>(bar_ofull(obuf), (it >> 1) & 1u, w);
           __syncwarp();
           tcgen05_fence_after_sync();
+          B2B_TRACE_POINT();  // S.V of the tile complete
           uint32_t v[32];
           tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + hh * 32, v);
 #pragma unroll
@@ -520,25 +528,27 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
             mbar_arrive_cluster_noflush(oempty_leader + 8u);
           }
         }
-        for (int g = 0; g < 2; ++g) {
-          if (store_thread) tma_store_wait_read<0>();
-          named_barrier_sync(3, kB2bEpiThreads);
-          if (kblk == g) {
+        // both halves at once: columns 0..63 go to the staging box, columns 64..127 to the idle eighth ring slot
+        if (store_thread) tma_store_wait_read<0>();  // the previous tile's stores have read both boxes
+        named_barrier_sync(3, kB2bEpiThreads);
+        {
+          const uint32_t box = kblk == 0 ? ybuf : ring_addr(kRingSlots - 1);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t a = ybuf + swz128(row, chunk0 + i);
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                           "r"(pk[4 * i + 3])
-                           : "memory");
-            }
-          }
-          fence_proxy_async_smem();
-          named_barrier_sync(3, kB2bEpiThreads);
-          if (store_thread) {
-            tma_store_3d(&tmO, ybuf, g * 64, m0, bz);
-            tma_store_commit();
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t a = box + swz128(row, chunk0 + i);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                         "r"(pk[4 * i + 3])
+                         : "memory");
           }
         }
+        fence_proxy_async_smem();
+        named_barrier_sync(3, kB2bEpiThreads);
+        if (store_thread) {
+          tma_store_3d(&tmO, ybuf, 0, m0, bz);
+          tma_store_3d(&tmO, ring_addr(kRingSlots - 1), 64, m0, bz);
+          tma_store_commit();
+        }
+        B2B_TRACE_POINT();  // tile stored
       };
       // Order (the S buffers and the O slots are handed back by the steps named behind the arrows):
       //   one sub-tile per row tile:   softmax(0) | softmax(t+1), finish(t) ...
@@ -630,7 +640,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       uint32_t pk[16];
       {
       const int s0 = ring.stage;
-      const int s1 = s0 + 1 == kRingSlots ? 0 : s0 + 1;
+      const int s1 = s0 + 1 == RING ? 0 : s0 + 1;
       // both residual slots are waited for by everybody (the phase bits must advance uniformly)
       mbar_wait<false>(bar_rfull(s0), (rfull_bits >> s0) & 1u, w);
       rfull_bits ^= 1u << s0;
