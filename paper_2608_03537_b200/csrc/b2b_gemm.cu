@@ -101,6 +101,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
   // The attention form's epilogue, not its loads, sets the pace: it walks seven of the eight ring slots and uses the
   // eighth as a second output staging box, so that both 64-column halves of a tile are staged and stored together.
+  // (The MLP form cannot give a slot away: X0, X1 stay at the head of the ring until ML1 of the last chunk has been
+  // issued, and W1 of that chunk is the eighth item behind them -- with seven slots the producer would wait for X0.)
   constexpr int RING = MODE == 1 ? kRingSlots - 1 : kRingSlots;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
