@@ -87,9 +87,10 @@ typedef struct {
 #define COMFUSE_FLAG_POST_RELU 1u      /* BIAS_RES_LAYERNORM kind only: Y = max(Y, 0) after the affine step            */
 #define COMFUSE_FLAG_NO_ACTIVATION 2u  /* BIAS_GELU_RES_RMSNORM_MAX kind only: H = alpha*A.B + bias + R, no GELU       */
 
-/* Runtime-parameter table of the op list.  bf16 device vectors of length N; NULL means absent
- * (bias, residual: 0; gamma: 1; beta: 0).  row_max / row_argmax: [batch*M] outputs of the
- * RMSNORM_MAX kind, required there and ignored elsewhere. */
+/* Runtime-parameter table of the op list.  bias, gamma, beta: bf16 device vectors of length N, shared by all batches;
+ * residual: bf16 [batch, M, N] with leading dimension desc->ldr; mask: see comfuse_mask_t.  NULL means absent (bias,
+ * residual: 0; gamma: 1; beta: 0).  row_max (fp32) / row_argmax (int32): [batch*M] outputs of the RMSNORM_MAX kind,
+ * required there and ignored elsewhere. */
 typedef struct {
   const void* bias;
   const void* residual;
