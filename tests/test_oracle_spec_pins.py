@@ -207,3 +207,30 @@ def test_programs_against_scalar_loops(name):
 def test_forward_edges_are_rejected():
     with pytest.raises(ValueError):
         spo.eval_nodes([("acc", -1, -1, -1, 0.0), ("add", 0, 2, -1, 0.0), ("const", -1, -1, -1, 1.0)], np.zeros((2, 2)))
+
+
+# ----------------------------------------------------------------------------- the two oracles agree where they overlap
+def test_programs_agree_with_the_op_list_oracle():
+    """The primitive spellings evaluated by the node-list oracle equal the op-list oracle's closed definitions (both are
+    pinned separately above and in test_oracle_pins.py; this ties the two together)."""
+    from oracle import comfuse_oracle as orc
+    M, K, N = 9, 16, 48
+    A, B = _inputs(31, M, K, N)
+    g = _rng(32)
+    bias, R, gamma, beta = g.standard_normal(N), g.standard_normal((M, N)), g.standard_normal(N), g.standard_normal(N)
+    p = wl.spec_layernorm(eps=1e-5, relu=True)
+    Y, _ = spo.gemm_spec(A, B, p.nodes, p.terminal, (bias, R, gamma, beta))
+    np.testing.assert_allclose(Y, orc.bias_res_layernorm(A, B, bias, R, gamma, beta, 1.0, 1e-5, relu=True), rtol=0, atol=1e-12)
+    p = wl.spec_rmsnorm_max(eps=1e-5)
+    Y, (mx, am) = spo.gemm_spec(A, B, p.nodes, p.terminal, (bias, R, gamma), p.row_outputs)
+    Y2, mx2, am2 = orc.bias_gelu_res_rmsnorm_max(A, B, bias, R, gamma, 1.0, 1e-5)
+    np.testing.assert_allclose(Y, Y2, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(mx, mx2, rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(am.astype(np.int64), am2)
+    p = wl.spec_rmsnorm_max(eps=1e-5, activation=False, residual=False)
+    Y, _ = spo.gemm_spec(A, B, p.nodes, p.terminal, (bias, gamma), p.row_outputs)
+    np.testing.assert_allclose(Y, orc.bias_gelu_res_rmsnorm_max(A, B, bias, None, gamma, 1.0, 1e-5, activation=False)[0], rtol=0, atol=1e-12)
+    As, Bs = _inputs(33, 12, 8, 12)
+    p = wl.spec_softmax(alpha=0.3, causal=True, softcap=2.5)
+    Y, _ = spo.gemm_spec(As, Bs, p.nodes, p.terminal)
+    np.testing.assert_allclose(Y, orc.scale_mask_softmax(As, Bs, 0.3, orc.causal_mask(12, 12), softcap=2.5), rtol=0, atol=1e-13)
