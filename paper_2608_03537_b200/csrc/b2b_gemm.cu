@@ -119,7 +119,9 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_pfull(a), 1);
       mbar_init(bar_sfull(a), 2 * kB2bEpiWarps);   // one arrival per epilogue warp of both CTAs
-      mbar_init(bar_sempty(a), 1);
+      // S buffer 1 of the MLP form doubles as the second output staging box: handing it back takes the UMMA commit AND
+      // the store thread's word that the previous tile's output store has read it (see Epi1 / Epi2 below)
+      mbar_init(bar_sempty(a), (MODE == 0 && a == 1) ? 2 : 1);
       mbar_init(bar_ofull(a), 1);
       mbar_init(bar_oempty(a), 2 * kB2bEpiWarps);
     }
@@ -587,7 +589,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         __syncwarp();
         tcgen05_fence_after_sync();
         B2B_TRACE_POINT();
-        // the S buffer is free once ML2 of chunk j-2 has read it
+        // the S buffer is free once ML2 of chunk j-2 has read it -- and, for buffer 1, once the output store that staged
+        // its second box there has read it: the store thread adds that arrival to the phase of the buffer's previous use
+        if (pb == 1 && store_thread && suses[1] > 0) {
+          tma_store_wait_read<0>();
+          mbar_arrive(bar_sempty(1));
+        }
         mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
         ++suses[pb];
         __syncwarp();
@@ -722,25 +729,27 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       tcgen05_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
-      // two 128 x 64 boxes (columns 0..63 from the hh = 0, 1 warps, 64..127 from hh = 2, 3) through one staging buffer
-      for (int g = 0; g < 2; ++g) {
-        if (store_thread) tma_store_wait_read<0>();
-        named_barrier_sync(3, kB2bEpiThreads);
-        if (kblk == g) {
+      // two 128 x 64 boxes (columns 0..63 from the hh = 0, 1 warps, 64..127 from hh = 2, 3), staged and stored together:
+      // the second box sits in S buffer 1 (first K block), which is idle between the last ML2 of this tile -- complete,
+      // the O slot was full -- and Epi1 of chunk 1 of the next tile, which waits for this store's read (above)
+      if (store_thread) tma_store_wait_read<0>();  // the previous tile's stores have read both boxes
+      named_barrier_sync(3, kB2bEpiThreads);
+      {
+        const uint32_t box = kblk == 0 ? ybuf : s_addr(1, 0);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t a = ybuf + swz128(row, chunk0 + i);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                         "r"(pk[4 * i + 3])
-                         : "memory");
-          }
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t a = box + swz128(row, chunk0 + i);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                       "r"(pk[4 * i + 3])
+                       : "memory");
         }
-        fence_proxy_async_smem();
-        named_barrier_sync(3, kB2bEpiThreads);
-        if (store_thread) {
-          tma_store_3d(&tmO, ybuf, g * 64, m0, bz);
-          tma_store_commit();
-        }
+      }
+      fence_proxy_async_smem();
+      named_barrier_sync(3, kB2bEpiThreads);
+      if (store_thread) {
+        tma_store_3d(&tmO, ybuf, 0, m0, bz);
+        tma_store_3d(&tmO, s_addr(1, 0), 64, m0, bz);
+        tma_store_commit();
       }
     }
     if (store_thread) tma_store_wait_read<0>();  // the staging buffer must outlive the last store's read
