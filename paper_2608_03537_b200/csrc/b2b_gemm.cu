@@ -36,7 +36,7 @@ constexpr int kMaxChunks = 4;             // N1 <= 512
 struct B2bSmem {
   static constexpr int OFF_RING = 0;
   static constexpr int OFF_S = kRingSlots * kSlotBytes;            // 2 buffers x 2 K blocks
-  static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // one output staging box
+  static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // output staging box (the second one is borrowed, see Epi2)
   static constexpr int OFF_B1 = OFF_YBUF + kSlotBytes;             // fp32 [512]
   static constexpr int OFF_VEC = OFF_B1 + kMaxChunks * 128 * 4;    // b2, gamma, beta fp32 [128] each
   static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][4][128]
@@ -488,7 +488,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         B2B_TRACE_POINT();  // S handed to the tensor pipe
         return tot;  // (row maximum in the log2 domain, sum of 2^(t - maximum)) of this sub-tile
       };
-      // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes through one staging buffer
+      // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes staged and stored together
       // `it` = number of the row tile's first sub-tile; ml0 / ml1 = (maximum, sum) of its one or two sub-tiles
       auto finish_tile = [&](int tile, uint32_t it, float2 ml0, float2 ml1) {
         const int bz = tile / p.mpairs;
