@@ -176,6 +176,20 @@ def b2b_from_intermediate(S, X, W2, b2, gamma=None, beta=None, eps=1e-5):
     return layernorm_rows(O, gamma, beta, eps)
 
 
+def relu(x: np.ndarray) -> np.ndarray:
+    """Unary activation node: max(x, 0) (the ReLU of the MBLR pattern, Sec. 6.1)."""
+    return np.maximum(np.asarray(x, dtype=np.float64), 0.0)
+
+
+def b2b_mlp_relu(X, W1, b1, W2, b2):
+    """Sec. 4, Eq. 2 with F = ReLU(. + b1) and a ReLU tail: the two-layer bottom MLP the paper evaluates as its DLRM
+    workload (Sec. 6.2, Table II: feature dimensions 1024 -> 512 -> 128):
+        P = X W1,  S = ReLU(P + b1),  O = ReLU(S W2 + b2).
+    X [M, K], W1 [K, N1], W2 [N1, N2]; K and N2 are independent (no residual)."""
+    S = relu(gemm(X, W1) + np.asarray(b1, dtype=np.float64))
+    return relu(gemm(S, W2) + np.asarray(b2, dtype=np.float64))
+
+
 def b2b_softmax_attention(Q, Kt, V, alpha=1.0):
     """Sec. 4, Eq. 2 with F = row softmax (the attention-form instance the paper evaluates as Target-Attention,
     Sec. 6.2, Table II):  P = alpha * Q Kt,  S = softmax(P) over the source positions,  O = S V.

@@ -427,3 +427,32 @@ def test_b2b_softmax_attention_brute_force_and_properties():
         np.testing.assert_allclose(Ob[b], orc.b2b_softmax_attention(Qb[b], Kb[b], Vb[b], alpha), atol=1e-14)
     lib = torch.softmax(torch.from_numpy(Q) @ torch.from_numpy(Kt) * alpha, dim=-1) @ torch.from_numpy(V)
     np.testing.assert_allclose(O, lib.numpy(), atol=1e-13)
+
+
+def test_b2b_mlp_relu_brute_force_and_properties():
+    """The ReLU two-layer MLP (Sec. 4, Eq. 2 with F = ReLU(. + b1) and a ReLU tail; the DLRM workload of Sec. 6.2).
+    Scalar-loop brute force; a hand-computed 2 x 2 case with one clipped unit per layer; outputs are non-negative; without
+    biases the map is positively homogeneous (f(aX) = a f(X) for a > 0); a large positive b1 keeps every hidden unit active,
+    which reduces the hidden layer to an affine map; W2 = I, b2 = 0 leaves ReLU(X W1 + b1); library cross-check in fp64."""
+    r = _rng(60)
+    X, W1, b1 = r.standard_normal((5, 7)), r.standard_normal((7, 6)), r.standard_normal(6)
+    W2, b2 = r.standard_normal((6, 3)), r.standard_normal(3)
+    O = orc.b2b_mlp_relu(X, W1, b1, W2, b2)
+    for i in range(5):
+        s = [max(sum(X[i, k] * W1[k, j] for k in range(7)) + b1[j], 0.0) for j in range(6)]
+        for c in range(3):
+            assert abs(O[i, c] - max(sum(s[j] * W2[j, c] for j in range(6)) + b2[c], 0.0)) < 1e-13
+    # hand-computed: X = [[1, -2]], W1 = [[1, 2], [3, 1]] -> P = [-5, 0]; + b1 = [6, -1] -> [1, -1] -> S = [1, 0];
+    # W2 = [[2, -3], [5, 7]] -> [2, -3]; + b2 = [0.5, 1] -> [2.5, -2] -> O = [2.5, 0]
+    Oh = orc.b2b_mlp_relu([[1.0, -2.0]], [[1.0, 2.0], [3.0, 1.0]], [6.0, -1.0], [[2.0, -3.0], [5.0, 7.0]], [0.5, 1.0])
+    np.testing.assert_array_equal(Oh, [[2.5, 0.0]])
+    assert (O >= 0.0).all() and (O == 0.0).any() and (O > 0.0).any()
+    z6, z3 = np.zeros(6), np.zeros(3)
+    np.testing.assert_allclose(orc.b2b_mlp_relu(3.5 * X, W1, z6, W2, z3), 3.5 * orc.b2b_mlp_relu(X, W1, z6, W2, z3), atol=1e-12)
+    big = np.full(6, 100.0)
+    np.testing.assert_allclose(orc.b2b_mlp_relu(X, W1, big, W2, b2), np.maximum((X @ W1 + big) @ W2 + b2, 0.0), atol=1e-11)
+    np.testing.assert_allclose(orc.b2b_mlp_relu(X, W1, b1, np.eye(6), z6), np.maximum(X @ W1 + b1, 0.0), atol=1e-14)
+    lin = torch.nn.functional.linear
+    tX, tW1, tW2 = torch.from_numpy(X), torch.from_numpy(W1), torch.from_numpy(W2)
+    lib = torch.relu(lin(torch.relu(lin(tX, tW1.T, torch.from_numpy(b1))), tW2.T, torch.from_numpy(b2)))
+    np.testing.assert_allclose(O, lib.numpy(), atol=1e-13)

@@ -53,6 +53,10 @@ def test_affine_and_b2b_shapes():
     m = wl.b2b_mlp(256, 128, 512, 128, seed=4)
     assert m.tensors["W1"].shape == (128, 512) and m.tensors["W2"].shape == (512, 128)
     assert m.gemm_flops() == 2 * 256 * 128 * 512 * 2
+    d = wl.dlrm_bottom_mlp(256, 1024, 512, 128)
+    assert d.tensors["X"].shape == (256, 1024) and d.tensors["W1"].shape == (1024, 512) and d.tensors["W2"].shape == (512, 128)
+    assert d.gemm_flops() == 2 * 256 * (1024 * 512 + 512 * 128)
+    assert d.min_hbm_bytes() == 2 * (256 * 1024 + 1024 * 512 + 512 * 128 + 512 + 128 + 256 * 128)
     s = wl.scaled_masked_softmax(2, 128, 128, 64, seed=3)
     assert s.scalars["alpha"] == 0.125 and s.tensors["B"].shape == (2, 64, 128)
 

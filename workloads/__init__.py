@@ -89,6 +89,7 @@ KIND_BIAS_GELU_RES_RMSNORM_MAX = "bias_gelu_res_rmsnorm_max"
 KIND_SCALE_MASK_SOFTMAX = "scale_mask_softmax"
 KIND_B2B_MLP_LAYERNORM = "b2b_mlp_layernorm"
 KIND_B2B_SOFTMAX_ATTENTION = "b2b_softmax_attention"
+KIND_B2B_MLP_RELU = "b2b_mlp_relu"
 KIND_GEMM_PROGRAM = "gemm_program"   # epilogue given as a node list (Workload.program)
 
 
@@ -105,7 +106,7 @@ class Workload:
 
     def gemm_flops(self) -> float:
         d = self.dims
-        if self.kind in (KIND_B2B_MLP_LAYERNORM, KIND_B2B_SOFTMAX_ATTENTION):
+        if self.kind in (KIND_B2B_MLP_LAYERNORM, KIND_B2B_SOFTMAX_ATTENTION, KIND_B2B_MLP_RELU):
             return d.get("batch", 1) * (2.0 * d["M"] * d["K"] * d["N1"] + 2.0 * d["M"] * d["N1"] * d["N2"])
         return 2.0 * d.get("batch", 1) * d["M"] * d["N"] * d["K"]
 
@@ -114,6 +115,9 @@ class Workload:
         d = self.dims
         if self.kind == KIND_B2B_SOFTMAX_ATTENTION:
             return 2.0 * d["batch"] * (d["M"] * d["K"] + d["K"] * d["N1"] + d["N1"] * d["N2"] + d["M"] * d["N2"])
+        if self.kind == KIND_B2B_MLP_RELU:
+            M, K, N1, N2 = d["M"], d["K"], d["N1"], d["N2"]
+            return 2.0 * (M * K + K * N1 + N1 * N2 + N1 + N2 + M * N2)
         if self.kind == KIND_B2B_MLP_LAYERNORM:
             M, K, N1, N2 = d["M"], d["K"], d["N1"], d["N2"]
             return 2.0 * (M * K + K * N1 + N1 * N2 + N1 + N2 + M * N2) + (
@@ -196,6 +200,20 @@ def b2b_mlp(M=32768, K=128, N1=512, N2=128, seed=4, affine=False, name=None) -> 
                     {"M": M, "K": K, "N1": N1, "N2": N2}, {"eps": 1e-5}, t)
 
 
+def dlrm_bottom_mlp(M=32768, K=1024, N1=512, N2=128, seed=8, name=None) -> Workload:
+    """O = ReLU(ReLU(X.W1 + b1).W2 + b2): the two-layer bottom MLP with the paper's DLRM feature dimensions
+    1024 -> 512 -> 128.  X ~ N(0, 1), weights ~ N(0, 1 / fan-in), biases ~ U(-0.1, 0.1)."""
+    t = {
+        "X": normal_bf16(seed, 0, (M, K)),
+        "W1": normal_bf16(seed, 1, (K, N1), std=1.0 / math.sqrt(K)),
+        "b1": uniform_bf16(seed, 2, (N1,), -0.1, 0.1),
+        "W2": normal_bf16(seed, 3, (N1, N2), std=1.0 / math.sqrt(N1)),
+        "b2": uniform_bf16(seed, 4, (N2,), -0.1, 0.1),
+    }
+    return Workload(name or f"dlrm_bottom_mlp_{M}x{K}x{N1}x{N2}", KIND_B2B_MLP_RELU,
+                    {"M": M, "K": K, "N1": N1, "N2": N2}, {}, t)
+
+
 # The five named configurations (index = position in the benchmark's config list).
 def target_attention(batch=32, M=4096, S=256, d=128, seed=5, name=None) -> Workload:
     """O = softmax(Q.Kt / sqrt(d)).V per batch: M target positions attend to S source positions (the paper's
@@ -224,6 +242,8 @@ def config(index: int) -> Workload:
         return target_attention(32, 4096, 256, 128, seed=5, name="a1_target_attention")
     if index == 7:   # beyond the five: the Self-Attention 512 x 512 shape of Sec. 6.2 (two sub-tiles of 256 source positions)
         return target_attention(256, 512, 512, 128, seed=7, name="a2_self_attention_512")
+    if index == 8:   # beyond the five: the DLRM bottom-MLP shape of Sec. 6.2 (K streamed through the first GEMM)
+        return dlrm_bottom_mlp(32768, 1024, 512, 128, seed=8, name="d1_dlrm_bottom_mlp")
     if index == 6:   # beyond the five: an epilogue given as data that no compiled kind covers
         return program_range_normalise(8192, 1024, 1024, seed=6, name="p1_program_range_normalise")
     raise IndexError(index)
