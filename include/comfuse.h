@@ -151,7 +151,14 @@ typedef enum {
    * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128 and N1 = 256 (a whole score row fits the
    * accumulators of one CTA pair) or N1 = 512 (two sub-tiles of 256 source positions, each exponentiated against its own
    * row maximum, combined when O is normalised); the probabilities are rounded to bf16 as the second GEMM's operand. */
-  COMFUSE_B2B_SOFTMAX_ATTENTION = 1
+  COMFUSE_B2B_SOFTMAX_ATTENTION = 1,
+  /* Two-layer ReLU MLP (Sec. 4, Eq. 2 with F = ReLU(. + b1); the DLRM workload of Sec. 6.2, 1024 -> 512 -> 128):
+   *   O = ReLU(ReLU(X.W1 + b1).W2 + b2),
+   * X [M, K], W1 [K, N1], W2 [N1, N2]; K and N2 independent, batch = 1, gamma and beta must be NULL, b1 / b2 may be NULL.
+   * Fused: N2 = 128, N1 = 256 or 512, any K (a multiple of 8) streamed through the first GEMM; the hidden layer is rounded
+   * to bf16 as the second GEMM's operand and never leaves the chip.  Unfused: any shape, the bf16 hidden layer [M, N1] in
+   * the workspace. */
+  COMFUSE_B2B_MLP_RELU = 2
 } comfuse_b2b_kind_t;
 
 typedef struct {

@@ -33,7 +33,7 @@ EPI_BIAS_ACTIVATION = 3   # reduction-free epilogue; reached through gemm_spec o
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
 FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2
-B2B_MLP_GELU_LAYERNORM, B2B_SOFTMAX_ATTENTION = 0, 1
+B2B_MLP_GELU_LAYERNORM, B2B_SOFTMAX_ATTENTION, B2B_MLP_RELU = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
@@ -308,6 +308,39 @@ def b2b_gemm(X, W1, b1, W2, b2, O, *, gamma=None, beta=None, eps=1e-5, fused=Tru
                                 ws_ptr, ws_bytes, _stream(stream))
     if st != OK:
         raise ComfuseError(st, "comfuse_b2b_gemm")
+    return O
+
+
+def b2b_mlp_relu(X, W1, b1, W2, b2, O, *, fused=True, workspace=None, stream=None):
+    """Enqueue O = ReLU(ReLU(X.W1 + b1).W2 + b2) (the two-layer ReLU MLP form of the back-to-back GEMM).  Dense row-major
+    CUDA bf16 tensors X [M, K], W1 [K, N1], W2 [N1, N2], O [M, N2]; b1, b2 may be None."""
+    M, K = X.shape
+    N1, N2 = W1.shape[1], W2.shape[1]
+    assert W1.shape == (K, N1) and W2.shape == (N1, N2) and O.shape == (M, N2)
+    for t in (X, W1, W2, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_MLP_RELU)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm(byref(d), _ptr(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), None, None, _ptr(O),
+                                ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm")
+    return O
+
+
+def b2b_mlp_relu_host(X, W1, b1, W2, b2, O, *, staging, fused=True, workspace=None, stream=None):
+    """b2b_mlp_relu with X and O in host memory (dense CPU tensors, pinned for asynchronous copies)."""
+    M, K = X.shape
+    N1, N2 = W1.shape[1], W2.shape[1]
+    for t in (X, W1, W2, O):
+        assert t.is_contiguous()
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_MLP_RELU)
+    ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
+    st = lib().comfuse_b2b_gemm_host(byref(d), _ptr(X), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), None, None, _ptr(O),
+                                     c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),
+                                     ws_ptr, ws_bytes, _stream(stream))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_b2b_gemm_host")
     return O
 
 

@@ -10,7 +10,8 @@ struct B2bParams {
   int M, K, N1, N2;
   int mblocks, mpairs;  // 128-row blocks and pairs of them (per batch)
   int batch;            // attention form: X, W1, W2, O are [batch, ., .]; MLP form: 1
-  int mode;             // 0: F = GELU(. + b1), tail = + b2 + X, LayerNorm; 1: F = softmax(alpha * .), tail = none
+  int mode;             // 0: F = GELU(. + b1), tail = + b2 + X, LayerNorm; 1: F = softmax(alpha * .), tail = none;
+                        // 2: F = ReLU(. + b1), tail = ReLU(. + b2) (the streamed-K kernel)
   float alpha;          // attention form: scale of the scores
   float eps;
   const uint16_t* X;  // also the residual of the tail
@@ -27,5 +28,8 @@ struct B2bParams {
 
 bool b2b_fused_supported(int K, int N1, int N2, int mode);
 cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
+// the ReLU MLP form with K streamed through the first GEMM (b2b_stream.cu)
+bool b2b_stream_supported(int K, int N1, int N2);
+cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
 
 }  // namespace comfuse

@@ -444,15 +444,22 @@ static comfuse_status_t validate_b2b_desc(const comfuse_b2b_desc_t* d) {
   if (!d) return COMFUSE_ERR_INVALID_ARG;
   if (d->M < 1 || d->K < 1 || d->N1 < 1 || d->N2 < 1) return COMFUSE_ERR_INVALID_ARG;
   if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
-  if (d->kind != COMFUSE_B2B_MLP_GELU_LAYERNORM && d->kind != COMFUSE_B2B_SOFTMAX_ATTENTION) return COMFUSE_ERR_INVALID_ARG;
+  if (d->kind != COMFUSE_B2B_MLP_GELU_LAYERNORM && d->kind != COMFUSE_B2B_SOFTMAX_ATTENTION && d->kind != COMFUSE_B2B_MLP_RELU)
+    return COMFUSE_ERR_INVALID_ARG;
   if (d->batch < 1 || d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
   if (d->kind == COMFUSE_B2B_MLP_GELU_LAYERNORM) {
     if (d->batch != 1) return COMFUSE_ERR_INVALID_ARG;
     if (d->N2 != d->K) return COMFUSE_ERR_INVALID_ARG;  // the residual is X itself
+  } else if (d->kind == COMFUSE_B2B_MLP_RELU) {
+    if (d->batch != 1) return COMFUSE_ERR_INVALID_ARG;
   } else if (!(d->alpha > 0.f)) {
     return COMFUSE_ERR_INVALID_ARG;
   }
   if (!mult8(d->K) || !mult8(d->N1) || !mult8(d->N2)) return COMFUSE_ERR_ALIGNMENT;
+  if (d->kind == COMFUSE_B2B_MLP_RELU) {
+    if (d->fused && !b2b_stream_supported(d->K, d->N1, d->N2)) return COMFUSE_ERR_UNSUPPORTED;
+    return COMFUSE_OK;  // unfused: two calls of the reduction-free GEMM kind, any N1 / N2
+  }
   if (d->fused && !b2b_fused_supported(d->K, d->N1, d->N2, d->kind)) return COMFUSE_ERR_UNSUPPORTED;
   if (!d->fused && (d->kind == COMFUSE_B2B_MLP_GELU_LAYERNORM ? d->N2 : d->N1) > 8192) return COMFUSE_ERR_UNSUPPORTED;
   return COMFUSE_OK;
@@ -464,6 +471,8 @@ comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size
   if (s != COMFUSE_OK) return s;
   if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1]
     *bytes = desc->fused ? 0 : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2;
+  else if (desc->kind == COMFUSE_B2B_MLP_RELU)  // unfused: the bf16 hidden layer [M, N1]
+    *bytes = desc->fused ? 0 : static_cast<size_t>(desc->M) * desc->N1 * 2;
   else
     *bytes = desc->fused ? 0 : (static_cast<size_t>(desc->M) * desc->N1 + static_cast<size_t>(desc->M) * desc->N2) * 2;
   return COMFUSE_OK;
@@ -477,6 +486,8 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
   if (!X || !W1 || !W2 || !O) return COMFUSE_ERR_INVALID_ARG;
   const bool attention = desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION;
   if (attention && (b1 || b2 || gamma || beta)) return COMFUSE_ERR_INVALID_ARG;
+  const bool relu_mlp = desc->kind == COMFUSE_B2B_MLP_RELU;
+  if (relu_mlp && (gamma || beta)) return COMFUSE_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W1) || !aligned16(W2) || !aligned16(O) || !aligned16(b1) || !aligned16(b2) ||
       !aligned16(gamma) || !aligned16(beta))
     return COMFUSE_ERR_ALIGNMENT;
@@ -494,7 +505,7 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
   if (desc->fused) {
     B2bParams bp = {};
     bp.M = M; bp.K = K; bp.N1 = N1; bp.N2 = N2;
-    bp.batch = desc->batch; bp.mode = attention ? 1 : 0; bp.alpha = desc->alpha;
+    bp.batch = desc->batch; bp.mode = attention ? 1 : (relu_mlp ? 2 : 0); bp.alpha = desc->alpha;
     bp.eps = desc->eps;
     bp.X = static_cast<const uint16_t*>(X);
     bp.b1 = static_cast<const uint16_t*>(b1);
@@ -508,8 +519,15 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) bp.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));
     if (const char* tf = std::getenv("COMFUSE_TRACE_FLAGS")) bp.trace_flags = std::atoi(tf);
 #endif
-    cudaError_t e = launch_b2b_fused(X, W1, W2, bp, st);
+    cudaError_t e = relu_mlp ? launch_b2b_stream(X, W1, W2, bp, st) : launch_b2b_fused(X, W1, W2, bp, st);
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+  }
+
+  if (relu_mlp) {
+    // unfused: S = ReLU(X.W1 + b1) as bf16 in the workspace, then O = ReLU(S.W2 + b2): the reduction-free GEMM kind twice
+    s = run_gemm_elementwise(1, M, N1, K, K, N1, N1, 0, 0, 0, X, W1, workspace, b1, 1.f, COMFUSE_OP_RELU, st);
+    if (s != COMFUSE_OK) return s;
+    return run_gemm_elementwise(1, M, N2, N1, N1, N2, N2, 0, 0, 0, workspace, W2, O, b2, 1.f, COMFUSE_OP_RELU, st);
   }
 
   if (attention) {

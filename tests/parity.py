@@ -55,6 +55,12 @@ def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
         ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
         cf.b2b_attention(T["X"], T["W1"], T["W2"], O, alpha=w.scalars["alpha"], fused=fused, workspace=ws)
         return {"Y": O}
+    if w.kind == wl.KIND_B2B_MLP_RELU:
+        O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
+        desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, fused, cf.B2B_MLP_RELU)
+        ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
+        cf.b2b_mlp_relu(T["X"], T["W1"], T.get("b1"), T["W2"], T.get("b2"), O, fused=fused, workspace=ws)
+        return {"Y": O}
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
         O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused)
@@ -102,6 +108,8 @@ def run_oracle(w: wl.Workload, rows=None, batches=None):
             Q = Q[:, rows, :]
         return {"Y": orc.b2b_softmax_attention(wl.bf16_to_f64(Q), wl.bf16_to_f64(w.tensors["W1"][bsel]),
                                                wl.bf16_to_f64(w.tensors["W2"][bsel]), w.scalars["alpha"])}
+    if w.kind == wl.KIND_B2B_MLP_RELU:
+        return {"Y": orc.b2b_mlp_relu(f64(w, "X", rows), f64(w, "W1"), f64(w, "b1"), f64(w, "W2"), f64(w, "b2"))}
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
         Y = orc.b2b_mlp_layernorm(f64(w, "X", rows), f64(w, "W1"), f64(w, "b1"), f64(w, "W2"), f64(w, "b2"),
                                   f64(w, "gamma"), f64(w, "beta"), w.scalars["eps"])

@@ -1,0 +1,93 @@
+"""GPU parity of the two-layer ReLU MLP form of the back-to-back GEMM (the DLRM workload's shape class): the fused kernel
+that streams K through the first GEMM and keeps the hidden layer on-chip, and the in-library unfused path (bf16 hidden layer
+in the workspace), against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_03537_b200 as cf
+import workloads as wl
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # M, K, N1
+    (256, 64, 256),      # one K block, one half: ML1 -> Epi1 -> ML2 -> Epi2 with nothing to overlap
+    (256, 128, 512),     # two K blocks, two halves: the two slots change roles once
+    (300, 1024, 512),    # the DLRM feature dimensions; ragged rows (a partial block and an empty one)
+    (1000, 1000, 256),   # K not a multiple of 64: the last K block is zero-filled
+    (77, 8, 256),        # the smallest K
+    (2048, 192, 512),    # odd number of K blocks
+    (40000, 128, 512),   # 157 tiles: up to three tiles per cluster, every slot reused in both roles
+    (41000, 64, 256),    # single-half tiles alternate between the two slots
+]
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("M,K,N1", CASES)
+def test_b2b_mlp_relu(M, K, N1, fused, cuda_device):
+    w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=M + K + N1)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    res = P.check_outputs(w, got, P.run_oracle(w), label=f"relu mlp M{M} K{K} N1{N1} fused={fused}")
+    assert (got["Y"].float() >= 0).all().item()
+    assert cf.last_device_status() == cf.OK
+    print(M, K, N1, fused, res)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_dlrm_shape_full_size_sampled(fused, cuda_device):
+    """32768 x (1024 -> 512 -> 128): sampled rows against the oracle, every element finite and non-negative."""
+    w = wl.config(8)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
+    Y = got["Y"].float()
+    assert torch.isfinite(Y).all().item() and (Y >= 0).all().item()
+    rows = wl.sample_rows(w.dims["M"], 512)
+    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"d1 fused={fused}")
+    print("d1", fused, res)
+
+
+def test_relu_mlp_without_biases_and_identity_second_layer(cuda_device):
+    """b1 = b2 = NULL; W2 = the first 128 columns of I: O = ReLU(X W1)[:, :128] (ReLU of a non-negative value is itself)."""
+    M, K, N1 = 512, 256, 256
+    w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=11)
+    T = P.dev_tensors(w)
+    W2 = torch.zeros(N1, 128, dtype=torch.bfloat16, device=T["X"].device)
+    W2[:128, :] = torch.eye(128, dtype=torch.bfloat16, device=W2.device)
+    O = torch.full((M, 128), float("nan"), dtype=torch.bfloat16, device=W2.device)
+    cf.b2b_mlp_relu(T["X"], T["W1"], None, W2, None, O, fused=True)
+    ref = np.maximum(wl.bf16_to_f64(w.tensors["X"]) @ wl.bf16_to_f64(w.tensors["W1"]), 0.0)[:, :128]
+    err = np.abs(P.to_f64(O) - ref)
+    assert err.max() <= 3e-2 and err.mean() <= 3e-3
+    # exact zeros where the hidden unit is clearly off
+    assert (P.to_f64(O)[ref == 0.0] == 0.0).all()
+
+
+def test_relu_mlp_bitwise_repeatable_and_equal_rows(cuda_device):
+    """Run twice: same bits.  Rows are independent: the result of a row does not depend on which tile it sits in."""
+    w = wl.dlrm_bottom_mlp(20000, 320, 512, 128, seed=5)
+    T = P.dev_tensors(w)
+    a = P.run_gpu(w, T, fused=True)["Y"]
+    b = P.run_gpu(w, T, fused=True)["Y"]
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    X2 = T["X"][19000:19300].contiguous()       # the same rows as their own problem
+    O2 = torch.empty(300, 128, dtype=torch.bfloat16, device=X2.device)
+    cf.b2b_mlp_relu(X2, T["W1"], T["b1"], T["W2"], T["b2"], O2, fused=True)
+    assert torch.equal(O2.view(torch.int16), a[19000:19300].view(torch.int16))
+
+
+def test_relu_mlp_argument_checks(cuda_device):
+    dev = "cuda:0"
+    X = torch.zeros(256, 64, dtype=torch.bfloat16, device=dev)
+    W1 = torch.zeros(64, 384, dtype=torch.bfloat16, device=dev)
+    W2 = torch.zeros(384, 128, dtype=torch.bfloat16, device=dev)
+    O = torch.zeros(256, 128, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(cf.ComfuseError) as e:     # N1 = 384 has no fused instantiation
+        cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=True)
+    assert e.value.status == cf.ERR_UNSUPPORTED
+    ws = torch.empty(256 * 384 * 2, dtype=torch.uint8, device=dev)
+    cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=False, workspace=ws)   # ... but runs unfused
+    assert cf.last_device_status() == cf.OK
+    with pytest.raises(cf.ComfuseError) as e:     # unfused without its workspace
+        cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=False)
+    assert e.value.status == cf.ERR_WORKSPACE
