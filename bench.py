@@ -33,10 +33,10 @@ import workloads as wl  # noqa: E402
 METRIC = "fused-kernel TFLOP/s (GEMM flops / time of the fused kernel)"
 # a1 (target attention), a2 (self-attention 512 x 512) and p1 (an epilogue given as data, on-chip interpreter) lie beyond
 # the five named configurations
-WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "a1": 5, "p1": 6, "a2": 7}
+WORKLOADS = {"c1": 0, "c2": 1, "c3": 2, "c4": 3, "c5": 4, "a1": 5, "p1": 6, "a2": 7, "d1": 8}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the ncu
 # captures summarised under profiles/, in bytes; None = not captured.
-NCU_TRAFFIC_BYTES = {"a2": None, "p1": 18_988_288, "a1": 39_041_536, "c1": None, "c2": 70_159_872, "c3": 217_753_600, "c4": 512_653_312, "c5": 8_713_216}
+NCU_TRAFFIC_BYTES = {"d1": None, "a2": None, "p1": 18_988_288, "a1": 39_041_536, "c1": None, "c2": 70_159_872, "c3": 217_753_600, "c4": 512_653_312, "c5": 8_713_216}
 
 
 def load_peaks():
@@ -114,6 +114,8 @@ def oracle_call(w, rows):
         return spo.gemm_spec(t["A"][rows], t["B"], pr.nodes, pr.terminal, params, pr.row_outputs)
     if w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION:
         return orc.b2b_softmax_attention(t["X"][0][rows], t["W1"][0], t["W2"][0], w.scalars["alpha"])
+    if w.kind == wl.KIND_B2B_MLP_RELU:
+        return orc.b2b_mlp_relu(t["X"][rows], t["W1"], t["b1"], t["W2"], t["b2"])
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
         return orc.b2b_mlp_layernorm(t["X"][rows], t["W1"], t["b1"], t["W2"], t["b2"], t.get("gamma"), t.get("beta"), w.scalars["eps"])
     if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
@@ -136,7 +138,7 @@ def widen_for_oracle(w, softmax_batches=1):
 
 def sample_flops(w, nrows):
     d = w.dims
-    if w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION):
+    if w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION, wl.KIND_B2B_MLP_RELU):
         return 2.0 * nrows * (d["K"] * d["N1"] + d["N1"] * d["N2"])
     return 2.0 * nrows * d["N"] * d["K"]
 
@@ -235,7 +237,8 @@ def run_comfuse(args):
     # ---- buffer sets: per-step activations (inputs read once per step and the outputs) are replicated until the
     # rotation exceeds 3x the L2 capacity; weights and row vectors are shared (they are meant to be L2 resident)
     attention = w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION
-    b2b = w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION)
+    relu_mlp = w.kind == wl.KIND_B2B_MLP_RELU
+    b2b = w.kind in (wl.KIND_B2B_MLP_LAYERNORM, wl.KIND_B2B_SOFTMAX_ATTENTION, wl.KIND_B2B_MLP_RELU)
     program = w.kind == wl.KIND_GEMM_PROGRAM
     if program:
         spec = cf.make_spec(w.program.nodes, w.program.terminal, len(w.program.param_kinds), w.program.row_outputs)
@@ -264,6 +267,8 @@ def run_comfuse(args):
     def b2b_desc(use_fused):
         if attention:
             return cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, use_fused, cf.B2B_SOFTMAX_ATTENTION, d["batch"], w.scalars["alpha"])
+        if relu_mlp:
+            return cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, use_fused, cf.B2B_MLP_RELU)
         return cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], use_fused)
 
     if b2b:
@@ -285,6 +290,8 @@ def run_comfuse(args):
                          row_out=s["row_out"], fused=use_fused, workspace=workspace)
         elif attention:
             cf.b2b_attention(s["X"], s["W1"], s["W2"], s["Y"], alpha=w.scalars["alpha"], fused=use_fused, workspace=workspace)
+        elif relu_mlp:
+            cf.b2b_mlp_relu(s["X"], s["W1"], s["b1"], s["W2"], s["b2"], s["Y"], fused=use_fused, workspace=workspace)
         elif w.kind == wl.KIND_B2B_MLP_LAYERNORM:
             cf.b2b_gemm(s["X"], s["W1"], s["b1"], s["W2"], s["b2"], s["Y"], gamma=s.get("gamma"), beta=s.get("beta"),
                         eps=w.scalars["eps"], fused=use_fused, workspace=workspace)
@@ -400,7 +407,7 @@ def run_comfuse(args):
         roof["kernel"] = {cf.SPEC_PATH_FUSED_KERNEL: "fused_pair_kernel (compiled kind)", cf.SPEC_PATH_FUSED_PROGRAM: "fused_pair_kernel<EPI_PROGRAM> (on-chip interpreter)",
                           cf.SPEC_PATH_ROW_PROGRAM: "fused_pair_kernel<EPI_NONE> + row_program_kernel"}[plan.path if fused else cf.SPEC_PATH_ROW_PROGRAM]
     elif b2b:
-        roof["kernel"] = "b2b_pair_kernel"
+        roof["kernel"] = "b2b_stream_kernel" if relu_mlp else "b2b_pair_kernel"
     elif w.kind == wl.KIND_SCALE_MASK_SOFTMAX and d["K"] <= 256:
         roof["kernel"] = "softmax_rows_kernel"      # short K: score chunks computed twice, no cluster exchange
     else:
@@ -468,6 +475,8 @@ def run_comfuse(args):
                 if "K_rows" not in sx:
                     sx["K_rows"] = sx["W1"].transpose(1, 2).contiguous()
                 return F.scaled_dot_product_attention(sx["X"].unsqueeze(0), sx["K_rows"].unsqueeze(0), sx["W2"].unsqueeze(0), scale=w.scalars["alpha"])
+            if relu_mlp:
+                return torch.relu(torch.addmm(sx["b2"], torch.relu(torch.addmm(sx["b1"], sx["X"], sx["W1"])), sx["W2"]))
             if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
                 hid = F.gelu(torch.addmm(sx["b1"], sx["X"], sx["W1"]), approximate="tanh")
                 return F.layer_norm(torch.addmm(sx["b2"], hid, sx["W2"]) + sx["X"], (d["N2"],), sx.get("gamma"), sx.get("beta"), w.scalars["eps"])
@@ -529,6 +538,9 @@ def run_comfuse(args):
             if attention:
                 cf.b2b_attention_host(host_in["X"], host_in["W1"], host_in["W2"], host_out, staging=staging,
                                       alpha=w.scalars["alpha"], fused=fused, workspace=ws)
+            elif relu_mlp:
+                cf.b2b_mlp_relu_host(host_in["X"], s0["W1"], s0["b1"], s0["W2"], s0["b2"], host_out, staging=staging, fused=fused,
+                                     workspace=ws)
             else:
                 cf.b2b_gemm_host(host_in["X"], s0["W1"], s0["b1"], s0["W2"], s0["b2"], host_out, staging=staging,
                                  gamma=s0.get("gamma"), beta=s0.get("beta"), eps=w.scalars["eps"], fused=fused, workspace=ws)

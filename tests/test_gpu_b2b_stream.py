@@ -91,3 +91,41 @@ def test_relu_mlp_argument_checks(cuda_device):
     with pytest.raises(cf.ComfuseError) as e:     # unfused without its workspace
         cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=False)
     assert e.value.status == cf.ERR_WORKSPACE
+
+
+def test_relu_mlp_random_shapes(cuda_device):
+    """Seeded random shapes (M 1 .. 3000 and a few beyond one wave of clusters, K any multiple of 8 up to 1536, N1 256 or
+    512), fused kernel against the oracle; the unfused path on every fourth shape."""
+    rng = np.random.default_rng(20240)
+    worst = 0.0
+    for i in range(60):
+        M = int(rng.integers(1, 3001)) if i % 10 else int(rng.integers(19000, 60000))
+        K = 8 * int(rng.integers(1, 193))
+        N1 = 256 * int(rng.integers(1, 3))
+        w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=1000 + i)
+        T = P.dev_tensors(w)
+        ref = P.run_oracle(w)
+        res = P.check_outputs(w, P.run_gpu(w, T, fused=True), ref, label=f"random relu mlp #{i} M{M} K{K} N1{N1}")
+        worst = max(worst, res["max_abs"])
+        if i % 4 == 0:
+            P.check_outputs(w, P.run_gpu(w, T, fused=False), ref, label=f"random relu mlp unfused #{i} M{M} K{K} N1{N1}")
+    assert cf.last_device_status() == cf.OK
+    print("worst max-abs", worst)
+
+
+@pytest.mark.parametrize("M", [600, 9000])
+def test_relu_mlp_host_buffers_match_device_buffers(M, cuda_device):
+    """X and O in pinned host memory (M = 9000 x K = 1024 is 18 MB of activations: the call runs as a pipeline of row ranges):
+    bit for bit the device-pointer call."""
+    w = wl.dlrm_bottom_mlp(M, 1024, 512, 128, seed=31)
+    T = P.dev_tensors(w)
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hX = T["X"].cpu().pin_memory()
+    hO = torch.empty(M, 128, dtype=torch.bfloat16).pin_memory()
+    desc = cf.make_b2b_desc(M, 1024, 512, 128, 0.0, True, cf.B2B_MLP_RELU)
+    staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=T["X"].device)
+    for _ in range(2):
+        cf.b2b_mlp_relu_host(hX, T["W1"], T["b1"], T["W2"], T["b2"], hO, staging=staging)
+    torch.cuda.synchronize()
+    assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+    assert cf.last_device_status() == cf.OK
