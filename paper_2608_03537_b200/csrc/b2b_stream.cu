@@ -263,6 +263,13 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       for (int part = 0; part < 2; ++part) {
         uint32_t v[32];
         tmem_ld_32cols(tmem_base + lane_sel + static_cast<uint32_t>(slot * 256 + hh * 64 + part * 32), v);
+        if (part == 1) {
+          // the slot has been read (the loads wait for their data).  Half 1 does not host O: its slot is free for the next
+          // tile's first half from here on -- the UMMA lane is waiting for exactly this
+          tcgen05_fence_before_sync();
+          __syncwarp();
+          if (h == 1 && lane == 0) mbar_arrive_cluster_noflush(pfree_leader + 8u * slot);
+        }
         const uint4* b4 = reinterpret_cast<const uint4*>(s_b1 + h * 256 + hh * 64 + part * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -275,10 +282,6 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           }
         }
       }
-      tcgen05_fence_before_sync();  // the slot's reads are complete before anybody is told so
-      __syncwarp();
-      // half 1 does not host O: its slot is free for the next tile's first half as soon as it has been read
-      if (h == 1 && lane == 0) mbar_arrive_cluster_noflush(pfree_leader + 8u * slot);
       // the S buffer: the output boxes that Epi2 staged there have been read by their stores ...
       if (h == 0 && it > 0) {
         if (store_thread) tma_store_wait_read<0>();
