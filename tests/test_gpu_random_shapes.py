@@ -101,5 +101,8 @@ def test_random_wide_rows(seed, cuda_device):
     ref = P.run_oracle(w)
     kw = {"norm_tol": max(4e-2, 2.0 ** -7 * float(np.abs(ref["Y"]).max()))}   # the un-normalised row passes through bf16 once
     if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
-        kw["rowmax_tol"] = 3e-2
+        # two columns whose un-normalised values were each moved by half a bf16 ulp (2^-9 relative) can swap places when they
+        # are closer than 2^-8 |y| g: with |y| up to 8 in rows of 12288+ columns that exceeds 3e-2 in about one row of 50 000
+        # (a CPU emulation of the rounding reproduces the same rows), so the slack follows the magnitude like `norm_tol`
+        kw["rowmax_tol"] = kw["norm_tol"]
     P.check_outputs(w, got, ref, label=f"{w.name} wide {sorted(w.tensors)} {w.scalars}", **kw)
