@@ -129,3 +129,33 @@ def test_relu_mlp_host_buffers_match_device_buffers(M, cuda_device):
     torch.cuda.synchronize()
     assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
     assert cf.last_device_status() == cf.OK
+
+
+def test_relu_mlp_back_to_back_dependent_launches(cuda_device):
+    """The kernel is launched with programmatic stream serialization (its set-up may overlap the previous kernel's tail; it
+    waits for that kernel before it touches global memory).  A chain in which every call consumes the previous call's
+    output, enqueued without synchronisation, gives bit for bit what the chain gives with a synchronisation per call."""
+    M, K, N1 = 3000, 128, 512
+    w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=41)
+    T = P.dev_tensors(w)
+    dev = T["X"].device
+    W2 = (T["W2"].float() * 4.0).to(torch.bfloat16)          # keeps the activations from dying out along the chain
+
+    def chain(sync):
+        x = T["X"].clone()                                    # [M, 128]; N2 == K so the output can feed the next call
+        bufs = [torch.empty(M, 128, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        for i in range(10):
+            y = bufs[i & 1]
+            cf.b2b_mlp_relu(x, T["W1"], T["b1"], W2, T["b2"], y, fused=True)
+            if sync:
+                torch.cuda.synchronize()
+            x = y
+        torch.cuda.synchronize()
+        return x.clone()
+
+    a = chain(sync=True)
+    assert a.float().abs().max().item() > 0
+    for _ in range(3):
+        b = chain(sync=False)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert cf.last_device_status() == cf.OK
