@@ -1,6 +1,8 @@
 """GPU parity of the two-layer ReLU MLP form of the back-to-back GEMM (the DLRM workload's shape class): the fused kernel
 that streams K through the first GEMM and keeps the hidden layer on-chip, and the in-library unfused path (bf16 hidden layer
 in the workspace), against the fp64 oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -95,10 +97,10 @@ def test_relu_mlp_argument_checks(cuda_device):
 
 def test_relu_mlp_random_shapes(cuda_device):
     """Seeded random shapes (M 1 .. 3000 and a few beyond one wave of clusters, K any multiple of 8 up to 1536, N1 256 or
-    512), fused kernel against the oracle; the unfused path on every fourth shape."""
+    512), fused kernel against the oracle; the unfused path on every fourth shape.  COMFUSE_FUZZ_SEEDS lengthens the sweep."""
     rng = np.random.default_rng(20240)
     worst = 0.0
-    for i in range(60):
+    for i in range(int(os.environ.get("COMFUSE_FUZZ_SEEDS", 60))):
         M = int(rng.integers(1, 3001)) if i % 10 else int(rng.integers(19000, 60000))
         K = 8 * int(rng.integers(1, 193))
         N1 = 256 * int(rng.integers(1, 3))
