@@ -4,19 +4,28 @@
 // global memory.
 //
 // Where it differs from the K = 128 kernel (b2b_gemm.cu): there a P chunk costs eight UMMAs, here it costs K / 16 of them,
-// so N1 is cut into HALVES of 256 columns (one UMMA N, X streamed once per half: the operand traffic per flop of a plain
-// 256 x 256 tile) and tensor memory is two slots of 256 columns that change roles:
-//   half 0 of tile t -> slot s0 = t & 1, half 1 -> the other slot; once Epi1 has read half 0 out of s0, O(t) accumulates in
-//   the first 128 columns of s0.  Tile t+1 starts in the slot that held half 1 of tile t.
-// One CTA pair (cta_group::2) owns 256 rows.  Per unit u = (tile, half) the UMMA lane issues
+// so N1 is cut into HALVES of 256 columns (one UMMA N) and tensor memory into two slots of 256 columns.  One CTA pair
+// (cta_group::2) owns 256 rows.  The output is staged in the S buffer, idle between the tile's last ML2 and the next Epi1.
+//
+// N1 = 512, both halves in LOCK-STEP (default): a ring stage (48 KB, three stages) holds one K block of X and this CTA's
+// 128 columns of W1 for BOTH halves; the X block in shared memory feeds the UMMAs of half 0 (slot 0) and half 1 (slot 1), so X
+// is streamed once and the MainLoop needs 109 B/clk of shared-memory traffic instead of 128.  Then Epi1(0) -> ML2(0),
+// Epi1(1) -> ML2(1) with O in the first 128 columns of slot 0 (read out by Epi1(0) before S of half 0 exists), Epi2; the next
+// tile's MainLoop waits for both slots, i.e. the epilogue of a tile is exposed, which the faster MainLoop more than pays for.
+//
+// N1 = 256 (and N1 = 512 with COMFUSE_B2B_STREAM_LOCK=0), ALTERNATING slots: the slots change roles -- half 0 of tile t ->
+// slot s0 = t & 1, half 1 -> the other slot; once Epi1 has read half 0 out of s0, O(t) accumulates in the first 128 columns of
+// s0; tile t+1 starts in the slot that held half 1 of tile t.  Per unit u = (tile, half) the UMMA lane issues
 //   ML1(u) first K blocks | ML2(u - 1) | ML1(u) remaining K blocks
 // so that Epi1(u - 1) (bias, ReLU, bf16, swizzled A operand in shared memory) has half a MainLoop to finish before the
 // tensor pipe asks for S, and S needs one shared-memory buffer only (Sec. 4.3's staggered pipeline with the second
 // MainLoop folded into the first one's stream).  The epilogue warps run Epi2(t - 1), Epi1(t, 0), Epi1(t, 1), ...
-// Ring (Sec. 4.2, unified circular buffer): stages of 32 KB in consumption order; an ML1 stage holds one K block of X
+// Ring (Sec. 4.2, unified circular buffer): five stages of 32 KB in consumption order; an ML1 stage holds one K block of X
 // (128 rows x 64) and of this CTA's 128 columns of W1 (two 64 x 64 boxes), an ML2 stage this CTA's 64 columns of the
-// 256 W2 rows of a half.  The output is staged in the S buffer, idle between the tile's last ML2 and the next Epi1.
+// 256 W2 rows of a half (in both schedules).
 #include <cuda_runtime.h>
+
+#include <cstdlib>
 
 #include "b2b_params.h"
 #include "fused_pair.cuh"
@@ -31,22 +40,25 @@ constexpr int kEpiWarps = 16;  // four per TMEM lane quarter
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreads = 32 * (2 + kEpiWarps);  // producer, UMMA, epilogue warps
 constexpr int kBoxBytes = 128 * 64 * 2;         // one 128 x 64 bf16 box
-constexpr int kStageBytes = 2 * kBoxBytes;
-constexpr int kStages = 5;
-
+// LOCK (N1 = 512): both halves of P are computed in lock-step from ONE copy of the X block (a stage = X block + the W1
+// blocks of both halves, 48 KB; three stages); otherwise a stage is 32 KB and there are five.
+template <bool LOCK>
 struct StreamSmem {
+  static constexpr int kStages = LOCK ? 3 : 5;
+  static constexpr int kStageBytes = LOCK ? 3 * kBoxBytes : 2 * kBoxBytes;
   static constexpr int OFF_RING = 0;
   static constexpr int OFF_S = kStages * kStageBytes;  // four K blocks of S; the output staging boxes live in the first two
   static constexpr int OFF_B1 = OFF_S + 4 * kBoxBytes;  // bf16 [512]
   static constexpr int OFF_B2 = OFF_B1 + 512 * 2;       // bf16 [128]
   static constexpr int OFF_BAR = OFF_B2 + 128 * 2;
-  // barriers: full[5] empty[5] pfull[2] pfree[2] sfull sempty ofull drain
+  // barriers: full[kStages] empty[kStages] pfull[2] pfree[2] sfull sempty ofull drain
   static constexpr int NUM_BARS = 2 * kStages + 8;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
-static_assert(StreamSmem::BYTES <= 232448, "shared memory budget");
+static_assert(StreamSmem<false>::BYTES <= 232448 && StreamSmem<true>::BYTES <= 232448, "shared memory budget");
 
+template <bool LOCK>
 __global__ void __launch_bounds__(kThreads, 1)
 b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                   const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
@@ -54,10 +66,13 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
   const uint32_t smem_base = smem_u32(smem);
+  using Smem = StreamSmem<LOCK>;
+  constexpr int kStages = Smem::kStages;
+  constexpr int kStageBytes = Smem::kStageBytes;
 
-  uint16_t* s_b1 = reinterpret_cast<uint16_t*>(smem + StreamSmem::OFF_B1);
-  uint16_t* s_b2 = reinterpret_cast<uint16_t*>(smem + StreamSmem::OFF_B2);
-  const uint32_t bar_base = smem_base + StreamSmem::OFF_BAR;
+  uint16_t* s_b1 = reinterpret_cast<uint16_t*>(smem + Smem::OFF_B1);
+  uint16_t* s_b2 = reinterpret_cast<uint16_t*>(smem + Smem::OFF_B2);
+  const uint32_t bar_base = smem_base + Smem::OFF_BAR;
   auto bar_full = [&](int s) { return bar_base + 8u * s; };               // stage landed in both CTAs (even CTA)
   auto bar_empty = [&](int s) { return bar_base + 8u * (kStages + s); };  // stage read by the tensor pipe
   auto bar_pfull = [&](int a) { return bar_base + 8u * (2 * kStages + a); };      // P half complete in slot a
@@ -66,8 +81,8 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const uint32_t bar_sempty = bar_sfull + 8u;                     // S read by ML2
   const uint32_t bar_ofull = bar_sfull + 16u;                     // O of a tile complete
   const uint32_t bar_drain = bar_sfull + 24u;
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + StreamSmem::OFF_MISC);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + StreamSmem::OFF_MISC + 4);
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + Smem::OFF_MISC);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Smem::OFF_MISC + 4);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -115,8 +130,8 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   cluster_sync_after_init();  // every CTA's barriers exist before any peer signals them
   const uint32_t tmem_base = *s_tmem_base;
   griddep_wait();  // global memory is touched only below
-  auto ring_addr = [&](int s) { return smem_base + StreamSmem::OFF_RING + s * kStageBytes; };
-  const uint32_t s_base = smem_base + StreamSmem::OFF_S;
+  auto ring_addr = [&](int s) { return smem_base + Smem::OFF_RING + s * kStageBytes; };
+  const uint32_t s_base = smem_base + Smem::OFF_S;
   // unit u of this cluster = half (u % NH) of its (u / NH)-th tile; P of that half goes to slot ((u / NH) & 1) ^ half,
   // O of the tile to the first 128 columns of slot (u / NH) & 1
   auto tile_m0 = [&](int it) { return (cluster_id + it * num_clusters) * 256 + static_cast<int>(pm) * 128; };
@@ -126,37 +141,50 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     if (lane == 0) {
       RingPos<kStages> ring;
       bool ok = true;
-      auto next_stage = [&](uint32_t& sa, uint32_t& full) {
+      auto next_stage = [&](uint32_t& sa, uint32_t& full, uint32_t bytes) {
         if (!ok) return false;
         if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; return false; }
         sa = ring_addr(ring.stage);
         full = map_to_cta(bar_full(ring.stage), leader);
-        mbar_arrive_expect_tx_cluster(full, kStageBytes);
+        mbar_arrive_expect_tx_cluster(full, bytes);
         ring.advance();
         return true;
       };
       auto push_ml1 = [&](int m0, int h, int kb) {
         uint32_t sa, full;
-        if (!next_stage(sa, full)) return;
+        if (!next_stage(sa, full, kStageBytes)) return;
         const int n0 = h * 256 + static_cast<int>(pm) * 128;  // this CTA's half of the UMMA's 256 columns
         tma_load_3d_pair(sa, &tmX, full, kb * 64, m0, 0);
         tma_load_3d_pair(sa + kBoxBytes, &tmW1, full, n0, kb * 64, 0);
         tma_load_3d_pair(sa + kBoxBytes + 8192, &tmW1, full, n0 + 64, kb * 64, 0);
+        if (LOCK) {  // the same columns of the second half behind them
+          tma_load_3d_pair(sa + 2 * kBoxBytes, &tmW1, full, n0 + 256, kb * 64, 0);
+          tma_load_3d_pair(sa + 2 * kBoxBytes + 8192, &tmW1, full, n0 + 256 + 64, kb * 64, 0);
+        }
       };
       auto push_w2 = [&](int h) {
         uint32_t sa, full;
-        if (!next_stage(sa, full)) return;
+        if (!next_stage(sa, full, 2 * kBoxBytes)) return;
         const int c0 = static_cast<int>(pm) * 64;  // this CTA's half of the 128 output columns
         tma_load_3d_pair(sa, &tmW2, full, c0, h * 256, 0);
         tma_load_3d_pair(sa + kBoxBytes, &tmW2, full, c0, h * 256 + 128, 0);
       };
-      for (int u = 0; u < nunits && ok; ++u) {
-        const int m0 = tile_m0(u / NH), h = u % NH;
-        for (int kb = 0; kb < KBa; ++kb) push_ml1(m0, h, kb);
-        if (u > 0) push_w2((u - 1) % NH);
-        for (int kb = KBa; kb < KB; ++kb) push_ml1(m0, h, kb);
+      if constexpr (LOCK) {
+        for (int it = 0; it < my_tiles && ok; ++it) {
+          const int m0 = tile_m0(it);
+          for (int kb = 0; kb < KB; ++kb) push_ml1(m0, 0, kb);
+          push_w2(0);
+          push_w2(1);
+        }
+      } else {
+        for (int u = 0; u < nunits && ok; ++u) {
+          const int m0 = tile_m0(u / NH), h = u % NH;
+          for (int kb = 0; kb < KBa; ++kb) push_ml1(m0, h, kb);
+          if (u > 0) push_w2((u - 1) % NH);
+          for (int kb = KBa; kb < KB; ++kb) push_ml1(m0, h, kb);
+        }
+        if (nunits > 0) push_w2((nunits - 1) % NH);
       }
-      if (nunits > 0) push_w2((nunits - 1) % NH);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------------------------------ UMMA issuer (even CTA)
@@ -198,7 +226,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         ++sfull_uses;
         tcgen05_fence_after_sync();
         const int it = u / NH, h = u % NH;
-        const uint32_t d_o = tmem_base + static_cast<uint32_t>((it & 1) * 256);
+        const uint32_t d_o = tmem_base + static_cast<uint32_t>(LOCK ? 0 : (it & 1) * 256);
         const uint64_t wdesc = make_smem_desc_sw128(sa, 8192, 1024);
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
@@ -213,7 +241,40 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           umma_commit_pair(map_to_cta(bar_ofull, peer));
         }
       };
-      for (int u = 0; u < nunits && ok; ++u) {
+      if constexpr (LOCK) {
+        // both halves in lock-step: the X block of a stage feeds the UMMAs of half 0 (slot 0) and of half 1 (slot 1); the tile's
+        // two ML2s follow its MainLoop, O in the first 128 columns of slot 0 (read out by Epi1 before S of half 0 exists)
+        for (int it = 0; it < my_tiles && ok; ++it) {
+          for (int slot = 0; slot < 2 && ok; ++slot) {
+            if (slot_uses[slot] > 0 && !mbar_wait<false>(bar_pfree(slot), (slot_uses[slot] - 1u) & 1u, w)) ok = false;
+            ++slot_uses[slot];
+          }
+          if (!ok) break;
+          tcgen05_fence_after_sync();
+          for (int kb = 0; kb < KB && ok; ++kb) {
+            const uint32_t sa = wait_stage();
+            if (!ok) break;
+            const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
+            const uint64_t bdesc0 = make_smem_desc_sw128(sa + kBoxBytes, 8192, 1024);
+            const uint64_t bdesc1 = make_smem_desc_sw128(sa + 2 * kBoxBytes, 8192, 1024);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+              umma_bf16_ss_pair(tmem_base, adesc + static_cast<uint64_t>(k * 2), bdesc0 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
+              umma_bf16_ss_pair(tmem_base + 256, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
+            }
+            release_stage();
+          }
+          if (!ok) break;
+          for (int slot = 0; slot < 2; ++slot) {
+            umma_commit_pair(bar_pfull(slot));
+            umma_commit_pair(map_to_cta(bar_pfull(slot), peer));
+          }
+          ml2(2 * it);
+          ml2(2 * it + 1);
+        }
+      }
+      for (int u = 0; !LOCK && u < nunits && ok; ++u) {
         const int it = u / NH, h = u % NH;
         const int slot = (it & 1) ^ h;
         // the slot's previous content (a P half read by Epi1, or an O read by Epi2) has been read by both CTAs
@@ -231,7 +292,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           umma_commit_pair(map_to_cta(bar_pfull(slot), peer));
         }
       }
-      if (nunits > 0 && ok) ml2(nunits - 1);
+      if (!LOCK && nunits > 0 && ok) ml2(nunits - 1);
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
       mbar_wait<false>(bar_drain, 0, w);
     }
@@ -253,7 +314,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     // ---------------- Epi1(u): S = bf16(ReLU(P + b1)) of one half, as the A operand of ML2(u)
     auto epi1 = [&](int u) {
       const int it = u / NH, h = u % NH;
-      const int slot = (it & 1) ^ h;
+      const int slot = LOCK ? h : ((it & 1) ^ h);
       mbar_wait<false>(bar_pfull(slot), puses[slot] & 1u, w);
       ++puses[slot];
       __syncwarp();
@@ -305,7 +366,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     };
     // ---------------- Epi2(it): O = bf16(ReLU(acc + b2)), two 128 x 64 boxes staged in the S buffer and stored together
     auto epi2 = [&](int it) {
-      const int oslot = it & 1;
+      const int oslot = LOCK ? 0 : (it & 1);
       mbar_wait<false>(bar_ofull, static_cast<uint32_t>(it) & 1u, w);  // also: the tile's last ML2 has read S
       __syncwarp();
       tcgen05_fence_after_sync();
@@ -364,6 +425,15 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
 }  // namespace
 
+// COMFUSE_B2B_STREAM_LOCK=0 runs N1 = 512 on the alternating-slot schedule as well (for comparison)
+static bool stream_lock_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("COMFUSE_B2B_STREAM_LOCK");
+    return !(e && e[0] == '0');
+  }();
+  return on;
+}
+
 bool b2b_stream_supported(int K, int N1, int N2) { return N2 == 128 && (N1 == 256 || N1 == 512) && K >= 8 && K % 8 == 0; }
 
 cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
@@ -387,7 +457,8 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = StreamSmem::BYTES;
+  const bool lock = p.N1 == 512 && stream_lock_enabled();
+  cfg.dynamicSmemBytes = lock ? StreamSmem<true>::BYTES : StreamSmem<false>::BYTES;
   cfg.stream = st;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
@@ -398,11 +469,15 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   if (max_clusters[di] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(b2b_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamSmem::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(b2b_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamSmem<false>::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(b2b_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamSmem<true>::BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
-    e = cudaOccupancyMaxActiveClusters(&n, b2b_stream_kernel, &cfg);
+    cfg.dynamicSmemBytes = StreamSmem<false>::BYTES;  // both instantiations: one CTA per SM
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_stream_kernel<false>, &cfg);
+    cfg.dynamicSmemBytes = lock ? StreamSmem<true>::BYTES : StreamSmem<false>::BYTES;
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di] = n;
@@ -411,7 +486,8 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
-  return cudaLaunchKernelEx(&cfg, b2b_stream_kernel, tmX, tmW1, tmW2, tmO, p);
+  return lock ? cudaLaunchKernelEx(&cfg, b2b_stream_kernel<true>, tmX, tmW1, tmW2, tmO, p)
+              : cudaLaunchKernelEx(&cfg, b2b_stream_kernel<false>, tmX, tmW1, tmW2, tmO, p);
 }
 
 }  // namespace comfuse

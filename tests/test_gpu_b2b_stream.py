@@ -161,3 +161,38 @@ def test_relu_mlp_back_to_back_dependent_launches(cuda_device):
         b = chain(sync=False)
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
     assert cf.last_device_status() == cf.OK
+
+
+_SCHEDULE_CHILD = r"""
+import sys, numpy as np, torch
+import workloads as wl
+from tests import parity as P
+import paper_2608_03537_b200 as cf
+out = {}
+for name, (M, K) in (("many_tiles", (40000, 128)), ("dlrm_dims", (300, 1024)), ("odd_blocks", (2048, 192))):
+    w = wl.dlrm_bottom_mlp(M, K, 512, 128, seed=M + K)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=name)
+    assert cf.last_device_status() == cf.OK
+    out[name] = got["Y"].view(torch.int16).cpu().numpy()
+np.savez(sys.argv[1], **out)
+"""
+
+
+def test_both_schedules_for_two_halves_agree_bit_for_bit(tmp_path, cuda_device):
+    """N1 = 512 runs with both halves in lock-step by default; COMFUSE_B2B_STREAM_LOCK=0 (read once per process, hence the
+    child processes) selects the alternating-slot schedule that N1 = 256 always uses.  Both accumulate every output element in
+    the same order: same bits, and each is checked against the oracle in its child."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = {}
+    for flag in ("1", "0"):
+        path = str(tmp_path / f"s{flag}.npz")
+        env = dict(os.environ, COMFUSE_B2B_STREAM_LOCK=flag, PYTHONPATH=root)
+        r = subprocess.run([sys.executable, "-c", _SCHEDULE_CHILD, path], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        res[flag] = np.load(path)
+    assert sorted(res["0"].files) == sorted(res["1"].files) and len(res["0"].files) == 3
+    for k in res["0"].files:
+        assert np.array_equal(res["0"][k], res["1"][k]), k
