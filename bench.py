@@ -426,6 +426,19 @@ def run_comfuse(args):
 
     extra = {}
     if not args.kernel_only:
+        # ---- the paper reports mean and minimum over its timed replays (Sec. 6 Setup): right behind the timed region, the
+        # minimum over groups of five replays of the step graph, each group between its own pair of events
+        if graph is not None and world == 1:
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(8)]
+            torch.cuda._sleep(400_000)
+            for a, b in evs:
+                a.record()
+                for _ in range(5):
+                    graph.replay()
+                b.record()
+            torch.cuda.synchronize()
+            extra["min_ms_per_step"] = min(a.elapsed_time(b) for a, b in evs) / (5 * nsets)
+            extra["min_over"] = f"8 groups of 5 graph replays ({5 * nsets} steps each)"
         # ---- the in-library unfused path on the same buffers (context: speedup of fusion)
         try:
             other = not fused
@@ -454,17 +467,6 @@ def run_comfuse(args):
         for i in range(3):
             step(sets[0])
         extra["warm_l2_ms_per_step"] = timed(n3, lambda i: step(sets[0])) / n3
-        # ---- the paper reports mean and minimum over its timed replays (Sec. 6 Setup): the minimum over single replays of
-        # the step graph (one launch per buffer set), each between its own pair of events, outside the main timed region
-        if graph is not None and world == 1:
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(30)]
-            torch.cuda._sleep(400_000)
-            for a, b in evs:
-                a.record()
-                graph.replay()
-                b.record()
-            torch.cuda.synchronize()
-            extra["min_ms_per_step"] = min(a.elapsed_time(b) for a, b in evs) / nsets
 
         def gemm_only(sx):
             if b2b:
