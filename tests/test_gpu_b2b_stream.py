@@ -196,3 +196,14 @@ def test_both_schedules_for_two_halves_agree_bit_for_bit(tmp_path, cuda_device):
     assert sorted(res["0"].files) == sorted(res["1"].files) and len(res["0"].files) == 3
     for k in res["0"].files:
         assert np.array_equal(res["0"][k], res["1"][k]), k
+
+
+def test_relu_mlp_million_rows_sampled(cuda_device):
+    """A million ragged rows (3907 tiles, 53 per CTA pair): sampled rows against the oracle, everything finite."""
+    M, K, N1 = 1_000_003, 64, 512
+    w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=77)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    assert torch.isfinite(got["Y"].float()).all().item()
+    rows = np.unique(np.concatenate([wl.sample_rows(M, 600), np.arange(M - 300, M)]))
+    P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label="relu mlp 1e6 rows")
+    assert cf.last_device_status() == cf.OK
