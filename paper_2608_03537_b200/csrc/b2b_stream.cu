@@ -257,19 +257,28 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
             const uint64_t bdesc0 = make_smem_desc_sw128(sa + kBoxBytes, 8192, 1024);
             const uint64_t bdesc1 = make_smem_desc_sw128(sa + 2 * kBoxBytes, 8192, 1024);
+            if (kb + 1 < KB) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-              umma_bf16_ss_pair(tmem_base, adesc + static_cast<uint64_t>(k * 2), bdesc0 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
-              umma_bf16_ss_pair(tmem_base + 256, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
+              for (int k = 0; k < 4; ++k) {
+                const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+                umma_bf16_ss_pair(tmem_base, adesc + static_cast<uint64_t>(k * 2), bdesc0 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
+                umma_bf16_ss_pair(tmem_base + 256, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc_ml1, acc);
+              }
+            } else {
+              // last K block: half 0 first, so that its epilogue starts while the tensor pipe finishes half 1
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  umma_bf16_ss_pair(tmem_base + half * 256, adesc + static_cast<uint64_t>(k * 2),
+                                    (half ? bdesc1 : bdesc0) + static_cast<uint64_t>(k * 128), idesc_ml1, (kb | k) != 0 ? 1u : 0u);
+                umma_commit_pair(bar_pfull(half));
+                umma_commit_pair(map_to_cta(bar_pfull(half), peer));
+              }
             }
             release_stage();
           }
           if (!ok) break;
-          for (int slot = 0; slot < 2; ++slot) {
-            umma_commit_pair(bar_pfull(slot));
-            umma_commit_pair(map_to_cta(bar_pfull(slot), peer));
-          }
           ml2(2 * it);
           ml2(2 * it + 1);
         }
