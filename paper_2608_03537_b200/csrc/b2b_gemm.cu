@@ -1,17 +1,11 @@
-// Fused back-to-back GEMM (Sec. 4):  P = X W1,  S = GELU_tanh(P + b1),  O' = S W2 + b2 + X,  O = LayerNorm(O').
-// Neither P nor S is written to global memory.
+// Fused back-to-back GEMM, attention form (Sec. 4 with a row softmax as F; the Target- and Self-Attention shapes of
+// Sec. 6.2):  P = alpha X W1,  S = exp(P - rowmax),  O = (S W2) / rowsum, per batch.  Neither P nor S is written to
+// global memory.  (The MLP form lives in b2b_mlp.cu, the ReLU MLP form with K streamed in b2b_stream.cu.)
 //
-// Dataflow (Sec. 4.1, adapted): N1 is cut into 128-column chunks.  Instead of spreading the chunks over the CTAs of
-// a cluster and summing partial O tiles at the commit, one CTA pair walks all chunks of its 256 rows and accumulates
-// O in tensor memory, which keeps the sum deterministic and needs no cross-CTA reduction.
-//
-// Consumer schedule (Sec. 4.3, ML1 -> Epi1 -> ML2 -> Epi2 staggered by one stage): the UMMA lane issues
-//   ML1(0) ML1(1) | ML2(0) ML1(2) | ML2(1) ML1(3) | ML2(2) | ML2(3)
-// so that Epi1(j) (bias + GELU + bf16 rounding into a swizzled shared-memory A operand) overlaps ML1(j+1) and
-// ML2(j-1); P has two TMEM slots, S two shared-memory buffers, O two TMEM slots (Epi2 of tile t overlaps tile t+1).
-//
-// Producer (Sec. 4.2, unified circular buffer): X, the W1 chunks, the W2 chunks and the residual copy of X all flow
-// through ONE ring of 16 KB slots (a 128-row x 64-element bf16 box each), in the order the consumers need them.
+// One CTA pair owns 256 rows; the two P slots hold a whole score row of 256 source positions (512 run as two sub-tiles
+// with their own maxima, combined when O is normalised); O accumulates in tensor memory.  X, the two W1 chunks and the
+// two W2 chunks flow through ONE ring of 16 KB slots (Sec. 4.2, unified circular buffer), in the order the consumers need
+// them; the roles are software-pipelined over the cluster's tiles (see the UMMA lane).
 //
 // CTA pairs (cta_group::2): each CTA holds its own 128 rows of X / S and half (64 columns) of every weight chunk.
 #include <cuda_runtime.h>
@@ -31,30 +25,23 @@ constexpr int kB2bEpiThreads = 32 * kB2bEpiWarps;
 constexpr int kB2bThreads = 32 * (2 + kB2bEpiWarps);  // producer, UMMA, epilogue warps
 constexpr int kSlotBytes = 128 * 64 * 2;  // one 128 x 64 bf16 box
 constexpr int kRingSlots = 8;
-constexpr int kMaxChunks = 4;             // N1 <= 512
 
 struct B2bSmem {
   static constexpr int OFF_RING = 0;
   static constexpr int OFF_S = kRingSlots * kSlotBytes;            // 2 buffers x 2 K blocks
-  static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // output staging box (the second one is borrowed, see Epi2)
-  static constexpr int OFF_B1 = OFF_YBUF + kSlotBytes;             // fp32 [512]
-  static constexpr int OFF_VEC = OFF_B1 + kMaxChunks * 128 * 4;    // b2, gamma, beta fp32 [128] each
-  static constexpr int OFF_PRE = OFF_VEC + 3 * 128 * 4;            // float2 [2][4][128]
+  static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // output staging box (the second one is the idle eighth ring slot)
+  static constexpr int OFF_PRE = OFF_YBUF + kSlotBytes;            // float2 [2][4][128]
   static constexpr int OFF_STATS = OFF_PRE + 2 * 4 * 128 * 8;      // float2 [2][1][128]
   static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
-  // barriers: full[8] empty[8] rfull[8] pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats[2] drain pfree
+  // barriers: full[8] empty[8] (8 unused) pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats[2] drain pfree
   static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 4;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
 static_assert(B2bSmem::BYTES <= 232448, "shared memory budget");
 
-// Ring items of one tile, in producer order (every role walks this sequence):
-//   X0 X1 | W1(0) W1(1) | { W2(j) W1(j+2) } for each chunk j | R0 R1      = 2 + 2*NC + 2 slots
-
-// MODE 0: MLP form (F = GELU(. + b1), tail = + b2 + X, LayerNorm); MODE 1: attention form (F = row softmax, no tail).
-// NHALF (attention form): sub-tiles of 256 source positions per score row, 1 or 2.
-template <int MODE, int NHALF = 1>
+// NHALF: sub-tiles of 256 source positions per score row, 1 or 2.
+template <int NHALF>
 __global__ void __launch_bounds__(kB2bThreads, 1)
 b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                 const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
@@ -63,16 +50,11 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
   const uint32_t smem_base = smem_u32(smem);
 
-  float* s_b1 = reinterpret_cast<float*>(smem + B2bSmem::OFF_B1);
-  float* s_b2 = reinterpret_cast<float*>(smem + B2bSmem::OFF_VEC);
-  float* s_gamma = s_b2 + 128;
-  float* s_beta = s_gamma + 128;
   float2* s_pre = reinterpret_cast<float2*>(smem + B2bSmem::OFF_PRE);
   float2* s_stats = reinterpret_cast<float2*>(smem + B2bSmem::OFF_STATS);
   const uint32_t bar_base = smem_base + B2bSmem::OFF_BAR;
   auto bar_full = [&](int s) { return bar_base + 8u * s; };                        // weight / X slot landed (even CTA)
   auto bar_empty = [&](int s) { return bar_base + 8u * (kRingSlots + s); };        // slot may be overwritten
-  auto bar_rfull = [&](int s) { return bar_base + 8u * (2 * kRingSlots + s); };    // residual slot landed (own CTA)
   auto bar_pfull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + a); };    // P slot complete
   auto bar_sfull = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 2 + a); };   // S buffer written by both CTAs (even CTA)
   auto bar_sempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 4 + a); };  // S buffer read by ML2
@@ -91,19 +73,15 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const uint32_t leader = 0u, peer = rank ^ 1u;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
-  const int NC = p.N1 / 128;
   const int total_tiles = p.batch * p.mpairs;
   // attention form: a score row of 512 source positions is processed as two sub-tiles of 256 (each with its own maximum
   // and its own O slot) that the normalisation step combines; nsub = sub-tiles this cluster walks
   constexpr int nhalf = NHALF;
   const int my_tiles = cluster_id < total_tiles ? (total_tiles - cluster_id + num_clusters - 1) / num_clusters : 0;
   const int nsub = my_tiles * nhalf;
-  constexpr bool has_tail_residual = MODE == 0;  // the MLP form adds X back before its LayerNorm
-  // The attention form's epilogue, not its loads, sets the pace: it walks seven of the eight ring slots and uses the
-  // eighth as a second output staging box, so that both 64-column halves of a tile are staged and stored together.
-  // (The MLP form cannot give a slot away: X0, X1 stay at the head of the ring until ML1 of the last chunk has been
-  // issued, and W1 of that chunk is the eighth item behind them -- with seven slots the producer would wait for X0.)
-  constexpr int RING = MODE == 1 ? kRingSlots - 1 : kRingSlots;
+  // The epilogue, not the loads, sets the pace: the ring walks seven of the eight slots and the eighth is a second output
+  // staging box, so that both 64-column halves of a tile are staged and stored together.
+  constexpr int RING = kRingSlots - 1;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 #ifdef COMFUSE_TRACE
@@ -114,14 +92,11 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     for (int s = 0; s < kRingSlots; ++s) {
       mbar_init(bar_full(s), 2);
       mbar_init(bar_empty(s), 1);
-      mbar_init(bar_rfull(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_pfull(a), 1);
       mbar_init(bar_sfull(a), 2 * kB2bEpiWarps);   // one arrival per epilogue warp of both CTAs
-      // S buffer 1 of the MLP form doubles as the second output staging box: handing it back takes the UMMA commit AND
-      // the store thread's word that the previous tile's output store has read it (see Epi1 / Epi2 below)
-      mbar_init(bar_sempty(a), (MODE == 0 && a == 1) ? 2 : 1);
+      mbar_init(bar_sempty(a), 1);
       mbar_init(bar_ofull(a), 1);
       mbar_init(bar_oempty(a), 2 * kB2bEpiWarps);
     }
@@ -155,24 +130,19 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     if (lane == 0) {
       RingPos<RING> ring;
       bool ok = true;
-      // one box into the current slot; kind 0: pair operand (signals the even CTA's full barrier), 1: residual
+      // one box into the current slot (a pair operand: signals the even CTA's full barrier)
       int bz = 0;  // batch coordinate of the current tile
-      auto push = [&](const CUtensorMap* tm, int x, int y, int kind) {
+      auto push = [&](const CUtensorMap* tm, int x, int y, int) {
         if (!ok) return;
         if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; return; }
-        if (kind == 0) {
-          const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
-          mbar_arrive_expect_tx_cluster(full, kSlotBytes);
-          tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, bz);
-        } else {
-          mbar_arrive_expect_tx(bar_rfull(ring.stage), kSlotBytes);
-          tma_load_3d(ring_addr(ring.stage), tm, bar_rfull(ring.stage), x, y, bz);
-        }
+        const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
+        mbar_arrive_expect_tx_cluster(full, kSlotBytes);
+        tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, bz);
         ring.advance();
       };
       const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
-      if constexpr (MODE == 1) {
-        // attention form, software-pipelined over tiles (see the UMMA lane): Q and K of tile t+1 go in before V of tile t
+      {
+        // software-pipelined over tiles (see the UMMA lane): Q and K of tile t+1 go in before V of tile t
         // sub-tile k of this cluster = 256 source positions (`half`) of its (k / nhalf)-th row tile
         auto push_qk = [&](int k) {
           const int tile = cluster_id + (k / nhalf) * num_clusters, half = k % nhalf;
@@ -190,22 +160,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           bz = tile / p.mpairs;
           push(&tmW2, wcol, half * 256 + 0 * 128, 0);
           push(&tmW2, wcol, half * 256 + 1 * 128, 0);
-        }
-      }
-      for (int tile = cluster_id; MODE == 0 && tile < total_tiles && ok; tile += num_clusters) {
-        bz = tile / p.mpairs;
-        const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
-        push(&tmX, 0, m0, 0);
-        push(&tmX, 64, m0, 0);
-        push(&tmW1, 0 * 128 + wcol, 0, 0);
-        if (NC > 1) push(&tmW1, 1 * 128 + wcol, 0, 0);
-        for (int j = 0; j < NC; ++j) {
-          push(&tmW2, wcol, j * 128, 0);
-          if (j + 2 < NC) push(&tmW1, (j + 2) * 128 + wcol, 0, 0);
-        }
-        if (has_tail_residual) {
-          push(&tmX, 0, m0, 1);
-          push(&tmX, 64, m0, 1);
         }
       }
     }
@@ -230,8 +184,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         umma_commit_pair(bar_empty(stage));
         umma_commit_pair(map_to_cta(bar_empty(stage), peer));
       };
-      if constexpr (MODE == 1) {
-        // Attention form, software-pipelined over the cluster's tiles: the scores of tile t+1 (ML1) are issued as soon
+      {
+        // Software-pipelined over the cluster's tiles: the scores of tile t+1 (ML1) are issued as soon
         // as the epilogue has read the scores of tile t out of the P slots, BEFORE S.V of tile t (ML2), so that the
         // epilogue can go from the softmax of tile t straight to the softmax of tile t+1 while ML2(t) runs, and finds
         // O(t) complete when it comes back for the normalisation.
@@ -298,74 +252,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           }
         }
       }
-      for (int tile = cluster_id; MODE == 0 && tile < total_tiles && ok; tile += num_clusters, ++tile_it) {
-        const int obuf = tile_it & 1u;
-        const uint32_t d_o = tmem_base + 256 + obuf * 128;
-        // X: two K blocks
-        const int xs0 = ring.stage;
-        const uint32_t x0 = wait_slot();
-        ring.advance();
-        const int xs1 = ring.stage;
-        const uint32_t x1 = wait_slot();
-        ring.advance();
-        const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
-        const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
-        auto issue_ml1 = [&](int j) {
-          // P[j & 1] = X . W1[:, chunk j]
-          const int wstage = ring.stage;
-          const uint32_t wa = wait_slot();
-          ring.advance();
-          if (!ok) return;
-          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
-          const uint32_t d_p = tmem_base + (j & 1) * 128;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_bf16_ss_pair(d_p, (k < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((k & 3) * 2), wdesc + static_cast<uint64_t>(k * 128),
-                              idesc_ml1, k != 0 ? 1u : 0u);
-          release_slot(wstage);
-          umma_commit_pair(bar_pfull(j & 1));
-          umma_commit_pair(map_to_cta(bar_pfull(j & 1), peer));
-          if (j == NC - 1) {  // X is no longer needed by the tensor pipe
-            release_slot(xs0);
-            release_slot(xs1);
-          }
-        };
-        auto issue_ml2 = [&](int j) {
-          // O += S_j . W2[chunk j, :]
-          const int wstage = ring.stage;
-          const uint32_t wa = wait_slot();
-          ring.advance();
-          if (!ok) return;
-          const int sb = j & 1;
-          if (!mbar_wait<false>(bar_sfull(sb), sfull_uses[sb] & 1u, w)) { ok = false; return; }
-          ++sfull_uses[sb];
-          tcgen05_fence_after_sync();
-          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
-          const uint64_t sdesc0 = make_smem_desc_sw128(s_addr(sb, 0), 16, 1024);
-          const uint64_t sdesc1 = make_smem_desc_sw128(s_addr(sb, 1), 16, 1024);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_bf16_ss_pair(d_o, (k < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((k & 3) * 2), wdesc + static_cast<uint64_t>(k * 128),
-                              idesc_ml2, (j | k) != 0 ? 1u : 0u);
-          release_slot(wstage);
-          umma_commit_pair(bar_sempty(sb));
-          umma_commit_pair(map_to_cta(bar_sempty(sb), peer));
-        };
-        // O slot must have been drained by Epi2 of the tile before the previous one
-        if (!mbar_wait<false>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
-        tcgen05_fence_after_sync();
-        issue_ml1(0);
-        if (NC > 1) issue_ml1(1);
-        for (int j = 0; j < NC && ok; ++j) {
-          issue_ml2(j);
-          if (j + 2 < NC) issue_ml1(j + 2);
-        }
-        if (ok) {
-          umma_commit_pair(bar_ofull(obuf));
-          umma_commit_pair(map_to_cta(bar_ofull(obuf), peer));
-        }
-        if (has_tail_residual) ring.skip(2);  // the residual slots belong to the epilogue
-      }
       umma_commit_pair(bar_drain);
       mbar_wait<false>(bar_drain, 0, w);
     }
@@ -376,14 +262,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int row = q * 32 + lane;
     const int epi_tid = threadIdx.x - 64;
     const bool store_thread = epi_tid == 0;
-    // the row vectors, widened to fp32 once, by the epilogue warps (idle until the first P chunk is complete)
-    for (int i = epi_tid; i < p.N1; i += kB2bEpiThreads) s_b1[i] = p.b1 ? bf16_lo(p.b1[i]) : 0.f;
-    for (int i = epi_tid; i < 128; i += kB2bEpiThreads) {
-      s_b2[i] = p.b2 ? bf16_lo(p.b2[i]) : 0.f;
-      s_gamma[i] = p.gamma ? bf16_lo(p.gamma[i]) : 1.f;
-      s_beta[i] = p.beta ? bf16_lo(p.beta[i]) : 0.f;
-    }
-    named_barrier_sync(2, kB2bEpiThreads);
     const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
     const uint32_t ybuf = smem_base + B2bSmem::OFF_YBUF;
     const uint32_t sfull_leader = map_to_cta(bar_sfull(0), leader);
@@ -391,9 +269,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     const int kblk = hh >> 1;            // K block of S (and residual box) this thread's columns fall into
     const int chunk0 = (hh & 1) * 4;     // first of its four 16-byte chunks inside that 128-byte row
     RingPos<RING> ring;
-    uint32_t rfull_bits = 0;
     uint32_t puses[2] = {0, 0}, suses[2] = {0, 0};
-    uint32_t tile_it = 0;
     int xpar = 0;
     uint32_t xphase = 0;
 #ifdef COMFUSE_TRACE
@@ -406,8 +282,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #define B2B_TRACE_POINT() do { } while (0)
 #endif
 
-    if constexpr (MODE == 1) {
-      // ================= attention form, software-pipelined over the cluster's tiles:
+    {
+      // ================= software-pipelined over the cluster's tiles:
       //   softmax(t0) | softmax(t1) finish(t0) | softmax(t2) finish(t1) | ... | finish(last)
       // so that S.V of tile t (ML2) runs under the softmax of tile t+1 and the UMMA lane never waits for this epilogue
       // longer than one softmax.
@@ -576,182 +452,6 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         }
       }
     }
-    for (int tile = cluster_id; MODE == 0 && tile < total_tiles; tile += num_clusters, ++tile_it) {
-      B2B_TRACE_POINT();
-      const int bz = tile / p.mpairs;
-      const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
-      const int obuf = tile_it & 1u;
-      // ---------------- Epi1(j): S_j = bf16(GELU(P_j + b1)) as the next UMMA's A operand
-      for (int j = 0; j < NC; ++j) {
-        const int pb = j & 1;
-        mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
-        ++puses[pb];
-        __syncwarp();
-        tcgen05_fence_after_sync();
-        B2B_TRACE_POINT();
-        // the S buffer is free once ML2 of chunk j-2 has read it -- and, for buffer 1, once the output store that staged
-        // its second box there has read it: the store thread adds that arrival to the phase of the buffer's previous use
-        if (pb == 1 && store_thread && suses[1] > 0) {
-          tma_store_wait_read<0>();
-          mbar_arrive(bar_sempty(1));
-        }
-        mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
-        ++suses[pb];
-        __syncwarp();
-        B2B_TRACE_POINT();
-        uint32_t v[32];
-        tmem_ld_32cols(tmem_base + lane_sel + pb * 128 + hh * 32, v);
-        const float4* b4 = reinterpret_cast<const float4*>(s_b1 + j * 128 + hh * 32);
-        uint32_t pk[16];
-#ifdef COMFUSE_TRACE
-        const int tf = p.trace_flags;
-#else
-        constexpr int tf = 0;
-#endif
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float4 bb = b4[i];
-          float2 g01, g23;
-          if (tf & 1) {  // experiment: no transcendental
-            g01 = add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y));
-            g23 = add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w));
-          } else {
-            g01 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)));
-            g23 = gelu_tanh_f32x2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)));
-          }
-          pk[2 * i] = pack_bf16x2_rn(g01);
-          pk[2 * i + 1] = pack_bf16x2_rn(g23);
-        }
-        const uint32_t sb = s_addr(pb, kblk);
-        if (!(tf & 2)) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t a = sb + swz128(row, chunk0 + i);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                       "r"(pk[4 * i + 3])
-                       : "memory");
-        }
-        }
-        B2B_TRACE_POINT();
-        tcgen05_fence_before_sync();  // P slot reads are complete before the UMMA lane is told to go on
-        if (!(tf & 4)) fence_proxy_async_smem();     // S writes are visible to the tensor core's shared-memory reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster_noflush(sfull_leader + 8u * pb);
-        B2B_TRACE_POINT();
-      }
-      ring.skip(2 + 2 * NC);  // X, W1 and W2 slots were the tensor pipe's
-      // ---------------- Epi2: O' = O + b2 + X, LayerNorm over the 128 columns, store
-      mbar_wait<false>(bar_ofull(obuf), (tile_it >> 1) & 1u, w);
-      __syncwarp();
-      tcgen05_fence_after_sync();
-      B2B_TRACE_POINT();
-      const uint32_t o_addr = tmem_base + lane_sel + 256 + obuf * 128 + hh * 32;
-      uint32_t pk[16];
-      {
-      const int s0 = ring.stage;
-      const int s1 = s0 + 1 == RING ? 0 : s0 + 1;
-      // both residual slots are waited for by everybody (the phase bits must advance uniformly)
-      mbar_wait<false>(bar_rfull(s0), (rfull_bits >> s0) & 1u, w);
-      rfull_bits ^= 1u << s0;
-      mbar_wait<false>(bar_rfull(s1), (rfull_bits >> s1) & 1u, w);
-      rfull_bits ^= 1u << s1;
-      __syncwarp();
-      uint32_t r32[16];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t a = ring_addr(kblk ? s1 : s0) + swz128(row, chunk0 + i);
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(r32[4 * i]), "=r"(r32[4 * i + 1]), "=r"(r32[4 * i + 2]), "=r"(r32[4 * i + 3])
-                     : "r"(a));
-      }
-      // hand the two residual slots back
-      __syncwarp();
-      named_barrier_sync(2, kB2bEpiThreads);
-      if (store_thread) {
-        mbar_arrive(bar_empty(s0));
-        mbar_arrive(bar_empty(s1));
-      }
-      ring.skip(2);
-      // stage 1: x = O + b2 + X ; thread-local (mean, M2) over this thread's 32 columns; x goes back into TMEM
-      float2 part;
-      {
-        uint32_t v[32];
-        tmem_ld_32cols(o_addr, v);
-        const float4* b4 = reinterpret_cast<const float4*>(s_b2 + hh * 32);
-        float2 s01 = splat2(0.f), s23 = splat2(0.f);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float4 bb = b4[i];
-          const float2 x01 = add2(add2(f2_from_bits(v[4 * i], v[4 * i + 1]), make_float2(bb.x, bb.y)), bf16x2_to_f2(r32[2 * i]));
-          const float2 x23 = add2(add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), make_float2(bb.z, bb.w)), bf16x2_to_f2(r32[2 * i + 1]));
-          v[4 * i] = __float_as_uint(x01.x); v[4 * i + 1] = __float_as_uint(x01.y);
-          v[4 * i + 2] = __float_as_uint(x23.x); v[4 * i + 3] = __float_as_uint(x23.y);
-          s01 = add2(s01, x01);
-          s23 = add2(s23, x23);
-        }
-        const float cmean = ((s01.x + s01.y) + (s23.x + s23.y)) * (1.f / 32.f);
-        const float2 nm = splat2(-cmean);
-        float2 q01 = splat2(0.f), q23 = splat2(0.f);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float2 d01 = add2(f2_from_bits(v[4 * i], v[4 * i + 1]), nm);
-          const float2 d23 = add2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), nm);
-          q01 = fma2(d01, d01, q01);
-          q23 = fma2(d23, d23, q23);
-        }
-        part = make_float2(cmean, (q01.x + q01.y) + (q23.x + q23.y));
-        tmem_st_32cols(o_addr, v);
-        tmem_st_wait();
-      }
-      // reduce: the row lives in this CTA only (four quarter-row threads)
-      const float2 tot =
-          cluster_row_reduce<1, MergeWelford, 4>(part, 32.f, MergeWelford(), s_pre, s_stats, bar_stats, row, hh, 0u, xpar, xphase, w);
-      B2B_TRACE_POINT();
-      const float mu = tot.x;
-      const float rstd = rsqrtf(tot.y * (1.f / 128.f) + p.eps);
-      // stage 2: normalise the resident x, round once
-      {
-        uint32_t v[32];
-        tmem_ld_32cols(o_addr, v);
-        const float4* g4 = reinterpret_cast<const float4*>(s_gamma + hh * 32);
-        const float4* be4 = reinterpret_cast<const float4*>(s_beta + hh * 32);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float4 gg = g4[i], be = be4[i];
-          const float2 n01 = fma2(f2_from_bits(v[4 * i], v[4 * i + 1]), splat2(rstd), splat2(-mu * rstd));
-          const float2 n23 = fma2(f2_from_bits(v[4 * i + 2], v[4 * i + 3]), splat2(rstd), splat2(-mu * rstd));
-          pk[2 * i] = pack_bf16x2_rn(fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y)));
-          pk[2 * i + 1] = pack_bf16x2_rn(fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w)));
-        }
-      }
-      }  // MLP form
-      // the accumulator has been read for the last time: the O slot can be reused by the tile after the next one
-      tcgen05_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
-      // two 128 x 64 boxes (columns 0..63 from the hh = 0, 1 warps, 64..127 from hh = 2, 3), staged and stored together:
-      // the second box sits in S buffer 1 (first K block), which is idle between the last ML2 of this tile -- complete,
-      // the O slot was full -- and Epi1 of chunk 1 of the next tile, which waits for this store's read (above)
-      if (store_thread) tma_store_wait_read<0>();  // the previous tile's stores have read both boxes
-      named_barrier_sync(3, kB2bEpiThreads);
-      {
-        const uint32_t box = kblk == 0 ? ybuf : s_addr(1, 0);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t a = box + swz128(row, chunk0 + i);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                       "r"(pk[4 * i + 3])
-                       : "memory");
-        }
-      }
-      fence_proxy_async_smem();
-      named_barrier_sync(3, kB2bEpiThreads);
-      if (store_thread) {
-        tma_store_3d(&tmO, ybuf, 0, m0, bz);
-        tma_store_3d(&tmO, s_addr(1, 0), 64, m0, bz);
-        tma_store_commit();
-      }
-    }
     if (store_thread) tma_store_wait_read<0>();  // the staging buffer must outlive the last store's read
   }
 
@@ -776,7 +476,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 bool b2b_fused_supported(int K, int N1, int N2, int mode) {
   // attention form: 256 source positions fill the two P slots; 512 run as two sub-tiles combined at the normalisation
   if (mode == 1) return K == 128 && N2 == 128 && (N1 == 256 || N1 == 512);
-  return K == 128 && N2 == 128 && N1 >= 128 && N1 <= 128 * kMaxChunks && N1 % 128 == 0;
+  return b2b_mlp_supported(K, N1, N2);
 }
 
 cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
@@ -785,7 +485,7 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   CUtensorMap tmX, tmW1, tmW2, tmO;
   const uint64_t M = p.M, K = p.K, N1 = p.N1, N2 = p.N2;
   if (p.batch < 1) p.batch = 1;
-  const uint64_t nb = static_cast<uint64_t>(p.batch);  // dense [batch, rows, cols] tensors (the MLP form has batch = 1)
+  const uint64_t nb = static_cast<uint64_t>(p.batch);  // dense [batch, rows, cols] tensors
   // all boxes are 64 elements x 128 rows
   if (!encode_tmap_bf16_3d(&tmX, X, K, M, nb, K * 2, M * K * 2, 128) ||
       !encode_tmap_bf16_3d(&tmW1, W1, N1, K, nb, N1 * 2, K * N1 * 2, 128) ||
@@ -812,15 +512,13 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   if (max_clusters[di] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    e = cudaFuncSetAttribute(b2b_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
-    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<0>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1>, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di] = n;
@@ -829,10 +527,9 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
-  if (p.mode == 1)
-    return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, 2>, tmX, tmW1, tmW2, tmO, p)
-                       : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, 1>, tmX, tmW1, tmW2, tmO, p);
-  return cudaLaunchKernelEx(&cfg, b2b_pair_kernel<0>, tmX, tmW1, tmW2, tmO, p);
+  if (p.mode != 1) return cudaErrorInvalidValue;  // the MLP forms have kernels of their own
+  return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2>, tmX, tmW1, tmW2, tmO, p)
+                     : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1>, tmX, tmW1, tmW2, tmO, p);
 }
 
 }  // namespace comfuse

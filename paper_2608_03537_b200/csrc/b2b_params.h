@@ -27,7 +27,11 @@ struct B2bParams {
 };
 
 bool b2b_fused_supported(int K, int N1, int N2, int mode);
+// the attention form (b2b_gemm.cu)
 cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
+// the MLP form (GELU, + b2 + X, LayerNorm) with the four stages on warps of their own (b2b_mlp.cu)
+bool b2b_mlp_supported(int K, int N1, int N2);
+cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);
 // the ReLU MLP form with K streamed through the first GEMM (b2b_stream.cu)
 bool b2b_stream_supported(int K, int N1, int N2);
 cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st);

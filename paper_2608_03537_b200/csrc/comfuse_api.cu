@@ -519,7 +519,9 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     if (const char* tp = std::getenv("COMFUSE_TRACE_PTR")) bp.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tp, nullptr, 0));
     if (const char* tf = std::getenv("COMFUSE_TRACE_FLAGS")) bp.trace_flags = std::atoi(tf);
 #endif
-    cudaError_t e = relu_mlp ? launch_b2b_stream(X, W1, W2, bp, st) : launch_b2b_fused(X, W1, W2, bp, st);
+    cudaError_t e = relu_mlp ? launch_b2b_stream(X, W1, W2, bp, st)
+                    : attention ? launch_b2b_fused(X, W1, W2, bp, st)
+                                : launch_b2b_mlp(X, W1, W2, bp, st);
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }
 
