@@ -70,7 +70,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // cluster of exactly two CTAs
   const uint32_t pm = rank & 1u;
-  const uint32_t leader = 0u, peer = rank ^ 1u;
+  const uint32_t leader = 0u;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
   const int total_tiles = p.batch * p.mpairs;
@@ -181,8 +181,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         return ring_addr(ring.stage);
       };
       auto release_slot = [&](int stage) {
-        umma_commit_pair(bar_empty(stage));
-        umma_commit_pair(map_to_cta(bar_empty(stage), peer));
+        umma_commit_pair_both(bar_empty(stage));
       };
       {
         // Software-pipelined over the cluster's tiles: the scores of tile t+1 (ML1) are issued as soon
@@ -209,8 +208,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
                                 wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
             release_slot(wstage);
-            umma_commit_pair(bar_pfull(j));
-            umma_commit_pair(map_to_cta(bar_pfull(j), peer));
+            umma_commit_pair_both(bar_pfull(j));
           }
           release_slot(xs0);
           release_slot(xs1);
@@ -243,12 +241,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               umma_bf16_ss_pair(d_o, (kk < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((kk & 3) * 2), wdesc + static_cast<uint64_t>(kk * 128),
                                 idesc_ml2, (j | kk) != 0 ? 1u : 0u);
             release_slot(wstage);
-            umma_commit_pair(bar_sempty(j));
-            umma_commit_pair(map_to_cta(bar_sempty(j), peer));
+            umma_commit_pair_both(bar_sempty(j));
           }
           if (ok) {
-            umma_commit_pair(bar_ofull(obuf));
-            umma_commit_pair(map_to_cta(bar_ofull(obuf), peer));
+            umma_commit_pair_both(bar_ofull(obuf));
           }
         }
       }

@@ -88,7 +88,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // cluster of exactly two CTAs
   const uint32_t pm = rank & 1u;
-  const uint32_t leader = 0u, peer = rank ^ 1u;
+  const uint32_t leader = 0u;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
   const int KB = (p.K + 63) / 64;   // K blocks of ML1 (the last one zero-filled past K)
@@ -202,8 +202,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         return ring_addr(ring.stage);
       };
       auto release_stage = [&]() {
-        umma_commit_pair(bar_empty(ring.stage));
-        umma_commit_pair(map_to_cta(bar_empty(ring.stage), peer));
+        umma_commit_pair_both(bar_empty(ring.stage));
         ring.advance();
       };
       auto ml1_blocks = [&](uint32_t d_p, int kb0, int kb1) {
@@ -234,11 +233,9 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           umma_bf16_ss_pair(d_o, sdesc, wdesc + static_cast<uint64_t>(k * 128), idesc_ml2, (h | k) != 0 ? 1u : 0u);
         }
         release_stage();
-        umma_commit_pair(bar_sempty);
-        umma_commit_pair(map_to_cta(bar_sempty, peer));
+        umma_commit_pair_both(bar_sempty);
         if (h == NH - 1) {
-          umma_commit_pair(bar_ofull);
-          umma_commit_pair(map_to_cta(bar_ofull, peer));
+          umma_commit_pair_both(bar_ofull);
         }
       };
       if constexpr (LOCK) {
@@ -272,8 +269,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 for (int k = 0; k < 4; ++k)
                   umma_bf16_ss_pair(tmem_base + half * 256, adesc + static_cast<uint64_t>(k * 2),
                                     (half ? bdesc1 : bdesc0) + static_cast<uint64_t>(k * 128), idesc_ml1, (kb | k) != 0 ? 1u : 0u);
-                umma_commit_pair(bar_pfull(half));
-                umma_commit_pair(map_to_cta(bar_pfull(half), peer));
+                umma_commit_pair_both(bar_pfull(half));
               }
             }
             release_stage();
@@ -297,8 +293,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         if (u > 0) ml2(u - 1);
         ml1_blocks(d_p, KBa, KB);
         if (ok) {
-          umma_commit_pair(bar_pfull(slot));
-          umma_commit_pair(map_to_cta(bar_pfull(slot), peer));
+          umma_commit_pair_both(bar_pfull(slot));
         }
       }
       if (!LOCK && nunits > 0 && ok) ml2(nunits - 1);

@@ -158,7 +158,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const uint32_t pm = rank & 1u;       // which row block of the pair
   const uint32_t crank = rank >> 1;    // which column range
   const uint32_t leader = rank & ~1u;  // cluster rank of the CTA that issues the pair's UMMAs
-  const uint32_t peer = rank ^ 1u;
+  const uint16_t pair_mask = static_cast<uint16_t>(3u << leader);  // the pair's two CTAs, for commits that signal both
   constexpr int CLUSTER = 2 * CN;
   const int cluster_id = blockIdx.x / CLUSTER;
   const int num_clusters = gridDim.x / CLUSTER;
@@ -346,13 +346,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 umma_bf16_ss_pair(d_tmem + BNS0, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc1, acc);
             }
             // the stage is free in both CTAs once these UMMAs have read it
-            umma_commit_pair(bar_empty(ring.stage));
-            umma_commit_pair(map_to_cta(bar_empty(ring.stage), peer));
+            umma_commit_pair_both(bar_empty(ring.stage), pair_mask);
             ring.advance();
           }
           if (ok) {
-            umma_commit_pair(bar_tfull(slot));
-            umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
+            umma_commit_pair_both(bar_tfull(slot), pair_mask);
             if (has_res) ring.skip((W / 64 + GPS - 1) / GPS);  // the residual stages belong to the epilogue
           }
         }

@@ -264,9 +264,10 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
 }
 // The same arrival delivered to the barrier at this shared-memory offset in BOTH CTAs of the pair by one instruction
 // (a commit occupies the issuing thread for tens of nanoseconds, so two plain commits per barrier add up on short tiles).
-__device__ __forceinline__ void umma_commit_pair_both(uint32_t bar_local_addr) {
+// `pair_mask` has the bits of the two CTAs' ranks in the cluster: 3 << (rank & ~1) for the pair that holds `rank`.
+__device__ __forceinline__ void umma_commit_pair_both(uint32_t bar_local_addr, uint16_t pair_mask = 3) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar_local_addr),
-               "h"(static_cast<uint16_t>(3))
+               "h"(pair_mask)
                : "memory");
 }
 __device__ __forceinline__ void umma_bf16_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,

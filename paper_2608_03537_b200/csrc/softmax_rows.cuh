@@ -83,7 +83,6 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t pm = cluster_ctarank();  // which 128-row block of the pair; rank 0 issues the UMMAs
-  const uint32_t peer = pm ^ 1u;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
   const int KB = (p.K + 63) >> 6;
@@ -200,13 +199,11 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside A's swizzled row, 2048 bytes in B
             umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
                               (kb | k) != 0 ? 1u : 0u);
-          umma_commit_pair(bar_empty(stage));
-          umma_commit_pair(map_to_cta(bar_empty(stage), peer));
+          umma_commit_pair_both(bar_empty(stage));
           if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit_pair(bar_tfull(slot));
-        umma_commit_pair(map_to_cta(bar_tfull(slot), peer));
+        umma_commit_pair_both(bar_tfull(slot));
       }
       umma_commit_pair(bar_drain);  // nothing may still be writing either CTA's TMEM when it is freed
       mbar_wait<false>(bar_drain, 0, w);
