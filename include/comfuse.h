@@ -118,8 +118,8 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
  * entry point: it exists for callers of this library, not for the method.)
  *
  * Some callers cannot provide the workspace that comfuse_gemm_epilogue(fused = 0) needs, because they cannot
- * allocate device memory where the call happens: code that runs while a stream is being captured or in a latency
- * critical loop where cudaMalloc (which synchronises the device) is not allowed, plug-ins that receive tensors from
+ * allocate device memory where the call happens: code in a latency-critical loop where cudaMalloc (which
+ * synchronises the device) is not allowed, plug-ins that receive tensors from
  * a host framework but have no access to its allocator, or processes whose device memory is handed out entirely by
  * another component.  For them the intermediate bf16 GEMM result is kept in a fixed array of
  * COMFUSE_STATIC_SCRATCH_BYTES that is part of the library's device image; every GPU on which the library is loaded
@@ -130,7 +130,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
  *   - batch * M * N * 2 bytes must fit in COMFUSE_STATIC_SCRATCH_BYTES; a larger problem is rejected with
  *     COMFUSE_ERR_WORKSPACE before anything is launched.
  *   - The first call on each device looks up the array's device address and configures the kernels it launches;
- *     make that first call outside any stream capture.
+ *     that first call should come before any stream capture.  The cached address does not survive cudaDeviceReset.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  Nothing in it
  *     needs clearing (each call overwrites the region it later reads), but two calls whose kernels can overlap on
  *     the GPU -- different streams without an ordering between them -- race on it.  Order such calls on one stream

@@ -230,12 +230,13 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 
 def gemm_epilogue_static_scratch(A, B, Y, kind, *, bias=None, residual=None, gamma=None, beta=None, mask_tensor=None,
-                                 row_max=None, row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, stream=None):
-    """The unfused GEMM -> row-kernel path for callers that cannot allocate a workspace (for instance inside a stream
-    capture, or a plug-in without access to the host framework's allocator): the intermediate lives in a fixed
+                                 row_max=None, row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, flags=0, softcap=0.0,
+                                 stream=None):
+    """The unfused GEMM -> row-kernel path for callers that cannot allocate a workspace (a loop in which cudaMalloc is not
+    allowed, a plug-in without access to the host framework's allocator): the intermediate lives in a fixed
     STATIC_SCRATCH_BYTES array inside the library.  batch*M*N*2 bytes must fit; calls that may overlap on the GPU race
-    on that array; make the first call on a device outside stream capture."""
-    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=False)
+    on that array; the first call on a device sets the array up and should come before any stream capture."""
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=False, flags=flags, softcap=softcap)
     args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
     st = lib().comfuse_gemm_epilogue_static_scratch(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), _stream(stream))
     if st != OK:

@@ -1,7 +1,7 @@
 // comfuse_gemm_epilogue_static_scratch: the unfused GEMM -> row-kernel path for callers that cannot hand the library
-// a workspace because they cannot allocate device memory at the time of the call -- code running inside a stream
-// capture or a real-time loop where cudaMalloc is forbidden, plug-ins that are given tensors but no allocator, or
-// processes whose memory pool is owned by another component.  The intermediate bf16 GEMM result lives in a
+// a workspace because they cannot allocate device memory at the time of the call -- a real-time loop where cudaMalloc
+// is forbidden, plug-ins that are given tensors but no allocator, or processes whose memory pool is owned by another
+// component.  The intermediate bf16 GEMM result lives in a
 // fixed-size array that is part of the loaded module instead.
 #include <cuda_runtime.h>
 
