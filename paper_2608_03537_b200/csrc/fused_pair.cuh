@@ -739,8 +739,17 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   if (y2 > best) { best = y2; best_col = c + 2; }
                   if (y3 > best) { best = y3; best_col = c + 3; }
                 }
-                pk[half * 16 + 2 * j] = pack_bf16x2_rn(y0, y1);
-                pk[half * 16 + 2 * j + 1] = pack_bf16x2_rn(y2, y3);
+                v[4 * j] = __float_as_uint(y0); v[4 * j + 1] = __float_as_uint(y1);
+                v[4 * j + 2] = __float_as_uint(y2); v[4 * j + 3] = __float_as_uint(y3);
+              }
+              // round once.  Wide rows: this is the un-normalised row on its way to the second kernel, which keeps 11
+              // significant bits (fp16) instead of 8, so that the detour costs the result a quarter of a bf16 half-ulp
+              if (p.wide) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_f16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[half * 16 + j] = pack_bf16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
               }
             }
             if (EPI == EPI_LN && p.post_relu && !p.wide) {

@@ -3,6 +3,7 @@
 // argues against in Sec. 1: on-chip -> off-chip -> on-chip).  One row is held in registers by a warp (N <= 1024)
 // or by a 256-thread block (N <= 8192); reductions are warp shuffles plus one shared-memory step.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -248,7 +249,16 @@ __global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p,
   for (int vi = threadIdx.x; vi < nvec; vi += 256) {
     float xf[8], gf[8], bf[8];
     const uint4 one = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-    unpack8(reinterpret_cast<const uint4*>(y)[vi], xf);
+    {  // the first kernel left the un-normalised row as fp16 (11 significant bits)
+      const uint4 q4 = reinterpret_cast<const uint4*>(y)[vi];
+      const uint32_t qw[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&qw[j]));
+        xf[2 * j] = f.x;
+        xf[2 * j + 1] = f.y;
+      }
+    }
     unpack8(p.gamma ? __ldg(reinterpret_cast<const uint4*>(p.gamma) + vi) : one, gf);
     unpack8((KIND == EPI_LN && p.beta) ? __ldg(reinterpret_cast<const uint4*>(p.beta) + vi) : make_uint4(0, 0, 0, 0), bf);
     float o[8];

@@ -31,12 +31,11 @@ def test_b2b_mlp_layernorm(M, N1, affine, fused, cuda_device):
 
 @pytest.mark.parametrize("fused", [True, False])
 def test_config_b2b_mlp_full_size(fused, cuda_device):
-    """c5 at full size: sampled rows against the oracle; over every row, the un-normalised statistics property."""
+    """c5 at full size: every element against the oracle; over every row, the un-normalised statistics property."""
     w = wl.config(4)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     assert torch.isfinite(got["Y"].float()).all().item()
-    rows = wl.sample_rows(w.dims["M"], 512)
-    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c5 fused={fused}")
+    res = P.check_outputs(w, got, P.run_oracle(w), label=f"c5 fused={fused}")
     Y = got["Y"].float()          # gamma = 1, beta = 0: every row has mean ~0 and variance ~1
     assert Y.mean(-1).abs().max().item() < 2e-2
     assert (Y.var(-1, unbiased=False) - 1).abs().max().item() < 3e-2
@@ -92,13 +91,12 @@ def test_b2b_softmax_attention_sharp_and_flat_rows(cuda_device):
     assert np.abs(P.to_f64(got["Y"][1, 128:]) - V1.mean(0)).max() < 2e-3
 
 
-def test_b2b_attention_full_size_sampled(cuda_device):
+def test_b2b_attention_full_size(cuda_device):
     w = wl.config(5)                               # 32 x (4096 x 128 -> 256 -> 128)
     got = P.run_gpu(w, P.dev_tensors(w), fused=True)
     assert torch.isfinite(got["Y"].float()).all().item()
-    rows = wl.sample_rows(w.dims["M"], 64)
-    batches = [0, 13, 31]
-    P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches, label="a1 target attention")
+    for b in range(w.dims["batch"]):               # every element, one batch at a time
+        P.check_outputs(w, got, P.run_oracle(w, batches=[b]), batches=[b], label=f"a1 target attention batch {b}")
 
 
 @pytest.mark.parametrize("fused", [True, False])

@@ -38,14 +38,13 @@ def test_b2b_mlp_relu(M, K, N1, fused, cuda_device):
 
 
 @pytest.mark.parametrize("fused", [True, False])
-def test_dlrm_shape_full_size_sampled(fused, cuda_device):
-    """32768 x (1024 -> 512 -> 128): sampled rows against the oracle, every element finite and non-negative."""
+def test_dlrm_shape_full_size(fused, cuda_device):
+    """32768 x (1024 -> 512 -> 128): every element against the oracle, every element finite and non-negative."""
     w = wl.config(8)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     Y = got["Y"].float()
     assert torch.isfinite(Y).all().item() and (Y >= 0).all().item()
-    rows = wl.sample_rows(w.dims["M"], 512)
-    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"d1 fused={fused}")
+    res = P.check_outputs(w, got, P.run_oracle(w), label=f"d1 fused={fused}")
     print("d1", fused, res)
 
 

@@ -1,6 +1,6 @@
 """GPU parity at the full sizes of the named configurations, in the launch configuration the benchmark times.
-The oracle evaluates a seeded sample of rows (always including both sides of the first and last 128-row block
-boundary) one by one; properties that hold at any size cover the rest of the output."""
+Every output element is compared with the fp64 oracle (the softmax configuration one batch at a time, to bound the
+oracle's memory); properties that need no oracle are checked over the whole output as well."""
 import numpy as np
 import pytest
 import torch
@@ -15,13 +15,24 @@ def _finite_everywhere(Y):
     assert torch.isfinite(Y.float()).all().item(), "some output elements were never written (NaN poison left)"
 
 
+def _unfused_bound(w, got, ref, label):
+    """The in-library unfused baseline rounds the GEMM result to bf16 before the subgraph, i.e. twice in all: an occasional
+    output of magnitude 4 .. 8 lands just above 3e-2.  It is held to 4e-2, with the number of elements above 3e-2 printed
+    and bounded."""
+    over = int((np.abs(P.to_f64(got["Y"]) - ref["Y"]) > P.TOL_NORM_MAX).sum())
+    print(f"{label}: {over} of {ref['Y'].size} elements above 3e-2")
+    assert over <= ref["Y"].size // 100_000
+    return 4e-2
+
+
 @pytest.mark.parametrize("fused", [True, False])
 def test_config_bert_ffn_out_post_norm(fused, cuda_device):
     w = wl.config(1)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     _finite_everywhere(got["Y"])
-    rows = wl.sample_rows(w.dims["M"], 192)
-    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c2 fused={fused}")
+    ref = P.run_oracle(w)
+    res = P.check_outputs(w, got, ref, label=f"c2 fused={fused}",
+                          norm_tol=P.TOL_NORM_MAX if fused else _unfused_bound(w, got, ref, "c2 unfused"))
     # property over every row: undoing the affine step leaves mean ~0 and variance ~1
     g = torch.from_numpy(wl.bf16_bits_to_f32(w.tensors["gamma"])).to(got["Y"].device)
     b = torch.from_numpy(wl.bf16_bits_to_f32(w.tensors["beta"])).to(got["Y"].device)
@@ -36,9 +47,9 @@ def test_config_complex_subgraph(fused, cuda_device):
     w = wl.config(2)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     _finite_everywhere(got["Y"])
-    rows = wl.sample_rows(w.dims["M"], 96)
-    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows), rows=rows, label=f"c3 fused={fused}",
-                          rowmax_tol=5e-3 if fused else 3e-2)
+    ref = P.run_oracle(w)
+    res = P.check_outputs(w, got, ref, label=f"c3 fused={fused}", rowmax_tol=5e-3 if fused else 3e-2,
+                          norm_tol=P.TOL_NORM_MAX if fused else _unfused_bound(w, got, ref, "c3 unfused"))
     # property over every row: the stored row attains its maximum at the reported column, and bf16(row_max) is it
     Y = got["Y"].float()
     ymax = Y.max(-1).values
@@ -53,10 +64,11 @@ def test_config_scaled_causal_softmax(fused, cuda_device):
     w = wl.config(3)
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     _finite_everywhere(got["Y"])
-    batches = [0, 17, 63]
-    rows = wl.sample_rows(w.dims["M"], 96)
-    res = P.check_outputs(w, got, P.run_oracle(w, rows=rows, batches=batches), rows=rows, batches=batches,
-                          label=f"c4 fused={fused}", softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+    res = {"max_abs": 0.0, "mean_abs": 0.0}
+    for b in range(w.dims["batch"]):   # every batch, one at a time (the oracle's fp64 scores of one batch are 34 MB)
+        r = P.check_outputs(w, got, P.run_oracle(w, batches=[b]), batches=[b], label=f"c4 fused={fused} batch {b}",
+                            softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+        res = {"max_abs": max(res["max_abs"], r["max_abs"]), "mean_abs": res["mean_abs"] + r["mean_abs"] / w.dims["batch"]}
     # properties over every row of every batch: strictly upper triangle exactly zero, rows sum to ~1, P[.,0,0] = 1
     Y = got["Y"]
     M = w.dims["M"]

@@ -58,15 +58,21 @@ def test_random_shape_and_operands(seed, cuda_device):
         kw["softmax_tol"] = P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED
     if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
         kw["rowmax_tol"] = 5e-3 if fused else 3e-2
-    if not fused and w.kind != wl.KIND_SCALE_MASK_SOFTMAX:
-        # the unfused baseline normalises the bf16-rounded GEMM result: on outputs of magnitude 4 .. 8 (half-ulp 1.56e-2) an
-        # occasional element lands just above 3e-2 (seen: 3.03e-2); the fused kernels are held to 3e-2
-        kw["norm_tol"] = 4e-2
     ref = P.run_oracle(w)
     if w.kind != wl.KIND_SCALE_MASK_SOFTMAX:
-        # the stated bound assumes outputs below 8 in magnitude (bf16 half-ulp 1.56e-2 on [4, 8)); the RMSNorm of GELU values
-        # without a residual reaches beyond that, where rounding alone is 3.1e-2: there the bound follows the magnitude
-        kw["norm_tol"] = max(kw.get("norm_tol", P.TOL_NORM_MAX), 2.0 ** -7 * float(np.abs(ref["Y"]).max()))
+        # the stated bound (3e-2) assumes outputs below 8 in magnitude (bf16 half-ulp 1.56e-2 on [4, 8)); the RMSNorm of GELU
+        # values without a residual reaches beyond that, where the output rounding alone is 3.1e-2: only there does the
+        # bound follow the magnitude
+        ymax = float(np.abs(ref["Y"]).max())
+        kw["norm_tol"] = P.TOL_NORM_MAX if ymax < 8.0 else max(P.TOL_NORM_MAX, 2.0 ** -7 * ymax)
+        if not fused:
+            # the unfused baseline normalises the bf16-rounded GEMM result, i.e. it rounds twice: an occasional output of
+            # magnitude 4 .. 8 lands just above 3e-2.  It is given 4e-2, and the number of elements above 3e-2 is printed
+            # and bounded so that "an occasional element" stays checkable
+            kw["norm_tol"] = max(kw["norm_tol"], 4e-2)
+            over = int((np.abs(P.to_f64(got["Y"]) - ref["Y"]) > max(P.TOL_NORM_MAX, 2.0 ** -7 * ymax if ymax >= 8.0 else 0.0)).sum())
+            print(f"unfused {w.name}: {over} of {ref['Y'].size} elements above the fused bound")
+            assert over <= max(2, ref["Y"].size // 100_000), over
     P.check_outputs(w, got, ref, label=f"{w.name} fused={fused} {sorted(w.tensors)} {w.scalars}", **kw)
 
 
@@ -99,10 +105,11 @@ def test_random_wide_rows(seed, cuda_device):
         w = wl.complex_subgraph(M, N, K, seed=seed, activation=bool(g.random() < 0.6), residual=bool(g.random() < 0.7))
     got = P.run_gpu(w, P.dev_tensors(w), fused=True)
     ref = P.run_oracle(w)
-    kw = {"norm_tol": max(4e-2, 2.0 ** -7 * float(np.abs(ref["Y"]).max()))}   # the un-normalised row passes through bf16 once
+    # the un-normalised row travels to the second kernel as fp16 (11 significant bits), so this path meets the bounds of
+    # the one-kernel path; beyond magnitude 8 the bound follows the output rounding, as above
+    ymax = float(np.abs(ref["Y"]).max())
+    kw = {"norm_tol": P.TOL_NORM_MAX if ymax < 8.0 else max(P.TOL_NORM_MAX, 2.0 ** -7 * ymax)}
     if w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
-        # two columns whose un-normalised values were each moved by half a bf16 ulp (2^-9 relative) can swap places when they
-        # are closer than 2^-8 |y| g: with |y| up to 8 in rows of 12288+ columns that exceeds 3e-2 in about one row of 50 000
-        # (a CPU emulation of the rounding reproduces the same rows), so the slack follows the magnitude like `norm_tol`
-        kw["rowmax_tol"] = kw["norm_tol"]
+        # the row maximum is taken over values that carry the fp16 rounding of the un-normalised row (2^-11 relative)
+        kw["rowmax_tol"] = max(5e-3, 2.0 ** -10 * ymax)
     P.check_outputs(w, got, ref, label=f"{w.name} wide {sorted(w.tensors)} {w.scalars}", **kw)
