@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     "c2": (70_159_872, "profiles/fused_layernorm_c2_bert_ffn_out.md"),
     "c3": (217_753_600, "profiles/fused_rmsnorm_max_c3_complex_subgraph.md"),
     "c4": (512_653_312, "profiles/softmax_rows_c4_scaled_causal_softmax.md"),
-    "c5": (8_713_216, "profiles/b2b_mlp_c5.md"),
+    "c5": (8_707_328, "profiles/b2b_mlp_c5.md"),
     "a1": (39_041_536, "profiles/b2b_attention_a1_target_attention.md"),
     "a2": (111_826_432, "profiles/b2b_attention_a2_self_attention_512.md"),
     "d1": (71_254_272, "profiles/b2b_stream_d1_dlrm_bottom_mlp.md"),

@@ -2,8 +2,9 @@
  * comfuse.h -- C ABI of the B200 (sm_100a) joint compute-memory fusion library.
  *
  * One bf16 tensor-core GEMM (or a back-to-back pair of GEMMs) whose fp32 result is consumed on-chip by
- * an elementwise/reduction subgraph, without writing the GEMM result to global memory (ComFuse, Sec. 1:
- * "joint compute-memory operator fusion"; Sec. 3: Stage-Stream Execution Model; Sec. 4: B2BGEMM).
+ * an elementwise/reduction subgraph, without writing the GEMM result to global memory (ComFuse: Sec. 1 states
+ * the problem of fusing the compute-bound operator with its memory-bound consumers; Sec. 3 gives the staged
+ * execution model of the epilogue; Sec. 4 the back-to-back GEMM).
  *
  * Conventions for every entry point
  *   - All tensor pointers are DEVICE pointers unless stated otherwise; the caller owns every buffer.
@@ -189,8 +190,11 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
  * computes on `cuda_stream` and range c-2's result is copied out on a second library-owned stream.  `cuda_stream` forks
  * into the two helper streams at the start of the call and joins them at its end, so work enqueued on it afterwards (an
  * event, the next call) is ordered behind the whole call; results are bit for bit those of the unpipelined form.  The
- * helper streams and events are created once per device at first use (COMFUSE_HOST_PIPELINE=0 disables the pipeline).
- * Errors: as comfuse_gemm_epilogue; COMFUSE_ERR_WORKSPACE also when `staging` is NULL or too small. */
+ * helper streams and events are created once per device at first use (COMFUSE_HOST_PIPELINE=0 disables the pipeline);
+ * they serve one call at a time, so host threads that call these forms on the same device take turns enqueueing.
+ * Errors: as comfuse_gemm_epilogue; COMFUSE_ERR_WORKSPACE also when `staging` is NULL or too small.  The description,
+ * the workspace and the staging size are checked before anything is enqueued; an error that a CUDA call reports later
+ * (COMFUSE_ERR_CUDA) can leave copies of this call on the stream, always joined back into `cuda_stream`'s order. */
 #define COMFUSE_HOST_A 1u
 #define COMFUSE_HOST_B 2u
 #define COMFUSE_HOST_RESIDUAL 4u /* args->residual is a host pointer */

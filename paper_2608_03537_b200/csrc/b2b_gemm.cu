@@ -10,6 +10,8 @@
 // CTA pairs (cta_group::2): each CTA holds its own 128 rows of X / S and half (64 columns) of every weight chunk.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "b2b_params.h"
 #include "epilogue_common.cuh"
 #include "fused_pair.cuh"
@@ -492,7 +494,7 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   p.mpairs = (p.mblocks + 1) / 2;
 
   constexpr int kMaxDev = 64;
-  static int max_clusters[kMaxDev] = {0};
+  static std::atomic<int> max_clusters[kMaxDev];  // 0 = kernel not configured yet on that device (set last, released)
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -507,7 +509,8 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
-  if (max_clusters[di] == 0) {
+  int ncl = max_clusters[di].load(std::memory_order_acquire);
+  if (ncl == 0) {
     cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(b2b_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
@@ -517,10 +520,11 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
     e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1>, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
-    max_clusters[di] = n;
+    max_clusters[di].store(n, std::memory_order_release);
+    ncl = n;
   }
   const int tiles = p.batch * p.mpairs;
-  const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
+  const int clusters = tiles < ncl ? tiles : ncl;
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
   if (p.mode != 1) return cudaErrorInvalidValue;  // the MLP forms have kernels of their own

@@ -19,6 +19,8 @@
 // LayerNorm(x) with eps.  The normalised row is staged over the tile's X buffer, idle by then, and stored from there by TMA.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "b2b_params.h"
 #include "fused_pair.cuh"
 #include "host_common.h"
@@ -551,7 +553,7 @@ cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bPar
   p.mpairs = (p.mblocks + 1) / 2;
 
   constexpr int kMaxDev = 64;
-  static int max_clusters[kMaxDev] = {0};
+  static std::atomic<int> max_clusters[kMaxDev];  // 0 = kernel not configured yet on that device (set last, released)
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -566,7 +568,8 @@ cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bPar
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
-  if (max_clusters[di] == 0) {
+  int ncl = max_clusters[di].load(std::memory_order_acquire);
+  if (ncl == 0) {
     cudaError_t e = cudaFuncSetAttribute(b2b_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MlpSmem::BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
@@ -574,10 +577,11 @@ cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bPar
     e = cudaOccupancyMaxActiveClusters(&n, b2b_mlp_kernel, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
-    max_clusters[di] = n;
+    max_clusters[di].store(n, std::memory_order_release);
+    ncl = n;
   }
   const int tiles = p.batch * p.mpairs;
-  const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
+  const int clusters = tiles < ncl ? tiles : ncl;
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
   return cudaLaunchKernelEx(&cfg, b2b_mlp_kernel, tmX, tmW1, tmW2, tmO, p);

@@ -25,6 +25,8 @@
 // 256 W2 rows of a half (in both schedules).
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include <cstdlib>
 
 #include "b2b_params.h"
@@ -456,7 +458,7 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   p.mpairs = (p.mblocks + 1) / 2;
 
   constexpr int kMaxDev = 64;
-  static int max_clusters[kMaxDev] = {0};
+  static std::atomic<int> max_clusters[kMaxDev];  // 0 = kernel not configured yet on that device (set last, released)
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -472,7 +474,8 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
-  if (max_clusters[di] == 0) {
+  int ncl = max_clusters[di].load(std::memory_order_acquire);
+  if (ncl == 0) {
     cudaError_t e = cudaFuncSetAttribute(b2b_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamSmem<false>::BYTES);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(b2b_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, StreamSmem<true>::BYTES);
@@ -484,10 +487,11 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
     cfg.dynamicSmemBytes = lock ? StreamSmem<true>::BYTES : StreamSmem<false>::BYTES;
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
-    max_clusters[di] = n;
+    max_clusters[di].store(n, std::memory_order_release);
+    ncl = n;
   }
   const int tiles = p.mpairs;
-  const int clusters = tiles < max_clusters[di] ? tiles : max_clusters[di];
+  const int clusters = tiles < ncl ? tiles : ncl;
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
   return lock ? cudaLaunchKernelEx(&cfg, b2b_stream_kernel<true>, tmX, tmW1, tmW2, tmO, p)

@@ -21,6 +21,7 @@ std::atomic<uint64_t> g_launches{0};
 std::mutex g_mutex;
 constexpr int kMaxDev = 64;
 DeviceInfo g_dev[kMaxDev];
+std::atomic<bool> g_dev_ready[kMaxDev];  // zero-initialised: false
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -77,9 +78,11 @@ bool programmatic_launch_enabled() {
 const DeviceInfo* current_device_info() {
   int d = -1;
   if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDev) return nullptr;
-  if (g_dev[d].device == d) return &g_dev[d];
+  // g_dev_ready[d] is set (release) after every field of g_dev[d] has been written, so a thread that sees it (acquire)
+  // sees the fields too.  The cached device addresses do not survive cudaDeviceReset.
+  if (g_dev_ready[d].load(std::memory_order_acquire)) return &g_dev[d];
   std::lock_guard<std::mutex> lock(g_mutex);
-  if (g_dev[d].device == d) return &g_dev[d];
+  if (g_dev_ready[d].load(std::memory_order_relaxed)) return &g_dev[d];
   DeviceInfo info;
   if (cudaDeviceGetAttribute(&info.cc_major, cudaDevAttrComputeCapabilityMajor, d) != cudaSuccess) return nullptr;
   if (cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, d) != cudaSuccess) return nullptr;
@@ -91,8 +94,9 @@ const DeviceInfo* current_device_info() {
     }
     info.status_word = static_cast<unsigned int*>(addr);
   }
+  info.device = d;
   g_dev[d] = info;
-  g_dev[d].device = d;
+  g_dev_ready[d].store(true, std::memory_order_release);
   return &g_dev[d];
 }
 

@@ -2,6 +2,7 @@
 // reduce phase of a stage (Sec. 3.1), and the bf16 row-chunk store.
 #pragma once
 
+#include "comfuse.h"
 #include "sm100_primitives.cuh"
 
 namespace comfuse {
@@ -31,9 +32,9 @@ struct MergeByOp {  // (value, unused) under a run-time reduction operator: comf
   __device__ __forceinline__ float2 operator()(float2 a, float, float2 b, float) const {
     float r;
     switch (op) {
-      case 50: r = fmaxf(a.x, b.x); break;  // COMFUSE_OP_RED_MAX
-      case 51: r = fminf(a.x, b.x); break;  // COMFUSE_OP_RED_MIN
-      case 52: r = a.x * b.x; break;        // COMFUSE_OP_RED_PROD
+      case COMFUSE_OP_RED_MAX: r = fmaxf(a.x, b.x); break;
+      case COMFUSE_OP_RED_MIN: r = fminf(a.x, b.x); break;
+      case COMFUSE_OP_RED_PROD: r = a.x * b.x; break;
       default: r = a.x + b.x; break;        // sum, mean
     }
     return make_float2(r, 0.f);

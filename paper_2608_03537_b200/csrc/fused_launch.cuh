@@ -2,6 +2,7 @@
 // non-portable size when above 8), persistent grid sized from the number of clusters the device can hold at once.
 #pragma once
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 
@@ -19,7 +20,7 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream
   if (!dev) return cudaErrorInvalidDevice;
   constexpr int kCluster = 2 * CN;
   constexpr int kMaxDev = 64;
-  static int max_clusters[kMaxDev] = {0};  // 0 = kernel not configured yet on that device
+  static std::atomic<int> max_clusters[kMaxDev];  // 0 = kernel not configured yet on that device (set last, released)
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
 
   p.mpairs = (p.mblocks + 1) / 2;
@@ -40,7 +41,8 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
 
-  if (max_clusters[di] == 0) {
+  int ncl = max_clusters[di].load(std::memory_order_acquire);
+  if (ncl == 0) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     if (kCluster > 8) {
@@ -52,12 +54,13 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, FusedParams p, cudaStream
     e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
-    max_clusters[di] = n;
+    max_clusters[di].store(n, std::memory_order_release);
+    ncl = n;
     if (std::getenv("COMFUSE_VERBOSE"))
       std::fprintf(stderr, "comfuse: kernel epi=%d bns=%d+%d cn=%d stages=%d lock=%d epw=%d: cluster of %d CTAs, %d clusters fit, %d B smem, %d staging boxes/warp\n",
                    EPI, BNS0, BNS1, CN, NSTAGES, LOCK, EPW, kCluster, n, Cfg::SMEM_BYTES, Cfg::YBOXES);
   }
-  const int clusters = p.total_tiles < max_clusters[di] ? p.total_tiles : max_clusters[di];
+  const int clusters = p.total_tiles < ncl ? p.total_tiles : ncl;
   if (clusters <= 0) return cudaSuccess;
   cfg.gridDim = dim3(clusters * kCluster, 1, 1);
   count_launch();

@@ -28,6 +28,7 @@ int pipe_chunks(size_t h2d_bytes) {
 constexpr int kMaxDevPipe = 64;
 struct Pipe {
   bool ready = false;
+  std::mutex use;  // held by a call while it enqueues: the helper streams and events serve one call at a time
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr, copied[kPipeChunks] = {}, computed[kPipeChunks] = {};
 };
@@ -101,6 +102,12 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
   if ((host_mask & COMFUSE_HOST_RESIDUAL) && !(args && args->residual)) return COMFUSE_ERR_INVALID_ARG;
   if (need > 0 && (!staging || staging_bytes < need)) return COMFUSE_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(staging) & 15u) return COMFUSE_ERR_ALIGNMENT;
+  {  // everything that can be checked on the host is checked before the first copy is enqueued
+    size_t ws_all = 0;
+    if (comfuse_workspace_size(desc, &ws_all) != COMFUSE_OK) return COMFUSE_ERR_INVALID_ARG;
+    if (ws_all > 0 && (!workspace || workspace_bytes < ws_all)) return COMFUSE_ERR_WORKSPACE;
+    if (ws_all > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return COMFUSE_ERR_ALIGNMENT;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Extents e = extents_of(desc, host_mask);
   unsigned char* cur = static_cast<unsigned char*>(staging);
@@ -122,6 +129,7 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
                 (host_mask & COMFUSE_HOST_Y) && desc->M >= 2 * rows_per_chunk)
                    ? pipe_for_current_device() : nullptr;
   if (pipe) {
+    std::lock_guard<std::mutex> one_call(pipe->use);  // two host threads must not interleave their use of the events
     unsigned char* sA = cur;
     cur += round_up(e.a);
     unsigned char* sB = cur;
@@ -145,20 +153,27 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
       ws_rows_bytes = ws_all / static_cast<size_t>(desc->M);
       if (ws_all > 0 && (!workspace || workspace_bytes < ws_all)) return COMFUSE_ERR_WORKSPACE;
     }
+    // from here on the helper streams are forked off the caller's stream: whatever happens, they are joined back
+    // (`rejoin`), so that an error return leaves no work of this call outside the caller's stream order
     if (cudaEventRecord(pipe->fork, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
-    if (cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
-    if (cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    auto rejoin = [&](comfuse_status_t status) {
+      const bool ok = cudaEventRecord(pipe->join, pipe->out) == cudaSuccess && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess &&
+                      cudaEventRecord(pipe->join, pipe->in) == cudaSuccess && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess;
+      return (status == COMFUSE_OK && !ok) ? COMFUSE_ERR_CUDA : status;
+    };
+    if (cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess) return rejoin(COMFUSE_ERR_CUDA);
+    if (cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess) return rejoin(COMFUSE_ERR_CUDA);
     int c = 0;
     for (int r0 = 0; r0 < desc->M; r0 += rows_per_chunk, ++c) {
       const int rows = desc->M - r0 < rows_per_chunk ? desc->M - r0 : rows_per_chunk;
       const size_t offA = static_cast<size_t>(r0) * desc->lda * 2, offR = static_cast<size_t>(r0) * desc->ldr * 2,
                    offY = static_cast<size_t>(r0) * desc->ldy * 2;
       if (cudaMemcpyAsync(sA + offA, hA + offA, extent_bytes(1, rows, desc->K, desc->lda, 0), cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       if (host_r && cudaMemcpyAsync(sR + offR, hR + offR, extent_bytes(1, rows, desc->N, desc->ldr, 0), cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       if (cudaEventRecord(pipe->copied[c], pipe->in) != cudaSuccess || cudaStreamWaitEvent(st, pipe->copied[c], 0) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       comfuse_gemm_desc_t dc = *desc;
       dc.M = rows;
       comfuse_epilogue_args_t ac = a;
@@ -167,14 +182,13 @@ extern "C" comfuse_status_t comfuse_gemm_epilogue_host(const comfuse_gemm_desc_t
       if (ac.row_argmax) ac.row_argmax += r0;
       unsigned char* wsc = workspace ? static_cast<unsigned char*>(workspace) + static_cast<size_t>(r0) * ws_rows_bytes : nullptr;
       s = comfuse_gemm_epilogue(&dc, sA + offA, dB, sY + offY, &ac, wsc, wsc ? workspace_bytes - static_cast<size_t>(r0) * ws_rows_bytes : 0, cuda_stream);
-      if (s != COMFUSE_OK) return s;
+      if (s != COMFUSE_OK) return rejoin(s);
       if (cudaEventRecord(pipe->computed[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->out, pipe->computed[c], 0) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       if (cudaMemcpyAsync(hY + offY, sY + offY, extent_bytes(1, rows, desc->N, desc->ldy, 0), cudaMemcpyDeviceToHost, pipe->out) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
     }
-    if (cudaEventRecord(pipe->join, pipe->out) != cudaSuccess || cudaStreamWaitEvent(st, pipe->join, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
-    return COMFUSE_OK;
+    return rejoin(COMFUSE_OK);
   }
   if ((host_mask & COMFUSE_HOST_A) && !stage_in(A, e.a, &dA)) return COMFUSE_ERR_CUDA;
   if ((host_mask & COMFUSE_HOST_B) && !stage_in(B, e.b, &dB)) return COMFUSE_ERR_CUDA;
@@ -208,6 +222,13 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
   if (!X || !O) return COMFUSE_ERR_INVALID_ARG;
   if (!staging || staging_bytes < need) return COMFUSE_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(staging) & 15u) return COMFUSE_ERR_ALIGNMENT;
+  {  // everything that can be checked on the host is checked before the first copy is enqueued
+    size_t ws_all = 0;
+    if (comfuse_b2b_workspace_size(desc, &ws_all) != COMFUSE_OK) return COMFUSE_ERR_INVALID_ARG;
+    if (ws_all > 0 && (!workspace || workspace_bytes < ws_all)) return COMFUSE_ERR_WORKSPACE;
+    if (ws_all > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return COMFUSE_ERR_ALIGNMENT;
+    if (!W1 || !W2) return COMFUSE_ERR_INVALID_ARG;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t nb = static_cast<size_t>(desc->batch);
   const size_t xb = nb * desc->M * desc->K * 2, ob = nb * desc->M * desc->N2 * 2;
@@ -222,6 +243,7 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
   const long long per_chunk = nchunks >= 2 ? ((units + nchunks - 1) / nchunks + grain - 1) / grain * grain : units;
   Pipe* pipe = (nchunks >= 2 && units >= 2 * per_chunk && (!attn || (W1 && W2))) ? pipe_for_current_device() : nullptr;
   if (pipe) {
+    std::lock_guard<std::mutex> one_call(pipe->use);  // two host threads must not interleave their use of the events
     const size_t w1b = nb * desc->K * desc->N1 * 2, w2b = nb * desc->N1 * desc->N2 * 2;
     unsigned char* dW1 = dO + round_up(ob);
     unsigned char* dW2 = dW1 + round_up(w1b);
@@ -232,21 +254,26 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
     // bytes per unit (row or batch) of each per-step tensor
     const size_t ux = static_cast<size_t>(attn ? desc->M : 1) * desc->K * 2, uo = static_cast<size_t>(attn ? desc->M : 1) * desc->N2 * 2;
     const size_t u1 = static_cast<size_t>(desc->K) * desc->N1 * 2, u2 = static_cast<size_t>(desc->N1) * desc->N2 * 2;
-    if (cudaEventRecord(pipe->fork, st) != cudaSuccess || cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess ||
-        cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess)
-      return COMFUSE_ERR_CUDA;
+    if (cudaEventRecord(pipe->fork, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+    auto rejoin = [&](comfuse_status_t status) {  // whatever happens, the helper streams are joined back into the caller's
+      const bool ok = cudaEventRecord(pipe->join, pipe->out) == cudaSuccess && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess &&
+                      cudaEventRecord(pipe->join, pipe->in) == cudaSuccess && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess;
+      return (status == COMFUSE_OK && !ok) ? COMFUSE_ERR_CUDA : status;
+    };
+    if (cudaStreamWaitEvent(pipe->in, pipe->fork, 0) != cudaSuccess || cudaStreamWaitEvent(pipe->out, pipe->fork, 0) != cudaSuccess)
+      return rejoin(COMFUSE_ERR_CUDA);
     int c = 0;
     for (long long u0 = 0; u0 < units; u0 += per_chunk, ++c) {
       const long long n = units - u0 < per_chunk ? units - u0 : per_chunk;
       const unsigned char* hX = static_cast<const unsigned char*>(X) + u0 * ux;
-      if (cudaMemcpyAsync(dX + u0 * ux, hX, n * ux, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess) return COMFUSE_ERR_CUDA;
+      if (cudaMemcpyAsync(dX + u0 * ux, hX, n * ux, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess) return rejoin(COMFUSE_ERR_CUDA);
       if (attn) {
         if (cudaMemcpyAsync(dW1 + u0 * u1, static_cast<const unsigned char*>(W1) + u0 * u1, n * u1, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess ||
             cudaMemcpyAsync(dW2 + u0 * u2, static_cast<const unsigned char*>(W2) + u0 * u2, n * u2, cudaMemcpyHostToDevice, pipe->in) != cudaSuccess)
-          return COMFUSE_ERR_CUDA;
+          return rejoin(COMFUSE_ERR_CUDA);
       }
       if (cudaEventRecord(pipe->copied[c], pipe->in) != cudaSuccess || cudaStreamWaitEvent(st, pipe->copied[c], 0) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       comfuse_b2b_desc_t dc = *desc;
       if (attn) dc.batch = static_cast<int32_t>(n);
       else dc.M = static_cast<int32_t>(n);
@@ -254,14 +281,13 @@ extern "C" comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc
       s = comfuse_b2b_gemm(&dc, dX + u0 * ux, attn ? static_cast<const void*>(dW1 + u0 * u1) : W1, b1,
                            attn ? static_cast<const void*>(dW2 + u0 * u2) : W2, b2, gamma, beta, dO + u0 * uo, wsc,
                            wsc ? workspace_bytes - u0 * ws_unit : 0, cuda_stream);
-      if (s != COMFUSE_OK) return s;
+      if (s != COMFUSE_OK) return rejoin(s);
       if (cudaEventRecord(pipe->computed[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->out, pipe->computed[c], 0) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
       if (cudaMemcpyAsync(static_cast<unsigned char*>(O) + u0 * uo, dO + u0 * uo, n * uo, cudaMemcpyDeviceToHost, pipe->out) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
+        return rejoin(COMFUSE_ERR_CUDA);
     }
-    if (cudaEventRecord(pipe->join, pipe->out) != cudaSuccess || cudaStreamWaitEvent(st, pipe->join, 0) != cudaSuccess) return COMFUSE_ERR_CUDA;
-    return COMFUSE_OK;
+    return rejoin(COMFUSE_OK);
   }
   if (cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
   if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION) {  // W1 (keys) and W2 (values) are host pointers as well

@@ -1,4 +1,5 @@
 // Host-side launch of the short-K row-softmax kernel (pairs of CTAs, persistent grid).
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 
@@ -16,7 +17,7 @@ cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_
   const DeviceInfo* dev = current_device_info();
   if (!dev) return cudaErrorInvalidDevice;
   constexpr int kMaxDev = 64;
-  static int max_clusters[kMaxDev] = {0};  // 0 = kernel not configured yet on that device
+  static std::atomic<int> max_clusters[kMaxDev];  // 0 = kernel not configured yet on that device (set last, released)
   const int di = dev->device < kMaxDev ? dev->device : kMaxDev - 1;
 
   p.mpairs = (p.mblocks + 1) / 2;
@@ -37,7 +38,8 @@ cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
 
-  if (max_clusters[di] == 0) {
+  int ncl = max_clusters[di].load(std::memory_order_acquire);
+  if (ncl == 0) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
@@ -45,11 +47,12 @@ cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_
     e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
-    max_clusters[di] = n;
+    max_clusters[di].store(n, std::memory_order_release);
+    ncl = n;
     if (std::getenv("COMFUSE_VERBOSE"))
       std::fprintf(stderr, "comfuse: row-softmax kernel: %d pairs fit, %d B smem\n", n, Cfg::SMEM_BYTES);
   }
-  const int clusters = p.total_tiles < max_clusters[di] ? p.total_tiles : max_clusters[di];
+  const int clusters = p.total_tiles < ncl ? p.total_tiles : ncl;
   if (clusters <= 0) return cudaSuccess;
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
