@@ -102,12 +102,18 @@ typedef struct {
   int32_t* row_argmax;
 } comfuse_epilogue_args_t;
 
-/* Bytes of caller-provided workspace the described call needs.  Fused calls need none, except LayerNorm / RMSNorm rows
- * wider than the largest cluster can hold on-chip (N > 4096; supported for N a multiple of 4096 up to 65536).  Those run as
- * two kernels: the fused kernel finishes stage 1 per 4096-column block, stores the un-normalised row (rounded to bf16) in
- * Y and one partial statistic per row and block in the workspace (batch * M * N/4096 * 8 bytes); a second kernel merges the
- * partials and rescales the row in place (the un-normalised values are materialised because they no longer fit on-chip,
- * Sec. 2.2).  Their results carry one extra bf16 rounding, like those of the unfused path. */
+/* Bytes of caller-provided workspace the described call can use.  Most fused calls need none.  Two cases of the LayerNorm /
+ * RMSNorm kinds run as TWO kernels and report batch * M * (N / block) * 8 bytes: the fused kernel finishes stage 1 per
+ * column block, stores the un-normalised row in Y as fp16 (11 significant bits) and one partial statistic per row and
+ * block in the workspace; a second kernel merges the partials and rescales the row in place to bf16.
+ *   - Rows wider than the largest cluster can hold on-chip (N > 4096; supported for N a multiple of 4096 up to 65536,
+ *     block = 4096): the un-normalised values are materialised because they no longer fit (Sec. 2.2).  The workspace is
+ *     required.
+ *   - Rows of 2048 .. 4096 columns (a multiple of 256) behind a long contraction (K >= 1024), block = 256: measured faster
+ *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
+ *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
+ *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.
+ * The results of both forms meet the same tolerances as the one-kernel path. */
 comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes);
 
 /* GEMM -> subgraph (Sec. 3).  A, B inputs; Y output [batch, M, N] bf16, rounded once, at the store. */

@@ -75,6 +75,21 @@ bool programmatic_launch_enabled() {
   return on;
 }
 
+int split_row_block(int epi, int N, int K) {
+  // COMFUSE_SPLIT_BLOCK=<width> forces the two-kernel form with that block width where N is a multiple of it (0 = never)
+  static const int forced = [] {
+    const char* e = std::getenv("COMFUSE_SPLIT_BLOCK");
+    return e ? std::atoi(e) : -1;
+  }();
+  (void)epi;
+  if (forced >= 0) return (forced > 0 && N > forced && N % forced == 0) ? forced : 0;
+  // Measured (8192 rows; on-chip / two kernels with 256-column blocks, us): N = 4096: K = 4096 242 / 212, K = 1024 101 / 87,
+  // K = 256 64 / 62 (LayerNorm 57 / 66); N = 2048: K = 4096 147 / 118, K = 1024 59 / 55; N = 1024, K = 4096: 55 / 69.
+  // The clusters of 16 and 8 CTAs that hold rows of 4096 and 2048 columns fill 112 and 120 of the 148 SMs and cannot overlap
+  // a tile's epilogue with the next MainLoop; the 256-column tiles of the two-kernel form can, on every SM.
+  return (N >= 2048 && N % 256 == 0 && K >= 1024) ? 256 : 0;
+}
+
 const DeviceInfo* current_device_info() {
   int d = -1;
   if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDev) return nullptr;
@@ -172,14 +187,15 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
   return COMFUSE_OK;
 }
 
-// Does a fused instantiation exist for this description?
-comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d) {
+// Does a fused instantiation exist for this description?  `on_chip_only`: without the two-kernel form.
+comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only = false) {
   if (d->mask == COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
   p.M = d->M;
   p.N = d->N;
   p.K = d->K;
-  p.wide = wide_row_blocks(kind_to_epi(d->kind), d->N) > 0;
+  p.wide_block = on_chip_only ? 0 : wide_row_block(kind_to_epi(d->kind), d->N, d->K);
+  p.wide = p.wide_block > 0;
   GemmMaps dummy;
   std::memset(&dummy, 0, sizeof(dummy));
   cudaError_t e = cudaErrorInvalidValue;
@@ -309,7 +325,7 @@ comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t*
     s = fused_supported(desc);
     if (s != COMFUSE_OK) return s;
     // rows wider than one cluster: one partial statistic (8 bytes) per row and 4096-column block
-    *bytes = static_cast<size_t>(wide_row_blocks(kind_to_epi(desc->kind), desc->N)) * desc->batch * desc->M * sizeof(float2);
+    *bytes = static_cast<size_t>(wide_row_blocks(kind_to_epi(desc->kind), desc->N, desc->K)) * desc->batch * desc->M * sizeof(float2);
   } else {
     if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
     *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
@@ -340,6 +356,11 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   size_t need = 0;
   s = comfuse_workspace_size(desc, &need);
   if (s != COMFUSE_OK) return s;
+  // For rows that fit a cluster (N <= 4096) the two-kernel form is an optimisation, not a need: a fused call that brings no
+  // (or too small a) workspace keeps the row on chip instead of being refused.
+  const bool split_optional = desc->fused && desc->N <= kWideRowBlock && need > 0 && fused_supported(desc, true) == COMFUSE_OK;
+  const bool have_ws = workspace && workspace_bytes >= need && aligned16(workspace);
+  if (split_optional && !have_ws) need = 0;
   if (need > 0 && (!workspace || workspace_bytes < need)) return COMFUSE_ERR_WORKSPACE;
   if (need > 0 && !aligned16(workspace)) return COMFUSE_ERR_ALIGNMENT;
 
@@ -390,8 +411,9 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
     p.Y = static_cast<uint16_t*>(Y);
     p.ldy = desc->ldy; p.batch_stride_y = bsy;
     p.row_max = a.row_max; p.row_argmax = a.row_argmax;
-    const int wide_blocks = wide_row_blocks(epi, desc->N);
-    if (wide_blocks) {  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace
+    const int wide_blocks = need > 0 ? wide_row_blocks(epi, desc->N, desc->K) : 0;
+    if (wide_blocks) {
+      p.wide_block = wide_row_block(epi, desc->N, desc->K);  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace
       p.wide = 1;
       p.nblocks = wide_blocks;
       p.wide_partials = static_cast<float2*>(workspace);

@@ -8,8 +8,8 @@ cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, c
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_LN, b0, b1, cn, nst, lock>(maps, p, st);
   // Two sub-tiles advance in lock step (lock = 1): the A tile is fetched once per K block for both.
-  // Wide rows (p.wide): every cluster covers one 4096-column block of the row, p.nblocks blocks per row.
-  switch (p.wide ? kWideRowBlock : p.N) {
+  // Two-kernel form (p.wide): every cluster covers one p.wide_block-column block of the row, p.nblocks blocks per row.
+  switch (p.wide ? p.wide_block : p.N) {
     COMFUSE_CASE(256, 256, 0, 1, 5, 0)
     COMFUSE_CASE(512, 256, 256, 1, 3, 1)
     COMFUSE_CASE(768, 256, 128, 2, 4, 1)

@@ -165,8 +165,9 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int KB = (p.K + 63) >> 6;
   const bool has_res = (EPI == EPI_LN || kIsRms || EPI == EPI_PROGRAM) && p.residual != nullptr;
   // The last tile's output boxes may be staged in the circular buffer only if nothing is still arriving there when they
-  // are written: a stage program that stores in its first pass does so while the residual boxes are still coming in.
-  const bool ring_idle_at_store = !(EPI == EPI_PROGRAM && has_res && p.program.terminal_pass == 0);
+  // are written: a stage program that stores in its first pass, and the two-kernel form, which stores in stage 1, do so
+  // while the residual boxes are still coming in.
+  const bool ring_idle_at_store = !(EPI == EPI_PROGRAM && has_res && p.program.terminal_pass == 0) && !(p.wide && has_res);
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 
@@ -617,6 +618,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
               for (int j = 0; j < 32; ++j) r32[j] = 0u;
             }
+            uint32_t pkw[32];  // two-kernel form: the group's un-normalised values as fp16 pairs
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               const int lc = lsub + g * 64 + half * 32;
@@ -674,10 +676,19 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 const float q0 = q01.x, q1 = q01.y, q2 = q23.x, q3 = q23.y;
                 part.x += (q0 + q1) + (q2 + q3);
               }
-              tmem_st_32cols(taddr + g * 64 + half * 32, v);
+              if (p.wide) {
+                // two-kernel form: x leaves the chip here, once, as fp16 (11 significant bits: the detour costs the result
+                // a quarter of a bf16 half-ulp); the second kernel normalises it.  No write-back, no stage 2.
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pkw[half * 16 + j] = pack_f16x2_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              } else {
+                tmem_st_32cols(taddr + g * 64 + half * 32, v);
+              }
             }
+            if (p.wide) store_box(pkw);
             COMFUSE_TRACE_POINT();
           }
+          if (p.wide) release_accumulator(sub);
         }
         tmem_st_wait();
         COMFUSE_TRACE_POINT();
@@ -696,9 +707,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const float mu = (EPI == EPI_LN && !p.wide) ? tot.x : 0.f;
         const float sq = EPI == EPI_LN ? tot.y : tot.x;
         const float rstd = p.wide ? 1.f : rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
-        if (p.wide && crank == 0 && h == 0 && valid) {
-          const int nb = (ncta0 / (CN * BN));
-          p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
+        if (p.wide) {
+          if (crank == 0 && h == 0 && valid) {
+            const int nb = (ncta0 / (CN * BN));
+            p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
+          }
+          continue;  // the row is finished by the second kernel
         }
         // ---------------- stage 2 (PostOp): normalise the resident x, round once, store
         float best = -INFINITY;

@@ -110,6 +110,7 @@ struct FusedParams {
   // column block only, stores the un-normalised values and writes the block's partial statistic of each row to
   // wide_partials[(batch * M + row) * nblocks + block]; a second kernel merges the partials and rescales in place.
   int wide;
+  int wide_block;   // columns per block of the two-kernel form (the instantiation that runs each block)
   float2* wide_partials;
   // Cross-CTA aggregation of the row statistics (Sec. 3.1): 0 = all-to-all (every CTA sends its partial to every peer),
   // 1 = leader-follower (partials go to column range 0, which merges and sends the result back).  Same merge order,

@@ -49,8 +49,20 @@ cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cud
 // Rows wider than the largest cluster (16 CTAs x 256 columns): LayerNorm / RMSNorm kinds run per 4096-column block and a
 // second kernel merges the blocks' statistics (the wide-row fallback).  Returns the number of blocks, 0 = not a wide row.
 constexpr int kWideRowBlock = 4096;
-inline int wide_row_blocks(int epi, int N) {
-  return ((epi == EPI_LN || epi == EPI_RMS_MAX) && N > kWideRowBlock && N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? N / kWideRowBlock : 0;
+// The same two-kernel form for rows that WOULD fit a cluster (N <= 4096), cut into narrower column blocks: clusters of 16
+// CTAs occupy 112 of the 148 SMs and leave tensor memory no room to overlap a tile's epilogue with the next MainLoop, so
+// for long K the detour through one fp16 copy of the row can be the faster path.  `split_row_block` = the block width
+// chosen for (epi, N, K), 0 = keep the row on chip.
+int split_row_block(int epi, int N, int K);
+// column block width of the two-kernel form (0 = one kernel) and the number of blocks per row
+inline int wide_row_block(int epi, int N, int K) {
+  if (epi != EPI_LN && epi != EPI_RMS_MAX) return 0;
+  if (N > kWideRowBlock) return (N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? kWideRowBlock : 0;
+  return split_row_block(epi, N, K);
+}
+inline int wide_row_blocks(int epi, int N, int K) {
+  const int w = wide_row_block(epi, N, K);
+  return w ? N / w : 0;
 }
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).
