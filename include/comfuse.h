@@ -63,8 +63,9 @@ typedef enum {
 typedef enum {
   COMFUSE_MASK_NONE = 0,
   COMFUSE_MASK_CAUSAL = 1,   /* 0 where column <= row, -inf elsewhere; requires M == N            */
-  COMFUSE_MASK_ADDITIVE = 2  /* bf16 [M, N] tensor (ld = N) added to the scaled scores, shared by all
-                                batches; may hold -inf; unfused path only                         */
+  COMFUSE_MASK_ADDITIVE = 2  /* bf16 [M, N] tensor (ld = N) added to the scaled (and soft-capped) scores,
+                                shared by all batches; may hold -inf: such entries give exact zeros, a
+                                row with nothing else gives a row of zeros                        */
 } comfuse_mask_t;
 
 typedef struct {

@@ -189,7 +189,6 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
 
 // Does a fused instantiation exist for this description?  `on_chip_only`: without the two-kernel form.
 comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only = false) {
-  if (d->mask == COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
   p.M = d->M;
   p.N = d->N;
@@ -411,6 +410,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
     p.Y = static_cast<uint16_t*>(Y);
     p.ldy = desc->ldy; p.batch_stride_y = bsy;
     p.row_max = a.row_max; p.row_argmax = a.row_argmax;
+    p.mask = desc->mask == COMFUSE_MASK_ADDITIVE ? static_cast<const uint16_t*>(a.mask) : nullptr;
     const int wide_blocks = need > 0 ? wide_row_blocks(epi, desc->N, desc->K) : 0;
     if (wide_blocks) {
       p.wide_block = wide_row_block(epi, desc->N, desc->K);  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace

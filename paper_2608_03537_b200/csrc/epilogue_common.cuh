@@ -134,6 +134,20 @@ __device__ __forceinline__ float2 cluster_row_reduce(float2 mine, float per_thre
   return acc;
 }
 
+// 32 consecutive values of one row of an additive mask (bf16, the segment starts on a 16-byte boundary), as log2-domain
+// addends: m * log2(e); -inf stays -inf.  `valid` = how many of the 32 columns exist (the rest, and every column of a row
+// that does not exist, read as 0: those scores are dropped by the caller's own bounds).
+__device__ __forceinline__ void load_mask_log2_32(const uint16_t* seg, int valid, float2 (&m2)[16]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 q = make_uint4(0u, 0u, 0u, 0u);
+    if (8 * i < valid) q = __ldg(reinterpret_cast<const uint4*>(seg) + i);
+    const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) m2[4 * i + k] = mul2(bf16x2_to_f2(w4[k]), splat2(1.4426950408889634f));
+  }
+}
+
 __device__ __forceinline__ void store_chunk_bf16(uint16_t* dst, const uint32_t (&pk)[16]) {
   uint4* d = reinterpret_cast<uint4*>(dst);
 #pragma unroll

@@ -1163,6 +1163,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const bool capped = p.softcap > 0.f;
         const SoftcapLog2 cap_fn(p.alpha, capped ? p.softcap : 1.f);
         const float sc = capped ? 1.f : p.alpha * 1.4426950408889634f;
+        const bool additive = p.mask != nullptr;  // additive mask tensor, applied behind the scale / soft-cap
         // fragment classification under the causal mask, uniform over the warp's 32 rows so that the warp-wide TMEM
         // loads stay convergent: 2 = all live, 1 = crosses the diagonal, 0 = all masked
         const int wrow0 = m0 + q * 32;
@@ -1189,16 +1190,33 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
               }
               float m0v = -INFINITY, m1v = -INFINITY;
+              if (additive) {
+                // a full-tensor operand of the epilogue (Sec. 5.2): t = score + mask, written back over the accumulator so
+                // that pass B finds it there
+                float2 m2[16];
+                load_mask_log2_32(p.mask + static_cast<long long>(grow) * p.N + col0, valid ? 32 : 0, m2);
 #pragma unroll
-              for (int j = 0; j < 32; j += 2) {
-                const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
-                if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
-                if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+                for (int j = 0; j < 16; ++j) {
+                  const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), m2[j]);
+                  v[2 * j] = __float_as_uint(t01.x);
+                  v[2 * j + 1] = __float_as_uint(t01.y);
+                  if (st == 2 || col0 + 2 * j <= grow) m0v = fmaxf(m0v, t01.x);
+                  if (st == 2 || col0 + 2 * j + 1 <= grow) m1v = fmaxf(m1v, t01.y);
+                }
+                tmem_st_32cols(tmem_of(sub) + g * 64 + half * 32, v);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                  const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
+                  if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
+                  if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+                }
               }
               mloc = fmaxf(mloc, fmaxf(m0v, m1v));
             }
           }
         }
+        if (additive) tmem_st_wait();
         COMFUSE_TRACE_POINT();
         // ---------------- pass B: e = 2^(t - mloc), thread-local sum, e written back over the scores
         float lloc = 0.f;
@@ -1216,14 +1234,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (st == 0) continue;
               uint32_t v[32];
               tmem_ld_32cols(tmem_of(sub) + g * 64 + half * 32, v);
-              if (capped) {
+              if (capped && !additive) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
               }
               float s0 = 0.f, s1 = 0.f;
+              const float scb = additive ? 1.f : sc;  // with a mask tensor pass A has left t itself in the accumulator
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
-                const float2 t01 = fma2(f2_from_bits(v[j], v[j + 1]), splat2(sc), splat2(-msub));
+                const float2 t01 = fma2(f2_from_bits(v[j], v[j + 1]), splat2(scb), splat2(-msub));
                 float e0 = ex2_approx(t01.x);
                 float e1 = ex2_approx(t01.y);
                 if (st != 2) {

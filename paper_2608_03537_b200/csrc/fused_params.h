@@ -109,6 +109,7 @@ struct FusedParams {
   // Rows wider than one cluster (nblocks > 1 with a normalising epilogue): every cluster finishes stage 1 for its
   // column block only, stores the un-normalised values and writes the block's partial statistic of each row to
   // wide_partials[(batch * M + row) * nblocks + block]; a second kernel merges the partials and rescales in place.
+  const uint16_t* mask;  // softmax kinds: additive bf16 mask [M, N] (ld = N), shared by all batches, or null
   int wide;
   int wide_block;   // columns per block of the two-kernel form (the instantiation that runs each block)
   float2* wide_partials;

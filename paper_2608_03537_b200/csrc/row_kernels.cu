@@ -213,14 +213,27 @@ __global__ void __launch_bounds__(256) row_epilogue_kernel(const RowParams p) {
   }
 }
 
-// Second kernel of the wide-row path: the fused kernel stored the un-normalised x (bf16) in Y and one partial statistic
-// per row and column block; merge the partials in block order, rescale the row in place, and (RMSNorm kind) take the row
-// maximum / lowest argmax of the normalised values.  One block per row.
+// Second kernel of the two-kernel form: the fused kernel stored the un-normalised x (fp16, 11 significant bits) in Y and
+// one partial statistic per row and column block; merge the partials in block order, rescale the row in place to bf16, and
+// (RMSNorm kind) take the row maximum / lowest arg max of the normalised values.  One WARP per row: a lane keeps up to
+// eight 16-byte loads in flight and the row reduce is a shuffle, so nothing waits on a block barrier.
+__device__ __forceinline__ void unpack8_f16(const uint4 q4, float (&xf)[8]) {
+  const uint32_t qw[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&qw[j]));
+    xf[2 * j] = f.x;
+    xf[2 * j + 1] = f.y;
+  }
+}
+
 template <int KIND>
-__global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p, const float2* partials, int nblocks) {
-  __shared__ float s_red[8];
-  __shared__ int s_idx[8];
-  const long long r = blockIdx.x;  // row over batch * M
+__global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p, const float2* partials, int nblocks, long long rows) {
+  // launched with programmatic stream serialization: everything above this line may overlap the first kernel's tail
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int lane = threadIdx.x & 31;
+  const long long r = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);  // row over batch * M
+  if (r >= rows) return;
   const int b = static_cast<int>(r / p.M);
   const int i = static_cast<int>(r - static_cast<long long>(b) * p.M);
   uint16_t* y = p.Y + static_cast<long long>(b) * p.batch_stride_y + static_cast<long long>(i) * p.ldy;
@@ -246,37 +259,38 @@ __global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p,
   float best = -INFINITY;
   int best_col = 0x7FFFFFFF;
   const int nvec = p.N >> 3;
-  for (int vi = threadIdx.x; vi < nvec; vi += 256) {
-    float xf[8], gf[8], bf[8];
-    const uint4 one = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
-    {  // the first kernel left the un-normalised row as fp16 (11 significant bits)
-      const uint4 q4 = reinterpret_cast<const uint4*>(y)[vi];
-      const uint32_t qw[4] = {q4.x, q4.y, q4.z, q4.w};
+  const uint4 one = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+  for (int v0 = 0; v0 < nvec; v0 += 32 * 8) {
+    uint4 xq[8];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&qw[j]));
-        xf[2 * j] = f.x;
-        xf[2 * j + 1] = f.y;
-      }
+    for (int u = 0; u < 8; ++u) {
+      const int vi = v0 + u * 32 + lane;
+      if (vi < nvec) xq[u] = __ldcs(reinterpret_cast<const uint4*>(y) + vi);  // read once: streaming
     }
-    unpack8(p.gamma ? __ldg(reinterpret_cast<const uint4*>(p.gamma) + vi) : one, gf);
-    unpack8((KIND == EPI_LN && p.beta) ? __ldg(reinterpret_cast<const uint4*>(p.beta) + vi) : make_uint4(0, 0, 0, 0), bf);
-    float o[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if constexpr (KIND == EPI_LN) {
-        o[j] = fmaf((xf[j] - mu) * rstd, gf[j], bf[j]);
-        if (p.post_relu) o[j] = fmaxf(o[j], 0.f);
-      } else {
-        o[j] = xf[j] * rstd * gf[j];
-        if (o[j] > best) { best = o[j]; best_col = vi * 8 + j; }
+    for (int u = 0; u < 8; ++u) {
+      const int vi = v0 + u * 32 + lane;
+      if (vi >= nvec) continue;
+      float xf[8], gf[8], bf[8], o[8];
+      unpack8_f16(xq[u], xf);
+      unpack8(p.gamma ? __ldg(reinterpret_cast<const uint4*>(p.gamma) + vi) : one, gf);
+      unpack8((KIND == EPI_LN && p.beta) ? __ldg(reinterpret_cast<const uint4*>(p.beta) + vi) : make_uint4(0, 0, 0, 0), bf);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if constexpr (KIND == EPI_LN) {
+          o[j] = fmaf((xf[j] - mu) * rstd, gf[j], bf[j]);
+          if (p.post_relu) o[j] = fmaxf(o[j], 0.f);
+        } else {
+          o[j] = xf[j] * rstd * gf[j];
+          if (o[j] > best) { best = o[j]; best_col = vi * 8 + j; }
+        }
       }
+      reinterpret_cast<uint4*>(y)[vi] = make_uint4(pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
     }
-    reinterpret_cast<uint4*>(y)[vi] = make_uint4(pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
   }
   if constexpr (KIND == EPI_RMS_MAX) {
-    row_argmax_reduce<256>(best, best_col, s_red, s_idx);
-    if (threadIdx.x == 0) {
+    row_argmax_reduce<32>(best, best_col, nullptr, nullptr);
+    if (lane == 0) {
       p.row_max[r] = best;
       p.row_argmax[r] = best_col;
     }
@@ -331,12 +345,20 @@ cudaError_t launch_row_epilogue(int kind, const RowParams& p, cudaStream_t st) {
 }
 
 cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, cudaStream_t st) {
-  const unsigned rows = static_cast<unsigned>(static_cast<long long>(p.batch) * p.M);
+  const long long rows = static_cast<long long>(p.batch) * p.M;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.gridDim = dim3(static_cast<unsigned>((rows + 7) / 8), 1, 1);  // eight rows (warps) per block
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // its launch overlaps the first kernel's tail
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = programmatic_launch_enabled() ? 1 : 0;
   count_launch();
-  if (kind == EPI_LN) wide_row_finish_kernel<EPI_LN><<<rows, 256, 0, st>>>(p, partials, nblocks);
-  else if (kind == EPI_RMS_MAX) wide_row_finish_kernel<EPI_RMS_MAX><<<rows, 256, 0, st>>>(p, partials, nblocks);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (kind == EPI_LN) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_LN>, p, partials, nblocks, rows);
+  if (kind == EPI_RMS_MAX) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_RMS_MAX>, p, partials, nblocks, rows);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_bias_gelu(uint16_t* P, const uint16_t* bias, long long rows, int n, cudaStream_t st) {

@@ -21,6 +21,7 @@
 // issues the TMA stores of the staged boxes.  Every wait is bounded.
 #pragma once
 
+#include "epilogue_common.cuh"
 #include "fused_params.h"
 #include "sm100_primitives.cuh"
 
@@ -286,6 +287,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool capped = p.softcap > 0.f;
     const SoftcapLog2 cap_fn(p.alpha, capped ? p.softcap : 1.f);
     const float sc = capped ? 1.f : p.alpha * 1.4426950408889634f;
+    const bool additive = p.mask != nullptr;  // additive mask tensor, applied behind the scale / soft-cap
     constexpr uint32_t poly_pairs = Cfg::POLY_PAIRS;
 
 #ifdef COMFUSE_TRACE
@@ -349,8 +351,15 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
               }
               float2 tv[16];
+              if (additive) {  // a full-tensor operand of the epilogue (Sec. 5.2): this thread's 32 mask values from global memory
+                float2 m2[16];
+                load_mask_log2_32(p.mask + static_cast<long long>(grow) * p.N + col0, grow < p.M ? p.N - col0 : 0, m2);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) tv[j] = mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc));
+                for (int j = 0; j < 16; ++j) tv[j] = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), m2[j]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) tv[j] = mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc));
+              }
               if (st != 2) {  // the fragment crosses the diagonal (or the end of the row): rare, kept out of the main path
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -365,7 +374,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 mx1 = max3(mx1, tv[j + 1].x, tv[j + 1].y);
               }
               const float m_new = fmaxf(mx0, mx1);
-              if (st == 2 || m_new != -INFINITY) {  // else every column seen so far is masked for this row
+              if ((st == 2 && !additive) || m_new != -INFINITY) {  // else every column seen so far is masked for this row
                 float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
                 const float2 neg_m = splat2(-m_new);
 #pragma unroll
@@ -398,10 +407,20 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                   for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(cap_fn(__uint_as_float(v[j])));
                 }
                 float2 ev[16];
+                if (additive) {
+                  float2 m2[16];
+                  load_mask_log2_32(p.mask + static_cast<long long>(grow) * p.N + col0, grow < p.M ? p.N - col0 : 0, m2);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), splat2(-off));
-                  ev[j] = ((poly_pairs >> j) & 1u) ? ex2_poly2(t01) : make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
+                  for (int j = 0; j < 16; ++j) {  // (a masked score is -inf, and so is -inf - off: its probability is an exact zero)
+                    const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), add2(m2[j], splat2(-off)));
+                    ev[j] = make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
+                  }
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) {
+                    const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), splat2(-off));
+                    ev[j] = ((poly_pairs >> j) & 1u) ? ex2_poly2(t01) : make_float2(ex2_approx(t01.x), ex2_approx(t01.y));
+                  }
                 }
                 if (st != 2) {  // crosses the diagonal (or the end of the row)
 #pragma unroll

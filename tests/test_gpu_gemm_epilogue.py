@@ -187,19 +187,39 @@ def test_softmax_large_scores_do_not_overflow(cuda_device):
     P.check_outputs(w, got, P.run_oracle(w), label="softmax large scores")
 
 
-def test_softmax_additive_mask_unfused_with_fully_masked_row(cuda_device):
-    """The additive-mask variant (unfused path): -inf entries give exact zeros; a fully masked row gives zeros."""
-    batch, M, N, K = 2, 96, 256, 64
-    w = wl.scaled_masked_softmax(batch, M, N, K, seed=31, causal=False)
-    g = np.random.default_rng(0)
+def _additive_mask(M, N, seed, dead_rows=(5,)):
+    """A mask tensor with moderate finite entries, 30 % of -inf, and whole rows of -inf."""
+    g = np.random.default_rng(seed)
     mask = (g.standard_normal((M, N)) * 0.5).astype(np.float32)
     mask[g.random((M, N)) < 0.3] = -np.inf
-    mask[5, :] = -np.inf
-    w.tensors["mask"] = wl.f32_to_bf16_bits(mask)
-    got = P.run_gpu(w, P.dev_tensors(w), fused=False)
+    for r in dead_rows:
+        if r < M:
+            mask[r, :] = -np.inf
+    return wl.f32_to_bf16_bits(mask)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M,N,K,softcap", [
+    (2, 96, 256, 64, 0.0),       # short K: the row kernel; fewer rows than a tile
+    (3, 300, 1000, 72, 0.0),     # ragged M and N, several chunks per row
+    (1, 512, 2048, 128, 3.0),    # soft-cap in front of the mask
+    (2, 200, 1024, 320, 0.0),    # long K: the cluster kernel (4 CTA pairs per row block)
+    (1, 256, 512, 512, 2.5),     # cluster kernel, soft-capped
+])
+def test_softmax_additive_mask_with_fully_masked_rows(batch, M, N, K, softcap, fused, cuda_device):
+    """The additive-mask variant: the mask tensor is one more operand of the epilogue; -inf entries give exact zeros, a
+    fully masked row gives a row of zeros (the plain definition would give NaN)."""
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=31 + K, causal=False, softcap=softcap)
+    dead = (5, M - 1, 130)
+    w.tensors["mask"] = _additive_mask(M, N, seed=K, dead_rows=dead)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     ref = P.run_oracle(w)
-    P.check_outputs(w, got, ref, label="softmax additive mask", softmax_tol=P.TOL_SOFTMAX_UNFUSED)
-    assert (got["Y"][:, 5, :] == 0).all()
+    P.check_outputs(w, got, ref, label=f"softmax additive mask fused={fused}", softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+    for r in dead:
+        if r < M:
+            assert (got["Y"][:, r, :] == 0).all()
+    rows_alive = [r for r in range(M) if r not in dead]
+    assert (got["Y"][:, rows_alive, :].float().sum(-1) - 1).abs().max().item() < 2e-2
 
 
 def test_fused_and_unfused_runs_are_bitwise_repeatable(cuda_device):

@@ -46,6 +46,11 @@ def _case(seed):
         if causal:
             M = N
         w = wl.scaled_masked_softmax(batch, M, N, K, seed=seed, causal=causal, softcap=softcap)
+        if not causal and g.random() < 0.4:   # an additive mask tensor with -inf entries and one fully masked row
+            mask = (g.standard_normal((M, N)) * 0.5).astype(np.float32)
+            mask[g.random((M, N)) < 0.25] = -np.inf
+            mask[int(g.integers(M)), :] = -np.inf
+            w.tensors["mask"] = wl.f32_to_bf16_bits(mask)
     return w, fused
 
 
