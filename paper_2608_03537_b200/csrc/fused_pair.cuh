@@ -799,6 +799,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const float* vecs[3] = {s_bias, s_gamma, s_beta};
         float racc[kStageMaxRed];  // thread-local partials (value; column for an arg max); indexed at run time
         int ridx[kStageMaxRed];
+        float2 sc_topk[kStageMaxRed];  // Top-K: the row's pick of round 0 (value, column bits), kept until its later rounds run
 #pragma unroll 1
         for (int r = 0; r < kStageMaxRed; ++r) {
           const int op = r < sp.n_red ? sp.red[r].op : COMFUSE_OP_RED_SUM;
@@ -817,15 +818,22 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int j = 0; j < 32; ++j) r32[j] = 0u;
         uint32_t ybox = 0, ybar = 0;
 
+        // A sweep runs a micro-instruction range over this thread's fragments.  Ordinary sweeps are the passes; behind a
+        // pass's merges every Top-K reduction of that pass adds K - 1 sweeps of its own code range (`topk_r` >= 0), each
+        // looking for the best element behind the previous pick (pv, pc).
+        int pass = 0, topk_r = -1, topk_round = 0;
+        float pv = 0.f;
+        int pc = 0;
 #pragma unroll 1
-        for (int pass = 0; pass < sp.n_passes; ++pass) {
-          const int i0 = sp.pass_off[pass], i1 = sp.pass_off[pass + 1];
+        while (pass < sp.n_passes) {
+          const int i0 = topk_r >= 0 ? sp.red[topk_r].code_lo : sp.pass_off[pass];
+          const int i1 = topk_r >= 0 ? sp.red[topk_r].code_hi : sp.pass_off[pass + 1];
 #pragma unroll 1
           for (int f = 0; f < kFrags; ++f) {
             const int g = h + EPW * (f >> 1), half = f & 1;
             const int lc = g * 64 + half * 32;  // first CTA-local column of the fragment
             const int col0 = ncta0 + lc;
-            if (pass == 0 && half == 0 && has_res) {
+            if (pass == 0 && topk_r < 0 && half == 0 && has_res) {
               // the residual box of this group rides the operand ring (one stage per warp pair and group)
               mbar_wait<false>(bar_rfull(ring.stage), (rfull_bits >> ring.stage) & 1u, w);
               rfull_bits ^= 1u << ring.stage;
@@ -1001,10 +1009,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
                   for (int j = 0; j < 32; ++j) v[j] = __fdividef(1.f, 1.f + ex2_approx(-1.4426950408889634f * v[j]));
                   break;
-                case kChainXsave: {  // x = v; written back over the accumulator when a later pass reads it
+                case kChainXsave: {  // x = v; written back over the accumulator when a later pass (or sweep) reads it
 #pragma unroll
                   for (int j = 0; j < 32; ++j) x[j] = v[j];
-                  if (sp.n_passes > 1) {
+                  if (sp.n_passes > 1 || sp.x_writeback) {
                     uint32_t vb[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) vb[j] = __float_as_uint(v[j]);
@@ -1018,6 +1026,20 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   break;
                 case kChainAcc: {  // thread-local partial of reduction ci.index over v
                   const int r = ci.index;
+                  if (topk_r >= 0) {
+                    if (r != topk_r) break;  // another reduction's accumulate inside this one's code range
+                    // best element behind the previous pick: smaller value, or the same value in a later column
+                    float a = racc[r];
+                    int ai = ridx[r];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                      const bool behind = v[j] < pv || (v[j] == pv && col0 + j > pc);
+                      if (behind && v[j] > a) { a = v[j]; ai = col0 + j; }  // columns rise: a strict compare keeps the lowest
+                    }
+                    racc[r] = a;
+                    ridx[r] = ai;
+                    break;
+                  }
                   float a = racc[r];
                   switch (sp.red[r].op) {
                     case COMFUSE_OP_RED_SUM:
@@ -1066,6 +1088,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   break;
                 }
                 default: {  // kChainEmit: round v once and put this half of the row into the warp's staging box
+                  if (topk_r >= 0) break;
                   if (half == 0) {
                     if (Cfg::RING_STAGING && in_ring) {
                       ybox = ring_box(warp - 2, ring_k);
@@ -1099,10 +1122,42 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               }
             }
           }
+          if (topk_r >= 0) {
+            // ---- a Top-K sweep is complete: merge the candidates, deliver the pick, go on to the next round / reduction / pass
+            const float2 tot = cluster_row_reduce<CN, MergeArgmax, EPW>(make_float2(racc[topk_r], __int_as_float(ridx[topk_r])), kThreadCount,
+                                                                       MergeArgmax(), s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase, w,
+                                                                       2u, pm, p.leader_reduce != 0);
+            pv = tot.x;
+            pc = __float_as_int(tot.y);
+            if (crank == 0 && h == 0 && valid) {
+              const long long o = (static_cast<long long>(b) * p.M + grow) * sp.red[topk_r].k + topk_round;
+              for (int q2 = 0; q2 < sp.n_row_out; ++q2)
+                if (sp.out[q2].topk_red == topk_r + 1) {
+                  if (sp.out[q2].is_int) static_cast<int*>(sp.out[q2].ptr)[o] = pc;
+                  else static_cast<float*>(sp.out[q2].ptr)[o] = pv;
+                }
+            }
+            if (++topk_round >= sp.red[topk_r].k) {
+              int nxt = -1;
+              for (int r = topk_r + 1; r < sp.n_red; ++r)
+                if (nxt < 0 && sp.red[r].pass == pass && sp.red[r].k > 1) nxt = r;
+              topk_r = nxt;
+              topk_round = 1;
+              if (topk_r >= 0) { pv = sc_topk[topk_r].x; pc = __float_as_int(sc_topk[topk_r].y); }
+            }
+            if (topk_r >= 0) {
+              racc[topk_r] = -INFINITY;
+              ridx[topk_r] = 0x7FFFFFFF;
+            } else {
+              if (pass == sp.n_passes - 1) release_accumulator(0);
+              ++pass;
+            }
+            continue;
+          }
           if (pass == 0) tmem_st_wait();
-          if (pass == sp.n_passes - 1) release_accumulator(0);
           // ---- stage boundary: merges of the pass's reductions in program order (every CTA of the group makes the same
           // calls), then the per-row arithmetic that depends on them
+          int first_topk = -1;
 #pragma unroll 1
           for (int r = 0; r < sp.n_red; ++r) {
             if (sp.red[r].pass != pass) continue;
@@ -1115,6 +1170,20 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             else
               tot = cluster_row_reduce<CN, MergeByOp, EPW>(mine, kThreadCount, MergeByOp{op}, s_pre, s_stats, bar_stats, row, h, crank, xpar, xphase,
                                                           w, 2u, pm, p.leader_reduce != 0);
+            if (sp.red[r].k > 0) {
+              // Top-K, round 0: the pass's own arg max; the later rounds follow behind the pass's merges
+              sc_topk[r] = tot;
+              if (crank == 0 && h == 0 && valid) {
+                const long long o = (static_cast<long long>(b) * p.M + grow) * sp.red[r].k;
+                for (int q2 = 0; q2 < sp.n_row_out; ++q2)
+                  if (sp.out[q2].topk_red == r + 1) {
+                    if (sp.out[q2].is_int) static_cast<int*>(sp.out[q2].ptr)[o] = __float_as_int(tot.y);
+                    else static_cast<float*>(sp.out[q2].ptr)[o] = tot.x;
+                  }
+              }
+              if (sp.red[r].k > 1 && first_topk < 0) first_topk = r;
+              continue;
+            }
             float val = op == COMFUSE_OP_RED_ARGMAX ? static_cast<float>(__float_as_int(tot.y)) : tot.x;
             if (op == COMFUSE_OP_RED_MEAN) val *= 1.f / static_cast<float>(CN * BN);
             scalar_set(sp.red[r].dst, val);
@@ -1148,10 +1217,22 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
             scalar_set(si.dst, rv);
           }
+          if (first_topk >= 0) {  // the pass's Top-K reductions take their further rounds before the next pass
+            topk_r = first_topk;
+            topk_round = 1;
+            pv = sc_topk[topk_r].x;
+            pc = __float_as_int(sc_topk[topk_r].y);
+            racc[topk_r] = -INFINITY;
+            ridx[topk_r] = 0x7FFFFFFF;
+          } else {
+            if (pass == sp.n_passes - 1) release_accumulator(0);
+            ++pass;
+          }
         }
         if (crank == 0 && h == 0 && valid) {
           const long long o = static_cast<long long>(b) * p.M + grow;
           for (int r = 0; r < sp.n_row_out; ++r) {
+            if (sp.out[r].topk_red) continue;  // delivered round by round
             const float val = scalar_get(CHO_SCALAR, sp.out[r].scalar, 0.f);
             if (sp.out[r].is_int) static_cast<int*>(sp.out[r].ptr)[o] = static_cast<int>(val);
             else static_cast<float*>(sp.out[r].ptr)[o] = val;

@@ -46,9 +46,16 @@ struct ChainInstr {
 
 struct StageReduction {
   uint8_t pass;        // the pass in which its input is available
-  uint8_t op;          // comfuse_op_t of the reduction (sum, mean, max, min, prod, argmax)
+  uint8_t op;          // comfuse_op_t of the reduction (sum, mean, max, min, prod, argmax; Top-K: argmax)
   uint8_t on_terminal; // input is y itself: accumulated in the terminal's pass from the unrounded y
-  uint8_t dst;         // per-row scalar it defines
+  uint8_t dst;         // per-row scalar it defines (unused by Top-K)
+  // Top-K (the StreamReduction node's parameter K, Sec. 5): K rounds of an arg max.  Round 0 is the arg max the pass's
+  // stream accumulates anyway; every further round sweeps the resident tensor again with code[code_lo .. code_hi) -- the
+  // instructions that lead from x to this reduction's ACC -- and takes the best element that ranks behind the previous
+  // pick (value falling, column rising).  The picks go straight to the row outputs that name this reduction.
+  uint8_t k;           // 0 = an ordinary reduction
+  uint8_t code_lo, code_hi;
+  uint8_t pad;
 };
 
 struct ScalarInstr {   // per-row arithmetic at a stage boundary: s[dst] = op(a, b)
@@ -62,18 +69,21 @@ struct ScalarInstr {   // per-row arithmetic at a stage boundary: s[dst] = op(a,
 };
 
 struct StageRowOutput {
-  void* ptr;        // fp32 [batch * M], int32 for an arg max
+  void* ptr;        // fp32 [batch * M], int32 for an arg max; [batch * M, K] for a Top-K output
   uint8_t scalar;
   uint8_t is_int;
-  uint8_t pad[6];
+  uint8_t topk_red; // 1 + the Top-K reduction whose values (is_int = 0) or columns (is_int = 1) this output takes, 0 = none
+  uint8_t pad[5];
 };
 
 constexpr int kStageMaxCode = 80, kStageMaxRed = 6, kStageMaxScalarInstr = 12, kStageMaxScalars = 16, kStageMaxRowOut = 6,
-              kStageMaxPasses = 4;
+              kStageMaxPasses = 4, kStageMaxTopK = 8;
 
 struct StageProgram {
   uint8_t n_red, n_scalar_instr, n_passes, terminal_pass;
-  uint8_t n_row_out, pad[3];
+  uint8_t n_row_out;
+  uint8_t x_writeback;  // x goes back to tensor memory even in a one-pass program (a Top-K re-reads it)
+  uint8_t pad[2];
   // per pass, the micro-instruction stream run on every 32-column fragment: code[pass_off[s] .. pass_off[s + 1]).
   // pass 0: entry chain, XSAVE; every pass: per reduction of the pass (XLOAD if v was changed,) its chain, ACC; the
   // terminal's pass: (XLOAD,) final chain, ACC of the reductions on y, EMIT.

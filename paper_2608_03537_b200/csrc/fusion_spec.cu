@@ -541,13 +541,39 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
   // reductions and per-row arithmetic, in node order
   int max_pass = an.stage[an.terminal];
   int& scalars = L.scalars;
+  int topk_input[kStageMaxRed];        // per reduction: the input node of a Top-K, else -1
+  std::vector<int> topk_of(n, -1);     // per Top-K node: its reduction
+  for (int r = 0; r < kStageMaxRed; ++r) topk_input[r] = -1;
   for (int k = 0; k < n; ++k) {
     if (!an.live[k] || an.type[k] != T_ROW) continue;
     const comfuse_spec_node_t& nd = an.nodes[k];
+    if (is_topk(nd.op)) {
+      // values and columns of the same input and K share one reduction; on chip K <= kStageMaxTopK
+      const int e = nd.in0;
+      if (nd.param > kStageMaxTopK || an.type[e] != T_TENSOR) return false;
+      int found = -1;
+      for (int r = 0; r < sp.n_red; ++r)
+        if (sp.red[r].k == nd.param && topk_input[r] == e) found = r;
+      if (found < 0) {
+        if (sp.n_red >= kStageMaxRed) return false;
+        StageReduction& r = sp.red[sp.n_red];
+        r.op = COMFUSE_OP_RED_ARGMAX;
+        r.k = static_cast<uint8_t>(nd.param);
+        r.pass = static_cast<uint8_t>(an.stage[e]);
+        red_chain.emplace_back();
+        if (e == an.terminal) r.on_terminal = 1;
+        else if (!L.chain(e, false, red_chain.back())) return false;
+        if (r.pass > max_pass) max_pass = r.pass;
+        topk_input[sp.n_red] = e;
+        found = sp.n_red++;
+      }
+      topk_of[k] = found;
+      continue;
+    }
     if (scalars >= kStageMaxScalars) return false;
     const int my = scalars++;  // before the chains below, which may allocate reciprocals
     if (is_reduce(nd.op)) {
-      if (is_topk(nd.op) || sp.n_red >= kStageMaxRed) return false;
+      if (sp.n_red >= kStageMaxRed) return false;
       const int e = nd.in0;
       if (an.type[e] != T_TENSOR) return false;
       StageReduction& r = sp.red[sp.n_red];
@@ -598,16 +624,23 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
     }
     for (int r = 0; r < sp.n_red; ++r) {
       if (sp.red[r].pass != pass || sp.red[r].on_terminal) continue;
+      sp.red[r].code_lo = static_cast<uint8_t>(nc);  // from here (v = x, reloaded if it was changed) to the ACC
       if (!v_is_x) micro(kChainXload);
       for (const ChainInstr& c : red_chain[r]) emit(c);
       v_is_x = red_chain[r].empty();
       micro(kChainAcc, r);
+      sp.red[r].code_hi = static_cast<uint8_t>(nc);
     }
     if (pass == sp.terminal_pass) {
+      const int fin_lo = nc;
       if (!v_is_x) micro(kChainXload);
       for (const ChainInstr& c : fin) emit(c);
       for (int r = 0; r < sp.n_red; ++r)
-        if (sp.red[r].on_terminal) micro(kChainAcc, r);
+        if (sp.red[r].on_terminal) {
+          micro(kChainAcc, r);
+          sp.red[r].code_lo = static_cast<uint8_t>(fin_lo);
+          sp.red[r].code_hi = static_cast<uint8_t>(nc);
+        }
       micro(kChainEmit);
     }
   }
@@ -615,10 +648,24 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
   if (!ok) return false;
   for (size_t r = 0; r < an.row_outputs.size(); ++r) {
     const int q = an.row_outputs[r];
+    if (is_topk(an.nodes[q].op)) {
+      if (topk_of[q] < 0) return false;
+      sp.out[r].topk_red = static_cast<uint8_t>(topk_of[q] + 1);
+      sp.out[r].is_int = an.nodes[q].op == COMFUSE_OP_RED_TOPK_INDICES;
+      sp.x_writeback = 1;
+      bind.row_out_pos[r] = static_cast<int>(r);
+      continue;
+    }
     if (an.type[q] != T_ROW || L.scalar_of[q] < 0) return false;
     sp.out[r].scalar = static_cast<uint8_t>(L.scalar_of[q]);
     sp.out[r].is_int = an.nodes[q].op == COMFUSE_OP_RED_ARGMAX;
     bind.row_out_pos[r] = static_cast<int>(r);
+  }
+  // a Top-K that no row output takes would still be swept K times: drop it back to a plain arg max
+  for (int r = 0; r < sp.n_red; ++r) {
+    bool used = false;
+    for (size_t o = 0; o < an.row_outputs.size(); ++o) used |= sp.out[o].topk_red == r + 1;
+    if (!used) sp.red[r].k = 0;
   }
   sp.n_row_out = static_cast<uint8_t>(an.row_outputs.size());
   return true;

@@ -212,7 +212,7 @@ def _topk_prog(k):
     return wl.SpecProgram(nodes, 3, (4, 5), ("rowvec",))
 
 
-def _run_topk(A, B, bias, k):
+def _run_topk(A, B, bias, k, fused=1):
     prog = _topk_prog(k)
     M, N = A.shape[0], B.shape[1]
     spec = cf.make_spec(prog.nodes, prog.terminal, 1, prog.row_outputs)
@@ -221,8 +221,8 @@ def _run_topk(A, B, bias, k):
     Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
     tv = torch.full((M, k), float("nan"), dtype=torch.float32, device=dev)
     ti = torch.full((M, k), -1, dtype=torch.int32, device=dev)
-    ws = torch.empty(cf.gemm_spec_workspace_size(spec, shape), dtype=torch.uint8, device=dev)
-    cf.gemm_spec(to_dev(A), to_dev(B), Y, spec, params=[to_dev(bias)], row_out=[tv, ti], workspace=ws)
+    ws = torch.empty(max(16, cf.gemm_spec_workspace_size(spec, shape, fused)), dtype=torch.uint8, device=dev)
+    cf.gemm_spec(to_dev(A), to_dev(B), Y, spec, params=[to_dev(bias)], row_out=[tv, ti], workspace=ws, fused=fused)
     torch.cuda.synchronize()
     assert cf.last_device_status() == cf.OK
     f = wl.bf16_to_f64
@@ -254,6 +254,38 @@ def test_topk_row_outputs_on_gaussian_data():
     assert np.all((ti >= 0) & (ti < N)) and all(len(set(r)) == k for r in ti.tolist())
     np.testing.assert_allclose(np.take_along_axis(Yref, ti.astype(np.int64), axis=1), tv, atol=3e-2)  # the picked columns hold those values
     assert np.mean(ti == ri.astype(np.int64)) > 0.9
+
+
+@pytest.mark.parametrize("M,N,K,k", [(70, 256, 16, 8), (300, 512, 16, 3), (200, 1024, 16, 8), (130, 2048, 16, 1), (257, 4096, 16, 4)])
+def test_topk_on_chip_exact_on_integer_data_with_ties(M, N, K, k):
+    """Top-K inside the fused kernel (K rounds of an arg max over the resident tensor, merged across the cluster): with
+    small integers the GEMM result is exact, so values AND columns must equal the oracle's, ties included.  Row lengths with
+    one, two, four, eight and sixteen CTAs per row block."""
+    g = np.random.default_rng(50 + N)
+    A = wl.f32_to_bf16_bits(g.integers(-1, 2, size=(M, K)).astype(np.float32))
+    B = wl.f32_to_bf16_bits(g.integers(-2, 3, size=(K, N)).astype(np.float32))
+    bias = wl.f32_to_bf16_bits(np.zeros(N, dtype=np.float32))
+    prog = _topk_prog(k)
+    plan = cf.spec_plan(cf.make_spec(prog.nodes, prog.terminal, 1, prog.row_outputs), cf.make_gemm_shape(1, M, N, K))
+    assert plan.path == cf.SPEC_PATH_FUSED_PROGRAM     # no detour through a materialised GEMM result
+    Y, tv, ti, Yref, rv, ri = _run_topk(A, B, bias, k, fused=2)
+    np.testing.assert_array_equal(to_f64(Y), Yref)
+    np.testing.assert_array_equal(tv.astype(np.float64), rv)
+    np.testing.assert_array_equal(ti.astype(np.int64), ri.astype(np.int64))
+    if k > 1:
+        assert (rv[:, :-1] == rv[:, 1:]).any()  # the data does contain ties
+
+
+def test_topk_on_chip_on_gaussian_data():
+    M, N, K, k = 300, 1024, 136, 5
+    A, B, (bias,) = _inputs(41, 1, M, N, K, ("rowvec",))
+    Y, tv, ti, Yref, rv, ri = _run_topk(A, B, bias, k, fused=2)
+    assert np.abs(to_f64(Y) - Yref).max() <= 3e-2
+    np.testing.assert_allclose(tv, rv, atol=1e-3)                 # fp32 values, not values that went through bf16
+    assert np.all(np.diff(tv, axis=1) <= 0)                       # falling order
+    assert np.all((ti >= 0) & (ti < N)) and all(len(set(r)) == k for r in ti.tolist())
+    np.testing.assert_allclose(np.take_along_axis(Yref, ti.astype(np.int64), axis=1), tv, atol=1e-3)
+    assert np.mean(ti == ri.astype(np.int64)) > 0.99
 
 
 def test_program_workload_at_bench_size_sampled_rows_and_graph_replay():
