@@ -20,6 +20,10 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
     COMFUSE_CASE(2048, 256, 256, 4, 2, 4)
     COMFUSE_CASE(4096, 256, 256, 8, 2, 4)
     default:
+      // Long K and a row length without a cluster instantiation -- above all rows wider than the largest cluster holds
+      // (N > 4096): the row kernel's statistics pass followed by a second MainLoop pass takes any N.  It pays the
+      // GEMM twice, which is still less than writing and re-reading the scores.
+      if (p.N >= 64) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
       return cudaErrorInvalidValue;
   }
 #undef COMFUSE_CASE

@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import paper_2608_03537_b200 as cf
 import workloads as wl
 from tests import parity as P
 
@@ -185,6 +186,18 @@ def test_softmax_large_scores_do_not_overflow(cuda_device):
     w.scalars["alpha"] = 4.0
     got = P.run_gpu(w, P.dev_tensors(w), fused=True)
     P.check_outputs(w, got, P.run_oracle(w), label="softmax large scores")
+
+
+@pytest.mark.parametrize("batch,M,N,K,causal", [(1, 300, 8192, 320, False), (2, 200, 1000, 512, False), (1, 1536, 1536, 320, True),
+                                               (1, 257, 12288, 264, False)])
+def test_softmax_long_k_rows_without_a_cluster_instantiation(batch, M, N, K, causal, cuda_device):
+    """Long K with a row wider than the largest cluster holds (or of a length without a cluster instantiation): fused through
+    the statistics pass + second MainLoop pass of the row kernel, at the fused tolerance."""
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=5 + N, causal=causal)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"softmax long K N={N}")
+    assert (got["Y"].float().sum(-1) - 1).abs().max().item() < 2e-2
+    assert cf.last_device_status() == cf.OK
 
 
 def _additive_mask(M, N, seed, dead_rows=(5,)):
