@@ -23,8 +23,9 @@ namespace comfuse {
 namespace {
 
 constexpr int kB2bEpiWarps = 16;                       // four per TMEM lane quarter, 32 columns of a 128-column chunk each
-constexpr int kB2bEpiThreads = 32 * kB2bEpiWarps;
-constexpr int kB2bThreads = 32 * (2 + kB2bEpiWarps);  // producer, UMMA, epilogue warps
+constexpr int kB2bFinWarps = 4;                        // one per TMEM lane quarter: a thread per row normalises and stores O
+constexpr int kMl2Warp = 2 + kB2bEpiWarps + kB2bFinWarps;  // its first lane issues S.V; the scores have a lane of their own (warp 1)
+constexpr int kB2bThreads = 32 * (kMl2Warp + 1);       // producer, score UMMAs, softmax warps, finish warps, S.V UMMAs
 constexpr int kSlotBytes = 128 * 64 * 2;  // one 128 x 64 bf16 box
 constexpr int kRingSlots = 8;
 
@@ -32,11 +33,11 @@ struct B2bSmem {
   static constexpr int OFF_RING = 0;
   static constexpr int OFF_S = kRingSlots * kSlotBytes;            // 2 buffers x 2 K blocks
   static constexpr int OFF_YBUF = OFF_S + 4 * kSlotBytes;          // output staging box (the second one is the idle eighth ring slot)
-  static constexpr int OFF_PRE = OFF_YBUF + kSlotBytes;            // float2 [2][4][128]
-  static constexpr int OFF_STATS = OFF_PRE + 2 * 4 * 128 * 8;      // float2 [2][1][128]
-  static constexpr int OFF_BAR = OFF_STATS + 2 * 128 * 8;
-  // barriers: full[8] empty[8] (8 unused) pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats[2] drain pfree
-  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 4;
+  static constexpr int OFF_PRE = OFF_YBUF + kSlotBytes;            // float [2][4][128]: the row maxima of the four threads of a row
+  static constexpr int OFF_ML = OFF_PRE + 2 * 4 * 128 * 4;         // float [4][5][128]: row maximum and four partial row sums of the last four sub-tiles
+  static constexpr int OFF_BAR = OFF_ML + 4 * 5 * 128 * 4;
+  // barriers: full[8] empty[8] (8 unused) pfull[2] sfull[2] sempty[2] ofull[2] oempty[2] stats[2] drain pfree drain2 lfull[4]
+  static constexpr int NUM_BARS = 3 * kRingSlots + 10 + 4 + 5;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
@@ -52,8 +53,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   uint8_t* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
   const uint32_t smem_base = smem_u32(smem);
 
-  float2* s_pre = reinterpret_cast<float2*>(smem + B2bSmem::OFF_PRE);
-  float2* s_stats = reinterpret_cast<float2*>(smem + B2bSmem::OFF_STATS);
+  float* s_mx = reinterpret_cast<float*>(smem + B2bSmem::OFF_PRE);
   const uint32_t bar_base = smem_base + B2bSmem::OFF_BAR;
   auto bar_full = [&](int s) { return bar_base + 8u * s; };                        // weight / X slot landed (even CTA)
   auto bar_empty = [&](int s) { return bar_base + 8u * (kRingSlots + s); };        // slot may be overwritten
@@ -64,7 +64,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   auto bar_oempty = [&](int a) { return bar_base + 8u * (3 * kRingSlots + 8 + a); };  // O slot drained by both CTAs (even CTA)
   const uint32_t bar_stats = bar_base + 8u * (3 * kRingSlots + 10);
   const uint32_t bar_drain = bar_stats + 16u;
-  const uint32_t bar_pfree = bar_drain + 8u;  // attention form: both P slots read by every epilogue warp (even CTA)
+  const uint32_t bar_pfree = bar_drain + 8u;  // both P slots read by every softmax warp (even CTA)
+  const uint32_t bar_drain2 = bar_pfree + 8u;
+  auto bar_lfull = [&](int a) { return bar_pfree + 16u + 8u * a; };  // row statistics of sub-tile k in slot k & 3 (this CTA)
+  float* s_ml = reinterpret_cast<float*>(smem + B2bSmem::OFF_ML);
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(smem + B2bSmem::OFF_MISC);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + B2bSmem::OFF_MISC + 4);
 
@@ -85,6 +88,11 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
   // staging box, so that both 64-column halves of a tile are staged and stored together.
   constexpr int RING = kRingSlots - 1;
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
+#ifdef COMFUSE_TRACE
+#define B2B_TRACE_AT(ix) do { if (p.trace && blockIdx.x == 0) p.trace[ix] = globaltimer_ns(); } while (0)
+#else
+#define B2B_TRACE_AT(ix) do { } while (0)
+#endif
   griddep_launch_dependents();  // the next kernel's set-up may overlap this kernel (it waits before touching memory)
 #ifdef COMFUSE_TRACE
   if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) p.trace[62] = globaltimer_ns();  // kernel entry
@@ -100,8 +108,10 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       mbar_init(bar_sfull(a), 2 * kB2bEpiWarps);   // one arrival per epilogue warp of both CTAs
       mbar_init(bar_sempty(a), 1);
       mbar_init(bar_ofull(a), 1);
-      mbar_init(bar_oempty(a), 2 * kB2bEpiWarps);
+      mbar_init(bar_oempty(a), 2 * kB2bFinWarps);
     }
+    for (int a = 0; a < 4; ++a) mbar_init(bar_lfull(a), kB2bEpiWarps);
+    mbar_init(bar_drain2, 1);
     mbar_init(bar_stats, 4);
     mbar_init(bar_stats + 8u, 4);
     mbar_init(bar_drain, 1);
@@ -166,110 +176,125 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------------------------------ UMMA issuer (even CTA)
+    // ------------------------------------------------------------------------------------------ score UMMAs (even CTA)
+    // The scores and S.V have an issuing lane each, so that a wait of one (the S buffers, an O slot) never holds back the
+    // other.  Both walk the same ring sequence, QK(0) | QK(k+1), V(k) ..., each taking its own items and stepping
+    // over the other's; the barrier parity of a slot is the ring's wrap count, whoever used the slot last.  A lane that
+    // steps over slots never saw their barriers complete, so each of its own waits must come behind an event that
+    // implies the slot's PREVIOUS fill has landed and been consumed (else the parity test passes on the older phase):
+    // here the scores of sub-tile k+1 wait for pfree(k) first, which lies behind S.V of sub-tile k-2 (the previous tenant
+    // of their first slot); the other three slots' previous tenants are this lane's own.
     if (lane == 0 && pm == 0) {
       constexpr uint32_t idesc_ml1 = make_idesc_bf16(256, 128, false, true);
-      constexpr uint32_t idesc_ml2 = make_idesc_bf16(256, 128, false, true);
       RingPos<RING> ring;
-      uint32_t full_bits = 0;
-      uint32_t sfull_uses[2] = {0, 0};
-      uint32_t tile_it = 0;
       bool ok = true;
       auto wait_slot = [&]() {  // the next ring item is a pair operand: wait until both halves have landed
         if (!ok) return 0u;
-        if (!mbar_wait<false>(bar_full(ring.stage), (full_bits >> ring.stage) & 1u, w)) { ok = false; return 0u; }
-        full_bits ^= 1u << ring.stage;
+        if (!mbar_wait<false>(bar_full(ring.stage), ring.phase, w)) { ok = false; return 0u; }
         tcgen05_fence_after_sync();
         return ring_addr(ring.stage);
       };
-      auto release_slot = [&](int stage) {
-        umma_commit_pair_both(bar_empty(stage));
-      };
-      {
-        // Software-pipelined over the cluster's tiles: the scores of tile t+1 (ML1) are issued as soon
-        // as the epilogue has read the scores of tile t out of the P slots, BEFORE S.V of tile t (ML2), so that the
-        // epilogue can go from the softmax of tile t straight to the softmax of tile t+1 while ML2(t) runs, and finds
-        // O(t) complete when it comes back for the normalisation.
-        auto ml1 = [&]() {  // P[0], P[1] = Q . Kt chunks 0, 1 of the next tile in the ring
-          const int xs0 = ring.stage;
-          const uint32_t x0 = wait_slot();
+      auto release_slot = [&](int stage) { umma_commit_pair_both(bar_empty(stage)); };
+      auto ml1 = [&]() {  // P[0], P[1] = Q . Kt chunks 0, 1 of the next sub-tile in the ring
+        const int xs0 = ring.stage;
+        const uint32_t x0 = wait_slot();
+        ring.advance();
+        const int xs1 = ring.stage;
+        const uint32_t x1 = wait_slot();
+        ring.advance();
+        const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
+        const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
+        for (int j = 0; j < 2 && ok; ++j) {
+          const int wstage = ring.stage;
+          const uint32_t wa = wait_slot();
           ring.advance();
-          const int xs1 = ring.stage;
-          const uint32_t x1 = wait_slot();
-          ring.advance();
-          const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
-          const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
-          for (int j = 0; j < 2 && ok; ++j) {
-            const int wstage = ring.stage;
-            const uint32_t wa = wait_slot();
-            ring.advance();
-            if (!ok) return;
-            const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+          if (!ok) return;
+          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
-                                wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
-            release_slot(wstage);
-            umma_commit_pair_both(bar_pfull(j));
-          }
-          release_slot(xs0);
-          release_slot(xs1);
-        };
-        if (nsub > 0) ml1();
-        for (int k = 0; k < nsub && ok; ++k, ++tile_it) {
-          const int obuf = tile_it & 1u;
-          const uint32_t d_o = tmem_base + 256 + obuf * 128;
-          if (k + 1 < nsub) {
-            if (!mbar_wait<false>(bar_pfree, tile_it & 1u, w)) { ok = false; break; }  // the epilogue holds tile t's scores in registers
-            tcgen05_fence_after_sync();
-            ml1();
-            if (!ok) break;
-          }
-          if (!mbar_wait<false>(bar_oempty(obuf), ((tile_it >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
-          tcgen05_fence_after_sync();
-          for (int j = 0; j < 2 && ok; ++j) {  // O = S . V, two K halves of 128 source positions
-            const int wstage = ring.stage;
-            const uint32_t wa = wait_slot();
-            ring.advance();
-            if (!ok) break;
-            if (!mbar_wait<false>(bar_sfull(j), sfull_uses[j] & 1u, w)) { ok = false; break; }
-            ++sfull_uses[j];
-            tcgen05_fence_after_sync();
-            const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
-            const uint64_t sdesc0 = make_smem_desc_sw128(s_addr(j, 0), 16, 1024);
-            const uint64_t sdesc1 = make_smem_desc_sw128(s_addr(j, 1), 16, 1024);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              umma_bf16_ss_pair(d_o, (kk < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((kk & 3) * 2), wdesc + static_cast<uint64_t>(kk * 128),
-                                idesc_ml2, (j | kk) != 0 ? 1u : 0u);
-            release_slot(wstage);
-            umma_commit_pair_both(bar_sempty(j));
-          }
-          if (ok) {
-            umma_commit_pair_both(bar_ofull(obuf));
-          }
+          for (int kk = 0; kk < 8; ++kk)
+            umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
+                              wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
+          release_slot(wstage);
+          umma_commit_pair_both(bar_pfull(j));
         }
+        release_slot(xs0);
+        release_slot(xs1);
+      };
+      if (nsub > 0) ml1();
+      for (int k = 0; k < nsub && ok; ++k) {
+        if (k + 1 < nsub) {
+          // the softmax warps hold sub-tile k's scores in registers: the P slots take the scores of sub-tile k+1
+          if (!mbar_wait<false>(bar_pfree, static_cast<uint32_t>(k) & 1u, w)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          if (k < 30) B2B_TRACE_AT(200 + 2 * k);
+          ml1();
+          if (k < 30) B2B_TRACE_AT(201 + 2 * k);
+        }
+        ring.skip(2);  // V(k) belongs to the other lane
       }
       umma_commit_pair(bar_drain);
       mbar_wait<false>(bar_drain, 0, w);
     }
-  } else {
-    // ------------------------------------------------------------------------------------------ epilogue warps
+  } else if (warp == kMl2Warp) {
+    // ------------------------------------------------------------------------------------------ S.V UMMAs (even CTA)
+    if (lane == 0 && pm == 0) {
+      constexpr uint32_t idesc_ml2 = make_idesc_bf16(256, 128, false, true);
+      RingPos<RING> ring;
+      bool ok = true;
+      auto wait_slot = [&]() {
+        if (!ok) return 0u;
+        if (!mbar_wait<false>(bar_full(ring.stage), ring.phase, w)) { ok = false; return 0u; }
+        tcgen05_fence_after_sync();
+        return ring_addr(ring.stage);
+      };
+      if (nsub > 0) ring.skip(4);  // QK(0)
+      for (int k = 0; k < nsub && ok; ++k) {
+        const uint32_t uk = static_cast<uint32_t>(k);
+        const int obuf = k & 1;
+        const uint32_t d_o = tmem_base + 256 + obuf * 128;
+        if (k + 1 < nsub) ring.skip(4);  // QK(k+1)
+        if (!mbar_wait<false>(bar_oempty(obuf), ((uk >> 1) & 1u) ^ 1u, w)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        if (k < 30) B2B_TRACE_AT(300 + 2 * k);
+        for (int j = 0; j < 2 && ok; ++j) {  // O = S . V, two K halves of 128 source positions
+          // S first, the V slot second.  A parity wait tells "the fill I expect has landed" from "the fill before it has not
+          // even landed yet" only if this lane looks at the slot AFTER that earlier fill has completed; the earlier fill
+          // of a V slot is a Q / K box of the same sub-tile (or this lane's own previous V box), which the score UMMAs
+          // consumed before the softmax that has just handed S over could start.  Looked at earlier (at kernel start, say),
+          // the wait would pass on an empty slot.
+          if (!mbar_wait<false>(bar_sfull(j), uk & 1u, w)) { ok = false; break; }
+          const int wstage = ring.stage;
+          const uint32_t wa = wait_slot();
+          ring.advance();
+          if (!ok) break;
+          tcgen05_fence_after_sync();
+          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+          const uint64_t sdesc0 = make_smem_desc_sw128(s_addr(j, 0), 16, 1024);
+          const uint64_t sdesc1 = make_smem_desc_sw128(s_addr(j, 1), 16, 1024);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            umma_bf16_ss_pair(d_o, (kk < 4 ? sdesc0 : sdesc1) + static_cast<uint64_t>((kk & 3) * 2), wdesc + static_cast<uint64_t>(kk * 128),
+                              idesc_ml2, (j | kk) != 0 ? 1u : 0u);
+          umma_commit_pair_both(bar_empty(wstage));
+          umma_commit_pair_both(bar_sempty(j));
+        }
+        if (ok) umma_commit_pair_both(bar_ofull(obuf));
+        if (k < 30) B2B_TRACE_AT(301 + 2 * k);
+      }
+      umma_commit_pair(bar_drain2);
+      mbar_wait<false>(bar_drain2, 0, w);
+    }
+  } else if (warp < 2 + kB2bEpiWarps) {
+    // ------------------------------------------------------------------------------------------ softmax warps
     const int q = warp & 3;          // TMEM lane quarter: rows 32q .. 32q+31
-    const int hh = (warp - 2) >> 2;  // which 32 columns of every 128-column chunk / of the 128 output columns
+    const int hh = (warp - 2) >> 2;  // which 32 columns of every 128-column chunk
     const int row = q * 32 + lane;
-    const int epi_tid = threadIdx.x - 64;
-    const bool store_thread = epi_tid == 0;
     const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
-    const uint32_t ybuf = smem_base + B2bSmem::OFF_YBUF;
     const uint32_t sfull_leader = map_to_cta(bar_sfull(0), leader);
-    const uint32_t oempty_leader = map_to_cta(bar_oempty(0), leader);
-    const int kblk = hh >> 1;            // K block of S (and residual box) this thread's columns fall into
+    const int kblk = hh >> 1;            // K block of S this thread's columns fall into
     const int chunk0 = (hh & 1) * 4;     // first of its four 16-byte chunks inside that 128-byte row
-    RingPos<RING> ring;
     uint32_t puses[2] = {0, 0}, suses[2] = {0, 0};
     int xpar = 0;
-    uint32_t xphase = 0;
 #ifdef COMFUSE_TRACE
     int trace_ix = 0;
 #define B2B_TRACE_POINT()                                                                                \
@@ -279,16 +304,12 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 #else
 #define B2B_TRACE_POINT() do { } while (0)
 #endif
-
     {
-      // ================= software-pipelined over the cluster's tiles:
-      //   softmax(t0) | softmax(t1) finish(t0) | softmax(t2) finish(t1) | ... | finish(last)
-      // so that S.V of tile t (ML2) runs under the softmax of tile t+1 and the UMMA lane never waits for this epilogue
-      // longer than one softmax.
-      // ---------------- Epi1 (N1 = 256: the two P slots hold one whole score row): row max and sum of exponentials
-      // across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next UMMAs' A operand;
-      // returns 1 / (row sum), applied in the tile's finish step (O = (S.V) / sum)
-      auto softmax_tile = [&]() -> float2 {
+      // One sub-tile after the other: the two P slots hold one whole score row of 256 source positions.  Row max and sum
+      // of exponentials across the two chunks and the four threads of the row, then S = bf16(2^(t - max)) as the next
+      // UMMAs' A operand.  S.V of sub-tile k runs under the softmax of sub-tile k+1; the division by the row sum is the
+      // finish warps' work.
+      auto softmax_tile = [&](int k) {
         for (int pb = 0; pb < 2; ++pb) {
           mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
           ++puses[pb];
@@ -300,7 +321,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         uint32_t v0[32], v1[32];
         tmem_ld_32cols(tmem_base + lane_sel + 0 * 128 + hh * 32, v0);
         tmem_ld_32cols(tmem_base + lane_sel + 1 * 128 + hh * 32, v1);
-        // the scores are in registers: the P slots may take the next tile's scores
+        // the scores are in registers: the P slots may take the next sub-tile's scores
         tcgen05_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster_noflush(map_to_cta(bar_pfree, leader));
@@ -310,147 +331,151 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           mx0 = max3(mx0, __uint_as_float(v0[i]), __uint_as_float(v0[i + 1]));
           mx1 = max3(mx1, __uint_as_float(v1[i]), __uint_as_float(v1[i + 1]));
         }
-        // sc > 0 is required (checked by the host): the maximum of the scaled scores is the scaled maximum
-        const float mloc = fmaxf(mx0, mx1) * sc;
-        float2 a0 = splat2(0.f), a1 = splat2(0.f);
+        // The row maximum first (the four threads of a row sit in the four warps of one lane quarter: shared memory and a
+        // barrier of those 128 threads), so that the exponentials come out against the final maximum and go straight
+        // into S; the row SUM is not needed here at all, the finish warps add the four partial sums.
+        // sc > 0 is required (checked by the host): the maximum of the scaled scores is the scaled maximum.
+        s_mx[(xpar * 4 + hh) * 128 + row] = fmaxf(mx0, mx1) * sc;
+        named_barrier_sync(1 + q, 128);
+        const float m = fmaxf(fmaxf(s_mx[(xpar * 4 + 0) * 128 + row], s_mx[(xpar * 4 + 1) * 128 + row]),
+                              fmaxf(s_mx[(xpar * 4 + 2) * 128 + row], s_mx[(xpar * 4 + 3) * 128 + row]));
+        xpar ^= 1;  // the write after next comes behind the next barrier, which every reader of this buffer passes first
+        B2B_TRACE_POINT();  // row maximum known
+        float2 acc = splat2(0.f);
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float2 d0 = fma2(f2_from_bits(v0[i], v0[i + 1]), splat2(sc), splat2(-mloc));
-          const float2 d1 = fma2(f2_from_bits(v1[i], v1[i + 1]), splat2(sc), splat2(-mloc));
-          // every other pair of the second chunk (a quarter of the scores) takes 2^x from the FMA-pipe polynomial (relative
-          // error 4e-6): the MUFU unit is the busiest pipe of this loop (measured: a quarter 29.4 us on a1, none 30.1, half 30.3)
-          const float2 e0 = make_float2(ex2_approx(d0.x), ex2_approx(d0.y));
-          const float2 e1 = (i & 2) ? ex2_poly2(d1) : make_float2(ex2_approx(d1.x), ex2_approx(d1.y));
-          v0[i] = __float_as_uint(e0.x); v0[i + 1] = __float_as_uint(e0.y);
-          v1[i] = __float_as_uint(e1.x); v1[i + 1] = __float_as_uint(e1.y);
-          a0 = add2(a0, e0);
-          a1 = add2(a1, e1);
-        }
-        const float lloc = (a0.x + a0.y) + (a1.x + a1.y);
-        const float2 tot = cluster_row_reduce<1, MergeMaxSumExp2, 4>(make_float2(mloc, lloc), 64.f, MergeMaxSumExp2(), s_pre, s_stats,
-                                                                     bar_stats, row, hh, 0u, xpar, xphase, w);
-        B2B_TRACE_POINT();  // exponentials done, row statistics merged
-        const float f = ex2_approx(mloc - tot.x);  // this thread's exponentials are relative to its own maximum
-        // the S buffers are free once ML2 of the previous tile has read them
         for (int pb = 0; pb < 2; ++pb) {
+          uint32_t(&vv)[32] = pb ? v1 : v0;
+          // S buffer pb is free once S.V of the previous sub-tile has read it
           mbar_wait<false>(bar_sempty(pb), (suses[pb] & 1u) ^ 1u, w);
           ++suses[pb];
-        }
-        __syncwarp();
-        B2B_TRACE_POINT();  // S buffers free
-#pragma unroll
-        for (int pb = 0; pb < 2; ++pb) {
-          const uint32_t(&vv)[32] = pb ? v1 : v0;
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(vv[2 * i], vv[2 * i + 1]), splat2(f)));
+          __syncwarp();
+          if (pb == 0) B2B_TRACE_POINT();  // first S buffer free
           const uint32_t sb = s_addr(pb, kblk);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t a = sb + swz128(row, chunk0 + i);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                         "r"(pk[4 * i + 3])
-                         : "memory");
+          for (int g = 0; g < 4; ++g) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int i = 8 * g + 2 * j;
+              const float2 d = fma2(f2_from_bits(vv[i], vv[i + 1]), splat2(sc), splat2(-m));
+              // a quarter of the scores takes 2^x from the FMA-pipe polynomial (relative error 4e-6): the MUFU unit is the
+              // busiest pipe of this loop
+              const float2 e = (pb == 1 && (j & 1)) ? ex2_poly2(d) : make_float2(ex2_approx(d.x), ex2_approx(d.y));
+              acc = add2(acc, e);
+              pk[j] = pack_bf16x2_rn(e);
+            }
+            const uint32_t a = sb + swz128(row, chunk0 + g);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
           }
+          fence_proxy_async_smem();  // S writes are visible to the tensor core's shared-memory reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster_noflush(sfull_leader + 8u * pb);  // S.V may start on this half
         }
-        fence_proxy_async_smem();  // S writes are visible to the tensor core's shared-memory reads
+        // (maximum in the log2 domain, partial sum of 2^(t - maximum)) of this sub-tile for the finish warps; the slot's
+        // previous tenant, sub-tile k-4, was read before the O slot that S.V of sub-tile k-1 needed was handed back
+        float* ml = s_ml + (k & 3) * 5 * 128;
+        if (hh == 0) ml[row] = m;
+        ml[(1 + hh) * 128 + row] = acc.x + acc.y;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_lfull(k & 3));
+        B2B_TRACE_POINT();  // S handed to the tensor pipe
+      };
+      for (int k = 0; k < nsub; ++k) softmax_tile(k);
+    }
+  } else if (warp < kMl2Warp) {
+    // ------------------------------------------------------------------------------------------ finish warps
+    // O = (S.V) / (row sum), rounded once: a thread per row walks the 128 output columns in four blocks, stages its warp's
+    // 32 rows in the two output boxes (columns 0..63 in the staging box, 64..127 in the idle eighth ring slot) and stores
+    // them, while the softmax warps are already on the next sub-tile.
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t lane_sel = static_cast<uint32_t>(q * 32) << 16;
+    const uint32_t oempty_leader = map_to_cta(bar_oempty(0), leader);
+    const uint32_t box0 = smem_base + B2bSmem::OFF_YBUF, box1 = ring_addr(kRingSlots - 1);
+    auto stage_block = [&](int cb, const uint32_t (&pk)[16]) {
+      const uint32_t box = cb < 2 ? box0 : box1;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t a = box + swz128(row, (cb & 1) * 4 + i);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                     "r"(pk[4 * i + 3])
+                     : "memory");
+      }
+    };
+    for (int i = 0; i < my_tiles; ++i) {
+      const int tile = cluster_id + i * num_clusters;
+      const uint32_t k0 = static_cast<uint32_t>(i * nhalf);  // the row tile's first sub-tile
+      const int bz = tile / p.mpairs;
+      const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
+      if (lane == 0) tma_store_wait_read<0>();  // the previous tile's stores have read this warp's rows of both boxes
+      __syncwarp();
+      if constexpr (NHALF == 1) {
+        const int obuf = k0 & 1u;
+        mbar_wait<false>(bar_lfull(k0 & 3u), (k0 >> 2) & 1u, w);
+        const float* ml = s_ml + (k0 & 3u) * 5 * 128 + row;
+        const float l = (ml[128] + ml[256]) + (ml[384] + ml[512]);
+        const float inv_l = l > 0.f ? 1.f / l : 0.f;
+        if (warp == 2 + kB2bEpiWarps && lane == 0 && i < 20) B2B_TRACE_AT(100 + 3 * i);
+        mbar_wait<false>(bar_ofull(obuf), (k0 >> 1) & 1u, w);
+        __syncwarp();
+        tcgen05_fence_after_sync();
+        if (warp == 2 + kB2bEpiWarps && lane == 0 && i < 20) B2B_TRACE_AT(101 + 3 * i);
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t v[32], pk[16];
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + cb * 32, v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(inv_l)));
+          stage_block(cb, pk);
+        }
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
+      } else {
+        // two sub-tiles, each exponentiated against its own maximum: O = (O0 2^(m0-m) + O1 2^(m1-m)) / (l0 2^(m0-m) + l1 2^(m1-m));
+        // k0 is even: slot 0 holds the first sub-tile's S.V, slot 1 the second's
+        mbar_wait<false>(bar_lfull(k0 & 3u), (k0 >> 2) & 1u, w);
+        mbar_wait<false>(bar_lfull((k0 + 1u) & 3u), (k0 >> 2) & 1u, w);
+        const float* pa = s_ml + (k0 & 3u) * 5 * 128 + row;
+        const float* pb = s_ml + ((k0 + 1u) & 3u) * 5 * 128 + row;
+        const float2 ml0 = make_float2(pa[0], (pa[128] + pa[256]) + (pa[384] + pa[512]));
+        const float2 ml1 = make_float2(pb[0], (pb[128] + pb[256]) + (pb[384] + pb[512]));
+        const float mm = fmaxf(ml0.x, ml1.x);
+        const float f0 = ml0.x == -INFINITY ? 0.f : ex2_approx(ml0.x - mm), f1 = ml1.x == -INFINITY ? 0.f : ex2_approx(ml1.x - mm);
+        const float l = ml0.y * f0 + ml1.y * f1;
+        const float inv_l = l > 0.f ? 1.f / l : 0.f;
+        const float2 w0 = splat2(f0 * inv_l), w1 = splat2(f1 * inv_l);
+        mbar_wait<false>(bar_ofull(0), (k0 >> 1) & 1u, w);
+        mbar_wait<false>(bar_ofull(1), (k0 >> 1) & 1u, w);
+        __syncwarp();
+        tcgen05_fence_after_sync();
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t v0[32], v1[32], pk[16];
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + 0 * 128 + cb * 32, v0);
+          tmem_ld_32cols(tmem_base + lane_sel + 256 + 1 * 128 + cb * 32, v1);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            pk[j] = pack_bf16x2_rn(fma2(f2_from_bits(v1[2 * j], v1[2 * j + 1]), w1, mul2(f2_from_bits(v0[2 * j], v0[2 * j + 1]), w0)));
+          stage_block(cb, pk);
+        }
+        tcgen05_fence_before_sync();
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive_cluster_noflush(sfull_leader);
-          mbar_arrive_cluster_noflush(sfull_leader + 8u);
-        }
-        B2B_TRACE_POINT();  // S handed to the tensor pipe
-        return tot;  // (row maximum in the log2 domain, sum of 2^(t - maximum)) of this sub-tile
-      };
-      // ---------------- Epi2: O = (S.V) / (row sum), rounded once, two 128 x 64 boxes staged and stored together
-      // `it` = number of the row tile's first sub-tile; ml0 / ml1 = (maximum, sum) of its one or two sub-tiles
-      auto finish_tile = [&](int tile, uint32_t it, float2 ml0, float2 ml1) {
-        const int bz = tile / p.mpairs;
-        const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
-        uint32_t pk[16];
-        if constexpr (NHALF == 1) {
-          const int obuf = it & 1u;
-          const float inv_l = ml0.y > 0.f ? 1.f / ml0.y : 0.f;
-          mbar_wait<false>(bar_ofull(obuf), (it >> 1) & 1u, w);
-          __syncwarp();
-          tcgen05_fence_after_sync();
-          B2B_TRACE_POINT();  // S.V of the tile complete
-          uint32_t v[32];
-          tmem_ld_32cols(tmem_base + lane_sel + 256 + obuf * 128 + hh * 32, v);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2_rn(mul2(f2_from_bits(v[2 * i], v[2 * i + 1]), splat2(inv_l)));
-          tcgen05_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster_noflush(oempty_leader + 8u * obuf);
-        } else {
-          // two sub-tiles, each exponentiated against its own maximum: O = (O0 2^(m0-m) + O1 2^(m1-m)) / (l0 2^(m0-m) + l1 2^(m1-m))
-          const float mm = fmaxf(ml0.x, ml1.x);
-          const float f0 = ml0.x == -INFINITY ? 0.f : ex2_approx(ml0.x - mm), f1 = ml1.x == -INFINITY ? 0.f : ex2_approx(ml1.x - mm);
-          const float l = ml0.y * f0 + ml1.y * f1;
-          const float inv_l = l > 0.f ? 1.f / l : 0.f;
-          const float2 w0 = splat2(f0 * inv_l), w1 = splat2(f1 * inv_l);
-          mbar_wait<false>(bar_ofull(0), (it >> 1) & 1u, w);  // `it` is even: slot 0 holds the first sub-tile's S.V, slot 1 the second's
-          mbar_wait<false>(bar_ofull(1), (it >> 1) & 1u, w);
-          __syncwarp();
-          tcgen05_fence_after_sync();
-          uint32_t v0[32], v1[32];
-          tmem_ld_32cols(tmem_base + lane_sel + 256 + 0 * 128 + hh * 32, v0);
-          tmem_ld_32cols(tmem_base + lane_sel + 256 + 1 * 128 + hh * 32, v1);
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            pk[i] = pack_bf16x2_rn(fma2(f2_from_bits(v1[2 * i], v1[2 * i + 1]), w1, mul2(f2_from_bits(v0[2 * i], v0[2 * i + 1]), w0)));
-          tcgen05_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive_cluster_noflush(oempty_leader);
-            mbar_arrive_cluster_noflush(oempty_leader + 8u);
-          }
-        }
-        // both halves at once: columns 0..63 go to the staging box, columns 64..127 to the idle eighth ring slot
-        if (store_thread) tma_store_wait_read<0>();  // the previous tile's stores have read both boxes
-        named_barrier_sync(3, kB2bEpiThreads);
-        {
-          const uint32_t box = kblk == 0 ? ybuf : ring_addr(kRingSlots - 1);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t a = box + swz128(row, chunk0 + i);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
-                         "r"(pk[4 * i + 3])
-                         : "memory");
-          }
-        }
-        fence_proxy_async_smem();
-        named_barrier_sync(3, kB2bEpiThreads);
-        if (store_thread) {
-          tma_store_3d(&tmO, ybuf, 0, m0, bz);
-          tma_store_3d(&tmO, ring_addr(kRingSlots - 1), 64, m0, bz);
-          tma_store_commit();
-        }
-        B2B_TRACE_POINT();  // tile stored
-      };
-      // Order (the S buffers and the O slots are handed back by the steps named behind the arrows):
-      //   one sub-tile per row tile:   softmax(0) | softmax(t+1), finish(t) ...
-      //   two sub-tiles per row tile:  softmax(0), softmax(1) | softmax(2t+2), finish(t), softmax(2t+3) ...
-      // (S.V of sub-tile 2t+2 needs O slot 0, which finish(t) releases; the softmax of 2t+3 needs the S buffers that
-      // S.V of 2t+2 releases, so it must come behind finish(t).)
-      float2 ml_a = make_float2(-INFINITY, 0.f), ml_b = ml_a;
-      if (nsub > 0) ml_a = softmax_tile();
-      if (nhalf == 2 && nsub > 1) ml_b = softmax_tile();
-      for (int i = 0; i < my_tiles; ++i) {
-        const int tile = cluster_id + i * num_clusters;
-        const int first = i * nhalf;
-        const float2 c0 = ml_a, c1 = ml_b;
-        if constexpr (NHALF == 1) {
-          if (first + 1 < nsub) ml_a = softmax_tile();
-          finish_tile(tile, static_cast<uint32_t>(first), c0, c0);
-        } else {
-          if (first + 2 < nsub) ml_a = softmax_tile();
-          finish_tile(tile, static_cast<uint32_t>(first), c0, c1);
-          if (first + 3 < nsub) ml_b = softmax_tile();
+          mbar_arrive_cluster_noflush(oempty_leader);
+          mbar_arrive_cluster_noflush(oempty_leader + 8u);
         }
       }
+      fence_proxy_async_smem();  // the staged rows are visible to the TMA store
+      __syncwarp();
+      if (warp == 2 + kB2bEpiWarps && lane == 0 && i < 20) B2B_TRACE_AT(102 + 3 * i);
+      if (lane == 0) {
+        tma_store_3d(&tmO, box0 + q * 4096, 0, m0 + q * 32, bz);
+        tma_store_3d(&tmO, box1 + q * 4096, 64, m0 + q * 32, bz);
+        tma_store_commit();
+      }
     }
-    if (store_thread) tma_store_wait_read<0>();  // the staging buffer must outlive the last store's read
+    if (lane == 0) tma_store_wait_read<0>();  // the staging boxes must outlive the last store's read
   }
 
 #ifdef COMFUSE_TRACE
@@ -488,7 +513,7 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   if (!encode_tmap_bf16_3d(&tmX, X, K, M, nb, K * 2, M * K * 2, 128) ||
       !encode_tmap_bf16_3d(&tmW1, W1, N1, K, nb, N1 * 2, K * N1 * 2, 128) ||
       !encode_tmap_bf16_3d(&tmW2, W2, N2, N1, nb, N2 * 2, N1 * N2 * 2, 128) ||
-      !encode_tmap_bf16_3d(&tmO, p.O, N2, M, nb, N2 * 2, M * N2 * 2, 128))
+      !encode_tmap_bf16_3d(&tmO, p.O, N2, M, nb, N2 * 2, M * N2 * 2, 32))  // a finish warp stores its 32 rows
     return cudaErrorInvalidValue;
   p.mblocks = (p.M + 127) / 128;
   p.mpairs = (p.mblocks + 1) / 2;

@@ -44,8 +44,9 @@ def f64(w: wl.Workload, name: str, rows=None):
 
 
 # --------------------------------------------------------------------------------------------- GPU side
-def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
-    """Run one workload through the library.  Returns dict of output tensors (on device)."""
+def prepare_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
+    """Allocate the outputs and the workspace of one workload once.  Returns (outputs on device, launch): launch()
+    enqueues one call of the library on the current stream and nothing else, so that calls can be queued back to back."""
     dev = T[next(iter(T))].device
     d = w.dims
     fill = float("nan") if poison else 0.0
@@ -53,21 +54,18 @@ def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
         O = torch.full((d["batch"], d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, fused, cf.B2B_SOFTMAX_ATTENTION, d["batch"], w.scalars["alpha"])
         ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
-        cf.b2b_attention(T["X"], T["W1"], T["W2"], O, alpha=w.scalars["alpha"], fused=fused, workspace=ws)
-        return {"Y": O}
+        return {"Y": O}, lambda: cf.b2b_attention(T["X"], T["W1"], T["W2"], O, alpha=w.scalars["alpha"], fused=fused, workspace=ws)
     if w.kind == wl.KIND_B2B_MLP_RELU:
         O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, fused, cf.B2B_MLP_RELU)
         ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
-        cf.b2b_mlp_relu(T["X"], T["W1"], T.get("b1"), T["W2"], T.get("b2"), O, fused=fused, workspace=ws)
-        return {"Y": O}
+        return {"Y": O}, lambda: cf.b2b_mlp_relu(T["X"], T["W1"], T.get("b1"), T["W2"], T.get("b2"), O, fused=fused, workspace=ws)
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
         O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused)
         ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
-        cf.b2b_gemm(T["X"], T["W1"], T["b1"], T["W2"], T["b2"], O, gamma=T.get("gamma"), beta=T.get("beta"),
-                    eps=w.scalars["eps"], fused=fused, workspace=ws)
-        return {"Y": O}
+        return {"Y": O}, lambda: cf.b2b_gemm(T["X"], T["W1"], T["b1"], T["W2"], T["b2"], O, gamma=T.get("gamma"), beta=T.get("beta"),
+                                             eps=w.scalars["eps"], fused=fused, workspace=ws)
     shape = (d["batch"], d["M"], d["N"]) if "batch" in d else (d["M"], d["N"])
     Y = torch.full(shape, fill, dtype=torch.bfloat16, device=dev)
     out = {"Y": Y}
@@ -93,7 +91,13 @@ def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
                              eps=kw.get("eps", 1e-5), mask=kw.get("mask", cf.MASK_NONE), fused=fused, flags=flags,
                              softcap=kw["softcap"])
     ws = torch.empty(max(cf.workspace_size(desc), 16), dtype=torch.uint8, device=dev)
-    cf.gemm_epilogue(T["A"], T["B"], Y, kind, fused=fused, workspace=ws, **kw)
+    return out, lambda: cf.gemm_epilogue(T["A"], T["B"], Y, kind, fused=fused, workspace=ws, **kw)
+
+
+def run_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
+    """Run one workload through the library.  Returns dict of output tensors (on device)."""
+    out, launch = prepare_gpu(w, T, fused, poison)
+    launch()
     return out
 
 
