@@ -57,8 +57,9 @@ int split_row_block(int epi, int N, int K);
 // column block width of the two-kernel form (0 = one kernel) and the number of blocks per row
 inline int wide_row_block(int epi, int N, int K) {
   if (epi != EPI_LN && epi != EPI_RMS_MAX) return 0;
-  if (N > kWideRowBlock) return (N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? kWideRowBlock : 0;
-  return split_row_block(epi, N, K);
+  const int narrow = N <= 16 * kWideRowBlock ? split_row_block(epi, N, K) : 0;
+  if (N > kWideRowBlock && narrow == 0) return (N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? kWideRowBlock : 0;
+  return narrow;
 }
 inline int wide_row_blocks(int epi, int N, int K) {
   const int w = wide_row_block(epi, N, K);

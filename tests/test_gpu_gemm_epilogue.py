@@ -75,8 +75,8 @@ WIDE_SHAPES = [(300, 8192, 72), (129, 12288, 64)]   # rows wider than the larges
 
 @pytest.mark.parametrize("M,N,K", WIDE_SHAPES)
 def test_layernorm_wide_rows_two_kernel_path(M, N, K, cuda_device):
-    """fused = 1 with N > 4096: per-4096-column-block stage 1 with partial statistics, then the rescaling kernel.  The row
-    passes through bf16 once before it is normalised, like the unfused path's intermediate, so it gets that path's budget."""
+    """fused = 1 with N > 4096 and a short contraction: per-4096-column-block stage 1 with partial statistics, then the
+    normalising kernel.  The row leaves the chip once as fp16 before it is normalised, so the fused tolerance holds."""
     import paper_2608_03537_b200 as cf
     w = wl.post_norm(M, N, K, seed=N + K, affine=True)
     T = P.dev_tensors(w)
@@ -92,6 +92,23 @@ def test_gelu_rmsnorm_max_wide_rows_two_kernel_path(M, N, K, cuda_device):
     w = wl.complex_subgraph(M, N, K, seed=M + N)
     got = P.run_gpu(w, P.dev_tensors(w), fused=True)
     P.check_outputs(w, got, P.run_oracle(w), label=f"RMS wide {M}x{N}x{K}", rowmax_tol=3e-2)
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 8192, 1024), (260, 6144, 1088), (129, 5120, 1024)])
+def test_wide_rows_behind_a_long_contraction_run_in_256_column_tiles(M, N, K, cuda_device):
+    """N > 4096 with K >= 1024: the first kernel works in 256-column tiles on every SM instead of 4096-column blocks on clusters
+    of sixteen (one partial per row and tile), which also covers row lengths that are multiples of 256 but not of 4096."""
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(M, N, K, seed=N + K, affine=True)
+    T = P.dev_tensors(w)
+    desc = cf.make_gemm_desc(T["A"], T["B"], torch.empty(M, N, dtype=torch.bfloat16, device=T["A"].device),
+                             cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=True)
+    assert cf.workspace_size(desc) == M * (N // 256) * 8
+    got = P.run_gpu(w, T, fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN wide 256-tiles {M}x{N}x{K}")
+    w = wl.complex_subgraph(M, N, K, seed=M + N)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"RMS wide 256-tiles {M}x{N}x{K}", rowmax_tol=3e-2)
 
 
 def test_wide_rows_need_their_workspace(cuda_device):
