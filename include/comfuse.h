@@ -107,9 +107,9 @@ typedef struct {
  * RMSNorm kinds run as TWO kernels and report batch * M * (N / block) * 8 bytes: the fused kernel finishes stage 1 per
  * column block, stores the un-normalised row in Y as fp16 (11 significant bits) and one partial statistic per row and
  * block in the workspace; a second kernel merges the partials and rescales the row in place to bf16.
- *   - Rows wider than the largest cluster can hold on-chip (N > 4096; supported for N a multiple of 4096 up to 65536,
- *     block = 4096): the un-normalised values are materialised because they no longer fit (Sec. 2.2).  The workspace is
- *     required.
+ *   - Rows wider than the largest cluster can hold on-chip (4096 < N <= 65536): the un-normalised values are materialised
+ *     because they no longer fit (Sec. 2.2).  block = 256 behind a long contraction (K >= 1024, N a multiple of 256),
+ *     otherwise block = 4096 (N a multiple of 4096).  The workspace is required.
  *   - Rows of 2048 .. 4096 columns (a multiple of 256) behind a long contraction (K >= 1024), block = 256: measured faster
  *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
  *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
