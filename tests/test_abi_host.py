@@ -61,8 +61,10 @@ def test_workspace_size_rules():
     sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldb=2048, ldr=2048, ldy=2048)
     assert _ws(_desc(**sm, mask=cf.MASK_CAUSAL))[0] == cf.ERR_UNSUPPORTED              # causal needs M == N
     assert _ws(_desc(**sm, M=2048, mask=cf.MASK_CAUSAL))[0] == cf.OK
-    assert _ws(_desc(**sm, mask=cf.MASK_ADDITIVE))[0] == cf.ERR_UNSUPPORTED            # additive mask: unfused only
+    assert _ws(_desc(**sm, mask=cf.MASK_ADDITIVE)) == (cf.OK, 0)                       # additive mask: fused and unfused
     assert _ws(_desc(**sm, mask=cf.MASK_ADDITIVE, fused=0))[0] == cf.OK
+    long_k = dict(sm, K=512, lda=512, N=8192, ldb=8192, ldr=8192, ldy=8192)
+    assert _ws(_desc(**long_k)) == (cf.OK, 0)                                          # softmax rows of any length run fused
     assert cf.lib().comfuse_workspace_size(None, None) == cf.ERR_INVALID_ARG
 
 
@@ -71,6 +73,11 @@ def test_wide_row_and_host_staging_sizes():
     assert _ws(_desc(**wide)) == (cf.OK, 256 * 2 * 8)                      # fused wide rows: (mean, M2) per row and 4096-column block
     assert _ws(_desc(**wide, kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX)) == (cf.OK, 256 * 2 * 8)
     assert _ws(_desc(N=8200, ldb=8200, ldr=8200, ldy=8200))[0] == cf.ERR_UNSUPPORTED   # wide rows come in whole 4096-column blocks
+    long_k = dict(K=1024, lda=1024)                                        # ... or, behind K >= 1024, in 256-column tiles
+    assert _ws(_desc(**wide, **long_k)) == (cf.OK, 256 * 32 * 8)
+    assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144, **long_k)) == (cf.OK, 256 * 24 * 8)
+    assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144))[0] == cf.ERR_UNSUPPORTED
+    assert _ws(_desc(N=4096, ldb=4096, ldr=4096, ldy=4096, **long_k)) == (cf.OK, 256 * 16 * 8)   # optional for rows that fit a cluster
     d = _desc()                                                            # A [256, 512], B [512, 768], R, Y [256, 768], dense
     n = ctypes.c_size_t(0)
     L = cf.lib()
