@@ -416,6 +416,79 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         MLP_TRACE_EPI1();
         if (++j == NC) j = 0;
       }
+      // ---------------------------------------------------------------------------------------- Epi2 of the LAST tile
+      // Nothing is left to overlap it with, so the sixteen Epi1 warps take it instead of the four Epi2 warps: a thread owns
+      // 32 of its row's 128 columns, the row statistics are merged across the four threads of the row through shared
+      // memory (an S buffer: every UMMA that read it is complete once the O slot is full).
+      if (my_tiles > 0) {
+        const int i = my_tiles - 1;
+        const int tile = tile_of(i);
+        const int bz = tile / p.mpairs;
+        const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128 + q * 32;
+        const int ob = i & 1;
+        const bool affine = p.gamma != nullptr || p.beta != nullptr;
+        float2* s_part = reinterpret_cast<float2*>(smem + MlpSmem::OFF_S);  // [4][128] (mean, M2) of a thread's 32 columns
+        mbar_wait<false>(bar_ofull(ob), (static_cast<uint32_t>(i) >> 1) & 1u, w);
+        __syncwarp();
+        tcgen05_fence_after_sync();
+        uint32_t v[32];
+        tmem_ld_32cols(tmem_base + lane_sel + 256 + ob * 128 + hh * 32, v);
+        const float4* b4 = reinterpret_cast<const float4*>(s_b2 + hh * 32);
+        const float shift = __uint_as_float(v[0]) + s_b2[hh * 32];
+        const float2 ns = splat2(-shift);
+        float2 s1 = splat2(0.f), s2 = splat2(0.f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float4 bb = b4[k];
+          const float2 x01 = add2(f2_from_bits(v[4 * k], v[4 * k + 1]), make_float2(bb.x, bb.y));
+          const float2 x23 = add2(f2_from_bits(v[4 * k + 2], v[4 * k + 3]), make_float2(bb.z, bb.w));
+          v[4 * k] = __float_as_uint(x01.x); v[4 * k + 1] = __float_as_uint(x01.y);
+          v[4 * k + 2] = __float_as_uint(x23.x); v[4 * k + 3] = __float_as_uint(x23.y);
+          const float2 d01 = add2(x01, ns), d23 = add2(x23, ns);
+          s1 = add2(s1, add2(d01, d23));
+          s2 = fma2(d01, d01, s2);
+          s2 = fma2(d23, d23, s2);
+        }
+        const float dsum = s1.x + s1.y;
+        const float2 mine = make_float2(shift + dsum * (1.f / 32.f), fmaxf((s2.x + s2.y) - dsum * dsum * (1.f / 32.f), 0.f));
+        s_part[hh * 128 + row] = mine;
+        named_barrier_sync(3 + q, 128);  // the four warps of this lane quarter
+        const float2 p0 = s_part[row], p1 = s_part[128 + row], p2 = s_part[256 + row], p3 = s_part[384 + row];
+        const float mu = ((p0.x + p1.x) + (p2.x + p3.x)) * 0.25f;
+        const float d0 = p0.x - mu, d1 = p1.x - mu, d2 = p2.x - mu, d3 = p3.x - mu;
+        const float m2 = ((p0.y + p1.y) + (p2.y + p3.y)) + 32.f * ((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3));  // equal-count Chan merge
+        const float rstd = rsqrtf(m2 * (1.f / 128.f) + 4.f * p.eps);
+        const float2 a2 = splat2(rstd), c2 = splat2(-mu * rstd);
+        uint32_t pk[16];
+        if (affine) {
+          const float4* g4 = reinterpret_cast<const float4*>(s_gamma + hh * 32);
+          const float4* be4 = reinterpret_cast<const float4*>(s_beta + hh * 32);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float4 gg = g4[k], be = be4[k];
+            const float2 n01 = fma2(f2_from_bits(v[4 * k], v[4 * k + 1]), a2, c2);
+            const float2 n23 = fma2(f2_from_bits(v[4 * k + 2], v[4 * k + 3]), a2, c2);
+            pk[2 * k] = pack_bf16x2_rn(fma2(n01, make_float2(gg.x, gg.y), make_float2(be.x, be.y)));
+            pk[2 * k + 1] = pack_bf16x2_rn(fma2(n23, make_float2(gg.z, gg.w), make_float2(be.z, be.w)));
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            pk[2 * k] = pack_bf16x2_rn(fma2(f2_from_bits(v[4 * k], v[4 * k + 1]), a2, c2));
+            pk[2 * k + 1] = pack_bf16x2_rn(fma2(f2_from_bits(v[4 * k + 2], v[4 * k + 3]), a2, c2));
+          }
+        }
+        // staged over the tile's X operand like the other tiles' rows (its UMMAs are complete), one pair of stores per quarter
+        store_row_chunks(pk, x_addr(i & 1, hh >> 1), row, (hh & 1) * 4);
+        fence_proxy_async_smem();
+        named_barrier_sync(3 + q, 128);
+        if (hh == 0 && lane == 0) {
+          tma_store_3d(&tmO, x_addr(i & 1, 0) + q * 32 * 128, 0, m0, bz);
+          tma_store_3d(&tmO, x_addr(i & 1, 1) + q * 32 * 128, 64, m0, bz);
+          tma_store_commit();
+          tma_store_wait_read<0>();  // the staging boxes must outlive the stores' reads
+        }
+      }
     } else {
       // ---------------------------------------------------------------------------------------- Epi2
       // The accumulator holds 2 (S W2 + X); x' = O + 2 b2 = 2 x; LayerNorm_eps(x) = (x' - mean') rsqrt(var' + 4 eps).
@@ -428,7 +501,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       const bool affine = p.gamma != nullptr || p.beta != nullptr;
       const float eps4 = 4.f * p.eps;
       int pending_x = -1;  // lane 0: X buffer whose output stores have not yet been seen to have read it
-      for (int i = 0; i < my_tiles; ++i) {
+      for (int i = 0; i + 1 < my_tiles; ++i) {  // the last tile is the Epi1 warps' (above)
         const int tile = tile_of(i);
         const int bz = tile / p.mpairs;
         const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128 + q * 32;
