@@ -155,7 +155,8 @@ typedef enum {
   COMFUSE_B2B_MLP_GELU_LAYERNORM = 0, /* as above                                                                   */
   /* Attention form (Sec. 4, Eq. 2 with a row reduction as F; the Target-Attention workload of Sec. 6.2):
    *   O = softmax(alpha * X.W1) . W2   per batch,  softmax over the N1 source positions,
-   * X [batch, M, K] queries, W1 [batch, K, N1] keys (already transposed), W2 [batch, N1, N2] values, O [batch, M, N2],
+   * X [batch, M, K] queries, W1 [batch, K, N1] keys (already transposed) -- or, with COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR,
+   * W1 [batch, N1, K], one key per row as an attention layer produces them --, W2 [batch, N1, N2] values, O [batch, M, N2],
    * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128 and N1 = 256 (a whole score row fits the
    * accumulators of one CTA pair) or N1 = 512 (two sub-tiles of 256 source positions, each exponentiated against its own
    * row maximum, combined when O is normalised); the probabilities are rounded to bf16 as the second GEMM's operand. */
@@ -176,8 +177,13 @@ typedef struct {
   int32_t kind;   /* comfuse_b2b_kind_t */
   int32_t batch;  /* >= 1; must be 1 for the MLP kind (its weights are shared by all rows) */
   float alpha;    /* attention kind: scale of the scores; ignored by the MLP kind */
-  int32_t reserved; /* must be 0 */
+  int32_t flags;  /* COMFUSE_B2B_FLAG_*; 0 otherwise (any other bit: COMFUSE_ERR_INVALID_ARG) */
 } comfuse_b2b_desc_t;
+
+/* Attention kind only: W1 is stored [batch, N1, K] (keys row-major, the contraction dimension contiguous).  The fused kernel
+ * reads it as a K-major tensor-core operand; the unfused path transposes it into its workspace first (K * N1 * 2 more bytes
+ * per batch). */
+#define COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR 1
 
 comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size_t* bytes);
 

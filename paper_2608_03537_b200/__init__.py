@@ -34,6 +34,7 @@ MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
 FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2
 B2B_MLP_GELU_LAYERNORM, B2B_SOFTMAX_ATTENTION, B2B_MLP_RELU = 0, 1, 2
+B2B_FLAG_KEYS_ROW_MAJOR = 1   # attention kind: W1 is [batch, N1, K] (one key per row)
 
 EXPORTED_SYMBOLS = (
     "comfuse_workspace_size",
@@ -74,7 +75,7 @@ class EpilogueArgs(Structure):
 
 class B2bDesc(Structure):
     _fields_ = [("M", c_int32), ("K", c_int32), ("N1", c_int32), ("N2", c_int32), ("eps", c_float), ("fused", c_int32),
-                ("kind", c_int32), ("batch", c_int32), ("alpha", c_float), ("reserved", c_int32)]
+                ("kind", c_int32), ("batch", c_int32), ("alpha", c_float), ("flags", c_int32)]
 
 
 # Epilogue programs as data: the node vocabulary (comfuse_op_t), by name
@@ -244,19 +245,20 @@ def gemm_epilogue_static_scratch(A, B, Y, kind, *, bias=None, residual=None, gam
     return Y
 
 
-def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True, kind=B2B_MLP_GELU_LAYERNORM, batch=1, alpha=1.0) -> B2bDesc:
-    return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)), int(kind), int(batch), float(alpha), 0)
+def make_b2b_desc(M, K, N1, N2, eps=1e-5, fused=True, kind=B2B_MLP_GELU_LAYERNORM, batch=1, alpha=1.0, flags=0) -> B2bDesc:
+    return B2bDesc(int(M), int(K), int(N1), int(N2), float(eps), int(bool(fused)), int(kind), int(batch), float(alpha), int(flags))
 
 
-def b2b_attention(Q, Kt, V, O, *, alpha, fused=True, workspace=None, stream=None):
+def b2b_attention(Q, Kt, V, O, *, alpha, fused=True, workspace=None, stream=None, keys_row_major=False):
     """Enqueue O = softmax(alpha * Q.Kt).V per batch (the attention form of the back-to-back GEMM).  Dense CUDA bf16
-    tensors Q [b, M, d], Kt [b, d, S] (keys already transposed), V [b, S, d2], O [b, M, d2]."""
+    tensors Q [b, M, d], Kt [b, d, S] (keys already transposed) or, with ``keys_row_major``, the keys as [b, S, d];
+    V [b, S, d2], O [b, M, d2]."""
     nb, M, K = Q.shape
-    N1, N2 = Kt.shape[2], V.shape[2]
-    assert Kt.shape == (nb, K, N1) and V.shape == (nb, N1, N2) and O.shape == (nb, M, N2)
+    N1, N2 = V.shape[1], V.shape[2]
+    assert Kt.shape == ((nb, N1, K) if keys_row_major else (nb, K, N1)) and V.shape == (nb, N1, N2) and O.shape == (nb, M, N2)
     for t in (Q, Kt, V, O):
         assert t.is_contiguous()
-    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha)
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha, B2B_FLAG_KEYS_ROW_MAJOR if keys_row_major else 0)
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
     st = lib().comfuse_b2b_gemm(byref(d), _ptr(Q), _ptr(Kt), None, _ptr(V), None, None, None, _ptr(O), ws_ptr, ws_bytes, _stream(stream))
     if st != OK:
@@ -370,14 +372,14 @@ def b2b_gemm_host(X, W1, b1, W2, b2, O, *, staging, gamma=None, beta=None, eps=1
     return O
 
 
-def b2b_attention_host(Q, Kt, V, O, *, staging, alpha, fused=True, workspace=None, stream=None):
+def b2b_attention_host(Q, Kt, V, O, *, staging, alpha, fused=True, workspace=None, stream=None, keys_row_major=False):
     """b2b_attention with Q, Kt, V and O in host memory (dense CPU tensors, pinned for asynchronous copies); ``staging`` is a
     CUDA uint8 tensor of at least b2b_host_staging_size(desc) bytes."""
     nb, M, K = Q.shape
-    N1, N2 = Kt.shape[2], V.shape[2]
+    N1, N2 = V.shape[1], V.shape[2]
     for t in (Q, Kt, V, O):
         assert t.is_contiguous()
-    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha)
+    d = make_b2b_desc(M, K, N1, N2, 0.0, fused, B2B_SOFTMAX_ATTENTION, nb, alpha, B2B_FLAG_KEYS_ROW_MAJOR if keys_row_major else 0)
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
     st = lib().comfuse_b2b_gemm_host(byref(d), _ptr(Q), _ptr(Kt), None, _ptr(V), None, None, None, _ptr(O),
                                      c_void_p(staging.data_ptr()), staging.numel() * staging.element_size(),

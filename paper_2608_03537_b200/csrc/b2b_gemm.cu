@@ -43,8 +43,10 @@ struct B2bSmem {
 };
 static_assert(B2bSmem::BYTES <= 232448, "shared memory budget");
 
-// NHALF: sub-tiles of 256 source positions per score row, 1 or 2.
-template <int NHALF>
+// NHALF: sub-tiles of 256 source positions per score row, 1 or 2.  KM: the keys (W1) are stored [batch, N1, K], one key per
+// row, and feed the score UMMAs as a K-major operand (two 64 x 64 boxes per slot: contraction elements 0..63 and 64..127 of
+// this CTA's 64 keys); else [batch, K, N1], an MN-major operand (one 128 x 64 box per slot).
+template <int NHALF, bool KM>
 __global__ void __launch_bounds__(kB2bThreads, 1)
 b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                 const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
@@ -152,6 +154,16 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         tma_load_3d_pair(ring_addr(ring.stage), tm, full, x, y, bz);
         ring.advance();
       };
+      // row-major keys: this CTA's 64 keys from `key0` on, as two boxes of 64 contraction elements each in one slot
+      auto push_keys = [&](int key0) {
+        if (!ok) return;
+        if (!mbar_wait<false>(bar_empty(ring.stage), ring.phase ^ 1u, w)) { ok = false; return; }
+        const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
+        mbar_arrive_expect_tx_cluster(full, kSlotBytes);
+        tma_load_3d_pair(ring_addr(ring.stage), &tmW1, full, 0, key0, bz);
+        tma_load_3d_pair(ring_addr(ring.stage) + kSlotBytes / 2, &tmW1, full, 64, key0, bz);
+        ring.advance();
+      };
       const int wcol = static_cast<int>(pm) * 64;  // this CTA's half of every 128-column weight chunk
       {
         // software-pipelined over tiles (see the UMMA lane): Q and K of tile t+1 go in before V of tile t
@@ -162,8 +174,13 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           const int m0 = (tile - bz * p.mpairs) * 256 + static_cast<int>(pm) * 128;
           push(&tmX, 0, m0, 0);
           push(&tmX, 64, m0, 0);
-          push(&tmW1, half * 256 + 0 * 128 + wcol, 0, 0);
-          push(&tmW1, half * 256 + 1 * 128 + wcol, 0, 0);
+          if constexpr (KM) {
+            push_keys(half * 256 + 0 * 128 + wcol);
+            push_keys(half * 256 + 1 * 128 + wcol);
+          } else {
+            push(&tmW1, half * 256 + 0 * 128 + wcol, 0, 0);
+            push(&tmW1, half * 256 + 1 * 128 + wcol, 0, 0);
+          }
         };
         if (nsub > 0) push_qk(0);
         for (int k = 0; k < nsub && ok; ++k) {
@@ -185,7 +202,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
     // here the scores of sub-tile k+1 wait for pfree(k) first, which lies behind S.V of sub-tile k-2 (the previous tenant
     // of their first slot); the other three slots' previous tenants are this lane's own.
     if (lane == 0 && pm == 0) {
-      constexpr uint32_t idesc_ml1 = make_idesc_bf16(256, 128, false, true);
+      constexpr uint32_t idesc_ml1 = make_idesc_bf16(256, 128, false, !KM);
       RingPos<RING> ring;
       bool ok = true;
       auto wait_slot = [&]() {  // the next ring item is a pair operand: wait until both halves have landed
@@ -209,11 +226,20 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
           const uint32_t wa = wait_slot();
           ring.advance();
           if (!ok) return;
-          const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+          if constexpr (KM) {
+            const uint64_t wdesc0 = make_smem_desc_sw128(wa, 16, 1024);
+            const uint64_t wdesc1 = make_smem_desc_sw128(wa + kSlotBytes / 2, 16, 1024);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
-                              wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
+            for (int kk = 0; kk < 8; ++kk)
+              umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
+                                (kk < 4 ? wdesc0 : wdesc1) + static_cast<uint64_t>((kk & 3) * 2), idesc_ml1, kk != 0 ? 1u : 0u);
+          } else {
+            const uint64_t wdesc = make_smem_desc_sw128(wa, 8192, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
+                                wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
+          }
           release_slot(wstage);
           umma_commit_pair_both(bar_pfull(j));
         }
@@ -516,7 +542,8 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   const uint64_t nb = static_cast<uint64_t>(p.batch);  // dense [batch, rows, cols] tensors
   // all boxes are 64 elements x 128 rows
   if (!encode_tmap_bf16_3d(&tmX, X, K, M, nb, K * 2, M * K * 2, 128) ||
-      !encode_tmap_bf16_3d(&tmW1, W1, N1, K, nb, N1 * 2, K * N1 * 2, 128) ||
+      !(p.keys_row_major ? encode_tmap_bf16_3d(&tmW1, W1, K, N1, nb, K * 2, N1 * K * 2, 64)   // [batch, N1, K]: 64 keys x 64 elements
+                         : encode_tmap_bf16_3d(&tmW1, W1, N1, K, nb, N1 * 2, K * N1 * 2, 128)) ||
       !encode_tmap_bf16_3d(&tmW2, W2, N2, N1, nb, N2 * 2, N1 * N2 * 2, 128) ||
       !encode_tmap_bf16_3d(&tmO, p.O, N2, M, nb, N2 * 2, M * N2 * 2, 32))  // a finish warp stores its 32 rows
     return cudaErrorInvalidValue;
@@ -541,13 +568,17 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   int ncl = max_clusters[di].load(std::memory_order_acquire);
   if (ncl == 0) {
-    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    e = cudaFuncSetAttribute(b2b_pair_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(b2b_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(b2b_pair_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
-    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1, false>, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di].store(n, std::memory_order_release);
@@ -558,8 +589,11 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
   if (p.mode != 1) return cudaErrorInvalidValue;  // the MLP forms have kernels of their own
-  return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2>, tmX, tmW1, tmW2, tmO, p)
-                     : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1>, tmX, tmW1, tmW2, tmO, p);
+  if (p.keys_row_major)
+    return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2, true>, tmX, tmW1, tmW2, tmO, p)
+                       : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, true>, tmX, tmW1, tmW2, tmO, p);
+  return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2, false>, tmX, tmW1, tmW2, tmO, p)
+                     : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, false>, tmX, tmW1, tmW2, tmO, p);
 }
 
 }  // namespace comfuse

@@ -13,6 +13,7 @@ struct B2bParams {
   int mode;             // 0: F = GELU(. + b1), tail = + b2 + X, LayerNorm; 1: F = softmax(alpha * .), tail = none;
                         // 2: F = ReLU(. + b1), tail = ReLU(. + b2) (the streamed-K kernel)
   float alpha;          // attention form: scale of the scores
+  int keys_row_major;   // attention form: W1 is [batch, N1, K] (K-major tensor-core operand) instead of [batch, K, N1]
   float eps;
   const uint16_t* X;  // also the residual of the tail
   const uint16_t* b1;

@@ -472,7 +472,8 @@ static comfuse_status_t validate_b2b_desc(const comfuse_b2b_desc_t* d) {
   if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
   if (d->kind != COMFUSE_B2B_MLP_GELU_LAYERNORM && d->kind != COMFUSE_B2B_SOFTMAX_ATTENTION && d->kind != COMFUSE_B2B_MLP_RELU)
     return COMFUSE_ERR_INVALID_ARG;
-  if (d->batch < 1 || d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->batch < 1 || (d->flags & ~COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) != 0) return COMFUSE_ERR_INVALID_ARG;
+  if (d->flags != 0 && d->kind != COMFUSE_B2B_SOFTMAX_ATTENTION) return COMFUSE_ERR_INVALID_ARG;
   if (d->kind == COMFUSE_B2B_MLP_GELU_LAYERNORM) {
     if (d->batch != 1) return COMFUSE_ERR_INVALID_ARG;
     if (d->N2 != d->K) return COMFUSE_ERR_INVALID_ARG;  // the residual is X itself
@@ -495,8 +496,10 @@ comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size
   if (!bytes) return COMFUSE_ERR_INVALID_ARG;
   comfuse_status_t s = validate_b2b_desc(desc);
   if (s != COMFUSE_OK) return s;
-  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1]
-    *bytes = desc->fused ? 0 : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2;
+  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1] (+ the transposed keys)
+    *bytes = desc->fused ? 0
+                         : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2 +
+                               ((desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) ? static_cast<size_t>(desc->batch) * desc->K * desc->N1 * 2 : 0);
   else if (desc->kind == COMFUSE_B2B_MLP_RELU)  // unfused: the bf16 hidden layer [M, N1]
     *bytes = desc->fused ? 0 : static_cast<size_t>(desc->M) * desc->N1 * 2;
   else
@@ -532,6 +535,7 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     B2bParams bp = {};
     bp.M = M; bp.K = K; bp.N1 = N1; bp.N2 = N2;
     bp.batch = desc->batch; bp.mode = attention ? 1 : (relu_mlp ? 2 : 0); bp.alpha = desc->alpha;
+    bp.keys_row_major = (desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) ? 1 : 0;
     bp.eps = desc->eps;
     bp.X = static_cast<const uint16_t*>(X);
     bp.b1 = static_cast<const uint16_t*>(b1);
@@ -562,6 +566,11 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     // unfused: P = X.W1 (bf16, workspace) -> row softmax of alpha * P in place -> O = P.W2, batched
     uint16_t* P = static_cast<uint16_t*>(workspace);
     const int nb = desc->batch;
+    if (desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) {  // keys [nb, N1, K] -> [nb, K, N1] behind the scores in the workspace
+      uint16_t* Kt = P + static_cast<size_t>(nb) * M * N1;
+      if (launch_transpose_bf16(static_cast<const uint16_t*>(W1), Kt, nb, N1, K, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
+      W1 = Kt;
+    }
     GemmMaps maps;
     FusedParams p = {};
     p.batch = nb; p.mblocks = (M + 127) / 128; p.alpha = 1.f;

@@ -185,3 +185,18 @@ def test_valid_call_without_a_usable_gpu_fails_cleanly():
     st = L.comfuse_gemm_epilogue(ctypes.byref(d), FAKE, FAKE, FAKE, ctypes.byref(args), None, 0, None)
     assert st in (cf.ERR_CUDA, cf.ERR_ARCH)
     assert cf.lib().comfuse_last_device_status(None) in (cf.ERR_CUDA, cf.ERR_ARCH)
+
+
+def test_b2b_flags_are_checked():
+    """The attention kind's layout flag: unknown bits and the flag on another kind are refused on the host."""
+    L = cf.lib()
+    n = ctypes.c_size_t(0)
+    att = cf.make_b2b_desc(256, 128, 256, 128, 0.0, True, cf.B2B_SOFTMAX_ATTENTION, 2, 0.1, cf.B2B_FLAG_KEYS_ROW_MAJOR)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK and n.value == 0
+    att.fused = 0
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK
+    assert n.value == 2 * 256 * 256 * 2 + 2 * 128 * 256 * 2          # scores + the transposed keys
+    att.flags = 2
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.ERR_INVALID_ARG
+    mlp = cf.make_b2b_desc(256, 128, 512, 128, 1e-5, True, cf.B2B_MLP_GELU_LAYERNORM, 1, 1.0, cf.B2B_FLAG_KEYS_ROW_MAJOR)
+    assert L.comfuse_b2b_workspace_size(ctypes.byref(mlp), ctypes.byref(n)) == cf.ERR_INVALID_ARG
