@@ -45,7 +45,7 @@ NCU_TRAFFIC = {
     # 227.6 MB in its window, the finish kernel another 77.1 MB
     "c3": (227_593_984, "profiles/fused_rmsnorm_max_c3_complex_subgraph.md"),
     "c4": (512_653_312, "profiles/softmax_rows_c4_scaled_causal_softmax.md"),
-    "c5": (8_707_328, "profiles/b2b_mlp_c5.md"),
+    "c5": (8_711_936, "profiles/b2b_mlp_c5.md"),
     "a1": (38_943_488, "profiles/b2b_attention_a1_target_attention.md"),
     "a2": (112_186_112, "profiles/b2b_attention_a2_self_attention_512.md"),
     "d1": (71_254_272, "profiles/b2b_stream_d1_dlrm_bottom_mlp.md"),
