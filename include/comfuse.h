@@ -88,6 +88,12 @@ typedef struct {
  * NO_ACTIVATION without a residual, and SOFTMAX with softcap > 0). */
 #define COMFUSE_FLAG_POST_RELU 1u      /* BIAS_RES_LAYERNORM kind only: Y = max(Y, 0) after the affine step            */
 #define COMFUSE_FLAG_NO_ACTIVATION 2u  /* BIAS_GELU_RES_RMSNORM_MAX kind only: H = alpha*A.B + bias + R, no GELU       */
+/* The second operand is stored [batch, N, K] (ldb >= K: the contraction dimension contiguous, one column of the product per
+ * row -- attention keys as a layer holds them), i.e. the call computes alpha * A.B^T of the stored tensors.  Fused: the
+ * softmax kind (the row softmax kernel reads it as a K-major tensor-core operand; any N >= 64, any K).  Unfused: every
+ * kind; the operand is transposed into the workspace first (batch * K * N * 2 more bytes).  Not taken by the host-buffer
+ * entry point (COMFUSE_ERR_UNSUPPORTED); the node-list entry point has no such flag. */
+#define COMFUSE_FLAG_B_ROW_MAJOR_NK 4u
 
 /* Runtime-parameter table of the op list.  bias, gamma, beta: bf16 device vectors of length N, shared by all batches;
  * residual: bf16 [batch, M, N] with leading dimension desc->ldr; mask: see comfuse_mask_t.  NULL means absent (bias,

@@ -32,7 +32,7 @@ EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 
 EPI_BIAS_ACTIVATION = 3   # reduction-free epilogue; reached through gemm_spec only
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
 HOST_A, HOST_B, HOST_RESIDUAL, HOST_Y = 1, 2, 4, 8
-FLAG_POST_RELU, FLAG_NO_ACTIVATION = 1, 2
+FLAG_POST_RELU, FLAG_NO_ACTIVATION, FLAG_B_ROW_MAJOR_NK = 1, 2, 4
 B2B_MLP_GELU_LAYERNORM, B2B_SOFTMAX_ATTENTION, B2B_MLP_RELU = 0, 1, 2
 B2B_FLAG_KEYS_ROW_MAJOR = 1   # attention kind: W1 is [batch, N1, K] (one key per row)
 
@@ -184,19 +184,21 @@ def _stream(stream=None):
 
 def make_gemm_desc(A, B, Y, kind, *, residual=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True, flags=0,
                    softcap=0.0) -> GemmDesc:
-    """Describe A [b, M, K] (or [M, K]), B [b, K, N] (or [K, N]), Y [b, M, N] from torch tensors' shapes and strides."""
+    """Describe A [b, M, K] (or [M, K]), B [b, K, N] (or [K, N]; with FLAG_B_ROW_MAJOR_NK in ``flags``: [b, N, K]),
+    Y [b, M, N] from torch tensors' shapes and strides."""
     batched = A.dim() == 3
     batch = A.shape[0] if batched else 1
     M, K = A.shape[-2], A.shape[-1]
-    N = B.shape[-1]
-    assert B.shape[-2] == K and Y.shape[-2] == M and Y.shape[-1] == N
+    b_nk = bool(int(flags) & FLAG_B_ROW_MAJOR_NK)
+    N = B.shape[-2] if b_nk else B.shape[-1]
+    assert (B.shape[-1] if b_nk else B.shape[-2]) == K and Y.shape[-2] == M and Y.shape[-1] == N
     assert A.stride(-1) == 1 and B.stride(-1) == 1 and Y.stride(-1) == 1
     d = GemmDesc()
     d.batch, d.M, d.N, d.K = batch, M, N, K
     d.lda, d.ldb, d.ldy = A.stride(-2), B.stride(-2), Y.stride(-2)
     d.ldr = residual.stride(-2) if residual is not None else N
     d.batch_stride_a = A.stride(0) if batched else M * d.lda
-    d.batch_stride_b = B.stride(0) if batched else K * d.ldb
+    d.batch_stride_b = B.stride(0) if batched else (N if b_nk else K) * d.ldb
     d.batch_stride_y = Y.stride(0) if batched else M * d.ldy
     d.batch_stride_r = (residual.stride(0) if batched else M * d.ldr) if residual is not None else M * N
     d.kind, d.mask, d.alpha, d.eps, d.fused, d.reserved = int(kind), int(mask), float(alpha), float(eps), int(bool(fused)), 0

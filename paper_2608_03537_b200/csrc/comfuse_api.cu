@@ -133,13 +133,17 @@ namespace {
 // Tensor maps of a GEMM -> subgraph call.  R may be null (no residual): its map is then left zeroed and never used.
 bool make_gemm_maps(GemmMaps* maps, const void* A, const void* B, const void* R, const void* Y, int batch, int M, int N, int K,
                     long long lda, long long ldb, long long ldr, long long ldy, long long bsa, long long bsb, long long bsr,
-                    long long bsy) {
+                    long long bsy, bool b_nk = false) {
   std::memset(maps, 0, sizeof(*maps));
   auto bs = [&](long long given, long long rows, long long ld) {
     return static_cast<uint64_t>(batch > 1 ? given : rows * ld) * 2;
   };
   if (!encode_tmap_bf16_3d(&maps->A, A, K, M, batch, static_cast<uint64_t>(lda) * 2, bs(bsa, M, lda), 128)) return false;
-  if (!encode_tmap_bf16_3d(&maps->B, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, K, ldb), 64)) return false;
+  if (b_nk) {  // B stored [N, K]: boxes of 128 rows (columns of the product) x 64 contraction elements, like A's
+    if (!encode_tmap_bf16_3d(&maps->B, B, K, N, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, N, ldb), 128)) return false;
+  } else if (!encode_tmap_bf16_3d(&maps->B, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, K, ldb), 64)) {
+    return false;
+  }
   if (!encode_tmap_bf16_3d(&maps->Y, Y, N, M, batch, static_cast<uint64_t>(ldy) * 2, bs(bsy, M, ldy), 32)) return false;
   if (R && !encode_tmap_bf16_3d(&maps->R, R, N, M, batch, static_cast<uint64_t>(ldr) * 2, bs(bsr, M, ldr), 128)) return false;
   return true;
@@ -169,17 +173,19 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
   if (d->mask < COMFUSE_MASK_NONE || d->mask > COMFUSE_MASK_ADDITIVE) return COMFUSE_ERR_INVALID_ARG;
   if (d->fused != 0 && d->fused != 1) return COMFUSE_ERR_INVALID_ARG;
   if (d->reserved != 0) return COMFUSE_ERR_INVALID_ARG;
-  if (d->flags & ~(COMFUSE_FLAG_POST_RELU | COMFUSE_FLAG_NO_ACTIVATION)) return COMFUSE_ERR_INVALID_ARG;
+  if (d->flags & ~(COMFUSE_FLAG_POST_RELU | COMFUSE_FLAG_NO_ACTIVATION | COMFUSE_FLAG_B_ROW_MAJOR_NK)) return COMFUSE_ERR_INVALID_ARG;
+  const bool b_nk = (d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0;
   if ((d->flags & COMFUSE_FLAG_POST_RELU) && d->kind != COMFUSE_EPI_BIAS_RES_LAYERNORM) return COMFUSE_ERR_INVALID_ARG;
   if ((d->flags & COMFUSE_FLAG_NO_ACTIVATION) && d->kind != COMFUSE_EPI_BIAS_GELU_RES_RMSNORM_MAX) return COMFUSE_ERR_INVALID_ARG;
   if (!(d->softcap >= 0.f) || (d->softcap > 0.f && d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX)) return COMFUSE_ERR_INVALID_ARG;
-  if (d->lda < d->K || d->ldb < d->N || d->ldy < d->N) return COMFUSE_ERR_INVALID_ARG;
+  if (d->lda < d->K || d->ldb < (b_nk ? d->K : d->N) || d->ldy < d->N) return COMFUSE_ERR_INVALID_ARG;
   if (d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX && d->mask != COMFUSE_MASK_NONE) return COMFUSE_ERR_INVALID_ARG;
   if (!mult8(d->N) || !mult8(d->K)) return COMFUSE_ERR_ALIGNMENT;
   if (!mult8(d->lda) || !mult8(d->ldb) || !mult8(d->ldy)) return COMFUSE_ERR_ALIGNMENT;
   if (d->batch > 1) {
     if (d->batch_stride_a < static_cast<long long>(d->M - 1) * d->lda + d->K) return COMFUSE_ERR_INVALID_ARG;
-    if (d->batch_stride_b < static_cast<long long>(d->K - 1) * d->ldb + d->N) return COMFUSE_ERR_INVALID_ARG;
+    if (d->batch_stride_b < (b_nk ? static_cast<long long>(d->N - 1) * d->ldb + d->K : static_cast<long long>(d->K - 1) * d->ldb + d->N))
+      return COMFUSE_ERR_INVALID_ARG;
     if (d->batch_stride_y < static_cast<long long>(d->M - 1) * d->ldy + d->N) return COMFUSE_ERR_INVALID_ARG;
     if (!mult8(d->batch_stride_a) || !mult8(d->batch_stride_b) || !mult8(d->batch_stride_y)) return COMFUSE_ERR_ALIGNMENT;
   }
@@ -189,7 +195,10 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
 
 // Does a fused instantiation exist for this description?  `on_chip_only`: without the two-kernel form.
 comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only = false) {
+  // a second operand stored [N, K]: the row softmax kernel is the one fused kernel that reads it
+  if ((d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) && d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
+  p.b_nk = (d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) ? 1 : 0;
   p.M = d->M;
   p.N = d->N;
   p.K = d->K;
@@ -328,6 +337,7 @@ comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t*
   } else {
     if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
     *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
+    if (desc->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) *bytes += static_cast<size_t>(desc->batch) * desc->K * desc->N * 2;  // + B transposed
   }
   return COMFUSE_OK;
 }
@@ -370,14 +380,26 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
 
   const long long bsr = desc->batch > 1 ? desc->batch_stride_r : 0;
   const long long bsy = desc->batch > 1 ? desc->batch_stride_y : 0;
+  const bool b_nk = (desc->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0;
   GemmMaps maps;
   if (desc->fused) {
     if (!make_gemm_maps(&maps, A, B, a.residual, Y, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, desc->ldr,
-                        desc->ldy, desc->batch_stride_a, desc->batch_stride_b, bsr, bsy))
+                        desc->ldy, desc->batch_stride_a, desc->batch_stride_b, bsr, bsy, b_nk))
       return COMFUSE_ERR_CUDA;
   } else {  // the GEMM's output is the dense bf16 Z in the workspace
-    if (!make_gemm_maps(&maps, A, B, nullptr, workspace, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, 0, desc->N,
-                        desc->batch_stride_a, desc->batch_stride_b, 0, static_cast<long long>(desc->M) * desc->N))
+    long long ldb = desc->ldb, bsb = desc->batch_stride_b;
+    if (b_nk) {
+      // B stored [batch, N, K]: a dense transposed copy [batch, K, N] behind Z in the workspace feeds the plain GEMM
+      uint16_t* Bt = static_cast<uint16_t*>(workspace) + static_cast<size_t>(desc->batch) * desc->M * desc->N;
+      if (launch_transpose_bf16_strided(static_cast<const uint16_t*>(B), Bt, desc->batch, desc->N, desc->K, desc->ldb,
+                                        desc->batch > 1 ? desc->batch_stride_b : 0, st) != cudaSuccess)
+        return COMFUSE_ERR_CUDA;
+      B = Bt;
+      ldb = desc->N;
+      bsb = static_cast<long long>(desc->K) * desc->N;
+    }
+    if (!make_gemm_maps(&maps, A, B, nullptr, workspace, desc->batch, desc->M, desc->N, desc->K, desc->lda, ldb, 0, desc->N,
+                        desc->batch_stride_a, bsb, 0, static_cast<long long>(desc->M) * desc->N))
       return COMFUSE_ERR_CUDA;
   }
 
@@ -388,6 +410,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.total_tiles = p.batch * p.mblocks;
   p.alpha = desc->alpha; p.eps = desc->eps;
   p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
+  p.b_nk = (desc->fused && b_nk) ? 1 : 0;
   p.post_relu = (desc->flags & COMFUSE_FLAG_POST_RELU) ? 1 : 0;
   p.no_activation = (desc->flags & COMFUSE_FLAG_NO_ACTIVATION) ? 1 : 0;
   p.softcap = desc->softcap;

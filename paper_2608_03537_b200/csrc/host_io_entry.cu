@@ -85,6 +85,7 @@ extern "C" comfuse_status_t comfuse_host_staging_size(const comfuse_gemm_desc_t*
   size_t ws = 0;
   const comfuse_status_t s = comfuse_workspace_size(desc, &ws);  // validates the description
   if (s != COMFUSE_OK) return s;
+  if (desc->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) return COMFUSE_ERR_UNSUPPORTED;  // the staged copies assume B [K, N]
   if ((host_mask & COMFUSE_HOST_RESIDUAL) && desc->ldr < desc->N) return COMFUSE_ERR_INVALID_ARG;
   const Extents e = extents_of(desc, host_mask);
   *bytes = round_up(e.a) + round_up(e.b) + round_up(e.r) + round_up(e.y);

@@ -13,7 +13,7 @@ bool softmax_rows_supported(const FusedParams& p) { return p.K <= 256 && p.N >= 
 cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_t stream) {
   constexpr int NSTAGES = 2, YBOXES = 2;
   using Cfg = RowSoftmaxCfg<NSTAGES, YBOXES>;
-  auto kern = softmax_rows_kernel<NSTAGES, YBOXES>;
+  auto kern = p.b_nk ? softmax_rows_kernel<NSTAGES, YBOXES, true> : softmax_rows_kernel<NSTAGES, YBOXES, false>;
   const DeviceInfo* dev = current_device_info();
   if (!dev) return cudaErrorInvalidDevice;
   constexpr int kMaxDev = 64;
@@ -40,7 +40,9 @@ cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_
 
   int ncl = max_clusters[di].load(std::memory_order_acquire);
   if (ncl == 0) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(softmax_rows_kernel<NSTAGES, YBOXES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(softmax_rows_kernel<NSTAGES, YBOXES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);

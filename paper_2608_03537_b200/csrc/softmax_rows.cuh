@@ -57,7 +57,9 @@ struct RowSoftmaxCfg {
   static_assert(NSTAGES >= 2 && NSTAGES <= 8 && YBOXES >= 1 && YBOXES <= 4, "ring and staging depths");
 };
 
-template <int NSTAGES, int YBOXES>
+// BKM: the B operand is stored [N, K] (one box of this CTA's 128 columns x 64 contraction elements per stage, K-major for the
+// UMMA, like A) instead of [K, N] (two boxes of 64 contraction rows x 64 columns, MN-major).
+template <int NSTAGES, int YBOXES, bool BKM>
 __global__ void __launch_bounds__(32 * 20, 1)
 softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmY, const FusedParams p) {
@@ -162,8 +164,12 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           tma_load_3d_pair_hint(sa, &tmA, full, kb * 64, m0, b, keep);
           // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
           const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
-          tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b, keep);
-          tma_load_3d_pair_hint(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b, keep);
+          if constexpr (BKM) {
+            tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, kb * 64, col, b, keep);
+          } else {
+            tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b, keep);
+            tma_load_3d_pair_hint(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b, keep);
+          }
           if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }
         }
         }
@@ -176,7 +182,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t phase = 0;
       uint32_t slot_uses[2] = {0, 0};
       uint32_t unit = 0;
-      constexpr uint32_t idesc = make_idesc_bf16(256, CHUNK, false, true);
+      constexpr uint32_t idesc = make_idesc_bf16(256, CHUNK, false, !BKM);
       bool ok = true;
       uint32_t total_units = 0;
       for (int r = 0; r < rounds; ++r) {
@@ -195,10 +201,11 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
-          const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
+          const uint64_t bdesc = BKM ? make_smem_desc_sw128(sa + Cfg::A_BYTES, 16, 1024)
+                                     : make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside A's swizzled row, 2048 bytes in B
-            umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc,
+          for (int k = 0; k < 4; ++k)  // K advances by 16 elements: 32 bytes inside a K-major operand's swizzled row, 2048 bytes in an MN-major B
+            umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(BKM ? k * 2 : k * 128), idesc,
                               (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair_both(bar_empty(stage));
           if (++stage == NSTAGES) { stage = 0; phase ^= 1u; }

@@ -96,7 +96,7 @@ def test_pattern_variant_flags_are_checked():
     assert _ws(_desc(flags=cf.FLAG_NO_ACTIVATION))[0] == cf.ERR_INVALID_ARG                 # belongs to the RMSNorm kind
     assert _ws(_desc(kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, flags=cf.FLAG_NO_ACTIVATION))[0] == cf.OK
     assert _ws(_desc(kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX, flags=cf.FLAG_POST_RELU))[0] == cf.ERR_INVALID_ARG
-    assert _ws(_desc(flags=4))[0] == cf.ERR_INVALID_ARG                                     # unknown bit
+    assert _ws(_desc(flags=8))[0] == cf.ERR_INVALID_ARG                                     # unknown bit
     assert _ws(_desc(softcap=30.0))[0] == cf.ERR_INVALID_ARG                                # soft-cap belongs to the softmax kind
     sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldb=2048, ldr=2048, ldy=2048)
     assert _ws(_desc(**sm, softcap=30.0))[0] == cf.OK
@@ -200,3 +200,19 @@ def test_b2b_flags_are_checked():
     assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.ERR_INVALID_ARG
     mlp = cf.make_b2b_desc(256, 128, 512, 128, 1e-5, True, cf.B2B_MLP_GELU_LAYERNORM, 1, 1.0, cf.B2B_FLAG_KEYS_ROW_MAJOR)
     assert L.comfuse_b2b_workspace_size(ctypes.byref(mlp), ctypes.byref(n)) == cf.ERR_INVALID_ARG
+
+
+def test_second_operand_layout_flag_rules():
+    """COMFUSE_FLAG_B_ROW_MAJOR_NK: ldb counts contraction elements, only the softmax kind has a fused kernel for it, the
+    unfused workspace also holds the transposed operand, the host-buffer form refuses it."""
+    nk = dict(flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=512)                       # B [768, 512]: ldb >= K
+    assert _ws(_desc(**nk))[0] == cf.ERR_UNSUPPORTED                        # LayerNorm kind, fused
+    assert _ws(_desc(fused=0, **nk)) == (cf.OK, 256 * 768 * 2 + 512 * 768 * 2)
+    assert _ws(_desc(fused=0, flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=504))[0] == cf.ERR_INVALID_ARG   # ldb < K
+    sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldr=2048, ldy=2048, K=64, lda=64, flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=64)
+    assert _ws(_desc(**sm)) == (cf.OK, 0)
+    assert _ws(_desc(**dict(sm, K=512, lda=512, ldb=512))) == (cf.OK, 0)   # long K: still the row kernel
+    assert _ws(_desc(flags=8))[0] == cf.ERR_INVALID_ARG                     # unknown bit
+    n = ctypes.c_size_t(0)
+    d = _desc(**sm)
+    assert cf.lib().comfuse_host_staging_size(ctypes.byref(d), cf.HOST_A, ctypes.byref(n)) == cf.ERR_UNSUPPORTED

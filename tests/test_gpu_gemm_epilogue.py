@@ -349,3 +349,52 @@ def test_layernorm_with_a_large_common_offset(fused, cuda_device):
     w.tensors["bias"] = wl.f32_to_bf16_bits(np.full(1024, 64.0, dtype=np.float32))
     got = P.run_gpu(w, P.dev_tensors(w), fused=fused)
     P.check_outputs(w, got, P.run_oracle(w), label=f"large offset fused={fused}")
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("batch,M,N,K,causal", [
+    (2, 256, 256, 64, True),       # one chunk
+    (3, 300, 1000, 72, False),     # ragged M, N and K
+    (2, 2048, 2048, 64, True),     # the attention-score shape of the fifth... fourth configuration, two batches
+    (1, 200, 1024, 320, False),    # long K: the row kernel's second MainLoop pass
+    (1, 129, 8192, 128, False),    # rows wider than a cluster
+])
+def test_softmax_second_operand_stored_n_by_k(batch, M, N, K, causal, fused, cuda_device):
+    """COMFUSE_FLAG_B_ROW_MAJOR_NK: the second operand as [batch, N, K] (attention keys, one per row).  The fused row softmax
+    kernel reads it as a K-major operand and gives the same bits as the call with the operand transposed; the unfused path
+    transposes it into its workspace."""
+    w = wl.scaled_masked_softmax(batch, M, N, K, seed=N + K, causal=causal)
+    T = P.dev_tensors(w)
+    Bnk = T["B"].transpose(1, 2).contiguous()                        # [batch, N, K]
+    Y = torch.full((batch, M, N), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    mask = cf.MASK_CAUSAL if causal else cf.MASK_NONE
+    desc = cf.make_gemm_desc(T["A"], Bnk, Y, cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"], mask=mask, fused=fused,
+                             flags=cf.FLAG_B_ROW_MAJOR_NK)
+    need = cf.workspace_size(desc)
+    assert need == (0 if fused else batch * M * N * 2 + batch * K * N * 2)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device=cuda_device)
+    cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"], mask=mask, fused=fused, workspace=ws,
+                     flags=cf.FLAG_B_ROW_MAJOR_NK)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK
+    P.check_outputs(w, {"Y": Y}, P.run_oracle(w), label=f"softmax B[N,K] {batch}x{M}x{N}x{K} fused={fused}",
+                    softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
+    if fused and K <= 256:   # same kernel, same arithmetic as with B [K, N]
+        ref = P.run_gpu(w, T, fused=True)["Y"]
+        assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
+
+
+def test_second_operand_n_by_k_other_kinds_run_unfused_only(cuda_device):
+    """LayerNorm kind with B [N, K]: no fused kernel reads that layout (UNSUPPORTED); the unfused path transposes and matches."""
+    w = wl.post_norm(300, 768, 200, seed=77, affine=True)
+    T = P.dev_tensors(w)
+    Bnk = T["B"].t().contiguous()
+    Y = torch.full((300, 768), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    kw = dict(bias=T["bias"], residual=T["residual"], gamma=T["gamma"], beta=T["beta"], alpha=w.scalars["alpha"], eps=w.scalars["eps"])
+    with pytest.raises(cf.ComfuseError) as e:
+        cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, fused=True, flags=cf.FLAG_B_ROW_MAJOR_NK, **kw)
+    assert e.value.status == cf.ERR_UNSUPPORTED
+    desc = cf.make_gemm_desc(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=False, flags=cf.FLAG_B_ROW_MAJOR_NK)
+    ws = torch.empty(cf.workspace_size(desc), dtype=torch.uint8, device=cuda_device)
+    cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, fused=False, workspace=ws, flags=cf.FLAG_B_ROW_MAJOR_NK, **kw)
+    P.check_outputs(w, {"Y": Y}, P.run_oracle(w), label="LN B[N,K] unfused", norm_tol=4e-2)
