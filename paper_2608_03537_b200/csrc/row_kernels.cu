@@ -232,8 +232,10 @@ __global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p,
   // launched with programmatic stream serialization: everything above this line may overlap the first kernel's tail
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int lane = threadIdx.x & 31;
-  const long long r = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);  // row over batch * M
-  if (r >= rows) return;
+  // rows from the last to the first: the first kernel wrote them in rising order, so the blocks that start first read what
+  // is most likely still in L2
+  const long long r = rows - 1 - (static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5));  // row over batch * M
+  if (r < 0) return;
   const int b = static_cast<int>(r / p.M);
   const int i = static_cast<int>(r - static_cast<long long>(b) * p.M);
   uint16_t* y = p.Y + static_cast<long long>(b) * p.batch_stride_y + static_cast<long long>(i) * p.ldy;
