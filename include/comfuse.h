@@ -89,10 +89,10 @@ typedef struct {
 #define COMFUSE_FLAG_POST_RELU 1u      /* BIAS_RES_LAYERNORM kind only: Y = max(Y, 0) after the affine step            */
 #define COMFUSE_FLAG_NO_ACTIVATION 2u  /* BIAS_GELU_RES_RMSNORM_MAX kind only: H = alpha*A.B + bias + R, no GELU       */
 /* The second operand is stored [batch, N, K] (ldb >= K: the contraction dimension contiguous, one column of the product per
- * row -- attention keys as a layer holds them), i.e. the call computes alpha * A.B^T of the stored tensors.  Fused: the
- * softmax kind (the row softmax kernel reads it as a K-major tensor-core operand; any N >= 64, any K).  Unfused: every
- * kind; the operand is transposed into the workspace first (batch * K * N * 2 more bytes).  Not taken by the host-buffer
- * entry point (COMFUSE_ERR_UNSUPPORTED); the node-list entry point has no such flag. */
+ * row -- a linear layer's weight [out, in], attention keys as a layer holds them), i.e. the call computes alpha * A.B^T of
+ * the stored tensors.  Every GEMM kernel of the library reads it in place as a K-major tensor-core operand (fused and
+ * unfused, all kinds, same results bit for bit as with the transposed operand).  Not taken by the host-buffer entry point
+ * (COMFUSE_ERR_UNSUPPORTED); the node-list entry point has no such flag. */
 #define COMFUSE_FLAG_B_ROW_MAJOR_NK 4u
 
 /* Runtime-parameter table of the op list.  bias, gamma, beta: bf16 device vectors of length N, shared by all batches;
@@ -187,8 +187,7 @@ typedef struct {
 } comfuse_b2b_desc_t;
 
 /* Attention kind only: W1 is stored [batch, N1, K] (keys row-major, the contraction dimension contiguous).  The fused kernel
- * reads it as a K-major tensor-core operand; the unfused path transposes it into its workspace first (K * N1 * 2 more bytes
- * per batch). */
+ * and the unfused path's GEMM read it in place as a K-major tensor-core operand. */
 #define COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR 1
 
 comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size_t* bytes);

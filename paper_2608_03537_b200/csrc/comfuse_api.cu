@@ -139,8 +139,8 @@ bool make_gemm_maps(GemmMaps* maps, const void* A, const void* B, const void* R,
     return static_cast<uint64_t>(batch > 1 ? given : rows * ld) * 2;
   };
   if (!encode_tmap_bf16_3d(&maps->A, A, K, M, batch, static_cast<uint64_t>(lda) * 2, bs(bsa, M, lda), 128)) return false;
-  if (b_nk) {  // B stored [N, K]: boxes of 128 rows (columns of the product) x 64 contraction elements, like A's
-    if (!encode_tmap_bf16_3d(&maps->B, B, K, N, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, N, ldb), 128)) return false;
+  if (b_nk) {  // B stored [N, K]: boxes of 64 rows (columns of the product) x 64 contraction elements
+    if (!encode_tmap_bf16_3d(&maps->B, B, K, N, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, N, ldb), 64)) return false;
   } else if (!encode_tmap_bf16_3d(&maps->B, B, N, K, batch, static_cast<uint64_t>(ldb) * 2, bs(bsb, K, ldb), 64)) {
     return false;
   }
@@ -195,8 +195,6 @@ comfuse_status_t validate_gemm_desc(const comfuse_gemm_desc_t* d) {
 
 // Does a fused instantiation exist for this description?  `on_chip_only`: without the two-kernel form.
 comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only = false) {
-  // a second operand stored [N, K]: the row softmax kernel is the one fused kernel that reads it
-  if ((d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) && d->kind != COMFUSE_EPI_SCALE_MASK_SOFTMAX) return COMFUSE_ERR_UNSUPPORTED;
   FusedParams p = {};
   p.b_nk = (d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) ? 1 : 0;
   p.M = d->M;
@@ -337,7 +335,6 @@ comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t*
   } else {
     if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
     *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
-    if (desc->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) *bytes += static_cast<size_t>(desc->batch) * desc->K * desc->N * 2;  // + B transposed
   }
   return COMFUSE_OK;
 }
@@ -387,19 +384,8 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
                         desc->ldy, desc->batch_stride_a, desc->batch_stride_b, bsr, bsy, b_nk))
       return COMFUSE_ERR_CUDA;
   } else {  // the GEMM's output is the dense bf16 Z in the workspace
-    long long ldb = desc->ldb, bsb = desc->batch_stride_b;
-    if (b_nk) {
-      // B stored [batch, N, K]: a dense transposed copy [batch, K, N] behind Z in the workspace feeds the plain GEMM
-      uint16_t* Bt = static_cast<uint16_t*>(workspace) + static_cast<size_t>(desc->batch) * desc->M * desc->N;
-      if (launch_transpose_bf16_strided(static_cast<const uint16_t*>(B), Bt, desc->batch, desc->N, desc->K, desc->ldb,
-                                        desc->batch > 1 ? desc->batch_stride_b : 0, st) != cudaSuccess)
-        return COMFUSE_ERR_CUDA;
-      B = Bt;
-      ldb = desc->N;
-      bsb = static_cast<long long>(desc->K) * desc->N;
-    }
-    if (!make_gemm_maps(&maps, A, B, nullptr, workspace, desc->batch, desc->M, desc->N, desc->K, desc->lda, ldb, 0, desc->N,
-                        desc->batch_stride_a, bsb, 0, static_cast<long long>(desc->M) * desc->N))
+    if (!make_gemm_maps(&maps, A, B, nullptr, workspace, desc->batch, desc->M, desc->N, desc->K, desc->lda, desc->ldb, 0, desc->N,
+                        desc->batch_stride_a, desc->batch_stride_b, 0, static_cast<long long>(desc->M) * desc->N, b_nk))
       return COMFUSE_ERR_CUDA;
   }
 
@@ -410,7 +396,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
   p.total_tiles = p.batch * p.mblocks;
   p.alpha = desc->alpha; p.eps = desc->eps;
   p.causal = desc->mask == COMFUSE_MASK_CAUSAL;
-  p.b_nk = (desc->fused && b_nk) ? 1 : 0;
+  p.b_nk = b_nk ? 1 : 0;  // every GEMM kernel reads the operand as stored
   p.post_relu = (desc->flags & COMFUSE_FLAG_POST_RELU) ? 1 : 0;
   p.no_activation = (desc->flags & COMFUSE_FLAG_NO_ACTIVATION) ? 1 : 0;
   p.softcap = desc->softcap;
@@ -519,10 +505,9 @@ comfuse_status_t comfuse_b2b_workspace_size(const comfuse_b2b_desc_t* desc, size
   if (!bytes) return COMFUSE_ERR_INVALID_ARG;
   comfuse_status_t s = validate_b2b_desc(desc);
   if (s != COMFUSE_OK) return s;
-  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1] (+ the transposed keys)
+  if (desc->kind == COMFUSE_B2B_SOFTMAX_ATTENTION)  // unfused: the bf16 scores / probabilities [batch, M, N1]
     *bytes = desc->fused ? 0
-                         : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2 +
-                               ((desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) ? static_cast<size_t>(desc->batch) * desc->K * desc->N1 * 2 : 0);
+                         : static_cast<size_t>(desc->batch) * desc->M * desc->N1 * 2;
   else if (desc->kind == COMFUSE_B2B_MLP_RELU)  // unfused: the bf16 hidden layer [M, N1]
     *bytes = desc->fused ? 0 : static_cast<size_t>(desc->M) * desc->N1 * 2;
   else
@@ -589,18 +574,15 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     // unfused: P = X.W1 (bf16, workspace) -> row softmax of alpha * P in place -> O = P.W2, batched
     uint16_t* P = static_cast<uint16_t*>(workspace);
     const int nb = desc->batch;
-    if (desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) {  // keys [nb, N1, K] -> [nb, K, N1] behind the scores in the workspace
-      uint16_t* Kt = P + static_cast<size_t>(nb) * M * N1;
-      if (launch_transpose_bf16(static_cast<const uint16_t*>(W1), Kt, nb, N1, K, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
-      W1 = Kt;
-    }
+    const bool keys_rm = (desc->flags & COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR) != 0;  // keys [nb, N1, K]: the plain GEMM reads them as stored
     GemmMaps maps;
     FusedParams p = {};
     p.batch = nb; p.mblocks = (M + 127) / 128; p.alpha = 1.f;
     p.status = dev->status_word; p.timeout_ns = timeout_ns();
-    if (!make_gemm_maps(&maps, X, W1, nullptr, P, nb, M, N1, K, K, N1, 0, N1, static_cast<long long>(M) * K,
-                        static_cast<long long>(K) * N1, 0, static_cast<long long>(M) * N1))
+    if (!make_gemm_maps(&maps, X, W1, nullptr, P, nb, M, N1, K, K, keys_rm ? K : N1, 0, N1, static_cast<long long>(M) * K,
+                        static_cast<long long>(K) * N1, 0, static_cast<long long>(M) * N1, keys_rm))
       return COMFUSE_ERR_CUDA;
+    p.b_nk = keys_rm ? 1 : 0;
     p.M = M; p.N = N1; p.K = K; p.Y = P; p.ldy = N1; p.batch_stride_y = static_cast<long long>(M) * N1;
     if (launch_plain_gemm(maps, p, st) != cudaSuccess) return COMFUSE_ERR_CUDA;
     RowParams r = {};
@@ -612,6 +594,7 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
     if (!make_gemm_maps(&maps, P, W2, nullptr, O, nb, M, N2, N1, N1, N2, 0, N2, static_cast<long long>(M) * N1,
                         static_cast<long long>(N1) * N2, 0, static_cast<long long>(M) * N2))
       return COMFUSE_ERR_CUDA;
+    p.b_nk = 0;
     p.N = N2; p.K = N1; p.Y = static_cast<uint16_t*>(O); p.ldy = N2; p.batch_stride_y = static_cast<long long>(M) * N2;
     return launch_plain_gemm(maps, p, st) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }

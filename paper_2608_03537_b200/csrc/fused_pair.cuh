@@ -272,11 +272,15 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const uint32_t full = map_to_cta(bar_full(ring.stage), leader);
             mbar_arrive_expect_tx_cluster(full, bytes);
             tma_load_3d_pair(sa, &tmA, full, kb * 64, m0, b);
-            // this CTA's half of each UMMA's B tile: boxes of 64 columns, 8 KB apart
+            // this CTA's half of each UMMA's B tile: boxes of 64 columns, 8 KB apart (B stored [K, N]: 64 contraction rows x
+            // 64 columns, MN-major for the UMMA; B stored [N, K]: 64 rows of B = columns of the product x 64 contraction
+            // elements, K-major like A -- same bytes, same places, the two coordinates change roles)
             auto load_b_half = [&](uint32_t dst, int first_group, int width) {
-              for (int j = 0; j < width / 128; ++j)
-                tma_load_3d_pair(dst + j * 8192, &tmB, full, group_col(ncta0, first_group + static_cast<int>(pm) * (width / 128) + j),
-                                 kb * 64, b);
+              for (int j = 0; j < width / 128; ++j) {
+                const int col = group_col(ncta0, first_group + static_cast<int>(pm) * (width / 128) + j);
+                if (p.b_nk) tma_load_3d_pair(dst + j * 8192, &tmB, full, kb * 64, col, b);
+                else tma_load_3d_pair(dst + j * 8192, &tmB, full, col, kb * 64, b);
+              }
             };
             if (LOCK) {
               load_b_half(sa + Cfg::A_BYTES, 0, BNS0);
@@ -312,6 +316,11 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       uint32_t slot_uses[2] = {0, 0};
       uint32_t unit_count = 0;
       bool ok = true;
+      // B stored [K, N] is an MN-major operand (64-column blocks 8 KB apart, 8 contraction rows 1 KB apart), B stored [N, K]
+      // a K-major one like A; everything that depends on it is computed once, outside the K loop
+      const bool bkm = p.b_nk != 0;
+      const uint64_t bdesc_layout = bkm ? make_smem_desc_sw128(0, 16, 1024) : make_smem_desc_sw128(0, 8192, 1024);
+      const uint64_t bstep[4] = {0, bkm ? 2u : 128u, bkm ? 4u : 256u, bkm ? 6u : 384u};
       for (int tile = cluster_id; tile < p.total_tiles && ok; tile += num_clusters) {
         int b, mpair0, ncta0;
         decode_tile(tile, b, mpair0, ncta0);
@@ -327,8 +336,8 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ++slot_uses[slot];
           tcgen05_fence_after_sync();
           const uint32_t d_tmem = tmem_base + (slot ? BNS0 : 0);
-          constexpr uint32_t idesc0 = make_idesc_bf16(256, BNS0, false, true);
-          constexpr uint32_t idesc1 = make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true);
+          const uint32_t idesc0 = bkm ? make_idesc_bf16(256, BNS0, false, false) : make_idesc_bf16(256, BNS0, false, true);
+          const uint32_t idesc1 = bkm ? make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, false) : make_idesc_bf16(256, BNS1 > 0 ? BNS1 : 16, false, true);
           const uint32_t idesc = (!LOCK && sub) ? idesc1 : idesc0;
           for (int kb = 0; kb < KB; ++kb) {
             if (!mbar_wait<false>(bar_full(ring.stage), (full_bits >> ring.stage) & 1u, w)) { ok = false; break; }
@@ -336,15 +345,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tcgen05_fence_after_sync();
             const uint32_t sa = smem_base + ring.stage * Cfg::STAGE_BYTES;
             const uint64_t adesc = make_smem_desc_sw128(sa, 16, 1024);
-            const uint64_t bdesc = make_smem_desc_sw128(sa + Cfg::A_BYTES, /*next 64-column block*/ 8192, /*next 8 K rows*/ 1024);
-            const uint64_t bdesc1 = make_smem_desc_sw128(sa + Cfg::A_BYTES + (BNS0 / 2) * 128, 8192, 1024);
+            // B: the descriptor's layout half was fixed before the loops; only the address field changes per stage
+            // (the address field takes the offset inside the CTA's shared-memory window: a shared address also carries the CTA's
+            // rank in the cluster above bit 18)
+            const uint64_t bdesc = bdesc_layout + (((sa + Cfg::A_BYTES) & 0x3FFFFu) >> 4);
+            const uint64_t bdesc1 = bdesc + (((BNS0 / 2) * 128) >> 4);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              // K advances by 16 elements: 32 bytes inside A's swizzled row, 16 K-lines (2048 bytes) in B
+              // K advances by 16 elements: 32 bytes inside A's (or a K-major B's) swizzled row, 16 K-lines (2048 bytes) in an MN-major B
               const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + static_cast<uint64_t>(k * 128), idesc, acc);
+              umma_bf16_ss_pair(d_tmem, adesc + static_cast<uint64_t>(k * 2), bdesc + bstep[k], idesc, acc);
               if (LOCK)  // the second sub-tile reuses the A tile that is already in shared memory
-                umma_bf16_ss_pair(d_tmem + BNS0, adesc + static_cast<uint64_t>(k * 2), bdesc1 + static_cast<uint64_t>(k * 128), idesc1, acc);
+                umma_bf16_ss_pair(d_tmem + BNS0, adesc + static_cast<uint64_t>(k * 2), bdesc1 + bstep[k], idesc1, acc);
             }
             // the stage is free in both CTAs once these UMMAs have read it
             umma_commit_pair_both(bar_empty(ring.stage), pair_mask);

@@ -9,8 +9,6 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   // COMFUSE_SOFTMAX_CLUSTER=1 forces the cluster kernel where it has an instantiation (for comparisons).
   static const bool force_cluster = std::getenv("COMFUSE_SOFTMAX_CLUSTER") != nullptr;
   if (softmax_rows_supported(p) && !force_cluster) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
-  // a second operand stored [N, K] is read by the row kernel only (it takes any K through its second MainLoop pass)
-  if (p.b_nk) return p.N >= 64 ? (supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st)) : cudaErrorInvalidValue;
 #define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
   case n:                                     \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, 0, epw>(maps, p, st);

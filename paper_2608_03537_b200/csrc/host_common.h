@@ -66,11 +66,6 @@ inline int wide_row_blocks(int epi, int N, int K) {
   return w ? N / w : 0;
 }
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
-// out[b][c][r] = in[b][r][c] for dense bf16 [batch, rows, cols] (rows, cols multiples of 8)
-cudaError_t launch_transpose_bf16(const uint16_t* in, uint16_t* out, int batch, int rows, int cols, cudaStream_t st);
-// the same from a strided source: row pitch `ld` elements, batch pitch `batch_stride` (0 = rows * ld); the result is dense
-cudaError_t launch_transpose_bf16_strided(const uint16_t* in, uint16_t* out, int batch, int rows, int cols, long long ld,
-                                          long long batch_stride, cudaStream_t st);
 // Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).
 bool softmax_rows_supported(const FusedParams& p);
 cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_t st);

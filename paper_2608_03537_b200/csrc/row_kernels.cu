@@ -363,32 +363,6 @@ cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* p
   return cudaErrorInvalidValue;
 }
 
-// out[b][c][r] = in[b][r][c]: 32 x 32 tiles through shared memory (unfused attention path with row-major keys)
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const uint16_t* in, uint16_t* out, int rows, int cols, long long ld,
-                                                             long long batch_stride) {
-  __shared__ uint16_t tile[32][33];
-  const long long ibase = static_cast<long long>(blockIdx.z) * batch_stride;
-  const long long base = static_cast<long long>(blockIdx.z) * rows * cols;
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int j = ty; j < 32; j += 8)
-    if (r0 + j < rows && c0 + tx < cols) tile[j][tx] = in[ibase + static_cast<long long>(r0 + j) * ld + c0 + tx];
-  __syncthreads();
-  for (int j = ty; j < 32; j += 8)
-    if (c0 + j < cols && r0 + tx < rows) out[base + static_cast<long long>(c0 + j) * rows + r0 + tx] = tile[tx][j];
-}
-
-cudaError_t launch_transpose_bf16_strided(const uint16_t* in, uint16_t* out, int batch, int rows, int cols, long long ld,
-                                          long long batch_stride, cudaStream_t st) {
-  count_launch();
-  transpose_bf16_kernel<<<dim3((cols + 31) / 32, (rows + 31) / 32, batch), 256, 0, st>>>(in, out, rows, cols, ld,
-                                                                                         batch_stride ? batch_stride : static_cast<long long>(rows) * ld);
-  return cudaGetLastError();
-}
-cudaError_t launch_transpose_bf16(const uint16_t* in, uint16_t* out, int batch, int rows, int cols, cudaStream_t st) {
-  return launch_transpose_bf16_strided(in, out, batch, rows, cols, cols, 0, st);
-}
-
 cudaError_t launch_bias_gelu(uint16_t* P, const uint16_t* bias, long long rows, int n, cudaStream_t st) {
   const long long nvec_total = rows * (n >> 3);
   const unsigned blocks = static_cast<unsigned>((nvec_total + 255) / 256);

@@ -164,8 +164,9 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           tma_load_3d_pair_hint(sa, &tmA, full, kb * 64, m0, b, keep);
           // this CTA's half of the UMMA's B tile: two boxes of 64 columns, 8 KB apart
           const int col = c * CHUNK + static_cast<int>(pm) * (CHUNK / 2);
-          if constexpr (BKM) {
+          if constexpr (BKM) {  // two boxes of 64 rows of B (columns of the product) x 64 contraction elements
             tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, kb * 64, col, b, keep);
+            tma_load_3d_pair_hint(sa + Cfg::A_BYTES + 8192, &tmB, full, kb * 64, col + 64, b, keep);
           } else {
             tma_load_3d_pair_hint(sa + Cfg::A_BYTES, &tmB, full, col, kb * 64, b, keep);
             tma_load_3d_pair_hint(sa + Cfg::A_BYTES + 8192, &tmB, full, col + 64, kb * 64, b, keep);

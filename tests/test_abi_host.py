@@ -195,7 +195,7 @@ def test_b2b_flags_are_checked():
     assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK and n.value == 0
     att.fused = 0
     assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK
-    assert n.value == 2 * 256 * 256 * 2 + 2 * 128 * 256 * 2          # scores + the transposed keys
+    assert n.value == 2 * 256 * 256 * 2                              # the scores; the keys are read in place
     att.flags = 2
     assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.ERR_INVALID_ARG
     mlp = cf.make_b2b_desc(256, 128, 512, 128, 1e-5, True, cf.B2B_MLP_GELU_LAYERNORM, 1, 1.0, cf.B2B_FLAG_KEYS_ROW_MAJOR)
@@ -203,11 +203,11 @@ def test_b2b_flags_are_checked():
 
 
 def test_second_operand_layout_flag_rules():
-    """COMFUSE_FLAG_B_ROW_MAJOR_NK: ldb counts contraction elements, only the softmax kind has a fused kernel for it, the
-    unfused workspace also holds the transposed operand, the host-buffer form refuses it."""
+    """COMFUSE_FLAG_B_ROW_MAJOR_NK: ldb counts contraction elements, every kind takes it fused and unfused with the usual
+    workspace, the host-buffer form refuses it."""
     nk = dict(flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=512)                       # B [768, 512]: ldb >= K
-    assert _ws(_desc(**nk))[0] == cf.ERR_UNSUPPORTED                        # LayerNorm kind, fused
-    assert _ws(_desc(fused=0, **nk)) == (cf.OK, 256 * 768 * 2 + 512 * 768 * 2)
+    assert _ws(_desc(**nk)) == (cf.OK, 0)                                   # LayerNorm kind, fused
+    assert _ws(_desc(fused=0, **nk)) == (cf.OK, 256 * 768 * 2)
     assert _ws(_desc(fused=0, flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=504))[0] == cf.ERR_INVALID_ARG   # ldb < K
     sm = dict(kind=cf.EPI_SCALE_MASK_SOFTMAX, N=2048, ldr=2048, ldy=2048, K=64, lda=64, flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=64)
     assert _ws(_desc(**sm)) == (cf.OK, 0)

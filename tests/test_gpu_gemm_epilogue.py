@@ -360,9 +360,8 @@ def test_layernorm_with_a_large_common_offset(fused, cuda_device):
     (1, 129, 8192, 128, False),    # rows wider than a cluster
 ])
 def test_softmax_second_operand_stored_n_by_k(batch, M, N, K, causal, fused, cuda_device):
-    """COMFUSE_FLAG_B_ROW_MAJOR_NK: the second operand as [batch, N, K] (attention keys, one per row).  The fused row softmax
-    kernel reads it as a K-major operand and gives the same bits as the call with the operand transposed; the unfused path
-    transposes it into its workspace."""
+    """COMFUSE_FLAG_B_ROW_MAJOR_NK: the second operand as [batch, N, K] (attention keys, one per row).  Every GEMM kernel
+    reads it in place as a K-major operand and gives the same bits as the call with the operand transposed."""
     w = wl.scaled_masked_softmax(batch, M, N, K, seed=N + K, causal=causal)
     T = P.dev_tensors(w)
     Bnk = T["B"].transpose(1, 2).contiguous()                        # [batch, N, K]
@@ -371,7 +370,7 @@ def test_softmax_second_operand_stored_n_by_k(batch, M, N, K, causal, fused, cud
     desc = cf.make_gemm_desc(T["A"], Bnk, Y, cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"], mask=mask, fused=fused,
                              flags=cf.FLAG_B_ROW_MAJOR_NK)
     need = cf.workspace_size(desc)
-    assert need == (0 if fused else batch * M * N * 2 + batch * K * N * 2)
+    assert need == (0 if fused else batch * M * N * 2)
     ws = torch.empty(max(need, 16), dtype=torch.uint8, device=cuda_device)
     cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_SCALE_MASK_SOFTMAX, alpha=w.scalars["alpha"], mask=mask, fused=fused, workspace=ws,
                      flags=cf.FLAG_B_ROW_MAJOR_NK)
@@ -379,22 +378,43 @@ def test_softmax_second_operand_stored_n_by_k(batch, M, N, K, causal, fused, cud
     assert cf.last_device_status() == cf.OK
     P.check_outputs(w, {"Y": Y}, P.run_oracle(w), label=f"softmax B[N,K] {batch}x{M}x{N}x{K} fused={fused}",
                     softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED)
-    if fused and K <= 256:   # same kernel, same arithmetic as with B [K, N]
-        ref = P.run_gpu(w, T, fused=True)["Y"]
-        assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
+    ref = P.run_gpu(w, T, fused=fused)["Y"]      # same kernels, same arithmetic as with B [K, N]
+    assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
 
 
-def test_second_operand_n_by_k_other_kinds_run_unfused_only(cuda_device):
-    """LayerNorm kind with B [N, K]: no fused kernel reads that layout (UNSUPPORTED); the unfused path transposes and matches."""
-    w = wl.post_norm(300, 768, 200, seed=77, affine=True)
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("kind", ["ln_small", "ln_lockstep", "rms_cluster16", "rms_two_kernels"])
+def test_second_operand_n_by_k_normalising_kinds(kind, fused, cuda_device):
+    """A linear layer's weight as it is stored, [out, in] = [N, K]: the LayerNorm and RMSNorm kinds on every tiling of the
+    fused kernel (one sub-tile, lock-step sub-tiles, clusters of sixteen, the two-kernel form) and on the unfused path give the
+    same bits as with the transposed operand, and match the oracle."""
+    w = {"ln_small": lambda: wl.post_norm(300, 256, 200, seed=71, affine=True),
+         "ln_lockstep": lambda: wl.post_norm(300, 768, 200, seed=72, affine=True),
+         "rms_cluster16": lambda: wl.complex_subgraph(150, 4096, 128, seed=73),
+         "rms_two_kernels": lambda: wl.complex_subgraph(520, 2048, 1024, seed=74)}[kind]()
     T = P.dev_tensors(w)
-    Bnk = T["B"].t().contiguous()
-    Y = torch.full((300, 768), float("nan"), dtype=torch.bfloat16, device=cuda_device)
-    kw = dict(bias=T["bias"], residual=T["residual"], gamma=T["gamma"], beta=T["beta"], alpha=w.scalars["alpha"], eps=w.scalars["eps"])
-    with pytest.raises(cf.ComfuseError) as e:
-        cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, fused=True, flags=cf.FLAG_B_ROW_MAJOR_NK, **kw)
-    assert e.value.status == cf.ERR_UNSUPPORTED
-    desc = cf.make_gemm_desc(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=False, flags=cf.FLAG_B_ROW_MAJOR_NK)
-    ws = torch.empty(cf.workspace_size(desc), dtype=torch.uint8, device=cuda_device)
-    cf.gemm_epilogue(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, fused=False, workspace=ws, flags=cf.FLAG_B_ROW_MAJOR_NK, **kw)
-    P.check_outputs(w, {"Y": Y}, P.run_oracle(w), label="LN B[N,K] unfused", norm_tol=4e-2)
+    ref, _ = P.prepare_gpu(w, T, fused=fused)
+    T2 = dict(T)
+    T2["B"] = T["B"].t().contiguous()
+    d = w.dims
+    Y = torch.full((d["M"], d["N"]), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
+        epi = cf.EPI_BIAS_RES_LAYERNORM
+        kw = dict(bias=T.get("bias"), residual=T.get("residual"), gamma=T.get("gamma"), beta=T.get("beta"), alpha=w.scalars["alpha"], eps=w.scalars["eps"])
+        outs = {"Y": Y}
+    else:
+        epi = cf.EPI_BIAS_GELU_RES_RMSNORM_MAX
+        outs = {"Y": Y, "row_max": torch.empty(d["M"], dtype=torch.float32, device=cuda_device),
+                "row_argmax": torch.empty(d["M"], dtype=torch.int32, device=cuda_device)}
+        kw = dict(bias=T.get("bias"), residual=T.get("residual"), gamma=T.get("gamma"), alpha=w.scalars["alpha"], eps=w.scalars["eps"],
+                  row_max=outs["row_max"], row_argmax=outs["row_argmax"])
+    desc = cf.make_gemm_desc(T["A"], T2["B"], Y, epi, residual=T.get("residual"), fused=fused, flags=cf.FLAG_B_ROW_MAJOR_NK)
+    ws = torch.empty(max(cf.workspace_size(desc), 16), dtype=torch.uint8, device=cuda_device)
+    cf.gemm_epilogue(T["A"], T2["B"], Y, epi, fused=fused, workspace=ws, flags=cf.FLAG_B_ROW_MAJOR_NK, **kw)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK
+    P.check_outputs(w, outs, P.run_oracle(w), label=f"{kind} B[N,K] fused={fused}", rowmax_tol=3e-2, norm_tol=P.TOL_NORM_MAX if fused else 4e-2)
+    base = P.run_gpu(w, T, fused=fused)
+    for k in outs:
+        a, b = outs[k], base[k]
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b), k
