@@ -91,8 +91,8 @@ typedef struct {
 /* The second operand is stored [batch, N, K] (ldb >= K: the contraction dimension contiguous, one column of the product per
  * row -- a linear layer's weight [out, in], attention keys as a layer holds them), i.e. the call computes alpha * A.B^T of
  * the stored tensors.  Every GEMM kernel of the library reads it in place as a K-major tensor-core operand (fused and
- * unfused, all kinds, same results bit for bit as with the transposed operand).  Not taken by the host-buffer entry point
- * (COMFUSE_ERR_UNSUPPORTED); the node-list entry point has no such flag. */
+ * unfused, all kinds, same results bit for bit as with the transposed operand); the host-buffer and workspace-free entry
+ * points take it too.  The node-list entry point has no such flag. */
 #define COMFUSE_FLAG_B_ROW_MAJOR_NK 4u
 
 /* Runtime-parameter table of the op list.  bias, gamma, beta: bf16 device vectors of length N, shared by all batches;

@@ -278,11 +278,11 @@ def host_staging_size(desc: GemmDesc, host_mask: int) -> int:
 
 def gemm_epilogue_host(A, B, Y, kind, *, staging, host_mask, bias=None, residual=None, gamma=None, beta=None,
                        mask_tensor=None, row_max=None, row_argmax=None, alpha=1.0, eps=1e-5, mask=MASK_NONE, fused=True,
-                       workspace=None, stream=None):
+                       workspace=None, stream=None, flags=0):
     """gemm_epilogue with the tensors named in ``host_mask`` (HOST_A | HOST_B | HOST_RESIDUAL | HOST_Y) living in host
     memory (CPU tensors, pinned for asynchronous copies); ``staging`` is a CUDA uint8 tensor of at least
     host_staging_size(desc, host_mask) bytes.  Copies and kernels are enqueued on the stream; nothing synchronises."""
-    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused)
+    d = make_gemm_desc(A, B, Y, kind, residual=residual, alpha=alpha, eps=eps, mask=mask, fused=fused, flags=flags)
     args = EpilogueArgs(_ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(mask_tensor), _ptr(row_max), _ptr(row_argmax))
     ws_ptr, ws_bytes = (None, 0) if workspace is None else (c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size())
     st = lib().comfuse_gemm_epilogue_host(byref(d), _ptr(A), _ptr(B), _ptr(Y), byref(args), int(host_mask),

@@ -71,7 +71,9 @@ struct Extents { size_t a, b, r, y; };
 Extents extents_of(const comfuse_gemm_desc_t* d, uint32_t mask) {
   Extents e = {0, 0, 0, 0};
   if (mask & COMFUSE_HOST_A) e.a = extent_bytes(d->batch, d->M, d->K, d->lda, d->batch_stride_a);
-  if (mask & COMFUSE_HOST_B) e.b = extent_bytes(d->batch, d->K, d->N, d->ldb, d->batch_stride_b);
+  if (mask & COMFUSE_HOST_B)  // stored [K, N], or [N, K] with COMFUSE_FLAG_B_ROW_MAJOR_NK
+    e.b = (d->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) ? extent_bytes(d->batch, d->N, d->K, d->ldb, d->batch_stride_b)
+                                                   : extent_bytes(d->batch, d->K, d->N, d->ldb, d->batch_stride_b);
   if (mask & COMFUSE_HOST_RESIDUAL) e.r = extent_bytes(d->batch, d->M, d->N, d->ldr, d->batch_stride_r);
   if (mask & COMFUSE_HOST_Y) e.y = extent_bytes(d->batch, d->M, d->N, d->ldy, d->batch_stride_y);
   return e;
@@ -85,7 +87,6 @@ extern "C" comfuse_status_t comfuse_host_staging_size(const comfuse_gemm_desc_t*
   size_t ws = 0;
   const comfuse_status_t s = comfuse_workspace_size(desc, &ws);  // validates the description
   if (s != COMFUSE_OK) return s;
-  if (desc->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) return COMFUSE_ERR_UNSUPPORTED;  // the staged copies assume B [K, N]
   if ((host_mask & COMFUSE_HOST_RESIDUAL) && desc->ldr < desc->N) return COMFUSE_ERR_INVALID_ARG;
   const Extents e = extents_of(desc, host_mask);
   *bytes = round_up(e.a) + round_up(e.b) + round_up(e.r) + round_up(e.y);

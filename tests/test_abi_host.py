@@ -204,7 +204,7 @@ def test_b2b_flags_are_checked():
 
 def test_second_operand_layout_flag_rules():
     """COMFUSE_FLAG_B_ROW_MAJOR_NK: ldb counts contraction elements, every kind takes it fused and unfused with the usual
-    workspace, the host-buffer form refuses it."""
+    workspace, the host-buffer form stages the operand with its own extent."""
     nk = dict(flags=cf.FLAG_B_ROW_MAJOR_NK, ldb=512)                       # B [768, 512]: ldb >= K
     assert _ws(_desc(**nk)) == (cf.OK, 0)                                   # LayerNorm kind, fused
     assert _ws(_desc(fused=0, **nk)) == (cf.OK, 256 * 768 * 2)
@@ -215,4 +215,5 @@ def test_second_operand_layout_flag_rules():
     assert _ws(_desc(flags=8))[0] == cf.ERR_INVALID_ARG                     # unknown bit
     n = ctypes.c_size_t(0)
     d = _desc(**sm)
-    assert cf.lib().comfuse_host_staging_size(ctypes.byref(d), cf.HOST_A, ctypes.byref(n)) == cf.ERR_UNSUPPORTED
+    assert cf.lib().comfuse_host_staging_size(ctypes.byref(d), cf.HOST_B, ctypes.byref(n)) == cf.OK
+    assert n.value == 2048 * 64 * 2                                         # the operand's own extent, [N, K]

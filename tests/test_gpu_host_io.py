@@ -53,6 +53,25 @@ def test_softmax_host_buffers_batched(cuda_device):
     assert torch.equal(hY.view(torch.int16), ref.cpu().view(torch.int16))
 
 
+def test_softmax_host_buffers_with_keys_stored_one_per_row(cuda_device):
+    """COMFUSE_FLAG_B_ROW_MAJOR_NK through the host-buffer form: the operand [batch, N, K] is staged with its own extent and
+    read in place; same bits as the device-pointer call with the transposed operand."""
+    import paper_2608_03537_b200 as cf
+    w = wl.scaled_masked_softmax(3, 256, 512, 72, seed=6, causal=False)
+    T = P.dev_tensors(w)
+    dev = T["A"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hA, hB = _pinned(T["A"]), _pinned(T["B"].transpose(1, 2).contiguous())
+    hY = torch.empty(3, 256, 512, dtype=torch.bfloat16).pin_memory()
+    mask = cf.HOST_A | cf.HOST_B | cf.HOST_Y
+    desc = cf.make_gemm_desc(hA, hB, hY, cf.EPI_SCALE_MASK_SOFTMAX, fused=True, flags=cf.FLAG_B_ROW_MAJOR_NK)
+    staging = torch.empty(cf.host_staging_size(desc, mask), dtype=torch.uint8, device=dev)
+    cf.gemm_epilogue_host(hA, hB, hY, cf.EPI_SCALE_MASK_SOFTMAX, staging=staging, host_mask=mask, alpha=w.scalars["alpha"],
+                          flags=cf.FLAG_B_ROW_MAJOR_NK)
+    torch.cuda.synchronize()
+    assert torch.equal(hY.view(torch.int16), ref.cpu().view(torch.int16))
+
+
 def test_b2b_host_buffers_match_device_buffers(cuda_device):
     import paper_2608_03537_b200 as cf
     w = wl.b2b_mlp(M=600, K=128, N1=512, N2=128, seed=8, affine=True)
