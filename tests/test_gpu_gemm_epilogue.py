@@ -418,3 +418,19 @@ def test_second_operand_n_by_k_normalising_kinds(kind, fused, cuda_device):
     for k in outs:
         a, b = outs[k], base[k]
         assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b), k
+
+
+def test_second_operand_n_by_k_through_the_workspace_free_entry_point(cuda_device):
+    """The workspace-free (unfused, fixed scratch) entry point passes the operand-layout flag through."""
+    w = wl.post_norm(300, 768, 200, seed=91, affine=True)
+    T = P.dev_tensors(w)
+    Bnk = T["B"].t().contiguous()
+    Y = torch.full((300, 768), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    cf.gemm_epilogue_static_scratch(T["A"], Bnk, Y, cf.EPI_BIAS_RES_LAYERNORM, bias=T["bias"], residual=T["residual"],
+                                    gamma=T["gamma"], beta=T["beta"], alpha=w.scalars["alpha"], eps=w.scalars["eps"],
+                                    flags=cf.FLAG_B_ROW_MAJOR_NK)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK
+    ref = P.run_gpu(w, T, fused=False)["Y"]
+    assert torch.equal(Y.view(torch.int16), ref.view(torch.int16))
+    P.check_outputs(w, {"Y": Y}, P.run_oracle(w), label="static scratch B[N,K]", norm_tol=4e-2)
