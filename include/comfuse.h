@@ -92,7 +92,7 @@ typedef struct {
  * row -- a linear layer's weight [out, in], attention keys as a layer holds them), i.e. the call computes alpha * A.B^T of
  * the stored tensors.  Every GEMM kernel of the library reads it in place as a K-major tensor-core operand (fused and
  * unfused, all kinds, same results bit for bit as with the transposed operand); the host-buffer and workspace-free entry
- * points take it too.  The node-list entry point has no such flag. */
+ * points take it too, the node-list entry point through comfuse_gemm_shape_t.flags. */
 #define COMFUSE_FLAG_B_ROW_MAJOR_NK 4u
 
 /* Runtime-parameter table of the op list.  bias, gamma, beta: bf16 device vectors of length N, shared by all batches;
@@ -319,6 +319,7 @@ typedef struct {
   int32_t batch, M, N, K;
   int64_t lda, ldb, ldy;
   int64_t batch_stride_a, batch_stride_b, batch_stride_y;  /* used when batch > 1 */
+  uint32_t flags;  /* 0, or COMFUSE_FLAG_B_ROW_MAJOR_NK: B stored [batch, N, K] (ldb >= K); any other bit: INVALID_ARG */
 } comfuse_gemm_shape_t;
 
 typedef enum {

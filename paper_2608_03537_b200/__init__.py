@@ -103,7 +103,7 @@ class FusionSpec(Structure):
 class GemmShape(Structure):
     _fields_ = [("batch", c_int32), ("M", c_int32), ("N", c_int32), ("K", c_int32),
                 ("lda", c_int64), ("ldb", c_int64), ("ldy", c_int64),
-                ("batch_stride_a", c_int64), ("batch_stride_b", c_int64), ("batch_stride_y", c_int64)]
+                ("batch_stride_a", c_int64), ("batch_stride_b", c_int64), ("batch_stride_y", c_int64), ("flags", ctypes.c_uint32)]
 
 
 class SpecPlan(Structure):
@@ -405,9 +405,12 @@ def make_spec(nodes, terminal, n_params=0, row_outputs=()) -> FusionSpec:
 
 
 def make_gemm_shape(batch, M, N, K, lda=None, ldb=None, ldy=None, batch_stride_a=None, batch_stride_b=None,
-                    batch_stride_y=None) -> GemmShape:
-    lda, ldb, ldy = lda or K, ldb or N, ldy or N
-    return GemmShape(batch, M, N, K, lda, ldb, ldy, batch_stride_a or M * lda, batch_stride_b or K * ldb, batch_stride_y or M * ldy)
+                    batch_stride_y=None, flags=0) -> GemmShape:
+    """Dense shapes by default; ``flags=FLAG_B_ROW_MAJOR_NK``: B is stored [batch, N, K]."""
+    b_nk = bool(int(flags) & FLAG_B_ROW_MAJOR_NK)
+    lda, ldb, ldy = lda or K, ldb or (K if b_nk else N), ldy or N
+    return GemmShape(batch, M, N, K, lda, ldb, ldy, batch_stride_a or M * lda, batch_stride_b or (N if b_nk else K) * ldb,
+                     batch_stride_y or M * ldy, int(flags))
 
 
 def spec_plan(spec: FusionSpec, shape: GemmShape) -> SpecPlan:
@@ -427,15 +430,17 @@ def gemm_spec_workspace_size(spec: FusionSpec, shape: GemmShape, fused=True) -> 
     return int(n.value)
 
 
-def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, workspace=None, stream=None):
+def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, workspace=None, stream=None, b_nk=False):
     """Enqueue Y = program(A.B): ``spec`` from make_spec, ``params`` the CUDA bf16 tensors of the parameter table
-    (row vectors [N], tensors [batch, M, N]), ``row_out`` the per-row output tensors (fp32, int32 for an arg max)."""
+    (row vectors [N], tensors [batch, M, N]), ``row_out`` the per-row output tensors (fp32, int32 for an arg max);
+    ``b_nk``: B is stored [batch, N, K]."""
     batched = A.dim() == 3
     batch = A.shape[0] if batched else 1
     M, K = A.shape[-2], A.shape[-1]
-    N = B.shape[-1]
+    N = B.shape[-2] if b_nk else B.shape[-1]
     shape = make_gemm_shape(batch, M, N, K, A.stride(-2), B.stride(-2), Y.stride(-2),
-                            A.stride(0) if batched else None, B.stride(0) if batched else None, Y.stride(0) if batched else None)
+                            A.stride(0) if batched else None, B.stride(0) if batched else None, Y.stride(0) if batched else None,
+                            flags=FLAG_B_ROW_MAJOR_NK if b_nk else 0)
     n = max(1, len(params))
     pp = (c_void_p * n)(*[None if t is None else t.data_ptr() for t in params])
     ld = (c_int64 * n)(*[0 if (t is None or t.dim() < 2) else t.stride(-2) for t in params])

@@ -217,15 +217,16 @@ comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only
 }  // namespace
 
 comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
-                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st) {
+                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st, bool b_nk) {
   const DeviceInfo* dev = nullptr;
   comfuse_status_t s = check_device(&dev);
   if (s != COMFUSE_OK) return s;
   GemmMaps maps;
   if (!make_gemm_maps(&maps, A, B, nullptr, Z, batch, M, N, K, lda, ldb, 0, N, batch_stride_a, batch_stride_b, 0,
-                      static_cast<long long>(M) * N))
+                      static_cast<long long>(M) * N, b_nk))
     return COMFUSE_ERR_CUDA;
   FusedParams p = {};
+  p.b_nk = b_nk ? 1 : 0;
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.mblocks = (M + 127) / 128;
   p.nblocks = 1;
@@ -241,15 +242,16 @@ comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, lon
 
 comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                       long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
-                                      const void* bias, float alpha, int activation, cudaStream_t st) {
+                                      const void* bias, float alpha, int activation, cudaStream_t st, bool b_nk) {
   const DeviceInfo* dev = nullptr;
   comfuse_status_t s = check_device(&dev);
   if (s != COMFUSE_OK) return s;
   GemmMaps maps;
   if (!make_gemm_maps(&maps, A, B, nullptr, Y, batch, M, N, K, lda, ldb, 0, ldy, batch_stride_a, batch_stride_b, 0,
-                      batch > 1 ? batch_stride_y : 0))
+                      batch > 1 ? batch_stride_y : 0, b_nk))
     return COMFUSE_ERR_CUDA;
   FusedParams p = {};
+  p.b_nk = b_nk ? 1 : 0;
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.mblocks = (M + 127) / 128;
   p.nblocks = 1;
@@ -268,9 +270,10 @@ comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long 
 comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
-                                   cudaStream_t st, bool query_only) {
+                                   cudaStream_t st, bool query_only, bool b_nk) {
   FusedParams p = {};
   p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.b_nk = b_nk ? 1 : 0;
   GemmMaps maps;
   if (query_only) {
     std::memset(&maps, 0, sizeof(maps));
@@ -281,7 +284,7 @@ comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda
   if (s != COMFUSE_OK) return s;
   const long long bsr = static_cast<long long>(M) * ldr;
   if (!make_gemm_maps(&maps, A, B, residual, Y, batch, M, N, K, lda, ldb, ldr, ldy, batch_stride_a, batch_stride_b, bsr,
-                      batch > 1 ? batch_stride_y : 0))
+                      batch > 1 ? batch_stride_y : 0, b_nk))
     return COMFUSE_ERR_CUDA;
   p.mblocks = (M + 127) / 128;
   p.nblocks = 1;

@@ -756,11 +756,14 @@ comfuse_status_t lower_row_program(const Analysis& an, int N, RowProgram& P, int
 comfuse_status_t validate_shape(const comfuse_gemm_shape_t* s) {
   if (!s) return COMFUSE_ERR_INVALID_ARG;
   if (s->batch < 1 || s->M < 1 || s->N < 1 || s->K < 1) return COMFUSE_ERR_INVALID_ARG;
-  if (s->lda < s->K || s->ldb < s->N || s->ldy < s->N) return COMFUSE_ERR_INVALID_ARG;
+  if (s->flags & ~COMFUSE_FLAG_B_ROW_MAJOR_NK) return COMFUSE_ERR_INVALID_ARG;
+  const bool b_nk = (s->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0;
+  if (s->lda < s->K || s->ldb < (b_nk ? s->K : s->N) || s->ldy < s->N) return COMFUSE_ERR_INVALID_ARG;
   if ((s->N & 7) || (s->K & 7) || (s->lda & 7) || (s->ldb & 7) || (s->ldy & 7)) return COMFUSE_ERR_ALIGNMENT;
   if (s->batch > 1) {
     if (s->batch_stride_a < static_cast<long long>(s->M - 1) * s->lda + s->K) return COMFUSE_ERR_INVALID_ARG;
-    if (s->batch_stride_b < static_cast<long long>(s->K - 1) * s->ldb + s->N) return COMFUSE_ERR_INVALID_ARG;
+    if (s->batch_stride_b < (b_nk ? static_cast<long long>(s->N - 1) * s->ldb + s->K : static_cast<long long>(s->K - 1) * s->ldb + s->N))
+      return COMFUSE_ERR_INVALID_ARG;
     if (s->batch_stride_y < static_cast<long long>(s->M - 1) * s->ldy + s->N) return COMFUSE_ERR_INVALID_ARG;
     if ((s->batch_stride_a & 7) || (s->batch_stride_b & 7) || (s->batch_stride_y & 7)) return COMFUSE_ERR_ALIGNMENT;
   }
@@ -777,7 +780,7 @@ comfuse_gemm_desc_t fused_desc(const comfuse_gemm_shape_t& s, const FusedMatch& 
   d.batch_stride_r = static_cast<long long>(s.M) * ldr;
   d.kind = m.kind;
   d.mask = m.causal ? COMFUSE_MASK_CAUSAL : COMFUSE_MASK_NONE;
-  d.alpha = m.alpha; d.eps = m.eps; d.fused = 1; d.flags = m.flags; d.softcap = m.softcap;
+  d.alpha = m.alpha; d.eps = m.eps; d.fused = 1; d.flags = m.flags | (s.flags & COMFUSE_FLAG_B_ROW_MAJOR_NK); d.softcap = m.softcap;
   return d;
 }
 
@@ -940,7 +943,7 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
     const FusedMatch& m = dc.match;
     return run_gemm_elementwise(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
                                 shape->batch_stride_b, shape->batch_stride_y, A, B, Y, m.bias >= 0 ? params[m.bias] : nullptr, m.alpha,
-                                m.activation, static_cast<cudaStream_t>(cuda_stream));
+                                m.activation, static_cast<cudaStream_t>(cuda_stream), (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0);
   }
   if (dc.fused) {
     const FusedMatch& m = dc.match;
@@ -969,7 +972,7 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
     const void* res = bd.tensor_param >= 0 ? params[bd.tensor_param] : nullptr;
     return run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
                              shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res,
-                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false);
+                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false, (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0);
   }
 
   // standard pathway: GEMM -> bf16 Z in the workspace -> row program
@@ -979,7 +982,7 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
   s = lower_row_program(an, shape->N, P, ni, ns);
   if (s != COMFUSE_OK) return s;
   s = gemm_to_bf16(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->batch_stride_a, shape->batch_stride_b, A, B,
-                   workspace, st);
+                   workspace, st, (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0);
   if (s != COMFUSE_OK) return s;
   P.batch = shape->batch; P.M = shape->M; P.N = shape->N;
   P.Z = static_cast<const uint16_t*>(workspace);

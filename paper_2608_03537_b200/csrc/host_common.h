@@ -85,13 +85,13 @@ namespace comfuse {
 comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
-                                   cudaStream_t st, bool query_only);
+                                   cudaStream_t st, bool query_only, bool b_nk = false);
 // Y = act(alpha * A . B + bias) (reduction-free epilogue), any N that is a multiple of 8; bias may be null.
 comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                       long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
-                                      const void* bias, float alpha, int activation, cudaStream_t st);
+                                      const void* bias, float alpha, int activation, cudaStream_t st, bool b_nk = false);
 // Z = bf16(A . B), dense [batch, M, N] (ld = N), with the plain tensor-core GEMM kernel; arguments already validated.
 comfuse_status_t gemm_to_bf16(int batch, int M, int N, int K, long long lda, long long ldb, long long batch_stride_a,
-                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st);
+                              long long batch_stride_b, const void* A, const void* B, void* Z, cudaStream_t st, bool b_nk = false);
 
 }  // namespace comfuse

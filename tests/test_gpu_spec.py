@@ -26,21 +26,23 @@ def _inputs(seed, batch, M, N, K, kinds):
     return A, B, params
 
 
-def _run(prog, A, B, params, fused, batch, M, N):
+def _run(prog, A, B, params, fused, batch, M, N, b_nk=False):
     fused = int(fused)
     dev = "cuda:0"
     spec = cf.make_spec(prog.nodes, prog.terminal, len(prog.param_kinds), prog.row_outputs)
     dA, dB = to_dev(A), to_dev(B)
+    if b_nk:
+        dB = dB.transpose(-1, -2).contiguous()      # the operand as a layer stores it: [N, K]
     dP = [to_dev(p) for p in params]
     Y = torch.full((batch, M, N) if batch > 1 else (M, N), float("nan"), dtype=torch.bfloat16, device=dev)
     rows = batch * M
     ro = [torch.full((rows,), -7, dtype=torch.int32 if prog.nodes[r][0] == "argmax" else torch.float32, device=dev)
           for r in prog.row_outputs]
-    shape = cf.make_gemm_shape(batch, M, N, A.shape[-1])
+    shape = cf.make_gemm_shape(batch, M, N, A.shape[-1], flags=cf.FLAG_B_ROW_MAJOR_NK if b_nk else 0)
     plan = cf.spec_plan(spec, shape)
     ws = torch.empty(max(16, cf.gemm_spec_workspace_size(spec, shape, fused)), dtype=torch.uint8, device=dev)
     before = cf.launch_count()
-    cf.gemm_spec(dA, dB, Y, spec, params=dP, row_out=ro, fused=fused, workspace=ws)
+    cf.gemm_spec(dA, dB, Y, spec, params=dP, row_out=ro, fused=fused, workspace=ws, b_nk=b_nk)
     torch.cuda.synchronize()
     assert cf.last_device_status() == cf.OK
     return Y, ro, plan, cf.launch_count() - before
@@ -95,6 +97,21 @@ def test_program_lowers_to_the_fused_kernel_and_matches_the_oracle(name):
     err = np.abs(to_f64(Y) - Yref)
     assert np.isfinite(err).all() and err.max() <= tmax and err.mean() <= tmean, (err.max(), err.mean())
     _check_rows(prog, ro, Rref, Yref)
+
+
+@pytest.mark.parametrize("fused", [1, 2, 0])
+@pytest.mark.parametrize("name", ["layernorm_relu", "rmsnorm_max", "softmax_causal"])
+def test_second_operand_stored_n_by_k_on_every_pathway(name, fused):
+    """comfuse_gemm_shape_t.flags = COMFUSE_FLAG_B_ROW_MAJOR_NK: the compiled kind (1), the on-chip interpreter (2) and the
+    GEMM + row-program pair (0) read B [N, K] in place and give the same bits as with B [K, N]."""
+    prog, batch, M, N, K, kind, tmax, tmean = CASES[name]
+    A, B, params = _inputs(37, batch, M, N, K, prog.param_kinds)
+    Y0, ro0, plan0, _ = _run(prog, A, B, params, fused, batch, M, N)
+    Y1, ro1, plan1, _ = _run(prog, A, B, params, fused, batch, M, N, b_nk=True)
+    assert plan0.path == plan1.path
+    assert torch.equal(Y0.view(torch.int16), Y1.view(torch.int16))
+    for a, b in zip(ro0, ro1):
+        assert torch.equal(a, b)
 
 
 @pytest.mark.parametrize("name", sorted(CASES))
