@@ -44,6 +44,41 @@ def f64(w: wl.Workload, name: str, rows=None):
 
 
 # --------------------------------------------------------------------------------------------- GPU side
+# Canary pads: every output (and the workspace) of prepare_gpu / run_gpu sits inside a larger allocation whose margins hold a
+# fixed bit pattern; check_outputs (or check_canaries) verifies that no launch wrote outside the tensor it was given.
+GUARD_BYTES = 4096
+CANARY = 0x5A
+
+
+def guarded(shape, dtype, fill, device):
+    """A contiguous tensor of `shape` with GUARD_BYTES of canary before and after it in the same allocation."""
+    n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+    pad = (-n) % 256
+    flat = torch.full((GUARD_BYTES + n + pad + GUARD_BYTES,), CANARY, dtype=torch.uint8, device=device)
+    t = flat[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(*shape)
+    t.fill_(fill)
+    t._guard = (flat, n)
+    return t
+
+
+def check_canaries(tensors, label=""):
+    """Every guarded tensor among `tensors`: the bytes around it still hold the canary."""
+    for name, t in (tensors.items() if isinstance(tensors, dict) else enumerate(tensors)):
+        for what, u in ((f"output {name}", t), (f"the workspace of {name}", getattr(t, "_guard_ws", None))):
+            g = getattr(u, "_guard", None) if u is not None else None
+            if g is None:
+                continue
+            flat, n = g
+            lead = flat[:GUARD_BYTES]
+            tail = flat[GUARD_BYTES + n:]
+            assert bool((lead == CANARY).all().item()), f"{label}: bytes in front of {what} were overwritten"
+            assert bool((tail == CANARY).all().item()), f"{label}: bytes behind {what} were overwritten"
+
+
+def _guarded_workspace(nbytes, device):
+    ws = guarded((max(int(nbytes), 16),), torch.uint8, 0xEE, device)
+    return ws
+
 def prepare_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True):
     """Allocate the outputs and the workspace of one workload once.  Returns (outputs on device, launch): launch()
     enqueues one call of the library on the current stream and nothing else, so that calls can be queued back to back."""
@@ -51,23 +86,26 @@ def prepare_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True
     d = w.dims
     fill = float("nan") if poison else 0.0
     if w.kind == wl.KIND_B2B_SOFTMAX_ATTENTION:
-        O = torch.full((d["batch"], d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
+        O = guarded((d["batch"], d["M"], d["N2"]), torch.bfloat16, fill, dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, fused, cf.B2B_SOFTMAX_ATTENTION, d["batch"], w.scalars["alpha"])
-        ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
+        ws = _guarded_workspace(cf.b2b_workspace_size(desc), dev)
+        O._guard_ws = ws
         return {"Y": O}, lambda: cf.b2b_attention(T["X"], T["W1"], T["W2"], O, alpha=w.scalars["alpha"], fused=fused, workspace=ws)
     if w.kind == wl.KIND_B2B_MLP_RELU:
-        O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
+        O = guarded((d["M"], d["N2"]), torch.bfloat16, fill, dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], 0.0, fused, cf.B2B_MLP_RELU)
-        ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
+        ws = _guarded_workspace(cf.b2b_workspace_size(desc), dev)
+        O._guard_ws = ws
         return {"Y": O}, lambda: cf.b2b_mlp_relu(T["X"], T["W1"], T.get("b1"), T["W2"], T.get("b2"), O, fused=fused, workspace=ws)
     if w.kind == wl.KIND_B2B_MLP_LAYERNORM:
-        O = torch.full((d["M"], d["N2"]), fill, dtype=torch.bfloat16, device=dev)
+        O = guarded((d["M"], d["N2"]), torch.bfloat16, fill, dev)
         desc = cf.make_b2b_desc(d["M"], d["K"], d["N1"], d["N2"], w.scalars["eps"], fused)
-        ws = torch.empty(max(cf.b2b_workspace_size(desc), 16), dtype=torch.uint8, device=dev)
+        ws = _guarded_workspace(cf.b2b_workspace_size(desc), dev)
+        O._guard_ws = ws
         return {"Y": O}, lambda: cf.b2b_gemm(T["X"], T["W1"], T["b1"], T["W2"], T["b2"], O, gamma=T.get("gamma"), beta=T.get("beta"),
                                              eps=w.scalars["eps"], fused=fused, workspace=ws)
     shape = (d["batch"], d["M"], d["N"]) if "batch" in d else (d["M"], d["N"])
-    Y = torch.full(shape, fill, dtype=torch.bfloat16, device=dev)
+    Y = guarded(shape, torch.bfloat16, fill, dev)
     out = {"Y": Y}
     kw = {}
     if w.kind == wl.KIND_BIAS_RES_LAYERNORM:
@@ -76,8 +114,8 @@ def prepare_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True
                   alpha=w.scalars["alpha"], eps=w.scalars["eps"])
     elif w.kind == wl.KIND_BIAS_GELU_RES_RMSNORM_MAX:
         kind = cf.EPI_BIAS_GELU_RES_RMSNORM_MAX
-        out["row_max"] = torch.full(shape[:-1], fill, dtype=torch.float32, device=dev)
-        out["row_argmax"] = torch.full(shape[:-1], -1, dtype=torch.int32, device=dev)
+        out["row_max"] = guarded(shape[:-1], torch.float32, fill, dev)
+        out["row_argmax"] = guarded(shape[:-1], torch.int32, -1, dev)
         kw = dict(bias=T.get("bias"), residual=T.get("residual"), gamma=T.get("gamma"), alpha=w.scalars["alpha"],
                   eps=w.scalars["eps"], row_max=out["row_max"], row_argmax=out["row_argmax"])
     else:
@@ -90,7 +128,8 @@ def prepare_gpu(w: wl.Workload, T: dict, fused: bool = True, poison: bool = True
     desc = cf.make_gemm_desc(T["A"], T["B"], Y, kind, residual=kw.get("residual"), alpha=kw.get("alpha", 1.0),
                              eps=kw.get("eps", 1e-5), mask=kw.get("mask", cf.MASK_NONE), fused=fused, flags=flags,
                              softcap=kw["softcap"])
-    ws = torch.empty(max(cf.workspace_size(desc), 16), dtype=torch.uint8, device=dev)
+    ws = _guarded_workspace(cf.workspace_size(desc), dev)
+    Y._guard_ws = ws
     return out, lambda: cf.gemm_epilogue(T["A"], T["B"], Y, kind, fused=fused, workspace=ws, **kw)
 
 
@@ -154,6 +193,7 @@ def check_outputs(w: wl.Workload, got: dict, ref: dict, rows=None, batches=None,
     `softmax_tol`: 2e-3 for the fused kernel; the unfused path exponentiates bf16-rounded scores (relative error
     2^-9 on |score| up to ~4 after scaling), which alone moves a probability near 0.5 by up to ~4e-3, so the tests
     give it 1e-2 and say so.  `norm_tol`: max-abs bound of normalised outputs (3e-2 unless a caller says otherwise)."""
+    check_canaries(got, label)
     Y = got["Y"]
     if batches is not None:
         Y = Y[list(batches)]
