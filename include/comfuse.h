@@ -39,7 +39,9 @@ typedef enum {
   COMFUSE_ERR_WORKSPACE = 4,    /* workspace NULL or smaller than comfuse_*_workspace_size() reports      */
   COMFUSE_ERR_ARCH = 5,         /* current device is not compute capability 10.x                           */
   COMFUSE_ERR_CUDA = 6,         /* a CUDA runtime / driver call failed (launch, tensor-map encode, ...)   */
-  COMFUSE_ERR_TIMEOUT = 7       /* a bounded device-side wait expired (reported by last_device_status)    */
+  COMFUSE_ERR_TIMEOUT = 7,      /* a bounded device-side wait expired (reported by last_device_status)    */
+  COMFUSE_ERR_BOUNDS = 8        /* checked build only (-DCOMFUSE_CHECKED): a bounds predicate inside a kernel failed;
+                                   the access was skipped (reported by last_device_status)                 */
 } comfuse_status_t;
 
 /* The memory-intensive subgraph fused behind the GEMM, as a fixed, topologically ordered op list
@@ -230,7 +232,8 @@ comfuse_status_t comfuse_b2b_gemm_host(const comfuse_b2b_desc_t* desc, const voi
                                        void* cuda_stream);
 
 /* Synchronises `cuda_stream`, then returns and clears the device status word of the current device:
- * COMFUSE_OK, COMFUSE_ERR_TIMEOUT, or COMFUSE_ERR_CUDA if the stream reports an error. */
+ * COMFUSE_OK, COMFUSE_ERR_TIMEOUT, COMFUSE_ERR_BOUNDS (checked build only), or COMFUSE_ERR_CUDA if the stream reports an
+ * error. */
 comfuse_status_t comfuse_last_device_status(void* cuda_stream);
 
 /* Number of kernels this library has launched in this process since it was loaded (for accounting). */
@@ -242,6 +245,13 @@ uint64_t comfuse_launch_count(void);
  * If `expired_waits` (a HOST pointer) is not NULL the call synchronises the stream and stores how many threads saw an
  * expired or aborted wait (all 64). */
 comfuse_status_t comfuse_selftest_bounded_wait(uint32_t timeout_ms, void* cuda_stream, uint32_t* expired_waits);
+
+/* Checked-build self-test (the paper has no counterpart).  Launches one small kernel that evaluates a bounds predicate
+ * which is false, in front of an access it therefore skips.  In a library built with -DCOMFUSE_CHECKED the device status
+ * word then reads COMFUSE_ERR_BOUNDS; in the ordinary build the predicates are compiled out, the kernel does nothing and
+ * the status stays COMFUSE_OK.  `*checked_build` (a HOST pointer, may be NULL) receives 1 or 0 accordingly.  Nothing is
+ * read or written out of bounds in either build. */
+comfuse_status_t comfuse_selftest_bounds_predicate(void* cuda_stream, int32_t* checked_build);
 
 const char* comfuse_status_string(comfuse_status_t status);
 

@@ -24,10 +24,11 @@ import os
 from ctypes import POINTER, Structure, byref, c_float, c_int32, c_int64, c_size_t, c_uint64, c_void_p
 
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG_DIR, "libcomfuse.so")
+LIB_PATH = os.environ.get("COMFUSE_LIB") or os.path.join(_PKG_DIR, "libcomfuse.so")   # COMFUSE_LIB: e.g. the checked build
 
 # status codes / enums of include/comfuse.h
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
+ERR_BOUNDS = 8   # checked build only: a bounds predicate failed, the access was skipped
 EPI_BIAS_RES_LAYERNORM, EPI_BIAS_GELU_RES_RMSNORM_MAX, EPI_SCALE_MASK_SOFTMAX = 0, 1, 2
 EPI_BIAS_ACTIVATION = 3   # reduction-free epilogue; reached through gemm_spec only
 MASK_NONE, MASK_CAUSAL, MASK_ADDITIVE = 0, 1, 2
@@ -49,6 +50,7 @@ EXPORTED_SYMBOLS = (
     "comfuse_spec_plan",
     "comfuse_gemm_spec_workspace_size",
     "comfuse_gemm_spec",
+    "comfuse_selftest_bounds_predicate",
     "comfuse_last_device_status",
     "comfuse_launch_count",
     "comfuse_selftest_bounded_wait",
@@ -164,6 +166,8 @@ def lib() -> ctypes.CDLL:
         L.comfuse_last_device_status.restype = c_int32
         L.comfuse_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, POINTER(ctypes.c_uint32)]
         L.comfuse_selftest_bounded_wait.restype = c_int32
+        L.comfuse_selftest_bounds_predicate.argtypes = [c_void_p, POINTER(c_int32)]
+        L.comfuse_selftest_bounds_predicate.restype = c_int32
         L.comfuse_launch_count.argtypes = []
         L.comfuse_launch_count.restype = c_uint64
         L.comfuse_status_string.argtypes = [c_int32]
@@ -454,7 +458,7 @@ def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, w
 
 
 def last_device_status(stream=None) -> int:
-    """Synchronise the stream and return (and clear) the device status word: OK or ERR_TIMEOUT."""
+    """Synchronise the stream and return (and clear) the device status word: OK, ERR_TIMEOUT, or (checked build) ERR_BOUNDS."""
     return int(lib().comfuse_last_device_status(_stream(stream)))
 
 
@@ -466,6 +470,16 @@ def selftest_bounded_wait(timeout_ms: int = 20, stream=None) -> int:
     if st != OK:
         raise ComfuseError(st, "comfuse_selftest_bounded_wait")
     return int(n.value)
+
+
+def selftest_bounds_predicate(stream=None) -> bool:
+    """Run the bounds-predicate self-test kernel; returns whether the loaded library is the checked build.  In that build
+    the device status word reads ERR_BOUNDS afterwards, in the ordinary build OK; no access is out of bounds in either."""
+    flag = ctypes.c_int32(-1)
+    st = lib().comfuse_selftest_bounds_predicate(_stream(stream), byref(flag))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_selftest_bounds_predicate")
+    return bool(flag.value)
 
 
 def launch_count() -> int:

@@ -496,7 +496,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       fence_proxy_async_smem();  // the staged rows are visible to the TMA store
       __syncwarp();
       if (warp == 2 + kB2bEpiWarps && lane == 0 && i < 20) B2B_TRACE_AT(102 + 3 * i);
-      if (lane == 0) {
+      if (lane == 0 && COMFUSE_IN_BOUNDS(m0 >= 0 && m0 + q * 32 < p.mpairs * 256 && bz >= 0 && bz < p.batch, p.status)) {
         tma_store_3d(&tmO, box0 + q * 4096, 0, m0 + q * 32, bz);
         tma_store_3d(&tmO, box1 + q * 4096, 64, m0 + q * 32, bz);
         tma_store_commit();

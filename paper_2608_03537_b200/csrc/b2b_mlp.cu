@@ -482,7 +482,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         store_row_chunks(pk, x_addr(i & 1, hh >> 1), row, (hh & 1) * 4);
         fence_proxy_async_smem();
         named_barrier_sync(3 + q, 128);
-        if (hh == 0 && lane == 0) {
+        if (hh == 0 && lane == 0 && COMFUSE_IN_BOUNDS(m0 >= 0 && m0 < p.mpairs * 256 && bz >= 0 && bz < p.batch, p.status)) {
           tma_store_3d(&tmO, x_addr(i & 1, 0) + q * 32 * 128, 0, m0, bz);
           tma_store_3d(&tmO, x_addr(i & 1, 1) + q * 32 * 128, 64, m0, bz);
           tma_store_commit();
@@ -576,7 +576,8 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           if (f & 1) {
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) tma_store_3d(&tmO, x_addr(i & 1, f >> 1) + q * 32 * 128, (f >> 1) * 64, m0, bz);
+            if (lane == 0 && COMFUSE_IN_BOUNDS(m0 >= 0 && m0 < p.mpairs * 256 && bz >= 0 && bz < p.batch, p.status))
+              tma_store_3d(&tmO, x_addr(i & 1, f >> 1) + q * 32 * 128, (f >> 1) * 64, m0, bz);
           }
         }
         if (lane == 0) {

@@ -406,8 +406,10 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       named_barrier_sync(3, kEpiThreads);
       if (store_thread) {
         const int m0 = tile_m0(it);
-        tma_store_3d(&tmO, s_base, 0, m0, 0);
-        tma_store_3d(&tmO, s_base + kBoxBytes, 64, m0, 0);
+        if (COMFUSE_IN_BOUNDS(m0 >= 0 && m0 < p.mpairs * 256, p.status)) {
+          tma_store_3d(&tmO, s_base, 0, m0, 0);
+          tma_store_3d(&tmO, s_base + kBoxBytes, 64, m0, 0);
+        }
         tma_store_commit();
       }
     };

@@ -320,6 +320,7 @@ const char* comfuse_status_string(comfuse_status_t s) {
     case COMFUSE_ERR_ARCH: return "device is not compute capability 10.x";
     case COMFUSE_ERR_CUDA: return "CUDA call failed";
     case COMFUSE_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case COMFUSE_ERR_BOUNDS: return "a bounds predicate of the checked build failed (access skipped)";
     default: return "unknown status";
   }
 }
@@ -638,7 +639,7 @@ comfuse_status_t comfuse_last_device_status(void* cuda_stream) {
   if (word != 0) {
     const unsigned int zero = 0;
     if (cudaMemcpy(dev->status_word, &zero, sizeof(zero), cudaMemcpyHostToDevice) != cudaSuccess) return COMFUSE_ERR_CUDA;
-    return COMFUSE_ERR_TIMEOUT;
+    return (word & 1u) ? COMFUSE_ERR_TIMEOUT : COMFUSE_ERR_BOUNDS;
   }
   return COMFUSE_OK;
 }

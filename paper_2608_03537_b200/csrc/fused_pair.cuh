@@ -402,6 +402,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
               if (!(p.trace_flags & 1))
 #endif
+              if (COMFUSE_IN_BOUNDS(col >= 0 && col < p.N && (col & 7) == 0 && m0 + q * 32 >= 0 && b >= 0 && b < p.batch, p.status))
               tma_store_3d_hint(&tmY, ring_box(e, kk), col, m0 + q * 32, b, once);
               tma_store_commit();
               ++kk;
@@ -412,6 +413,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
             if (!(p.trace_flags & 1))
 #endif
+            if (COMFUSE_IN_BOUNDS(col >= 0 && col < p.N && (col & 7) == 0 && m0 + q * 32 >= 0 && b >= 0 && b < p.batch, p.status))
             tma_store_3d_hint(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, m0 + q * 32, b, once);
             tma_store_commit();
             if (n >= static_cast<uint32_t>(D)) {
@@ -722,6 +724,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (p.wide) {
           if (crank == 0 && h == 0 && valid) {
             const int nb = (ncta0 / (CN * BN));
+            if (COMFUSE_IN_BOUNDS(nb >= 0 && nb < p.nblocks && grow >= 0 && grow < p.M && b >= 0 && b < p.batch, p.status))
             p.wide_partials[(static_cast<long long>(b) * p.M + grow) * p.nblocks + nb] = tot;
           }
           continue;  // the row is finished by the second kernel
@@ -795,8 +798,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                                    s_stats, bar_stats, row, h, crank, xpar, xphase, w, 2u, pm, p.leader_reduce != 0);
           if (crank == 0 && h == 0 && valid) {
             const long long o = static_cast<long long>(b) * p.M + grow;
-            p.row_max[o] = mx.x;
-            p.row_argmax[o] = __float_as_int(mx.y);
+            if (COMFUSE_IN_BOUNDS(o >= 0 && o < static_cast<long long>(p.batch) * p.M, p.status)) {
+              p.row_max[o] = mx.x;
+              p.row_argmax[o] = __float_as_int(mx.y);
+            }
           }
         }
       } else if constexpr (EPI == EPI_PROGRAM) {

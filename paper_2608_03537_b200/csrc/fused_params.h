@@ -120,7 +120,7 @@ struct FusedParams {
   // column block only, stores the un-normalised values and writes the block's partial statistic of each row to
   // wide_partials[(batch * M + row) * nblocks + block]; a second kernel merges the partials and rescales in place.
   const uint16_t* mask;  // softmax kinds: additive bf16 mask [M, N] (ld = N), shared by all batches, or null
-  int b_nk;              // the B operand is stored [N, K] (K-major tensor-core operand; row softmax kernel only)
+  int b_nk;              // the B operand is stored [N, K] (K-major tensor-core operand)
   int wide;
   int wide_block;   // columns per block of the two-kernel form (the instantiation that runs each block)
   float2* wide_partials;

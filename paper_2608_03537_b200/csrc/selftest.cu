@@ -30,6 +30,17 @@ __global__ void bounded_wait_selftest_kernel(unsigned int* status, unsigned long
 
 __device__ unsigned int g_selftest_counter = 0;
 
+// One element past the end of a 32-element array: the predicate is false, the store is skipped (checked build), or the
+// predicate is compiled out and the kernel's own `false &&` keeps the store from happening (ordinary build).
+__global__ void bounds_predicate_selftest_kernel(unsigned int* status, unsigned int* arr, int n) {
+  const int i = n + static_cast<int>(threadIdx.x);  // always >= n
+#ifdef COMFUSE_CHECKED
+  if (COMFUSE_IN_BOUNDS(i < n, status)) arr[i] = 1u;
+#else
+  (void)status; (void)arr; (void)i;
+#endif
+}
+
 }  // namespace
 }  // namespace comfuse
 
@@ -54,5 +65,23 @@ extern "C" comfuse_status_t comfuse_selftest_bounded_wait(uint32_t timeout_ms, v
     if (cudaStreamSynchronize(st) != cudaSuccess) return COMFUSE_ERR_CUDA;
     *expired_waits = h;
   }
+  return COMFUSE_OK;
+}
+
+extern "C" comfuse_status_t comfuse_selftest_bounds_predicate(void* cuda_stream, int32_t* checked_build) {
+  const DeviceInfo* dev = current_device_info();
+  if (!dev) return COMFUSE_ERR_CUDA;
+  if (dev->cc_major != 10) return COMFUSE_ERR_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  void* counter = nullptr;
+  if (cudaGetSymbolAddress(&counter, g_selftest_counter) != cudaSuccess) return COMFUSE_ERR_CUDA;
+  count_launch();
+  bounds_predicate_selftest_kernel<<<1, 32, 0, st>>>(dev->status_word, static_cast<unsigned int*>(counter), 1);
+  if (cudaGetLastError() != cudaSuccess) return COMFUSE_ERR_CUDA;
+#ifdef COMFUSE_CHECKED
+  if (checked_build) *checked_build = 1;
+#else
+  if (checked_build) *checked_build = 0;
+#endif
   return COMFUSE_OK;
 }

@@ -12,6 +12,16 @@ namespace comfuse {
 
 // Device status word (bit set = event happened since the last read).  Lives in the module: no allocation.
 constexpr unsigned int kStatusTimeout = 1u;
+constexpr unsigned int kStatusBounds = 2u;
+
+// Checked build (-DCOMFUSE_CHECKED): `if (COMFUSE_IN_BOUNDS(index < limit, status)) access;` -- a predicate that fails
+// records kStatusBounds in the device status word and the access is skipped; nothing traps.  In the ordinary build the
+// predicate is compiled out (the surrounding logic already guarantees it).
+#ifdef COMFUSE_CHECKED
+#define COMFUSE_IN_BOUNDS(cond, status_ptr) ((cond) || (atomicOr((status_ptr), ::comfuse::kStatusBounds), false))
+#else
+#define COMFUSE_IN_BOUNDS(cond, status_ptr) (true)
+#endif
 
 // What a bounded wait needs: the CTA-shared abort flag, the device status word and the time limit.
 struct WaitCtx {

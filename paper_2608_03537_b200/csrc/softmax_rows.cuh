@@ -240,6 +240,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #ifdef COMFUSE_TRACE
         if (!(p.trace_flags & 1))
 #endif
+        if (COMFUSE_IN_BOUNDS(col >= 0 && col < p.N && (col & 7) == 0 && mpair0 >= 0 && b >= 0 && b < p.batch, p.status))
         tma_store_3d_hint(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, mpair0 + static_cast<int>(pm) * 128 + q * 32, b, stream_out);
         tma_store_commit();
         if (n >= static_cast<uint32_t>(D)) {
@@ -273,6 +274,7 @@ softmax_rows_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #ifdef COMFUSE_TRACE
             if (!(p.trace_flags & 4))
 #endif
+            if (COMFUSE_IN_BOUNDS(col >= 0 && (col & 7) == 0 && y0 >= 0 && b >= 0 && b < p.batch, p.status))
             tma_store_3d_hint(&tmY, smem_base + Cfg::OFF_ZERO, col, y0 + (i & 3) * 32, b, stream_out);
             tma_store_commit();
           }

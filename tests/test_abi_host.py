@@ -38,8 +38,8 @@ def test_library_exports_every_declared_function():
 
 def test_status_strings_and_launch_counter():
     L = cf.lib()
-    texts = [L.comfuse_status_string(i).decode() for i in range(8)]
-    assert texts[0] == "ok" and len(set(texts)) == 8
+    texts = [L.comfuse_status_string(i).decode() for i in range(9)]
+    assert texts[0] == "ok" and len(set(texts)) == 9
     assert "unknown" in L.comfuse_status_string(99).decode()
     assert cf.launch_count() >= 0
 
