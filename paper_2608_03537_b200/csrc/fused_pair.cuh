@@ -809,7 +809,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // ONE interpreter loop (one copy of every operation's code: the kernel is instruction-fetch bound otherwise)
         // runs the pass's micro-instruction stream on each 32-column fragment: v is the working fragment, x the resident one.
         static_assert(ESUB == 1, "stage programs run on single-unit tiles");
+        // `sp` is the program's structure, `rp` its run-time part (immediates, row-output pointers).  In the ordinary build
+        // both are the kernel parameter and the loops below are an interpreter; when the program is compiled into the
+        // kernel (COMFUSE_COMPILED_PROGRAM: a constant table in front of this header, Sec. 5's code generation), the sweep and
+        // instruction loops unroll and every dispatch below folds to the one operation it selects.
+        const StageProgram& rp = p.program;
+#ifdef COMFUSE_COMPILED_PROGRAM
+        const StageProgram& sp = kCompiledProgram;
+#define COMFUSE_PROGRAM_LOOP _Pragma("unroll")
+#else
         const StageProgram& sp = p.program;
+#define COMFUSE_PROGRAM_LOOP _Pragma("unroll 1")
+#endif
         float sc[kStageMaxScalars];  // this row's scalars (reduction results and arithmetic on them)
 #pragma unroll
         for (int i = 0; i < kStageMaxScalars; ++i) sc[i] = 0.f;
@@ -817,7 +828,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         float racc[kStageMaxRed];  // thread-local partials (value; column for an arg max); indexed at run time
         int ridx[kStageMaxRed];
         float2 sc_topk[kStageMaxRed];  // Top-K: the row's pick of round 0 (value, column bits), kept until its later rounds run
-#pragma unroll 1
+COMFUSE_PROGRAM_LOOP
         for (int r = 0; r < kStageMaxRed; ++r) {
           const int op = r < sp.n_red ? sp.red[r].op : COMFUSE_OP_RED_SUM;
           racc[r] = op == COMFUSE_OP_RED_PROD ? 1.f : (op == COMFUSE_OP_RED_MAX || op == COMFUSE_OP_RED_ARGMAX) ? -INFINITY
@@ -837,14 +848,18 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
         // A sweep runs a micro-instruction range over this thread's fragments.  Ordinary sweeps are the passes; behind a
         // pass's merges every Top-K reduction of that pass adds K - 1 sweeps of its own code range (`topk_r` >= 0), each
-        // looking for the best element behind the previous pick (pv, pc).
-        int pass = 0, topk_r = -1, topk_round = 0;
+        // looking for the best element behind the previous pick (pv, pc).  The host laid the order down in sp.sweep[].
         float pv = 0.f;
         int pc = 0;
-#pragma unroll 1
-        while (pass < sp.n_passes) {
-          const int i0 = topk_r >= 0 ? sp.red[topk_r].code_lo : sp.pass_off[pass];
-          const int i1 = topk_r >= 0 ? sp.red[topk_r].code_hi : sp.pass_off[pass + 1];
+COMFUSE_PROGRAM_LOOP
+        for (int s = 0; s < sp.n_sweeps; ++s) {
+          const int pass = sp.sweep[s].pass, topk_r = sp.sweep[s].topk_r, topk_round = sp.sweep[s].topk_round;
+          const int i0 = sp.sweep[s].i0, i1 = sp.sweep[s].i1;
+          if (topk_r >= 0) {
+            if (topk_round == 1) { pv = sc_topk[topk_r].x; pc = __float_as_int(sc_topk[topk_r].y); }
+            racc[topk_r] = -INFINITY;
+            ridx[topk_r] = 0x7FFFFFFF;
+          }
 #pragma unroll 1
           for (int f = 0; f < kFrags; ++f) {
             const int g = h + EPW * (f >> 1), half = f & 1;
@@ -867,14 +882,14 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
               for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(vb[j]); x[j] = v[j]; }
             }
-#pragma unroll 1
+COMFUSE_PROGRAM_LOOP
             for (int i = i0; i < i1; ++i) {
               const ChainInstr ci = sp.code[i];
               const int op = ci.op;
               if (op >= COMFUSE_OP_ADD && op <= kChainRdiv) {
                 // ---- binary with a row-uniform operand (constant or per-row scalar): applied directly
                 if (ci.operand == CHO_SCALAR || ci.operand == CHO_CONST) {
-                  const float sv = scalar_get(ci.operand, ci.index, ci.imm);
+                  const float sv = scalar_get(ci.operand, ci.index, rp.code[i].imm);
                   const float2 s2 = make_float2(sv, sv);
                   switch (op) {
                     case COMFUSE_OP_ADD:
@@ -1148,34 +1163,20 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             pc = __float_as_int(tot.y);
             if (crank == 0 && h == 0 && valid) {
               const long long o = (static_cast<long long>(b) * p.M + grow) * sp.red[topk_r].k + topk_round;
+COMFUSE_PROGRAM_LOOP
               for (int q2 = 0; q2 < sp.n_row_out; ++q2)
                 if (sp.out[q2].topk_red == topk_r + 1) {
-                  if (sp.out[q2].is_int) static_cast<int*>(sp.out[q2].ptr)[o] = pc;
-                  else static_cast<float*>(sp.out[q2].ptr)[o] = pv;
+                  if (sp.out[q2].is_int) static_cast<int*>(rp.out[q2].ptr)[o] = pc;
+                  else static_cast<float*>(rp.out[q2].ptr)[o] = pv;
                 }
             }
-            if (++topk_round >= sp.red[topk_r].k) {
-              int nxt = -1;
-              for (int r = topk_r + 1; r < sp.n_red; ++r)
-                if (nxt < 0 && sp.red[r].pass == pass && sp.red[r].k > 1) nxt = r;
-              topk_r = nxt;
-              topk_round = 1;
-              if (topk_r >= 0) { pv = sc_topk[topk_r].x; pc = __float_as_int(sc_topk[topk_r].y); }
-            }
-            if (topk_r >= 0) {
-              racc[topk_r] = -INFINITY;
-              ridx[topk_r] = 0x7FFFFFFF;
-            } else {
-              if (pass == sp.n_passes - 1) release_accumulator(0);
-              ++pass;
-            }
+            if (sp.sweep[s].release) release_accumulator(0);
             continue;
           }
           if (pass == 0) tmem_st_wait();
           // ---- stage boundary: merges of the pass's reductions in program order (every CTA of the group makes the same
           // calls), then the per-row arithmetic that depends on them
-          int first_topk = -1;
-#pragma unroll 1
+COMFUSE_PROGRAM_LOOP
           for (int r = 0; r < sp.n_red; ++r) {
             if (sp.red[r].pass != pass) continue;
             const int op = sp.red[r].op;
@@ -1192,25 +1193,25 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               sc_topk[r] = tot;
               if (crank == 0 && h == 0 && valid) {
                 const long long o = (static_cast<long long>(b) * p.M + grow) * sp.red[r].k;
+COMFUSE_PROGRAM_LOOP
                 for (int q2 = 0; q2 < sp.n_row_out; ++q2)
                   if (sp.out[q2].topk_red == r + 1) {
-                    if (sp.out[q2].is_int) static_cast<int*>(sp.out[q2].ptr)[o] = __float_as_int(tot.y);
-                    else static_cast<float*>(sp.out[q2].ptr)[o] = tot.x;
+                    if (sp.out[q2].is_int) static_cast<int*>(rp.out[q2].ptr)[o] = __float_as_int(tot.y);
+                    else static_cast<float*>(rp.out[q2].ptr)[o] = tot.x;
                   }
               }
-              if (sp.red[r].k > 1 && first_topk < 0) first_topk = r;
               continue;
             }
             float val = op == COMFUSE_OP_RED_ARGMAX ? static_cast<float>(__float_as_int(tot.y)) : tot.x;
             if (op == COMFUSE_OP_RED_MEAN) val *= 1.f / static_cast<float>(CN * BN);
             scalar_set(sp.red[r].dst, val);
           }
-#pragma unroll 1
+COMFUSE_PROGRAM_LOOP
           for (int i = 0; i < sp.n_scalar_instr; ++i) {
             const ScalarInstr si = sp.sc[i];
             if (si.after_pass != pass) continue;
-            const float a = scalar_get(si.a_kind, si.a, si.a_imm);
-            const float bq = scalar_get(si.b_kind, si.b, si.b_imm);
+            const float a = scalar_get(si.a_kind, si.a, rp.sc[i].a_imm);
+            const float bq = scalar_get(si.b_kind, si.b, rp.sc[i].b_imm);
             float rv;
             switch (si.op) {
               case COMFUSE_OP_NEG: rv = -a; break;
@@ -1234,27 +1235,19 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
             scalar_set(si.dst, rv);
           }
-          if (first_topk >= 0) {  // the pass's Top-K reductions take their further rounds before the next pass
-            topk_r = first_topk;
-            topk_round = 1;
-            pv = sc_topk[topk_r].x;
-            pc = __float_as_int(sc_topk[topk_r].y);
-            racc[topk_r] = -INFINITY;
-            ridx[topk_r] = 0x7FFFFFFF;
-          } else {
-            if (pass == sp.n_passes - 1) release_accumulator(0);
-            ++pass;
-          }
+          if (sp.sweep[s].release) release_accumulator(0);
         }
         if (crank == 0 && h == 0 && valid) {
           const long long o = static_cast<long long>(b) * p.M + grow;
+COMFUSE_PROGRAM_LOOP
           for (int r = 0; r < sp.n_row_out; ++r) {
             if (sp.out[r].topk_red) continue;  // delivered round by round
             const float val = scalar_get(CHO_SCALAR, sp.out[r].scalar, 0.f);
-            if (sp.out[r].is_int) static_cast<int*>(sp.out[r].ptr)[o] = static_cast<int>(val);
-            else static_cast<float*>(sp.out[r].ptr)[o] = val;
+            if (sp.out[r].is_int) static_cast<int*>(rp.out[r].ptr)[o] = static_cast<int>(val);
+            else static_cast<float*>(rp.out[r].ptr)[o] = val;
           }
         }
+#undef COMFUSE_PROGRAM_LOOP
       } else {  // EPI_SOFTMAX
         // log2 domain: t = Acc * (alpha * log2 e), so exp(x - m) = 2^(t - m_t)
         // with a soft-cap the accumulators are mapped to capped log2-domain scores right after they are loaded, and sc = 1

@@ -79,6 +79,19 @@ struct StageRowOutput {
 constexpr int kStageMaxCode = 80, kStageMaxRed = 6, kStageMaxScalarInstr = 12, kStageMaxScalars = 16, kStageMaxRowOut = 6,
               kStageMaxPasses = 4, kStageMaxTopK = 8;
 
+// The order in which the kernel takes a program's sweeps over the resident tensor: every pass, and behind a pass's merges
+// the further rounds of its Top-K reductions.  Built on the host, so the kernel walks a table instead of deciding -- and
+// the table is a compile-time constant when the program is compiled into the kernel.
+struct SweepStep {
+  uint8_t i0, i1;      // micro-instruction range code[i0 .. i1)
+  int8_t topk_r;       // -1: a pass (its merges and per-row arithmetic follow); >= 0: a Top-K sweep of this reduction
+  uint8_t topk_round;  // Top-K sweep: which pick it looks for (1 .. K-1; round 0 is the pass's own arg max)
+  uint8_t pass;
+  uint8_t release;     // the accumulator is handed back behind this step (the last one)
+  uint8_t pad[2];
+};
+constexpr int kStageMaxSweeps = kStageMaxPasses + kStageMaxRed * (kStageMaxTopK - 1);
+
 struct StageProgram {
   uint8_t n_red, n_scalar_instr, n_passes, terminal_pass;
   uint8_t n_row_out;
@@ -88,7 +101,9 @@ struct StageProgram {
   // pass 0: entry chain, XSAVE; every pass: per reduction of the pass (XLOAD if v was changed,) its chain, ACC; the
   // terminal's pass: (XLOAD,) final chain, ACC of the reductions on y, EMIT.
   uint8_t pass_off[kStageMaxPasses + 1];
-  uint8_t pad2[3];
+  uint8_t n_sweeps;
+  uint8_t pad2[2];
+  SweepStep sweep[kStageMaxSweeps];
   ChainInstr code[kStageMaxCode];
   StageReduction red[kStageMaxRed];
   ScalarInstr sc[kStageMaxScalarInstr];

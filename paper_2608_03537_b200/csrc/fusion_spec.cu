@@ -668,6 +668,19 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
     if (!used) sp.red[r].k = 0;
   }
   sp.n_row_out = static_cast<uint8_t>(an.row_outputs.size());
+  // the sweep table: each pass, then the further rounds of that pass's Top-K reductions in program order
+  int ns = 0;
+  for (int pass = 0; pass < sp.n_passes; ++pass) {
+    sp.sweep[ns++] = SweepStep{sp.pass_off[pass], sp.pass_off[pass + 1], -1, 0, static_cast<uint8_t>(pass), 0, {0, 0}};
+    for (int r = 0; r < sp.n_red; ++r) {
+      if (sp.red[r].pass != pass) continue;
+      for (int round = 1; round < sp.red[r].k; ++round)
+        sp.sweep[ns++] = SweepStep{sp.red[r].code_lo, sp.red[r].code_hi, static_cast<int8_t>(r), static_cast<uint8_t>(round),
+                                   static_cast<uint8_t>(pass), 0, {0, 0}};
+    }
+  }
+  sp.sweep[ns - 1].release = 1;
+  sp.n_sweeps = static_cast<uint8_t>(ns);
   return true;
 }
 
