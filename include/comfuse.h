@@ -281,6 +281,15 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      max, min, prod, argmax merge across the cluster); any other valid program runs on the standard pathway
  *      (COMFUSE_SPEC_PATH_ROW_PROGRAM): the GEMM kernel writes bf16 Z to the workspace and one row-program kernel
  *      evaluates the node list per row with the row resident in shared memory, one pass per stage.
+ *   3. on request (`fused` = 3) GENERATES the fused kernel for the program (Sec. 5: the fused epilogue as generated code):
+ *      the FUSED_PROGRAM kernel is compiled at run time with the program's structure as a compile-time table, so that the
+ *      interpreter's loops unroll and its dispatches fold into straight-line code; same lowering, same limits, same
+ *      merge order.  Results equal the interpreter's except where the compiler contracts a multiply and the addition of
+ *      the next node into one fused multiply-add (one rounding instead of two); with COMFUSE_GENERATED_FMAD=0 in the
+ *      environment kernels are compiled without contraction and the results are bit-identical.  Constants (CONST nodes) and pointers stay run-time
+ *      arguments: programs that differ only in those share a kernel.  The first call that needs a kernel compiles it
+ *      (NVRTC from the CUDA toolkit, a few seconds, on the calling thread) and keeps it for the life of the process; make
+ *      that call, or comfuse_gemm_spec_prepare, before any stream capture.
  */
 typedef enum {
   COMFUSE_OP_ACC = 0,          /* accumulator entry: (A.B)[i, j]                                      */
@@ -359,14 +368,27 @@ typedef struct {
 comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape,
                                    comfuse_spec_plan_t* plan);
 
-/* Workspace comfuse_gemm_spec needs (bytes): 0 or row scratch for the fused kernel, batch*M*N*2 for the row program. */
+/* Workspace comfuse_gemm_spec needs (bytes): 0 or row scratch for the fused kernel, batch*M*N*2 for the row program,
+ * 0 for `fused` = 3. */
 comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape,
                                                   int32_t fused, size_t* bytes);
+
+/* Whether programs can be compiled at run time on this machine: COMFUSE_OK, or COMFUSE_ERR_UNSUPPORTED with *why (may be
+ * NULL) pointing at a static string that names what is missing (the toolkit's libnvrtc or its headers; CUDA_HOME is
+ * searched, then /usr/local/cuda).  Touches no device. */
+comfuse_status_t comfuse_program_compiler_status(const char** why);
+
+/* Does whatever comfuse_gemm_spec(..., fused, ...) would do ahead of its first launch for this program and shape -- for
+ * `fused` = 3 it generates and compiles the kernel (no device is needed for that; the module is loaded by the first
+ * launch) -- and nothing for the other pathways.  OK, the errors of comfuse_spec_plan, or UNSUPPORTED when `fused` = 3
+ * and the program has no on-chip lowering, the shape no instantiation, or the compiler is not available. */
+comfuse_status_t comfuse_gemm_spec_prepare(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused);
 
 /* Y = program(A . B).  `params`: HOST array of spec->n_params DEVICE pointers (bf16; ROWVEC [N], TENSOR [batch, M, N]
  * with leading dimension param_ld[k], 0 = N); `param_ld` may be NULL.  `row_out`: HOST array of n_row_outputs DEVICE
  * pointers.  `fused` = 1: the best path (compiled fused kind, else on-chip interpreter, else row program); 2: skip the
- * compiled kinds (on-chip interpreter, else row program); 0: always the row-program pathway.
+ * compiled kinds (on-chip interpreter, else row program); 0: always the row-program pathway; 3: the kernel generated for
+ * this program (UNSUPPORTED where the program has no on-chip lowering or the compiler is not available; no fallback).
  * Asynchronous on `cuda_stream`; the host arrays are not read after the call returns. */
 comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A,
                                    const void* B, void* Y, const void* const* params, const int64_t* param_ld,

@@ -50,6 +50,8 @@ EXPORTED_SYMBOLS = (
     "comfuse_spec_plan",
     "comfuse_gemm_spec_workspace_size",
     "comfuse_gemm_spec",
+    "comfuse_gemm_spec_prepare",
+    "comfuse_program_compiler_status",
     "comfuse_selftest_bounds_predicate",
     "comfuse_last_device_status",
     "comfuse_launch_count",
@@ -162,6 +164,10 @@ def lib() -> ctypes.CDLL:
         L.comfuse_gemm_spec.argtypes = [POINTER(FusionSpec), POINTER(GemmShape), c_void_p, c_void_p, c_void_p, POINTER(c_void_p),
                                         POINTER(c_int64), POINTER(c_void_p), c_int32, c_void_p, c_size_t, c_void_p]
         L.comfuse_gemm_spec.restype = c_int32
+        L.comfuse_gemm_spec_prepare.argtypes = [POINTER(FusionSpec), POINTER(GemmShape), c_int32]
+        L.comfuse_gemm_spec_prepare.restype = c_int32
+        L.comfuse_program_compiler_status.argtypes = [POINTER(ctypes.c_char_p)]
+        L.comfuse_program_compiler_status.restype = c_int32
         L.comfuse_last_device_status.argtypes = [c_void_p]
         L.comfuse_last_device_status.restype = c_int32
         L.comfuse_selftest_bounded_wait.argtypes = [ctypes.c_uint32, c_void_p, POINTER(ctypes.c_uint32)]
@@ -434,10 +440,28 @@ def gemm_spec_workspace_size(spec: FusionSpec, shape: GemmShape, fused=True) -> 
     return int(n.value)
 
 
+GENERATED = 3   # `fused` value of the spec calls: the kernel generated (compiled at run time) for the program
+
+
+def program_compiler_status():
+    """(status, reason): OK and "" when programs can be compiled at run time on this machine (needs no GPU)."""
+    why = ctypes.c_char_p()
+    st = int(lib().comfuse_program_compiler_status(byref(why)))
+    return st, (why.value or b"").decode()
+
+
+def gemm_spec_prepare(spec: FusionSpec, shape: GemmShape, fused=GENERATED) -> None:
+    """Compile ahead of the first launch what gemm_spec(..., fused=fused) would compile on it (needs no GPU)."""
+    st = lib().comfuse_gemm_spec_prepare(byref(spec), byref(shape), int(fused))
+    if st != OK:
+        raise ComfuseError(st, "comfuse_gemm_spec_prepare")
+
+
 def gemm_spec(A, B, Y, spec: FusionSpec, *, params=(), row_out=(), fused=True, workspace=None, stream=None, b_nk=False):
     """Enqueue Y = program(A.B): ``spec`` from make_spec, ``params`` the CUDA bf16 tensors of the parameter table
     (row vectors [N], tensors [batch, M, N]), ``row_out`` the per-row output tensors (fp32, int32 for an arg max);
-    ``b_nk``: B is stored [batch, N, K]."""
+    ``b_nk``: B is stored [batch, N, K].  ``fused``: 1 best path, 2 on-chip interpreter, 0 row program, GENERATED (3) the
+    kernel compiled for this program (the first call compiles it: seconds)."""
     batched = A.dim() == 3
     batch = A.shape[0] if batched else 1
     M, K = A.shape[-2], A.shape[-1]

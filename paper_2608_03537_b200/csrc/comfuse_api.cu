@@ -270,14 +270,15 @@ comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long 
 comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
-                                   cudaStream_t st, bool query_only, bool b_nk) {
+                                   cudaStream_t st, bool query_only, bool b_nk, bool compiled) {
   FusedParams p = {};
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.b_nk = b_nk ? 1 : 0;
   GemmMaps maps;
   if (query_only) {
     std::memset(&maps, 0, sizeof(maps));
-    return launch_fused_program(maps, p, nullptr, true) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
+    const cudaError_t e = compiled ? launch_compiled_program(maps, p, nullptr, true, false) : launch_fused_program(maps, p, nullptr, true);
+    return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
   }
   const DeviceInfo* dev = nullptr;
   comfuse_status_t s = check_device(&dev);
@@ -301,7 +302,20 @@ comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda
   p.Y = static_cast<uint16_t*>(Y);
   p.ldy = ldy; p.batch_stride_y = batch > 1 ? batch_stride_y : 0;
   p.program = prog;
+  if (compiled) {
+    const cudaError_t e = launch_compiled_program(maps, p, st, false, true);
+    return e == cudaSuccess ? COMFUSE_OK : (e == cudaErrorInvalidValue ? COMFUSE_ERR_UNSUPPORTED : COMFUSE_ERR_CUDA);
+  }
   return launch_fused_program(maps, p, st, false) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
+}
+
+comfuse_status_t prepare_compiled_program(int N, const StageProgram& prog) {
+  FusedParams p = {};
+  p.N = N;
+  p.program = prog;
+  GemmMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  return launch_compiled_program(maps, p, nullptr, false, false) == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_UNSUPPORTED;
 }
 
 }  // namespace comfuse

@@ -12,9 +12,7 @@ cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cud
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_PROGRAM, b0, b1, cn, nst, lock>(maps, p, st);
   switch (p.N) {
-    COMFUSE_CASE(256, 256, 0, 1, 5, 0)
-    COMFUSE_CASE(512, 256, 256, 1, 3, 1)
-    COMFUSE_CASE(768, 256, 128, 2, 4, 1)
+    COMFUSE_PROGRAM_INSTANCES_SMALL(COMFUSE_CASE)
     default:
       return launch_fused_program_large(maps, p, st, supported_only);  // N = 1024, 2048, 4096: a translation unit of their own
   }

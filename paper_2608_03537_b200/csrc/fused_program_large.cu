@@ -9,9 +9,7 @@ cudaError_t launch_fused_program_large(const GemmMaps& maps, const FusedParams& 
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_PROGRAM, b0, b1, cn, nst, lock>(maps, p, st);
   switch (p.N) {
-    COMFUSE_CASE(1024, 256, 256, 2, 3, 1)
-    COMFUSE_CASE(2048, 256, 256, 4, 3, 1)
-    COMFUSE_CASE(4096, 256, 256, 8, 3, 1)
+    COMFUSE_PROGRAM_INSTANCES_LARGE(COMFUSE_CASE)
     default:
       return cudaErrorInvalidValue;
   }

@@ -851,7 +851,7 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
   if (want_fused && !dc.fused && lower_stage_program(dc.an, dc.stage_prog, dc.stage_bind)) {
     const void* none[3] = {nullptr, nullptr, nullptr};
     dc.on_chip = run_fused_program(shape->batch, shape->M, shape->N, shape->K, 0, 0, 0, 0, 0, 0, nullptr, nullptr, nullptr, dc.stage_prog,
-                                   none, nullptr, 0, nullptr, true) == COMFUSE_OK;
+                                   none, nullptr, 0, nullptr, true, false, want_fused == 3) == COMFUSE_OK;
     if (dc.on_chip && want_fused == 1 && !on_chip_is_cheaper(dc.an, dc.stage_prog, shape->N)) dc.on_chip = false;
   }
   return COMFUSE_OK;
@@ -896,12 +896,24 @@ comfuse_status_t comfuse_spec_plan(const comfuse_fusion_spec_t* spec, const comf
   return (plan->path == COMFUSE_SPEC_PATH_ROW_PROGRAM) ? s : COMFUSE_OK;
 }
 
+comfuse_status_t comfuse_program_compiler_status(const char** why) { return program_compiler_status(why); }
+
+comfuse_status_t comfuse_gemm_spec_prepare(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused) {
+  if (fused < 0 || fused > 3) return COMFUSE_ERR_INVALID_ARG;
+  Decision dc;
+  comfuse_status_t s = decide(spec, shape, fused, dc);
+  if (s != COMFUSE_OK || fused != 3) return s;
+  if (!dc.on_chip) return COMFUSE_ERR_UNSUPPORTED;
+  return prepare_compiled_program(shape->N, dc.stage_prog);
+}
+
 comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused,
                                                   size_t* bytes) {
-  if (!bytes || fused < 0 || fused > 2) return COMFUSE_ERR_INVALID_ARG;
+  if (!bytes || fused < 0 || fused > 3) return COMFUSE_ERR_INVALID_ARG;
   Decision dc;
   comfuse_status_t s = decide(spec, shape, fused, dc);
   if (s != COMFUSE_OK) return s;
+  if (fused == 3 && !dc.on_chip) return COMFUSE_ERR_UNSUPPORTED;
   if (dc.fused) {
     *bytes = dc.fused_inner_ws + dc.fused_scratch;
     return COMFUSE_OK;
@@ -922,10 +934,11 @@ comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* s
 comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A, const void* B,
                                    void* Y, const void* const* params, const int64_t* param_ld, void* const* row_out, int32_t fused,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  if (fused < 0 || fused > 2) return COMFUSE_ERR_INVALID_ARG;
+  if (fused < 0 || fused > 3) return COMFUSE_ERR_INVALID_ARG;
   Decision dc;
   comfuse_status_t s = decide(spec, shape, fused, dc);
   if (s != COMFUSE_OK) return s;
+  if (fused == 3 && !dc.on_chip) return COMFUSE_ERR_UNSUPPORTED;  // the generated kernel is asked for by name: no other path stands in
   if (!A || !B || !Y) return COMFUSE_ERR_INVALID_ARG;
   const Analysis& an = dc.an;
   // the parameter table: every slot a live node reads must be there, aligned, with a usable leading dimension
@@ -985,7 +998,8 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
     const void* res = bd.tensor_param >= 0 ? params[bd.tensor_param] : nullptr;
     return run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
                              shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res,
-                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false, (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0);
+                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false, (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0,
+                             fused == 3);
   }
 
   // standard pathway: GEMM -> bf16 Z in the workspace -> row program

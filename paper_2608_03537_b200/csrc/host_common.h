@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "comfuse.h"
 #include "fused_params.h"
 
 namespace comfuse {
@@ -46,6 +47,10 @@ cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, c
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Epilogue = the stage program in p.program, interpreted on-chip (N in {256, 512, 768, 1024, 2048, 4096}).
 cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+// The same kernel with p.program compiled in (generated at run time, cached per program structure and N).  `launch` =
+// false stops after the compilation.  cudaErrorInvalidValue: no instantiation for N, or the compiler is unavailable / failed.
+cudaError_t launch_compiled_program(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only, bool launch);
+comfuse_status_t program_compiler_status(const char** why);
 // Rows wider than the largest cluster (16 CTAs x 256 columns): LayerNorm / RMSNorm kinds run per 4096-column block and a
 // second kernel merges the blocks' statistics (the wide-row fallback).  Returns the number of blocks, 0 = not a wide row.
 constexpr int kWideRowBlock = 4096;
@@ -85,7 +90,9 @@ namespace comfuse {
 comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                    long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,
                                    const StageProgram& prog, const void* const vecs[3], const void* residual, long long ldr,
-                                   cudaStream_t st, bool query_only, bool b_nk = false);
+                                   cudaStream_t st, bool query_only, bool b_nk = false, bool compiled = false);
+// Compiles the kernel run_fused_program(..., compiled = true) would launch for this program and N (no device needed).
+comfuse_status_t prepare_compiled_program(int N, const StageProgram& prog);
 // Y = act(alpha * A . B + bias) (reduction-free epilogue), any N that is a multiple of 8; bias may be null.
 comfuse_status_t run_gemm_elementwise(int batch, int M, int N, int K, long long lda, long long ldb, long long ldy, long long batch_stride_a,
                                       long long batch_stride_b, long long batch_stride_y, const void* A, const void* B, void* Y,

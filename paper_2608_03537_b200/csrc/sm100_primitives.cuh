@@ -387,9 +387,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
 }
 // Three-input maximum (one instruction on sm_100).
 __device__ __forceinline__ float max3(float a, float b, float c) {
+#if defined(__CUDACC_RTC__) && (__CUDACC_VER_MAJOR__ * 100 + __CUDACC_VER_MINOR__ < 1209)
+  return fmaxf(fmaxf(a, b), c);  // a run-time compiler older than the three-input form
+#else
   float y;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
+#endif
 }
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
@@ -410,8 +414,16 @@ struct SoftcapLog2 {
 };
 // Packed fp32x2 arithmetic (one instruction for two lanes of a float2): halves the issue slots of the epilogue math.
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+#ifdef COMFUSE_NO_CONTRACTION
+// Measured: a packed multiply followed by a packed add is contracted into one packed fused multiply-add when both end up in
+// one basic block, whatever the contraction option says; the scalar round-to-nearest forms never are.  A kernel generated
+// for a program uses these when it has to reproduce the interpreter (a dispatch between any two nodes) bit for bit.
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return make_float2(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y)); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return make_float2(__fmul_rn(a.x, b.x), __fmul_rn(a.y, b.y)); }
+#else
 __device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
 __device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+#endif
 __device__ __forceinline__ float2 splat2(float a) { return make_float2(a, a); }
 __device__ __forceinline__ float2 f2_from_bits(uint32_t a, uint32_t b) { return make_float2(__uint_as_float(a), __uint_as_float(b)); }
 // the two bf16 halves of a packed word, widened exactly
