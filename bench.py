@@ -259,6 +259,14 @@ def measure(name, args, env, full):
         spec = cf.make_spec(w.program.nodes, w.program.terminal, len(w.program.param_kinds), w.program.row_outputs)
         pshape = cf.make_gemm_shape(1, w.dims["M"], w.dims["N"], w.dims["K"])
         plan = cf.spec_plan(spec, pshape)
+        # the fused path of a program: the kernel generated for it (compiled at run time, ahead of the timed region and of
+        # any graph capture), else the on-chip interpreter of the same lowering
+        generated = (args.program_path == "generated" and plan.program_path == cf.SPEC_PATH_FUSED_PROGRAM
+                     and plan.path != cf.SPEC_PATH_FUSED_KERNEL and cf.program_compiler_status()[0] == cf.OK)
+        if generated:
+            cf.gemm_spec_prepare(spec, pshape, cf.GENERATED)
+        interpreted = 2 if plan.path == cf.SPEC_PATH_FUSED_PROGRAM else 1
+        pmode = lambda use_fused: (cf.GENERATED if generated else interpreted) if use_fused else 0
     act_names = {"A", "B"} if w.kind == wl.KIND_SCALE_MASK_SOFTMAX else ({"X", "W1", "W2"} if attention else {"A", "residual", "X"})
     base = {k: to_dev(v) for k, v in w.tensors.items()}
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
@@ -289,7 +297,7 @@ def measure(name, args, env, full):
     if b2b:
         ws_bytes = cf.b2b_workspace_size(b2b_desc(fused))
     elif program:
-        ws_bytes = cf.gemm_spec_workspace_size(spec, pshape, fused)
+        ws_bytes = cf.gemm_spec_workspace_size(spec, pshape, pmode(fused))
     else:
         kind = {wl.KIND_BIAS_RES_LAYERNORM: cf.EPI_BIAS_RES_LAYERNORM,
                 wl.KIND_BIAS_GELU_RES_RMSNORM_MAX: cf.EPI_BIAS_GELU_RES_RMSNORM_MAX,
@@ -302,7 +310,7 @@ def measure(name, args, env, full):
     def step(s, use_fused=fused, workspace=ws):
         if program:
             cf.gemm_spec(s["A"], s["B"], s["Y"], spec, params=[s[f"p{k}"] for k in range(len(w.program.param_kinds))],
-                         row_out=s["row_out"], fused=use_fused, workspace=workspace)
+                         row_out=s["row_out"], fused=pmode(use_fused), workspace=workspace)
         elif attention:
             cf.b2b_attention(s["X"], s["W1"], s["W2"], s["Y"], alpha=w.scalars["alpha"], fused=use_fused, workspace=workspace)
         elif relu_mlp:
@@ -426,7 +434,7 @@ def measure(name, args, env, full):
     roof["traffic"], roof["traffic_source"] = NCU_TRAFFIC.get(name, (None, None))
     roof["peak_source"] = f"of {peaks['source']} (burst figure, kernel timed alone)"
     if program:
-        roof["kernel"] = {cf.SPEC_PATH_FUSED_KERNEL: "fused_pair_kernel (compiled kind)", cf.SPEC_PATH_FUSED_PROGRAM: "fused_pair_kernel<EPI_PROGRAM> (on-chip interpreter)",
+        roof["kernel"] = {cf.SPEC_PATH_FUSED_KERNEL: "fused_pair_kernel (compiled kind)", cf.SPEC_PATH_FUSED_PROGRAM: "fused_pair_kernel<EPI_PROGRAM> (generated for the program)" if generated else "fused_pair_kernel<EPI_PROGRAM> (on-chip interpreter)",
                           cf.SPEC_PATH_ROW_PROGRAM: "fused_pair_kernel<EPI_NONE> + row_program_kernel"}[plan.path if fused else cf.SPEC_PATH_ROW_PROGRAM]
     elif b2b:
         roof["kernel"] = "b2b_stream_kernel" if relu_mlp else ("b2b_pair_kernel" if attention else "b2b_mlp_kernel")
@@ -481,7 +489,7 @@ def measure(name, args, env, full):
         if b2b:
             ob = cf.b2b_workspace_size(b2b_desc(other))
         elif program:
-            ob = cf.gemm_spec_workspace_size(spec, pshape, other)
+            ob = cf.gemm_spec_workspace_size(spec, pshape, pmode(other))
         else:
             desc.fused = int(other)
             ob = cf.workspace_size(desc)
@@ -496,6 +504,16 @@ def measure(name, args, env, full):
         del ws2
     except cf.ComfuseError as e:
         extra["unfused_error"] = str(e)
+    if program and fused and generated:
+        # context: the same lowering run as data by the on-chip interpreter (what the generated kernel replaces)
+        def interp(i):
+            s = sets[i % nsets]
+            cf.gemm_spec(s["A"], s["B"], s["Y"], spec, params=[s[f"p{k}"] for k in range(len(w.program.param_kinds))],
+                         row_out=s["row_out"], fused=2, workspace=ws)
+        for i in range(3):
+            interp(i)
+        n2 = max(3, min(args.steps, 50))
+        extra["interpreter_ms_per_step"] = timed(n2, interp) / n2
     res.update(extra)
     if not full:
         return res
@@ -575,7 +593,7 @@ def measure(name, args, env, full):
         def e2e_step(i):
             dA.copy_(host_in["A"], non_blocking=True)
             cf.gemm_spec(dA, s0["B"], s0["Y"], spec, params=[s0[f"p{k}"] for k in range(len(w.program.param_kinds))],
-                         row_out=s0["row_out"], fused=fused, workspace=ws)
+                         row_out=s0["row_out"], fused=pmode(fused), workspace=ws)
             host_out.copy_(s0["Y"], non_blocking=True)
     elif b2b:
         bdesc = b2b_desc(fused)
@@ -694,6 +712,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--kernel-only", action="store_true", help="skip the unfused, end-to-end and CPU legs (for profiler runs)")
+    ap.add_argument("--program-path", default="generated", choices=["generated", "interpreter"],
+                    help="workload p1: the kernel generated for the program (default where the run-time compiler is there) or the on-chip interpreter")
     ap.add_argument("--no-per-workload", action="store_true", help="only the headline workload, not the c2-c5 list")
     args = ap.parse_args()
     if args.impl == "reference":

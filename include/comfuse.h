@@ -288,8 +288,10 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      the next node into one fused multiply-add (one rounding instead of two); with COMFUSE_GENERATED_FMAD=0 in the
  *      environment kernels are compiled without contraction and the results are bit-identical.  Constants (CONST nodes) and pointers stay run-time
  *      arguments: programs that differ only in those share a kernel.  The first call that needs a kernel compiles it
- *      (NVRTC from the CUDA toolkit, a few seconds, on the calling thread) and keeps it for the life of the process; make
- *      that call, or comfuse_gemm_spec_prepare, before any stream capture.
+ *      (NVRTC from the CUDA toolkit, one to three seconds, on the calling thread) and keeps it for the life of the process;
+ *      make that call, or comfuse_gemm_spec_prepare, before any stream capture.  Where the compiler is available `fused` = 1
+ *      takes this form too whenever it would otherwise interpret (COMFUSE_GENERATE=0 in the environment keeps the
+ *      interpreter); comfuse_spec_plan reports COMFUSE_SPEC_PATH_FUSED_PROGRAM for both, they are the same lowering.
  */
 typedef enum {
   COMFUSE_OP_ACC = 0,          /* accumulator entry: (A.B)[i, j]                                      */
@@ -379,15 +381,16 @@ comfuse_status_t comfuse_gemm_spec_workspace_size(const comfuse_fusion_spec_t* s
 comfuse_status_t comfuse_program_compiler_status(const char** why);
 
 /* Does whatever comfuse_gemm_spec(..., fused, ...) would do ahead of its first launch for this program and shape -- for
- * `fused` = 3 it generates and compiles the kernel (no device is needed for that; the module is loaded by the first
- * launch) -- and nothing for the other pathways.  OK, the errors of comfuse_spec_plan, or UNSUPPORTED when `fused` = 3
+ * `fused` = 3, and for `fused` = 1 where that takes the generated form, it generates and compiles the kernel (no device
+ * is needed for that; the module is loaded by the first launch) -- and nothing for the other pathways.  OK, the errors of comfuse_spec_plan, or UNSUPPORTED when `fused` = 3
  * and the program has no on-chip lowering, the shape no instantiation, or the compiler is not available. */
 comfuse_status_t comfuse_gemm_spec_prepare(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, int32_t fused);
 
 /* Y = program(A . B).  `params`: HOST array of spec->n_params DEVICE pointers (bf16; ROWVEC [N], TENSOR [batch, M, N]
  * with leading dimension param_ld[k], 0 = N); `param_ld` may be NULL.  `row_out`: HOST array of n_row_outputs DEVICE
- * pointers.  `fused` = 1: the best path (compiled fused kind, else on-chip interpreter, else row program); 2: skip the
- * compiled kinds (on-chip interpreter, else row program); 0: always the row-program pathway; 3: the kernel generated for
+ * pointers.  `fused` = 1: the best path (compiled fused kind, else the on-chip program -- as generated code where the run-time
+ * compiler is available, else interpreted --, else row program); 2: skip the compiled kinds and interpret (on-chip
+ * interpreter, else row program); 0: always the row-program pathway; 3: the kernel generated for
  * this program (UNSUPPORTED where the program has no on-chip lowering or the compiler is not available; no fallback).
  * Asynchronous on `cuda_stream`; the host arrays are not read after the call returns. */
 comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comfuse_gemm_shape_t* shape, const void* A,

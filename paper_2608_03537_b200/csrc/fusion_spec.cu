@@ -9,6 +9,7 @@
 //   lower_row_program(): the standard pathway -- one instruction per live computed node, shared-memory slots assigned
 //               by liveness (a node's buffer is released at its last use and may be overwritten in place).
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -802,6 +803,14 @@ comfuse_gemm_desc_t fused_desc(const comfuse_gemm_shape_t& s, const FusedMatch& 
 // chains re-run in every pass, transcendental operations counted three times -- against 0.9 ns per instruction plus 0.6 ns for
 // the bf16 round trip of Z in the row program, which has every SM's full occupancy).  A coarse model, good enough to send
 // exponential-heavy three-pass programs to the row program and the rest on-chip.
+// Whether `fused` = 1 runs an on-chip program as a kernel generated for it: where the run-time compiler is there, unless
+// COMFUSE_GENERATE=0 asks for the interpreter.
+bool generate_by_default() {
+  const char* v = std::getenv("COMFUSE_GENERATE");
+  if (v && v[0] == '0') return false;
+  return program_compiler_status(nullptr) == COMFUSE_OK;
+}
+
 bool on_chip_is_cheaper(const Analysis& an, const StageProgram& sp, int N) {
   RowProgram P;
   std::memset(&P, 0, sizeof(P));
@@ -817,7 +826,9 @@ bool on_chip_is_cheaper(const Analysis& an, const StageProgram& sp, int N) {
       units += transcendental ? 3.f : 1.f;
     }
   }
-  return 0.36f * units <= 0.9f * static_cast<float>(ni) + 0.6f;
+  // compiled into the kernel, the same stream costs about 0.14 ns per unit (measured on the same programs: 2.2 to 2.8 times
+  // the interpreter's rate)
+  return (generate_by_default() ? 0.14f : 0.36f) * units <= 0.9f * static_cast<float>(ni) + 0.6f;
 }
 
 struct Decision {
@@ -902,7 +913,12 @@ comfuse_status_t comfuse_gemm_spec_prepare(const comfuse_fusion_spec_t* spec, co
   if (fused < 0 || fused > 3) return COMFUSE_ERR_INVALID_ARG;
   Decision dc;
   comfuse_status_t s = decide(spec, shape, fused, dc);
-  if (s != COMFUSE_OK || fused != 3) return s;
+  if (s != COMFUSE_OK) return s;
+  if (fused == 1 && dc.on_chip && generate_by_default()) {
+    (void)prepare_compiled_program(shape->N, dc.stage_prog);  // a failure leaves the interpreter
+    return COMFUSE_OK;
+  }
+  if (fused != 3) return COMFUSE_OK;
   if (!dc.on_chip) return COMFUSE_ERR_UNSUPPORTED;
   return prepare_compiled_program(shape->N, dc.stage_prog);
 }
@@ -939,6 +955,7 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
   comfuse_status_t s = decide(spec, shape, fused, dc);
   if (s != COMFUSE_OK) return s;
   if (fused == 3 && !dc.on_chip) return COMFUSE_ERR_UNSUPPORTED;  // the generated kernel is asked for by name: no other path stands in
+  const bool try_generated = fused == 1 && dc.on_chip && generate_by_default();
   if (!A || !B || !Y) return COMFUSE_ERR_INVALID_ARG;
   const Analysis& an = dc.an;
   // the parameter table: every slot a live node reads must be there, aligned, with a usable leading dimension
@@ -996,10 +1013,16 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
     StageProgram sp = dc.stage_prog;
     for (int r = 0; r < sp.n_row_out; ++r) sp.out[r].ptr = row_out[bd.row_out_pos[r]];
     const void* res = bd.tensor_param >= 0 ? params[bd.tensor_param] : nullptr;
+    const long long ldres = bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N;
+    const bool b_nk = (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0;
+    if (try_generated) {
+      // the best path: the kernel generated for this program; where it cannot be had (the compilation failed), the interpreter
+      s = run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
+                            shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res, ldres, st, false, b_nk, true);
+      if (s != COMFUSE_ERR_UNSUPPORTED) return s;
+    }
     return run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
-                             shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res,
-                             bd.tensor_param >= 0 ? ld[bd.tensor_param] : shape->N, st, false, (shape->flags & COMFUSE_FLAG_B_ROW_MAJOR_NK) != 0,
-                             fused == 3);
+                             shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res, ldres, st, false, b_nk, fused == 3);
   }
 
   // standard pathway: GEMM -> bf16 Z in the workspace -> row program

@@ -63,10 +63,10 @@ def test_ordinary_build_has_no_predicates(cuda_device):
 
 
 def test_checked_build_runs_every_kernel_family_with_a_clear_status_word(cuda_device):
-    if not os.path.exists(CHECKED_LIB):
-        try:
-            cf_build.build(checked=True)
-        except Exception as e:  # no nvcc on this machine
+    try:
+        cf_build.build(checked=True)     # incremental: nothing happens when the library is up to date
+    except Exception as e:               # no nvcc on this machine: a library that came with the tree will do
+        if not os.path.exists(CHECKED_LIB):
             pytest.skip(f"checked library not built: {e}")
     env = dict(os.environ, COMFUSE_LIB=CHECKED_LIB, PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
     r = subprocess.run([sys.executable, "-c", CHILD], cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)

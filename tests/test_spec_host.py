@@ -83,8 +83,15 @@ def test_recovered_constants():
     assert _plan(p.nodes, p.terminal, 4).eps == pytest.approx(3e-4)
 
 
-def test_near_misses_do_not_take_a_compiled_kind():
-    PROG, ROW = cf.SPEC_PATH_FUSED_PROGRAM, cf.SPEC_PATH_ROW_PROGRAM
+@pytest.mark.parametrize("generate", [False, True])
+def test_near_misses_do_not_take_a_compiled_kind(generate, monkeypatch):
+    """With COMFUSE_GENERATE=0 an on-chip program is interpreted, and the cost model sends exponential-heavy three-pass
+    programs to the row program; run as generated code (the default where the run-time compiler is there) they stay on-chip."""
+    if generate and cf.program_compiler_status()[0] != cf.OK:
+        pytest.skip("no run-time compiler on this machine")
+    monkeypatch.setenv("COMFUSE_GENERATE", "1" if generate else "0")
+    PROG = cf.SPEC_PATH_FUSED_PROGRAM
+    ROW = PROG if generate else cf.SPEC_PATH_ROW_PROGRAM
     # residual added INSIDE the activation: not the compiled RMSNorm entry, but still one resident tensor -> on-chip interpreter
     g = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("tensor", -1, -1, 1, 0), ("add", 2, 3, -1, 0), ("gelu_tanh", 4, -1, -1, 0),
          ("square", 5, -1, -1, 0), ("mean", 6, -1, -1, 0), ("const", -1, -1, -1, 1e-5), ("add", 7, 8, -1, 0), ("rsqrt", 9, -1, -1, 0),
@@ -105,7 +112,7 @@ def test_near_misses_do_not_take_a_compiled_kind():
     assert pl.path == ROW and pl.program_path == PROG
     # a row length without any fused instantiation
     p = wl.spec_layernorm()
-    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == ROW
+    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
 
 
 def test_on_chip_lowering_needs_one_resident_tensor():
@@ -165,7 +172,8 @@ def test_malformed_programs_are_rejected():
     assert _status([("acc", 0, -1, -1, 0)], 0) == INV                                          # entry node with an input
 
 
-def test_topk_nodes_are_row_outputs_only():
+def test_topk_nodes_are_row_outputs_only(monkeypatch):
+    monkeypatch.setenv("COMFUSE_GENERATE", "0")   # the path expected below is the cost model's choice for interpreted programs
     INV = cf.ERR_INVALID_ARG
     tk = ("topk_values", 0, -1, 4, 0.0)
     assert _plan([N_, tk], 0, row_outputs=(1,)).path == cf.SPEC_PATH_ROW_PROGRAM
