@@ -49,7 +49,7 @@ NCU_TRAFFIC = {
     "a1": (38_943_488, "profiles/b2b_attention_a1_target_attention.md"),
     "a2": (112_186_112, "profiles/b2b_attention_a2_self_attention_512.md"),
     "d1": (69_688_832, "profiles/b2b_stream_d1_dlrm_bottom_mlp.md"),
-    "p1": (18_984_704, "profiles/fused_program_p1_range_normalise.md"),
+    "p1": (18_941_184, "profiles/fused_program_p1_range_normalise.md"),
 }
 PER_WORKLOAD = ("c2", "c3", "c4", "c5")   # the full-size configurations whose kernels carry a roofline target
 
