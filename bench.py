@@ -52,6 +52,7 @@ NCU_TRAFFIC = {
     "p1": (18_941_184, "profiles/fused_program_p1_range_normalise.md"),
 }
 PER_WORKLOAD = ("c2", "c3", "c4", "c5")   # the full-size configurations whose kernels carry a roofline target
+BEYOND_CONFIGS = ("a1", "a2", "d1", "p1")  # the shapes beyond the named configurations, measured the same way after them
 
 
 def load_peaks():
@@ -674,7 +675,7 @@ def run_comfuse(args):
     per = []
     if world == 1 and not args.kernel_only and not args.no_per_workload:
         # the kernel-level figures of every full-size configuration, in this process, under the same clock sampler
-        for name in PER_WORKLOAD:
+        for name in PER_WORKLOAD + (() if args.no_beyond_configs else BEYOND_CONFIGS):
             if name == args.workload:
                 r = head
             else:
@@ -683,7 +684,9 @@ def run_comfuse(args):
             per.append({"workload": name, "ms_per_step": r["ms_per_step"], "value": r["value"], "unit": "TFLOP/s",
                         "roofline": r["roofline"], "min_ms_per_step": r.get("min_ms_per_step"),
                         "unfused_ms_per_step": r.get("unfused_ms_per_step"), "speedup_vs_unfused": r.get("speedup_vs_unfused"),
-                        "gpu_launches": r["gpu_launches"], "clocks": r["clocks"]})
+                        "gpu_launches": r["gpu_launches"], "clocks": r["clocks"], "named_config": name in PER_WORKLOAD})
+            if "interpreter_ms_per_step" in r:
+                per[-1]["interpreter_ms_per_step"] = r["interpreter_ms_per_step"]
     all_clocks = sampler.stop()
 
     if rank == 0:
@@ -714,6 +717,7 @@ def main():
     ap.add_argument("--kernel-only", action="store_true", help="skip the unfused, end-to-end and CPU legs (for profiler runs)")
     ap.add_argument("--program-path", default="generated", choices=["generated", "interpreter"],
                     help="workload p1: the kernel generated for the program (default where the run-time compiler is there) or the on-chip interpreter")
+    ap.add_argument("--no-beyond-configs", action="store_true", help="per_workload: c2-c5 only, not a1, a2, d1, p1")
     ap.add_argument("--no-per-workload", action="store_true", help="only the headline workload, not the c2-c5 list")
     args = ap.parse_args()
     if args.impl == "reference":
