@@ -948,6 +948,10 @@ COMFUSE_PROGRAM_LOOP
                       o[2 * j] = t2.x; o[2 * j + 1] = t2.y;
                     }
                     break;
+                  case CHO_X:  // the resident tensor (before XSAVE: the accumulator as loaded)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = x[j];
+                    break;
                   default:  // CHO_MASK
 #pragma unroll
                     for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;

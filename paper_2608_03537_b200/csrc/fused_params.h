@@ -26,7 +26,8 @@ enum ChainOperand : uint8_t {
   CHO_SCALAR,    // per-row scalar `index`
   CHO_ROWVEC,    // row-vector parameter staged in shared memory, `index` = 0..2
   CHO_RESIDUAL,  // the full-tensor parameter (entry chain only; delivered through the operand ring)
-  CHO_MASK       // causal mask: 0 where column <= row, -inf above the diagonal
+  CHO_MASK,      // causal mask: 0 where column <= row, -inf above the diagonal
+  CHO_X          // the resident tensor itself (the accumulator, inside the entry chain): gates such as x * sigmoid(x)
 };
 // chain opcodes: the comfuse_op_t values of the unary / binary nodes, plus the reversed non-commutative forms
 constexpr int kChainRsub = 38;  // v = operand - v

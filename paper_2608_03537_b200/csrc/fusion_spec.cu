@@ -492,6 +492,18 @@ struct StageLowering {
       out.push_back(ci);
       return true;
     }
+    // a computed tensor combined with the root itself (a gate: x * sigmoid(x)): the root is at hand in every pass
+    if (is_root(a, entry_mode) && carrier(b) && !is_root(b, entry_mode)) {
+      if (!chain(b, entry_mode, out)) return false;
+      out.push_back(ChainInstr{static_cast<uint8_t>(nd.op == COMFUSE_OP_SUB ? kChainRsub : nd.op == COMFUSE_OP_DIV ? kChainRdiv : nd.op),
+                               CHO_X, 0, 0.f});
+      return true;
+    }
+    if (is_root(b, entry_mode) && carrier(a) && !is_root(a, entry_mode)) {
+      if (!chain(a, entry_mode, out)) return false;
+      out.push_back(ChainInstr{static_cast<uint8_t>(nd.op), CHO_X, 0, 0.f});
+      return true;
+    }
     return false;  // two computed tensors (needs a second resident tensor), or two broadcasts
   }
 };
@@ -517,9 +529,13 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
     }
   }
   if (cand.size() > 1) return false;
-  if (cand.size() == 1) return lower_stage_program_from(an, cand[0], sp, bind);
-  // no later stage reads a stage-0 tensor (the reductions only feed row outputs): any stage-0 tensor from which the
-  // terminal and every reduction input can be reached by chains will do; try them from the last to the first
+  if (cand.size() == 1) {
+    StageBinding b1;
+    if (lower_stage_program_from(an, cand[0], sp, b1)) { bind = b1; return true; }
+  }
+  // no later stage reads a stage-0 tensor (the reductions only feed row outputs), or the one they read is not a chain on
+  // the accumulator (a gate x * f(x)): any stage-0 tensor from which the terminal, every reduction input and every tensor
+  // the later stages read can be reached by chains will do; try them from the last to the first
   for (int k = n - 1; k >= 0; --k) {
     if (!an.live[k] || an.type[k] != T_TENSOR || an.stage[k] != 0) continue;
     if (is_leaf(an.nodes[k].op) && an.nodes[k].op != COMFUSE_OP_ACC) continue;

@@ -43,7 +43,9 @@ def test_topk_program_compiles(compiler):
 
 
 def test_requests_the_pathway_refuses(compiler):
-    dag = wl.spec_gated_minmax()      # two tensors live across a reduction: no on-chip lowering
+    N_ = ("acc", -1, -1, -1, 0.0)     # relu(x) * tanh(x): two computed tensors meet in one node, no on-chip lowering
+    dag = wl.SpecProgram([N_, ("relu", 0, -1, -1, 0.0), ("tanh", 0, -1, -1, 0.0), ("mul", 1, 2, -1, 0.0), ("rmax", 3, -1, -1, 0.0),
+                          ("sub", 3, 4, -1, 0.0)], 5, (), ())
     with pytest.raises(cf.ComfuseError) as e:
         cf.gemm_spec_prepare(_spec(dag), cf.make_gemm_shape(1, 300, 1024, 64), cf.GENERATED)
     assert e.value.status == cf.ERR_UNSUPPORTED

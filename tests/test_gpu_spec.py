@@ -206,13 +206,36 @@ def test_program_outside_the_compiled_patterns(M, N, K):
     prog = wl.spec_gated_minmax()
     A, B, params = _inputs(34, 1, M, N, K, prog.param_kinds)
     Y, ro, plan, launches = _run(prog, A, B, params, True, 1, M, N)
-    assert plan.path == cf.SPEC_PATH_ROW_PROGRAM and plan.n_stages == 2 and launches == 2
+    # a gate x * sigmoid(x): on-chip where the row length has an instantiation (x stays resident, the gate is a chain with x
+    # as its operand), else GEMM + row program
+    on_chip = N == 4096
+    assert plan.path == (cf.SPEC_PATH_FUSED_PROGRAM if on_chip else cf.SPEC_PATH_ROW_PROGRAM) and plan.n_stages == 2
+    assert launches == (1 if on_chip else 2)
     Yref, Rref = _oracle(prog, A, B, params, 1)
     err = np.abs(to_f64(Y) - Yref)
     assert np.isfinite(err).all() and err.max() <= 1.5e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
     np.testing.assert_allclose(ro[0].cpu().numpy(), Rref[0], atol=3e-2)   # row min of the gate
     np.testing.assert_allclose(ro[1].cpu().numpy(), Rref[1], atol=3e-2)   # row max
     np.testing.assert_allclose(ro[2].cpu().numpy(), Rref[2], rtol=2e-3)   # row product
+
+
+@pytest.mark.parametrize("fused", [2, 0])
+@pytest.mark.parametrize("M,N,K", [(300, 256, 72), (260, 1024, 136), (4000, 2048, 64)])
+def test_gated_program_on_the_interpreter_and_on_the_row_program(M, N, K, fused):
+    """x * sigmoid(x) spelled with two uses of x, rescaled to the row's range, plus the row product of a function of the
+    sigmoid: the resident tensor is an operand of its own chain."""
+    prog = wl.spec_gated_minmax()
+    A, B, params = _inputs(37, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, fused, 1, M, N)
+    assert plan.program_path == cf.SPEC_PATH_FUSED_PROGRAM and plan.n_passes == 2
+    assert launches == (1 if fused else 2)
+    Yref, Rref = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    tol = 4e-3 if fused else 1.5e-2
+    assert np.isfinite(err).all() and err.max() <= tol and err.mean() <= tol / 4, (err.max(), err.mean())
+    np.testing.assert_allclose(ro[0].cpu().numpy(), Rref[0], atol=1e-4 if fused else 3e-2)   # row min of the gate
+    np.testing.assert_allclose(ro[1].cpu().numpy(), Rref[1], atol=1e-4 if fused else 3e-2, rtol=1e-5)   # row max
+    np.testing.assert_allclose(ro[2].cpu().numpy(), Rref[2], rtol=2e-4 if fused else 2e-3)   # row product
 
 
 def test_row_program_rejects_rows_that_do_not_fit_shared_memory():

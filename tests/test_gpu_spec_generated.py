@@ -83,6 +83,18 @@ def test_generated_range_normalise_over_every_instantiation(M, N, K, no_contract
     assert np.isfinite(err).all() and err.max() <= 4e-3 and err.mean() <= 1e-3
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 256, 72), (260, 1024, 136), (4000, 2048, 64)])
+def test_generated_gated_program_equals_the_interpreter(M, N, K, no_contraction):
+    prog = wl.spec_gated_minmax()       # the resident tensor is an operand of its own chain: x * sigmoid(x)
+    A, B, params = _inputs(67, 1, M, N, K, prog.param_kinds)
+    Yi, roi, _, _ = _run(prog, A, B, params, 2, 1, M, N)
+    Yg, rog, _, launches = _run(prog, A, B, params, cf.GENERATED, 1, M, N)
+    assert launches == 1 and _same(Yi, Yg) and all(_same(a, b) for a, b in zip(roi, rog))
+    Yref, Rref = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Yg) - Yref)
+    assert np.isfinite(err).all() and err.max() <= 4e-3
+
+
 def test_generated_kernel_with_the_operand_stored_n_by_k(no_contraction):
     prog = wl.spec_range_normalise()
     A, B, params = _inputs(64, 1, 300, 1024, 136, prog.param_kinds)
@@ -153,7 +165,9 @@ def test_programs_that_differ_in_constants_share_a_kernel():
 
 
 def test_generated_kernel_is_refused_where_the_program_has_no_on_chip_lowering():
-    prog = wl.spec_gated_minmax()       # a DAG on two tensors, not a chain on one
+    N_ = ("acc", -1, -1, -1, 0.0)       # relu(x) * tanh(x): two computed tensors meet in one node
+    prog = wl.SpecProgram([N_, ("relu", 0, -1, -1, 0.0), ("tanh", 0, -1, -1, 0.0), ("mul", 1, 2, -1, 0.0), ("rmax", 3, -1, -1, 0.0),
+                           ("sub", 3, 4, -1, 0.0)], 5, (), ())
     A, B, params = _inputs(66, 1, 130, 256, 64, prog.param_kinds)
     with pytest.raises(cf.ComfuseError) as e:
         _run(prog, A, B, params, cf.GENERATED, 1, 130, 256)

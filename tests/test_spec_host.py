@@ -121,9 +121,15 @@ def test_on_chip_lowering_needs_one_resident_tensor():
     for prog, n_params, passes in ((wl.spec_layernorm(relu=True), 4, 3), (wl.spec_rmsnorm_max(), 3, 2), (wl.spec_softmax(0.2, True, 3.0), 0, 3)):
         pl = _plan(prog.nodes, prog.terminal, n_params, prog.row_outputs, shape=cf.make_gemm_shape(1, 1024, 1024, 64))
         assert pl.path == cf.SPEC_PATH_FUSED_KERNEL and pl.program_path == PROG and pl.n_passes == passes
-    # x * sigmoid(x): two computed tensors meet in one node -> needs a second resident tensor -> row program
+    # x * sigmoid(x): a computed tensor meets the resident tensor itself (a gate) -> x = acc + bias stays resident and the
+    # gate is a chain with x as its operand, recomputed where a later stage reads it
     p = wl.spec_gated_minmax()
     pl = _plan(p.nodes, p.terminal, 1, p.row_outputs)
+    assert pl.path == PROG and pl.program_path == PROG and pl.n_passes == 2
+    # relu(x) * tanh(x): two COMPUTED tensors meet in one node -> needs a second resident tensor -> row program
+    nodes = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0), ("tanh", 2, -1, -1, 0), ("mul", 3, 4, -1, 0),
+             ("rmax", 5, -1, -1, 0), ("sub", 5, 6, -1, 0)]
+    pl = _plan(nodes, 7, 1)
     assert pl.path == ROW and pl.program_path == ROW
     # no reduction at all: act(acc + bias) is a compiled reduction-free kind (the plain GEMM's tiling, any N); on the
     # interpreter it is a single pass
@@ -134,10 +140,12 @@ def test_on_chip_lowering_needs_one_resident_tensor():
     # two element-wise steps behind the bias: not that kind, still one resident tensor
     pl = _plan([N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("relu", 2, -1, -1, 0), ("square", 3, -1, -1, 0)], 4, 1)
     assert pl.path == PROG and pl.n_passes == 1
-    # a reduction of something below the resident tensor (max of the raw accumulator while x = acc + bias is kept)
+    # a reduction of something below the tensor the later stages read (max of the raw accumulator, x = acc + bias used later):
+    # the accumulator itself stays resident and acc + bias is recomputed from it
     nodes = [N_, ("rowvec", -1, -1, 0, 0), ("add", 0, 1, -1, 0), ("rmax", 0, -1, -1, 0), ("mean", 2, -1, -1, 0), ("sub", 2, 4, -1, 0),
              ("mul", 5, 3, -1, 0)]
-    assert _plan(nodes, 6, 1).path == ROW
+    pl = _plan(nodes, 6, 1)
+    assert pl.path == PROG and pl.n_passes == 2
     # four row vectors: more than the kernel stages in shared memory
     nodes = [N_] + [("rowvec", -1, -1, q, 0) for q in range(4)] + [("add", 0, 1, -1, 0), ("mul", 5, 2, -1, 0), ("add", 6, 3, -1, 0), ("mul", 7, 4, -1, 0)]
     assert _plan(nodes, 8, 4).path == ROW
