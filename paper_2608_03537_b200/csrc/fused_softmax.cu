@@ -12,7 +12,21 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
 #define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
   case n:                                     \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, 0, epw>(maps, p, st);
-  // The softmax passes are latency-bound on few warps and need few registers: four epilogue warps per lane quarter.
+  // Behind a long contraction the MainLoop is what counts: three pipeline stages with both sub-tiles in lock step (the A
+  // tile fetched once per K block) and eight epilogue warps, instead of two stages and sixteen warps.  Measured: 8192 x 1024,
+  // K = 1024: 24.1 us against 28.7; 8192 x 4096, K = 1024: 106.6 against 126.1; but K = 320 / 512 (causal): 39.2 / 44.9
+  // against 36.4 / 43.1.  COMFUSE_SOFTMAX_STAGES=2 or 3 forces either form.
+  static const char* stages_env = std::getenv("COMFUSE_SOFTMAX_STAGES");
+  const bool long_k = stages_env ? stages_env[0] == '3' : p.K >= 768;
+  if (long_k) {
+    switch (p.N) {
+      case 1024: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 2, 3, 1, 2>(maps, p, st);
+      case 2048: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 4, 3, 1, 2>(maps, p, st);
+      case 4096: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 8, 3, 1, 2>(maps, p, st);
+      default: break;
+    }
+  }
+  // Else the softmax passes are latency-bound on few warps and need few registers: four epilogue warps per lane quarter.
   switch (p.N) {
     COMFUSE_CASE(256, 256, 0, 1, 3, 4)
     COMFUSE_CASE(512, 256, 256, 1, 2, 4)

@@ -182,6 +182,11 @@ SOFTMAX_CASES = [
     (1, 300, 512, 320, False),
     (2, 200, 2048, 272, False),
     (1, 4096, 4096, 264, True),
+    # K >= 768: the cluster kernel's long-contraction form (three stages, sub-tiles in lock step, eight epilogue warps)
+    (1, 300, 1024, 776, False),
+    (2, 1024, 1024, 768, True),
+    (1, 2048, 2048, 1032, True),
+    (1, 260, 4096, 800, False),
 ]
 
 
@@ -235,6 +240,8 @@ def _additive_mask(M, N, seed, dead_rows=(5,)):
     (1, 512, 2048, 128, 3.0),    # soft-cap in front of the mask
     (2, 200, 1024, 320, 0.0),    # long K: the cluster kernel (4 CTA pairs per row block)
     (1, 256, 512, 512, 2.5),     # cluster kernel, soft-capped
+    (1, 300, 1024, 840, 2.0),    # cluster kernel behind a long contraction, soft-capped
+    (2, 260, 2048, 768, 0.0),
 ])
 def test_softmax_additive_mask_with_fully_masked_rows(batch, M, N, K, softcap, fused, cuda_device):
     """The additive-mask variant: the mask tensor is one more operand of the epilogue; -inf entries give exact zeros, a
