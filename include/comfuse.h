@@ -9,7 +9,8 @@
  * Conventions for every entry point
  *   - All tensor pointers are DEVICE pointers unless stated otherwise; the caller owns every buffer.
  *     The library allocates no device memory; its only device state is a small status word that lives
- *     in the loaded module.
+ *     in the loaded module.  (A kernel generated at run time for an epilogue program -- comfuse_gemm_spec, below -- is a
+ *     module of its own, loaded by the first launch that needs it.)
  *   - Tensors are row-major bf16 (2 bytes/element); leading dimensions are in ELEMENTS.
  *     Pointers must be 16-byte aligned and leading dimensions / batch strides multiples of 8 elements.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and
