@@ -274,12 +274,15 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      [activation] [+ residual] -> LayerNorm | RMSNorm [-> max/argmax] | softmax, or a reduction-free act(alpha*acc + bias),
  *      in any spelling the canonicaliser recognises: operand order of commutative nodes, optional nodes absent) runs as
  *      that ONE fused kernel
- *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); a program in which ONE tensor stays resident across the reductions and
- *      every tensor-valued expression is a chain on it (element-wise nodes whose other operand is a constant, a per-row
- *      value, a row vector, the causal mask or -- before the first reduction -- one full tensor; at most 3 row vectors,
- *      6 reductions, 6 row outputs, 4 passes) runs as ONE fused kernel whose epilogue interprets the stages over the on-chip
- *      accumulator (COMFUSE_SPEC_PATH_FUSED_PROGRAM; N in {256, 512, 768, 1024, 2048, 4096}: the reductions sum, mean,
- *      max, min, prod, argmax merge across the cluster); any other valid program runs on the standard pathway
+ *      (path COMFUSE_SPEC_PATH_FUSED_KERNEL); a program in which ONE tensor can stay resident across the reductions --
+ *      the accumulator or something computed from it before the first reduction -- and every other tensor-valued
+ *      expression can be recomputed from it, from constants, per-row values, row vectors, the causal mask and (in the
+ *      first pass only) one full tensor, runs as ONE fused kernel whose epilogue executes the stages over the on-chip
+ *      accumulator (COMFUSE_SPEC_PATH_FUSED_PROGRAM; N in {256, 512, 768, 1024, 2048, 4096}; at most 3 row vectors, 6
+ *      reductions, 6 row outputs, 4 passes, 80 micro-instructions; the reductions sum, mean, max, min, prod, argmax merge
+ *      across the cluster).  Expressions in which two COMPUTED tensors meet (relu(x) * tanh(x)) need temporaries, which
+ *      exist in the generated form of the kernel only (3. below): the interpreter (`fused` = 2) sends such a program to the
+ *      row program; any other valid program runs on the standard pathway
  *      (COMFUSE_SPEC_PATH_ROW_PROGRAM): the GEMM kernel writes bf16 Z to the workspace and one row-program kernel
  *      evaluates the node list per row with the row resident in shared memory, one pass per stage.
  *   3. on request (`fused` = 3) GENERATES the fused kernel for the program (Sec. 5: the fused epilogue as generated code):

@@ -274,6 +274,7 @@ comfuse_status_t run_fused_program(int batch, int M, int N, int K, long long lda
   FusedParams p = {};
   p.M = M; p.N = N; p.K = K; p.batch = batch;
   p.b_nk = b_nk ? 1 : 0;
+  p.program = prog;  // (the query looks at it too: a program with temporaries runs as generated code only)
   GemmMaps maps;
   if (query_only) {
     std::memset(&maps, 0, sizeof(maps));

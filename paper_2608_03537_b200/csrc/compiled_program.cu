@@ -97,7 +97,8 @@ std::string constant_table(const StageProgram& sp) {
   char buf[160];
   auto put = [&](const char* fmt, auto... a) { std::snprintf(buf, sizeof(buf), fmt, a...); t += buf; };
   t += "#include \"fused_params.h\"\nnamespace comfuse {\n__device__ const StageProgram kCompiledProgram = {\n";
-  put("  %d, %d, %d, %d, %d, %d, {0, 0},\n", sp.n_red, sp.n_scalar_instr, sp.n_passes, sp.terminal_pass, sp.n_row_out, sp.x_writeback);
+  put("  %d, %d, %d, %d, %d, %d, %d, {0},\n", sp.n_red, sp.n_scalar_instr, sp.n_passes, sp.terminal_pass, sp.n_row_out, sp.x_writeback,
+      sp.uses_temps);
   t += "  {";
   for (int i = 0; i <= kStageMaxPasses; ++i) put("%d, ", sp.pass_off[i]);
   put("}, %d, {0, 0},\n  {", sp.n_sweeps);

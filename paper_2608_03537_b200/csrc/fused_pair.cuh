@@ -876,6 +876,9 @@ COMFUSE_PROGRAM_LOOP
               ring.advance();
             }
             float v[32], x[32];
+#ifdef COMFUSE_COMPILED_PROGRAM
+            float tq[kStageMaxTemps][32];  // temporaries: constant indices after unrolling, so registers (unused ones vanish)
+#endif
             {
               uint32_t vb[32];
               tmem_ld_32cols(taddr + lc, vb);
@@ -886,7 +889,7 @@ COMFUSE_PROGRAM_LOOP
             for (int i = i0; i < i1; ++i) {
               const ChainInstr ci = sp.code[i];
               const int op = ci.op;
-              if (op >= COMFUSE_OP_ADD && op <= kChainRdiv) {
+              if (op >= COMFUSE_OP_ADD && op <= kChainMov) {
                 // ---- binary with a row-uniform operand (constant or per-row scalar): applied directly
                 if (ci.operand == CHO_SCALAR || ci.operand == CHO_CONST) {
                   const float sv = scalar_get(ci.operand, ci.index, rp.code[i].imm);
@@ -922,6 +925,10 @@ COMFUSE_PROGRAM_LOOP
 #pragma unroll
                       for (int j = 0; j < 32; ++j) v[j] = sv - v[j];
                       break;
+                    case kChainMov:
+#pragma unroll
+                      for (int j = 0; j < 32; ++j) v[j] = sv;
+                      break;
                     default:  // kChainRdiv
 #pragma unroll
                       for (int j = 0; j < 32; ++j) v[j] = __fdividef(sv, v[j]);
@@ -952,6 +959,12 @@ COMFUSE_PROGRAM_LOOP
 #pragma unroll
                     for (int j = 0; j < 32; ++j) o[j] = x[j];
                     break;
+#ifdef COMFUSE_COMPILED_PROGRAM
+                  case CHO_T:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) o[j] = tq[ci.index][j];
+                    break;
+#endif
                   default:  // CHO_MASK
 #pragma unroll
                     for (int j = 0; j < 32; ++j) o[j] = (col0 + j <= grow) ? 0.f : -INFINITY;
@@ -985,6 +998,10 @@ COMFUSE_PROGRAM_LOOP
                   case kChainRsub:
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = o[j] - v[j];
+                    break;
+                  case kChainMov:
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = o[j];
                     break;
                   default:  // kChainRdiv
 #pragma unroll
@@ -1056,6 +1073,12 @@ COMFUSE_PROGRAM_LOOP
                   }
                   break;
                 }
+#ifdef COMFUSE_COMPILED_PROGRAM
+                case kChainTsave:
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) tq[ci.index][j] = v[j];
+                  break;
+#endif
                 case kChainXload:
 #pragma unroll
                   for (int j = 0; j < 32; ++j) v[j] = x[j];

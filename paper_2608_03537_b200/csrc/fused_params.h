@@ -27,16 +27,20 @@ enum ChainOperand : uint8_t {
   CHO_ROWVEC,    // row-vector parameter staged in shared memory, `index` = 0..2
   CHO_RESIDUAL,  // the full-tensor parameter (entry chain only; delivered through the operand ring)
   CHO_MASK,      // causal mask: 0 where column <= row, -inf above the diagonal
-  CHO_X          // the resident tensor itself (the accumulator, inside the entry chain): gates such as x * sigmoid(x)
+  CHO_X,         // the resident tensor itself (the accumulator, inside the entry chain): gates such as x * sigmoid(x)
+  CHO_T          // temporary fragment `index` (kernels generated for the program only): two computed tensors meet in a node
 };
 // chain opcodes: the comfuse_op_t values of the unary / binary nodes, plus the reversed non-commutative forms
 constexpr int kChainRsub = 38;  // v = operand - v
 constexpr int kChainRdiv = 39;  // v = operand / v
+constexpr int kChainMov = 40;   // v = operand (a chain that starts from a broadcast: sigmoid(row vector), ...)
 // micro-instructions of a pass's stream (besides the chain operations)
 constexpr int kChainXsave = 66;  // x = v (pass 0, after the entry chain)
 constexpr int kChainXload = 67;  // v = x
 constexpr int kChainAcc = 68;    // accumulate v into the thread-local partial of reduction `index`
 constexpr int kChainEmit = 69;   // round v and stage it for the output store
+constexpr int kChainTsave = 70;  // temporary `index` = v (generated kernels only: the temporaries are registers there)
+constexpr int kStageMaxTemps = 3;
 
 struct ChainInstr {
   uint8_t op;
@@ -97,7 +101,8 @@ struct StageProgram {
   uint8_t n_red, n_scalar_instr, n_passes, terminal_pass;
   uint8_t n_row_out;
   uint8_t x_writeback;  // x goes back to tensor memory even in a one-pass program (a Top-K re-reads it)
-  uint8_t pad[2];
+  uint8_t uses_temps;   // the code uses temporaries (CHO_T, TSAVE): runs as generated code only, the interpreter refuses it
+  uint8_t pad[1];
   // per pass, the micro-instruction stream run on every 32-column fragment: code[pass_off[s] .. pass_off[s + 1]).
   // pass 0: entry chain, XSAVE; every pass: per reduction of the pass (XLOAD if v was changed,) its chain, ACC; the
   // terminal's pass: (XLOAD,) final chain, ACC of the reductions on y, EMIT.

@@ -8,6 +8,7 @@ namespace comfuse {
 cudaError_t launch_fused_program_large(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 
 cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
+  if (p.program.uses_temps) return cudaErrorInvalidValue;  // temporaries exist as registers of generated code only
 #define COMFUSE_CASE(n, b0, b1, cn, nst, lock) \
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_PROGRAM, b0, b1, cn, nst, lock>(maps, p, st);

@@ -403,6 +403,9 @@ struct StageLowering {
   std::vector<int> scalar_of;  // per node: its per-row scalar index, -1 = none
   std::vector<int> recip_of;   // per node: the scalar holding its reciprocal, -1 = not needed yet
   int x_root = -1;
+  bool pass0 = false;          // the code being emitted runs in pass 0 (the full-tensor operand is at hand there)
+  int temps_in_use = 0;        // temporaries holding a value at this point of the code being emitted
+  bool uses_temps = false;
   int scalars = 0;             // per-row scalars allocated so far
   StageProgram* sp = nullptr;
   explicit StageLowering(const Analysis& a, StageBinding& b) : an(a), bind(b), scalar_of(a.n, -1), recip_of(a.n, -1) {}
@@ -450,7 +453,7 @@ struct StageLowering {
         return true;
       }
       case COMFUSE_OP_TENSOR:
-        if (!entry_mode) return false;  // the operand ring delivers it once, in pass 0
+        if (!entry_mode && !pass0) return false;  // the operand ring delivers it once, in pass 0
         if (bind.tensor_param >= 0 && bind.tensor_param != an.nodes[k].param) return false;
         bind.tensor_param = an.nodes[k].param;
         ci.operand = CHO_RESIDUAL;
@@ -460,51 +463,101 @@ struct StageLowering {
     }
   }
   bool is_root(int k, bool entry_mode) const { return entry_mode ? an.nodes[k].op == COMFUSE_OP_ACC : k == x_root; }
-  // code that turns the root's value into node k's value
-  bool chain(int k, bool entry_mode, std::vector<ChainInstr>& out) {
-    if (is_root(k, entry_mode)) return true;
+  // code that turns the root's value into node k's value (v holds the root's value where the code starts)
+  bool chain(int k, bool entry_mode, std::vector<ChainInstr>& out, bool in_pass0 = false) {
+    bool v_root = true;
+    pass0 = entry_mode || in_pass0;
+    return emit(k, entry_mode, out, v_root);
+  }
+  // code that leaves node k's value in v; `v_root`: v holds the root's value at this point
+  bool emit(int k, bool entry_mode, std::vector<ChainInstr>& out, bool& v_root) {
+    const size_t mark = out.size();
+    const bool v_root_in = v_root;
+    const int temps_in = temps_in_use;
+    if (emit_node(k, entry_mode, out, v_root)) return true;
+    out.resize(mark);  // a failed attempt leaves no code behind
+    v_root = v_root_in;
+    temps_in_use = temps_in;
+    return false;
+  }
+  bool emit_node(int k, bool entry_mode, std::vector<ChainInstr>& out, bool& v_root) {
+    if (is_root(k, entry_mode)) {
+      if (!v_root) out.push_back(ChainInstr{static_cast<uint8_t>(kChainXload), CHO_NONE, 0, 0.f});  // x: the root (before XSAVE: the accumulator)
+      v_root = true;
+      return true;
+    }
     if (!tensor(k)) return false;
     const comfuse_spec_node_t& nd = an.nodes[k];
     if (is_unary(nd.op)) {
-      if (!chain(nd.in0, entry_mode, out)) return false;
+      if (!emit(nd.in0, entry_mode, out, v_root)) return false;
+      v_root = false;
       out.push_back(ChainInstr{static_cast<uint8_t>(nd.op), CHO_NONE, 0, 0.f});
       return true;
     }
-    if (!is_binary(nd.op)) return false;  // a tensor leaf that is not the root cannot start a chain
-    const int a = nd.in0, b = nd.in1;
     ChainInstr ci;
-    auto carrier = [&](int q) { return is_root(q, entry_mode) || (tensor(q) && !is_leaf(an.nodes[q].op)); };
-    if (a == b && nd.op == COMFUSE_OP_MUL && carrier(a)) {
-      if (!chain(a, entry_mode, out)) return false;
-      out.push_back(ChainInstr{COMFUSE_OP_SQUARE, CHO_NONE, 0, 0.f});
+    if (is_leaf(nd.op)) {
+      // a chain that starts from a broadcast (row vector, causal mask, in pass 0 the full tensor): v = operand
+      if (!operand(k, entry_mode, ci)) return false;
+      ci.op = static_cast<uint8_t>(kChainMov);
+      out.push_back(ci);
+      v_root = false;
       return true;
     }
-    if (carrier(a) && !carrier(b) && operand(b, entry_mode, ci)) {
-      if (!chain(a, entry_mode, out)) return false;
+    if (!is_binary(nd.op)) return false;
+    const int a = nd.in0, b = nd.in1;
+    auto carrier = [&](int q) { return is_root(q, entry_mode) || (tensor(q) && !is_leaf(an.nodes[q].op)); };
+    if (a == b && nd.op == COMFUSE_OP_MUL && carrier(a)) {
+      if (!emit(a, entry_mode, out, v_root)) return false;
+      out.push_back(ChainInstr{COMFUSE_OP_SQUARE, CHO_NONE, 0, 0.f});
+      v_root = false;
+      return true;
+    }
+    auto starts = [&](int q) { return carrier(q) || (tensor(q) && is_leaf(an.nodes[q].op)); };  // something a chain can begin with
+    if (starts(a) && !carrier(b) && operand(b, entry_mode, ci)) {
+      if (!emit(a, entry_mode, out, v_root)) return false;
       ci.op = static_cast<uint8_t>(nd.op);
       if (nd.op == COMFUSE_OP_DIV && !divide_by(b, ci)) return false;
       out.push_back(ci);
+      v_root = false;
       return true;
     }
-    if (carrier(b) && !carrier(a) && operand(a, entry_mode, ci)) {
-      if (!chain(b, entry_mode, out)) return false;
+    if (starts(b) && !carrier(a) && operand(a, entry_mode, ci)) {
+      if (!emit(b, entry_mode, out, v_root)) return false;
       ci.op = static_cast<uint8_t>(nd.op == COMFUSE_OP_SUB ? kChainRsub : nd.op == COMFUSE_OP_DIV ? kChainRdiv : nd.op);
       out.push_back(ci);
+      v_root = false;
       return true;
     }
     // a computed tensor combined with the root itself (a gate: x * sigmoid(x)): the root is at hand in every pass
     if (is_root(a, entry_mode) && carrier(b) && !is_root(b, entry_mode)) {
-      if (!chain(b, entry_mode, out)) return false;
+      if (!emit(b, entry_mode, out, v_root)) return false;
       out.push_back(ChainInstr{static_cast<uint8_t>(nd.op == COMFUSE_OP_SUB ? kChainRsub : nd.op == COMFUSE_OP_DIV ? kChainRdiv : nd.op),
                                CHO_X, 0, 0.f});
+      v_root = false;
       return true;
     }
     if (is_root(b, entry_mode) && carrier(a) && !is_root(a, entry_mode)) {
-      if (!chain(a, entry_mode, out)) return false;
+      if (!emit(a, entry_mode, out, v_root)) return false;
       out.push_back(ChainInstr{static_cast<uint8_t>(nd.op), CHO_X, 0, 0.f});
+      v_root = false;
       return true;
     }
-    return false;  // two computed tensors (needs a second resident tensor), or two broadcasts
+    // two computed tensors meet: the first goes into a temporary while the second is computed (generated kernels only: the
+    // temporaries are registers of straight-line code there; shared sub-expressions are the compiler's to find)
+    if (carrier(a) && carrier(b) && temps_in_use < kStageMaxTemps) {
+      if (!emit(a, entry_mode, out, v_root)) return false;
+      const int t = temps_in_use++;
+      out.push_back(ChainInstr{static_cast<uint8_t>(kChainTsave), CHO_NONE, static_cast<int16_t>(t), 0.f});
+      if (!emit(b, entry_mode, out, v_root)) return false;
+      // v = b, temporary = a: a (op) b in the reversed forms where the order matters
+      out.push_back(ChainInstr{static_cast<uint8_t>(nd.op == COMFUSE_OP_SUB ? kChainRsub : nd.op == COMFUSE_OP_DIV ? kChainRdiv : nd.op),
+                               CHO_T, static_cast<int16_t>(t), 0.f});
+      --temps_in_use;
+      uses_temps = true;
+      v_root = false;
+      return true;
+    }
+    return false;  // more live tensors than temporaries, or two broadcasts
   }
 };
 
@@ -528,7 +581,8 @@ bool lower_stage_program(const Analysis& an, StageProgram& sp, StageBinding& bin
       if (!seen) cand.push_back(e);
     }
   }
-  if (cand.size() > 1) return false;
+  // (several such tensors: none of them can be THE resident one, but a tensor below them all -- in the end the accumulator
+  // itself -- can, with the others recomputed from it in every pass that reads them: the loop below)
   if (cand.size() == 1) {
     StageBinding b1;
     if (lower_stage_program_from(an, cand[0], sp, b1)) { bind = b1; return true; }
@@ -579,7 +633,7 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
         r.pass = static_cast<uint8_t>(an.stage[e]);
         red_chain.emplace_back();
         if (e == an.terminal) r.on_terminal = 1;
-        else if (!L.chain(e, false, red_chain.back())) return false;
+        else if (!L.chain(e, false, red_chain.back())) return false;  // (no full tensor: the later rounds re-run this code)
         if (r.pass > max_pass) max_pass = r.pass;
         topk_input[sp.n_red] = e;
         found = sp.n_red++;
@@ -599,7 +653,7 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
       r.dst = static_cast<uint8_t>(my);
       red_chain.emplace_back();
       if (e == an.terminal) r.on_terminal = 1;
-      else if (!L.chain(e, false, red_chain.back())) return false;
+      else if (!L.chain(e, false, red_chain.back(), r.pass == 0)) return false;
       if (r.pass > max_pass) max_pass = r.pass;
       ++sp.n_red;
     } else {
@@ -620,7 +674,7 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
     L.scalar_of[k] = my;
   }
   // the terminal: x -> y
-  if (!L.chain(an.terminal, false, fin)) return false;
+  if (!L.chain(an.terminal, false, fin, an.stage[an.terminal] == 0)) return false;
   sp.terminal_pass = static_cast<uint8_t>(an.stage[an.terminal]);
   if (max_pass + 1 > kStageMaxPasses) return false;
   sp.n_passes = static_cast<uint8_t>(max_pass + 1);
@@ -698,6 +752,7 @@ bool lower_stage_program_from(const Analysis& an, int x_root, StageProgram& sp, 
   }
   sp.sweep[ns - 1].release = 1;
   sp.n_sweeps = static_cast<uint8_t>(ns);
+  sp.uses_temps = L.uses_temps ? 1 : 0;
   return true;
 }
 
@@ -851,7 +906,8 @@ struct Decision {
   Analysis an;
   FusedMatch match;
   bool fused = false;       // a compiled fused kind
-  bool on_chip = false;     // the on-chip stage-program interpreter
+  bool on_chip = false;     // the on-chip stage program (generated kernel or interpreter)
+  bool interp_ok = false;   // ... which the interpreter can run (no temporaries)
   StageProgram stage_prog;
   StageBinding stage_bind;
   size_t fused_inner_ws = 0;  // what the fused entry point itself needs
@@ -877,8 +933,13 @@ comfuse_status_t decide(const comfuse_fusion_spec_t* spec, const comfuse_gemm_sh
   }
   if (want_fused && !dc.fused && lower_stage_program(dc.an, dc.stage_prog, dc.stage_bind)) {
     const void* none[3] = {nullptr, nullptr, nullptr};
-    dc.on_chip = run_fused_program(shape->batch, shape->M, shape->N, shape->K, 0, 0, 0, 0, 0, 0, nullptr, nullptr, nullptr, dc.stage_prog,
-                                   none, nullptr, 0, nullptr, true, false, want_fused == 3) == COMFUSE_OK;
+    auto query = [&](bool compiled) {
+      return run_fused_program(shape->batch, shape->M, shape->N, shape->K, 0, 0, 0, 0, 0, 0, nullptr, nullptr, nullptr, dc.stage_prog, none,
+                               nullptr, 0, nullptr, true, false, compiled) == COMFUSE_OK;
+    };
+    dc.interp_ok = want_fused != 3 && query(false);
+    const bool generated_ok = (want_fused == 3 || (want_fused == 1 && generate_by_default())) && query(true);
+    dc.on_chip = dc.interp_ok || generated_ok;
     if (dc.on_chip && want_fused == 1 && !on_chip_is_cheaper(dc.an, dc.stage_prog, shape->N)) dc.on_chip = false;
   }
   return COMFUSE_OK;
@@ -1035,7 +1096,7 @@ comfuse_status_t comfuse_gemm_spec(const comfuse_fusion_spec_t* spec, const comf
       // the best path: the kernel generated for this program; where it cannot be had (the compilation failed), the interpreter
       s = run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
                             shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res, ldres, st, false, b_nk, true);
-      if (s != COMFUSE_ERR_UNSUPPORTED) return s;
+      if (s != COMFUSE_ERR_UNSUPPORTED || !dc.interp_ok) return s;
     }
     return run_fused_program(shape->batch, shape->M, shape->N, shape->K, shape->lda, shape->ldb, shape->ldy, shape->batch_stride_a,
                              shape->batch_stride_b, shape->batch_stride_y, A, B, Y, sp, vecs, res, ldres, st, false, b_nk, fused == 3);

@@ -43,9 +43,9 @@ def test_topk_program_compiles(compiler):
 
 
 def test_requests_the_pathway_refuses(compiler):
-    N_ = ("acc", -1, -1, -1, 0.0)     # relu(x) * tanh(x): two computed tensors meet in one node, no on-chip lowering
-    dag = wl.SpecProgram([N_, ("relu", 0, -1, -1, 0.0), ("tanh", 0, -1, -1, 0.0), ("mul", 1, 2, -1, 0.0), ("rmax", 3, -1, -1, 0.0),
-                          ("sub", 3, 4, -1, 0.0)], 5, (), ())
+    N_ = ("acc", -1, -1, -1, 0.0)     # a full tensor used behind a reduction: no on-chip lowering
+    dag = wl.SpecProgram([N_, ("mean", 0, -1, -1, 0.0), ("sub", 0, 1, -1, 0.0), ("tensor", -1, -1, 0, 0.0), ("add", 2, 3, -1, 0.0)], 4, (),
+                         ("tensor",))
     with pytest.raises(cf.ComfuseError) as e:
         cf.gemm_spec_prepare(_spec(dag), cf.make_gemm_shape(1, 300, 1024, 64), cf.GENERATED)
     assert e.value.status == cf.ERR_UNSUPPORTED
@@ -73,6 +73,21 @@ def test_without_a_toolkit_the_pathway_says_so():
     r = subprocess.run([sys.executable, "-c", "import paper_2608_03537_b200 as cf; print(cf.program_compiler_status())"],
                        cwd=ROOT, capture_output=True, text=True, env=dict(os.environ, CUDA_HOME="/nonexistent"))
     assert r.returncode == 0 and "not found" in r.stdout
+
+
+def test_two_computed_tensors_meet_in_generated_code_only(compiler, monkeypatch):
+    """relu(x) * tanh(x): the first factor waits in a temporary while the second is computed -- registers of the generated
+    kernel; the interpreter has none, so `fused` = 2 plans the row program and `fused` = 1 the on-chip form."""
+    N_ = ("acc", -1, -1, -1, 0.0)
+    nodes = [N_, ("rowvec", -1, -1, 0, 0.0), ("add", 0, 1, -1, 0.0), ("relu", 2, -1, -1, 0.0), ("tanh", 2, -1, -1, 0.0),
+             ("mul", 3, 4, -1, 0.0), ("rmax", 5, -1, -1, 0.0), ("sub", 5, 6, -1, 0.0)]
+    prog = wl.SpecProgram(nodes, 7, (6,), ("rowvec",))
+    shape = cf.make_gemm_shape(1, 300, 1024, 64)
+    plan = cf.spec_plan(_spec(prog), shape)
+    assert plan.path == cf.SPEC_PATH_FUSED_PROGRAM and plan.program_path == cf.SPEC_PATH_ROW_PROGRAM
+    cf.gemm_spec_prepare(_spec(prog), shape, cf.GENERATED)
+    monkeypatch.setenv("COMFUSE_GENERATE", "0")
+    assert cf.spec_plan(_spec(prog), shape).path == cf.SPEC_PATH_ROW_PROGRAM
 
 
 def test_the_generated_translation_unit_can_be_dumped(compiler, tmp_path, monkeypatch):

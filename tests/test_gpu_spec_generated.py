@@ -95,6 +95,46 @@ def test_generated_gated_program_equals_the_interpreter(M, N, K, no_contraction)
     assert np.isfinite(err).all() and err.max() <= 4e-3
 
 
+def _dag_programs():
+    N_ = ("acc", -1, -1, -1, 0.0)
+    progs = {}
+    # relu(x) * tanh(x) with x = acc + bias, minus its row maximum
+    progs["two_factors"] = wl.SpecProgram(
+        [N_, ("rowvec", -1, -1, 0, 0.0), ("add", 0, 1, -1, 0.0), ("relu", 2, -1, -1, 0.0), ("tanh", 2, -1, -1, 0.0), ("mul", 3, 4, -1, 0.0),
+         ("rmax", 5, -1, -1, 0.0), ("sub", 5, 6, -1, 0.0)], 7, (6,), ("rowvec",))
+    # three computed tensors alive at once: (sigmoid(x) - tanh(x)) / (1.5 + tanh(abs(x) * g)), normalised by its row mean square
+    progs["three_live"] = wl.SpecProgram(
+        [N_, ("sigmoid", 0, -1, -1, 0.0), ("tanh", 0, -1, -1, 0.0), ("sub", 1, 2, -1, 0.0), ("abs", 0, -1, -1, 0.0), ("rowvec", -1, -1, 0, 0.0),
+         ("mul", 4, 5, -1, 0.0), ("tanh", 6, -1, -1, 0.0), ("const", -1, -1, -1, 1.5), ("add", 7, 8, -1, 0.0), ("div", 3, 9, -1, 0.0),
+         ("square", 10, -1, -1, 0.0), ("mean", 11, -1, -1, 0.0), ("const", -1, -1, -1, 1e-3), ("add", 12, 13, -1, 0.0), ("rsqrt", 14, -1, -1, 0.0),
+         ("mul", 10, 15, -1, 0.0)], 16, (12,), ("rowvec",))
+    # the two factors are used again behind the reduction, with a residual tensor inside one of them
+    progs["residual_gate"] = wl.SpecProgram(
+        [N_, ("tensor", -1, -1, 0, 0.0), ("add", 0, 1, -1, 0.0), ("gelu_tanh", 2, -1, -1, 0.0), ("neg", 0, -1, -1, 0.0), ("sigmoid", 4, -1, -1, 0.0),
+         ("mul", 3, 5, -1, 0.0), ("rmin", 6, -1, -1, 0.0), ("rmax", 6, -1, -1, 0.0), ("sub", 8, 7, -1, 0.0), ("const", -1, -1, -1, 1e-3),
+         ("add", 9, 10, -1, 0.0), ("sub", 6, 7, -1, 0.0), ("div", 12, 11, -1, 0.0)], 13, (7, 8), ("tensor",))
+    return progs
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 256, 72), (260, 1024, 136), (1100, 2048, 64)])
+@pytest.mark.parametrize("name", ["two_factors", "three_live", "residual_gate"])
+def test_programs_in_which_computed_tensors_meet_run_as_generated_code(name, M, N, K):
+    """Two or three computed tensors alive at once: temporaries of the generated kernel (registers); the interpreter has
+    none, so `fused` = 2 takes the row program, and both are compared with the node-list oracle."""
+    prog = _dag_programs()[name]
+    A, B, params = _inputs(68, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, cf.GENERATED, 1, M, N)
+    assert launches == 1 and plan.path == cf.SPEC_PATH_FUSED_PROGRAM and plan.program_path == cf.SPEC_PATH_ROW_PROGRAM
+    Yref, Rref = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    scale = max(1.0, float(np.abs(Yref).max()))
+    assert np.isfinite(err).all() and err.max() <= 8e-3 * scale and err.mean() <= 1e-3 * scale, (err.max(), err.mean(), scale)
+    for got, ref in zip(ro, Rref):
+        np.testing.assert_allclose(got.cpu().numpy(), ref, rtol=2e-3, atol=2e-3)
+    Y1, ro1, _, launches1 = _run(prog, A, B, params, 1, 1, M, N)     # the best path is the same kernel
+    assert launches1 == 1 and _same(Y, Y1)
+
+
 def test_generated_kernel_with_the_operand_stored_n_by_k(no_contraction):
     prog = wl.spec_range_normalise()
     A, B, params = _inputs(64, 1, 300, 1024, 136, prog.param_kinds)
@@ -165,9 +205,9 @@ def test_programs_that_differ_in_constants_share_a_kernel():
 
 
 def test_generated_kernel_is_refused_where_the_program_has_no_on_chip_lowering():
-    N_ = ("acc", -1, -1, -1, 0.0)       # relu(x) * tanh(x): two computed tensors meet in one node
-    prog = wl.SpecProgram([N_, ("relu", 0, -1, -1, 0.0), ("tanh", 0, -1, -1, 0.0), ("mul", 1, 2, -1, 0.0), ("rmax", 3, -1, -1, 0.0),
-                           ("sub", 3, 4, -1, 0.0)], 5, (), ())
+    N_ = ("acc", -1, -1, -1, 0.0)       # a full tensor used behind a reduction
+    prog = wl.SpecProgram([N_, ("mean", 0, -1, -1, 0.0), ("sub", 0, 1, -1, 0.0), ("tensor", -1, -1, 0, 0.0), ("add", 2, 3, -1, 0.0)], 4, (),
+                          ("tensor",))
     A, B, params = _inputs(66, 1, 130, 256, 64, prog.param_kinds)
     with pytest.raises(cf.ComfuseError) as e:
         _run(prog, A, B, params, cf.GENERATED, 1, 130, 256)
