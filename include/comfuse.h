@@ -112,7 +112,7 @@ typedef struct {
   int32_t* row_argmax;
 } comfuse_epilogue_args_t;
 
-/* Bytes of caller-provided workspace the described call can use.  Most fused calls need none.  Two cases of the LayerNorm /
+/* Bytes of caller-provided workspace the described call can use.  Most fused calls need none.  Three cases of the LayerNorm /
  * RMSNorm kinds run as TWO kernels and report batch * M * (N / block) * 8 bytes: the fused kernel finishes stage 1 per
  * column block, stores the un-normalised row in Y as fp16 (11 significant bits) and one partial statistic per row and
  * block in the workspace; a second kernel merges the partials and rescales the row in place to bf16.
@@ -123,6 +123,10 @@ typedef struct {
  *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
  *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
  *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.
+ *   - Row lengths that are a multiple of 256 but have no on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048,
+ *     4096) -- 1280, 1536, 2560, 3072, 5120, ... up to 65536 -- at any K, block = 256.  The workspace is required.
+ *   Other row lengths of these two kinds (not a multiple of 256) are COMFUSE_ERR_UNSUPPORTED with fused = 1; the softmax kind
+ *   takes any N that is a multiple of 8.
  * The results of both forms meet the same tolerances as the one-kernel path. */
 comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes);
 

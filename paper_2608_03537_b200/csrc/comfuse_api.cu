@@ -87,7 +87,12 @@ int split_row_block(int epi, int N, int K) {
   // K = 256 64 / 62 (LayerNorm 57 / 66); N = 2048: K = 4096 147 / 118, K = 1024 59 / 55; N = 1024, K = 4096: 55 / 69.
   // The clusters of 16 and 8 CTAs that hold rows of 4096 and 2048 columns fill 112 and 120 of the 148 SMs and cannot overlap
   // a tile's epilogue with the next MainLoop; the 256-column tiles of the two-kernel form can, on every SM.
-  return (N >= 2048 && N % 256 == 0 && K >= 1024) ? 256 : 0;
+  if (N >= 2048 && N % 256 == 0 && K >= 1024) return 256;
+  // A row length that no single-kernel instantiation covers (1280, 1536, 2560, 3072, 5120, ...): the two-kernel form takes
+  // any multiple of 256, at any K -- one fp16 trip of the row, which is still cheaper than the unfused path's bf16 Z plus
+  // a row kernel.
+  const bool on_chip = N == 256 || N == 512 || N == 768 || N == 1024 || N == 2048 || N == 4096;
+  return (!on_chip && N % kWideRowBlock != 0 && N % 256 == 0 && N <= 16 * kWideRowBlock) ? 256 : 0;  // (multiples of 4096: 4096-column blocks)
 }
 
 const DeviceInfo* current_device_info() {

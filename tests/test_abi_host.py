@@ -76,7 +76,9 @@ def test_wide_row_and_host_staging_sizes():
     long_k = dict(K=1024, lda=1024)                                        # ... or, behind K >= 1024, in 256-column tiles
     assert _ws(_desc(**wide, **long_k)) == (cf.OK, 256 * 32 * 8)
     assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144, **long_k)) == (cf.OK, 256 * 24 * 8)
-    assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144))[0] == cf.ERR_UNSUPPORTED
+    assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144)) == (cf.OK, 256 * 24 * 8)   # no single-kernel form for this row length: any K
+    assert _ws(_desc(N=1536, ldb=1536, ldr=1536, ldy=1536)) == (cf.OK, 256 * 6 * 8)
+    assert _ws(_desc(N=1408, ldb=1408, ldr=1408, ldy=1408))[0] == cf.ERR_UNSUPPORTED   # not a multiple of 256
     assert _ws(_desc(N=4096, ldb=4096, ldr=4096, ldy=4096, **long_k)) == (cf.OK, 256 * 16 * 8)   # optional for rows that fit a cluster
     d = _desc()                                                            # A [256, 512], B [512, 768], R, Y [256, 768], dense
     n = ctypes.c_size_t(0)

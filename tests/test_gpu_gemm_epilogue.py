@@ -111,6 +111,22 @@ def test_wide_rows_behind_a_long_contraction_run_in_256_column_tiles(M, N, K, cu
     P.check_outputs(w, got, P.run_oracle(w), label=f"RMS wide 256-tiles {M}x{N}x{K}", rowmax_tol=3e-2)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 1536, 200), (520, 3072, 64), (129, 1280, 520), (260, 5120, 136), (4100, 2560, 72)])
+def test_row_lengths_without_a_single_kernel_form_run_in_256_column_tiles(M, N, K, cuda_device):
+    """Multiples of 256 that no on-chip instantiation covers (1280, 1536, 2560, 3072, 5120, ...), at any K: the two-kernel form."""
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(M, N, K, seed=N + K, affine=True, relu=(N == 3072))
+    T = P.dev_tensors(w)
+    desc = cf.make_gemm_desc(T["A"], T["B"], torch.empty(M, N, dtype=torch.bfloat16, device=T["A"].device),
+                             cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=True)
+    assert cf.workspace_size(desc) == M * (N // 256) * 8
+    got = P.run_gpu(w, T, fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN 256-tiles {M}x{N}x{K}")
+    w = wl.complex_subgraph(M, N, K, seed=M + N)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"RMS 256-tiles {M}x{N}x{K}", rowmax_tol=3e-2)
+
+
 def test_wide_rows_need_their_workspace(cuda_device):
     import paper_2608_03537_b200 as cf
     w = wl.post_norm(128, 8192, 64, seed=3, affine=False)
