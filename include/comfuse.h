@@ -123,10 +123,10 @@ typedef struct {
  *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
  *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
  *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.
- *   - Row lengths that are a multiple of 256 but have no on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048,
- *     4096) -- 1280, 1536, 2560, 3072, 5120, ... up to 65536 -- at any K, block = 256.  The workspace is required.
- *   Other row lengths of these two kinds (not a multiple of 256) are COMFUSE_ERR_UNSUPPORTED with fused = 1; the softmax kind
- *   takes any N that is a multiple of 8.
+ *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096) that are not a
+ *     multiple of 4096 -- 1000, 1280, 1536, 1600, 3072, 5120, ... any multiple of 8 up to 65536 -- at any K, block = 256,
+ *     (N + 255) / 256 blocks: the last tile may be a partial one.  The workspace is required.
+ *   With these every row length that is a multiple of 8 (up to 65536 columns) has a fused form for all three kinds.
  * The results of both forms meet the same tolerances as the one-kernel path. */
 comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t* bytes);
 

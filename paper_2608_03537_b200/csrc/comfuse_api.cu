@@ -92,7 +92,9 @@ int split_row_block(int epi, int N, int K) {
   // any multiple of 256, at any K -- one fp16 trip of the row, which is still cheaper than the unfused path's bf16 Z plus
   // a row kernel.
   const bool on_chip = N == 256 || N == 512 || N == 768 || N == 1024 || N == 2048 || N == 4096;
-  return (!on_chip && N % kWideRowBlock != 0 && N % 256 == 0 && N <= 16 * kWideRowBlock) ? 256 : 0;  // (multiples of 4096: 4096-column blocks)
+  // (multiples of 4096: 4096-column blocks.)  N need not be a multiple of 256: the last tile is a partial one -- operands
+  // outside the matrix read as zeros, stores are clipped, and the second kernel corrects that tile's statistic for them.
+  return (!on_chip && N % kWideRowBlock != 0 && N <= 16 * kWideRowBlock) ? 256 : 0;
 }
 
 const DeviceInfo* current_device_info() {
@@ -468,7 +470,7 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
       r.Y = static_cast<uint16_t*>(Y);
       r.ldy = desc->ldy; r.batch_stride_y = bsy;
       r.row_max = a.row_max; r.row_argmax = a.row_argmax;
-      e = launch_wide_row_finish(epi, r, p.wide_partials, wide_blocks, st);
+      e = launch_wide_row_finish(epi, r, p.wide_partials, wide_blocks, p.wide_block, st);
     }
     return e == cudaSuccess ? COMFUSE_OK : COMFUSE_ERR_CUDA;
   }

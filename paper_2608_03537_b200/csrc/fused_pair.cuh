@@ -402,6 +402,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
               if (!(p.trace_flags & 1))
 #endif
+              if (col < p.N)  // (a group of a partial last tile may lie outside the matrix altogether: nothing to store)
               if (COMFUSE_IN_BOUNDS(col >= 0 && col < p.N && (col & 7) == 0 && m0 + q * 32 >= 0 && b >= 0 && b < p.batch, p.status))
               tma_store_3d_hint(&tmY, ring_box(e, kk), col, m0 + q * 32, b, once);
               tma_store_commit();
@@ -413,6 +414,7 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #ifdef COMFUSE_TRACE
             if (!(p.trace_flags & 1))
 #endif
+            if (col < p.N)
             if (COMFUSE_IN_BOUNDS(col >= 0 && col < p.N && (col & 7) == 0 && m0 + q * 32 >= 0 && b >= 0 && b < p.batch, p.status))
             tma_store_3d_hint(&tmY, ybox0 + sel * Cfg::WARP_BOX_BYTES, col, m0 + q * 32, b, once);
             tma_store_commit();

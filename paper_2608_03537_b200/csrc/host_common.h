@@ -68,7 +68,7 @@ inline int wide_row_block(int epi, int N, int K) {
 }
 inline int wide_row_blocks(int epi, int N, int K) {
   const int w = wide_row_block(epi, N, K);
-  return w ? N / w : 0;
+  return w ? (N + w - 1) / w : 0;
 }
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).

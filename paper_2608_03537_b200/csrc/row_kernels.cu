@@ -228,7 +228,7 @@ __device__ __forceinline__ void unpack8_f16(const uint4 q4, float (&xf)[8]) {
 }
 
 template <int KIND>
-__global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p, const float2* partials, int nblocks, long long rows) {
+__global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p, const float2* partials, int nblocks, int block, long long rows) {
   // launched with programmatic stream serialization: everything above this line may overlap the first kernel's tail
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int lane = threadIdx.x & 31;
@@ -240,19 +240,42 @@ __global__ void __launch_bounds__(256) wide_row_finish_kernel(const RowParams p,
   const int i = static_cast<int>(r - static_cast<long long>(b) * p.M);
   uint16_t* y = p.Y + static_cast<long long>(b) * p.batch_stride_y + static_cast<long long>(i) * p.ldy;
   const float2* q = partials + r * nblocks;
-  const float wb = static_cast<float>(p.N / nblocks);  // columns per block (equal by construction)
+  const float wb = static_cast<float>(block);                    // columns per block
+  const int last = p.N - (nblocks - 1) * block;                  // valid columns of the last block (== block: none partial)
   float mu = 0.f, rstd;
   if constexpr (KIND == EPI_LN) {
-    // equal-count Chan merge: mean of the block means, M2 = sum M2_b + wb * sum (mean_b - mean)^2
-    float ms = 0.f;
-    for (int k = 0; k < nblocks; ++k) ms += q[k].x;
-    mu = ms / static_cast<float>(nblocks);
-    float m2 = 0.f;
-    for (int k = 0; k < nblocks; ++k) {
-      const float d = q[k].x - mu;
-      m2 += q[k].y + wb * d * d;
+    if (last == block) {
+      // equal-count Chan merge: mean of the block means, M2 = sum M2_b + wb * sum (mean_b - mean)^2
+      float ms = 0.f;
+      for (int k = 0; k < nblocks; ++k) ms += q[k].x;
+      mu = ms / static_cast<float>(nblocks);
+      float m2 = 0.f;
+      for (int k = 0; k < nblocks; ++k) {
+        const float d = q[k].x - mu;
+        m2 += q[k].y + wb * d * d;
+      }
+      rstd = rsqrtf(m2 / static_cast<float>(p.N) + p.eps);
+    } else {
+      // The last block is a partial one: the first kernel's statistic covers its `block` columns, of which block - last
+      // are exact zeros (operands outside the matrix read as zero, the bias is masked).  Zeros add nothing to the sum and
+      // to the sum of squares, so the statistic of the valid columns alone follows: S = wb mean', Sxx = M2' + wb mean'^2,
+      // mean = S / last, M2 = Sxx - last mean^2.  Then the merge with the blocks' true counts.
+      const float lf = static_cast<float>(last);
+      float2 ql = q[nblocks - 1];
+      const float s_last = wb * ql.x, sxx = ql.y + wb * ql.x * ql.x;
+      ql.x = s_last / lf;
+      ql.y = fmaxf(sxx - lf * ql.x * ql.x, 0.f);
+      float ms = lf * ql.x;
+      for (int k = 0; k + 1 < nblocks; ++k) ms += wb * q[k].x;
+      mu = ms / static_cast<float>(p.N);
+      const float dl = ql.x - mu;
+      float m2 = ql.y + lf * dl * dl;
+      for (int k = 0; k + 1 < nblocks; ++k) {
+        const float d = q[k].x - mu;
+        m2 += q[k].y + wb * d * d;
+      }
+      rstd = rsqrtf(m2 / static_cast<float>(p.N) + p.eps);
     }
-    rstd = rsqrtf(m2 / static_cast<float>(p.N) + p.eps);
   } else {
     float ss = 0.f;
     for (int k = 0; k < nblocks; ++k) ss += q[k].x;
@@ -346,7 +369,7 @@ cudaError_t launch_row_epilogue(int kind, const RowParams& p, cudaStream_t st) {
   }
 }
 
-cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, cudaStream_t st) {
+cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, int block, cudaStream_t st) {
   const long long rows = static_cast<long long>(p.batch) * p.M;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
@@ -358,8 +381,8 @@ cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* p
   cfg.attrs = attr;
   cfg.numAttrs = programmatic_launch_enabled() ? 1 : 0;
   count_launch();
-  if (kind == EPI_LN) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_LN>, p, partials, nblocks, rows);
-  if (kind == EPI_RMS_MAX) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_RMS_MAX>, p, partials, nblocks, rows);
+  if (kind == EPI_LN) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_LN>, p, partials, nblocks, block, rows);
+  if (kind == EPI_RMS_MAX) return cudaLaunchKernelEx(&cfg, wide_row_finish_kernel<EPI_RMS_MAX>, p, partials, nblocks, block, rows);
   return cudaErrorInvalidValue;
 }
 

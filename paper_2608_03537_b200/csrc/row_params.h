@@ -28,7 +28,8 @@ struct RowParams {
 
 cudaError_t launch_row_epilogue(int kind, const RowParams& p, cudaStream_t st);
 // Wide rows: merge the per-block partial statistics of each row and rescale the un-normalised row stored in p.Y in place.
-cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, cudaStream_t st);
+// `block` = columns per block of the first kernel; the last block may be a partial one (N not a multiple of `block`)
+cudaError_t launch_wide_row_finish(int kind, const RowParams& p, const float2* partials, int nblocks, int block, cudaStream_t st);
 cudaError_t launch_bias_gelu(uint16_t* P, const uint16_t* bias, long long rows, int n, cudaStream_t st);
 
 }  // namespace comfuse

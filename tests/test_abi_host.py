@@ -49,7 +49,9 @@ def test_workspace_size_rules():
     assert _ws(_desc(fused=0)) == (cf.OK, 256 * 768 * 2)                   # unfused: dense bf16 Z
     assert _ws(_desc(fused=0, batch=3, batch_stride_a=256 * 512, batch_stride_b=512 * 768, batch_stride_y=256 * 768,
                      batch_stride_r=256 * 768)) == (cf.OK, 3 * 256 * 768 * 2)
-    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776))[0] == cf.ERR_UNSUPPORTED      # no fused instantiation for N = 776
+    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776)) == (cf.OK, 256 * 4 * 8)        # no on-chip instantiation for N = 776: two kernels,
+                                                                                      # 256-column tiles, the last one partial
+    assert _ws(_desc(N=70000, ldb=70000, ldr=70000, ldy=70000))[0] == cf.ERR_UNSUPPORTED   # beyond 65536 columns
     assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776, fused=0))[0] == cf.OK          # ... but the unfused path takes it
     assert _ws(_desc(N=770, ldb=776, ldr=776, ldy=776))[0] == cf.ERR_ALIGNMENT        # N must be a multiple of 8
     assert _ws(_desc(lda=516))[0] == cf.ERR_ALIGNMENT                                  # leading dims too
@@ -72,13 +74,13 @@ def test_wide_row_and_host_staging_sizes():
     wide = dict(N=8192, ldb=8192, ldr=8192, ldy=8192)
     assert _ws(_desc(**wide)) == (cf.OK, 256 * 2 * 8)                      # fused wide rows: (mean, M2) per row and 4096-column block
     assert _ws(_desc(**wide, kind=cf.EPI_BIAS_GELU_RES_RMSNORM_MAX)) == (cf.OK, 256 * 2 * 8)
-    assert _ws(_desc(N=8200, ldb=8200, ldr=8200, ldy=8200))[0] == cf.ERR_UNSUPPORTED   # wide rows come in whole 4096-column blocks
+    assert _ws(_desc(N=8200, ldb=8200, ldr=8200, ldy=8200)) == (cf.OK, 256 * 33 * 8)   # not a multiple of 4096: 256-column tiles, a partial last one
     long_k = dict(K=1024, lda=1024)                                        # ... or, behind K >= 1024, in 256-column tiles
     assert _ws(_desc(**wide, **long_k)) == (cf.OK, 256 * 32 * 8)
     assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144, **long_k)) == (cf.OK, 256 * 24 * 8)
     assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144)) == (cf.OK, 256 * 24 * 8)   # no single-kernel form for this row length: any K
     assert _ws(_desc(N=1536, ldb=1536, ldr=1536, ldy=1536)) == (cf.OK, 256 * 6 * 8)
-    assert _ws(_desc(N=1408, ldb=1408, ldr=1408, ldy=1408))[0] == cf.ERR_UNSUPPORTED   # not a multiple of 256
+    assert _ws(_desc(N=1408, ldb=1408, ldr=1408, ldy=1408)) == (cf.OK, 256 * 6 * 8)    # not a multiple of 256: the last tile is partial
     assert _ws(_desc(N=4096, ldb=4096, ldr=4096, ldy=4096, **long_k)) == (cf.OK, 256 * 16 * 8)   # optional for rows that fit a cluster
     d = _desc()                                                            # A [256, 512], B [512, 768], R, Y [256, 768], dense
     n = ctypes.c_size_t(0)

@@ -110,9 +110,12 @@ def test_near_misses_do_not_take_a_compiled_kind(generate, monkeypatch):
     p = wl.spec_softmax(0.5, True)
     pl = _plan(p.nodes, p.terminal, shape=cf.make_gemm_shape(1, 256, 512, 64))
     assert pl.path == ROW and pl.program_path == PROG
-    # a row length without any fused instantiation
+    # a row length without an on-chip instantiation: the compiled LayerNorm kind takes it as two kernels (256-column tiles,
+    # a partial last one); a program outside the compiled kinds has no on-chip form there and goes to the row program
     p = wl.spec_layernorm()
-    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
+    assert _plan(p.nodes, p.terminal, 4, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_FUSED_KERNEL
+    p = wl.spec_range_normalise()
+    assert _plan(p.nodes, p.terminal, 1, p.row_outputs, shape=cf.make_gemm_shape(1, 256, 1000, 64)).path == cf.SPEC_PATH_ROW_PROGRAM
 
 
 def test_on_chip_lowering_needs_one_resident_tensor():
