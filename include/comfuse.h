@@ -286,7 +286,7 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      reductions, 6 row outputs, 4 passes, 80 micro-instructions; the reductions sum, mean, max, min, prod, argmax merge
  *      across the cluster).  Expressions in which two COMPUTED tensors meet (relu(x) * tanh(x)) need temporaries, which
  *      exist in the generated form of the kernel only (3. below): the interpreter (`fused` = 2) sends such a program to the
- *      row program; any other valid program runs on the standard pathway
+ *      row program; the generated form also exists at N in {1280, 1536, 1792, 2560, 3072, 3584}; any other valid program runs on the standard pathway
  *      (COMFUSE_SPEC_PATH_ROW_PROGRAM): the GEMM kernel writes bf16 Z to the workspace and one row-program kernel
  *      evaluates the node list per row with the row resident in shared memory, one pass per stage.
  *   3. on request (`fused` = 3) GENERATES the fused kernel for the program (Sec. 5: the fused epilogue as generated code):

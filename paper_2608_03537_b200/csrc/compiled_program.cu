@@ -225,6 +225,7 @@ cudaError_t launch_compiled_program(const GemmMaps& maps, const FusedParams& p, 
   switch (p.N) {
     COMFUSE_PROGRAM_INSTANCES_SMALL(COMFUSE_CASE)
     COMFUSE_PROGRAM_INSTANCES_LARGE(COMFUSE_CASE)
+    COMFUSE_PROGRAM_INSTANCES_GENERATED_ONLY(COMFUSE_CASE)
     default:
       return cudaErrorInvalidValue;
   }

@@ -86,5 +86,10 @@ cudaError_t launch_pair_instance(const GemmMaps& maps, const FusedParams& p, cud
 // X(N, BNS0, BNS1, CN, NSTAGES, LOCK).  One table for the interpreter's instantiations and for the kernels compiled at run time.
 #define COMFUSE_PROGRAM_INSTANCES_SMALL(X) X(256, 256, 0, 1, 5, 0) X(512, 256, 256, 1, 3, 1) X(768, 256, 128, 2, 4, 1)
 #define COMFUSE_PROGRAM_INSTANCES_LARGE(X) X(1024, 256, 256, 2, 3, 1) X(2048, 256, 256, 4, 3, 1) X(4096, 256, 256, 8, 3, 1)
+// Further row lengths for the kernels generated at run time (an instantiation there costs a table entry, not a translation
+// unit): clusters of 6, 10, 12 and 14 CTAs.
+#define COMFUSE_PROGRAM_INSTANCES_GENERATED_ONLY(X) \
+  X(1280, 256, 0, 5, 5, 0) X(1536, 256, 256, 3, 3, 1) X(1792, 256, 0, 7, 5, 0) X(2560, 256, 256, 5, 3, 1) X(3072, 256, 256, 6, 3, 1) \
+  X(3584, 256, 256, 7, 3, 1)
 
 }  // namespace comfuse

@@ -92,6 +92,34 @@ def test_generated_gated_program_equals_the_interpreter(M, N, K, no_contraction)
     assert np.isfinite(err).all() and err.max() <= 4e-3
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 1280, 72), (520, 1536, 136), (260, 1792, 64), (300, 2560, 72), (1300, 3072, 64), (260, 3584, 200)])
+def test_generated_kernels_at_row_lengths_the_library_has_no_instantiation_for(M, N, K):
+    """Clusters of 10, 6, 14, 10, 12 and 14 CTAs: an instantiation of a generated kernel is a table entry.  The interpreter
+    and the compiled kinds' on-chip forms do not exist at these row lengths."""
+    prog = wl.spec_range_normalise()
+    A, B, params = _inputs(69, 1, M, N, K, prog.param_kinds)
+    Y, ro, plan, launches = _run(prog, A, B, params, 1, 1, M, N)
+    assert launches == 1 and plan.path == cf.SPEC_PATH_FUSED_PROGRAM and plan.program_path == cf.SPEC_PATH_ROW_PROGRAM
+    Yref, Rref = _oracle(prog, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    assert np.isfinite(err).all() and err.max() <= 4e-3 and err.mean() <= 1e-3
+    lo, hi, pr, sm, am = [t.cpu().numpy() for t in ro]
+    np.testing.assert_allclose(lo, Rref[0], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(hi, Rref[1], atol=1e-4, rtol=1e-5)
+    np.testing.assert_allclose(pr, Rref[2], rtol=1e-4)
+    np.testing.assert_allclose(sm, Rref[3], rtol=1e-4)
+    assert np.mean(am == Rref[4].astype(np.int64)) > 0.995
+    # a LayerNorm with an extra row output (not a compiled kind) with its residual through the operand ring
+    ln = wl.spec_layernorm(relu=True)
+    ln = wl.SpecProgram(ln.nodes, ln.terminal, (ln.nodes.index(("mean", 4, -1, -1, 0.0)),), ln.param_kinds)
+    A, B, params = _inputs(70, 1, M, N, K, ln.param_kinds)
+    Y, ro, plan, launches = _run(ln, A, B, params, cf.GENERATED, 1, M, N)
+    Yref, Rref = _oracle(ln, A, B, params, 1)
+    err = np.abs(to_f64(Y) - Yref)
+    assert launches == 1 and np.isfinite(err).all() and err.max() <= 3e-2 and err.mean() <= 3e-3
+    np.testing.assert_allclose(ro[0].cpu().numpy(), Rref[0], atol=2e-3)
+
+
 def _dag_programs():
     N_ = ("acc", -1, -1, -1, 0.0)
     progs = {}
