@@ -297,7 +297,8 @@ const char* comfuse_status_string(comfuse_status_t status);
  *      environment kernels are compiled without contraction and the results are bit-identical.  Constants (CONST nodes) and pointers stay run-time
  *      arguments: programs that differ only in those share a kernel.  The first call that needs a kernel compiles it
  *      (NVRTC from the CUDA toolkit, one to three seconds, on the calling thread) and keeps it for the life of the process;
- *      make that call, or comfuse_gemm_spec_prepare, before any stream capture.  Where the compiler is available `fused` = 1
+ *      make that call, or comfuse_gemm_spec_prepare, before any stream capture.  With COMFUSE_KERNEL_CACHE=<directory>
+ *      in the environment the device images are also kept on disk, and a later process loads them instead of compiling.  Where the compiler is available `fused` = 1
  *      takes this form too whenever it would otherwise interpret (COMFUSE_GENERATE=0 in the environment keeps the
  *      interpreter); comfuse_spec_plan reports COMFUSE_SPEC_PATH_FUSED_PROGRAM for both, they are the same lowering.
  */

@@ -6,9 +6,10 @@
 // the per-row scalars live in registers.  Immediates and row-output pointers stay run-time parameters, so programs that
 // differ only in constants share a kernel.  The compiler is NVRTC, loaded with dlopen when the first program asks for it;
 // the kernel sources are embedded in this library at build time.  A kernel is compiled on the first call that needs it
-// (seconds) and kept for the life of the process.
+// (seconds) and kept for the life of the process; COMFUSE_KERNEL_CACHE=<directory> also keeps the device images on disk.
 #include <dlfcn.h>
 #include <nvrtc.h>
+#include <unistd.h>
 
 #include <cstring>
 #include <memory>
@@ -199,6 +200,58 @@ std::unique_ptr<CompiledKernel> compile_kernel(const std::string& source, const 
   return out;
 }
 
+// Optional cache of device images on disk (COMFUSE_KERNEL_CACHE=<directory>): a process finds the kernels earlier processes
+// compiled.  The file name is a hash of everything the image depends on: instantiation, options, constant table, the embedded
+// kernel sources and the compiler's version.  File = "comfuse-cubin-1\n" lowered-name "\n" image.  Written through a
+// temporary name and renamed, so a reader never sees half a file.
+uint64_t fnv1a(const std::string& text, uint64_t h = 1469598103934665603ull) {
+  for (unsigned char c : text) { h ^= c; h *= 1099511628211ull; }
+  return h;
+}
+std::string disk_cache_path(const std::string& key) {
+  const char* dir = std::getenv("COMFUSE_KERNEL_CACHE");
+  if (!dir || !dir[0]) return std::string();
+  static const uint64_t build = [] {
+    uint64_t h = 1469598103934665603ull;
+    for (int i = 0; i < kEmbeddedSourceCount; ++i) h = fnv1a(kEmbeddedSources[i], h);
+    int major = 0, minor = 0;
+    if (auto version = reinterpret_cast<decltype(&nvrtcVersion)>(compiler().lib ? dlsym(compiler().lib, "nvrtcVersion") : nullptr))
+      version(&major, &minor);
+    return fnv1a(std::to_string(major) + "." + std::to_string(minor), h);
+  }();
+  char name[64];
+  std::snprintf(name, sizeof(name), "/comfuse-%016llx.cubin", static_cast<unsigned long long>(fnv1a(key, build)));
+  return std::string(dir) + name;
+}
+const char kDiskMagic[] = "comfuse-cubin-1\n";
+std::unique_ptr<CompiledKernel> disk_cache_load(const std::string& path) {
+  FILE* f = path.empty() ? nullptr : std::fopen(path.c_str(), "rb");
+  if (!f) return nullptr;
+  std::string all;
+  char buf[1 << 16];
+  for (size_t n; (n = std::fread(buf, 1, sizeof(buf), f)) > 0;) all.append(buf, n);
+  std::fclose(f);
+  const size_t m = sizeof(kDiskMagic) - 1;
+  if (all.compare(0, m, kDiskMagic) != 0) return nullptr;
+  const size_t nl = all.find('\n', m);
+  if (nl == std::string::npos || nl + 1 >= all.size()) return nullptr;
+  std::unique_ptr<CompiledKernel> k(new CompiledKernel);
+  k->lowered_name = all.substr(m, nl - m);
+  k->image.assign(all.begin() + nl + 1, all.end());
+  return k;
+}
+void disk_cache_store(const std::string& path, const CompiledKernel& k) {
+  if (path.empty()) return;
+  const std::string tmp = path + ".tmp" + std::to_string(static_cast<long long>(getpid()));
+  FILE* f = std::fopen(tmp.c_str(), "wb");
+  if (!f) return;
+  bool ok = std::fwrite(kDiskMagic, 1, sizeof(kDiskMagic) - 1, f) == sizeof(kDiskMagic) - 1;
+  ok = ok && std::fwrite(k.lowered_name.data(), 1, k.lowered_name.size(), f) == k.lowered_name.size() && std::fputc('\n', f) != EOF;
+  ok = ok && std::fwrite(k.image.data(), 1, k.image.size(), f) == k.image.size();
+  ok = (std::fclose(f) == 0) && ok;
+  if (!ok || std::rename(tmp.c_str(), path.c_str()) != 0) std::remove(tmp.c_str());
+}
+
 std::mutex g_cache_mutex;
 std::unordered_map<std::string, std::unique_ptr<CompiledKernel>> g_cache;     // key: instance name + constant table
 std::unordered_map<std::string, std::string> g_failed;                         // key -> reason (not retried)
@@ -248,20 +301,28 @@ cudaError_t launch_compiled_program(const GemmMaps& maps, const FusedParams& p, 
       return cudaErrorInvalidValue;
     } else {
       std::string why;
+      const std::string on_disk = disk_cache_path(key);
+      std::unique_ptr<CompiledKernel> made = disk_cache_load(on_disk);
+      if (made) {
+        k = made.get();
+        g_cache[key] = std::move(made);
+      } else {
       if (const char* dump = std::getenv("COMFUSE_GENERATED_DUMP")) {  // the generated translation unit, for inspection
         if (FILE* f = std::fopen(dump, "w")) {
           std::fprintf(f, "// %s\n%s", name, table.c_str());
           std::fclose(f);
         }
       }
-      std::unique_ptr<CompiledKernel> made = compile_kernel(table, name, contract, why);
+      made = compile_kernel(table, name, contract, why);
       if (!made) {
         std::fprintf(stderr, "comfuse: %s\n", why.c_str());
         g_failed[key] = why;
         return cudaErrorInvalidValue;
       }
+      disk_cache_store(on_disk, *made);
       k = made.get();
       g_cache[key] = std::move(made);
+      }
     }
   }
   if (!launch) return cudaSuccess;

@@ -100,3 +100,31 @@ def test_the_generated_translation_unit_can_be_dumped(compiler, tmp_path, monkey
     text = path.read_text()
     assert "kCompiledProgram" in text and "fused_pair_kernel<comfuse::EPI_PROGRAM, 256, 256, 1, 3, 1, 2>" in text
     assert "0.37" not in text            # constants stay run-time arguments: programs that differ only in them share the kernel
+
+
+def test_device_images_can_be_kept_on_disk(compiler, tmp_path):
+    """COMFUSE_KERNEL_CACHE=<directory>: a second process finds the image the first one compiled (the generated translation
+    unit is dumped only when a kernel is actually compiled, so the second process leaves no dump behind)."""
+    cache = tmp_path / "cache"
+    cache.mkdir()
+    code = (
+        "import sys, paper_2608_03537_b200 as cf, workloads as wl\n"
+        "p = wl.spec_range_normalise()\n"
+        "spec = cf.make_spec(p.nodes, p.terminal, len(p.param_kinds), p.row_outputs)\n"
+        "cf.gemm_spec_prepare(spec, cf.make_gemm_shape(1, 300, 2048, 64), cf.GENERATED)\n"
+    )
+    for dump in ("first.cu", "second.cu"):
+        env = dict(os.environ, COMFUSE_KERNEL_CACHE=str(cache), COMFUSE_GENERATED_DUMP=str(tmp_path / dump),
+                   PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
+        r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr[-2000:]
+    files = [f for f in os.listdir(cache) if f.endswith(".cubin")]
+    assert len(files) == 1 and os.path.getsize(cache / files[0]) > 10_000
+    assert (tmp_path / "first.cu").exists() and not (tmp_path / "second.cu").exists()
+    # a damaged file is ignored (and replaced by a fresh compilation), not trusted
+    with open(cache / files[0], "r+b") as f:
+        f.write(b"garbage")
+    env = dict(os.environ, COMFUSE_KERNEL_CACHE=str(cache), COMFUSE_GENERATED_DUMP=str(tmp_path / "third.cu"),
+               PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0 and (tmp_path / "third.cu").exists()
