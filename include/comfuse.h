@@ -123,7 +123,8 @@ typedef struct {
  *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
  *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
  *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.
- *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096) that are not a
+ *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096, and behind
+ *     contractions short enough for it to pay 1280, 1536, 1792: ask this function) that are not a
  *     multiple of 4096 -- 1000, 1280, 1536, 1600, 3072, 5120, ... any multiple of 8 up to 65536 -- at any K, block = 256,
  *     (N + 255) / 256 blocks: the last tile may be a partial one.  The workspace is required.
  *   With these every row length that is a multiple of 8 (up to 65536 columns) has a fused form for all three kinds.

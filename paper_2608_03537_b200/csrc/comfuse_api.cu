@@ -81,7 +81,6 @@ int split_row_block(int epi, int N, int K) {
     const char* e = std::getenv("COMFUSE_SPLIT_BLOCK");
     return e ? std::atoi(e) : -1;
   }();
-  (void)epi;
   if (forced >= 0) return (forced > 0 && N > forced && N % forced == 0) ? forced : 0;
   // Measured (8192 rows; on-chip / two kernels with 256-column blocks, us): N = 4096: K = 4096 242 / 212, K = 1024 101 / 87,
   // K = 256 64 / 62 (LayerNorm 57 / 66); N = 2048: K = 4096 147 / 118, K = 1024 59 / 55; N = 1024, K = 4096: 55 / 69.
@@ -91,7 +90,13 @@ int split_row_block(int epi, int N, int K) {
   // A row length that no single-kernel instantiation covers (1280, 1536, 2560, 3072, 5120, ...): the two-kernel form takes
   // any multiple of 256, at any K -- one fp16 trip of the row, which is still cheaper than the unfused path's bf16 Z plus
   // a row kernel.
-  const bool on_chip = N == 256 || N == 512 || N == 768 || N == 1024 || N == 2048 || N == 4096;
+  // 1280, 1536 and 1792 columns have on-chip forms too, on clusters of 10, 6 and 14 CTAs.  Measured (8192 rows; on chip / two
+  // kernels, us; K = 256, 1024, 2048, 4096): LayerNorm N = 1280: 20 / 27, 29 / 38, 44 / 54, 75 / 87; N = 1536: 24 / 29, 39 / 40,
+  // 58 / 57, 98 / 90; N = 1792: 30 / 33, 42 / 48, 67 / 70, 117 / 114.  RMSNorm N = 1280: 23 / 26, 30 / 37, 46 / 53, 77 / 86;
+  // N = 1536: 27 / 28, 42 / 39, 61 / 55, 102 / 89; N = 1792: 36 / 32, 45 / 46, 70 / 69, 120 / 112.
+  const bool ln = epi == EPI_LN;
+  const bool more_rows = N == 1280 || (N == 1536 && K <= (ln ? 1024 : 256)) || (N == 1792 && ln && K <= 2048);
+  const bool on_chip = N == 256 || N == 512 || N == 768 || N == 1024 || N == 2048 || N == 4096 || more_rows;
   // (multiples of 4096: 4096-column blocks.)  N need not be a multiple of 256: the last tile is a partial one -- operands
   // outside the matrix read as zeros, stores are clipped, and the second kernel corrects that tile's statistic for them.
   return (!on_chip && N % kWideRowBlock != 0 && N <= 16 * kWideRowBlock) ? 256 : 0;

@@ -17,7 +17,7 @@ cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, c
     COMFUSE_CASE(2048, 256, 256, 4, 3, 1)
     COMFUSE_CASE(4096, 256, 256, 8, 3, 1)
     default:
-      return cudaErrorInvalidValue;
+      return launch_fused_norm_more_rows(EPI_LN, maps, p, st, supported_only);  // 1280, 1536, 1792: a translation unit of their own
   }
 #undef COMFUSE_CASE
 }

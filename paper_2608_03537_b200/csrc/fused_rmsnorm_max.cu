@@ -20,7 +20,7 @@ cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p,
     COMFUSE_CASE(2048, 256, 256, 4, 3, 1)
     COMFUSE_CASE(4096, 256, 256, 8, 3, 1)
     default:
-      return cudaErrorInvalidValue;
+      return launch_fused_norm_more_rows(EPI_RMS_MAX, maps, p, st, supported_only);  // 1280, 1536, 1792
   }
 #undef COMFUSE_CASE
 }

@@ -45,6 +45,7 @@ struct GemmMaps {
 // exists without launching.
 cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 cudaError_t launch_fused_rmsnorm_max(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+cudaError_t launch_fused_norm_more_rows(int epi, const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Epilogue = the stage program in p.program, interpreted on-chip (N in {256, 512, 768, 1024, 2048, 4096}).
 cudaError_t launch_fused_program(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // The same kernel with p.program compiled in (generated at run time, cached per program structure and N).  `launch` =

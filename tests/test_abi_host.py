@@ -79,7 +79,9 @@ def test_wide_row_and_host_staging_sizes():
     assert _ws(_desc(**wide, **long_k)) == (cf.OK, 256 * 32 * 8)
     assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144, **long_k)) == (cf.OK, 256 * 24 * 8)
     assert _ws(_desc(N=6144, ldb=6144, ldr=6144, ldy=6144)) == (cf.OK, 256 * 24 * 8)   # no single-kernel form for this row length: any K
-    assert _ws(_desc(N=1536, ldb=1536, ldr=1536, ldy=1536)) == (cf.OK, 256 * 6 * 8)
+    assert _ws(_desc(N=1536, ldb=1536, ldr=1536, ldy=1536)) == (cf.OK, 0)   # K = 512: the on-chip form on a cluster of 6 CTAs
+    assert _ws(_desc(N=1536, ldb=1536, ldr=1536, ldy=1536, K=2048, lda=2048)) == (cf.OK, 256 * 6 * 8)   # long K: two kernels
+    assert _ws(_desc(N=2560, ldb=2560, ldr=2560, ldy=2560)) == (cf.OK, 256 * 10 * 8)
     assert _ws(_desc(N=1408, ldb=1408, ldr=1408, ldy=1408)) == (cf.OK, 256 * 6 * 8)    # not a multiple of 256: the last tile is partial
     assert _ws(_desc(N=4096, ldb=4096, ldr=4096, ldy=4096, **long_k)) == (cf.OK, 256 * 16 * 8)   # optional for rows that fit a cluster
     d = _desc()                                                            # A [256, 512], B [512, 768], R, Y [256, 768], dense

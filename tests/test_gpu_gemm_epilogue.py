@@ -111,7 +111,26 @@ def test_wide_rows_behind_a_long_contraction_run_in_256_column_tiles(M, N, K, cu
     P.check_outputs(w, got, P.run_oracle(w), label=f"RMS wide 256-tiles {M}x{N}x{K}", rowmax_tol=3e-2)
 
 
-@pytest.mark.parametrize("M,N,K", [(300, 1536, 200), (520, 3072, 64), (129, 1280, 520), (260, 5120, 136), (4100, 2560, 72)])
+@pytest.mark.parametrize("M,N,K", [(300, 1536, 200), (129, 1280, 520), (1100, 1280, 2056), (260, 1792, 136), (4100, 1536, 72), (520, 1792, 1032)])
+def test_on_chip_forms_on_clusters_of_six_ten_and_fourteen_ctas(M, N, K, cuda_device):
+    """1536, 1280 and 1792 columns: three, five and seven column ranges per row block.  Which of these shapes run on chip and
+    which as two kernels follows the measured rule of the library; here whatever it picks is checked against the oracle, and
+    the on-chip form where the rule says so needs no workspace."""
+    import paper_2608_03537_b200 as cf
+    w = wl.post_norm(M, N, K, seed=N + K, affine=True, relu=(N == 1792))
+    T = P.dev_tensors(w)
+    desc = cf.make_gemm_desc(T["A"], T["B"], torch.empty(M, N, dtype=torch.bfloat16, device=T["A"].device),
+                             cf.EPI_BIAS_RES_LAYERNORM, residual=T["residual"], fused=True)
+    on_chip = N == 1280 or (N == 1536 and K <= 1024) or (N == 1792 and K <= 2048)
+    assert cf.workspace_size(desc) == (0 if on_chip else M * (N // 256) * 8)
+    got = P.run_gpu(w, T, fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"LN {M}x{N}x{K}")
+    w = wl.complex_subgraph(M, N, K, seed=M + N)
+    got = P.run_gpu(w, P.dev_tensors(w), fused=True)
+    P.check_outputs(w, got, P.run_oracle(w), label=f"RMS {M}x{N}x{K}", rowmax_tol=3e-2)
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 1536, 2048), (520, 3072, 64), (260, 5120, 136), (4100, 2560, 72)])
 def test_row_lengths_without_a_single_kernel_form_run_in_256_column_tiles(M, N, K, cuda_device):
     """Multiples of 256 that no on-chip instantiation covers (1280, 1536, 2560, 3072, 5120, ...), at any K: the two-kernel form."""
     import paper_2608_03537_b200 as cf
