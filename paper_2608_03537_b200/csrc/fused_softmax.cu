@@ -33,6 +33,10 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
     COMFUSE_CASE(1024, 256, 256, 2, 2, 4)
     COMFUSE_CASE(2048, 256, 256, 4, 2, 4)
     COMFUSE_CASE(4096, 256, 256, 8, 2, 4)
+    case 1280: case 1536: case 1792:
+      return launch_fused_softmax_more_rows_a(maps, p, st, supported_only);  // translation units of their own
+    case 2560: case 3072: case 3584:
+      return launch_fused_softmax_more_rows_b(maps, p, st, supported_only);
     default:
       // Long K and a row length without a cluster instantiation -- above all rows wider than the largest cluster holds
       // (N > 4096): the row kernel's statistics pass followed by a second MainLoop pass takes any N.  It pays the

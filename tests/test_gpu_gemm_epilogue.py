@@ -235,6 +235,13 @@ SOFTMAX_CASES = [
     (1, 300, 512, 320, False),
     (2, 200, 2048, 272, False),
     (1, 4096, 4096, 264, True),
+    # row lengths on clusters of 10, 6, 14, 10, 12 and 14 CTAs (instead of the row kernel's two MainLoop passes)
+    (1, 300, 1280, 320, False),
+    (1, 1536, 1536, 264, True),
+    (2, 200, 1792, 520, False),
+    (1, 520, 2560, 776, False),
+    (1, 3072, 3072, 264, True),
+    (1, 260, 3584, 1032, False),
     # K >= 768: the cluster kernel's long-contraction form (three stages, sub-tiles in lock step, eight epilogue warps)
     (1, 300, 1024, 776, False),
     (2, 1024, 1024, 768, True),
@@ -295,6 +302,8 @@ def _additive_mask(M, N, seed, dead_rows=(5,)):
     (1, 256, 512, 512, 2.5),     # cluster kernel, soft-capped
     (1, 300, 1024, 840, 2.0),    # cluster kernel behind a long contraction, soft-capped
     (2, 260, 2048, 768, 0.0),
+    (1, 300, 1536, 320, 0.0),    # cluster of 6 CTAs
+    (1, 260, 3072, 520, 2.0),    # cluster of 12 CTAs, soft-capped
 ])
 def test_softmax_additive_mask_with_fully_masked_rows(batch, M, N, K, softcap, fused, cuda_device):
     """The additive-mask variant: the mask tensor is one more operand of the epilogue; -inf entries give exact zeros, a
