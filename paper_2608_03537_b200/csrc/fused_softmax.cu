@@ -33,7 +33,7 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
     COMFUSE_CASE(1024, 256, 256, 2, 2, 4)
     COMFUSE_CASE(2048, 256, 256, 4, 2, 4)
     COMFUSE_CASE(4096, 256, 256, 8, 2, 4)
-    case 1280: case 1536: case 1792:
+    case 768: case 1280: case 1536: case 1792:
       return launch_fused_softmax_more_rows_a(maps, p, st, supported_only);  // translation units of their own
     case 2560: case 3072: case 3584:
       return launch_fused_softmax_more_rows_b(maps, p, st, supported_only);

@@ -1,4 +1,4 @@
-// Cluster instantiations of the softmax kind at 1280, 1536 and 1792 columns (clusters of 10, 6 and 14 CTAs), in a translation unit of their
+// Cluster instantiations of the softmax kind at 768, 1280, 1536 and 1792 columns (clusters of 4, 10, 6 and 14 CTAs), in a translation unit of their
 // own.  Behind a contraction longer than 256 such rows would otherwise take the row kernel, which computes the scores twice:
 // measured (8192 rows) 8192 x 1536, K = 4096: 433 us there against 99 us on chip; 2560, K = 2048: 321 against 95.
 #include "fused_launch.cuh"
@@ -10,6 +10,7 @@ cudaError_t launch_fused_softmax_more_rows_a(const GemmMaps& maps, const FusedPa
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, lock, 2>(maps, p, st);
   switch (p.N) {
+    COMFUSE_CASE(768, 256, 128, 2, 4, 1)
     COMFUSE_CASE(1280, 256, 0, 5, 5, 0)
     COMFUSE_CASE(1536, 256, 256, 3, 3, 1)
     COMFUSE_CASE(1792, 256, 0, 7, 5, 0)

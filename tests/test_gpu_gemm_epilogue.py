@@ -236,6 +236,8 @@ SOFTMAX_CASES = [
     (2, 200, 2048, 272, False),
     (1, 4096, 4096, 264, True),
     # row lengths on clusters of 10, 6, 14, 10, 12 and 14 CTAs (instead of the row kernel's two MainLoop passes)
+    (1, 300, 768, 320, False),
+    (2, 768, 768, 520, True),
     (1, 300, 1280, 320, False),
     (1, 1536, 1536, 264, True),
     (2, 200, 1792, 520, False),
@@ -303,6 +305,7 @@ def _additive_mask(M, N, seed, dead_rows=(5,)):
     (1, 300, 1024, 840, 2.0),    # cluster kernel behind a long contraction, soft-capped
     (2, 260, 2048, 768, 0.0),
     (1, 300, 1536, 320, 0.0),    # cluster of 6 CTAs
+    (2, 200, 768, 264, 3.0),     # sub-tiles of 256 and 128 columns in lock step
     (1, 260, 3072, 520, 2.0),    # cluster of 12 CTAs, soft-capped
 ])
 def test_softmax_additive_mask_with_fully_masked_rows(batch, M, N, K, softcap, fused, cuda_device):
