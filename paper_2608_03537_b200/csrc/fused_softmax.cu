@@ -8,7 +8,15 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   // Short K: recomputing a score chunk is cheaper than keeping the row block on-chip across a cluster.
   // COMFUSE_SOFTMAX_CLUSTER=1 forces the cluster kernel where it has an instantiation (for comparisons).
   static const bool force_cluster = std::getenv("COMFUSE_SOFTMAX_CLUSTER") != nullptr;
-  if (softmax_rows_supported(p) && !force_cluster) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
+  // ... unless the problem is so small that the row kernel's CTA pairs do not fill the machine: up to 32 pairs of row blocks
+  // (8192 rows) of 768 columns or more run faster on clusters, which put 4 to 16 CTAs on every pair.  Measured at 8192 rows,
+  // K = 64 (row kernel / cluster kernel, us): N = 768: 22.3 / 15.2, 1024: 19.1 / 15.7, 2048 causal: 31.8 / 26.5, 4096: 59.1 / 50.7;
+  // at 16384 rows the row kernel is ahead again (N = 2048 causal: 32.5 / 41.4), and far ahead once the output outgrows L2.
+  const long long row_pairs = static_cast<long long>(p.batch) * ((p.M + 255) / 256);
+  const bool cluster_form = p.N == 768 || p.N == 1024 || p.N == 1280 || p.N == 1536 || p.N == 1792 || p.N == 2048 || p.N == 2560 ||
+                            p.N == 3072 || p.N == 3584 || p.N == 4096;
+  const bool small = row_pairs <= 32 && cluster_form;
+  if (softmax_rows_supported(p) && !force_cluster && !small) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
 #define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
   case n:                                     \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, 0, epw>(maps, p, st);
@@ -20,6 +28,8 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   const bool long_k = stages_env ? stages_env[0] == '3' : p.K >= 768;
   if (long_k) {
     switch (p.N) {
+      case 256: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 0, 1, 5, 0, 2>(maps, p, st);
+      case 512: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 1, 3, 1, 2>(maps, p, st);
       case 1024: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 2, 3, 1, 2>(maps, p, st);
       case 2048: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 4, 3, 1, 2>(maps, p, st);
       case 4096: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 8, 3, 1, 2>(maps, p, st);
