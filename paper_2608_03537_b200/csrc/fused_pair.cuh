@@ -1284,10 +1284,16 @@ COMFUSE_PROGRAM_LOOP
         const SoftcapLog2 cap_fn(p.alpha, capped ? p.softcap : 1.f);
         const float sc = capped ? 1.f : p.alpha * 1.4426950408889634f;
         const bool additive = p.mask != nullptr;  // additive mask tensor, applied behind the scale / soft-cap
-        // fragment classification under the causal mask, uniform over the warp's 32 rows so that the warp-wide TMEM
-        // loads stay convergent: 2 = all live, 1 = crosses the diagonal, 0 = all masked
+        // The last live column of a row: the diagonal under the causal mask, and never beyond the row's end -- the
+        // instantiation may be wider than the row (N = 1000 on the 1024-column form), columns from N on are masked.
+        // Fragment classification, uniform over the warp's 32 rows so that the warp-wide TMEM loads stay convergent:
+        // 2 = all live, 1 = crosses the limit of some row, 0 = all masked
         const int wrow0 = m0 + q * 32;
-        auto frag_state = [&](int col0) { return !p.causal ? 2 : (col0 + 31 <= wrow0 ? 2 : (col0 > wrow0 + 31 ? 0 : 1)); };
+        const int nlast = p.N - 1;
+        const int rlim = p.causal ? (grow < nlast ? grow : nlast) : nlast;
+        const int wlim_lo = p.causal ? (wrow0 < nlast ? wrow0 : nlast) : nlast;
+        const int wlim_hi = p.causal ? (wrow0 + 31 < nlast ? wrow0 + 31 : nlast) : nlast;
+        auto frag_state = [&](int col0) { return col0 + 31 <= wlim_lo ? 2 : (col0 > wlim_hi ? 0 : 1); };
         COMFUSE_TRACE_POINT();
         // ---------------- pass A: thread-local row max
         float mloc = -INFINITY;
@@ -1314,22 +1320,22 @@ COMFUSE_PROGRAM_LOOP
                 // a full-tensor operand of the epilogue (Sec. 5.2): t = score + mask, written back over the accumulator so
                 // that pass B finds it there
                 float2 m2[16];
-                load_mask_log2_32(p.mask + static_cast<long long>(grow) * p.N + col0, valid ? 32 : 0, m2);
+                load_mask_log2_32(p.mask + static_cast<long long>(grow) * p.N + col0, valid ? (p.N - col0 < 32 ? p.N - col0 : 32) : 0, m2);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   const float2 t01 = fma2(f2_from_bits(v[2 * j], v[2 * j + 1]), splat2(sc), m2[j]);
                   v[2 * j] = __float_as_uint(t01.x);
                   v[2 * j + 1] = __float_as_uint(t01.y);
-                  if (st == 2 || col0 + 2 * j <= grow) m0v = fmaxf(m0v, t01.x);
-                  if (st == 2 || col0 + 2 * j + 1 <= grow) m1v = fmaxf(m1v, t01.y);
+                  if (st == 2 || col0 + 2 * j <= rlim) m0v = fmaxf(m0v, t01.x);
+                  if (st == 2 || col0 + 2 * j + 1 <= rlim) m1v = fmaxf(m1v, t01.y);
                 }
                 tmem_st_32cols(tmem_of(sub) + g * 64 + half * 32, v);
               } else {
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                   const float t0 = __uint_as_float(v[j]) * sc, t1 = __uint_as_float(v[j + 1]) * sc;
-                  if (st == 2 || col0 + j <= grow) m0v = fmaxf(m0v, t0);
-                  if (st == 2 || col0 + j + 1 <= grow) m1v = fmaxf(m1v, t1);
+                  if (st == 2 || col0 + j <= rlim) m0v = fmaxf(m0v, t0);
+                  if (st == 2 || col0 + j + 1 <= rlim) m1v = fmaxf(m1v, t1);
                 }
               }
               mloc = fmaxf(mloc, fmaxf(m0v, m1v));
@@ -1366,8 +1372,8 @@ COMFUSE_PROGRAM_LOOP
                 float e0 = ex2_approx(t01.x);
                 float e1 = ex2_approx(t01.y);
                 if (st != 2) {
-                  if (col0 + j > grow) e0 = 0.f;
-                  if (col0 + j + 1 > grow) e1 = 0.f;
+                  if (col0 + j > rlim) e0 = 0.f;
+                  if (col0 + j + 1 > rlim) e1 = 0.f;
                 }
                 v[j] = __float_as_uint(e0);
                 v[j + 1] = __float_as_uint(e1);

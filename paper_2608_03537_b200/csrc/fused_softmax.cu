@@ -12,10 +12,14 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   // (8192 rows) of 768 columns or more run faster on clusters, which put 4 to 16 CTAs on every pair.  Measured at 8192 rows,
   // K = 64 (row kernel / cluster kernel, us): N = 768: 22.3 / 15.2, 1024: 19.1 / 15.7, 2048 causal: 31.8 / 26.5, 4096: 59.1 / 50.7;
   // at 16384 rows the row kernel is ahead again (N = 2048 causal: 32.5 / 41.4), and far ahead once the output outgrows L2.
+  // A row length between two instantiations runs on the next wider one: the columns from N on read as zeros and are
+  // masked like the ones above the diagonal of a causal mask.
+  static const int kForms[] = {256, 512, 768, 1024, 1280, 1536, 1792, 2048, 2560, 3072, 3584, 4096};
+  int form = 0;
+  for (int f : kForms)
+    if (form == 0 && p.N <= f) form = f;
   const long long row_pairs = static_cast<long long>(p.batch) * ((p.M + 255) / 256);
-  const bool cluster_form = p.N == 768 || p.N == 1024 || p.N == 1280 || p.N == 1536 || p.N == 1792 || p.N == 2048 || p.N == 2560 ||
-                            p.N == 3072 || p.N == 3584 || p.N == 4096;
-  const bool small = row_pairs <= 32 && cluster_form;
+  const bool small = row_pairs <= 32 && form >= 768 && p.N > form / 2;
   if (softmax_rows_supported(p) && !force_cluster && !small) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
 #define COMFUSE_CASE(n, b0, b1, cn, nst, epw) \
   case n:                                     \
@@ -27,7 +31,7 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
   static const char* stages_env = std::getenv("COMFUSE_SOFTMAX_STAGES");
   const bool long_k = stages_env ? stages_env[0] == '3' : p.K >= 768;
   if (long_k) {
-    switch (p.N) {
+    switch (form) {
       case 256: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 0, 1, 5, 0, 2>(maps, p, st);
       case 512: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 1, 3, 1, 2>(maps, p, st);
       case 1024: return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, 256, 256, 2, 3, 1, 2>(maps, p, st);
@@ -37,20 +41,19 @@ cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cud
     }
   }
   // Else the softmax passes are latency-bound on few warps and need few registers: four epilogue warps per lane quarter.
-  switch (p.N) {
+  switch (form) {
     COMFUSE_CASE(256, 256, 0, 1, 3, 4)
     COMFUSE_CASE(512, 256, 256, 1, 2, 4)
     COMFUSE_CASE(1024, 256, 256, 2, 2, 4)
     COMFUSE_CASE(2048, 256, 256, 4, 2, 4)
     COMFUSE_CASE(4096, 256, 256, 8, 2, 4)
     case 768: case 1280: case 1536: case 1792:
-      return launch_fused_softmax_more_rows_a(maps, p, st, supported_only);  // translation units of their own
+      return launch_fused_softmax_more_rows_a(form, maps, p, st, supported_only);  // translation units of their own
     case 2560: case 3072: case 3584:
-      return launch_fused_softmax_more_rows_b(maps, p, st, supported_only);
+      return launch_fused_softmax_more_rows_b(form, maps, p, st, supported_only);
     default:
-      // Long K and a row length without a cluster instantiation -- above all rows wider than the largest cluster holds
-      // (N > 4096): the row kernel's statistics pass followed by a second MainLoop pass takes any N.  It pays the
-      // GEMM twice, which is still less than writing and re-reading the scores.
+      // Long K and rows wider than the largest cluster holds (N > 4096): the row kernel's statistics pass followed by a
+      // second MainLoop pass takes any N.  It pays the GEMM twice, which is still less than writing and re-reading the scores.
       if (p.N >= 64) return supported_only ? cudaSuccess : launch_softmax_rows(maps, p, st);
       return cudaErrorInvalidValue;
   }

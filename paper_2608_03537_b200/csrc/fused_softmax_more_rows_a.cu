@@ -5,11 +5,11 @@
 
 namespace comfuse {
 
-cudaError_t launch_fused_softmax_more_rows_a(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
+cudaError_t launch_fused_softmax_more_rows_a(int form, const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
 #define COMFUSE_CASE(n, b0, b1, cn, nst, lock) \
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, lock, 2>(maps, p, st);
-  switch (p.N) {
+  switch (form) {  // the instantiation's row length: p.N, or the next wider one
     COMFUSE_CASE(768, 256, 128, 2, 4, 1)
     COMFUSE_CASE(1280, 256, 0, 5, 5, 0)
     COMFUSE_CASE(1536, 256, 256, 3, 3, 1)

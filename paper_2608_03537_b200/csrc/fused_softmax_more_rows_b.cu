@@ -5,11 +5,11 @@
 
 namespace comfuse {
 
-cudaError_t launch_fused_softmax_more_rows_b(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
+cudaError_t launch_fused_softmax_more_rows_b(int form, const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only) {
 #define COMFUSE_CASE(n, b0, b1, cn, nst, lock) \
   case n:                                      \
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_SOFTMAX, b0, b1, cn, nst, lock, 2>(maps, p, st);
-  switch (p.N) {
+  switch (form) {  // the instantiation's row length: p.N, or the next wider one
     COMFUSE_CASE(2560, 256, 256, 5, 3, 1)
     COMFUSE_CASE(3072, 256, 256, 6, 3, 1)
     COMFUSE_CASE(3584, 256, 256, 7, 3, 1)

@@ -72,8 +72,8 @@ inline int wide_row_blocks(int epi, int N, int K) {
   return w ? (N + w - 1) / w : 0;
 }
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
-cudaError_t launch_fused_softmax_more_rows_a(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
-cudaError_t launch_fused_softmax_more_rows_b(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+cudaError_t launch_fused_softmax_more_rows_a(int form, const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
+cudaError_t launch_fused_softmax_more_rows_b(int form, const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
 // Short-K row softmax (pairs of CTAs, score chunks computed twice instead of exchanged across a cluster).
 bool softmax_rows_supported(const FusedParams& p);
 cudaError_t launch_softmax_rows(const GemmMaps& maps, FusedParams p, cudaStream_t st);

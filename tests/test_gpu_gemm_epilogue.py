@@ -244,6 +244,13 @@ SOFTMAX_CASES = [
     (1, 520, 2560, 776, False),
     (1, 3072, 3072, 264, True),
     (1, 260, 3584, 1032, False),
+    # row lengths between two instantiations run on the next wider one, the columns from N on masked
+    (1, 300, 1000, 320, False),
+    (2, 1000, 1000, 264, True),
+    (1, 200, 72, 520, False),
+    (1, 260, 2056, 776, False),
+    (1, 3000, 3000, 328, True),
+    (3, 130, 4088, 1032, False),
     # K >= 768: the cluster kernel's long-contraction form (three stages, sub-tiles in lock step, eight epilogue warps)
     (1, 300, 1024, 776, False),
     (2, 1024, 1024, 768, True),
@@ -306,6 +313,8 @@ def _additive_mask(M, N, seed, dead_rows=(5,)):
     (2, 260, 2048, 768, 0.0),
     (1, 300, 1536, 320, 0.0),    # cluster of 6 CTAs
     (2, 200, 768, 264, 3.0),     # sub-tiles of 256 and 128 columns in lock step
+    (1, 300, 1000, 328, 0.0),    # the 1024-column form with 24 columns masked, the mask tensor's rows 1000 long
+    (2, 200, 1160, 64, 2.5),     # a small problem behind a short contraction: the cluster kernel, 1280-column form
     (1, 260, 3072, 520, 2.0),    # cluster of 12 CTAs, soft-capped
 ])
 def test_softmax_additive_mask_with_fully_masked_rows(batch, M, N, K, softcap, fused, cuda_device):

@@ -41,8 +41,10 @@ def _case(seed):
         softcap = float(np.round(g.uniform(1.0, 8.0), 2)) if g.random() < 0.3 else 0.0
         if K <= 256:
             N = int(g.integers(8, 160)) * 8               # any row length for the short-K kernel: 64 .. 1272
+        elif g.random() < 0.5:
+            N = [256, 512, 768, 1024, 1536, 2048][int(g.integers(6))]   # row lengths with a cluster instantiation of their own
         else:
-            N = [256, 512, 1024, 2048][int(g.integers(4))]   # the cluster kernel's instantiations
+            N = int(g.integers(8, 320)) * 8               # any other: the next wider instantiation, the columns from N on masked
         if causal:
             M = N
         w = wl.scaled_masked_softmax(batch, M, N, K, seed=seed, causal=causal, softcap=softcap)
