@@ -156,4 +156,7 @@ struct FusedParams {
   int trace_flags;            // tracing builds: bit 0 = skip the output stores, bit 1 = skip the UMMAs
 };
 
+// the kernels take four 128-byte tensor maps and this block by value: 4 KB of parameter space
+static_assert(sizeof(FusedParams) + 4 * 128 <= 4096, "kernel parameter space");
+
 }  // namespace comfuse
