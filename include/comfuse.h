@@ -122,7 +122,9 @@ typedef struct {
  *   - Rows of 2048 .. 4096 columns (a multiple of 256) behind a long contraction (K >= 1024), block = 256: measured faster
  *     than keeping the row on chip, because the 8- and 16-CTA clusters that hold such rows leave SMs idle and cannot
  *     overlap a tile's epilogue with the next MainLoop.  Here the workspace is optional where the row length has an
- *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.
+ *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.  The same holds for rows of 512 ..
+ *     1024 columns when there are so few rows that the on-chip clusters would leave most of the machine idle (fewer than about
+ *     6000 rows; K >= 1536 for the LayerNorm kind, K >= 1024 for the RMSNorm kind).
  *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096, and behind
  *     contractions short enough for it to pay 1280, 1536, 1792: ask this function) that are not a
  *     multiple of 4096 -- 1000, 1280, 1536, 1600, 3072, 5120, ... any multiple of 8 up to 65536 -- at any K, block = 256,

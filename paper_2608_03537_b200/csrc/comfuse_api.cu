@@ -75,7 +75,7 @@ bool programmatic_launch_enabled() {
   return on;
 }
 
-int split_row_block(int epi, int N, int K) {
+int split_row_block(int epi, int N, int K, long long row_pairs) {
   // COMFUSE_SPLIT_BLOCK=<width> forces the two-kernel form with that block width where N is a multiple of it (0 = never)
   static const int forced = [] {
     const char* e = std::getenv("COMFUSE_SPLIT_BLOCK");
@@ -87,6 +87,17 @@ int split_row_block(int epi, int N, int K) {
   // The clusters of 16 and 8 CTAs that hold rows of 4096 and 2048 columns fill 112 and 120 of the 148 SMs and cannot overlap
   // a tile's epilogue with the next MainLoop; the 256-column tiles of the two-kernel form can, on every SM.
   if (N >= 2048 && N % 256 == 0 && K >= 1024) return 256;
+  // Few rows behind a long contraction: the on-chip forms put one cluster on every pair of row blocks, which leaves most of
+  // the machine idle when there are few pairs; 256-column tiles give N / 256 times as many work items.  Measured at 2048
+  // rows (on chip / two kernels, us): N = 1024: K = 1024 20.3 / 16.7, K = 4096 48.0 / 32.2; at 8192 rows the clusters fill
+  // the machine and the on-chip form is ahead again (K = 4096: 55 / 69).
+  // (N = 512, 512 .. 4096 rows: K = 1536 LayerNorm 24 / 20, K = 2048 28 / 21, K = 4096 46 / 30; the RMSNorm kind gains from
+  // K = 1024 on: 21 / 15; LayerNorm at K = 1024 is level.)
+  if (std::getenv("COMFUSE_NO_SMALL_SPLIT") == nullptr && K >= (epi == EPI_LN ? 1536 : 1024) && N % 256 == 0 && N >= 512 && N <= 1024) {
+    const long long cluster = N >= 768 ? 4 : 2;
+    const long long two_kernel = row_pairs * (N / 256) * 2 < 148 ? row_pairs * (N / 256) * 2 : 148;
+    if (row_pairs * cluster * 10 < two_kernel * 6) return 256;
+  }
   // A row length that no single-kernel instantiation covers (1280, 1536, 2560, 3072, 5120, ...): the two-kernel form takes
   // any multiple of 256, at any K -- one fp16 trip of the row, which is still cheaper than the unfused path's bf16 Z plus
   // a row kernel.
@@ -212,7 +223,7 @@ comfuse_status_t fused_supported(const comfuse_gemm_desc_t* d, bool on_chip_only
   p.M = d->M;
   p.N = d->N;
   p.K = d->K;
-  p.wide_block = on_chip_only ? 0 : wide_row_block(kind_to_epi(d->kind), d->N, d->K);
+  p.wide_block = on_chip_only ? 0 : wide_row_block(kind_to_epi(d->kind), d->N, d->K, static_cast<long long>(d->batch) * ((d->M + 255) / 256));
   p.wide = p.wide_block > 0;
   GemmMaps dummy;
   std::memset(&dummy, 0, sizeof(dummy));
@@ -362,7 +373,8 @@ comfuse_status_t comfuse_workspace_size(const comfuse_gemm_desc_t* desc, size_t*
     s = fused_supported(desc);
     if (s != COMFUSE_OK) return s;
     // rows wider than one cluster: one partial statistic (8 bytes) per row and 4096-column block
-    *bytes = static_cast<size_t>(wide_row_blocks(kind_to_epi(desc->kind), desc->N, desc->K)) * desc->batch * desc->M * sizeof(float2);
+    *bytes = static_cast<size_t>(wide_row_blocks(kind_to_epi(desc->kind), desc->N, desc->K, static_cast<long long>(desc->batch) * ((desc->M + 255) / 256))) *
+             desc->batch * desc->M * sizeof(float2);
   } else {
     if (desc->N > 8192) return COMFUSE_ERR_UNSUPPORTED;
     *bytes = static_cast<size_t>(desc->batch) * desc->M * desc->N * 2;  // dense bf16 Z
@@ -451,9 +463,10 @@ comfuse_status_t comfuse_gemm_epilogue(const comfuse_gemm_desc_t* desc, const vo
     p.ldy = desc->ldy; p.batch_stride_y = bsy;
     p.row_max = a.row_max; p.row_argmax = a.row_argmax;
     p.mask = desc->mask == COMFUSE_MASK_ADDITIVE ? static_cast<const uint16_t*>(a.mask) : nullptr;
-    const int wide_blocks = need > 0 ? wide_row_blocks(epi, desc->N, desc->K) : 0;
+    const long long row_pairs = static_cast<long long>(desc->batch) * ((desc->M + 255) / 256);
+    const int wide_blocks = need > 0 ? wide_row_blocks(epi, desc->N, desc->K, row_pairs) : 0;
     if (wide_blocks) {
-      p.wide_block = wide_row_block(epi, desc->N, desc->K);  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace
+      p.wide_block = wide_row_block(epi, desc->N, desc->K, row_pairs);  // first kernel: per-block stage 1, un-normalised x to Y, partial statistics to the workspace
       p.wide = 1;
       p.nblocks = wide_blocks;
       p.wide_partials = static_cast<float2*>(workspace);

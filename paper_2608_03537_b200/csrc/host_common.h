@@ -59,16 +59,16 @@ constexpr int kWideRowBlock = 4096;
 // CTAs occupy 112 of the 148 SMs and leave tensor memory no room to overlap a tile's epilogue with the next MainLoop, so
 // for long K the detour through one fp16 copy of the row can be the faster path.  `split_row_block` = the block width
 // chosen for (epi, N, K), 0 = keep the row on chip.
-int split_row_block(int epi, int N, int K);
+int split_row_block(int epi, int N, int K, long long row_pairs);  // row_pairs = batch * ceil(M / 256): how many tiles a row length gives
 // column block width of the two-kernel form (0 = one kernel) and the number of blocks per row
-inline int wide_row_block(int epi, int N, int K) {
+inline int wide_row_block(int epi, int N, int K, long long row_pairs) {
   if (epi != EPI_LN && epi != EPI_RMS_MAX) return 0;
-  const int narrow = N <= 16 * kWideRowBlock ? split_row_block(epi, N, K) : 0;
+  const int narrow = N <= 16 * kWideRowBlock ? split_row_block(epi, N, K, row_pairs) : 0;
   if (N > kWideRowBlock && narrow == 0) return (N % kWideRowBlock == 0 && N <= 16 * kWideRowBlock) ? kWideRowBlock : 0;
   return narrow;
 }
-inline int wide_row_blocks(int epi, int N, int K) {
-  const int w = wide_row_block(epi, N, K);
+inline int wide_row_blocks(int epi, int N, int K, long long row_pairs) {
+  const int w = wide_row_block(epi, N, K, row_pairs);
   return w ? (N + w - 1) / w : 0;
 }
 cudaError_t launch_fused_softmax(const GemmMaps& maps, const FusedParams& p, cudaStream_t st, bool supported_only);
