@@ -51,6 +51,23 @@ for i, w in enumerate(cases):
             P.check_outputs(w, got, P.run_oracle(w), label=f"{w.name} fused={fused}", rowmax_tol=5e-3 if fused else 3e-2,
                             softmax_tol=P.TOL_SOFTMAX_MAX if fused else P.TOL_SOFTMAX_UNFUSED,
                             norm_tol=P.TOL_NORM_MAX if fused else 4e-2)
+# an epilogue program on the interpreter and as a generated kernel (compiled with the predicates as well)
+import numpy as np
+from oracle import fusion_spec_oracle as spo
+prog = wl.spec_range_normalise()
+M, N, K = 300, 1024, 72
+A = wl.normal_bf16(21, 0, (M, K)); B = wl.normal_bf16(21, 1, (K, N), std=K ** -0.5); bias = wl.normal_bf16(21, 2, (N,), std=0.1)
+f = wl.bf16_to_f64
+Yref, Rref = spo.gemm_spec(f(A), f(B), prog.nodes, prog.terminal, [f(bias)], prog.row_outputs)
+spec = cf.make_spec(prog.nodes, prog.terminal, 1, prog.row_outputs)
+modes = [2] + ([cf.GENERATED] if cf.program_compiler_status()[0] == cf.OK else [])
+for fused in modes:
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    ro = [torch.zeros(M, dtype=torch.int32 if prog.nodes[r][0] == "argmax" else torch.float32, device="cuda:0") for r in prog.row_outputs]
+    cf.gemm_spec(P.to_dev(A), P.to_dev(B), Y, spec, params=[P.to_dev(bias)], row_out=ro, fused=fused)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK, ("program", fused)
+    assert float(np.abs(P.to_f64(Y) - Yref).max()) <= 4e-3, ("program", fused)
 print("checked build ok")
 """
 
