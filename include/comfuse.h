@@ -125,8 +125,9 @@ typedef struct {
  *     on-chip instantiation (2048, 4096): a call that brings none keeps the row on chip.  The same holds for rows of 512 ..
  *     1024 columns when there are so few rows that the on-chip clusters would leave most of the machine idle (fewer than about
  *     6000 rows; K >= 1536 for the LayerNorm kind, K >= 1024 for the RMSNorm kind).
- *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096, and behind
- *     contractions short enough for it to pay 1280, 1536, 1792: ask this function) that are not a
+ *   - Row lengths without an on-chip instantiation (the on-chip ones: 256, 512, 768, 1024, 2048, 4096 and row lengths up to
+ *     a quarter shorter than one of these, which run on it with the surplus columns masked; behind contractions short
+ *     enough for it to pay also 1280, 1536, 1792: ask this function) that are not a
  *     multiple of 4096 -- 1000, 1280, 1536, 1600, 3072, 5120, ... any multiple of 8 up to 65536 -- at any K, block = 256,
  *     (N + 255) / 256 blocks: the last tile may be a partial one.  The workspace is required.
  *   With these every row length that is a multiple of 8 (up to 65536 columns) has a fused form for all three kinds.

@@ -87,6 +87,8 @@ int split_row_block(int epi, int N, int K, long long row_pairs) {
   // The clusters of 16 and 8 CTAs that hold rows of 4096 and 2048 columns fill 112 and 120 of the 148 SMs and cannot overlap
   // a tile's epilogue with the next MainLoop; the 256-column tiles of the two-kernel form can, on every SM.
   if (N >= 2048 && N % 256 == 0 && K >= 1024) return 256;
+  const int form = norm_on_chip_form(N);
+  if (form >= 2048 && form != N && K >= 1024) return 256;  // the same behind a row a little shorter than 2048 / 4096
   // Few rows behind a long contraction: the on-chip forms put one cluster on every pair of row blocks, which leaves most of
   // the machine idle when there are few pairs; 256-column tiles give N / 256 times as many work items.  Measured at 2048
   // rows (on chip / two kernels, us): N = 1024: K = 1024 20.3 / 16.7, K = 4096 48.0 / 32.2; at 8192 rows the clusters fill
@@ -107,7 +109,7 @@ int split_row_block(int epi, int N, int K, long long row_pairs) {
   // N = 1536: 27 / 28, 42 / 39, 61 / 55, 102 / 89; N = 1792: 36 / 32, 45 / 46, 70 / 69, 120 / 112.
   const bool ln = epi == EPI_LN;
   const bool more_rows = N == 1280 || (N == 1536 && K <= (ln ? 1024 : 256)) || (N == 1792 && ln && K <= 2048);
-  const bool on_chip = N == 256 || N == 512 || N == 768 || N == 1024 || N == 2048 || N == 4096 || more_rows;
+  const bool on_chip = form != 0 || more_rows;
   // (multiples of 4096: 4096-column blocks.)  N need not be a multiple of 256: the last tile is a partial one -- operands
   // outside the matrix read as zeros, stores are clipped, and the second kernel corrects that tile's statistic for them.
   return (!on_chip && N % kWideRowBlock != 0 && N <= 16 * kWideRowBlock) ? 256 : 0;

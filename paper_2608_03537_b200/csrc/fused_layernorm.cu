@@ -9,7 +9,8 @@ cudaError_t launch_fused_layernorm(const GemmMaps& maps, const FusedParams& p, c
     return supported_only ? cudaSuccess : launch_pair_instance<EPI_LN, b0, b1, cn, nst, lock>(maps, p, st);
   // Two sub-tiles advance in lock step (lock = 1): the A tile is fetched once per K block for both.
   // Two-kernel form (p.wide): every cluster covers one p.wide_block-column block of the row, p.nblocks blocks per row.
-  switch (p.wide ? p.wide_block : p.N) {
+  const int form = norm_on_chip_form(p.N);  // a row a little shorter than an instantiation runs on it, the surplus masked
+  switch (p.wide ? p.wide_block : (form ? form : p.N)) {
     COMFUSE_CASE(256, 256, 0, 1, 5, 0)
     COMFUSE_CASE(512, 256, 256, 1, 3, 1)
     COMFUSE_CASE(768, 256, 128, 2, 4, 1)

@@ -229,7 +229,10 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto group_col = [&](int ncta0, int lg) { return Cfg::INTERLEAVE ? (lg * CN + static_cast<int>(crank)) * 64 : ncta0 + lg * 64; };
   // A sub-tile is not computed when it lies past N, or when the causal mask removes it for BOTH row blocks of the
   // pair (its first group has the smallest columns).  Every role evaluates the same predicate.
-  auto unit_live = [&](int mpair0, int n0) { return n0 < p.N && !(EPI == EPI_SOFTMAX && p.causal && n0 > mpair0 + 255); };
+  // (the normalising kinds read every accumulator column of the instantiation: where it is wider than the row, the columns
+  // from N on must BE zeros -- computed from operands that read as zeros -- not whatever the slot held before)
+  constexpr bool kAllUnitsLive = EPI == EPI_LN || kIsRms || EPI == EPI_PROGRAM;
+  auto unit_live = [&](int mpair0, int n0) { return (kAllUnitsLive || n0 < p.N) && !(EPI == EPI_SOFTMAX && p.causal && n0 > mpair0 + 255); };
 
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------ TMA producer
@@ -720,9 +723,21 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         COMFUSE_TRACE_POINT();
         // wide rows: the statistic covers this column block only; store x as it is (gamma = 1, beta = 0 were loaded) and
         // leave the normalisation to the second kernel
-        const float mu = (EPI == EPI_LN && !p.wide) ? tot.x : 0.f;
-        const float sq = EPI == EPI_LN ? tot.y : tot.x;
-        const float rstd = p.wide ? 1.f : rsqrtf(sq * (1.f / static_cast<float>(CN * BN)) + p.eps);
+        float mu = (EPI == EPI_LN && !p.wide) ? tot.x : 0.f;
+        float sq = EPI == EPI_LN ? tot.y : tot.x;
+        // The instantiation may be wider than the row (N = 1000 on the 1024-column form): the columns from N on hold exact
+        // zeros (operands outside the matrix read as zeros, the row vectors are masked), which add nothing to a sum or to a
+        // sum of squares.  The statistic of the N valid columns follows from the one over all W: S = W mean', Sxx = M2' +
+        // W mean'^2, mean = S / N, M2 = Sxx - N mean^2.
+        constexpr float kW = static_cast<float>(CN * BN);
+        const bool ragged = !p.wide && p.N != CN * BN;
+        const float nf = ragged ? static_cast<float>(p.N) : kW;
+        if (EPI == EPI_LN && ragged) {
+          const float s_all = kW * mu, sxx = sq + kW * mu * mu;
+          mu = s_all / nf;
+          sq = fmaxf(sxx - nf * mu * mu, 0.f);
+        }
+        const float rstd = p.wide ? 1.f : rsqrtf(sq / nf + p.eps);
         if (p.wide) {
           if (crank == 0 && h == 0 && valid) {
             const int nb = (ncta0 / (CN * BN));
@@ -765,10 +780,12 @@ fused_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const float2 y23 = mul2(mul2(f2_from_bits(v[4 * j + 2], v[4 * j + 3]), splat2(rstd)), make_float2(gg.z, gg.w));
                   y0 = y01.x; y1 = y01.y; y2 = y23.x; y3 = y23.y;
                   const int c = ncta0 + lc + 4 * j;
-                  if (y0 > best) { best = y0; best_col = c; }
-                  if (y1 > best) { best = y1; best_col = c + 1; }
-                  if (y2 > best) { best = y2; best_col = c + 2; }
-                  if (y3 > best) { best = y3; best_col = c + 3; }
+                  if (c + 3 < p.N) {  // (four columns at a time: N is a multiple of 8, so a group of four is inside or outside)
+                    if (y0 > best) { best = y0; best_col = c; }
+                    if (y1 > best) { best = y1; best_col = c + 1; }
+                    if (y2 > best) { best = y2; best_col = c + 2; }
+                    if (y3 > best) { best = y3; best_col = c + 3; }
+                  }
                 }
                 v[4 * j] = __float_as_uint(y0); v[4 * j + 1] = __float_as_uint(y1);
                 v[4 * j + 2] = __float_as_uint(y2); v[4 * j + 3] = __float_as_uint(y3);

@@ -59,6 +59,15 @@ constexpr int kWideRowBlock = 4096;
 // CTAs occupy 112 of the 148 SMs and leave tensor memory no room to overlap a tile's epilogue with the next MainLoop, so
 // for long K the detour through one fp16 copy of the row can be the faster path.  `split_row_block` = the block width
 // chosen for (epi, N, K), 0 = keep the row on chip.
+// The on-chip form a LayerNorm / RMSNorm row of N columns runs on: N itself where it has one, else the next wider one when
+// at most a quarter of it would be masked columns (the columns from N on then hold exact zeros, and the kernel takes its
+// statistic over N), else 0 (two kernels).
+inline int norm_on_chip_form(int N) {
+  if (N == 1280 || N == 1536 || N == 1792) return 0;  // forms of their own, with rules of their own (split_row_block)
+  for (int f : {256, 512, 768, 1024, 2048, 4096})
+    if (N <= f) return (N == f || 4 * N > 3 * f) ? f : 0;
+  return 0;
+}
 int split_row_block(int epi, int N, int K, long long row_pairs);  // row_pairs = batch * ceil(M / 256): how many tiles a row length gives
 // column block width of the two-kernel form (0 = one kernel) and the number of blocks per row
 inline int wide_row_block(int epi, int N, int K, long long row_pairs) {

@@ -49,7 +49,8 @@ def test_workspace_size_rules():
     assert _ws(_desc(fused=0)) == (cf.OK, 256 * 768 * 2)                   # unfused: dense bf16 Z
     assert _ws(_desc(fused=0, batch=3, batch_stride_a=256 * 512, batch_stride_b=512 * 768, batch_stride_y=256 * 768,
                      batch_stride_r=256 * 768)) == (cf.OK, 3 * 256 * 768 * 2)
-    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776)) == (cf.OK, 256 * 4 * 8)        # no on-chip instantiation for N = 776: two kernels,
+    assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776)) == (cf.OK, 0)                  # N = 776 runs on the 1024-column form, 248 columns masked
+    assert _ws(_desc(N=520, ldb=520, ldr=520, ldy=520)) == (cf.OK, 256 * 3 * 8)        # too short for the 768-column form: two kernels,
                                                                                       # 256-column tiles, the last one partial
     assert _ws(_desc(N=70000, ldb=70000, ldr=70000, ldy=70000))[0] == cf.ERR_UNSUPPORTED   # beyond 65536 columns
     assert _ws(_desc(N=776, ldb=776, ldr=776, ldy=776, fused=0))[0] == cf.OK          # ... but the unfused path takes it
