@@ -167,7 +167,8 @@ comfuse_status_t comfuse_gemm_epilogue_static_scratch(const comfuse_gemm_desc_t*
 /* Back-to-back GEMM (Sec. 4, Eq. 2) with F = GELU_tanh(. + b1) and the tail
  *   O = LayerNorm(S.W2 + b2 + X) * gamma + beta,   S = F(X.W1),
  * X [M, K], W1 [K, N1], W2 [N1, N2], all dense row-major bf16, N2 == K.  In the fused path S (and P) never
- * leave the chip: S is rounded to bf16 as the second GEMM's tensor-core operand. */
+ * leave the chip: S is rounded to bf16 as the second GEMM's tensor-core operand.  Fused: K = N2 = 128, N1 a multiple of
+ * 128 up to 4096 (the hidden layer streams through in chunks of 128 columns); other shapes: fused = 0. */
 typedef enum {
   COMFUSE_B2B_MLP_GELU_LAYERNORM = 0, /* as above                                                                   */
   /* Attention form (Sec. 4, Eq. 2 with a row reduction as F; the Target-Attention workload of Sec. 6.2):

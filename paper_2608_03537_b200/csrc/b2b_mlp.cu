@@ -1,5 +1,6 @@
 // Fused back-to-back GEMM, MLP form (Sec. 4):  P = X W1,  S = GELU_tanh(P + b1),  O' = S W2 + b2 + X,  O = LayerNorm(O'),
-// K = N2 = 128, N1 = 128 .. 512.  Neither P nor S is written to global memory.
+// K = N2 = 128, N1 = 128 .. 4096 (the chunks of N1 stream through; only the bias b1 is held whole).  Neither P nor S is
+// written to global memory.
 //
 // Dataflow (Sec. 4.1, adapted): N1 is cut into 128-column chunks; one CTA pair walks all chunks of its 256 rows and
 // accumulates O in tensor memory (deterministic, no cross-CTA partial sums).  The chunks of all the pair's tiles form ONE
@@ -43,8 +44,9 @@ struct MlpSmem {
   static constexpr int OFF_W = OFF_X + 4 * kBoxBytes;           // ring
   static constexpr int OFF_S = OFF_W + kWSlots * kBoxBytes;     // [2 buffers][2 K blocks]
   static constexpr int OFF_I = OFF_S + 4 * kBoxBytes;           // this CTA's 64 columns of 2 I (128 x 128), laid out like a W2 chunk
-  static constexpr int OFF_B1 = OFF_I + kBoxBytes;              // fp32 [512]
-  static constexpr int OFF_VEC = OFF_B1 + 512 * 4;              // 2 b2, gamma, beta fp32 [128] each
+  static constexpr int kMaxN1 = 4096;
+  static constexpr int OFF_B1 = OFF_I + kBoxBytes;              // fp32 [kMaxN1]
+  static constexpr int OFF_VEC = OFF_B1 + kMaxN1 * 4;           // 2 b2, gamma, beta fp32 [128] each
   static constexpr int OFF_BAR = OFF_VEC + 3 * 128 * 4;
   // xfull[2] xempty[2] wfull[4] (4 unused) pfull[2] pfree[2] sfull[2] sempty[2] ofull[2] oempty[2] drain[2] eye
   static constexpr int NUM_BARS = 4 + 2 * kWSlots + 12 + 3;
@@ -608,7 +610,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
 }  // namespace
 
-bool b2b_mlp_supported(int K, int N1, int N2) { return K == 128 && N2 == 128 && N1 >= 128 && N1 <= 512 && N1 % 128 == 0; }
+bool b2b_mlp_supported(int K, int N1, int N2) { return K == 128 && N2 == 128 && N1 >= 128 && N1 <= MlpSmem::kMaxN1 && N1 % 128 == 0; }
 
 cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
   const DeviceInfo* dev = current_device_info();

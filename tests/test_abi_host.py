@@ -139,7 +139,7 @@ def test_b2b_validation():
     assert n.value == (1024 * 512 + 1024 * 128) * 2
     for bad, code in [(cf.make_b2b_desc(1024, 128, 512, 256), cf.ERR_INVALID_ARG),      # residual needs N2 == K
                       (cf.make_b2b_desc(1024, 256, 512, 256), cf.ERR_UNSUPPORTED),      # fused kernel: K = N2 = 128
-                      (cf.make_b2b_desc(1024, 128, 1024, 128), cf.ERR_UNSUPPORTED),     # N1 <= 512
+                      (cf.make_b2b_desc(1024, 128, 4224, 128), cf.ERR_UNSUPPORTED),     # N1 <= 4096
                       (cf.make_b2b_desc(1024, 128, 516, 128), cf.ERR_ALIGNMENT),
                       (cf.make_b2b_desc(0, 128, 512, 128), cf.ERR_INVALID_ARG)]:
         assert L.comfuse_b2b_workspace_size(ctypes.byref(bad), ctypes.byref(n)) == code

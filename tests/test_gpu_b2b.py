@@ -17,6 +17,9 @@ CASES = [
     (1000, 256, True),     # two chunks
     (130, 128, False),     # a single chunk: ML1 -> Epi1 -> ML2 with no overlap partner
     (2048, 384, True),     # three chunks, several tiles per cluster on small grids
+    (300, 640, True),      # five chunks: an odd count beyond four
+    (520, 2048, False),    # sixteen chunks per tile
+    (260, 4096, True),     # the widest hidden layer the bias buffer holds
 ]
 
 
@@ -60,11 +63,11 @@ def test_b2b_bitwise_repeatable(cuda_device):
 
 
 def test_b2b_unsupported_shapes_are_refused_for_the_fused_path(cuda_device):
-    d = cf.make_b2b_desc(256, 128, 640, 128, fused=True)      # N1 > 512
+    d = cf.make_b2b_desc(256, 128, 4224, 128, fused=True)      # N1 > 4096
     with pytest.raises(cf.ComfuseError) as e:
         cf.b2b_workspace_size(d)
     assert e.value.status == cf.ERR_UNSUPPORTED
-    assert cf.b2b_workspace_size(cf.make_b2b_desc(256, 128, 640, 128, fused=False)) == 256 * 640 * 2 + 256 * 128 * 2
+    assert cf.b2b_workspace_size(cf.make_b2b_desc(256, 128, 4224, 128, fused=False)) == 256 * 4224 * 2 + 256 * 128 * 2
 
 
 # --------------------------------------------------------------------------------------------- attention form (F = softmax)
