@@ -175,9 +175,11 @@ typedef enum {
    *   O = softmax(alpha * X.W1) . W2   per batch,  softmax over the N1 source positions,
    * X [batch, M, K] queries, W1 [batch, K, N1] keys (already transposed) -- or, with COMFUSE_B2B_FLAG_KEYS_ROW_MAJOR,
    * W1 [batch, N1, K], one key per row as an attention layer produces them --, W2 [batch, N1, N2] values, O [batch, M, N2],
-   * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128 and N1 = 256 (a whole score row fits the
-   * accumulators of one CTA pair) or N1 = 512 (two sub-tiles of 256 source positions, each exponentiated against its own
-   * row maximum, combined when O is normalised); the probabilities are rounded to bf16 as the second GEMM's operand. */
+   * all dense.  b1, b2, gamma, beta must be NULL, alpha > 0.  Fused: K = N2 = 128 and N1 <= 512, a multiple of 8: up to
+   * 256 source positions a whole score row fits the accumulators of one CTA pair, above that it is two sub-tiles of 256
+   * source positions, each exponentiated against its own row maximum, combined when O is normalised; positions from N1 up
+   * to the end of the last sub-tile are loaded as zeros and take no part in the softmax.  The probabilities are rounded
+   * to bf16 as the second GEMM's operand. */
   COMFUSE_B2B_SOFTMAX_ATTENTION = 1,
   /* Two-layer ReLU MLP (Sec. 4, Eq. 2 with F = ReLU(. + b1); the DLRM workload of Sec. 6.2, 1024 -> 512 -> 128):
    *   O = ReLU(ReLU(X.W1 + b1).W2 + b2),

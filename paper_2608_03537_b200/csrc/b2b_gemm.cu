@@ -45,8 +45,9 @@ static_assert(B2bSmem::BYTES <= 232448, "shared memory budget");
 
 // NHALF: sub-tiles of 256 source positions per score row, 1 or 2.  KM: the keys (W1) are stored [batch, N1, K], one key per
 // row, and feed the score UMMAs as a K-major operand (two 64 x 64 boxes per slot: contraction elements 0..63 and 64..127 of
-// this CTA's 64 keys); else [batch, K, N1], an MN-major operand (one 128 x 64 box per slot).
-template <int NHALF, bool KM>
+// this CTA's 64 keys); else [batch, K, N1], an MN-major operand (one 128 x 64 box per slot).  RAGGED: N1 is not NHALF * 256;
+// scores of the source positions from N1 on (zeros: their keys were loaded out of bounds) are set to -inf before the softmax.
+template <int NHALF, bool KM, bool RAGGED>
 __global__ void __launch_bounds__(kB2bThreads, 1)
 b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                 const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmO, const B2bParams p) {
@@ -351,6 +352,23 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         tcgen05_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster_noflush(map_to_cta(bar_pfree, leader));
+        {
+          // A source length that is not a multiple of 256: the keys from N1 on read as zeros (the loads fill outside the
+          // tensor), their scores count as -inf -- 2^(-inf - m) = 0 goes into S for them, and nothing into the row sum.
+          // The thread's two blocks of 32 columns are the same for every row: the test is uniform over the warp.
+          const int key0 = (k % nhalf) * 256 + hh * 32;
+          const int nv0 = p.N1 - key0, nv1 = p.N1 - (key0 + 128);
+          if (RAGGED && nv0 < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i >= nv0) v0[i] = 0xFF800000u;
+          }
+          if (RAGGED && nv1 < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i >= nv1) v1[i] = 0xFF800000u;
+          }
+        }
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
@@ -529,7 +547,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
 
 bool b2b_fused_supported(int K, int N1, int N2, int mode) {
   // attention form: 256 source positions fill the two P slots; 512 run as two sub-tiles combined at the normalisation
-  if (mode == 1) return K == 128 && N2 == 128 && (N1 == 256 || N1 == 512);
+  // (any source length up to 512 that is a multiple of 8: the positions from N1 on are masked)
+  if (mode == 1) return K == 128 && N2 == 128 && N1 >= 8 && N1 <= 512 && N1 % 8 == 0;
   return b2b_mlp_supported(K, N1, N2);
 }
 
@@ -568,17 +587,17 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.numAttrs = programmatic_launch_enabled() ? 2 : 1;
   int ncl = max_clusters[di].load(std::memory_order_acquire);
   if (ncl == 0) {
-    cudaError_t e = cudaFuncSetAttribute(b2b_pair_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(b2b_pair_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    for (void (*k)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, B2bParams) :
+         {b2b_pair_kernel<1, false, false>, b2b_pair_kernel<2, false, false>, b2b_pair_kernel<1, true, false>,
+          b2b_pair_kernel<2, true, false>, b2b_pair_kernel<1, false, true>, b2b_pair_kernel<2, false, true>,
+          b2b_pair_kernel<1, true, true>, b2b_pair_kernel<2, true, true>}) {
+      e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, B2bSmem::BYTES);
+      if (e != cudaSuccess) return e;
+    }
     int n = 0;
     cfg.gridDim = dim3(2 * dev->sm_count, 1, 1);
-    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1, false>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, b2b_pair_kernel<1, false, false>, &cfg);
     if (e != cudaSuccess) return e;
     if (n <= 0) return cudaErrorLaunchOutOfResources;
     max_clusters[di].store(n, std::memory_order_release);
@@ -589,11 +608,14 @@ cudaError_t launch_b2b_fused(const void* X, const void* W1, const void* W2, B2bP
   cfg.gridDim = dim3(clusters * 2, 1, 1);
   count_launch();
   if (p.mode != 1) return cudaErrorInvalidValue;  // the MLP forms have kernels of their own
-  if (p.keys_row_major)
-    return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2, true>, tmX, tmW1, tmW2, tmO, p)
-                       : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, true>, tmX, tmW1, tmW2, tmO, p);
-  return p.N1 == 512 ? cudaLaunchKernelEx(&cfg, b2b_pair_kernel<2, false>, tmX, tmW1, tmW2, tmO, p)
-                     : cudaLaunchKernelEx(&cfg, b2b_pair_kernel<1, false>, tmX, tmW1, tmW2, tmO, p);
+  const bool two = p.N1 > 256, ragged = p.N1 % 256 != 0;
+  auto go = [&](auto kern) { return cudaLaunchKernelEx(&cfg, kern, tmX, tmW1, tmW2, tmO, p); };
+  if (p.keys_row_major) {
+    if (ragged) return two ? go(b2b_pair_kernel<2, true, true>) : go(b2b_pair_kernel<1, true, true>);
+    return two ? go(b2b_pair_kernel<2, true, false>) : go(b2b_pair_kernel<1, true, false>);
+  }
+  if (ragged) return two ? go(b2b_pair_kernel<2, false, true>) : go(b2b_pair_kernel<1, false, true>);
+  return two ? go(b2b_pair_kernel<2, false, false>) : go(b2b_pair_kernel<1, false, false>);
 }
 
 }  // namespace comfuse

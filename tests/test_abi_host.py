@@ -151,7 +151,8 @@ def test_b2b_validation():
     assert L.comfuse_b2b_workspace_size(ctypes.byref(att), ctypes.byref(n)) == cf.OK and n.value == 0
     attu = cf.make_b2b_desc(4096, 128, 256, 128, 0.0, False, A, 32, 0.088)
     assert L.comfuse_b2b_workspace_size(ctypes.byref(attu), ctypes.byref(n)) == cf.OK and n.value == 32 * 4096 * 256 * 2
-    for bad, code in [(cf.make_b2b_desc(4096, 128, 512, 128, 0.0, True, A, 2, 0.1), cf.OK),                # fused: N1 = 256 or 512
+    for bad, code in [(cf.make_b2b_desc(4096, 128, 512, 128, 0.0, True, A, 2, 0.1), cf.OK),                # fused: N1 <= 512, a multiple of 8
+                      (cf.make_b2b_desc(4096, 128, 200, 128, 0.0, True, A, 2, 0.1), cf.OK),                # (positions from N1 on are masked)
                       (cf.make_b2b_desc(4096, 128, 1024, 128, 0.0, True, A, 2, 0.1), cf.ERR_UNSUPPORTED),
                       (cf.make_b2b_desc(4096, 128, 1024, 128, 0.0, False, A, 2, 0.1), cf.OK),              # unfused takes it
                       (cf.make_b2b_desc(4096, 64, 256, 64, 0.0, False, A, 2, 0.1), cf.OK),                  # N2 != K is fine here

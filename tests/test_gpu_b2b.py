@@ -122,6 +122,26 @@ def test_b2b_softmax_attention_512_sharp_rows_in_either_half(cuda_device):
     P.check_outputs(w, got, P.run_oracle(w), label="attention S=512 sharp")
 
 
+@pytest.mark.parametrize("keys_row_major", [False, True])
+@pytest.mark.parametrize("batch,M,S", [(2, 300, 8), (3, 260, 64), (2, 600, 200), (5, 256, 248), (2, 300, 264), (3, 520, 384), (40, 256, 504)])
+def test_b2b_softmax_attention_any_source_length_up_to_512(batch, M, S, keys_row_major, cuda_device):
+    """Source lengths that are not 256 or 512: the fused kernel masks the positions from S on (their keys and values read as
+    zeros, their scores count as -inf), in the 256-position form up to 256 and in the two-sub-tile form beyond."""
+    import paper_2608_03537_b200 as cf
+    w = wl.target_attention(batch, M, S, 128, seed=5 * batch + M + S)
+    T = P.dev_tensors(w)
+    O = torch.full((batch, M, 128), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    keys = T["W1"].transpose(1, 2).contiguous() if keys_row_major else T["W1"]
+    desc = cf.make_b2b_desc(M, 128, S, 128, 0.0, True, cf.B2B_SOFTMAX_ATTENTION, batch, w.scalars["alpha"],
+                            cf.B2B_FLAG_KEYS_ROW_MAJOR if keys_row_major else 0)
+    assert cf.b2b_workspace_size(desc) == 0
+    before = cf.launch_count()
+    cf.b2b_attention(T["X"], keys, T["W2"], O, alpha=w.scalars["alpha"], fused=True, keys_row_major=keys_row_major)
+    torch.cuda.synchronize()
+    assert cf.last_device_status() == cf.OK and cf.launch_count() - before == 1
+    P.check_outputs(w, {"Y": O}, P.run_oracle(w), label=f"attention b{batch} M{M} S{S} keys_row_major={keys_row_major}")
+
+
 @pytest.mark.parametrize("batch,M,S,d", [(4, 512, 1024, 128), (2, 300, 1000, 64)])
 def test_b2b_softmax_attention_other_shapes_unfused_path(batch, M, S, d, cuda_device):
     """Shapes without a fused instantiation: the fused call says UNSUPPORTED, the in-library unfused path (batched GEMM, row
