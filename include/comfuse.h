@@ -168,7 +168,8 @@ comfuse_status_t comfuse_gemm_epilogue_static_scratch(const comfuse_gemm_desc_t*
  *   O = LayerNorm(S.W2 + b2 + X) * gamma + beta,   S = F(X.W1),
  * X [M, K], W1 [K, N1], W2 [N1, N2], all dense row-major bf16, N2 == K.  In the fused path S (and P) never
  * leave the chip: S is rounded to bf16 as the second GEMM's tensor-core operand.  Fused: K = N2 = 128, N1 a multiple of
- * 128 up to 4096 (the hidden layer streams through in chunks of 128 columns); other shapes: fused = 0. */
+ * 8 up to 4096 (the hidden layer streams through in chunks of 128 columns; a partial last chunk is filled with zeros,
+ * which GELU keeps); other shapes: fused = 0. */
 typedef enum {
   COMFUSE_B2B_MLP_GELU_LAYERNORM = 0, /* as above                                                                   */
   /* Attention form (Sec. 4, Eq. 2 with a row reduction as F; the Target-Attention workload of Sec. 6.2):
@@ -184,7 +185,7 @@ typedef enum {
   /* Two-layer ReLU MLP (Sec. 4, Eq. 2 with F = ReLU(. + b1); the DLRM workload of Sec. 6.2, 1024 -> 512 -> 128):
    *   O = ReLU(ReLU(X.W1 + b1).W2 + b2),
    * X [M, K], W1 [K, N1], W2 [N1, N2]; K and N2 independent, batch = 1, gamma and beta must be NULL, b1 / b2 may be NULL.
-   * Fused: N2 = 128, N1 = 256 or 512, any K (a multiple of 8) streamed through the first GEMM; the hidden layer is rounded
+   * Fused: N2 = 128, N1 <= 512 (a multiple of 8), any K (a multiple of 8) streamed through the first GEMM; the hidden layer is rounded
    * to bf16 as the second GEMM's operand and never leaves the chip.  Unfused: any shape, the bf16 hidden layer [M, N1] in
    * the workspace. */
   COMFUSE_B2B_MLP_RELU = 2

@@ -1,5 +1,5 @@
 // Fused back-to-back GEMM, MLP form (Sec. 4):  P = X W1,  S = GELU_tanh(P + b1),  O' = S W2 + b2 + X,  O = LayerNorm(O'),
-// K = N2 = 128, N1 = 128 .. 4096 (the chunks of N1 stream through; only the bias b1 is held whole).  Neither P nor S is
+// K = N2 = 128, N1 = 8 .. 4096, a multiple of 8 (the chunks of N1 stream through; only the bias b1 is held whole).  Neither P nor S is
 // written to global memory.
 //
 // Dataflow (Sec. 4.1, adapted): N1 is cut into 128-column chunks; one CTA pair walks all chunks of its 256 rows and
@@ -159,7 +159,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   const uint32_t leader = 0u;
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
-  const int NC = p.N1 / 128;
+  const int NC = (p.N1 + 127) / 128;  // a partial last chunk: W1 columns and W2 rows past N1 load as zeros, GELU(0 + 0) = 0
   const int total_tiles = p.batch * p.mpairs;
   const int my_tiles = cluster_id < total_tiles ? (total_tiles - cluster_id + num_clusters - 1) / num_clusters : 0;
   const int total = my_tiles * NC;  // chunks of this cluster's flat stream
@@ -353,7 +353,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   } else {
     // the row vectors, widened to fp32 once, by the epilogue warps (idle until the first P chunk is complete)
     const int epi_tid = threadIdx.x - 64;
-    for (int i = epi_tid; i < p.N1; i += kEpiThreads) s_b1[i] = p.b1 ? bf16_lo(p.b1[i]) : 0.f;
+    for (int i = epi_tid; i < NC * 128; i += kEpiThreads) s_b1[i] = (p.b1 && i < p.N1) ? bf16_lo(p.b1[i]) : 0.f;
     {
       // this CTA's 64 columns of 2 I as a B operand: row k is one 128-byte line, 16-byte chunks swizzled by k & 7 (the
       // layout a TMA load of a W2 chunk half produces); column n of the half is column 64 pm + n of the identity
@@ -610,7 +610,7 @@ b2b_mlp_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
 }  // namespace
 
-bool b2b_mlp_supported(int K, int N1, int N2) { return K == 128 && N2 == 128 && N1 >= 128 && N1 <= MlpSmem::kMaxN1 && N1 % 128 == 0; }
+bool b2b_mlp_supported(int K, int N1, int N2) { return K == 128 && N2 == 128 && N1 >= 8 && N1 <= MlpSmem::kMaxN1 && N1 % 8 == 0; }
 
 cudaError_t launch_b2b_mlp(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
   const DeviceInfo* dev = current_device_info();

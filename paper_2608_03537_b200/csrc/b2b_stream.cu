@@ -95,7 +95,7 @@ b2b_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   const int num_clusters = gridDim.x >> 1;
   const int KB = (p.K + 63) / 64;   // K blocks of ML1 (the last one zero-filled past K)
   const int KBa = (KB + 1) / 2;     // ML2 of the previous unit is issued behind this many of them
-  const int NH = p.N1 / 256;        // halves of N1: 1 or 2
+  const int NH = (p.N1 + 255) / 256;  // halves of N1: 1 or 2; hidden columns past N1 load as zeros and stay zero (ReLU(0 + 0))
   const int total_tiles = p.mpairs;
   const int my_tiles = cluster_id < total_tiles ? (total_tiles - cluster_id + num_clusters - 1) / num_clusters : 0;
   const int nunits = my_tiles * NH;
@@ -442,7 +442,7 @@ static bool stream_lock_enabled() {
   return on;
 }
 
-bool b2b_stream_supported(int K, int N1, int N2) { return N2 == 128 && (N1 == 256 || N1 == 512) && K >= 8 && K % 8 == 0; }
+bool b2b_stream_supported(int K, int N1, int N2) { return N2 == 128 && N1 >= 8 && N1 <= 512 && N1 % 8 == 0 && K >= 8 && K % 8 == 0; }
 
 cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2bParams p, cudaStream_t st) {
   const DeviceInfo* dev = current_device_info();
@@ -465,7 +465,7 @@ cudaError_t launch_b2b_stream(const void* X, const void* W1, const void* W2, B2b
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(kThreads, 1, 1);
-  const bool lock = p.N1 == 512 && stream_lock_enabled();
+  const bool lock = p.N1 > 256 && stream_lock_enabled();
   cfg.dynamicSmemBytes = lock ? StreamSmem<true>::BYTES : StreamSmem<false>::BYTES;
   cfg.stream = st;
   attr[0].id = cudaLaunchAttributeClusterDimension;

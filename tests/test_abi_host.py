@@ -163,14 +163,15 @@ def test_b2b_validation():
         assert L.comfuse_b2b_workspace_size(ctypes.byref(bad), ctypes.byref(n)) == code
     # the attention form has no bias / affine vectors
     assert L.comfuse_b2b_gemm(ctypes.byref(att), FAKE, FAKE, FAKE, FAKE, None, None, None, FAKE, None, 0, None) == cf.ERR_INVALID_ARG
-    # the two-layer ReLU MLP kind: K and N2 independent; fused for N2 = 128, N1 = 256 or 512, any K that is a multiple of 8
+    # the two-layer ReLU MLP kind: K and N2 independent; fused for N2 = 128, N1 <= 512, any K that is a multiple of 8
     R = cf.B2B_MLP_RELU
     relu = cf.make_b2b_desc(32768, 1024, 512, 128, 0.0, True, R)
     assert L.comfuse_b2b_workspace_size(ctypes.byref(relu), ctypes.byref(n)) == cf.OK and n.value == 0
     reluu = cf.make_b2b_desc(32768, 1024, 512, 128, 0.0, False, R)
     assert L.comfuse_b2b_workspace_size(ctypes.byref(reluu), ctypes.byref(n)) == cf.OK and n.value == 32768 * 512 * 2
     for bad, code in [(cf.make_b2b_desc(1024, 8, 256, 128, 0.0, True, R), cf.OK),
-                      (cf.make_b2b_desc(1024, 1024, 384, 128, 0.0, True, R), cf.ERR_UNSUPPORTED),    # N1: 256 or 512
+                      (cf.make_b2b_desc(1024, 1024, 384, 128, 0.0, True, R), cf.OK),                 # N1: any multiple of 8 up to 512
+                      (cf.make_b2b_desc(1024, 1024, 520, 128, 0.0, True, R), cf.ERR_UNSUPPORTED),
                       (cf.make_b2b_desc(1024, 1024, 1024, 128, 0.0, True, R), cf.ERR_UNSUPPORTED),
                       (cf.make_b2b_desc(1024, 1024, 512, 256, 0.0, True, R), cf.ERR_UNSUPPORTED),    # N2: 128
                       (cf.make_b2b_desc(1024, 1024, 1024, 256, 0.0, False, R), cf.OK),               # unfused takes any shape

@@ -20,6 +20,10 @@ CASES = [
     (300, 640, True),      # five chunks: an odd count beyond four
     (520, 2048, False),    # sixteen chunks per tile
     (260, 4096, True),     # the widest hidden layer the bias buffer holds
+    (300, 8, True),        # the narrowest: 8 of the chunk's 128 columns, the rest zero-filled
+    (520, 200, False),     # a whole chunk and a partial one
+    (260, 1000, True),     # seven chunks and 104 columns
+    (300, 4088, False),    # the last 8 columns missing
 ]
 
 

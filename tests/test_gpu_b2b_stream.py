@@ -23,6 +23,11 @@ CASES = [
     (2048, 192, 512),    # odd number of K blocks
     (40000, 128, 512),   # 157 tiles: up to three tiles per cluster, every slot reused in both roles
     (41000, 64, 256),    # single-half tiles alternate between the two slots
+    (300, 200, 8),       # the narrowest hidden layer: all but 8 columns of the half are zero-filled
+    (520, 1024, 200),    # a partial single half
+    (1000, 136, 264),    # the second half holds 8 columns
+    (300, 64, 384),      # one and a half halves
+    (2048, 1024, 504),   # the last 8 columns missing
 ]
 
 
@@ -80,13 +85,13 @@ def test_relu_mlp_bitwise_repeatable_and_equal_rows(cuda_device):
 def test_relu_mlp_argument_checks(cuda_device):
     dev = "cuda:0"
     X = torch.zeros(256, 64, dtype=torch.bfloat16, device=dev)
-    W1 = torch.zeros(64, 384, dtype=torch.bfloat16, device=dev)
-    W2 = torch.zeros(384, 128, dtype=torch.bfloat16, device=dev)
+    W1 = torch.zeros(64, 640, dtype=torch.bfloat16, device=dev)
+    W2 = torch.zeros(640, 128, dtype=torch.bfloat16, device=dev)
     O = torch.zeros(256, 128, dtype=torch.bfloat16, device=dev)
-    with pytest.raises(cf.ComfuseError) as e:     # N1 = 384 has no fused instantiation
+    with pytest.raises(cf.ComfuseError) as e:     # N1 = 640: more than the two halves of 256 columns tensor memory holds
         cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=True)
     assert e.value.status == cf.ERR_UNSUPPORTED
-    ws = torch.empty(256 * 384 * 2, dtype=torch.uint8, device=dev)
+    ws = torch.empty(256 * 640 * 2, dtype=torch.uint8, device=dev)
     cf.b2b_mlp_relu(X, W1, None, W2, None, O, fused=False, workspace=ws)   # ... but runs unfused
     assert cf.last_device_status() == cf.OK
     with pytest.raises(cf.ComfuseError) as e:     # unfused without its workspace
@@ -95,14 +100,14 @@ def test_relu_mlp_argument_checks(cuda_device):
 
 
 def test_relu_mlp_random_shapes(cuda_device):
-    """Seeded random shapes (M 1 .. 3000 and a few beyond one wave of clusters, K any multiple of 8 up to 1536, N1 256 or
-    512), fused kernel against the oracle; the unfused path on every fourth shape.  COMFUSE_FUZZ_SEEDS lengthens the sweep."""
+    """Seeded random shapes (M 1 .. 3000 and a few beyond one wave of clusters, K any multiple of 8 up to 1536, N1 any
+    multiple of 8 up to 512), fused kernel against the oracle; the unfused path on every fourth shape.  COMFUSE_FUZZ_SEEDS lengthens the sweep."""
     rng = np.random.default_rng(20240)
     worst = 0.0
     for i in range(int(os.environ.get("COMFUSE_FUZZ_SEEDS", 60))):
         M = int(rng.integers(1, 3001)) if i % 10 else int(rng.integers(19000, 60000))
         K = 8 * int(rng.integers(1, 193))
-        N1 = 256 * int(rng.integers(1, 3))
+        N1 = 256 * int(rng.integers(1, 3)) if i % 3 else 8 * int(rng.integers(1, 65))
         w = wl.dlrm_bottom_mlp(M, K, N1, 128, seed=1000 + i)
         T = P.dev_tensors(w)
         ref = P.run_oracle(w)

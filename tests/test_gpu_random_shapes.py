@@ -112,13 +112,13 @@ def test_random_row_lengths_of_the_normalising_kinds(seed, cuda_device):
 @pytest.mark.parametrize("seed", _N(150))
 def test_random_b2b_shapes(seed, cuda_device):
     """Back-to-back GEMM, both forms: random row counts (ragged tiles, fewer and more tiles than CTA pairs), every chunk count
-    of the MLP form, both source lengths of the attention form, random scale; fused and unfused."""
+    and partial last chunks of the MLP form, source lengths up to 512 of the attention form, random scale; fused and unfused."""
     g = np.random.default_rng(9000 + seed)
     fused = bool(g.random() < 0.7)
     if g.random() < 0.5:
-        w = wl.b2b_mlp(M=int(g.integers(1, 3000)), K=128, N1=128 * int(g.integers(1, 5) if g.random() < 0.7 else g.integers(5, 33)), N2=128, seed=seed, affine=bool(g.random() < 0.5))
+        w = wl.b2b_mlp(M=int(g.integers(1, 3000)), K=128, N1=(128 * int(g.integers(1, 5) if g.random() < 0.7 else g.integers(5, 33))) if g.random() < 0.6 else 8 * int(g.integers(1, 257)), N2=128, seed=seed, affine=bool(g.random() < 0.5))
     else:
-        w = wl.target_attention(int(g.integers(1, 6)), int(g.integers(1, 1200)), [256, 512][int(g.integers(2))], 128, seed=seed)
+        w = wl.target_attention(int(g.integers(1, 6)), int(g.integers(1, 1200)), [256, 512][int(g.integers(2))] if g.random() < 0.6 else 8 * int(g.integers(1, 65)), 128, seed=seed)
         # scores of standard deviation up to ~7 for the fused kernel; the unfused baseline rounds the scores to bf16 before it
         # exponentiates them (absolute error 2^-9 |score|), so it is only held to the tolerance on moderate scores
         w.scalars["alpha"] = float(np.round(g.uniform(0.02, 0.6 if fused else 0.12), 3))
