@@ -223,7 +223,8 @@ comfuse_status_t comfuse_b2b_gemm(const comfuse_b2b_desc_t* desc, const void* X,
  * computes on `cuda_stream` and range c-2's result is copied out on a second library-owned stream.  `cuda_stream` forks
  * into the two helper streams at the start of the call and joins them at its end, so work enqueued on it afterwards (an
  * event, the next call) is ordered behind the whole call; results are bit for bit those of the unpipelined form.  The
- * helper streams and events are created once per device at first use (COMFUSE_HOST_PIPELINE=0 disables the pipeline);
+ * helper streams and events are created once per device at first use (COMFUSE_HOST_PIPELINE=0 disables the pipeline,
+ * COMFUSE_HOST_CHUNKS=<2..32> sets the most ranges, default 8);
  * they serve one call at a time, so host threads that call these forms on the same device take turns enqueueing.
  * Errors: as comfuse_gemm_epilogue; COMFUSE_ERR_WORKSPACE also when `staging` is NULL or too small.  The description,
  * the workspace and the staging size are checked before anything is enqueued; an error that a CUDA call reports later

@@ -17,13 +17,19 @@ namespace {
 // result goes back on a copy-out stream (both copy engines and the SMs busy at once).  The two helper streams and the
 // events are created once per device and reused; the caller's stream forks into them at the start of the call and joins
 // them at its end, so the call keeps its stream-ordered semantics.  COMFUSE_HOST_PIPELINE=0 turns it off.
-constexpr int kPipeChunks = 8;
+constexpr int kPipeChunks = 32;   // events held per device; the default cut is kPipeDefault ranges (COMFUSE_HOST_CHUNKS=<n> overrides it)
+constexpr int kPipeDefault = 8;
 // Every range costs host time (tensor-map encodes, launches, event records): cut only into ranges whose host -> device
 // traffic is worth it.
 constexpr size_t kPipeMinChunkBytes = 4u << 20;
 int pipe_chunks(size_t h2d_bytes) {
+  static const int most = [] {
+    const char* e = std::getenv("COMFUSE_HOST_CHUNKS");
+    const int v = e ? std::atoi(e) : 0;
+    return v >= 2 && v <= kPipeChunks ? v : kPipeDefault;
+  }();
   const size_t n = h2d_bytes / kPipeMinChunkBytes;
-  return n >= static_cast<size_t>(kPipeChunks) ? kPipeChunks : static_cast<int>(n);
+  return n >= static_cast<size_t>(most) ? most : static_cast<int>(n);
 }
 constexpr int kMaxDevPipe = 64;
 struct Pipe {
