@@ -222,6 +222,7 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
         ring.advance();
         const uint64_t xdesc0 = make_smem_desc_sw128(x0, 16, 1024);
         const uint64_t xdesc1 = make_smem_desc_sw128(x1, 16, 1024);
+        int wst[2] = {0, 0};
         for (int j = 0; j < 2 && ok; ++j) {
           const int wstage = ring.stage;
           const uint32_t wa = wait_slot();
@@ -241,9 +242,13 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
               umma_bf16_ss_pair(tmem_base + j * 128, (kk < 4 ? xdesc0 : xdesc1) + static_cast<uint64_t>((kk & 3) * 2),
                                 wdesc + static_cast<uint64_t>(kk * 128), idesc_ml1, kk != 0 ? 1u : 0u);
           }
-          release_slot(wstage);
-          umma_commit_pair_both(bar_pfull(j));
+          wst[j] = wstage;
         }
+        // one commit tells the softmax warps that both chunks are complete (it is the one on the critical path: the slots
+        // are handed back behind it)
+        if (ok) umma_commit_pair_both(bar_pfull(0));
+        release_slot(wst[0]);
+        release_slot(wst[1]);
         release_slot(xs0);
         release_slot(xs1);
       };
@@ -337,10 +342,8 @@ b2b_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__
       // UMMAs' A operand.  S.V of sub-tile k runs under the softmax of sub-tile k+1; the division by the row sum is the
       // finish warps' work.
       auto softmax_tile = [&](int k) {
-        for (int pb = 0; pb < 2; ++pb) {
-          mbar_wait<false>(bar_pfull(pb), puses[pb] & 1u, w);
-          ++puses[pb];
-        }
+        mbar_wait<false>(bar_pfull(0), puses[0] & 1u, w);  // both chunks: the score lane commits once per sub-tile
+        ++puses[0];
         __syncwarp();
         tcgen05_fence_after_sync();
         B2B_TRACE_POINT();  // scores of the sub-tile complete
