@@ -24,3 +24,17 @@ def cuda_device():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     return torch.device("cuda:0")
+
+
+@pytest.fixture(autouse=True)
+def _device_status_stays_clear(request):
+    """Every GPU test ends with a clear device status word: no bounded wait ran out and (checked build) no bounds
+    predicate failed in any kernel the test launched.  Tests that provoke a status read it themselves, which clears it."""
+    yield
+    if request.node.get_closest_marker("gpu") is None:
+        return
+    import torch
+    if not torch.cuda.is_available():
+        return
+    import paper_2608_03537_b200 as cf
+    assert cf.last_device_status() == cf.OK, "a kernel launched by this test left a device status behind"
