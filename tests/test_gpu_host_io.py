@@ -180,3 +180,42 @@ def test_pipelined_b2b_host_forms_match_device_forms(cuda_device):
         cf.b2b_attention_host(hQ, hK, hV, hO, staging=staging, alpha=w.scalars["alpha"])
         torch.cuda.synchronize()
         assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_b2b_host_forms_with_partial_last_chunks(cuda_device):
+    """The host-buffer forms with a hidden width / source length that ends in a partial chunk (zero-filled loads on the
+    device side), large enough to run as pipelines: bit for bit the device-pointer results, oracle parity on sampled rows."""
+    import paper_2608_03537_b200 as cf
+    w = wl.b2b_mlp(M=40000, K=128, N1=200, N2=128, seed=41, affine=True)
+    T = P.dev_tensors(w)
+    dev = T["X"].device
+    ref = P.run_gpu(w, T, fused=True)["Y"]
+    hX = _pinned(T["X"])
+    hO = torch.empty(40000, 128, dtype=torch.bfloat16).pin_memory()
+    desc = cf.make_b2b_desc(40000, 128, 200, 128, w.scalars["eps"], True)
+    staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=dev)
+    hO.fill_(3.0)
+    cf.b2b_gemm_host(hX, T["W1"], T["b1"], T["W2"], T["b2"], hO, staging=staging, gamma=T.get("gamma"), beta=T.get("beta"),
+                     eps=w.scalars["eps"])
+    torch.cuda.synchronize()
+    assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+    rows = wl.sample_rows(40000, 64)
+    P.check_outputs(w, {"Y": ref}, P.run_oracle(w, rows=rows), rows=rows, label="b2b host, N1 = 200")
+    for keys_row_major in (False, True):
+        w = wl.target_attention(20, 2048, 200, 128, seed=42)
+        T = P.dev_tensors(w)
+        Kd = T["W1"].transpose(1, 2).contiguous() if keys_row_major else T["W1"]
+        ref = torch.empty(20, 2048, 128, dtype=torch.bfloat16, device=dev)
+        cf.b2b_attention(T["X"], Kd, T["W2"], ref, alpha=w.scalars["alpha"], keys_row_major=keys_row_major)
+        hQ, hK, hV = _pinned(T["X"]), _pinned(Kd), _pinned(T["W2"])
+        hO = torch.empty(20, 2048, 128, dtype=torch.bfloat16).pin_memory()
+        desc = cf.make_b2b_desc(2048, 128, 200, 128, 0.0, True, cf.B2B_SOFTMAX_ATTENTION, 20, w.scalars["alpha"],
+                                cf.B2B_FLAG_KEYS_ROW_MAJOR if keys_row_major else 0)
+        staging = torch.empty(cf.b2b_host_staging_size(desc), dtype=torch.uint8, device=dev)
+        hO.fill_(3.0)
+        cf.b2b_attention_host(hQ, hK, hV, hO, staging=staging, alpha=w.scalars["alpha"], keys_row_major=keys_row_major)
+        torch.cuda.synchronize()
+        assert torch.equal(hO.view(torch.int16), ref.cpu().view(torch.int16))
+        rows = wl.sample_rows(2048, 32)
+        want = P.run_oracle(w, rows=rows)
+        P.check_outputs(w, {"Y": ref}, want, rows=rows, label=f"attention host, 200 source positions, keys_row_major={keys_row_major}")
